@@ -1,0 +1,199 @@
+// CPU oracle for relay-buffer-free MoE dispatch / combine.
+//
+// TEST INFRASTRUCTURE ONLY (see moe_oracle.h).  Plain sequential C++17; the
+// definition written out, no blocking, no fusion.  Build:
+//   g++ -std=c++17 -O2 -ffp-contract=off -fPIC -shared -pthread moe_oracle.cpp -o liboracle.so
+//
+// Pins (tests marked "not gpu"): histogram vs a library bincount; s vs the
+// literal set-cardinality definition by O(B^2) counting; o vs a library
+// cumulative sum; slots vs a library stable sort by expert; dispatch vs
+// row-by-row lookup; combine vs exact rational arithmetic, vs an fp64 sum, and
+// vs closed forms (identity experts, W = 1/K, one-hot W); bf16 conversion vs a
+// library conversion; a hand-worked example.  No function here is unpinned.
+
+#include "moe_oracle.h"
+
+#include <cmath>
+#include <cstring>
+#include <thread>
+#include <vector>
+
+namespace {
+
+// Source rank of token t: the r with rank_tok_start[r] <= t < rank_tok_start[r+1]
+// (Algorithm 1: "source rank of token t").
+int32_t src_rank(const int32_t* rank_tok_start, int32_t R, int32_t t) {
+  for (int32_t r = 0; r < R; ++r)
+    if (t < rank_tok_start[r + 1]) return r;
+  return R - 1;
+}
+
+bool shape_ok(int32_t T, int32_t K, int32_t E, int32_t R, const int32_t* rank_tok_start) {
+  if (T < 0 || K < 1 || E < 1 || R < 1 || E % R != 0 || rank_tok_start == nullptr) return false;
+  if (rank_tok_start[0] != 0 || rank_tok_start[R] != T) return false;
+  for (int32_t r = 0; r < R; ++r)
+    if (rank_tok_start[r + 1] < rank_tok_start[r]) return false;
+  return true;
+}
+
+template <class F>
+void for_token_ranges(int32_t T, int32_t n_threads, F body) {
+  if (n_threads <= 1 || T < 2) {
+    body(0, T);
+    return;
+  }
+  std::vector<std::thread> pool;
+  for (int32_t i = 0; i < n_threads; ++i) {
+    int32_t lo = (int32_t)((int64_t)T * i / n_threads);
+    int32_t hi = (int32_t)((int64_t)T * (i + 1) / n_threads);
+    pool.emplace_back([=] { body(lo, hi); });
+  }
+  for (auto& th : pool) th.join();
+}
+
+}  // namespace
+
+extern "C" {
+
+float oracle_bf16_to_float(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+
+uint16_t oracle_float_to_bf16(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u)          // NaN: keep sign, force a quiet NaN
+    return (uint16_t)((u >> 16) | 0x0040u);
+  uint32_t lsb = (u >> 16) & 1u;                // ties to even
+  u += 0x7fffu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
+                const int32_t* rank_tok_start,
+                int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
+                int32_t* n_exp, int32_t* n_recv) {
+  if (!shape_ok(T, K, E, R, rank_tok_start)) return ORACLE_ERR_INVALID_ARG;
+  if (T > 0 && topk_idx == nullptr) return ORACLE_ERR_INVALID_ARG;
+  const int32_t E_r = E / R;
+  const int64_t B = (int64_t)T * K;
+
+  // Routing indexes lie in {0..E-1} (Section 5.1); anything else is an error.
+  for (int64_t b = 0; b < B; ++b)
+    if (topk_idx[b] < 0 || topk_idx[b] >= E) return ORACLE_ERR_BAD_INDEX;
+
+  // Layout: one pass over branches in flat order (t, j).  run[r][e] is the
+  // number of branches of source rank r seen so far that chose expert e, so the
+  // value read before the increment is s[t,j]; its final value is M[r,e].
+  std::vector<int32_t> run((size_t)R * E, 0);
+  for (int32_t t = 0; t < T; ++t) {
+    const int32_t r = src_rank(rank_tok_start, R, t);
+    for (int32_t j = 0; j < K; ++j) {
+      const int32_t e = topk_idx[(int64_t)t * K + j];
+      s[(int64_t)t * K + j] = run[(size_t)r * E + e]++;
+    }
+  }
+  for (int32_t r = 0; r < R; ++r)
+    for (int32_t e = 0; e < E; ++e) M[(size_t)r * E + e] = run[(size_t)r * E + e];
+
+  // Per-rank branch counts: c_rank[r,d] = sum over experts of rank d of M[r,e].
+  for (int32_t r = 0; r < R; ++r)
+    for (int32_t d = 0; d < R; ++d) {
+      int32_t acc = 0;
+      for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) acc += M[(size_t)r * E + e];
+      c_rank[(size_t)r * R + d] = acc;
+    }
+
+  // Notify: receive counts, then large offsets.  Inside the window of rank d
+  // the blocks follow each other expert by expert (ascending), and inside an
+  // expert source rank by source rank (ascending); o[e,r] is where block
+  // (r -> e) begins, counted from the start of rank d's window.
+  for (int32_t e = 0; e < E; ++e) {
+    int32_t acc = 0;
+    for (int32_t r = 0; r < R; ++r) acc += M[(size_t)r * E + e];
+    n_exp[e] = acc;
+  }
+  for (int32_t d = 0; d < R; ++d) {
+    int32_t acc = 0;
+    for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e)
+      for (int32_t r = 0; r < R; ++r) {
+        o[(size_t)e * R + r] = acc;
+        acc += M[(size_t)r * E + e];
+      }
+    n_recv[d] = acc;
+  }
+  return ORACLE_OK;
+}
+
+int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
+                 const int32_t* rank_tok_start, const int32_t* s, const int32_t* o,
+                 const int32_t* n_recv, int64_t C, int64_t* slots) {
+  if (!shape_ok(T, K, E, R, rank_tok_start) || C < 0) return ORACLE_ERR_INVALID_ARG;
+  const int32_t E_r = E / R;
+  for (int32_t d = 0; d < R; ++d)
+    if (n_recv[d] > C) return ORACLE_ERR_CAPACITY;
+  for (int64_t b = 0; b < (int64_t)T * K; ++b)
+    if (topk_idx[b] < 0 || topk_idx[b] >= E) return ORACLE_ERR_BAD_INDEX;
+  for (int32_t t = 0; t < T; ++t) {
+    const int32_t r_src = src_rank(rank_tok_start, R, t);
+    for (int32_t j = 0; j < K; ++j) {
+      const int64_t b = (int64_t)t * K + j;
+      const int32_t e = topk_idx[b];
+      const int32_t r_dst = e / E_r;                       // destination rank of the branch
+      slots[b] = (int64_t)r_dst * C + o[(size_t)e * R + r_src] + s[b];
+    }
+  }
+  return ORACLE_OK;
+}
+
+int oracle_dispatch(const uint16_t* X, int32_t T, int32_t H, int32_t K,
+                    const int64_t* slots, uint16_t* windows, int32_t n_threads) {
+  if (T < 0 || H < 1 || K < 1) return ORACLE_ERR_INVALID_ARG;
+  for_token_ranges(T, n_threads, [=](int32_t lo, int32_t hi) {
+    for (int32_t t = lo; t < hi; ++t)
+      for (int32_t j = 0; j < K; ++j)
+        std::memcpy(windows + slots[(int64_t)t * K + j] * H, X + (int64_t)t * H,
+                    (size_t)H * sizeof(uint16_t));
+  });
+  return ORACLE_OK;
+}
+
+int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int64_t C,
+                        const int32_t* n_exp, const uint16_t* scale) {
+  if (H < 1 || E < 1 || R < 1 || E % R != 0) return ORACLE_ERR_INVALID_ARG;
+  const int32_t E_r = E / R;
+  for (int32_t d = 0; d < R; ++d) {
+    int64_t row = (int64_t)d * C;
+    for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) {
+      const float sc = oracle_bf16_to_float(scale[e]);
+      for (int32_t i = 0; i < n_exp[e]; ++i, ++row)
+        for (int32_t h = 0; h < H; ++h) {
+          uint16_t* p = windows + row * H + h;
+          *p = oracle_float_to_bf16(oracle_bf16_to_float(*p) * sc);
+        }
+    }
+  }
+  return ORACLE_OK;
+}
+
+int oracle_combine(const uint16_t* windows, int32_t T, int32_t H, int32_t K,
+                   const int64_t* slots, const float* W, uint16_t* Y, int32_t n_threads) {
+  if (T < 0 || H < 1 || K < 1) return ORACLE_ERR_INVALID_ARG;
+  for_token_ranges(T, n_threads, [=](int32_t lo, int32_t hi) {
+    for (int32_t t = lo; t < hi; ++t)
+      for (int32_t h = 0; h < H; ++h) {
+        float acc = 0.0f;
+        for (int32_t j = 0; j < K; ++j) {
+          const int64_t b = (int64_t)t * K + j;
+          acc = std::fmaf(W[b], oracle_bf16_to_float(windows[slots[b] * H + h]), acc);
+        }
+        Y[(int64_t)t * H + h] = oracle_float_to_bf16(acc);
+      }
+  });
+  return ORACLE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,89 @@
+/* CPU oracle for relay-buffer-free MoE dispatch / combine.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is the plain, slow, sequential definition of
+ * what the path computes.  It shares no source, header, helper or constant with
+ * the CUDA library, and the CUDA library never calls it.  Only the tests, the
+ * smoke check and the benchmark's cpu-baseline leg may load it.
+ *
+ * All pointers are HOST pointers.  Integer tensors are int32 (slots: int64),
+ * hidden states are bf16 stored as uint16_t, routing weights are fp32.
+ *
+ * Notation follows the paper (Section 5.1, Table 1):
+ *   T tokens, H hidden size, K top-k degree, E experts, R ranks, E_r = E / R,
+ *   K[t,j] routing index, W[t,j] routing weight, s small offset, o large
+ *   offset, M gathered count matrix, n_exp / n_recv receive counts.
+ * Tokens of all source ranks are concatenated in rank order; source rank r owns
+ * tokens rank_tok_start[r] .. rank_tok_start[r+1]-1.
+ *
+ * Every function returns one of the ORACLE_* codes below and leaves its outputs
+ * untouched when it returns an error.
+ */
+#ifndef MOE_ORACLE_H
+#define MOE_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  ORACLE_OK = 0,
+  ORACLE_ERR_INVALID_ARG = 1,
+  ORACLE_ERR_BAD_INDEX = 2,
+  ORACLE_ERR_CAPACITY = 3
+};
+
+/* Planning state of the prefill schedule (Layout + Notify, Section 5.2):
+ *   M      [R,E]  M[r,e]  = #branches from source rank r to expert e      (gathered count matrix)
+ *   c_rank [R,R]  c_rank[r,d] = #branches from source rank r to rank d    (per-rank branch counts)
+ *   s      [T,K]  small offset: #earlier branches (flat order t*K+j) of the
+ *                 same source rank that chose the same expert             (Layout, definition of s)
+ *   o      [E,R]  large offset: first row, local to the window of rank
+ *                 dst(e) = e / E_r, of the block (source rank r -> expert e);
+ *                 blocks are laid out expert-major, then source rank       (Notify, definition of o)
+ *   n_exp  [E]    rows received by expert e;  n_recv [R] rows received by rank d.
+ * The decode schedule keeps only (o, s); its values are these same ones (Section 5.3). */
+int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
+                const int32_t* rank_tok_start,
+                int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
+                int32_t* n_exp, int32_t* n_recv);
+
+/* Expert-window row of every branch (two-level offset rule, Section 5.1; Algorithm 1):
+ *   slot[t,j] = dst(e) * C + o[e, src(t)] + s[t,j],  e = K[t,j].
+ * The windows of the R ranks are R equal segments of C rows of one allocation.
+ * ORACLE_ERR_CAPACITY if some n_recv[d] > C. */
+int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
+                 const int32_t* rank_tok_start, const int32_t* s, const int32_t* o,
+                 const int32_t* n_recv, int64_t C, int64_t* slots);
+
+/* Dispatch (Algorithm 1, first loop): copy row X[t,:] to window row slot[t,j]
+ * for every branch.  Rows no branch maps to are left as the caller set them.
+ * n_threads > 1 splits the token range over std::thread workers (same result). */
+int oracle_dispatch(const uint16_t* X, int32_t T, int32_t H, int32_t K,
+                    const int64_t* slots, uint16_t* windows, int32_t n_threads);
+
+/* Stand-in for the expert FFN (not part of the method): multiply, in place,
+ * every received row of expert e by the bf16 scalar scale[e]:
+ *   y = bf16_rne(float(x) * float(scale[e])).
+ * Rows of expert e are rows start_e .. start_e + n_exp[e] - 1 of its rank's
+ * segment, start_e = sum of n_exp over earlier experts of the same rank. */
+int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int64_t C,
+                        const int32_t* n_exp, const uint16_t* scale);
+
+/* Combine (Algorithm 1, second loop):
+ *   acc = +0.0f; for j = 0..K-1: acc = fmaf(W[t,j], float(Yexp[slot[t,j], h]), acc);
+ *   Y[t,h] = bf16_rne(acc).
+ * Y is fully overwritten. */
+int oracle_combine(const uint16_t* windows, int32_t T, int32_t H, int32_t K,
+                   const int64_t* slots, const float* W, uint16_t* Y, int32_t n_threads);
+
+/* bf16 <-> fp32 conversions used above, exported so that tests can pin them
+ * against a library conversion.  Round to nearest, ties to even; NaN stays NaN. */
+uint16_t oracle_float_to_bf16(float f);
+float oracle_bf16_to_float(uint16_t b);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,440 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+Each test compares the oracle with a textbook/library routine, the literal
+definition evaluated by brute force, exact rational arithmetic, a closed form or
+a hand-worked example -- never with a retyped copy of the oracle's own loop.
+No GPU is needed.
+"""
+import itertools
+import json
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06055_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------- helpers
+def src_of_tokens(rts):
+    rts = np.asarray(rts)
+    return np.repeat(np.arange(len(rts) - 1), np.diff(rts))
+
+
+def literal_small_offsets(idx, rts):
+    """Definition of s (Prefill Layout): the number of branches that come before
+    (t,j) in (t,j) order, belong to the same source rank, and chose the same
+    expert -- counted one pair at a time."""
+    T, K = idx.shape
+    src = src_of_tokens(rts)
+    flat = [(t, j) for t in range(T) for j in range(K)]
+    s = np.zeros((T, K), np.int64)
+    for a, (t, j) in enumerate(flat):
+        s[t, j] = sum(1 for (t2, j2) in flat[:a] if src[t2] == src[t] and idx[t2, j2] == idx[t, j])
+    return s
+
+
+def round_to_format(x: Fraction, mant_bits: int, emin: int) -> Fraction:
+    """Round an exact rational to a binary float format with `mant_bits` stored
+    mantissa bits and minimum normal exponent `emin`: nearest, ties to even."""
+    if x == 0:
+        return Fraction(0)
+    sign = -1 if x < 0 else 1
+    a = abs(x)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    e = max(e, emin)
+    quantum = Fraction(2) ** (e - mant_bits)
+    n = a / quantum
+    fl = n.numerator // n.denominator
+    rem = n - fl
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+        fl += 1
+    return sign * fl * quantum
+
+
+def f32(x: Fraction) -> Fraction:
+    return round_to_format(x, 23, -126)
+
+
+def bf16(x: Fraction) -> Fraction:
+    return round_to_format(x, 7, -126)
+
+
+def u16_to_float(a):
+    return (np.asarray(a, np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def rand_bf16(rng, shape):
+    x = torch.from_numpy(rng.standard_normal(shape).astype(np.float32)).to(torch.bfloat16)
+    return synth.bf16_to_u16(x).copy()
+
+
+def random_case(rng, T, K, E, R, replace=False, uniform_ranks=False):
+    if replace:
+        idx = rng.integers(0, E, (T, K)).astype(np.int32)
+    else:
+        idx = np.stack([rng.permutation(E)[:K] for _ in range(T)]).astype(np.int32) if T else np.zeros((0, K), np.int32)
+    if uniform_ranks and T % R == 0:
+        rts = oracle.uniform_rank_tok_start(T, R)
+    else:
+        cuts = np.sort(rng.integers(0, T + 1, R - 1))
+        rts = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    return idx, rts
+
+
+SHAPES = [  # T, K, E, R
+    (0, 2, 4, 2), (1, 1, 1, 1), (7, 1, 4, 4), (37, 2, 8, 4), (64, 4, 16, 1), (100, 3, 12, 3),
+    (256, 2, 16, 4), (513, 8, 64, 8), (300, 6, 6, 6),
+]
+
+
+def cases():
+    rng = np.random.default_rng(20260506)
+    for (T, K, E, R) in SHAPES:
+        for replace in (False, True):
+            if not replace and K > E:
+                continue
+            yield (T, K, E, R, replace) + random_case(rng, T, K, E, R, replace)
+
+
+# ----------------------------------------------------------------------------- golden
+def test_hand_worked_example():
+    g = json.load(open(os.path.join(GOLDEN, "worked_example.json")))
+    idx = np.array(g["topk_idx"], np.int32)
+    T, K, E, R, H, C = (g[k] for k in "TKERHC")
+    rts = np.array(g["rank_tok_start"], np.int32)
+    p = oracle.plan(idx, E, R, rts)
+    assert p.status == oracle.OK
+    for name in ("M", "c_rank", "s", "o", "n_exp", "n_recv"):
+        assert getattr(p, name).tolist() == g[name], name
+    st, slots = oracle.slots(idx, E, R, p, C, rts)
+    assert st == oracle.OK and slots.tolist() == g["slots"]
+
+    xv = torch.tensor(g["x_row_value"], dtype=torch.float32)
+    X = synth.bf16_to_u16(xv[:, None].expand(T, H).to(torch.bfloat16).contiguous())
+    canary = 0xDEAD
+    win = np.full((R * C, H), canary, np.uint16)
+    assert oracle.dispatch(X, slots, win) == oracle.OK
+    for row, tok in enumerate(g["window_row_token"]):
+        want = canary if tok < 0 else X[tok, 0]
+        assert (win[row] == want).all(), row
+    W = np.array(g["topk_w"], np.float32)
+    st, Y = oracle.combine(win, slots, W, H)
+    assert st == oracle.OK
+    assert np.array_equal(u16_to_float(Y), np.repeat(np.array(g["y_identity_row_value"], np.float32)[:, None], H, 1))
+    scale = synth.bf16_to_u16(torch.tensor(g["scale"]).to(torch.bfloat16))
+    assert oracle.expert_scale(win, H, E, R, C, p.n_exp, scale) == oracle.OK
+    assert (win[8:] == canary).all()
+    st, Y = oracle.combine(win, slots, W, H)
+    assert np.array_equal(u16_to_float(Y), np.repeat(np.array(g["y_scale_row_value"], np.float32)[:, None], H, 1))
+
+
+# ----------------------------------------------------------------------------- plan
+@pytest.mark.parametrize("case", list(cases()), ids=lambda c: f"T{c[0]}K{c[1]}E{c[2]}R{c[3]}{'rep' if c[4] else ''}")
+def test_plan_against_library_routines(case):
+    T, K, E, R, _, idx, rts = case
+    p = oracle.plan(idx, E, R, rts)
+    assert p.status == oracle.OK
+    E_r = E // R
+    src = src_of_tokens(rts)
+
+    # Counts: a histogram of (source rank, expert) pairs (library bincount).
+    key = (np.repeat(src, K) * E + idx.reshape(-1)).astype(np.int64)
+    M = np.bincount(key, minlength=R * E).reshape(R, E)
+    assert np.array_equal(p.M, M)
+    assert p.M.sum() == T * K
+    assert np.array_equal(p.M.sum(1), np.diff(rts) * K)
+    assert np.array_equal(p.c_rank, M.reshape(R, R, E_r).sum(2))
+    assert np.array_equal(p.c_rank.sum(1), np.diff(rts) * K)
+    assert np.array_equal(p.n_exp, M.sum(0))
+    assert np.array_equal(p.n_recv, M.sum(0).reshape(R, E_r).sum(1))
+
+    # Large offsets: exclusive cumulative sum of M laid out [dst rank][local expert][src rank],
+    # restarting in every destination window.
+    blocks = M.T.reshape(R, E_r * R)                       # row d: (e_local, r) blocks in window order
+    excl = np.cumsum(blocks, 1) - blocks
+    assert np.array_equal(p.o, excl.reshape(E, R))
+    assert np.array_equal(excl[:, -1] + blocks[:, -1], p.n_recv)
+
+    # Small offsets: within each (r, e) group they are 0..M[r,e]-1, increasing in flat order.
+    flat_s = p.s.reshape(-1)
+    for k_ in np.unique(key):
+        assert np.array_equal(flat_s[key == k_], np.arange(M.reshape(-1)[k_]))
+
+    # Slots: a stable sort of the branches by expert IS the packed window order,
+    # because the source rank never decreases with the token index.
+    C = int(p.n_recv.max()) + 3 if T else 3
+    st, slots = oracle.slots(idx, E, R, p, C, rts)
+    assert st == oracle.OK
+    order = np.argsort(idx.reshape(-1), kind="stable")
+    pos = np.empty(T * K, np.int64)
+    pos[order] = np.arange(T * K)
+    dst = idx.reshape(-1) // E_r
+    before = np.concatenate([[0], np.cumsum(p.n_recv)])[dst]   # branches bound for earlier ranks
+    assert np.array_equal(slots.reshape(-1), dst * C + pos - before)
+
+    # Bijection onto the used part of each segment; each expert's rows contiguous.
+    used = np.sort(slots.reshape(-1))
+    want = np.concatenate([d * C + np.arange(p.n_recv[d]) for d in range(R)]) if T else np.zeros(0)
+    assert np.array_equal(used, want)
+    start = (np.cumsum(p.n_exp.reshape(R, E_r), 1) - p.n_exp.reshape(R, E_r)).reshape(-1)
+    for e in range(E):
+        rows = np.sort(slots.reshape(-1)[idx.reshape(-1) == e])
+        assert np.array_equal(rows, (e // E_r) * C + start[e] + np.arange(p.n_exp[e]))
+
+
+@pytest.mark.parametrize("T,K,E,R", [(5, 2, 4, 2), (40, 3, 6, 3), (64, 8, 16, 4), (129, 2, 3, 1)])
+def test_small_offsets_literal_definition(T, K, E, R):
+    rng = np.random.default_rng(T * 1000 + K)
+    for replace in (False, True):
+        if not replace and K > E:
+            continue
+        idx, rts = random_case(rng, T, K, E, R, replace)
+        p = oracle.plan(idx, E, R, rts)
+        assert np.array_equal(p.s, literal_small_offsets(idx, rts))
+
+
+def test_brute_force_all_routings_tiny():
+    """Every routing of T=3, K=2 over E=4 experts, R=2 ranks (4^6 cases), against
+    the definitions evaluated literally in Python."""
+    T, K, E, R, C = 3, 2, 4, 2, 6
+    rts = np.array([0, 2, 3], np.int32)
+    src = [0, 0, 1]
+    E_r = E // R
+    for combo in itertools.product(range(E), repeat=T * K):
+        idx = np.array(combo, np.int32).reshape(T, K)
+        p = oracle.plan(idx, E, R, rts)
+        st, slots = oracle.slots(idx, E, R, p, C, rts)
+        assert st == oracle.OK
+        branches = [(t, j) for t in range(T) for j in range(K)]
+        for a, (t, j) in enumerate(branches):
+            e = idx[t, j]
+            s_lit = sum(1 for (t2, j2) in branches[:a] if src[t2] == src[t] and idx[t2, j2] == e)
+            # block (r -> e) starts after every block (e', r') that precedes it in the window of dst(e)
+            o_lit = sum(1 for (t2, j2) in branches
+                        if idx[t2, j2] // E_r == e // E_r and (idx[t2, j2], src[t2]) < (e, src[t]))
+            assert p.s[t, j] == s_lit and p.o[e, src[t]] == o_lit
+            assert slots[t, j] == (e // E_r) * C + o_lit + s_lit
+
+
+def test_error_codes_and_untouched_outputs():
+    idx = np.array([[0, 1], [2, 4]], np.int32)
+    p = oracle.plan(idx, 4, 2)
+    assert p.status == oracle.ERR_BAD_INDEX
+    assert (p.M == -7).all() and (p.s == -7).all() and (p.o == -7).all()
+    idx[1, 1] = -1
+    assert oracle.plan(idx, 4, 2).status == oracle.ERR_BAD_INDEX
+    idx[1, 1] = 3
+    assert oracle.plan(idx, 4, 3, np.array([0, 1, 1, 2], np.int32)).status == oracle.ERR_INVALID_ARG   # E % R != 0
+    assert oracle.plan(idx, 4, 2, np.array([0, 2, 1], np.int32)).status == oracle.ERR_INVALID_ARG
+    assert oracle.plan(idx, 4, 2, np.array([0, 3, 2], np.int32)).status == oracle.ERR_INVALID_ARG
+    p = oracle.plan(idx, 4, 2)
+    assert p.status == oracle.OK
+    C = int(p.n_recv.max())
+    st, sl = oracle.slots(idx, 4, 2, p, C)
+    assert st == oracle.OK
+    st, sl = oracle.slots(idx, 4, 2, p, C - 1)
+    assert st == oracle.ERR_CAPACITY and (sl == -1).all()
+
+
+def test_edge_shapes():
+    # T = 0
+    p = oracle.plan(np.zeros((0, 2), np.int32), 4, 2)
+    assert p.status == oracle.OK and not p.M.any() and not p.o.any() and not p.n_recv.any()
+    # all branches to one expert; a rank with no tokens; E == R; K == 1
+    idx = np.full((10, 1), 2, np.int32)
+    rts = np.array([0, 0, 4, 10], np.int32)
+    p = oracle.plan(idx, 3, 3, rts)
+    assert p.n_exp.tolist() == [0, 0, 10] and p.n_recv.tolist() == [0, 0, 10]
+    assert p.o[2].tolist() == [0, 0, 4] and p.s.reshape(-1).tolist() == [0, 1, 2, 3, 0, 1, 2, 3, 4, 5]
+    # the same expert twice in one token: consecutive slots in j order
+    idx = np.array([[1, 1, 1]], np.int32)
+    p = oracle.plan(idx, 2, 1)
+    assert p.s.tolist() == [[0, 1, 2]]
+
+
+# ----------------------------------------------------------------------------- dispatch
+@pytest.mark.parametrize("T,K,E,R,H", [(37, 2, 8, 4, 8), (100, 3, 12, 3, 24), (256, 2, 16, 4, 64)])
+def test_dispatch_rows_and_canaries(T, K, E, R, H):
+    rng = np.random.default_rng(T)
+    idx, rts = random_case(rng, T, K, E, R, replace=True)
+    X = rand_bf16(rng, (T, H))
+    p = oracle.plan(idx, E, R, rts)
+    C = int(p.n_recv.max()) + 2
+    _, slots = oracle.slots(idx, E, R, p, C, rts)
+    win = np.full((R * C, H), 0xBEEF, np.uint16)
+    assert oracle.dispatch(X, slots, win) == oracle.OK
+    owner = np.full(R * C, -1)
+    owner[slots.reshape(-1)] = np.repeat(np.arange(T), K)
+    for row in range(R * C):
+        if owner[row] < 0:
+            assert (win[row] == 0xBEEF).all()
+        else:
+            assert np.array_equal(win[row], X[owner[row]])
+    win2 = np.full((R * C, H), 0xBEEF, np.uint16)
+    oracle.dispatch(X, slots, win2, n_threads=3)
+    assert np.array_equal(win, win2)
+
+
+# ----------------------------------------------------------------------------- bf16
+def test_bf16_conversion_against_torch():
+    rng = np.random.default_rng(7)
+    vals = np.concatenate([
+        rng.standard_normal(20000).astype(np.float32),
+        (rng.standard_normal(5000) * 1e30).astype(np.float32),
+        (rng.standard_normal(5000) * 1e-38).astype(np.float32),           # subnormal range
+        rng.integers(0, 2 ** 32, 20000, dtype=np.uint64).astype(np.uint32).view(np.float32),
+        np.array([0.0, -0.0, np.inf, -np.inf, 1.0, 1.00390625, 1.01171875, 3.3895314e38, 3.4e38], np.float32),
+    ])
+    want = synth.bf16_to_u16(torch.from_numpy(vals).to(torch.bfloat16))
+    for v, w in zip(vals, want):
+        got = oracle.float_to_bf16(v)
+        if np.isnan(v):
+            assert (got & 0x7F80) == 0x7F80 and (got & 0x7F) != 0
+        else:
+            assert got == w, (v, got, w)
+    for b in list(range(0, 65536, 37)) + [0x7F80, 0xFF80, 0x8000]:
+        f = oracle.bf16_to_float(b)
+        t = torch.tensor([b], dtype=torch.int32).to(torch.int16).view(torch.bfloat16).float().item()
+        assert (np.isnan(f) and np.isnan(t)) or f == t
+
+
+# ----------------------------------------------------------------------------- combine
+def _mk(rng, T, K, E, R, H, replace=False):
+    idx, rts = random_case(rng, T, K, E, R, replace)
+    X = rand_bf16(rng, (T, H))
+    p = oracle.plan(idx, E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(idx, E, R, p, C, rts)
+    win = np.full((R * C, H), 0x7FC1, np.uint16)       # NaN canary: a wrong row poisons the sum
+    oracle.dispatch(X, slots, win)
+    return idx, rts, X, p, C, slots, win
+
+
+def test_combine_exact_rational_fma_chain():
+    """acc_j = round_f32(W_j * y_j + acc_{j-1}) exactly (one rounding per term, j
+    ascending), then one round to bf16 -- evaluated with exact rationals."""
+    rng = np.random.default_rng(11)
+    T, K, E, R, H = 12, 4, 8, 2, 8
+    idx, rts, X, p, C, slots, win = _mk(rng, T, K, E, R, H)
+    scale = rand_bf16(rng, (E,))
+    oracle.expert_scale(win, H, E, R, C, p.n_exp, scale)
+    W = rng.random((T, K)).astype(np.float32)
+    st, Y = oracle.combine(win, slots, W, H)
+    assert st == oracle.OK
+    Xf, sf = u16_to_float(X), u16_to_float(scale)
+    for t in range(T):
+        for h in range(H):
+            acc = Fraction(0)
+            for j in range(K):
+                y = bf16(Fraction(float(Xf[t, h])) * Fraction(float(sf[idx[t, j]])))   # stand-in expert, exact
+                acc = f32(Fraction(float(W[t, j])) * y + acc)
+            assert Fraction(float(u16_to_float(Y[t, h]))) == bf16(acc), (t, h)
+
+
+def test_combine_order_matters_and_is_j_ascending():
+    """Three terms chosen so that the fp32 result depends on the summation
+    order; only j = 0,1,2 ascending gives the expected value."""
+    H = 8
+    idx = np.array([[0, 1, 2]], np.int32)
+    p = oracle.plan(idx, 3, 1)
+    _, slots = oracle.slots(idx, 3, 1, p, 3)
+    win = np.zeros((3, H), np.uint16)
+    one = synth.bf16_to_u16(torch.tensor([1.0]).to(torch.bfloat16))[0]
+    win[:] = one
+    W = np.array([[2.0 ** 24, 1.0, 1.0]], np.float32)   # (2^24 + 1) + 1 = 2^24 in fp32; 2^24 + (1 + 1) = 2^24 + 2
+    st, Y = oracle.combine(win, slots, W, H)
+    assert u16_to_float(Y[0, 0]) == np.float32(2.0 ** 24)
+    W = np.array([[1.0, 1.0, 2.0 ** 24]], np.float32)
+    st, Y2 = oracle.combine(win, slots, W, H)
+    assert u16_to_float(Y2[0, 0]) == np.float32(2.0 ** 24)     # bf16 rounding hides +2 ...
+    # ... so check the fp32 chain through a case bf16 can see: 256 + 1 + 1 in units of 2^-16 ulp is
+    # invisible as well; instead use cancellation: (2^24 + 1) - 2^24 = 0 but 1 + (2^24 - 2^24) = 1.
+    W = np.array([[2.0 ** 24, 1.0, -(2.0 ** 24)]], np.float32)
+    _, Ya = oracle.combine(win, slots, W, H)
+    assert u16_to_float(Ya[0, 0]) == 0.0
+    W = np.array([[2.0 ** 24, -(2.0 ** 24), 1.0]], np.float32)
+    _, Yb = oracle.combine(win, slots, W, H)
+    assert u16_to_float(Yb[0, 0]) == 1.0
+
+
+@pytest.mark.parametrize("T,K,E,R,H", [(64, 8, 32, 4, 64), (200, 2, 8, 8, 128), (33, 6, 12, 3, 40)])
+def test_combine_within_one_ulp_of_fp64(T, K, E, R, H):
+    rng = np.random.default_rng(T + K)
+    idx, rts, X, p, C, slots, win = _mk(rng, T, K, E, R, H)
+    scale = rand_bf16(rng, (E,))
+    oracle.expert_scale(win, H, E, R, C, p.n_exp, scale)
+    logits = rng.standard_normal((T, K)).astype(np.float32)
+    W = (np.exp(logits) / np.exp(logits).sum(1, keepdims=True)).astype(np.float32)
+    st, Y = oracle.combine(win, slots, W, H, n_threads=2)
+    # closed form that never builds windows: Y[t] = sum_j W[t,j] * f_{K[t,j]}(X[t]) in fp64
+    Xf = u16_to_float(X).astype(np.float64)
+    sf = u16_to_float(scale)
+    ref = np.zeros((T, H))
+    mag = np.zeros((T, H))
+    for j in range(K):
+        y = torch.from_numpy((Xf * sf[idx[:, j]][:, None].astype(np.float64)).astype(np.float32)).to(torch.bfloat16)
+        term = W[:, j:j + 1].astype(np.float64) * y.double().numpy()
+        ref += term
+        mag += np.abs(term)
+    got = u16_to_float(Y).astype(np.float64)
+    # Error budget of the fp32 chain: K roundings of relative size 2^-24 on partial sums bounded by
+    # sum|W y|, then one bf16 rounding (half an ulp <= 2^-8 relative to the result).
+    bound = np.abs(ref) * 2.0 ** -8 * (1 + 1e-6) + K * 2.0 ** -24 * mag + 1e-45
+    assert (np.abs(got - ref) <= bound).all()
+    # and where no cancellation occurred it is within one bf16 ulp of the rounded fp64 value
+    ref_b = synth.bf16_to_u16(torch.from_numpy(ref).to(torch.float32).to(torch.bfloat16)).astype(np.int32)
+    key = lambda a: np.where(a & 0x8000, 0x8000 - (a & 0x7FFF), 0x8000 + a)
+    no_cancel = mag <= 4 * np.abs(ref)
+    assert no_cancel.mean() > 0.5
+    assert np.abs(key(Y.astype(np.int32)) - key(ref_b))[no_cancel].max() <= 1
+
+
+@pytest.mark.parametrize("K", [1, 2, 8])
+def test_combine_round_trip_closed_forms(K):
+    rng = np.random.default_rng(K)
+    T, E, R, H = 96, 16, 4, 32
+    idx, rts, X, p, C, slots, win = _mk(rng, T, K, E, R, H)
+    # identity experts, softmax weights (sum to 1 up to fp32 rounding): Y == X exactly,
+    # because the fp32 error is far below half a bf16 ulp and X is already bf16.
+    logits = rng.standard_normal((T, K)).astype(np.float32)
+    W = (np.exp(logits) / np.exp(logits).sum(1, keepdims=True)).astype(np.float32)
+    _, Y = oracle.combine(win, slots, W, H)
+    assert np.array_equal(u16_to_float(Y), u16_to_float(X))
+    # W = 1/K with K a power of two: every product and partial sum is exact.
+    _, Y = oracle.combine(win, slots, np.full((T, K), 1.0 / K, np.float32), H)
+    assert np.array_equal(u16_to_float(Y), u16_to_float(X))
+    # one-hot weights select exactly the chosen expert's output.
+    scale = rand_bf16(rng, (E,))
+    oracle.expert_scale(win, H, E, R, C, p.n_exp, scale)
+    hot = rng.integers(0, K, T)
+    W = np.zeros((T, K), np.float32)
+    W[np.arange(T), hot] = 1.0
+    _, Y = oracle.combine(win, slots, W, H)
+    want = torch.from_numpy(u16_to_float(X) * u16_to_float(scale)[idx[np.arange(T), hot]][:, None]).to(torch.bfloat16)
+    assert np.array_equal(u16_to_float(Y), want.float().numpy())
+
+
+# ----------------------------------------------------------------------------- workloads
+def test_benchmark_routing_recipes():
+    for n in (1, 2):
+        wl = synth.config(n)
+        idx, w, _, _ = synth.make_routing(wl)
+        assert idx.shape == (wl.T, wl.K) and idx.min() >= 0 and idx.max() < wl.E
+        srt = np.sort(idx.numpy(), 1)
+        assert (np.diff(srt, axis=1) > 0).all()                 # top-k without replacement
+        assert np.allclose(w.sum(1).numpy(), 1.0, atol=1e-6)
+        p = oracle.plan(idx.numpy(), wl.E, wl.R)
+        assert p.status == oracle.OK and p.M.sum() == wl.B
+    wl = synth.config(4)
+    idx, w, extra, _ = synth.make_routing(wl)
+    p = oracle.plan(idx.numpy(), wl.E, wl.R)
+    assert p.n_exp.max() >= 10 * wl.B / wl.E                     # hot experts hold > 10x the mean load
+    assert (np.diff(np.sort(idx.numpy(), 1), axis=1) > 0).all()
