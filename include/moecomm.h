@@ -1,0 +1,157 @@
+/* libmoecomm -- relay-buffer-free MoE dispatch / combine on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only.  Every pointer parameter says whether
+ * it is a HOST or a DEVICE pointer.  The library allocates no device memory:
+ * payload tensors and the control-state workspace are caller-owned.  All work
+ * is enqueued on the caller's CUDA stream (a cudaStream_t passed as void*; NULL
+ * is the default stream) and nothing synchronises except moe_status().
+ *
+ * Model (paper Section 3.2, Section 5.1).  The pooled, symmetric HBM of an
+ * expert-parallel group of R ranks is one allocation `windows` of R equal
+ * segments of C rows of H bf16 values; segment d is the expert window of rank
+ * d, which hosts experts d*E_r .. (d+1)*E_r-1, E_r = E / R.  Tokens of all
+ * source ranks are concatenated in rank order; source rank r owns tokens
+ * rank_tok_start[r] .. rank_tok_start[r+1]-1.  A routed branch (t, j) with
+ * expert e = K[t,j] lives in window row
+ *
+ *     slot(t,j) = dst(e) * C + o[e, src(t)] + s[t,j],      dst(e) = e / E_r
+ *
+ * (two-level offset rule, Section 5.1): o is the large offset (start of the
+ * block "source rank r -> expert e" inside rank dst(e)'s window; blocks are laid
+ * out expert-major, then by source rank), s is the small offset (number of
+ * earlier branches, in (t, j) order, of the same source rank to the same
+ * expert).  Slots are therefore deterministic and stable in token order.
+ *
+ * Limits: 1 <= R <= MOE_MAX_R, E % R == 0, E <= MOE_MAX_E, 1 <= K <= MOE_MAX_K,
+ * H % 8 == 0 (rows are whole 16-byte chunks), T_max * K < 2^31.
+ * Thread safety: one context per stream; a context holds no global state.
+ */
+#ifndef MOECOMM_H
+#define MOECOMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOE_MAX_R 256
+#define MOE_MAX_E 4096
+#define MOE_MAX_K 32
+
+typedef enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = 1, /* host-detected: null/misaligned pointer, bad shape, T > T_max ...      */
+  MOE_ERR_BAD_INDEX = 2,   /* device-detected by moe_plan: a routing index outside [0, E)           */
+  MOE_ERR_CAPACITY = 3,    /* device-detected: some n_recv[d] > capacity_rows; nothing was written  */
+  MOE_ERR_NOT_PLANNED = 4, /* dispatch / combine / slots / view before a successful moe_plan        */
+  MOE_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired                                    */
+  MOE_ERR_CUDA = 6         /* a CUDA runtime call or kernel launch failed                           */
+} moe_status_t;
+
+/* The two schedules of Section 4.  PREFILL runs Layout + Notify as separate
+ * planning passes and keeps the whole planning table readable.  DECODE keeps
+ * only the compact state (o_dec, delta, n_recv); delta is produced inside the
+ * dispatch launch (Section 5.3, Decode Dispatch). */
+typedef enum { MOE_SCHED_PREFILL = 0, MOE_SCHED_DECODE = 1 } moe_schedule_t;
+
+typedef struct {
+  int32_t T_max; /* largest total token count a plan may be asked for */
+  int32_t H;     /* hidden size, multiple of 8                        */
+  int32_t E;     /* experts                                           */
+  int32_t R;     /* virtual expert-parallel ranks                     */
+  int32_t K;     /* top-k routing degree                              */
+} moe_shape_t;
+
+typedef struct moe_ctx moe_ctx_t; /* opaque, HOST-side handle */
+
+/* Bytes of DEVICE workspace a context of this shape needs (control state only:
+ * O(T_max*K + R*E) int32).  0 if the shape is invalid. */
+size_t moe_workspace_bytes(const moe_shape_t* shape /*HOST*/);
+
+/* Creates a context over a caller-owned DEVICE workspace (256-byte aligned, at
+ * least moe_workspace_bytes(shape) bytes, must outlive the context).  Clears
+ * the control words with a synchronous memset; call it outside stream capture.
+ * The context is bound to the CUDA device that is current at this call. */
+moe_status_t moe_create(const moe_shape_t* shape /*HOST*/, void* workspace /*DEVICE*/,
+                        size_t workspace_bytes, moe_ctx_t** out /*HOST*/);
+moe_status_t moe_destroy(moe_ctx_t* ctx);
+
+/* Planning (Section 5.2 Prefill Layout + Prefill Notify; Section 5.3 first step
+ * of Decode Dispatch): from the routing indexes computes the count matrix M,
+ * the small offsets s and the large offsets o (exclusive scan of M in window
+ * order), plus c_rank, n_exp, n_recv.
+ *   topk_idx        DEVICE [T,K] int32, values in [0,E)
+ *   rank_tok_start  HOST   [R+1] int32, nondecreasing, [0]=0, [R]=T; NULL means
+ *                   uniform T/R tokens per rank (T % R must be 0).  Read before
+ *                   the call returns.
+ * An index outside [0,E) sets the device status word to MOE_ERR_BAD_INDEX; the
+ * offending branch is ignored by the counts and later calls write nothing
+ * until moe_status() has cleared the word. */
+moe_status_t moe_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE*/,
+                      int32_t T, const int32_t* rank_tok_start /*HOST*/, void* stream);
+
+/* DEVICE views into the workspace, valid until the next moe_plan on this
+ * context.  Shapes: counts M [R,E], c_rank [R,R], small_off s|delta [T,K],
+ * large_off o|o_dec [E,R] (window-local row), n_exp [E], n_recv [R].
+ * PREFILL fills every field.  DECODE leaves counts, c_rank and n_exp NULL, and
+ * small_off holds delta only after moe_dispatch has run. */
+typedef struct {
+  const int32_t* counts;
+  const int32_t* c_rank;
+  const int32_t* small_off;
+  const int32_t* large_off;
+  const int32_t* n_exp;
+  const int32_t* n_recv;
+} moe_plan_view_t;
+moe_status_t moe_plan_view(const moe_ctx_t* ctx, moe_plan_view_t* out /*HOST*/);
+
+/* Dispatch (Algorithm 1 / Algorithm 2, first loop; Section 5.2 Prefill Dispatch):
+ * copies row X[t,:] to window row slot(t,j) for every branch.
+ *   x        DEVICE [T,H] bf16, 16-byte aligned
+ *   windows  DEVICE [R, capacity_rows, H] bf16, 16-byte aligned
+ * Rows >= n_recv[d] of segment d are never written.  If some n_recv[d] exceeds
+ * capacity_rows the status word becomes MOE_ERR_CAPACITY and nothing is written. */
+moe_status_t moe_dispatch(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows /*DEVICE*/,
+                          int64_t capacity_rows, void* stream);
+
+/* Combine (Algorithm 1 / Algorithm 2, second loop; Section 5.2 Prefill Combine):
+ *   Y[t,h] = bf16_rne( sum_{j=0..K-1} W[t,j] * float(windows[slot(t,j), h]) )
+ * accumulated in fp32 from +0 with one fused multiply-add per term, j ascending.
+ *   windows  DEVICE expert outputs, same layout as in moe_dispatch
+ *   topk_w   DEVICE [T,K] fp32
+ *   y        DEVICE [T,H] bf16, 16-byte aligned, fully overwritten */
+moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows /*DEVICE*/, int64_t capacity_rows,
+                         const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
+
+/* Materialises slot(t,j) into caller memory (parity checks, expert-side
+ * consumers).  slots DEVICE [T,K] int32; needs R * capacity_rows < 2^31. */
+moe_status_t moe_slots(moe_ctx_t* ctx, int64_t capacity_rows, int32_t* slots /*DEVICE*/, void* stream);
+
+/* One whole layer call from HOST buffers, enqueued on `stream`:
+ * host->device copies of x, topk_idx, topk_w; plan; dispatch; combine reading
+ * the dispatched windows (identity experts); device->host copy of y.
+ * The *_dev arguments are caller-owned DEVICE staging buffers of the shapes
+ * given above.  Pass pinned host memory for the copies to be asynchronous.
+ * rank_tok_start as in moe_plan.  Call moe_status() to wait for the result. */
+moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T,
+                              const int32_t* rank_tok_start /*HOST*/,
+                              const void* x_host, const int32_t* topk_idx_host, const float* topk_w_host,
+                              void* x_dev, int32_t* topk_idx_dev, float* topk_w_dev,
+                              void* windows_dev, int64_t capacity_rows, void* y_dev,
+                              void* y_host, void* stream);
+
+/* Synchronises `stream`, then returns and clears the device status word
+ * (first device-detected error since the last call, or MOE_OK). */
+moe_status_t moe_status(moe_ctx_t* ctx, void* stream);
+
+const char* moe_status_string(moe_status_t status);
+
+/* Number of kernel launches this context has enqueued so far (for benchmarks). */
+int64_t moe_launch_count(const moe_ctx_t* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,230 @@
+"""Thin ctypes binding of libmoecomm (argument marshalling only).
+
+Function names mirror the C ABI in ``include/moecomm.h``.  Tensors are torch
+CUDA tensors used purely as device memory; every step of the path runs in the
+library's CUDA kernels.  There is no CPU fallback: if ``libmoecomm.so`` has not
+been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmoecomm.so")
+
+MOE_OK, MOE_ERR_INVALID_ARG, MOE_ERR_BAD_INDEX, MOE_ERR_CAPACITY = 0, 1, 2, 3
+MOE_ERR_NOT_PLANNED, MOE_ERR_TIMEOUT, MOE_ERR_CUDA = 4, 5, 6
+MOE_SCHED_PREFILL, MOE_SCHED_DECODE = 0, 1
+
+EXPORTS = [
+    "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
+    "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
+]
+
+
+class MoeShape(ctypes.Structure):
+    _fields_ = [("T_max", ctypes.c_int32), ("H", ctypes.c_int32), ("E", ctypes.c_int32),
+                ("R", ctypes.c_int32), ("K", ctypes.c_int32)]
+
+
+class MoePlanView(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("counts", "c_rank", "small_off", "large_off", "n_exp", "n_recv")]
+
+
+class MoeError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads the built library; raises if it is missing (no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is not built; run `python -m paper_2605_06055_b200.build` "
+                           "(or __graft_entry__.build()). There is no CPU fallback.")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    L.moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeShape)]
+    L.moe_workspace_bytes.restype = ctypes.c_size_t
+    L.moe_create.argtypes = [ctypes.POINTER(MoeShape), vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    L.moe_destroy.argtypes = [vp]
+    L.moe_plan.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp]
+    L.moe_plan_view.argtypes = [vp, ctypes.POINTER(MoePlanView)]
+    L.moe_dispatch.argtypes = [vp, vp, vp, i64, vp]
+    L.moe_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.moe_slots.argtypes = [vp, i64, vp, vp]
+    L.moe_forward_host.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
+    L.moe_status.argtypes = [vp, vp]
+    L.moe_status_string.argtypes = [ctypes.c_int]
+    L.moe_status_string.restype = ctypes.c_char_p
+    L.moe_launch_count.argtypes = [vp]
+    L.moe_launch_count.restype = i64
+    for name in ("moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch", "moe_combine",
+                 "moe_slots", "moe_forward_host", "moe_status"):
+        getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return load().moe_status_string(int(code)).decode()
+
+
+def moe_workspace_bytes(T_max: int, H: int, E: int, R: int, K: int) -> int:
+    return int(load().moe_workspace_bytes(ctypes.byref(MoeShape(T_max, H, E, R, K))))
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, (t.dtype, dtype)
+    return t.data_ptr()
+
+
+def _host_ptr(t, dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"]
+        return t.ctypes.data
+    assert not t.is_cuda and t.is_contiguous()
+    if dtype is not None:
+        assert t.dtype == dtype
+    return t.data_ptr()
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+class MoeComm:
+    """One libmoecomm context (opaque handle + its torch-allocated workspace)."""
+
+    def __init__(self, T_max: int, H: int, E: int, R: int, K: int, device="cuda:0"):
+        self.lib = load()
+        self.device = torch.device(device)
+        self.T_max, self.H, self.E, self.R, self.K = T_max, H, E, R, K
+        self._shape = MoeShape(T_max, H, E, R, K)
+        nbytes = int(self.lib.moe_workspace_bytes(ctypes.byref(self._shape)))
+        if nbytes == 0:
+            raise MoeError(MOE_ERR_INVALID_ARG, "moe_workspace_bytes")
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            h = ctypes.c_void_p()
+            rc = self.lib.moe_create(ctypes.byref(self._shape), self.workspace.data_ptr(), nbytes, ctypes.byref(h))
+        if rc != MOE_OK:
+            raise MoeError(rc, "moe_create")
+        self._h = h
+        self.T = 0
+        self.schedule = None
+        self._keep = None  # routing tensor of the live plan (the library re-reads it)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.moe_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- C ABI calls, same names -------------------------------------------------
+    def moe_plan(self, schedule: int, topk_idx: torch.Tensor, T: Optional[int] = None, rank_tok_start=None,
+                 stream=None, check: bool = True) -> int:
+        T = topk_idx.shape[0] if T is None else T
+        rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_plan(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, _host_ptr(rts),
+                                   _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx
+        elif check:
+            raise MoeError(rc, "moe_plan")
+        return rc
+
+    def moe_plan_view(self) -> dict:
+        """Zero-copy int32 tensors over the planning state in the workspace."""
+        v = MoePlanView()
+        rc = self.lib.moe_plan_view(self._h, ctypes.byref(v))
+        if rc != MOE_OK:
+            raise MoeError(rc, "moe_plan_view")
+        base = self.workspace.data_ptr()
+        shapes = {"counts": (self.R, self.E), "c_rank": (self.R, self.R), "small_off": (self.T, self.K),
+                  "large_off": (self.E, self.R), "n_exp": (self.E,), "n_recv": (self.R,)}
+        out = {}
+        for name, shp in shapes.items():
+            p = getattr(v, name)
+            if p is None:
+                out[name] = None
+                continue
+            n = int(np.prod(shp))
+            off = p - base
+            out[name] = self.workspace[off:off + 4 * n].view(torch.int32).view(*shp)
+        return out
+
+    def moe_dispatch(self, x: torch.Tensor, windows: torch.Tensor, capacity_rows: int, stream=None,
+                     check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_dispatch(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(windows, torch.bfloat16),
+                                       int(capacity_rows), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch")
+        return rc
+
+    def moe_combine(self, windows: torch.Tensor, capacity_rows: int, topk_w: torch.Tensor, y: torch.Tensor,
+                    stream=None, check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_combine(self._h, _dev_ptr(windows, torch.bfloat16), int(capacity_rows),
+                                      _dev_ptr(topk_w, torch.float32), _dev_ptr(y, torch.bfloat16),
+                                      _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_combine")
+        return rc
+
+    def moe_slots(self, capacity_rows: int, slots: torch.Tensor, stream=None, check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_slots(self._h, int(capacity_rows), _dev_ptr(slots, torch.int32),
+                                    _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_slots")
+        return rc
+
+    def moe_forward_host(self, schedule: int, T: int, rank_tok_start, x_host, topk_idx_host, topk_w_host,
+                         x_dev, topk_idx_dev, topk_w_dev, windows_dev, capacity_rows: int, y_dev, y_host,
+                         stream=None, check: bool = True) -> int:
+        rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_forward_host(
+                self._h, schedule, T, _host_ptr(rts), _host_ptr(x_host), _host_ptr(topk_idx_host),
+                _host_ptr(topk_w_host), _dev_ptr(x_dev), _dev_ptr(topk_idx_dev), _dev_ptr(topk_w_dev),
+                _dev_ptr(windows_dev), int(capacity_rows), _dev_ptr(y_dev), _host_ptr(y_host),
+                _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx_dev
+        elif check:
+            raise MoeError(rc, "moe_forward_host")
+        return rc
+
+    def moe_status(self, stream=None) -> int:
+        with torch.cuda.device(self.device):
+            return int(self.lib.moe_status(self._h, _stream_handle(stream)))
+
+    def moe_launch_count(self) -> int:
+        return int(self.lib.moe_launch_count(self._h))

@@ -1,0 +1,391 @@
+// libmoecomm: host side of the C ABI declared in include/moecomm.h.
+// Argument validation, workspace layout, launch configuration.  Every step of
+// the path runs in the kernels of plan_kernels.cuh and row_kernels.cuh.
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "plan_kernels.cuh"
+#include "row_kernels.cuh"
+
+using namespace moe;
+
+struct moe_ctx {
+  moe_shape_t shape;
+  int device;
+  int num_sms;
+  char* ws;
+  size_t ws_bytes;
+  // workspace views (device)
+  Control* ctl;
+  int32_t *M, *c_rank, *o, *n_exp, *n_recv, *s, *tile_rank, *tile_hist;
+  // plan state (host)
+  bool planned;
+  moe_schedule_t schedule;
+  int32_t T;
+  int32_t n_tiles;
+  const int32_t* topk_idx;  // device; routing indexes of the current plan, read again by dispatch/combine
+  RankMap map;
+  int64_t launches;
+};
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+bool shape_valid(const moe_shape_t* s) {
+  if (s == nullptr) return false;
+  if (s->R < 1 || s->R > MOE_MAX_R || s->E < 1 || s->E > MOE_MAX_E || s->E % s->R != 0) return false;
+  if (s->K < 1 || s->K > MOE_MAX_K || s->H < 8 || s->H % 8 != 0 || s->T_max < 0) return false;
+  if ((int64_t)s->T_max * s->K >= (int64_t)1 << 31) return false;
+  return true;
+}
+
+int64_t max_tiles(const moe_shape_t* s) {
+  const int64_t B = (int64_t)s->T_max * s->K;
+  const int64_t smallest_tile = ROUNDS_DECODE * PLAN_THREADS;
+  return (B + smallest_tile - 1) / smallest_tile + s->R;  // every rank may end in a partial tile
+}
+
+struct Layout {
+  size_t ctl, M, c_rank, o, n_exp, n_recv, s, tile_rank, tile_hist, total;
+};
+
+Layout layout_of(const moe_shape_t* s) {
+  Layout L;
+  size_t at = 0;
+  auto take = [&](size_t bytes) {
+    size_t here = at;
+    at = align_up(at + bytes);
+    return here;
+  };
+  const size_t B = (size_t)s->T_max * s->K;
+  L.ctl = take(sizeof(Control));
+  L.M = take(sizeof(int32_t) * s->R * s->E);
+  L.c_rank = take(sizeof(int32_t) * s->R * s->R);
+  L.o = take(sizeof(int32_t) * s->E * s->R);
+  L.n_exp = take(sizeof(int32_t) * s->E);
+  L.n_recv = take(sizeof(int32_t) * s->R);
+  L.s = take(sizeof(int32_t) * B);
+  L.tile_rank = take(sizeof(int32_t) * B);
+  L.tile_hist = take(sizeof(int32_t) * (size_t)max_tiles(s) * s->E);
+  L.total = at;
+  return L;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+moe_status_t launch_ok(moe_ctx* ctx, int n = 1) {
+  ctx->launches += n;
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
+  RowArgs a;
+  const moe_shape_t& sh = ctx->shape;
+  a.topk_idx = nullptr;  // set by caller
+  // DECODE: small offsets are finished on the fly (in-tile rank + tile base) by every consumer, so a
+  // dispatch that aborted on the device can never leave a later call with half-written state; the
+  // dispatch launch also records them, which is what moe_plan_view exposes as delta.
+  const bool finish_delta = ctx->schedule == MOE_SCHED_DECODE;
+  a.small_off = finish_delta ? ctx->tile_rank : ctx->s;
+  a.small_out = (finish_delta && dispatching) ? ctx->s : nullptr;
+  a.tile_base = finish_delta ? ctx->tile_hist : nullptr;
+  a.large_off = ctx->o;
+  a.n_recv = ctx->n_recv;
+  a.status = &ctx->ctl->status;
+  a.C = C;
+  a.T = ctx->T;
+  a.K = sh.K;
+  a.E = sh.E;
+  a.R = sh.R;
+  a.E_r = sh.E / sh.R;
+  a.H16 = sh.H / 8;
+  return a;
+}
+
+int row_grid(const moe_ctx* ctx, int warps_per_cta, int ctas_per_sm) {
+  const int64_t need = ((int64_t)ctx->T + warps_per_cta - 1) / warps_per_cta;
+  const int64_t cap = (int64_t)ctx->num_sms * ctas_per_sm;
+  return (int)(need < cap ? (need < 1 ? 1 : need) : cap);
+}
+
+template <int KT>
+void launch_dispatch(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
+  const int grid = row_grid(ctx, 8, 8);
+  dispatch_rows_kernel<KT, 4><<<grid, 256, 0, st>>>(x, win, a, ctx->map);
+}
+
+template <int KT>
+void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const float* w, uint4* y, cudaStream_t st) {
+  const int grid = row_grid(ctx, 8, 8);
+  combine_rows_kernel<KT, (KT > 4 ? 1 : 2)><<<grid, 256, 0, st>>>(win, w, y, a, ctx->map);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t moe_workspace_bytes(const moe_shape_t* shape) {
+  if (!shape_valid(shape)) return 0;
+  return layout_of(shape).total;
+}
+
+moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t workspace_bytes, moe_ctx_t** out) {
+  if (out == nullptr) return MOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!shape_valid(shape) || workspace == nullptr) return MOE_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % ALIGN != 0) return MOE_ERR_INVALID_ARG;
+  const Layout L = layout_of(shape);
+  if (workspace_bytes < L.total) return MOE_ERR_INVALID_ARG;
+
+  moe_ctx* ctx = new (std::nothrow) moe_ctx();
+  if (ctx == nullptr) return MOE_ERR_CUDA;
+  ctx->shape = *shape;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess) {
+    delete ctx;
+    return MOE_ERR_CUDA;
+  }
+  ctx->ws = static_cast<char*>(workspace);
+  ctx->ws_bytes = workspace_bytes;
+  ctx->ctl = reinterpret_cast<Control*>(ctx->ws + L.ctl);
+  ctx->M = reinterpret_cast<int32_t*>(ctx->ws + L.M);
+  ctx->c_rank = reinterpret_cast<int32_t*>(ctx->ws + L.c_rank);
+  ctx->o = reinterpret_cast<int32_t*>(ctx->ws + L.o);
+  ctx->n_exp = reinterpret_cast<int32_t*>(ctx->ws + L.n_exp);
+  ctx->n_recv = reinterpret_cast<int32_t*>(ctx->ws + L.n_recv);
+  ctx->s = reinterpret_cast<int32_t*>(ctx->ws + L.s);
+  ctx->tile_rank = reinterpret_cast<int32_t*>(ctx->ws + L.tile_rank);
+  ctx->tile_hist = reinterpret_cast<int32_t*>(ctx->ws + L.tile_hist);
+  ctx->planned = false;
+  ctx->launches = 0;
+  ctx->topk_idx = nullptr;
+
+  // Shared memory of the planning kernels grows with E; opt in above 48 KB.
+  const int tile_smem = PLAN_WARPS * shape->E * (int)sizeof(int32_t);
+  bool ok = cudaMemset(ctx->ctl, 0, sizeof(Control)) == cudaSuccess;
+  if (ok && tile_smem > 48 * 1024) {
+    ok = cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_PREFILL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              tile_smem) == cudaSuccess &&
+         cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_DECODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              tile_smem) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    delete ctx;
+    return MOE_ERR_CUDA;
+  }
+  *out = ctx;
+  return MOE_OK;
+}
+
+moe_status_t moe_destroy(moe_ctx_t* ctx) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  delete ctx;
+  return MOE_OK;
+}
+
+moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                      const int32_t* rank_tok_start, void* stream) {
+  moe_ctx* ctx = c;
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  const moe_shape_t& sh = ctx->shape;
+  if (schedule != MOE_SCHED_PREFILL && schedule != MOE_SCHED_DECODE) return MOE_ERR_INVALID_ARG;
+  if (T < 0 || T > sh.T_max || (T > 0 && topk_idx == nullptr)) return MOE_ERR_INVALID_ARG;
+  if (rank_tok_start == nullptr && T % sh.R != 0) return MOE_ERR_INVALID_ARG;
+  if (rank_tok_start != nullptr) {
+    if (rank_tok_start[0] != 0 || rank_tok_start[sh.R] != T) return MOE_ERR_INVALID_ARG;
+    for (int r = 0; r < sh.R; ++r)
+      if (rank_tok_start[r + 1] < rank_tok_start[r]) return MOE_ERR_INVALID_ARG;
+  }
+  ctx->planned = false;
+
+  const int rounds = schedule == MOE_SCHED_PREFILL ? ROUNDS_PREFILL : ROUNDS_DECODE;
+  const int tile_branches = rounds * PLAN_THREADS;
+  RankMap& map = ctx->map;
+  std::memset(&map, 0, sizeof(map));
+  map.R = sh.R;
+  map.uniform_tokens = (rank_tok_start == nullptr && T > 0) ? T / sh.R : 0;
+  map.tile_shift = 0;
+  while ((1 << map.tile_shift) < tile_branches) ++map.tile_shift;
+  int32_t tiles = 0;
+  for (int r = 0; r <= sh.R; ++r) {
+    const int32_t tok = rank_tok_start != nullptr ? rank_tok_start[r] : (int32_t)((int64_t)T / sh.R * r);
+    map.tok_start[r] = tok;
+    map.tile_start[r] = tiles;
+    if (r < sh.R) {
+      const int32_t next = rank_tok_start != nullptr ? rank_tok_start[r + 1] : (int32_t)((int64_t)T / sh.R * (r + 1));
+      const int64_t branches = (int64_t)(next - tok) * sh.K;
+      tiles += (int32_t)((branches + tile_branches - 1) / tile_branches);
+    }
+  }
+  ctx->n_tiles = tiles;
+  ctx->T = T;
+  ctx->schedule = schedule;
+  ctx->topk_idx = topk_idx;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int tile_smem = PLAN_WARPS * sh.E * (int)sizeof(int32_t);
+  const int scan_smem = (2 * sh.E + 1) * (int)sizeof(int32_t);
+  const int full = schedule == MOE_SCHED_PREFILL;
+  int n = 0;
+  if (tiles > 0) {
+    if (full)
+      plan_tile_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, tile_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
+    else
+      plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, tile_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
+    ++n;
+  }
+  plan_scan_kernel<<<sh.R, PLAN_THREADS, scan_smem, st>>>(ctx->tile_hist, map, sh.E, full, ctx->M, ctx->c_rank,
+                                                          ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+  ++n;
+  if (full && tiles > 0) {
+    plan_finalize_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, 0, st>>>(topk_idx, map, sh.K, sh.E, ctx->tile_rank,
+                                                                        ctx->tile_hist, ctx->s);
+    ++n;
+  }
+  const moe_status_t rc = launch_ok(ctx, n);
+  if (rc == MOE_OK) ctx->planned = true;
+  return rc;
+}
+
+moe_status_t moe_plan_view(const moe_ctx_t* c, moe_plan_view_t* out) {
+  if (c == nullptr || out == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!c->planned) return MOE_ERR_NOT_PLANNED;
+  const bool full = c->schedule == MOE_SCHED_PREFILL;
+  out->counts = full ? c->M : nullptr;
+  out->c_rank = full ? c->c_rank : nullptr;
+  out->small_off = c->s;
+  out->large_off = c->o;
+  out->n_exp = full ? c->n_exp : nullptr;
+  out->n_recv = c->n_recv;
+  return MOE_OK;
+}
+
+moe_status_t moe_dispatch(moe_ctx_t* c, const void* x, void* windows, int64_t capacity_rows, void* stream) {
+  moe_ctx* ctx = c;
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || windows == nullptr))) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(windows)) return MOE_ERR_INVALID_ARG;
+  RowArgs a = row_args(ctx, capacity_rows, true);
+  a.topk_idx = ctx->topk_idx;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const uint4* xs = static_cast<const uint4*>(x);
+  uint4* win = static_cast<uint4*>(windows);
+  switch (ctx->shape.K) {
+    case 1: launch_dispatch<1>(ctx, a, xs, win, st); break;
+    case 2: launch_dispatch<2>(ctx, a, xs, win, st); break;
+    case 4: launch_dispatch<4>(ctx, a, xs, win, st); break;
+    case 6: launch_dispatch<6>(ctx, a, xs, win, st); break;
+    case 8: launch_dispatch<8>(ctx, a, xs, win, st); break;
+    default: launch_dispatch<0>(ctx, a, xs, win, st); break;
+  }
+  return launch_ok(ctx);
+}
+
+moe_status_t moe_combine(moe_ctx_t* c, const void* windows, int64_t capacity_rows, const float* topk_w, void* y,
+                         void* stream) {
+  moe_ctx* ctx = c;
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  if (capacity_rows < 0 || (ctx->T > 0 && (windows == nullptr || topk_w == nullptr || y == nullptr)))
+    return MOE_ERR_INVALID_ARG;
+  if (!aligned16(windows) || !aligned16(y)) return MOE_ERR_INVALID_ARG;
+  RowArgs a = row_args(ctx, capacity_rows, false);
+  a.topk_idx = ctx->topk_idx;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const uint4* win = static_cast<const uint4*>(windows);
+  uint4* ys = static_cast<uint4*>(y);
+  switch (ctx->shape.K) {
+    case 1: launch_combine<1>(ctx, a, win, topk_w, ys, st); break;
+    case 2: launch_combine<2>(ctx, a, win, topk_w, ys, st); break;
+    case 4: launch_combine<4>(ctx, a, win, topk_w, ys, st); break;
+    case 6: launch_combine<6>(ctx, a, win, topk_w, ys, st); break;
+    case 8: launch_combine<8>(ctx, a, win, topk_w, ys, st); break;
+    default: launch_combine<0>(ctx, a, win, topk_w, ys, st); break;
+  }
+  return launch_ok(ctx);
+}
+
+moe_status_t moe_slots(moe_ctx_t* c, int64_t capacity_rows, int32_t* slots, void* stream) {
+  moe_ctx* ctx = c;
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  if (capacity_rows < 0 || (int64_t)ctx->shape.R * capacity_rows >= (int64_t)1 << 31) return MOE_ERR_INVALID_ARG;
+  if (ctx->T > 0 && slots == nullptr) return MOE_ERR_INVALID_ARG;
+  RowArgs a = row_args(ctx, capacity_rows, false);
+  a.topk_idx = ctx->topk_idx;
+  const int64_t B = (int64_t)ctx->T * ctx->shape.K;
+  int grid = (int)((B + 255) / 256);
+  if (grid < 1) grid = 1;
+  if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
+  slots_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(slots, a, ctx->map);
+  return launch_ok(ctx);
+}
+
+moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T, const int32_t* rank_tok_start,
+                              const void* x_host, const int32_t* topk_idx_host, const float* topk_w_host,
+                              void* x_dev, int32_t* topk_idx_dev, float* topk_w_dev, void* windows_dev,
+                              int64_t capacity_rows, void* y_dev, void* y_host, void* stream) {
+  if (ctx == nullptr || T < 0 || T > ctx->shape.T_max) return MOE_ERR_INVALID_ARG;
+  if (T > 0 && (x_host == nullptr || topk_idx_host == nullptr || topk_w_host == nullptr || x_dev == nullptr ||
+                topk_idx_dev == nullptr || topk_w_dev == nullptr || windows_dev == nullptr || y_dev == nullptr ||
+                y_host == nullptr))
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t row_bytes = (size_t)ctx->shape.H * 2, B = (size_t)T * ctx->shape.K;
+  if (T > 0) {
+    if (cudaMemcpyAsync(topk_idx_dev, topk_idx_host, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(topk_w_dev, topk_w_host, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(x_dev, x_host, (size_t)T * row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return MOE_ERR_CUDA;
+  }
+  moe_status_t rc = moe_plan(ctx, schedule, topk_idx_dev, T, rank_tok_start, stream);
+  if (rc != MOE_OK) return rc;
+  rc = moe_dispatch(ctx, x_dev, windows_dev, capacity_rows, stream);
+  if (rc != MOE_OK) return rc;
+  rc = moe_combine(ctx, windows_dev, capacity_rows, topk_w_dev, y_dev, stream);
+  if (rc != MOE_OK) return rc;
+  if (T > 0 && cudaMemcpyAsync(y_host, y_dev, (size_t)T * row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+moe_status_t moe_status(moe_ctx_t* ctx, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t word = 0;
+  if (cudaMemcpyAsync(&word, &ctx->ctl->status, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (word != 0) {
+    if (cudaMemsetAsync(&ctx->ctl->status, 0, sizeof(word), st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+      return MOE_ERR_CUDA;
+  }
+  return (word >= 0 && word <= MOE_ERR_CUDA) ? static_cast<moe_status_t>(word) : MOE_ERR_CUDA;
+}
+
+const char* moe_status_string(moe_status_t status) {
+  switch (status) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_ERR_BAD_INDEX: return "routing index outside [0, E)";
+    case MOE_ERR_CAPACITY: return "expert window capacity too small";
+    case MOE_ERR_NOT_PLANNED: return "no plan: call moe_plan first";
+    case MOE_ERR_TIMEOUT: return "bounded device wait expired";
+    case MOE_ERR_CUDA: return "CUDA error";
+  }
+  return "unknown status";
+}
+
+int64_t moe_launch_count(const moe_ctx_t* ctx) { return ctx == nullptr ? 0 : ctx->launches; }
+
+}  // extern "C"

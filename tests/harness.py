@@ -1,0 +1,134 @@
+"""Test harness: runs one workload through the CUDA library (via the C ABI
+binding) and through the CPU oracle on the same seeded inputs.
+
+The harness owns what is not part of the method: device buffers, canary fill,
+and the stand-in expert op between dispatch and combine.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2605_06055_b200 import binding, synth
+
+CANARY = 0x7FC1  # a bf16 NaN pattern: a stray read poisons the sum, a stray write is visible
+
+
+def bf16_key(a: np.ndarray) -> np.ndarray:
+    """Monotone integer view of bf16 bit patterns (difference = distance in ulps)."""
+    a = a.astype(np.int32)
+    return np.where(a & 0x8000, 0x8000 - (a & 0x7FFF), 0x8000 + a)
+
+
+def max_ulp_diff(got_u16: np.ndarray, want_u16: np.ndarray) -> int:
+    """Largest bf16 ulp distance; NaN matches NaN, +0 matches -0."""
+    g, w = got_u16.astype(np.int32), want_u16.astype(np.int32)
+    g_nan = ((g & 0x7F80) == 0x7F80) & ((g & 0x7F) != 0)
+    w_nan = ((w & 0x7F80) == 0x7F80) & ((w & 0x7F) != 0)
+    if not np.array_equal(g_nan, w_nan):
+        return 1 << 30
+    d = np.abs(bf16_key(g) - bf16_key(w))
+    d[g_nan] = 0
+    return int(d.max()) if d.size else 0
+
+
+def gpu_expert_scale(windows: torch.Tensor, topk_idx: torch.Tensor, E: int, R: int, C: int,
+                     scale: torch.Tensor) -> None:
+    """Stand-in expert op on the device (harness code, not the library):
+    every received row of expert e is multiplied by the bf16 scalar scale[e]."""
+    n_exp = torch.bincount(topk_idx.reshape(-1).long(), minlength=E)
+    E_r = E // R
+    win = windows.view(R, C, -1)
+    for d in range(R):
+        cnt = n_exp[d * E_r:(d + 1) * E_r]
+        rows = int(cnt.sum())
+        if rows == 0:
+            continue
+        row_scale = torch.repeat_interleave(scale[d * E_r:(d + 1) * E_r], cnt)
+        win[d, :rows] = win[d, :rows] * row_scale[:, None]     # bf16*bf16: fp32 product, one RNE rounding
+
+
+@dataclass
+class OracleRun:
+    plan: oracle.Plan
+    slots: np.ndarray
+    windows: np.ndarray
+    Y: np.ndarray
+
+
+def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4) -> OracleRun:
+    wl = inp.wl
+    idx = inp.topk_idx.numpy()
+    p = oracle.plan(idx, wl.E, wl.R, inp.rank_tok_start)
+    assert p.status == oracle.OK
+    st, slots = oracle.slots(idx, wl.E, wl.R, p, C, inp.rank_tok_start)
+    assert st == oracle.OK
+    win = np.full((wl.R * C, wl.H), CANARY, np.uint16)
+    assert oracle.dispatch(synth.bf16_to_u16(inp.X), slots, win, n_threads) == oracle.OK
+    win_after_dispatch = win.copy()
+    if wl.expert_op == "scale":
+        assert oracle.expert_scale(win, wl.H, wl.E, wl.R, C, p.n_exp, synth.bf16_to_u16(inp.scale)) == oracle.OK
+    st, Y = oracle.combine(win, slots, inp.topk_w.numpy(), wl.H, n_threads)
+    assert st == oracle.OK
+    return OracleRun(p, slots, win_after_dispatch, Y)
+
+
+@dataclass
+class GpuRun:
+    view: dict          # plan tensors copied to host (numpy) after the run
+    slots: np.ndarray
+    windows: np.ndarray  # after dispatch, before the expert op
+    Y: np.ndarray
+    statuses: list
+
+
+def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Optional[binding.MoeComm] = None,
+            T_max: Optional[int] = None) -> GpuRun:
+    wl = inp.wl
+    dev = torch.device("cuda:0")
+    schedule = wl.schedule if schedule is None else schedule
+    own = comm is None
+    if own:
+        comm = binding.MoeComm(T_max or max(wl.T, 1), wl.H, wl.E, wl.R, wl.K, dev)
+    idx = inp.topk_idx.to(dev)
+    w = inp.topk_w.to(dev)
+    X = inp.X.to(dev)
+    rts = None if wl.rank_tokens is None else inp.rank_tok_start
+    statuses = []
+    comm.moe_plan(schedule, idx, wl.T, rts)
+    statuses.append(comm.moe_status())
+    slots = torch.full((wl.T, wl.K), -5, dtype=torch.int32, device=dev)
+    comm.moe_slots(C, slots)
+    windows = torch.from_numpy(np.full((wl.R * C, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    comm.moe_dispatch(X, windows, C)
+    statuses.append(comm.moe_status())
+    view = {k: (None if v is None else v.cpu().numpy().copy()) for k, v in comm.moe_plan_view().items()}
+    win_host = windows.cpu().view(torch.int16).numpy().view(np.uint16).copy()
+    if wl.expert_op == "scale":
+        gpu_expert_scale(windows, idx, wl.E, wl.R, C, inp.scale.to(dev))
+    Y = torch.from_numpy(np.full((wl.T, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    comm.moe_combine(windows, C, w, Y)
+    statuses.append(comm.moe_status())
+    out = GpuRun(view, slots.cpu().numpy(), win_host, Y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), statuses)
+    if own:
+        comm.close()
+    return out
+
+
+def assert_parity(g: GpuRun, o: OracleRun, schedule: int, combine_ulp: int = 1):
+    assert g.statuses == [0, 0, 0], g.statuses
+    names = {"counts": "M", "c_rank": "c_rank", "small_off": "s", "large_off": "o", "n_exp": "n_exp", "n_recv": "n_recv"}
+    for k, on in names.items():
+        if g.view[k] is None:
+            assert schedule == synth.DECODE and k in ("counts", "c_rank", "n_exp")
+            continue
+        assert np.array_equal(g.view[k], getattr(o.plan, on)), k          # bit-exact integers
+    assert np.array_equal(g.slots.astype(np.int64), o.slots)
+    assert np.array_equal(g.windows, o.windows)                           # bit-exact rows and canaries
+    ulp = max_ulp_diff(g.Y, o.Y)
+    assert ulp <= combine_ulp, ulp
+    return ulp

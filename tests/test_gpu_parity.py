@@ -1,0 +1,268 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle,
+element by element, on the same seeded inputs.
+
+Bar: bit-exact counts, offsets, slots and dispatched window bytes (canaries
+included); combine within 1 bf16 ulp (both sides accumulate in fp32 with one
+fma per term, j ascending, so the observed distance is normally 0).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06055_b200 import binding, synth
+from paper_2605_06055_b200.synth import DECODE, PREFILL, Workload
+
+import harness
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_check(wl, schedule=None, slack=3):
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R, inp.rank_tok_start)
+    C = int(p.n_recv.max()) + slack if wl.T else slack
+    o = harness.oracle_run(inp, C)
+    sch = wl.schedule if schedule is None else schedule
+    g = harness.gpu_run(inp, C, sch)
+    return harness.assert_parity(g, o, sch)
+
+
+# ------------------------------------------------------------------ the benchmark configurations
+def test_config1_tiny_prefill():
+    assert run_and_check(synth.config(1)) == 0
+
+
+def test_config1_under_decode_schedule():
+    run_and_check(synth.config(1), DECODE)
+
+
+def test_config2_decode_dsv3_full_size():
+    run_and_check(synth.config(2))
+
+
+def test_config2_under_prefill_schedule():
+    run_and_check(synth.config(2), PREFILL)
+
+
+@pytest.mark.parametrize("T", [128, 1024, 8192])
+@pytest.mark.parametrize("schedule", [PREFILL, DECODE])
+def test_config5_mixtral_sweep(T, schedule):
+    run_and_check(synth.config(5, T, schedule))
+
+
+def test_config3_shape_reduced_tokens():
+    # DeepSeek-V3-like prefill shape at 1/8 of the tokens: several 2048-branch tiles per rank plus a ragged tail.
+    wl = Workload("c3_reduced", 8 * 517, 7168, 256, 8, 8, PREFILL, "uniform", "identity", 3003)
+    run_and_check(wl)
+
+
+def test_config4_zipf_reduced_tokens():
+    wl = Workload("c4_reduced", 4096, 7168, 256, 8, 8, PREFILL, "zipf", "identity", 3004)
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    assert p.n_exp.max() >= 10 * wl.B / wl.E
+    C = int(p.n_recv.max())                      # capacity sized exactly from the actual counts
+    g = harness.gpu_run(inp, C)
+    harness.assert_parity(g, harness.oracle_run(inp, C), PREFILL)
+
+
+# ------------------------------------------------------------------ shapes, tails, degenerate cases
+EDGE = [
+    # name, T, H, E, R, K, routing, rank_tokens
+    ("K1", 200, 64, 8, 4, 1, "uniform", None),
+    ("R1", 96, 128, 8, 1, 2, "uniform", None),
+    ("E_eq_R", 64, 64, 4, 4, 2, "uniform", None),
+    ("H8", 300, 8, 16, 4, 4, "uniform", None),
+    ("H_not_mult_of_warp_row", 77, 1000, 16, 2, 6, "uniform", None),
+    ("K3_generic", 129, 264, 12, 3, 3, "replace", (40, 0, 89)),
+    ("K5_generic_dups", 250, 520, 10, 5, 5, "replace", (1, 100, 49, 0, 100)),
+    ("K32_max", 40, 64, 64, 2, 32, "uniform", None),
+    ("duplicates_in_token", 333, 72, 4, 2, 4, "replace", (300, 33)),
+    ("empty_rank_ragged", 1000, 256, 32, 4, 8, "uniform", (0, 517, 0, 483)),
+    ("many_ranks", 512, 64, 256, 64, 8, "uniform", None),
+    ("big_E", 3000, 32, 2048, 2, 8, "uniform", None),
+    ("tile_boundary_exact", 2048, 32, 8, 2, 2, "uniform", None),   # 2048 branches per rank = exactly one tile
+    ("tile_boundary_plus1", 2050, 32, 8, 2, 2, "uniform", None),
+]
+
+
+@pytest.mark.parametrize("schedule", [PREFILL, DECODE])
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+def test_edge_shapes(case, schedule):
+    name, T, H, E, R, K, routing, rank_tokens = case
+    wl = Workload(name, T, H, E, R, K, schedule, routing, "scale", 4000 + T, rank_tokens=rank_tokens)
+    run_and_check(wl)
+
+
+def test_empty_batch():
+    dev = torch.device("cuda:0")
+    comm = binding.MoeComm(64, 64, 8, 2, 2, dev)
+    idx = torch.zeros((0, 2), dtype=torch.int32, device=dev)
+    for sch in (PREFILL, DECODE):
+        comm.moe_plan(sch, idx, 0)
+        win = torch.zeros((2 * 4, 64), dtype=torch.bfloat16, device=dev)
+        comm.moe_dispatch(torch.zeros((0, 64), dtype=torch.bfloat16, device=dev), win, 4)
+        comm.moe_combine(win, 4, torch.zeros((0, 2), device=dev), torch.zeros((0, 64), dtype=torch.bfloat16, device=dev))
+        assert comm.moe_status() == 0
+        v = comm.moe_plan_view()
+        assert int(v["n_recv"].abs().sum()) == 0 and int(v["large_off"].abs().sum()) == 0
+
+
+def test_all_branches_to_one_expert_and_one_empty_expert():
+    T, H, E, R, K = 700, 64, 8, 4, 2
+    g = torch.Generator().manual_seed(5)
+    idx = torch.full((T, K), 5, dtype=torch.int32)
+    idx[:, 1] = torch.randint(0, 4, (T,), generator=g).to(torch.int32)     # experts 6,7 (rank 3) and 4 stay empty
+    wl = Workload("one_hot_expert", T, H, E, R, K, PREFILL, "replace", "scale", 77)
+    inp = synth.make_inputs(wl)
+    inp.topk_idx = idx
+    p = oracle.plan(idx.numpy(), E, R, inp.rank_tok_start)
+    assert p.n_exp[5] == T and p.n_exp[6] == 0
+    C = int(p.n_recv.max())
+    for sch in (PREFILL, DECODE):
+        harness.assert_parity(harness.gpu_run(inp, C, sch), harness.oracle_run(inp, C), sch)
+
+
+# ------------------------------------------------------------------ properties of the path
+def test_identity_round_trip_returns_x_exactly():
+    wl = Workload("roundtrip", 1024, 2048, 64, 8, 8, PREFILL, "uniform", "identity", 99)
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max())
+    g = harness.gpu_run(inp, C)
+    assert np.array_equal(g.Y, synth.bf16_to_u16(inp.X))       # sum_j W_j = 1 and identity experts => Y == X
+
+
+def test_schedules_agree_and_runs_are_bitwise_repeatable():
+    wl = synth.config(5, 1024, PREFILL)
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max()) + 1
+    a = harness.gpu_run(inp, C, PREFILL)
+    b = harness.gpu_run(inp, C, DECODE)
+    c = harness.gpu_run(inp, C, PREFILL)
+    for x in (b, c):
+        assert np.array_equal(a.slots, x.slots) and np.array_equal(a.windows, x.windows) and np.array_equal(a.Y, x.Y)
+        assert np.array_equal(a.view["small_off"], x.view["small_off"])
+        assert np.array_equal(a.view["large_off"], x.view["large_off"])
+    assert b.view["counts"] is None and b.view["c_rank"] is None and b.view["n_exp"] is None
+
+
+def test_context_reuse_across_plans_and_repeated_dispatch():
+    dev = torch.device("cuda:0")
+    comm = binding.MoeComm(1024, 256, 16, 4, 2, dev)
+    for seed, T, sch in [(1, 1024, DECODE), (2, 512, PREFILL), (3, 768, DECODE), (4, 1024, PREFILL)]:
+        wl = Workload("reuse", T, 256, 16, 4, 2, sch, "uniform", "identity", seed)
+        inp = synth.make_inputs(wl)
+        p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+        C = int(p.n_recv.max()) + 2
+        o = harness.oracle_run(inp, C)
+        g = harness.gpu_run(inp, C, sch, comm=comm)
+        harness.assert_parity(g, o, sch)
+        # a second dispatch + combine on the same plan gives the same bytes
+        X = inp.X.to(dev)
+        win = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
+        Y = torch.empty((T, wl.H), dtype=torch.bfloat16, device=dev)
+        comm.moe_dispatch(X, win, C)
+        comm.moe_combine(win, C, inp.topk_w.to(dev), Y)
+        assert comm.moe_status() == 0
+        assert np.array_equal(Y.cpu().view(torch.int16).numpy().view(np.uint16), g.Y)
+    comm.close()
+
+
+def test_decode_combine_without_dispatch_resolves_the_same_rows():
+    dev = torch.device("cuda:0")
+    wl = Workload("combine_only", 640, 128, 32, 4, 4, DECODE, "uniform", "identity", 31)
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max())
+    o = harness.oracle_run(inp, C)
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    idx = inp.topk_idx.to(dev)
+    comm.moe_plan(DECODE, idx)
+    win = torch.from_numpy(o.windows.view(np.int16)).to(dev).view(torch.bfloat16)   # expert outputs from elsewhere
+    Y = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    comm.moe_combine(win, C, inp.topk_w.to(dev), Y)
+    assert comm.moe_status() == 0
+    assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), o.Y) <= 1
+
+
+# ------------------------------------------------------------------ errors (made on the host; nothing faults)
+def test_errors_leave_memory_untouched():
+    dev = torch.device("cuda:0")
+    T, H, E, R, K = 256, 64, 16, 4, 2
+    comm = binding.MoeComm(T, H, E, R, K, dev)
+    wl = Workload("err", T, H, E, R, K, PREFILL, "uniform", "identity", 8)
+    inp = synth.make_inputs(wl)
+    X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
+    p = oracle.plan(inp.topk_idx.numpy(), E, R)
+    C = int(p.n_recv.max())
+    win = torch.from_numpy(np.full((R * C, H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    Y = torch.from_numpy(np.full((T, H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    canary_only = lambda t: bool((t.view(torch.int16) == np.int16(harness.CANARY)).all())
+
+    # before any plan
+    assert comm.moe_dispatch(X, win, C, check=False) == binding.MOE_ERR_NOT_PLANNED
+    assert comm.moe_combine(win, C, w, Y, check=False) == binding.MOE_ERR_NOT_PLANNED
+    with pytest.raises(binding.MoeError):
+        comm.moe_plan_view()
+    # host-detected argument errors
+    assert comm.moe_plan(PREFILL, idx, T + 1, check=False) == binding.MOE_ERR_INVALID_ARG
+    assert comm.moe_plan(PREFILL, idx, T, np.array([0, 10, 5, 100, T]), check=False) == binding.MOE_ERR_INVALID_ARG
+    assert comm.moe_plan(PREFILL, idx, T - 1, check=False) == binding.MOE_ERR_INVALID_ARG    # T % R with no map
+    assert comm.moe_plan(7, idx, T, check=False) == binding.MOE_ERR_INVALID_ARG
+
+    for sch in (PREFILL, DECODE):
+        # capacity one row short: status CAPACITY, no row written, Y untouched
+        comm.moe_plan(sch, idx)
+        assert comm.moe_status() == 0
+        comm.moe_dispatch(X, win, C - 1)
+        assert comm.moe_status() == binding.MOE_ERR_CAPACITY
+        comm.moe_combine(win, C - 1, w, Y)
+        assert comm.moe_status() == binding.MOE_ERR_CAPACITY
+        assert canary_only(win) and canary_only(Y)
+        # misaligned payload pointer
+        assert comm.moe_dispatch(X.view(-1)[1:], win, C, check=False) == binding.MOE_ERR_INVALID_ARG
+
+        # index == E and index == -1: BAD_INDEX, later calls write nothing until the status is read
+        for bad in (E, -1):
+            idx_bad = idx.clone()
+            idx_bad[T // 2, 1] = bad
+            comm.moe_plan(sch, idx_bad)
+            comm.moe_dispatch(X, win, C)
+            comm.moe_combine(win, C, w, Y)
+            assert comm.moe_status() == binding.MOE_ERR_BAD_INDEX
+            assert comm.moe_status() == 0                      # cleared by the read
+            assert canary_only(win) and canary_only(Y)
+
+    # and the context still works afterwards
+    comm.moe_plan(PREFILL, idx)
+    comm.moe_dispatch(X, win, C)
+    comm.moe_combine(win, C, w, Y)
+    assert comm.moe_status() == 0
+    assert np.array_equal(Y.cpu().view(torch.int16).numpy().view(np.uint16), synth.bf16_to_u16(inp.X))
+    comm.close()
+
+
+def test_forward_host_entry_point():
+    dev = torch.device("cuda:0")
+    wl = synth.config(5, 1024, DECODE)
+    inp = synth.make_inputs(wl, pin=True)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max())
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    x_dev = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    idx_dev = torch.empty((wl.T, wl.K), dtype=torch.int32, device=dev)
+    w_dev = torch.empty((wl.T, wl.K), dtype=torch.float32, device=dev)
+    win = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
+    y_dev = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    y_host = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16).pin_memory()
+    for sch in (DECODE, PREFILL):
+        y_host.zero_()
+        comm.moe_forward_host(sch, wl.T, None, inp.X, inp.topk_idx.pin_memory(), inp.topk_w.pin_memory(),
+                              x_dev, idx_dev, w_dev, win, C, y_dev, y_host)
+        assert comm.moe_status() == 0
+        o = harness.oracle_run(inp, C)
+        assert harness.max_ulp_diff(synth.bf16_to_u16(y_host), o.Y) <= 1
+    comm.close()
