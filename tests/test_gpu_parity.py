@@ -74,7 +74,7 @@ EDGE = [
     ("R1", 96, 128, 8, 1, 2, "uniform", None),
     ("E_eq_R", 64, 64, 4, 4, 2, "uniform", None),
     ("H8", 300, 8, 16, 4, 4, "uniform", None),
-    ("H_not_mult_of_warp_row", 77, 1000, 16, 2, 6, "uniform", None),
+    ("H_not_mult_of_warp_row", 77, 1000, 16, 2, 6, "uniform", (30, 47)),
     ("K3_generic", 129, 264, 12, 3, 3, "replace", (40, 0, 89)),
     ("K5_generic_dups", 250, 520, 10, 5, 5, "replace", (1, 100, 49, 0, 100)),
     ("K32_max", 40, 64, 64, 2, 32, "uniform", None),
