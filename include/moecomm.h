@@ -142,6 +142,30 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
                               void* windows_dev, int64_t capacity_rows, void* y_dev,
                               void* y_host, void* stream);
 
+/* Window slots straight from the routing indexes, for callers that cannot give the library a
+ * workspace.  (No counterpart in the paper: this is a packaging convenience of this library.)
+ * Who needs it: code that runs inside an engine which claimed all device memory for its own pool
+ * at start-up and offers no allocation hook, and decode loops in which nothing may allocate once
+ * serving has begun because a device allocation can stall every stream.  The planning scratch is
+ * a fixed array inside the library image (about 1.2 MB, resident on every GPU that loads the
+ * library until the process exits); this call allocates and frees nothing.
+ *   topk_idx        DEVICE [T,K] int32          rank_tok_start  HOST [R+1] or NULL, as in moe_plan
+ *   slots           DEVICE [T,K] int32, out     slot(t,j) as moe_plan(DECODE) + moe_slots gives it
+ *   n_recv          DEVICE [R] int32, out       rows received per window
+ *   status          DEVICE [1] int32, out       0, MOE_ERR_BAD_INDEX (that branch's slot is -1) or
+ *                                               MOE_ERR_CAPACITY (no slot written)
+ * Limits: T*K <= 65536, E <= 512, R <= 64, K <= MOE_MAX_K, R*capacity_rows < 2^31; larger problems
+ * are rejected with MOE_ERR_INVALID_ARG and a message on stderr -- use moe_plan with a workspace.
+ * The first call on each device looks up the array's device address; make that call with the
+ * device current and before any stream capture begins.  All calls on one device share the array
+ * (it keeps the previous call's contents; the words that must start at zero are cleared on the
+ * stream each time), so two calls whose kernels may overlap on the GPU -- different streams with
+ * no ordering between them -- race; order them on one stream or with events. */
+moe_status_t moe_slots_noalloc(const int32_t* topk_idx /*DEVICE*/, int32_t T, int32_t K, int32_t E, int32_t R,
+                               const int32_t* rank_tok_start /*HOST*/, int64_t capacity_rows,
+                               int32_t* slots /*DEVICE*/, int32_t* n_recv /*DEVICE*/, int32_t* status /*DEVICE*/,
+                               void* stream);
+
 /* Synchronises `stream`, then returns and clears the device status word
  * (first device-detected error since the last call, or MOE_OK). */
 moe_status_t moe_status(moe_ctx_t* ctx, void* stream);

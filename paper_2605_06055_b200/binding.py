@@ -24,6 +24,7 @@ MOE_SCHED_PREFILL, MOE_SCHED_DECODE = 0, 1
 EXPORTS = [
     "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
+    "moe_slots_noalloc",
 ]
 
 
@@ -66,6 +67,8 @@ def load() -> ctypes.CDLL:
     L.moe_slots.argtypes = [vp, i64, vp, vp]
     L.moe_forward_host.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     L.moe_status.argtypes = [vp, vp]
+    L.moe_slots_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp, vp, vp, vp]
+    L.moe_slots_noalloc.restype = ctypes.c_int
     L.moe_status_string.argtypes = [ctypes.c_int]
     L.moe_status_string.restype = ctypes.c_char_p
     L.moe_launch_count.argtypes = [vp]
@@ -228,3 +231,19 @@ class MoeComm:
 
     def moe_launch_count(self) -> int:
         return int(self.lib.moe_launch_count(self._h))
+
+
+def moe_slots_noalloc(topk_idx: torch.Tensor, E: int, R: int, capacity_rows: int, slots: torch.Tensor,
+                      n_recv: torch.Tensor, status: torch.Tensor, rank_tok_start=None, stream=None) -> int:
+    """Slots from routing indexes using the library's built-in scratch (see include/moecomm.h).
+
+    For callers that cannot hand the library a workspace.  Every tensor here is the caller's; this
+    wrapper allocates nothing and neither does the call.  Returns the host-side status code.
+    """
+    T, K = topk_idx.shape
+    rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
+    with torch.cuda.device(topk_idx.device):
+        return int(load().moe_slots_noalloc(_dev_ptr(topk_idx, torch.int32), T, K, E, R, _host_ptr(rts),
+                                            int(capacity_rows), _dev_ptr(slots, torch.int32),
+                                            _dev_ptr(n_recv, torch.int32), _dev_ptr(status, torch.int32),
+                                            _stream_handle(stream)))

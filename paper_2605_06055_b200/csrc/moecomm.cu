@@ -389,3 +389,125 @@ const char* moe_status_string(moe_status_t status) {
 int64_t moe_launch_count(const moe_ctx_t* ctx) { return ctx == nullptr ? 0 : ctx->launches; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// moe_slots_noalloc: routing indexes -> window slots with no caller workspace.
+//
+// Some callers of this library have no device memory to hand over for control state and may not
+// obtain any: a plug-in running inside an engine that reserved the whole HBM for its own pool at
+// start-up, or a latency-critical decode loop where a device allocation (which can stall the
+// device) is forbidden after initialisation.  For them the planning scratch lives in the
+// file-scope device array below, which every GPU that loads this library holds until the process
+// exits.  The entry point runs the same planning kernels as moe_plan(DECODE) + moe_slots, pointed
+// at that array.
+namespace {
+
+constexpr int32_t NOALLOC_MAX_BRANCHES = 65536;  // T * K
+constexpr int32_t NOALLOC_MAX_E = 512;
+constexpr int32_t NOALLOC_MAX_R = 64;
+constexpr int32_t NOALLOC_MAX_TILES = NOALLOC_MAX_BRANCHES / (ROUNDS_DECODE * PLAN_THREADS) + NOALLOC_MAX_R;
+
+struct NoallocScratch {
+  Control ctl;
+  int32_t M[NOALLOC_MAX_R * NOALLOC_MAX_E];
+  int32_t c_rank[NOALLOC_MAX_R * NOALLOC_MAX_R];
+  int32_t o[NOALLOC_MAX_E * NOALLOC_MAX_R];
+  int32_t n_exp[NOALLOC_MAX_E];
+  int32_t tile_rank[NOALLOC_MAX_BRANCHES];
+  int32_t tile_hist[(size_t)NOALLOC_MAX_TILES * NOALLOC_MAX_E];
+};
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoallocScratch)];  // about 1.2 MB
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+NoallocScratch* g_noalloc_ptr[NOALLOC_MAX_DEVICES];  // device address of the array, per device; 0 = not set up
+
+// In host code g_noalloc_scratch is only a handle for the runtime, not a device address, so the
+// address each device uses is looked up once, with that device current.
+NoallocScratch* noalloc_scratch_for_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return nullptr;
+  if (g_noalloc_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    g_noalloc_ptr[dev] = static_cast<NoallocScratch*>(p);
+  }
+  return g_noalloc_ptr[dev];
+}
+
+}  // namespace
+
+extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
+                                          const int32_t* rank_tok_start, int64_t capacity_rows, int32_t* slots,
+                                          int32_t* n_recv, int32_t* status, void* stream) {
+  if (T < 0 || K < 1 || K > MOE_MAX_K || E < 1 || R < 1 || E % R != 0 || capacity_rows < 0) return MOE_ERR_INVALID_ARG;
+  if (E > NOALLOC_MAX_E || R > NOALLOC_MAX_R || (int64_t)T * K > NOALLOC_MAX_BRANCHES) {
+    std::fprintf(stderr,
+                 "moe_slots_noalloc: T*K=%lld, E=%d, R=%d exceed the built-in scratch (T*K <= %d, E <= %d, R <= %d); "
+                 "use moe_plan + moe_slots with a caller workspace instead\n",
+                 (long long)T * K, E, R, NOALLOC_MAX_BRANCHES, NOALLOC_MAX_E, NOALLOC_MAX_R);
+    return MOE_ERR_INVALID_ARG;
+  }
+  if ((int64_t)R * capacity_rows >= (int64_t)1 << 31) return MOE_ERR_INVALID_ARG;
+  if (n_recv == nullptr || status == nullptr || (T > 0 && (topk_idx == nullptr || slots == nullptr)))
+    return MOE_ERR_INVALID_ARG;
+  if (rank_tok_start == nullptr && T % R != 0) return MOE_ERR_INVALID_ARG;
+  if (rank_tok_start != nullptr) {
+    if (rank_tok_start[0] != 0 || rank_tok_start[R] != T) return MOE_ERR_INVALID_ARG;
+    for (int r = 0; r < R; ++r)
+      if (rank_tok_start[r + 1] < rank_tok_start[r]) return MOE_ERR_INVALID_ARG;
+  }
+  NoallocScratch* sc = noalloc_scratch_for_current_device();
+  if (sc == nullptr) return MOE_ERR_CUDA;
+
+  const int tile_branches = ROUNDS_DECODE * PLAN_THREADS;
+  RankMap map;
+  std::memset(&map, 0, sizeof(map));
+  map.R = R;
+  map.uniform_tokens = (rank_tok_start == nullptr && T > 0) ? T / R : 0;
+  while ((1 << map.tile_shift) < tile_branches) ++map.tile_shift;
+  int32_t tiles = 0;
+  for (int r = 0; r <= R; ++r) {
+    const int32_t tok = rank_tok_start != nullptr ? rank_tok_start[r] : (int32_t)((int64_t)T / R * r);
+    map.tok_start[r] = tok;
+    map.tile_start[r] = tiles;
+    if (r < R) {
+      const int32_t next = rank_tok_start != nullptr ? rank_tok_start[r + 1] : (int32_t)((int64_t)T / R * (r + 1));
+      tiles += (int32_t)(((int64_t)(next - tok) * K + tile_branches - 1) / tile_branches);
+    }
+  }
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left; only the control words and the caller's
+  // status word must start at zero, everything else is fully rewritten before it is read.
+  if (cudaMemsetAsync(&sc->ctl, 0, sizeof(Control), st) != cudaSuccess ||
+      cudaMemsetAsync(status, 0, sizeof(int32_t), st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (tiles > 0)
+    plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, PLAN_WARPS * E * (int)sizeof(int32_t), st>>>(
+        topk_idx, map, K, E, sc->tile_rank, sc->tile_hist, status);
+  plan_scan_kernel<<<R, PLAN_THREADS, (2 * E + 1) * (int)sizeof(int32_t), st>>>(
+      sc->tile_hist, map, E, 0, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl);
+  RowArgs a;
+  a.topk_idx = topk_idx;
+  a.small_off = sc->tile_rank;
+  a.small_out = nullptr;
+  a.tile_base = sc->tile_hist;
+  a.large_off = sc->o;
+  a.n_recv = n_recv;
+  a.status = status;
+  a.C = capacity_rows;
+  a.T = T;
+  a.K = K;
+  a.E = E;
+  a.R = R;
+  a.E_r = E / R;
+  a.H16 = 0;
+  int grid = (int)(((int64_t)T * K + 255) / 256);
+  if (grid < 1) grid = 1;
+  slots_kernel<<<grid, 256, 0, st>>>(slots, a, map);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
