@@ -47,6 +47,9 @@ WORKLOADS = {
     "c3": lambda: synth.config(3),
     "c4": lambda: synth.config(4),
     "c5": lambda: synth.config(5, 65536, synth.PREFILL),
+    # c3 at a quarter of the tokens: the same kernels and row size, sized for ncu captures (about 1.2 GB resident)
+    "c3s": lambda: synth.Workload("c3_prefill_dsv3_T8192", 8192, 7168, 256, 8, 8, synth.PREFILL, "uniform",
+                                  "identity", 1003),
 }
 
 
@@ -285,6 +288,20 @@ def run_cuda(args, wl):
         ms_per_step = float(t.item())
 
     # ---- end to end through the C ABI from HOST buffers (copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        e2e = measure_e2e(args, wl, comm, inp, idx_h, w_h, X, idx, w, windows, C, Y, barrier, dist, dev, world,
+                          step_bytes)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    return finish(args, wl, world, dist, ms_per_step, step_bytes, b_plan, b_disp, b_comb, plan_us, disp_us, comb_us,
+                  clocks, launches, e2e, C, big, inp)
+
+
+def measure_e2e(args, wl, comm, inp, idx_h, w_h, X, idx, w, windows, C, Y, barrier, dist, dev, world, step_bytes):
     y_host = torch.empty((wl.T, wl.H), dtype=torch.bfloat16).pin_memory()
     x_dev2, idx_dev2, w_dev2 = torch.empty_like(X), torch.empty_like(idx), torch.empty_like(w)
     e2e_steps = max(3, min(args.steps, 10))
@@ -307,12 +324,12 @@ def run_cuda(args, wl):
         e2e_ms = float(t.item())
     h2d = wl.T * wl.H * 2 + wl.T * wl.K * 8
     d2h = wl.T * wl.H * 2
+    return {"value": world * step_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
 
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
 
+def finish(args, wl, world, dist, ms_per_step, step_bytes, b_plan, b_disp, b_comb, plan_us, disp_us, comb_us, clocks,
+           launches, e2e, C, big, inp):
     peak, peak_kind = measured_peak()
     med = statistics.median
     kernels = {
@@ -341,12 +358,10 @@ def run_cuda(args, wl):
         "dispatch_plus_combine_us": med(disp_us) + med(comb_us),
         "frac_of_8TBps": (b_disp + b_comb) / ((med(disp_us) + med(comb_us)) * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
         "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": launches,
-        "e2e": {"value": world * step_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "e2e": e2e,
     }
 
     if world == 1 and not args.no_cpu_baseline:
-        del windows, Y, x_dev2
         sample = wl if wl.T * wl.K * wl.H <= 2 * (1 << 30) else oracle_sample(wl, 2)
         times, cores = time_oracle(sample, 1, 1, inp if sample is wl else None)
         sb = bytes_plan(sample) + bytes_dispatch(sample) + bytes_combine(sample)
@@ -368,6 +383,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]()
     if args.impl == "reference":

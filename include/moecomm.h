@@ -142,6 +142,16 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
                               void* windows_dev, int64_t capacity_rows, void* y_dev,
                               void* y_host, void* stream);
 
+/* Tuning knobs of a context (tests use them to reach every kernel; defaults are the measured best).
+ *   MOE_OPT_DISPATCH_PATH  which dispatch kernel runs: AUTO (currently the bulk-copy kernel),
+ *                          REGISTERS (16-byte ld/st through registers, K-specialised), or
+ *                          BULK (cp.async.bulk through shared-memory stages).  Same result.
+ *   MOE_OPT_GRANULE        512-byte units per work item of dispatch/combine; 0 = chosen from the
+ *                          job size.  Any value gives the same result. */
+typedef enum { MOE_OPT_DISPATCH_PATH = 0, MOE_OPT_GRANULE = 1 } moe_option_t;
+enum { MOE_DISPATCH_AUTO = 0, MOE_DISPATCH_REGISTERS = 1, MOE_DISPATCH_BULK = 2 };
+moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);
+
 /* Window slots straight from the routing indexes, for callers that cannot give the library a
  * workspace.  (No counterpart in the paper: this is a packaging convenience of this library.)
  * Who needs it: code that runs inside an engine which claimed all device memory for its own pool

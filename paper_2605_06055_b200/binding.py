@@ -24,8 +24,10 @@ MOE_SCHED_PREFILL, MOE_SCHED_DECODE = 0, 1
 EXPORTS = [
     "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
-    "moe_slots_noalloc",
+    "moe_slots_noalloc", "moe_set_option",
 ]
+MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE = 0, 1
+MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
 
 
 class MoeShape(ctypes.Structure):
@@ -69,6 +71,8 @@ def load() -> ctypes.CDLL:
     L.moe_status.argtypes = [vp, vp]
     L.moe_slots_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp, vp, vp, vp]
     L.moe_slots_noalloc.restype = ctypes.c_int
+    L.moe_set_option.argtypes = [vp, ctypes.c_int, i64]
+    L.moe_set_option.restype = ctypes.c_int
     L.moe_status_string.argtypes = [ctypes.c_int]
     L.moe_status_string.restype = ctypes.c_char_p
     L.moe_launch_count.argtypes = [vp]
@@ -223,6 +227,12 @@ class MoeComm:
             self.T, self.schedule, self._keep = T, schedule, topk_idx_dev
         elif check:
             raise MoeError(rc, "moe_forward_host")
+        return rc
+
+    def moe_set_option(self, option: int, value: int, check: bool = True) -> int:
+        rc = int(self.lib.moe_set_option(self._h, option, int(value)))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_set_option")
         return rc
 
     def moe_status(self, stream=None) -> int:

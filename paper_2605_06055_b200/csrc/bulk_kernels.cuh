@@ -1,0 +1,145 @@
+// Dispatch through the bulk-copy engine (TMA, 1-D cp.async.bulk, no tensor map,
+// no multicast).
+//
+// Same work items and same result as dispatch_rows_kernel, but the bytes never
+// pass through registers: every warp drives a small ring of shared-memory
+// stages.  Lane 0 asks the copy engine to load one work item (up to a whole
+// 14 KB row) into a stage, and when the stage's mbarrier completes, to store it
+// to the K destination rows.  One request covers the whole contiguous span, so
+// HBM sees long sequential bursts per row, and the number of bytes in flight is
+// set by shared memory (about 170 KB per SM), not by registers or warp count.
+//
+// Every wait is bounded: an mbarrier that does not complete within WAIT_LIMIT
+// polls raises MOE_ERR_TIMEOUT and the warp stops taking work.
+#pragma once
+
+#include "row_kernels.cuh"
+
+namespace moe {
+
+constexpr int BULK_WARPS = 4;
+constexpr int BULK_STAGES = 3;
+constexpr int BULK_MAX_GRANULE = 32;   // a stage holds at most 16 KB of one row
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+// Bounded wait; false if the barrier did not complete.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Dynamic shared memory: [BULK_WARPS][BULK_STAGES][stage_bytes] payload, then
+// [BULK_WARPS][BULK_STAGES] mbarriers.  stage_bytes = granule * 512.
+__global__ void __launch_bounds__(BULK_WARPS * 32)
+dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows, const RowArgs a,
+                     const __grid_constant__ RankMap map) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  begin_work(a);
+  if (must_abort(a)) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t stage_bytes = (uint32_t)a.granule * 512u;
+  const uint32_t row_bytes = (uint32_t)a.H16 * 16u;
+  const uint32_t buf0 = smem_addr(smem) + warp * BULK_STAGES * stage_bytes;
+  const uint32_t bar0 = smem_addr(smem) + BULK_WARPS * BULK_STAGES * stage_bytes + warp * BULK_STAGES * 8;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < BULK_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  // Asks the copy engine for work item `item` into stage `s` (lane 0 only).
+  auto issue_load = [&](int32_t item, int s) {
+    const WorkItem w = decode_item(a, item);
+    const uint32_t off = (uint32_t)w.i0 * 512u;
+    const uint32_t bytes = min((uint32_t)w.i1 * 512u, row_bytes) - off;
+    mbar_expect_tx(bar0 + 8 * s, bytes);
+    bulk_load(buf0 + s * stage_bytes, X + (size_t)w.t * row_bytes + off, bytes, bar0 + 8 * s);
+  };
+
+  // Items in flight: q0 is consumed this iteration, q1 is loading, q2 is fetched now.
+  int32_t q0 = fetch_item(a);
+  int32_t q1 = fetch_item(a);
+  if (lane == 0) {
+    if (q0 < a.n_items) issue_load(q0, 0);
+    if (q1 < a.n_items) issue_load(q1, 1);
+  }
+  uint32_t it = 0;
+  bool alive = true;
+  while (q0 < a.n_items && alive) {
+    const int32_t q2 = fetch_item(a);
+    const int s = it % BULK_STAGES;
+    const uint32_t parity = (it / BULK_STAGES) & 1u;
+    const WorkItem w = decode_item(a, q0);
+    const int64_t slot = resolve_slot(a, map, w.t, lane, w.i0 == 0);   // overlaps the load in flight
+    const uint32_t off = (uint32_t)w.i0 * 512u;
+    const uint32_t bytes = min((uint32_t)w.i1 * 512u, row_bytes) - off;
+
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) {
+      if (lane == 0) raise_status(a.status, MOE_ERR_TIMEOUT);
+      alive = false;
+      break;
+    }
+    for (int j = 0; j < a.K; ++j) {
+      const int64_t row = __shfl_sync(0xffffffffu, slot, j);
+      if (lane == 0 && row >= 0) bulk_store(windows + (size_t)row * row_bytes + off, buf0 + s * stage_bytes, bytes);
+    }
+    if (lane == 0) {
+      bulk_commit();
+      // The stage that held the previous item is refilled next: its stores must have read it.
+      bulk_wait_read<1>();
+      if (q2 < a.n_items) issue_load(q2, (it + 2) % BULK_STAGES);
+    }
+    q0 = q1;
+    q1 = q2;
+    ++it;
+  }
+  if (lane == 0) bulk_wait_all();
+}
+
+}  // namespace moe

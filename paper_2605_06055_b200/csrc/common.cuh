@@ -33,7 +33,8 @@ struct RankMap {
 struct Control {
   int32_t status;       // first device-detected error (moe_status_t), 0 = none
   int32_t scan_ticket;  // "last block done" counter of the offset scan
-  int32_t pad[62];
+  int32_t work[2];      // work-item counters of the row kernels, used alternately (see row_kernels.cuh)
+  int32_t pad[60];
 };
 
 __device__ __forceinline__ void raise_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }

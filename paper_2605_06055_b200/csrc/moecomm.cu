@@ -3,12 +3,14 @@
 // the path runs in the kernels of plan_kernels.cuh and row_kernels.cuh.
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
 #include "common.cuh"
 #include "plan_kernels.cuh"
 #include "row_kernels.cuh"
+#include "bulk_kernels.cuh"
 
 using namespace moe;
 
@@ -29,6 +31,9 @@ struct moe_ctx {
   const int32_t* topk_idx;  // device; routing indexes of the current plan, read again by dispatch/combine
   RankMap map;
   int64_t launches;
+  int32_t work_parity;      // which of the two work-item counters the next row-kernel launch uses
+  int32_t dispatch_path;    // MOE_OPT_DISPATCH_PATH
+  int32_t granule_override; // MOE_OPT_GRANULE
 };
 
 namespace {
@@ -104,25 +109,83 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.R = sh.R;
   a.E_r = sh.E / sh.R;
   a.H16 = sh.H / 8;
+  a.work = nullptr;
+  a.work_next = nullptr;
+  a.granule = 1;
+  a.items_per_row = 0;
+  a.n_items = 0;
   return a;
 }
 
-int row_grid(const moe_ctx* ctx, int warps_per_cta, int ctas_per_sm) {
-  const int64_t need = ((int64_t)ctx->T + warps_per_cta - 1) / warps_per_cta;
-  const int64_t cap = (int64_t)ctx->num_sms * ctas_per_sm;
+// Chooses the work-item size and hands the launch its counter.  Large jobs take whole rows (at
+// most max_granule units) per item; small, decode-sized jobs take a fraction of a row so that every
+// warp of the grid has work.
+void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
+  const int upr = (a.H16 + 31) / 32;
+  const int64_t total = (int64_t)ctx->T * upr;
+  int64_t g = upr < max_granule ? upr : max_granule;
+  if (total < nwarps * g * 4) g = total / (nwarps * 2);
+  if (ctx->granule_override > 0) g = ctx->granule_override;
+  if (g > max_granule) g = max_granule;
+  if (g > upr) g = upr;
+  if (g < 1) g = 1;
+  while (((int64_t)ctx->T * ((upr + g - 1) / g)) > ((int64_t)1 << 30) && g < upr) ++g;   // n_items stays in int32
+  a.granule = (int32_t)g;
+  a.items_per_row = (int32_t)((upr + g - 1) / g);
+  a.n_items = (int32_t)((int64_t)ctx->T * a.items_per_row);
+  a.work = &ctx->ctl->work[ctx->work_parity];
+  a.work_next = &ctx->ctl->work[ctx->work_parity ^ 1];
+  ctx->work_parity ^= 1;
+}
+
+// One persistent wave: as many CTAs as fit on the device at once (from the occupancy calculator),
+// but no more warps than there are 512-byte units of work.
+template <class Kernel>
+int row_grid(const moe_ctx* ctx, Kernel kernel) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    per_sm = 2;
+  }
+  const int64_t units = (int64_t)ctx->T * ((ctx->shape.H / 8 + 31) / 32);
+  const int64_t need = (units + 7) / 8;
+  const int64_t cap = (int64_t)ctx->num_sms * per_sm;
   return (int)(need < cap ? (need < 1 ? 1 : need) : cap);
 }
 
+// Loads in flight per lane before the dependent stores / fma chain.  Few fat warps (one 256-thread
+// CTA per SM with about 32 16-byte loads per lane) measured faster than many thin ones: every warp
+// then streams long contiguous runs of each row, which HBM serves with far fewer page switches.
+constexpr int combine_unroll(int K) { return K >= 8 ? 4 : K >= 6 ? 5 : K >= 4 ? 8 : 16; }
+constexpr int DISPATCH_UNROLL = 14;
+
 template <int KT>
-void launch_dispatch(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
-  const int grid = row_grid(ctx, 8, 8);
-  dispatch_rows_kernel<KT, 4><<<grid, 256, 0, st>>>(x, win, a, ctx->map);
+void launch_dispatch_regs(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
+  auto kernel = dispatch_rows_kernel<KT, (KT > 0 ? DISPATCH_UNROLL : 1)>;
+  const int grid = row_grid(ctx, kernel);
+  RowArgs b = a;
+  set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
+  kernel<<<grid, 256, 0, st>>>(x, win, b, ctx->map);
+}
+
+// Bulk-copy path: one CTA of BULK_WARPS warps per SM, a ring of BULK_STAGES stages per warp.
+void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
+  const int upr = (a.H16 + 31) / 32;
+  const int grid = ctx->num_sms;
+  RowArgs b = a;
+  set_work(ctx, b, (int64_t)grid * BULK_WARPS, upr < BULK_MAX_GRANULE ? upr : BULK_MAX_GRANULE);
+  const int smem = BULK_WARPS * BULK_STAGES * (b.granule * 512 + 8);
+  dispatch_bulk_kernel<<<grid, BULK_WARPS * 32, smem, st>>>(reinterpret_cast<const unsigned char*>(x),
+                                                          reinterpret_cast<unsigned char*>(win), b, ctx->map);
 }
 
 template <int KT>
 void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const float* w, uint4* y, cudaStream_t st) {
-  const int grid = row_grid(ctx, 8, 8);
-  combine_rows_kernel<KT, (KT > 4 ? 1 : 2)><<<grid, 256, 0, st>>>(win, w, y, a, ctx->map);
+  auto kernel = combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 1)>;
+  const int grid = row_grid(ctx, kernel);
+  RowArgs b = a;
+  set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
+  kernel<<<grid, 256, 0, st>>>(win, w, y, b, ctx->map);
 }
 
 }  // namespace
@@ -164,10 +227,16 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->planned = false;
   ctx->launches = 0;
   ctx->topk_idx = nullptr;
+  ctx->work_parity = 0;
+  ctx->dispatch_path = MOE_DISPATCH_AUTO;
+  ctx->granule_override = 0;
 
   // Shared memory of the planning kernels grows with E; opt in above 48 KB.
   const int tile_smem = PLAN_WARPS * shape->E * (int)sizeof(int32_t);
   bool ok = cudaMemset(ctx->ctl, 0, sizeof(Control)) == cudaSuccess;
+  if (ok)
+    ok = cudaFuncSetAttribute(dispatch_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              BULK_WARPS * BULK_STAGES * (BULK_MAX_GRANULE * 512 + 8)) == cudaSuccess;
   if (ok && tile_smem > 48 * 1024) {
     ok = cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_PREFILL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               tile_smem) == cudaSuccess &&
@@ -279,13 +348,17 @@ moe_status_t moe_dispatch(moe_ctx_t* c, const void* x, void* windows, int64_t ca
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* xs = static_cast<const uint4*>(x);
   uint4* win = static_cast<uint4*>(windows);
-  switch (ctx->shape.K) {
-    case 1: launch_dispatch<1>(ctx, a, xs, win, st); break;
-    case 2: launch_dispatch<2>(ctx, a, xs, win, st); break;
-    case 4: launch_dispatch<4>(ctx, a, xs, win, st); break;
-    case 6: launch_dispatch<6>(ctx, a, xs, win, st); break;
-    case 8: launch_dispatch<8>(ctx, a, xs, win, st); break;
-    default: launch_dispatch<0>(ctx, a, xs, win, st); break;
+  if (ctx->dispatch_path != MOE_DISPATCH_REGISTERS) {
+    launch_dispatch_bulk(ctx, a, xs, win, st);
+  } else {
+    switch (ctx->shape.K) {
+      case 1: launch_dispatch_regs<1>(ctx, a, xs, win, st); break;
+      case 2: launch_dispatch_regs<2>(ctx, a, xs, win, st); break;
+      case 4: launch_dispatch_regs<4>(ctx, a, xs, win, st); break;
+      case 6: launch_dispatch_regs<6>(ctx, a, xs, win, st); break;
+      case 8: launch_dispatch_regs<8>(ctx, a, xs, win, st); break;
+      default: launch_dispatch_regs<0>(ctx, a, xs, win, st); break;
+    }
   }
   return launch_ok(ctx);
 }
@@ -356,6 +429,22 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
   if (T > 0 && cudaMemcpyAsync(y_host, y_dev, (size_t)T * row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   return MOE_OK;
+}
+
+moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  switch (option) {
+    case MOE_OPT_DISPATCH_PATH:
+      if (value != MOE_DISPATCH_AUTO && value != MOE_DISPATCH_REGISTERS && value != MOE_DISPATCH_BULK)
+        return MOE_ERR_INVALID_ARG;
+      ctx->dispatch_path = (int32_t)value;
+      return MOE_OK;
+    case MOE_OPT_GRANULE:
+      if (value < 0 || value > (1 << 20)) return MOE_ERR_INVALID_ARG;
+      ctx->granule_override = (int32_t)value;
+      return MOE_OK;
+  }
+  return MOE_ERR_INVALID_ARG;
 }
 
 moe_status_t moe_status(moe_ctx_t* ctx, void* stream) {
@@ -506,6 +595,11 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.R = R;
   a.E_r = E / R;
   a.H16 = 0;
+  a.work = nullptr;
+  a.work_next = nullptr;
+  a.granule = 1;
+  a.items_per_row = 0;
+  a.n_items = 0;
   int grid = (int)(((int64_t)T * K + 255) / 256);
   if (grid < 1) grid = 1;
   slots_kernel<<<grid, 256, 0, st>>>(slots, a, map);

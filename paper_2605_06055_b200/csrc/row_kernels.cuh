@@ -1,10 +1,10 @@
 // Payload kernels: dispatch (scatter rows into expert windows) and combine
 // (gather rows from expert windows + fp32 weighted sum), both token-major.
 //
-// Algorithm 1 / Algorithm 2 of the paper.  One warp owns one token at a time:
-// lane j < K resolves branch (t, j) to its window row with the two-level offset
-// rule slot = dst(e)*C + o[e, src(t)] + s[t,j]; then the whole warp moves the
-// row in 16-byte chunks.  Dispatch reads X[t,:] from HBM exactly once and
+// Algorithm 1 / Algorithm 2 of the paper.  A warp works on (part of) one token
+// row at a time: lane j < K resolves branch (t, j) to its window row with the
+// two-level offset rule slot = dst(e)*C + o[e, src(t)] + s[t,j]; then the whole
+// warp moves its share of the row in 16-byte chunks.  Dispatch reads X[t,:] from HBM exactly once and
 // stores it K times; combine issues the K loads of a chunk before its
 // j-ordered fma chain.  There is no relay, permute or unpermute buffer.
 #pragma once
@@ -24,6 +24,11 @@ struct RowArgs {
   int64_t C;                 // rows per window segment
   int32_t T, K, E, R, E_r;
   int32_t H16;               // 16-byte chunks per row
+  int32_t* work;             // this launch's work-item counter (zero on entry)
+  int32_t* work_next;        // the next launch's counter, zeroed by this launch
+  int32_t granule;           // units (512-byte slabs) per work item
+  int32_t items_per_row;     // ceil(units per row / granule)
+  int32_t n_items;           // T * items_per_row
 };
 
 // Window row of branch (t, lane) for lane < K, -1 otherwise.  Small offsets of
@@ -66,24 +71,61 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                : "memory");
 }
 
+// Work partition shared by dispatch and combine.  A "unit" is one 512-byte
+// column slab of one token row (32 lanes x 16 bytes).  A row is cut into
+// items_per_row work items of `granule` units (the last may be shorter); the job
+// is T * items_per_row items.  Warps take items from an atomic counter, fetching
+// the next one while the current one is processed, so a warp that the memory
+// system serves slowly simply takes fewer items: no wave quantisation at prefill
+// sizes, full-GPU parallelism at decode sizes, no static tail.  Which warp moves
+// which bytes does not affect the result.  The counter is one of two used
+// alternately: each launch zeroes the one the next launch will use.
+struct WorkItem {
+  int32_t t;       // token
+  int32_t i0, i1;  // unit range inside the row
+};
+
+__device__ __forceinline__ void begin_work(const RowArgs& a) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) *a.work_next = 0;
+}
+
+__device__ __forceinline__ int32_t fetch_item(const RowArgs& a) {
+  int32_t v = 0;
+  if ((threadIdx.x & 31) == 0) v = atomicAdd(a.work, 1);
+  return __shfl_sync(0xffffffffu, v, 0);
+}
+
+__device__ __forceinline__ WorkItem decode_item(const RowArgs& a, int32_t item) {
+  WorkItem w;
+  w.t = item / a.items_per_row;
+  w.i0 = (item - w.t * a.items_per_row) * a.granule;
+  w.i1 = min(w.i0 + a.granule, (a.H16 + 31) >> 5);
+  return w;
+}
+
 // ---------------------------------------------------------------- dispatch
 // KT > 0: K known at compile time (row pointers live in registers).
 // KT == 0: any K <= 32 (row index fetched by shuffle per store).
-template <int KT, int UNROLL>
-__global__ void __launch_bounds__(256)
+// UNROLL 16-byte loads are in flight per lane before the K x UNROLL stores; few
+// warps with deep unrolling beat many thin warps here, because each warp then
+// writes long contiguous runs of every destination row.
+template <int KT, int UNROLL, int MINB = 1>
+__global__ void __launch_bounds__(256, MINB)
 dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, const RowArgs a,
                      const __grid_constant__ RankMap map) {
+  begin_work(a);
   if (must_abort(a)) return;
   const int lane = threadIdx.x & 31;
-  const int warps_per_cta = blockDim.x >> 5;
-  const int32_t warp0 = blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
-  const int32_t nwarps = gridDim.x * warps_per_cta;
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
 
-  for (int32_t t = warp0; t < a.T; t += nwarps) {
-    const int64_t slot = resolve_slot(a, map, t, lane, true);
-    const uint4* src = X + (size_t)t * H16;
+  int32_t item = fetch_item(a);
+  while (item < a.n_items) {
+    const int32_t next_item = fetch_item(a);   // in flight while this item is processed
+    const WorkItem w = decode_item(a, item);
+    item = next_item;
+    const int64_t slot = resolve_slot(a, map, w.t, lane, w.i0 == 0);   // the owner of the row start records delta
+    const uint4* src = X + (size_t)w.t * H16;
     if constexpr (KT > 0) {
       uint4* dst[KT];
 #pragma unroll
@@ -91,27 +133,26 @@ dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, c
         const int64_t row = __shfl_sync(0xffffffffu, slot, j);
         dst[j] = row >= 0 ? windows + (size_t)row * H16 : nullptr;
       }
-      int c = lane;
-      for (; c + 32 * (UNROLL - 1) < H16; c += 32 * UNROLL) {
+      for (int i = w.i0; i < w.i1; i += UNROLL) {
         uint4 v[UNROLL];
+        bool ok[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(src + c + 32 * u);
+        for (int u = 0; u < UNROLL; ++u) {
+          const int c = (i + u) * 32 + lane;
+          ok[u] = (i + u < w.i1) && (c < H16);
+          if (ok[u]) v[u] = ld_stream(src + c);
+        }
 #pragma unroll
         for (int j = 0; j < KT; ++j)
           if (dst[j] != nullptr) {
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) st_stream(dst[j] + c + 32 * u, v[u]);
+            for (int u = 0; u < UNROLL; ++u)
+              if (ok[u]) st_stream(dst[j] + (i + u) * 32 + lane, v[u]);
           }
       }
-      for (; c < H16; c += 32) {
-        const uint4 v = ld_stream(src + c);
-#pragma unroll
-        for (int j = 0; j < KT; ++j)
-          if (dst[j] != nullptr) st_stream(dst[j] + c, v);
-      }
     } else {
-      for (int c0 = 0; c0 < H16; c0 += 32) {   // warp-uniform trip count: shuffles stay convergent
-        const int c = c0 + lane;
+      for (int i = w.i0; i < w.i1; ++i) {   // warp-uniform trip count: shuffles stay convergent
+        const int c = i * 32 + lane;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (c < H16) v = ld_stream(src + c);
         for (int j = 0; j < K; ++j) {
@@ -143,22 +184,24 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float (&acc)[8]) {
   return make_uint4(u[0], u[1], u[2], u[3]);
 }
 
-template <int KT, int UNROLL>
-__global__ void __launch_bounds__(256)
+template <int KT, int UNROLL, int MINB = 1>
+__global__ void __launch_bounds__(256, MINB)
 combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__ topk_w, uint4* __restrict__ Y,
                     const RowArgs a, const __grid_constant__ RankMap map) {
+  begin_work(a);
   if (must_abort(a)) return;
   const int lane = threadIdx.x & 31;
-  const int warps_per_cta = blockDim.x >> 5;
-  const int32_t warp0 = blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
-  const int32_t nwarps = gridDim.x * warps_per_cta;
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
 
-  for (int32_t t = warp0; t < a.T; t += nwarps) {
-    const int64_t slot = resolve_slot(a, map, t, lane, false);
-    const float w_lane = lane < K ? __ldg(topk_w + (size_t)t * K + lane) : 0.0f;
-    uint4* out = Y + (size_t)t * H16;
+  int32_t item = fetch_item(a);
+  while (item < a.n_items) {
+    const int32_t next_item = fetch_item(a);
+    const WorkItem wi = decode_item(a, item);
+    item = next_item;
+    const int64_t slot = resolve_slot(a, map, wi.t, lane, false);
+    const float w_lane = lane < K ? __ldg(topk_w + (size_t)wi.t * K + lane) : 0.0f;
+    uint4* out = Y + (size_t)wi.t * H16;
     if constexpr (KT > 0) {
       const uint4* src[KT];
       float w[KT];
@@ -168,34 +211,28 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
         src[j] = row >= 0 ? windows + (size_t)row * H16 : nullptr;
         w[j] = __shfl_sync(0xffffffffu, w_lane, j);
       }
-      int c = lane;
-      for (; c + 32 * (UNROLL - 1) < H16; c += 32 * UNROLL) {
+      for (int i = wi.i0; i < wi.i1; i += UNROLL) {
         uint4 v[UNROLL][KT];
+        bool ok[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u)
+        for (int u = 0; u < UNROLL; ++u) {
+          const int c = (i + u) * 32 + lane;
+          ok[u] = (i + u < wi.i1) && (c < H16);
 #pragma unroll
           for (int j = 0; j < KT; ++j)
-            v[u][j] = src[j] != nullptr ? ld_stream(src[j] + c + 32 * u) : make_uint4(0, 0, 0, 0);
+            v[u][j] = (ok[u] && src[j] != nullptr) ? ld_stream(src[j] + c) : make_uint4(0, 0, 0, 0);
+        }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
           float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int j = 0; j < KT; ++j) fma_bf16x8(acc, w[j], v[u][j]);   // j ascending, one fma per term
-          out[c + 32 * u] = pack_bf16x8(acc);
+          if (ok[u]) out[(i + u) * 32 + lane] = pack_bf16x8(acc);
         }
       }
-      for (; c < H16; c += 32) {
-        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        uint4 v[KT];
-#pragma unroll
-        for (int j = 0; j < KT; ++j) v[j] = src[j] != nullptr ? ld_stream(src[j] + c) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-        for (int j = 0; j < KT; ++j) fma_bf16x8(acc, w[j], v[j]);
-        out[c] = pack_bf16x8(acc);
-      }
     } else {
-      for (int c0 = 0; c0 < H16; c0 += 32) {
-        const int c = c0 + lane;
+      for (int i = wi.i0; i < wi.i1; ++i) {
+        const int c = i * 32 + lane;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int j = 0; j < K; ++j) {
           const int64_t row = __shfl_sync(0xffffffffu, slot, j);

@@ -87,13 +87,15 @@ class GpuRun:
 
 
 def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Optional[binding.MoeComm] = None,
-            T_max: Optional[int] = None) -> GpuRun:
+            T_max: Optional[int] = None, dispatch_path: int = binding.MOE_DISPATCH_AUTO, granule: int = 0) -> GpuRun:
     wl = inp.wl
     dev = torch.device("cuda:0")
     schedule = wl.schedule if schedule is None else schedule
     own = comm is None
     if own:
         comm = binding.MoeComm(T_max or max(wl.T, 1), wl.H, wl.E, wl.R, wl.K, dev)
+    comm.moe_set_option(binding.MOE_OPT_DISPATCH_PATH, dispatch_path)
+    comm.moe_set_option(binding.MOE_OPT_GRANULE, granule)
     idx = inp.topk_idx.to(dev)
     w = inp.topk_w.to(dev)
     X = inp.X.to(dev)

@@ -18,14 +18,20 @@ import harness
 pytestmark = pytest.mark.gpu
 
 
-def run_and_check(wl, schedule=None, slack=3):
+PATHS = [binding.MOE_DISPATCH_BULK, binding.MOE_DISPATCH_REGISTERS]
+
+
+def run_and_check(wl, schedule=None, slack=3, paths=PATHS, granule=0):
     inp = synth.make_inputs(wl)
     p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R, inp.rank_tok_start)
     C = int(p.n_recv.max()) + slack if wl.T else slack
     o = harness.oracle_run(inp, C)
     sch = wl.schedule if schedule is None else schedule
-    g = harness.gpu_run(inp, C, sch)
-    return harness.assert_parity(g, o, sch)
+    worst = 0
+    for path in paths:                      # every dispatch kernel must give the same bytes
+        g = harness.gpu_run(inp, C, sch, dispatch_path=path, granule=granule)
+        worst = max(worst, harness.assert_parity(g, o, sch))
+    return worst
 
 
 # ------------------------------------------------------------------ the benchmark configurations
@@ -93,6 +99,14 @@ def test_edge_shapes(case, schedule):
     name, T, H, E, R, K, routing, rank_tokens = case
     wl = Workload(name, T, H, E, R, K, schedule, routing, "scale", 4000 + T, rank_tokens=rank_tokens)
     run_and_check(wl)
+
+
+@pytest.mark.parametrize("granule", [1, 3, 5, 28, 1000])
+def test_any_work_item_size_gives_the_same_result(granule):
+    wl = Workload("granule", 300, 7168, 64, 4, 8, DECODE, "uniform", "scale", 4242)
+    run_and_check(wl, granule=granule)
+    wl = Workload("granule_ragged_row", 123, 1000, 16, 2, 6, PREFILL, "uniform", "scale", 4243, rank_tokens=(23, 100))
+    run_and_check(wl, granule=granule)
 
 
 def test_empty_batch():
