@@ -39,7 +39,13 @@ L2_BYTES = 126 << 20
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures summarised under
 # profiles/; keyed by (kernel, workload).  None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # captured at T=8192 (1009.5 MB / 998.4 MB per launch) and scaled by 4: every token moves the same bytes
+    ("combine_rows_kernel", "c3_prefill_dsv3"): 4 * 1009.5e6,
+    ("dispatch_bulk_kernel", "c3_prefill_dsv3"): 4 * 998.4e6,
+    ("combine_rows_kernel", "c3_prefill_dsv3_T8192"): 1009.5e6,
+    ("dispatch_bulk_kernel", "c3_prefill_dsv3_T8192"): 998.4e6,
+}
 
 WORKLOADS = {
     "c1": lambda: synth.config(1),
@@ -343,7 +349,7 @@ def finish(args, wl, world, dist, ms_per_step, step_bytes, b_plan, b_disp, b_com
         kernels[k]["frac_of_measured_peak"] = kernels[k]["GBps"] / peak
         kernels[k]["frac_of_8TBps"] = kernels[k]["GBps"] / NOMINAL_HBM_GBS
     dom = "moe_dispatch" if sum(disp_us) >= sum(comb_us) else "moe_combine"
-    dom_kernel = "dispatch_rows_kernel" if dom == "moe_dispatch" else "combine_rows_kernel"
+    dom_kernel = "dispatch_bulk_kernel" if dom == "moe_dispatch" else "combine_rows_kernel"
     roofline = {"bound": "hbm", "kernel": dom_kernel, "achieved": kernels[dom]["GBps"], "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kernels[dom]["GBps"] / peak,
                 "traffic": NCU_TRAFFIC_BYTES.get((dom_kernel, wl.name))}
