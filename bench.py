@@ -8,10 +8,12 @@ reads the dispatched windows in place).  Prints ONE JSON line.
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3]
   python bench.py --impl reference ...     # the CPU oracle, timed on the host cores
 
-Multi-GPU: the path does not shard (the R expert-parallel ranks are virtual
-segments of one GPU's memory), so N > 1 runs N independent replicas, one
-process per GPU, with no data-path collective; value is the sum over replicas
-divided by the slowest replica's time ("weak" scaling).
+Default workload: c3, the DeepSeek-V3-like prefill shape on which the HBM
+roofline target is stated; the same line carries the decode-step latency (c2)
+under "decode".  Multi-GPU: the path does not shard (the R expert-parallel
+ranks are virtual segments of one GPU's memory), so N > 1 runs N independent
+replicas, one process per GPU, with no data-path collective; value is the sum
+over replicas divided by the slowest replica's time ("weak" scaling).
 """
 from __future__ import annotations
 
@@ -33,12 +35,13 @@ import torch
 
 from paper_2605_06055_b200 import synth
 
+METRIC = "moe_plan_dispatch_combine_hbm_gbps"
 NOMINAL_HBM_GBS = 8000.0          # the metric's nominal denominator ("~8 TB/s")
 FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used only without MEASURED_PEAKS.json
 L2_BYTES = 126 << 20
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures summarised under
-# profiles/; keyed by (kernel, workload).  None = not captured.
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/; keyed by (kernel, workload).  Absent = not captured.
 NCU_TRAFFIC_BYTES = {
     # captured at T=8192 (1009.5 MB / 998.4 MB per launch) and scaled by 4: every token moves the same bytes
     ("combine_rows_kernel", "c3_prefill_dsv3"): 4 * 1009.5e6,
@@ -75,6 +78,10 @@ def bytes_plan(wl) -> int:
     return 8 * wl.T * wl.K + 8 * wl.E * wl.R
 
 
+def bytes_step(wl) -> int:
+    return bytes_plan(wl) + bytes_dispatch(wl) + bytes_combine(wl)
+
+
 def describe(wl) -> dict:
     return {"workload": wl.name, "T": wl.T, "H": wl.H, "E": wl.E, "R": wl.R, "K": wl.K,
             "schedule": "prefill" if wl.schedule == synth.PREFILL else "decode", "routing": wl.routing,
@@ -93,7 +100,7 @@ def measured_peak():
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the device is under load."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -107,7 +114,8 @@ class ClockSampler:
             sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
         except Exception:
             pass
-        self.cmd = ["nvidia-smi", "-i", sel, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        self.cmd = ["nvidia-smi", "-i", sel, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                    "-lms", "50"]
 
     def start(self):
         try:
@@ -124,7 +132,6 @@ class ClockSampler:
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -183,17 +190,15 @@ def time_oracle(wl, steps: int, warmup: int, inp=None):
 
 
 def run_reference(args, wl):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     sample = oracle_sample(wl, 8)
     times, cores = time_oracle(sample, args.steps, args.warmup)
     sec = sum(times) / len(times)
-    nbytes = bytes_plan(sample) + bytes_dispatch(sample) + bytes_combine(sample)
-    value = nbytes / sec / 1e9
-    what = f"first 1/8 of every rank's tokens of {wl.name} (T={sample.T}) per step"
+    value = bytes_step(sample) / sec / 1e9
+    what = f"first 1/8 of every rank's tokens of {wl.name} (T={sample.T}) per step, token-parallel over all cores"
     line = {
-        "impl": "reference", "metric": "moe_plan_dispatch_combine_hbm_gbps", "value": value, "unit": "GB/s",
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": describe(wl),
@@ -204,13 +209,146 @@ def run_reference(args, wl):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
-def flush_l2(buf):
-    buf.add_(1)
+def reduce_max_over_ranks(value: float, dist, dev) -> float:
+    """Slowest replica's time (device-timed), as the contract asks for multi-GPU numbers."""
+    if dist is None:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(step_bytes: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` replicas that each move step_bytes per step."""
+    return world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+
+class Layer:
+    """Device buffers and the library context for one workload."""
+
+    def __init__(self, wl, dev, pin=False):
+        from paper_2605_06055_b200 import binding
+        self.wl, self.dev = wl, dev
+        self.inp = synth.make_inputs(wl, pin=pin)
+        self.X, self.idx, self.w = self.inp.X.to(dev), self.inp.topk_idx.to(dev), self.inp.topk_w.to(dev)
+        self.comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+        # capacity sized from the actual counts (plan -> status -> n_recv), as the prefill schedule allows
+        self.comm.moe_plan(wl.schedule, self.idx)
+        assert self.comm.moe_status() == 0
+        C = int(self.comm.moe_plan_view()["n_recv"].max().item())
+        self.C = (C + 7) // 8 * 8
+        self.windows = torch.zeros((wl.R * self.C, wl.H), dtype=torch.bfloat16, device=dev)
+        self.Y = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+        self.big = bytes_dispatch(wl) > 2 * L2_BYTES
+
+    def step(self, events=None):
+        c, wl = self.comm, self.wl
+        if events is not None:
+            events[0].record()
+        c.moe_plan(wl.schedule, self.idx)
+        if events is not None:
+            events[1].record()
+        c.moe_dispatch(self.X, self.windows, self.C)
+        if events is not None:
+            events[2].record()
+        c.moe_combine(self.windows, self.C, self.w, self.Y)
+        if events is not None:
+            events[3].record()
+
+
+def time_steps(layer: Layer, steps: int, warmup: int, barrier, scratch=None):
+    """K steps bracketed by CUDA events on the launching stream, plus per-call events inside."""
+    for _ in range(max(warmup, 3)):
+        layer.step()
+    assert layer.comm.moe_status() == 0
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    gaps = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps)]
+    barrier()
+    launches0 = layer.comm.moe_launch_count()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(steps):
+        if scratch is not None:         # small workload: flush L2 between steps, outside the per-call events
+            gaps[2 * i].record()
+            scratch.add_(1)
+            gaps[2 * i + 1].record()
+        layer.step(ev[i])
+    t_end.record()
+    barrier()
+    assert layer.comm.moe_status() == 0
+    total_ms = t_start.elapsed_time(t_end)
+    if scratch is not None:
+        total_ms -= sum(gaps[2 * i].elapsed_time(gaps[2 * i + 1]) for i in range(steps))
+    return {
+        "ms_per_step": total_ms / steps,
+        "plan_us": [e[0].elapsed_time(e[1]) * 1e3 for e in ev],
+        "dispatch_us": [e[1].elapsed_time(e[2]) * 1e3 for e in ev],
+        "combine_us": [e[2].elapsed_time(e[3]) * 1e3 for e in ev],
+        "launches": layer.comm.moe_launch_count() - launches0,
+    }
+
+
+def time_graph_steps(layer: Layer, steps: int, scratch=None):
+    """The same step captured once in a CUDA graph and replayed (what a decode loop would do)."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        layer.step()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        if scratch is not None:
+            scratch.add_(1)
+        a.record()
+        g.replay()
+        b.record()
+    torch.cuda.synchronize()
+    assert layer.comm.moe_status() == 0
+    return [a.elapsed_time(b) * 1e3 for a, b in ev]
+
+
+def time_e2e(layer: Layer, steps: int, barrier):
+    """Whole layer through the C ABI from pinned HOST buffers: H2D of X, K, W and D2H of Y every step."""
+    wl, c = layer.wl, layer.comm
+    idx_h, w_h = layer.inp.topk_idx.pin_memory(), layer.inp.topk_w.pin_memory()
+    x_h = layer.inp.X if layer.inp.X.is_pinned() else layer.inp.X.pin_memory()
+    y_h = torch.empty((wl.T, wl.H), dtype=torch.bfloat16).pin_memory()
+    x_d, idx_d, w_d = torch.empty_like(layer.X), torch.empty_like(layer.idx), torch.empty_like(layer.w)
+
+    def one():
+        c.moe_forward_host(wl.schedule, wl.T, None, x_h, idx_h, w_h, x_d, idx_d, w_d, layer.windows, layer.C,
+                           layer.Y, y_h)
+    for _ in range(2):
+        one()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        one()
+    t1.record()
+    barrier()
+    assert c.moe_status() == 0
+    return t0.elapsed_time(t1) / steps, wl.T * wl.H * 2 + wl.T * wl.K * 8, wl.T * wl.H * 2
+
+
+def kernel_table(wl, r, peak):
+    med = statistics.median
+    mean = lambda v: sum(v) / len(v)
+    k = {
+        "moe_plan": {"us": med(r["plan_us"]), "bytes": bytes_plan(wl)},
+        "moe_dispatch": {"us": med(r["dispatch_us"]), "us_min": min(r["dispatch_us"]), "bytes": bytes_dispatch(wl),
+                         "GBps": bytes_dispatch(wl) / mean(r["dispatch_us"]) / 1e3},
+        "moe_combine": {"us": med(r["combine_us"]), "us_min": min(r["combine_us"]), "bytes": bytes_combine(wl),
+                        "GBps": bytes_combine(wl) / mean(r["combine_us"]) / 1e3},
+    }
+    for name in ("moe_dispatch", "moe_combine"):
+        k[name]["frac_of_measured_peak"] = k[name]["GBps"] / peak
+        k[name]["frac_of_8TBps"] = k[name]["GBps"] / NOMINAL_HBM_GBS
+    return k
 
 
 def run_cuda(args, wl):
-    from paper_2605_06055_b200 import binding
-
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -221,158 +359,79 @@ def run_cuda(args, wl):
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
 
-    inp = synth.make_inputs(wl, pin=True)
-    idx_h, w_h = inp.topk_idx.pin_memory(), inp.topk_w.pin_memory()
-    X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
-    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
-
-    # capacity sized from the actual counts (plan -> status -> n_recv), as the prefill schedule allows
-    comm.moe_plan(wl.schedule, idx)
-    assert comm.moe_status() == 0
-    C = int(comm.moe_plan_view()["n_recv"].max().item())
-    C = (C + 7) // 8 * 8
-    windows = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
-    Y = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
-    b_plan, b_disp, b_comb = bytes_plan(wl), bytes_dispatch(wl), bytes_combine(wl)
-    step_bytes = b_plan + b_disp + b_comb
-    big = (b_disp > 2 * L2_BYTES)
-    scratch = None if big else torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-
-    def step(events=None):
-        if events is not None:
-            events[0].record()
-        comm.moe_plan(wl.schedule, idx)
-        if events is not None:
-            events[1].record()
-        comm.moe_dispatch(X, windows, C)
-        if events is not None:
-            events[2].record()
-        comm.moe_combine(windows, C, w, Y)
-        if events is not None:
-            events[3].record()
-
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    assert comm.moe_status() == 0
-
-    # ---- timed region: exactly K steps, CUDA events on the launching stream
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    gaps = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps)]
     sampler = ClockSampler(local)
+    layer = Layer(wl, dev, pin=not args.no_e2e)
+    scratch = None if layer.big else torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
     sampler.start()
-    barrier()
-    launches0 = comm.moe_launch_count()
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for i in range(args.steps):
-        if scratch is not None:         # small workload: flush L2 between steps, outside the per-call events
-            gaps[2 * i].record()
-            flush_l2(scratch)
-            gaps[2 * i + 1].record()
-        step(ev[i])
-    t_end.record()
-    barrier()
-    launches = comm.moe_launch_count() - launches0
-    total_ms = t_start.elapsed_time(t_end)
-    if scratch is not None:
-        total_ms -= sum(gaps[2 * i].elapsed_time(gaps[2 * i + 1]) for i in range(args.steps))
-    clocks = sampler.stop()
-    assert comm.moe_status() == 0
-    plan_us = [e[0].elapsed_time(e[1]) * 1e3 for e in ev]
-    disp_us = [e[1].elapsed_time(e[2]) * 1e3 for e in ev]
-    comb_us = [e[2].elapsed_time(e[3]) * 1e3 for e in ev]
-    ms_per_step = total_ms / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_per_step], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
-
-    # ---- end to end through the C ABI from HOST buffers (copies inside the timed region)
+    r = time_steps(layer, args.steps, args.warmup, barrier, scratch)
+    ms_per_step = reduce_max_over_ranks(r["ms_per_step"], dist, dev)
     e2e = None
     if not args.no_e2e:
-        e2e = measure_e2e(args, wl, comm, inp, idx_h, w_h, X, idx, w, windows, C, Y, barrier, dist, dev, world,
-                          step_bytes)
-
+        e2e_steps = max(3, min(args.steps, 10))
+        e2e_ms, h2d, d2h = time_e2e(layer, e2e_steps, barrier)
+        e2e_ms = reduce_max_over_ranks(e2e_ms, dist, dev)
+        e2e = {"value": aggregate_value(bytes_step(wl), world, e2e_ms), "unit": "GB/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+    clocks = sampler.stop()
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
-    return finish(args, wl, world, dist, ms_per_step, step_bytes, b_plan, b_disp, b_comb, plan_us, disp_us, comb_us,
-                  clocks, launches, e2e, C, big, inp)
 
-
-def measure_e2e(args, wl, comm, inp, idx_h, w_h, X, idx, w, windows, C, Y, barrier, dist, dev, world, step_bytes):
-    y_host = torch.empty((wl.T, wl.H), dtype=torch.bfloat16).pin_memory()
-    x_dev2, idx_dev2, w_dev2 = torch.empty_like(X), torch.empty_like(idx), torch.empty_like(w)
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
-        comm.moe_forward_host(wl.schedule, wl.T, None, inp.X, idx_h, w_h, x_dev2, idx_dev2, w_dev2, windows, C, Y,
-                              y_host)
-    barrier()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(e2e_steps):
-        comm.moe_forward_host(wl.schedule, wl.T, None, inp.X, idx_h, w_h, x_dev2, idx_dev2, w_dev2, windows, C, Y,
-                              y_host)
-    t1.record()
-    barrier()
-    assert comm.moe_status() == 0
-    e2e_ms = t0.elapsed_time(t1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    h2d = wl.T * wl.H * 2 + wl.T * wl.K * 8
-    d2h = wl.T * wl.H * 2
-    return {"value": world * step_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
-            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
-
-
-def finish(args, wl, world, dist, ms_per_step, step_bytes, b_plan, b_disp, b_comb, plan_us, disp_us, comb_us, clocks,
-           launches, e2e, C, big, inp):
     peak, peak_kind = measured_peak()
-    med = statistics.median
-    kernels = {
-        "moe_plan": {"us": med(plan_us), "bytes": b_plan},
-        "moe_dispatch": {"us": med(disp_us), "us_min": min(disp_us), "bytes": b_disp,
-                         "GBps": b_disp / (sum(disp_us) / len(disp_us)) / 1e3},
-        "moe_combine": {"us": med(comb_us), "us_min": min(comb_us), "bytes": b_comb,
-                        "GBps": b_comb / (sum(comb_us) / len(comb_us)) / 1e3},
-    }
-    for k in ("moe_dispatch", "moe_combine"):
-        kernels[k]["frac_of_measured_peak"] = kernels[k]["GBps"] / peak
-        kernels[k]["frac_of_8TBps"] = kernels[k]["GBps"] / NOMINAL_HBM_GBS
-    dom = "moe_dispatch" if sum(disp_us) >= sum(comb_us) else "moe_combine"
+    kernels = kernel_table(wl, r, peak)
+    dom = "moe_dispatch" if sum(r["dispatch_us"]) >= sum(r["combine_us"]) else "moe_combine"
     dom_kernel = "dispatch_bulk_kernel" if dom == "moe_dispatch" else "combine_rows_kernel"
     roofline = {"bound": "hbm", "kernel": dom_kernel, "achieved": kernels[dom]["GBps"], "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kernels[dom]["GBps"] / peak,
                 "traffic": NCU_TRAFFIC_BYTES.get((dom_kernel, wl.name))}
-
+    dc_us = kernels["moe_dispatch"]["us"] + kernels["moe_combine"]["us"]
     line = {
-        "metric": "moe_plan_dispatch_combine_hbm_gbps", "value": world * step_bytes / (ms_per_step * 1e-3) / 1e9,
+        "metric": METRIC, "value": aggregate_value(bytes_step(wl), world, ms_per_step),
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": dict(describe(wl), capacity_rows=C, replicas=world,
-                       l2="inputs larger than L2" if big else "256 MB L2 flush between steps (untimed)"),
-        "dispatch_plus_combine_us": med(disp_us) + med(comb_us),
-        "frac_of_8TBps": (b_disp + b_comb) / ((med(disp_us) + med(comb_us)) * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
-        "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": launches,
-        "e2e": e2e,
+        "config": dict(describe(wl), capacity_rows=layer.C, replicas=world,
+                       l2="inputs larger than L2" if layer.big else "256 MB L2 flush between steps (untimed)"),
+        "dispatch_plus_combine_us": dc_us,
+        "frac_of_8TBps": (bytes_dispatch(wl) + bytes_combine(wl)) / (dc_us * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+        "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": r["launches"], "e2e": e2e,
     }
+
+    cpu_inp = layer.inp
+    del layer, scratch
+    torch.cuda.empty_cache()
+
+    if world == 1 and not args.no_decode and wl.name != synth.config(2).name:
+        # decode-step latency (config 2) in the same line: stream launches and CUDA-graph replay
+        dwl = synth.config(2)
+        dl = Layer(dwl, dev)
+        flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+        dr = time_steps(dl, 100, 5, barrier, flush)
+        gk = kernel_table(dwl, dr, peak)
+        graph_us = time_graph_steps(dl, 100, flush)
+        line["decode"] = {
+            "config": describe(dwl), "l2": "256 MB L2 flush between steps (untimed)",
+            "plan_us": gk["moe_plan"]["us"], "dispatch_us": gk["moe_dispatch"]["us"],
+            "combine_us": gk["moe_combine"]["us"], "step_us_stream_launches": dr["ms_per_step"] * 1e3,
+            "step_us_cuda_graph": statistics.median(graph_us),
+            "dispatch_GBps": gk["moe_dispatch"]["GBps"], "combine_GBps": gk["moe_combine"]["GBps"],
+            "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3,
+        }
+        del dl, flush
+        torch.cuda.empty_cache()
 
     if world == 1 and not args.no_cpu_baseline:
         sample = wl if wl.T * wl.K * wl.H <= 2 * (1 << 30) else oracle_sample(wl, 2)
-        times, cores = time_oracle(sample, 1, 1, inp if sample is wl else None)
-        sb = bytes_plan(sample) + bytes_dispatch(sample) + bytes_combine(sample)
-        line["cpu_baseline"] = {"value": sb / times[0] / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                                "ms": times[0] * 1e3,
+        times, cores = time_oracle(sample, 1, 1, cpu_inp if sample is wl else None)
+        line["cpu_baseline"] = {"value": bytes_step(sample) / times[0] / 1e9, "unit": "GB/s", "cores": cores,
+                                "kind": "oracle", "ms": times[0] * 1e3,
                                 "sample": ("whole workload" if sample is wl else
                                            f"first half of every rank's tokens (T={sample.T})") +
                                           ", one timed pass after one warm-up pass, token-parallel over all cores"}
@@ -384,17 +443,22 @@ def finish(args, wl, world, dist, ms_per_step, step_bytes, b_plan, b_disp, b_com
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None, help="default 200 (cuda) / 10 (reference)")
+    ap.add_argument("--warmup", type=int, default=None, help="default 10 (cuda) / 2 (reference)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-decode", action="store_true", help="skip the decode-latency leg (profiling runs)")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]()
-    if args.impl == "reference":
+    if args.impl == "reference":                 # the oracle takes ~0.3 s per step on its 1/8 sample
+        args.steps = 10 if args.steps is None else args.steps
+        args.warmup = 2 if args.warmup is None else args.warmup
         run_reference(args, wl)
     else:
+        args.steps = 200 if args.steps is None else args.steps
+        args.warmup = 10 if args.warmup is None else args.warmup
         run_cuda(args, wl)
 
 

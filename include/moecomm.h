@@ -53,7 +53,8 @@ typedef enum {
 /* The two schedules of Section 4.  PREFILL runs Layout + Notify as separate
  * planning passes and keeps the whole planning table readable.  DECODE keeps
  * only the compact state (o_dec, delta, n_recv); delta is produced inside the
- * dispatch launch (Section 5.3, Decode Dispatch). */
+ * dispatch launch (Section 5.3, Decode Dispatch), or already by the single
+ * planning launch when every source rank holds at most 4096 branches. */
 typedef enum { MOE_SCHED_PREFILL = 0, MOE_SCHED_DECODE = 1 } moe_schedule_t;
 
 typedef struct {
@@ -96,7 +97,9 @@ moe_status_t moe_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* to
  * context.  Shapes: counts M [R,E], c_rank [R,R], small_off s|delta [T,K],
  * large_off o|o_dec [E,R] (window-local row), n_exp [E], n_recv [R].
  * PREFILL fills every field.  DECODE leaves counts, c_rank and n_exp NULL, and
- * small_off holds delta only after moe_dispatch has run. */
+ * small_off is guaranteed to hold delta only after moe_dispatch has run (small
+ * decode batches, at most 4096 branches per source rank, are planned in a single
+ * launch that already leaves it final after moe_plan). */
 typedef struct {
   const int32_t* counts;
   const int32_t* c_rank;

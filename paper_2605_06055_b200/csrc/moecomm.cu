@@ -25,6 +25,7 @@ struct moe_ctx {
   int32_t *M, *c_rank, *o, *n_exp, *n_recv, *s, *tile_rank, *tile_hist;
   // plan state (host)
   bool planned;
+  bool compact_plan;  // DECODE plan done by plan_rank_kernel: small offsets are final after moe_plan
   moe_schedule_t schedule;
   int32_t T;
   int32_t n_tiles;
@@ -37,6 +38,10 @@ struct moe_ctx {
 };
 
 namespace {
+
+// DECODE plans whose ranks each hold at most this many branches take the single-launch planner.
+constexpr int64_t RANK_PLAN_MAX_BRANCHES = 4096;
+constexpr int RANK_PLAN_WIDE_MAX_E = 768;   // 32-warp CTAs while 33*E counters fit comfortably in shared memory
 
 constexpr size_t ALIGN = 256;
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
@@ -95,7 +100,7 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   // DECODE: small offsets are finished on the fly (in-tile rank + tile base) by every consumer, so a
   // dispatch that aborted on the device can never leave a later call with half-written state; the
   // dispatch launch also records them, which is what moe_plan_view exposes as delta.
-  const bool finish_delta = ctx->schedule == MOE_SCHED_DECODE;
+  const bool finish_delta = ctx->schedule == MOE_SCHED_DECODE && !ctx->compact_plan;
   a.small_off = finish_delta ? ctx->tile_rank : ctx->s;
   a.small_out = (finish_delta && dispatching) ? ctx->s : nullptr;
   a.tile_base = finish_delta ? ctx->tile_hist : nullptr;
@@ -225,6 +230,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->tile_rank = reinterpret_cast<int32_t*>(ctx->ws + L.tile_rank);
   ctx->tile_hist = reinterpret_cast<int32_t*>(ctx->ws + L.tile_hist);
   ctx->planned = false;
+  ctx->compact_plan = false;
   ctx->launches = 0;
   ctx->topk_idx = nullptr;
   ctx->work_parity = 0;
@@ -237,6 +243,13 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   if (ok)
     ok = cudaFuncSetAttribute(dispatch_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               BULK_WARPS * BULK_STAGES * (BULK_MAX_GRANULE * 512 + 8)) == cudaSuccess;
+  if (ok) {
+    const int wide = 33 * shape->E * (int)sizeof(int32_t), narrow = 9 * shape->E * (int)sizeof(int32_t);
+    if (shape->E <= RANK_PLAN_WIDE_MAX_E && wide > 48 * 1024)
+      ok = cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide) == cudaSuccess;
+    if (ok && shape->E > RANK_PLAN_WIDE_MAX_E && narrow > 48 * 1024)
+      ok = cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, narrow) == cudaSuccess;
+  }
   if (ok && tile_smem > 48 * 1024) {
     ok = cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_PREFILL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               tile_smem) == cudaSuccess &&
@@ -301,23 +314,39 @@ moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk
   const int tile_smem = PLAN_WARPS * sh.E * (int)sizeof(int32_t);
   const int scan_smem = (2 * sh.E + 1) * (int)sizeof(int32_t);
   const int full = schedule == MOE_SCHED_PREFILL;
-  int n = 0;
-  if (tiles > 0) {
-    if (full)
-      plan_tile_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, tile_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
-    else
-      plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, tile_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
-    ++n;
+  int64_t max_rank_branches = 0;
+  for (int r = 0; r < sh.R; ++r) {
+    const int64_t br = (int64_t)(map.tok_start[r + 1] - map.tok_start[r]) * sh.K;
+    if (br > max_rank_branches) max_rank_branches = br;
   }
-  plan_scan_kernel<<<sh.R, PLAN_THREADS, scan_smem, st>>>(ctx->tile_hist, map, sh.E, full, ctx->M, ctx->c_rank,
-                                                          ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
-  ++n;
-  if (full && tiles > 0) {
-    plan_finalize_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, 0, st>>>(topk_idx, map, sh.K, sh.E, ctx->tile_rank,
-                                                                        ctx->tile_hist, ctx->s);
+  ctx->compact_plan = !full && max_rank_branches <= RANK_PLAN_MAX_BRANCHES;
+  int n = 0;
+  if (ctx->compact_plan) {
+    if (sh.E <= RANK_PLAN_WIDE_MAX_E)
+      plan_rank_kernel<32><<<sh.R, 32 * 32, 33 * sh.E * (int)sizeof(int32_t), st>>>(
+          topk_idx, map, sh.K, sh.E, ctx->s, ctx->M, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+    else
+      plan_rank_kernel<8><<<sh.R, 8 * 32, 9 * sh.E * (int)sizeof(int32_t), st>>>(
+          topk_idx, map, sh.K, sh.E, ctx->s, ctx->M, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     ++n;
+  } else {
+    if (tiles > 0) {
+      if (full)
+        plan_tile_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, tile_smem, st>>>(
+            topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
+      else
+        plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, tile_smem, st>>>(
+            topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
+      ++n;
+    }
+    plan_scan_kernel<<<sh.R, PLAN_THREADS, scan_smem, st>>>(ctx->tile_hist, map, sh.E, full, ctx->M, ctx->c_rank,
+                                                            ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+    ++n;
+    if (full && tiles > 0) {
+      plan_finalize_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, 0, st>>>(topk_idx, map, sh.K, sh.E, ctx->tile_rank,
+                                                                          ctx->tile_hist, ctx->s);
+      ++n;
+    }
   }
   const moe_status_t rc = launch_ok(ctx, n);
   if (rc == MOE_OK) ctx->planned = true;

@@ -18,6 +18,7 @@
 //                      (exclusive scan in window order: expert, then source rank).
 //   plan_finalize_kernel  PREFILL only: s = in-tile rank + tile base.
 //                      (DECODE folds this step into the dispatch launch.)
+//   plan_rank_kernel   DECODE with few branches per rank: the whole plan in one launch.
 #pragma once
 
 #include "common.cuh"
@@ -120,6 +121,44 @@ __device__ __forceinline__ void warp0_exclusive_scan(const int32_t* in, int32_t*
   }
 }
 
+// Notify step proper: turns the complete count matrix M into receive counts and large offsets.
+// Run by ONE CTA (the last to finish counting).  sm: 2*E + 1 ints of shared memory.
+__device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ M, int32_t E, int32_t R,
+                                                    int32_t full_table, int32_t* __restrict__ c_rank,
+                                                    int32_t* __restrict__ o, int32_t* __restrict__ n_exp,
+                                                    int32_t* __restrict__ n_recv, int32_t* sm) {
+  int32_t* nexp_s = sm;
+  int32_t* pre_s = sm + E;
+  const int E_r = E / R;
+  for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
+    int32_t acc = 0;
+    for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);
+    nexp_s[e] = acc;
+    n_exp[e] = acc;
+  }
+  __syncthreads();
+  warp0_exclusive_scan(nexp_s, pre_s, E);
+  __syncthreads();
+  // Window of rank d = experts d*E_r ..; offsets restart at 0 in every window.
+  for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
+    const int d = e / E_r;
+    int32_t run = pre_s[e] - pre_s[d * E_r];
+    for (int rr = 0; rr < R; ++rr) {
+      o[(size_t)e * R + rr] = run;
+      run += __ldcg(M + (size_t)rr * E + e);
+    }
+  }
+  for (int d = threadIdx.x; d < R; d += (int)blockDim.x) n_recv[d] = pre_s[(d + 1) * E_r] - pre_s[d * E_r];
+  if (full_table) {
+    for (int i = threadIdx.x; i < R * R; i += (int)blockDim.x) {
+      const int rr = i / R, d = i % R;
+      int32_t acc = 0;
+      for (int e = d * E_r; e < (d + 1) * E_r; ++e) acc += __ldcg(M + (size_t)rr * E + e);
+      c_rank[i] = acc;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(PLAN_THREADS)
 plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusive bases */,
                  const __grid_constant__ RankMap map, int32_t E, int32_t full_table,
@@ -151,37 +190,70 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
   if (!is_last) return;
   __threadfence();
 
-  int32_t* nexp_s = sm;
-  int32_t* pre_s = sm + E;
-  const int E_r = E / R;
-  for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
-    int32_t acc = 0;
-    for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);
-    nexp_s[e] = acc;
-    n_exp[e] = acc;
-  }
-  __syncthreads();
-  warp0_exclusive_scan(nexp_s, pre_s, E);
-  __syncthreads();
-  // Window of rank d = experts d*E_r ..; offsets restart at 0 in every window.
-  for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
-    const int d = e / E_r;
-    int32_t run = pre_s[e] - pre_s[d * E_r];
-    for (int rr = 0; rr < R; ++rr) {
-      o[(size_t)e * R + rr] = run;
-      run += __ldcg(M + (size_t)rr * E + e);
-    }
-  }
-  for (int d = threadIdx.x; d < R; d += PLAN_THREADS) n_recv[d] = pre_s[(d + 1) * E_r] - pre_s[d * E_r];
-  if (full_table) {
-    for (int i = threadIdx.x; i < R * R; i += PLAN_THREADS) {
-      const int rr = i / R, d = i % R;
-      int32_t acc = 0;
-      for (int e = d * E_r; e < (d + 1) * E_r; ++e) acc += __ldcg(M + (size_t)rr * E + e);
-      c_rank[i] = acc;
-    }
-  }
+  build_large_offsets(M, E, R, full_table, c_rank, o, n_exp, n_recv, sm);
   if (threadIdx.x == 0) ctl->scan_ticket = 0;  // ready for the next plan on this stream
+}
+
+// Compact planner of the DECODE schedule when every source rank holds few branches: ONE launch, one
+// CTA per source rank.  The CTA walks its rank's branches in passes of WARPS*32, carrying the running
+// per-expert count in shared memory, so the small offsets come out final (no tile bases), row r of M
+// falls out at the end, and the last CTA to finish builds the large offsets.
+template <int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
+plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
+                 int32_t* __restrict__ s, int32_t* __restrict__ M, int32_t* __restrict__ o,
+                 int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
+  extern __shared__ int32_t sm[];   // [WARPS][E] per-warp counts, [E] running base  (reused: 2E+1 scan area)
+  __shared__ int is_last;
+  int32_t* warp_hist = sm;
+  int32_t* rank_base = sm + WARPS * E;
+  const int r = blockIdx.x, R = map.R;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int32_t b_begin = map.tok_start[r] * K, b_end = map.tok_start[r + 1] * K;
+  const unsigned lt = lanemask_lt();
+
+  for (int e = threadIdx.x; e < E; e += WARPS * 32) rank_base[e] = 0;
+  for (int32_t pass = b_begin; pass < b_end; pass += WARPS * 32) {
+    for (int i = threadIdx.x; i < WARPS * E; i += WARPS * 32) warp_hist[i] = 0;
+    __syncthreads();
+    const int32_t b = pass + warp * 32 + lane;
+    int32_t e = -1;
+    if (b < b_end) {
+      e = __ldg(topk_idx + b);
+      if (e < 0 || e >= E) {
+        raise_status(&ctl->status, MOE_ERR_BAD_INDEX);
+        e = -1;
+      }
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    const int ahead = __popc(peers & lt);
+    if (e >= 0 && ahead == 0) warp_hist[warp * E + e] = __popc(peers);   // one round per pass: no carry inside a warp
+    __syncthreads();
+    for (int x = threadIdx.x; x < E; x += WARPS * 32) {
+      int32_t run = rank_base[x];
+#pragma unroll 8
+      for (int w = 0; w < WARPS; ++w) {
+        const int32_t c = warp_hist[w * E + x];
+        warp_hist[w * E + x] = run;
+        run += c;
+      }
+      rank_base[x] = run;
+    }
+    __syncthreads();
+    if (b < b_end) s[b] = e >= 0 ? warp_hist[warp * E + e] + ahead : 0;
+    __syncthreads();
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += WARPS * 32) M[(size_t)r * E + e] = rank_base[e];
+
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(&ctl->scan_ticket, 1) == R - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  build_large_offsets(M, E, R, 0, nullptr, o, n_exp, n_recv, sm);
+  if (threadIdx.x == 0) ctl->scan_ticket = 0;
 }
 
 template <int ROUNDS>

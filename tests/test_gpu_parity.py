@@ -90,6 +90,8 @@ EDGE = [
     ("big_E", 3000, 32, 2048, 2, 8, "uniform", None),
     ("tile_boundary_exact", 2048, 32, 8, 2, 2, "uniform", None),   # 2048 branches per rank = exactly one tile
     ("tile_boundary_plus1", 2050, 32, 8, 2, 2, "uniform", None),
+    ("rank_above_compact_decode_limit", 6000, 16, 16, 2, 2, "uniform", (5000, 1000)),   # 10000 branches in rank 0
+    ("compact_decode_several_passes", 1200, 16, 1024, 2, 6, "uniform", (682, 518)),     # E > 768: 8-warp planner
 ]
 
 
