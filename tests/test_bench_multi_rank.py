@@ -1,0 +1,47 @@
+"""Host logic of the multi-GPU bench path on CPU: two gloo ranks, the reduction
+that turns per-replica device times into the job's number (max over ranks), and
+the replica aggregation."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = 1.25 if rank == 0 else 2.5            # ms per step measured by this replica
+    slowest = bench.reduce_max_over_ranks(mine, dist, torch.device("cpu"))
+    dist.barrier()
+    out[rank] = slowest
+    dist.destroy_process_group()
+
+
+def test_two_replicas_report_the_slowest_time_and_the_summed_bytes():
+    import bench
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, 29000 + os.getpid() % 2000, out), nprocs=world, join=True)
+        assert out[0] == 2.5 and out[1] == 2.5
+    wl = bench.WORKLOADS["c2"]()
+    one = bench.aggregate_value(bench.bytes_step(wl), 1, 2.5)
+    two = bench.aggregate_value(bench.bytes_step(wl), 2, 2.5)
+    assert abs(two - 2 * one) < 1e-9 * two
+    assert bench.reduce_max_over_ranks(3.0, None, torch.device("cpu")) == 3.0
+
+
+def test_algorithmic_bytes_match_the_stated_formulas():
+    import bench
+    wl = bench.WORKLOADS["c3"]()
+    # per token: one row read + K rows written (dispatch) / K rows read + one written (combine), rows of 2H bytes
+    assert bench.bytes_dispatch(wl) == 2 * 7168 * 32768 * 9 + 8 * 32768 * 8 + 4 * 256 * 8 == 4229963776
+    assert bench.bytes_combine(wl) == 2 * 7168 * 32768 * 9 + 12 * 32768 * 8 + 4 * 256 * 8
+    assert round(bench.bytes_dispatch(bench.WORKLOADS["c2"]()) / 1e6, 1) == 264.4
