@@ -232,6 +232,8 @@ class Layer:
         self.inp = synth.make_inputs(wl, pin=pin)
         self.X, self.idx, self.w = self.inp.X.to(dev), self.inp.topk_idx.to(dev), self.inp.topk_w.to(dev)
         self.comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+        if os.environ.get("MOE_BENCH_GRANULE"):      # tuning aid: work-item size override
+            self.comm.moe_set_option(binding.MOE_OPT_GRANULE, int(os.environ["MOE_BENCH_GRANULE"]))
         # capacity sized from the actual counts (plan -> status -> n_recv), as the prefill schedule allows
         self.comm.moe_plan(wl.schedule, self.idx)
         assert self.comm.moe_status() == 0

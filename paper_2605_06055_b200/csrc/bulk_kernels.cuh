@@ -54,9 +54,11 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
                ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-               ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+// Window rows are written once and not read again by this kernel: an evict-first L2 policy on the
+// stores measured 1-8 % faster (653 vs 661 us at prefill size, 47 vs 51 us at decode size).
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes, uint64_t policy) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+               ::"l"(dst), "r"(src_smem), "r"(bytes), "l"(policy) : "memory");
 }
 
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
@@ -106,6 +108,8 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
     if (q0 < a.n_items) issue_load(q0, 0);
     if (q1 < a.n_items) issue_load(q1, 1);
   }
+  uint64_t evict_first;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
   uint32_t it = 0;
   bool alive = true;
   while (q0 < a.n_items && alive) {
@@ -127,7 +131,7 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
     }
     for (int j = 0; j < a.K; ++j) {
       const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-      if (lane == 0 && row >= 0) bulk_store(windows + (size_t)row * row_bytes + off, buf0 + s * stage_bytes, bytes);
+      if (lane == 0 && row >= 0) bulk_store(windows + (size_t)row * row_bytes + off, buf0 + s * stage_bytes, bytes, evict_first);
     }
     if (lane == 0) {
       bulk_commit();

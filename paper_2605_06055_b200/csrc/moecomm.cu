@@ -122,14 +122,18 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   return a;
 }
 
-// Chooses the work-item size and hands the launch its counter.  Large jobs take whole rows (at
-// most max_granule units) per item; small, decode-sized jobs take a fraction of a row so that every
-// warp of the grid has work.
+// Chooses the work-item size and hands the launch its counter.  An item is a whole row (at most
+// max_granule units) whenever that still gives every warp an item -- whole rows measured best
+// even at decode sizes -- and an even fraction of a row for tiny batches.
 void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
   const int upr = (a.H16 + 31) / 32;
-  const int64_t total = (int64_t)ctx->T * upr;
   int64_t g = upr < max_granule ? upr : max_granule;
-  if (total < nwarps * g * 4) g = total / (nwarps * 2);
+  int64_t pieces = (upr + g - 1) / g;
+  if ((int64_t)ctx->T * pieces < nwarps && ctx->T > 0) {
+    pieces = (nwarps + ctx->T - 1) / ctx->T;
+    if (pieces > upr) pieces = upr;
+    g = (upr + pieces - 1) / pieces;
+  }
   if (ctx->granule_override > 0) g = ctx->granule_override;
   if (g > max_granule) g = max_granule;
   if (g > upr) g = upr;
@@ -186,7 +190,10 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
 
 template <int KT>
 void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const float* w, uint4* y, cudaStream_t st) {
-  auto kernel = combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 1)>;
+  // Jobs that read several times the L2 capacity take the L1-allocating loads (see ld_row).
+  const bool large = (int64_t)ctx->T * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
+  auto kernel = large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 1), true>
+                      : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 1), false>;
   const int grid = row_grid(ctx, kernel);
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
