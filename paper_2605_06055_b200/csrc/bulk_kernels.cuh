@@ -17,7 +17,8 @@
 
 namespace moe {
 
-constexpr int BULK_WARPS = 4;
+constexpr int BULK_MAX_WARPS = 8;      // warps per CTA: as many 3-stage rings as fit in BULK_SMEM_BUDGET
+constexpr int BULK_SMEM_BUDGET = 200 * 1024;
 constexpr int BULK_STAGES = 3;
 constexpr int BULK_MAX_GRANULE = 32;   // a stage holds at most 16 KB of one row
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
@@ -70,19 +71,19 @@ __device__ __forceinline__ void bulk_wait_read() {
 
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// Dynamic shared memory: [BULK_WARPS][BULK_STAGES][stage_bytes] payload, then
-// [BULK_WARPS][BULK_STAGES] mbarriers.  stage_bytes = granule * 512.
-__global__ void __launch_bounds__(BULK_WARPS * 32)
+// Dynamic shared memory: [warps][BULK_STAGES][stage_bytes] payload, then
+// [warps][BULK_STAGES] mbarriers.  stage_bytes = granule * 512; warps = blockDim.x / 32.
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32)
 dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows, const RowArgs a,
                      const __grid_constant__ RankMap map) {
   extern __shared__ __align__(128) unsigned char smem[];
   begin_work(a);
   if (must_abort(a)) return;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t stage_bytes = (uint32_t)a.granule * 512u;
   const uint32_t row_bytes = (uint32_t)a.H16 * 16u;
   const uint32_t buf0 = smem_addr(smem) + warp * BULK_STAGES * stage_bytes;
-  const uint32_t bar0 = smem_addr(smem) + BULK_WARPS * BULK_STAGES * stage_bytes + warp * BULK_STAGES * 8;
+  const uint32_t bar0 = smem_addr(smem) + n_warps * BULK_STAGES * stage_bytes + warp * BULK_STAGES * 8;
 
   if (lane == 0) {
 #pragma unroll

@@ -177,15 +177,21 @@ void launch_dispatch_regs(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   kernel<<<grid, 256, 0, st>>>(x, win, b, ctx->map);
 }
 
-// Bulk-copy path: one CTA of BULK_WARPS warps per SM, a ring of BULK_STAGES stages per warp.
+// Bulk-copy path: one CTA per SM; each warp drives a ring of BULK_STAGES stages, and the CTA has as
+// many warps (up to BULK_MAX_WARPS) as fit their rings into the shared-memory budget: 4 for 14 KB
+// rows, 8 for rows of 8 KB or less (short rows need more requests in flight to cover the latency).
 void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
   const int upr = (a.H16 + 31) / 32;
+  const int g_max = upr < BULK_MAX_GRANULE ? upr : BULK_MAX_GRANULE;
+  int warps = BULK_SMEM_BUDGET / (BULK_STAGES * (g_max * 512 + 8));
+  if (warps > BULK_MAX_WARPS) warps = BULK_MAX_WARPS;
+  if (warps < 1) warps = 1;
   const int grid = ctx->num_sms;
   RowArgs b = a;
-  set_work(ctx, b, (int64_t)grid * BULK_WARPS, upr < BULK_MAX_GRANULE ? upr : BULK_MAX_GRANULE);
-  const int smem = BULK_WARPS * BULK_STAGES * (b.granule * 512 + 8);
-  dispatch_bulk_kernel<<<grid, BULK_WARPS * 32, smem, st>>>(reinterpret_cast<const unsigned char*>(x),
-                                                          reinterpret_cast<unsigned char*>(win), b, ctx->map);
+  set_work(ctx, b, (int64_t)grid * warps, g_max);
+  const int smem = warps * BULK_STAGES * (b.granule * 512 + 8);
+  dispatch_bulk_kernel<<<grid, warps * 32, smem, st>>>(reinterpret_cast<const unsigned char*>(x),
+                                                     reinterpret_cast<unsigned char*>(win), b, ctx->map);
 }
 
 template <int KT>
@@ -249,7 +255,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   bool ok = cudaMemset(ctx->ctl, 0, sizeof(Control)) == cudaSuccess;
   if (ok)
     ok = cudaFuncSetAttribute(dispatch_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              BULK_WARPS * BULK_STAGES * (BULK_MAX_GRANULE * 512 + 8)) == cudaSuccess;
+                              BULK_SMEM_BUDGET + 1024) == cudaSuccess;
   if (ok) {
     const int wide = 33 * shape->E * (int)sizeof(int32_t), narrow = 9 * shape->E * (int)sizeof(int32_t);
     if (shape->E <= RANK_PLAN_WIDE_MAX_E && wide > 48 * 1024)
