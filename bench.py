@@ -56,6 +56,8 @@ WORKLOADS = {
     "c3": lambda: synth.config(3),
     "c4": lambda: synth.config(4),
     "c5": lambda: synth.config(5, 65536, synth.PREFILL),
+    # a top-k degree without a specialised kernel (K = 7): exercises the any-K paths
+    "k7": lambda: synth.Workload("k7_prefill", 16384, 7168, 256, 8, 7, synth.PREFILL, "uniform", "identity", 1007),
     # c3 at a quarter of the tokens: the same kernels and row size, sized for ncu captures (about 1.2 GB resident)
     "c3s": lambda: synth.Workload("c3_prefill_dsv3_T8192", 8192, 7168, 256, 8, 8, synth.PREFILL, "uniform",
                                   "identity", 1003),
@@ -427,6 +429,26 @@ def run_cuda(args, wl):
             "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3,
         }
         del dl, flush
+        torch.cuda.empty_cache()
+
+    if world == 1 and args.workload == "c5" and not args.no_decode:
+        # config 5: both schedules timed at each T of the sweep (per-call medians, L2 flushed between steps)
+        line["sweep"] = []
+        flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+        for T in (128, 1024, 8192, 65536):
+            for sch in (synth.PREFILL, synth.DECODE):
+                swl = synth.config(5, T, sch)
+                sl = Layer(swl, dev)
+                sr = time_steps(sl, 50, 5, barrier, flush)
+                sk = kernel_table(swl, sr, peak)
+                line["sweep"].append({"T": T, "schedule": "prefill" if sch == synth.PREFILL else "decode",
+                                      "plan_us": sk["moe_plan"]["us"], "dispatch_us": sk["moe_dispatch"]["us"],
+                                      "combine_us": sk["moe_combine"]["us"],
+                                      "dispatch_GBps": sk["moe_dispatch"]["GBps"],
+                                      "combine_GBps": sk["moe_combine"]["GBps"],
+                                      "bytes_per_call": bytes_dispatch(swl)})
+                del sl
+        del flush
         torch.cuda.empty_cache()
 
     if world == 1 and not args.no_cpu_baseline:

@@ -198,8 +198,8 @@ template <int KT>
 void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const float* w, uint4* y, cudaStream_t st) {
   // Jobs that read several times the L2 capacity take the L1-allocating loads (see ld_row).
   const bool large = (int64_t)ctx->T * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
-  auto kernel = large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 1), true>
-                      : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 1), false>;
+  auto kernel = large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), true>
+                      : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), false>;
   const int grid = row_grid(ctx, kernel);
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * 8, 1 << 20);

@@ -242,17 +242,40 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
         }
       }
     } else {
-      for (int i = wi.i0; i < wi.i1; ++i) {
-        const int c = i * 32 + lane;
-        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int j = 0; j < K; ++j) {
-          const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-          const float w = __shfl_sync(0xffffffffu, w_lane, j);
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (row >= 0 && c < H16) v = ld_row<L1_ALLOC>(windows + (size_t)row * H16 + c);
-          fma_bf16x8(acc, w, v);
+      // Any K <= 32: branches are taken eight at a time, still in ascending j, so the fma chain
+      // is the same; UNROLL x 8 loads are in flight per lane.
+      for (int i = wi.i0; i < wi.i1; i += UNROLL) {   // warp-uniform trip counts: shuffles stay convergent
+        float acc[UNROLL][8];
+        bool ok[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          ok[u] = (i + u < wi.i1) && ((i + u) * 32 + lane < H16);
+#pragma unroll
+          for (int x = 0; x < 8; ++x) acc[u][x] = 0.f;
         }
-        if (c < H16) out[c] = pack_bf16x8(acc);
+        for (int jc = 0; jc < K; jc += 8) {
+          uint4 v[UNROLL][8];
+          float wv[8];
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) {
+            const int j = jc + jj;
+            const int64_t row = __shfl_sync(0xffffffffu, slot, j & 31);
+            wv[jj] = __shfl_sync(0xffffffffu, w_lane, j & 31);
+            const uint4* src = (j < K && row >= 0) ? windows + (size_t)row * H16 : nullptr;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u)
+              v[u][jj] = (ok[u] && src != nullptr) ? ld_row<L1_ALLOC>(src + (i + u) * 32 + lane)
+                                                   : make_uint4(0, 0, 0, 0);
+          }
+#pragma unroll
+          for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj)
+              if (jc + jj < K) fma_bf16x8(acc[u], wv[jj], v[u][jj]);
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+          if (ok[u]) out[(i + u) * 32 + lane] = pack_bf16x8(acc[u]);
       }
     }
   }
