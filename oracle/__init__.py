@@ -48,6 +48,12 @@ def lib() -> ctypes.CDLL:
         L.oracle_dispatch.argtypes = [p, i32, i32, i32, p, p, i32]
         L.oracle_expert_scale.argtypes = [p, i32, i32, i32, i64, p, p]
         L.oracle_combine.argtypes = [p, i32, i32, i32, p, p, p, i32]
+        L.oracle_dispatch_quant.argtypes = [p, i32, i32, i32, p, p, p, i32]
+        L.oracle_dispatch_quant.restype = ctypes.c_int
+        L.oracle_float_to_e4m3.argtypes = [ctypes.c_float]
+        L.oracle_float_to_e4m3.restype = ctypes.c_uint8
+        L.oracle_e4m3_to_float.argtypes = [ctypes.c_uint8]
+        L.oracle_e4m3_to_float.restype = ctypes.c_float
         L.oracle_float_to_bf16.argtypes = [ctypes.c_float]
         L.oracle_float_to_bf16.restype = ctypes.c_uint16
         L.oracle_bf16_to_float.argtypes = [ctypes.c_uint16]
@@ -117,6 +123,25 @@ def dispatch(X_u16, slots_, windows_u16, n_threads: int = 1) -> int:
     K = slots_.shape[1] if slots_.ndim == 2 else 1
     assert windows_u16.dtype == np.uint16 and windows_u16.flags["C_CONTIGUOUS"]
     return lib().oracle_dispatch(_ptr(X_u16), T, H, K, _ptr(slots_), _ptr(windows_u16), n_threads)
+
+
+def dispatch_quant(X_u16, slots_, windows_q, scales, n_threads: int = 1) -> int:
+    """Quantise rows of X [T,H] to e4m3 with one fp32 scale per row and scatter codes + scales."""
+    X_u16 = _c(X_u16, np.uint16)
+    slots_ = _c(slots_, np.int64)
+    T, H = X_u16.shape
+    K = slots_.shape[1]
+    assert windows_q.dtype == np.uint8 and windows_q.flags["C_CONTIGUOUS"]
+    assert scales.dtype == np.float32 and scales.flags["C_CONTIGUOUS"]
+    return lib().oracle_dispatch_quant(_ptr(X_u16), T, H, K, _ptr(slots_), _ptr(windows_q), _ptr(scales), n_threads)
+
+
+def float_to_e4m3(x: float) -> int:
+    return int(lib().oracle_float_to_e4m3(float(np.float32(x))))
+
+
+def e4m3_to_float(c: int) -> float:
+    return float(lib().oracle_e4m3_to_float(int(c)))
 
 
 def expert_scale(windows_u16, H: int, E: int, R: int, C: int, n_exp, scale_u16) -> int:

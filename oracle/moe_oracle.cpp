@@ -72,6 +72,56 @@ uint16_t oracle_float_to_bf16(float f) {
   return (uint16_t)(u >> 16);
 }
 
+float oracle_e4m3_to_float(uint8_t c) {
+  const int sign = c >> 7, exp = (c >> 3) & 15, man = c & 7;
+  float v;
+  if (exp == 15 && man == 7) v = std::nanf("");
+  else if (exp == 0) v = std::ldexp((float)man, -9);             // subnormal: man * 2^-9
+  else v = std::ldexp(1.0f + (float)man / 8.0f, exp - 7);
+  return sign ? -v : v;
+}
+
+uint8_t oracle_float_to_e4m3(float f) {
+  if (std::isnan(f)) return 0x7f;
+  const uint8_t sign = std::signbit(f) ? 0x80 : 0x00;
+  const float a = std::fabs(f);
+  if (a >= 448.0f) return sign | 0x7e;                            // clamp to the largest finite value
+  if (a < std::ldexp(1.0f, -6)) {                                 // subnormal range: multiples of 2^-9
+    const int q = (int)std::nearbyint(std::ldexp(a, 9));          // exact scaling, ties to even
+    return sign | (uint8_t)q;                                     // q == 8 is the smallest normal
+  }
+  int e = std::ilogb(a);                                          // a = m * 2^e, m in [1,2)
+  int q = (int)std::nearbyint(std::ldexp(a, 3 - e)) - 8;          // (m - 1) * 8, ties to even
+  if (q == 8) { q = 0; ++e; }
+  const int code = ((e + 7) << 3) | q;
+  return sign | (uint8_t)(code > 0x7e ? 0x7e : code);
+}
+
+int oracle_dispatch_quant(const uint16_t* X, int32_t T, int32_t H, int32_t K, const int64_t* slots,
+                          uint8_t* windows_q, float* scales, int32_t n_threads) {
+  if (T < 0 || H < 1 || K < 1) return ORACLE_ERR_INVALID_ARG;
+  for_token_ranges(T, n_threads, [=](int32_t lo, int32_t hi) {
+    std::vector<uint8_t> code((size_t)H);
+    for (int32_t t = lo; t < hi; ++t) {
+      const uint16_t* x = X + (int64_t)t * H;
+      float amax = 0.0f;
+      for (int32_t h = 0; h < H; ++h) amax = std::fmax(amax, std::fabs(oracle_bf16_to_float(x[h])));
+      float scale = 1.0f, inv = 1.0f;
+      if (amax > 0.0f) {
+        scale = amax / 448.0f;
+        inv = 448.0f / amax;
+      }
+      for (int32_t h = 0; h < H; ++h) code[h] = oracle_float_to_e4m3(oracle_bf16_to_float(x[h]) * inv);
+      for (int32_t j = 0; j < K; ++j) {
+        const int64_t row = slots[(int64_t)t * K + j];
+        std::memcpy(windows_q + row * H, code.data(), (size_t)H);
+        scales[row] = scale;
+      }
+    }
+  });
+  return ORACLE_OK;
+}
+
 int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
                 const int32_t* rank_tok_start,
                 int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,

@@ -78,6 +78,22 @@ int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int6
 int oracle_combine(const uint16_t* windows, int32_t T, int32_t H, int32_t K,
                    const int64_t* slots, const float* W, uint16_t* Y, int32_t n_threads);
 
+/* Row-wise quantised dispatch (Section 5.2, Prefill Dispatch: "if row-wise quantization is enabled,
+ * the corresponding scale values are written into a parallel scale tensor in the same row order").
+ * The paper fixes no format; the reading taken here is fp8 e4m3 (1-4-3, bias 7, largest finite value
+ * 448, no infinities) with one fp32 scale per row:
+ *   amax  = max_h |float(X[t,h])|
+ *   scale = amax / 448.0f, inv = 448.0f / amax    (fp32, round to nearest; both 1.0f if amax == 0)
+ *   code[t,h] = e4m3_rne_sat(float(X[t,h]) * inv) (fp32 product, then round to nearest even, clamped to +-448)
+ * and every branch (t,j) gets the same code row and the same scale at window row slot[t,j]:
+ *   windows_q [rows, H] uint8,  scales [rows] fp32.   A consumer reads x ~ e4m3_to_float(code) * scale. */
+int oracle_dispatch_quant(const uint16_t* X, int32_t T, int32_t H, int32_t K, const int64_t* slots,
+                          uint8_t* windows_q, float* scales, int32_t n_threads);
+
+/* e4m3 conversions used above, exported so that tests can pin them against a library conversion. */
+uint8_t oracle_float_to_e4m3(float f);
+float oracle_e4m3_to_float(uint8_t c);
+
 /* bf16 <-> fp32 conversions used above, exported so that tests can pin them
  * against a library conversion.  Round to nearest, ties to even; NaN stays NaN. */
 uint16_t oracle_float_to_bf16(float f);

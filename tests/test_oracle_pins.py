@@ -438,3 +438,73 @@ def test_benchmark_routing_recipes():
     p = oracle.plan(idx.numpy(), wl.E, wl.R)
     assert p.n_exp.max() >= 10 * wl.B / wl.E                     # hot experts hold > 10x the mean load
     assert (np.diff(np.sort(idx.numpy(), 1), axis=1) > 0).all()
+
+
+# ----------------------------------------------------------------------------- quantised dispatch
+def test_e4m3_conversions_against_torch():
+    # decoding: all 256 codes against torch's float8_e4m3fn
+    codes = torch.arange(256, dtype=torch.int32).to(torch.uint8)
+    want = codes.view(torch.float8_e4m3fn).float().numpy()
+    for c in range(256):
+        got = oracle.e4m3_to_float(c)
+        assert (np.isnan(got) and np.isnan(want[c])) or got == want[c], c
+    # encoding: every representable value, every midpoint between neighbours, and random values in [-448, 448]
+    finite = np.sort(np.unique(want[np.isfinite(want)]))
+    mids = (finite[:-1].astype(np.float64) + finite[1:].astype(np.float64)) / 2
+    rng = np.random.default_rng(3)
+    vals = np.concatenate([finite, mids.astype(np.float32), np.nextafter(mids.astype(np.float32), np.float32(1e9)),
+                           np.nextafter(mids.astype(np.float32), np.float32(-1e9)),
+                           rng.uniform(-448, 448, 20000).astype(np.float32),
+                           (rng.standard_normal(20000) * 0.01).astype(np.float32)]).astype(np.float32)
+    ref = torch.from_numpy(vals).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    for v, r in zip(vals, ref):
+        got = oracle.float_to_e4m3(v)
+        if v == 0:
+            assert got & 0x7F == 0
+        else:
+            assert got == r, (v, got, r)
+    # beyond the largest finite value the conversion clamps (it never produces NaN from a finite input)
+    for v in (448.0, 449.0, 463.9, 464.0, 480.0, 1e9, np.inf):
+        assert oracle.float_to_e4m3(v) == 0x7E and oracle.float_to_e4m3(-v) == 0xFE
+    assert oracle.float_to_e4m3(float("nan")) & 0x7F == 0x7F
+
+
+@pytest.mark.parametrize("T,K,E,R,H", [(40, 2, 8, 4, 64), (77, 8, 16, 2, 256)])
+def test_dispatch_quant_against_torch_pipeline_and_error_bound(T, K, E, R, H):
+    rng = np.random.default_rng(T)
+    idx, rts = random_case(rng, T, K, E, R)
+    X = rand_bf16(rng, (T, H))
+    X[3] = 0                                          # an all-zero row: scale 1, codes 0
+    X[5, 7] = synth.bf16_to_u16(torch.tensor([300.0]).to(torch.bfloat16))[0]     # a row with an outlier
+    p = oracle.plan(idx, E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(idx, E, R, p, C, rts)
+    wq = np.full((R * C, H), 0xAB, np.uint8)
+    sc = np.full((R * C,), -1.0, np.float32)
+    assert oracle.dispatch_quant(X, slots, wq, sc) == oracle.OK
+
+    # the same pipeline with library ops: fp32 amax, two fp32 divisions, fp32 product, torch's e4m3 rounding
+    xf = torch.from_numpy(u16_to_float(X))
+    amax = xf.abs().amax(dim=1)
+    scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+    # (scalar / tensor would be reciprocal-then-multiply in torch: two roundings; divide tensor by tensor)
+    inv = torch.where(amax > 0, torch.full_like(amax, 448.0) / amax, torch.ones_like(amax))
+    codes = (xf * inv[:, None]).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    owner = np.full(R * C, -1)
+    owner[slots.reshape(-1)] = np.repeat(np.arange(T), K)
+    for row in range(R * C):
+        t = owner[row]
+        if t < 0:
+            assert (wq[row] == 0xAB).all() and sc[row] == -1.0          # untouched
+        else:
+            assert np.array_equal(wq[row] & 0x7F != 0, codes[t] & 0x7F != 0)
+            nz = codes[t] & 0x7F != 0
+            assert np.array_equal(wq[row][nz], codes[t][nz]) and sc[row] == scale[t].item()
+    # the largest element of every non-zero row maps to the largest code, and the round trip is within the
+    # format's error: half an ulp of a 3-bit mantissa (2^-4 relative) or half a subnormal step of the scaled row
+    deq = torch.from_numpy(wq[slots[:, 0]]).view(torch.float8_e4m3fn).float() * torch.from_numpy(sc[slots[:, 0]])[:, None]
+    err = (deq - xf).abs()
+    bound = xf.abs() * 2.0 ** -4 * (1 + 1e-5) + scale[:, None] * 2.0 ** -10 * (1 + 1e-5)
+    assert bool((err <= bound).all())
+    top = (wq[slots[:, 0]] & 0x7F).max(1)
+    assert (top[amax.numpy() > 0] == 0x7E).all() and top[3] == 0
