@@ -119,6 +119,20 @@ moe_status_t moe_plan_view(const moe_ctx_t* ctx, moe_plan_view_t* out /*HOST*/);
 moe_status_t moe_dispatch(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows /*DEVICE*/,
                           int64_t capacity_rows, void* stream);
 
+/* Row-wise quantised dispatch (Section 5.2, Prefill Dispatch: with row-wise quantisation the scale
+ * values go to a parallel scale tensor in the same row order).  The paper names no format; this
+ * library's definition is fp8 e4m3 (1-4-3, bias 7, largest finite 448, no infinities) with one fp32
+ * scale per row:  amax = max_h |x[t,h]|,  scale = amax / 448,  inv = 448 / amax  (fp32, round to
+ * nearest; both 1 when amax == 0),  code[h] = e4m3_round_nearest_even_saturating(x[t,h] * inv).
+ * Every branch (t,j) receives the same code row and scale at window row slot(t,j); a consumer
+ * reconstructs x ~ e4m3_to_float(code) * scale.  Inputs must be finite.
+ *   x          DEVICE [T,H] bf16, 16-byte aligned; H % 16 == 0 and H <= 16384
+ *   windows_q  DEVICE [R, capacity_rows, H] uint8 (e4m3 codes), 16-byte aligned
+ *   scales     DEVICE [R, capacity_rows] fp32
+ * Errors and untouched padding rows as in moe_dispatch. */
+moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows_q /*DEVICE*/,
+                                float* scales /*DEVICE*/, int64_t capacity_rows, void* stream);
+
 /* Combine (Algorithm 1 / Algorithm 2, second loop; Section 5.2 Prefill Combine):
  *   Y[t,h] = bf16_rne( sum_{j=0..K-1} W[t,j] * float(windows[slot(t,j), h]) )
  * accumulated in fp32 from +0 with one fused multiply-add per term, j ascending.

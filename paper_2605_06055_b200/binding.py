@@ -24,7 +24,7 @@ MOE_SCHED_PREFILL, MOE_SCHED_DECODE = 0, 1
 EXPORTS = [
     "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
-    "moe_slots_noalloc", "moe_set_option",
+    "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE = 0, 1
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -66,6 +66,8 @@ def load() -> ctypes.CDLL:
     L.moe_plan_view.argtypes = [vp, ctypes.POINTER(MoePlanView)]
     L.moe_dispatch.argtypes = [vp, vp, vp, i64, vp]
     L.moe_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.moe_dispatch_quant.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.moe_dispatch_quant.restype = ctypes.c_int
     L.moe_slots.argtypes = [vp, i64, vp, vp]
     L.moe_forward_host.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     L.moe_status.argtypes = [vp, vp]
@@ -193,6 +195,16 @@ class MoeComm:
                                        int(capacity_rows), _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_dispatch")
+        return rc
+
+    def moe_dispatch_quant(self, x: torch.Tensor, windows_q: torch.Tensor, scales: torch.Tensor, capacity_rows: int,
+                           stream=None, check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_dispatch_quant(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(windows_q, torch.uint8),
+                                             _dev_ptr(scales, torch.float32), int(capacity_rows),
+                                             _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_quant")
         return rc
 
     def moe_combine(self, windows: torch.Tensor, capacity_rows: int, topk_w: torch.Tensor, y: torch.Tensor,

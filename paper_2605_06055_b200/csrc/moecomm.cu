@@ -11,6 +11,7 @@
 #include "plan_kernels.cuh"
 #include "row_kernels.cuh"
 #include "bulk_kernels.cuh"
+#include "quant_kernels.cuh"
 
 using namespace moe;
 
@@ -256,6 +257,9 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   if (ok)
     ok = cudaFuncSetAttribute(dispatch_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               BULK_SMEM_BUDGET + 1024) == cudaSuccess;
+  if (ok)
+    ok = cudaFuncSetAttribute(dispatch_quant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              BULK_SMEM_BUDGET + 1024) == cudaSuccess;
   if (ok) {
     const int wide = 33 * shape->E * (int)sizeof(int32_t), narrow = 9 * shape->E * (int)sizeof(int32_t);
     if (shape->E <= RANK_PLAN_WIDE_MAX_E && wide > 48 * 1024)
@@ -402,6 +406,36 @@ moe_status_t moe_dispatch(moe_ctx_t* c, const void* x, void* windows, int64_t ca
       default: launch_dispatch_regs<0>(ctx, a, xs, win, st); break;
     }
   }
+  return launch_ok(ctx);
+}
+
+moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, float* scales, int64_t capacity_rows,
+                                void* stream) {
+  moe_ctx* ctx = c;
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  const int H = ctx->shape.H;
+  if (H % 16 != 0 || H * 2 > QUANT_MAX_ROW_BYTES) return MOE_ERR_INVALID_ARG;
+  if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || windows_q == nullptr || scales == nullptr)))
+    return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(windows_q) || (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)
+    return MOE_ERR_INVALID_ARG;
+  RowArgs a = row_args(ctx, capacity_rows, true);
+  a.topk_idx = ctx->topk_idx;
+  // One work item per token: the whole row is needed for its scale.
+  const int upr = (a.H16 + 31) / 32;
+  const int stage = ((H * 2 + 127) / 128 + (H + 127) / 128) * 128;
+  int warps = BULK_SMEM_BUDGET / (QUANT_STAGES * (stage + 8));
+  if (warps > BULK_MAX_WARPS) warps = BULK_MAX_WARPS;
+  if (warps < 1) return MOE_ERR_INVALID_ARG;
+  const int grid = ctx->num_sms;
+  const int32_t keep = ctx->granule_override;
+  ctx->granule_override = upr;
+  set_work(ctx, a, (int64_t)grid * warps, upr);
+  ctx->granule_override = keep;
+  const int smem = warps * QUANT_STAGES * (stage + 8);
+  dispatch_quant_kernel<<<grid, warps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
   return launch_ok(ctx);
 }
 

@@ -1,0 +1,155 @@
+// Row-wise quantised dispatch: bf16 rows in, fp8 e4m3 codes + one fp32 scale per
+// row out, written straight into the destination expert windows and a parallel
+// scale tensor in the same row order (Section 5.2, Prefill Dispatch).
+//
+// Format (the paper names none; this is the library's definition):
+//   amax  = max_h |x[h]|                         (inputs are finite)
+//   scale = amax / 448, inv = 448 / amax         (fp32, round to nearest; 1 and 1 when amax == 0)
+//   code[h] = e4m3( x[h] * inv )                 (fp32 product, round to nearest even, clamped to +-448)
+// Each token is quantised once; its K branches receive the same code row and scale.
+//
+// Structure: the bulk-copy ring of dispatch_bulk_kernel with a compute step in
+// the middle.  A stage holds one whole row (needed for amax) plus its code row.
+// Lane 0 loads the row with cp.async.bulk; the warp reduces amax and converts
+// from shared memory into the stage's code buffer; lane 0 stores the code row K
+// times with cp.async.bulk while lanes j < K store the scale.  X is read from
+// HBM once and only H + 4 bytes per branch are written.
+#pragma once
+
+#include <cuda_fp8.h>
+
+#include "bulk_kernels.cuh"
+
+namespace moe {
+
+constexpr int QUANT_STAGES = 2;
+constexpr int QUANT_MAX_ROW_BYTES = 32 * 1024;
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t lo, uint32_t hi) {
+  asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(addr), "r"(lo), "r"(hi) : "memory");
+}
+
+// Two bf16 values packed in one word -> two e4m3 codes (low half first).
+__device__ __forceinline__ uint32_t quant_pair(uint32_t two_bf16, float inv) {
+  float2 f;
+  f.x = __fmul_rn(__uint_as_float(two_bf16 << 16), inv);
+  f.y = __fmul_rn(__uint_as_float(two_bf16 & 0xffff0000u), inv);
+  return (uint32_t)__nv_cvt_float2_to_fp8x2(f, __NV_SATFINITE, __NV_E4M3);
+}
+
+// Dynamic shared memory: [warps][QUANT_STAGES] stages of (in_stride + out_stride) bytes, then
+// [warps][QUANT_STAGES] mbarriers.  in_stride / out_stride: row bytes / code-row bytes rounded up to 128.
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32)
+dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
+                      float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  begin_work(a);
+  if (must_abort(a)) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  const uint32_t row_bytes = (uint32_t)a.H16 * 16u;          // bf16 row
+  const uint32_t code_bytes = (uint32_t)a.H16 * 8u;          // e4m3 row
+  const uint32_t in_stride = (row_bytes + 127u) & ~127u, out_stride = (code_bytes + 127u) & ~127u;
+  const uint32_t stage_stride = in_stride + out_stride;
+  const uint32_t buf0 = smem_addr(smem) + warp * QUANT_STAGES * stage_stride;
+  const uint32_t bar0 = smem_addr(smem) + n_warps * QUANT_STAGES * stage_stride + warp * QUANT_STAGES * 8;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < QUANT_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  auto issue_load = [&](int32_t token, int s) {   // lane 0 only
+    mbar_expect_tx(bar0 + 8 * s, row_bytes);
+    bulk_load(buf0 + s * stage_stride, X + (size_t)token * row_bytes, row_bytes, bar0 + 8 * s);
+  };
+
+  uint64_t evict_first;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
+
+  // One work item = one token row (items_per_row == 1).  q0 is consumed now, q1 is loading.
+  int32_t q0 = fetch_item(a);
+  int32_t q1 = fetch_item(a);
+  if (lane == 0) {
+    if (q0 < a.n_items) issue_load(q0, 0);
+    if (q1 < a.n_items) issue_load(q1, 1 % QUANT_STAGES);
+  }
+  uint32_t it = 0;
+  while (q0 < a.n_items) {
+    const int32_t q2 = fetch_item(a);
+    const int s = it % QUANT_STAGES;
+    const uint32_t parity = (it / QUANT_STAGES) & 1u;
+    const int64_t slot = resolve_slot(a, map, q0, lane, true);   // overlaps the load in flight
+    const uint32_t in = buf0 + s * stage_stride, out = in + in_stride;
+
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) {
+      if (lane == 0) raise_status(a.status, MOE_ERR_TIMEOUT);
+      break;
+    }
+
+    // amax: |bf16| patterns order like the values, so a per-halfword unsigned max of the
+    // sign-cleared words is the maximum magnitude.
+    uint32_t m2 = 0;
+    for (int c = lane; c < a.H16; c += 32) {
+      const uint4 v = lds128(in + c * 16);
+      m2 = __vmaxu2(m2, v.x & 0x7fff7fffu);
+      m2 = __vmaxu2(m2, v.y & 0x7fff7fffu);
+      m2 = __vmaxu2(m2, v.z & 0x7fff7fffu);
+      m2 = __vmaxu2(m2, v.w & 0x7fff7fffu);
+    }
+    uint32_t mbits = max(m2 & 0xffffu, m2 >> 16);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mbits = max(mbits, __shfl_xor_sync(0xffffffffu, mbits, d));
+    const float amax = __uint_as_float(mbits << 16);
+    float scale = 1.0f, inv = 1.0f;
+    if (amax > 0.0f) {
+      scale = __fdiv_rn(amax, 448.0f);
+      inv = __fdiv_rn(448.0f, amax);
+    }
+
+    // The code buffer of this stage was last read by the stores of item it - QUANT_STAGES: allow only
+    // the QUANT_STAGES - 1 younger store groups to be still reading before it is overwritten.
+    if (lane == 0) bulk_wait_read<QUANT_STAGES - 1>();
+    __syncwarp();
+    for (int c = lane; c < a.H16; c += 32) {
+      const uint4 v = lds128(in + c * 16);
+      const uint32_t lo = quant_pair(v.x, inv) | (quant_pair(v.y, inv) << 16);
+      const uint32_t hi = quant_pair(v.z, inv) | (quant_pair(v.w, inv) << 16);
+      sts64(out + c * 8, lo, hi);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // code row: generic writes -> bulk-copy reads
+    __syncwarp();
+
+    for (int j = 0; j < a.K; ++j) {
+      const int64_t row = __shfl_sync(0xffffffffu, slot, j);
+      if (lane == 0 && row >= 0) bulk_store(windows_q + (size_t)row * code_bytes, out, code_bytes, evict_first);
+    }
+    if (lane < a.K && slot >= 0) scales[slot] = scale;
+    if (lane == 0) {
+      bulk_commit();
+      // The row buffer of this stage is free again (every lane has read it): refill it.
+      if (QUANT_STAGES == 2) {
+        if (q2 < a.n_items) issue_load(q2, s);
+      } else {
+        if (q2 < a.n_items) issue_load(q2, (it + 2) % QUANT_STAGES);
+      }
+    }
+    q0 = q1;
+    q1 = q2;
+    ++it;
+  }
+  if (lane == 0) bulk_wait_all();
+}
+
+}  // namespace moe

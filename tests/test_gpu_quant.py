@@ -1,0 +1,89 @@
+"""Row-wise quantised dispatch on the GPU against the CPU oracle.
+
+Codes are bytes and the scale comes from two IEEE fp32 divisions of the same
+operands on both sides, so everything is compared bit for bit: e4m3 code rows,
+fp32 scales, and the untouched padding rows / scale slots.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06055_b200 import binding, synth
+from paper_2605_06055_b200.synth import DECODE, PREFILL, Workload
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # name, T, H, E, R, K, schedule, routing, rank_tokens
+    ("c2_decode_full", 2048, 7168, 256, 16, 8, DECODE, "uniform", None),
+    ("c3_reduced", 2048, 7168, 256, 8, 8, PREFILL, "uniform", None),
+    ("mixtral_like", 1024, 4096, 8, 8, 2, PREFILL, "uniform", None),
+    ("H16_min", 300, 16, 16, 4, 4, PREFILL, "uniform", None),
+    ("ragged_units", 123, 1008, 16, 2, 6, DECODE, "uniform", (23, 100)),
+    ("K5_dups_empty_rank", 250, 528, 10, 5, 5, PREFILL, "replace", (1, 100, 49, 0, 100)),
+    ("max_row", 64, 16384, 8, 2, 2, DECODE, "uniform", None),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_quantised_dispatch_bit_exact(case):
+    name, T, H, E, R, K, sch, routing, per = case
+    dev = torch.device("cuda:0")
+    wl = Workload(name, T, H, E, R, K, sch, routing, "identity", 5000 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    X = inp.X.clone()
+    X[T // 3] = 0                                     # an all-zero row
+    X[T // 2, H // 2] = 3.0e4                         # an outlier: the rest of that row lands in the subnormal codes
+    X[1, 0] = -0.0
+    idx_np = inp.topk_idx.numpy()
+    p = oracle.plan(idx_np, E, R, inp.rank_tok_start)
+    C = int(p.n_recv.max()) + 2
+    _, slots = oracle.slots(idx_np, E, R, p, C, inp.rank_tok_start)
+    want_q = np.full((R * C, H), 0xAB, np.uint8)
+    want_s = np.full((R * C,), -1.0, np.float32)
+    assert oracle.dispatch_quant(synth.bf16_to_u16(X), slots, want_q, want_s, 4) == oracle.OK
+
+    comm = binding.MoeComm(T, H, E, R, K, dev)
+    rts = None if per is None else inp.rank_tok_start
+    comm.moe_plan(sch, inp.topk_idx.to(dev), T, rts)
+    wq = torch.full((R * C, H), 0xAB, dtype=torch.uint8, device=dev)
+    sc = torch.full((R * C,), -1.0, dtype=torch.float32, device=dev)
+    comm.moe_dispatch_quant(X.to(dev), wq, sc, C)
+    assert comm.moe_status() == 0
+    assert np.array_equal(wq.cpu().numpy(), want_q)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+    if sch == DECODE:                                 # the launch also records delta, like moe_dispatch
+        assert np.array_equal(comm.moe_plan_view()["small_off"].cpu().numpy(), p.s)
+    # a consumer's view: dequantised rows are within the format's error of the bf16 rows
+    deq = wq[torch.from_numpy(slots[:, 0]).to(dev)].view(torch.float8_e4m3fn).float() * \
+        sc[torch.from_numpy(slots[:, 0]).to(dev)][:, None]
+    xf = X.to(dev).float()
+    scale = xf.abs().amax(1) / 448.0
+    assert bool(((deq - xf).abs() <= xf.abs() * 2.0 ** -4 * 1.00001 + scale[:, None] * 2.0 ** -10 * 1.00001).all())
+    comm.close()
+
+
+def test_quantised_dispatch_errors():
+    dev = torch.device("cuda:0")
+    comm = binding.MoeComm(64, 24, 8, 2, 2, dev)      # H % 16 != 0
+    idx = torch.zeros((64, 2), dtype=torch.int32, device=dev)
+    comm.moe_plan(PREFILL, idx)
+    x = torch.zeros((64, 24), dtype=torch.bfloat16, device=dev)
+    wq = torch.zeros((2 * 128, 24), dtype=torch.uint8, device=dev)
+    sc = torch.zeros((2 * 128,), dtype=torch.float32, device=dev)
+    assert comm.moe_dispatch_quant(x, wq, sc, 128, check=False) == binding.MOE_ERR_INVALID_ARG
+    comm.close()
+    comm = binding.MoeComm(64, 32, 8, 2, 2, dev)
+    x = torch.ones((64, 32), dtype=torch.bfloat16, device=dev)
+    wq = torch.full((2 * 128, 32), 0xAB, dtype=torch.uint8, device=dev)
+    sc = torch.full((2 * 128,), -1.0, dtype=torch.float32, device=dev)
+    assert comm.moe_dispatch_quant(x, wq, sc, 128, check=False) == binding.MOE_ERR_NOT_PLANNED
+    comm.moe_plan(PREFILL, idx)                        # all 128 branches go to expert 0 of rank 0
+    comm.moe_dispatch_quant(x, wq, sc, 127)            # one row short
+    assert comm.moe_status() == binding.MOE_ERR_CAPACITY
+    assert bool((wq == 0xAB).all()) and bool((sc == -1.0).all())
+    comm.moe_dispatch_quant(x, wq, sc, 128)
+    assert comm.moe_status() == 0
+    assert bool((wq[:128] == 0x7E).all()) and bool((sc[:128] == 1.0 / 448.0).all()) and bool((wq[128:] == 0xAB).all())
+    comm.close()
