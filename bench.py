@@ -80,6 +80,11 @@ def bytes_plan(wl) -> int:
     return 8 * wl.T * wl.K + 8 * wl.E * wl.R
 
 
+def bytes_dispatch_quant(wl) -> int:
+    # read each bf16 row once; per branch write H e4m3 codes and one fp32 scale; same metadata as dispatch
+    return 2 * wl.H * wl.T + wl.K * wl.T * (wl.H + 4) + 8 * wl.T * wl.K + 4 * wl.E * wl.R
+
+
 def bytes_step(wl) -> int:
     return bytes_plan(wl) + bytes_dispatch(wl) + bytes_combine(wl)
 
@@ -292,6 +297,25 @@ def time_steps(layer: Layer, steps: int, warmup: int, barrier, scratch=None):
     }
 
 
+def time_dispatch_quant(layer: Layer, steps: int, scratch=None):
+    """The row-wise quantised variant of dispatch (e4m3 codes + fp32 scale per row), same plan."""
+    wl = layer.wl
+    wq = torch.zeros((wl.R * layer.C, wl.H), dtype=torch.uint8, device=layer.dev)
+    sc = torch.zeros((wl.R * layer.C,), dtype=torch.float32, device=layer.dev)
+    for _ in range(3):
+        layer.comm.moe_dispatch_quant(layer.X, wq, sc, layer.C)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        if scratch is not None:
+            scratch.add_(1)
+        a.record()
+        layer.comm.moe_dispatch_quant(layer.X, wq, sc, layer.C)
+        b.record()
+    torch.cuda.synchronize()
+    assert layer.comm.moe_status() == 0
+    return [a.elapsed_time(b) * 1e3 for a, b in ev]
+
+
 def time_graph_steps(layer: Layer, steps: int, scratch=None):
     """The same step captured once in a CUDA graph and replayed (what a decode loop would do)."""
     g = torch.cuda.CUDAGraph()
@@ -375,6 +399,9 @@ def run_cuda(args, wl):
     sampler.start()
     r = time_steps(layer, args.steps, args.warmup, barrier, scratch)
     ms_per_step = reduce_max_over_ranks(r["ms_per_step"], dist, dev)
+    quant_us = None
+    if wl.H % 16 == 0 and not args.no_decode:
+        quant_us = time_dispatch_quant(layer, min(args.steps, 50), scratch)
     e2e = None
     if not args.no_e2e:
         e2e_steps = max(3, min(args.steps, 10))
@@ -390,6 +417,12 @@ def run_cuda(args, wl):
 
     peak, peak_kind = measured_peak()
     kernels = kernel_table(wl, r, peak)
+    if quant_us is not None:
+        gbps = bytes_dispatch_quant(wl) / (sum(quant_us) / len(quant_us)) / 1e3
+        kernels["moe_dispatch_quant"] = {"us": statistics.median(quant_us), "us_min": min(quant_us),
+                                         "bytes": bytes_dispatch_quant(wl), "GBps": gbps,
+                                         "frac_of_measured_peak": gbps / peak, "frac_of_8TBps": gbps / NOMINAL_HBM_GBS,
+                                         "note": "row-wise e4m3 + fp32 scale variant of dispatch; not part of the step"}
     dom = "moe_dispatch" if sum(r["dispatch_us"]) >= sum(r["combine_us"]) else "moe_combine"
     dom_kernel = "dispatch_bulk_kernel" if dom == "moe_dispatch" else "combine_rows_kernel"
     roofline = {"bound": "hbm", "kernel": dom_kernel, "achieved": kernels[dom]["GBps"], "peak": peak,
