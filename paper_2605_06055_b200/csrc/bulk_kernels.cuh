@@ -103,8 +103,9 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
   };
 
   // Items in flight: q0 is consumed this iteration, q1 is loading, q2 is fetched now.
-  int32_t q0 = fetch_item(a);
-  int32_t q1 = fetch_item(a);
+  ItemFeed feed = begin_feed();
+  int32_t q0 = fetch_item(a, feed);
+  int32_t q1 = fetch_item(a, feed);
   if (lane == 0) {
     if (q0 < a.n_items) issue_load(q0, 0);
     if (q1 < a.n_items) issue_load(q1, 1);
@@ -114,7 +115,7 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
   uint32_t it = 0;
   bool alive = true;
   while (q0 < a.n_items && alive) {
-    const int32_t q2 = fetch_item(a);
+    const int32_t q2 = fetch_item(a, feed);
     const int s = it % BULK_STAGES;
     const uint32_t parity = (it / BULK_STAGES) & 1u;
     const WorkItem w = decode_item(a, q0);

@@ -132,7 +132,8 @@ __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ 
   const int E_r = E / R;
   for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
     int32_t acc = 0;
-    for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);
+#pragma unroll 16
+    for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);   // independent loads: keep many in flight
     nexp_s[e] = acc;
     n_exp[e] = acc;
   }
@@ -143,6 +144,7 @@ __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ 
   for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
     const int d = e / E_r;
     int32_t run = pre_s[e] - pre_s[d * E_r];
+#pragma unroll 16
     for (int rr = 0; rr < R; ++rr) {
       o[(size_t)e * R + rr] = run;
       run += __ldcg(M + (size_t)rr * E + e);
@@ -153,6 +155,7 @@ __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ 
     for (int i = threadIdx.x; i < R * R; i += (int)blockDim.x) {
       const int rr = i / R, d = i % R;
       int32_t acc = 0;
+#pragma unroll 16
       for (int e = d * E_r; e < (d + 1) * E_r; ++e) acc += __ldcg(M + (size_t)rr * E + e);
       c_rank[i] = acc;
     }
@@ -172,7 +175,7 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
 
   for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
     int32_t run = 0;
-#pragma unroll 4
+#pragma unroll 16
     for (int t = t0; t < t1; ++t) {
       const size_t at = (size_t)t * E + e;
       const int32_t c = tile_hist[at];

@@ -76,15 +76,16 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
 
   // One work item = one token row (items_per_row == 1).  q0 is consumed now, q1 is loading.
-  int32_t q0 = fetch_item(a);
-  int32_t q1 = fetch_item(a);
+  ItemFeed feed = begin_feed();
+  int32_t q0 = fetch_item(a, feed);
+  int32_t q1 = fetch_item(a, feed);
   if (lane == 0) {
     if (q0 < a.n_items) issue_load(q0, 0);
     if (q1 < a.n_items) issue_load(q1, 1 % QUANT_STAGES);
   }
   uint32_t it = 0;
   while (q0 < a.n_items) {
-    const int32_t q2 = fetch_item(a);
+    const int32_t q2 = fetch_item(a, feed);
     const int s = it % QUANT_STAGES;
     const uint32_t parity = (it / QUANT_STAGES) & 1u;
     const int64_t slot = resolve_slot(a, map, q0, lane, true);   // overlaps the load in flight

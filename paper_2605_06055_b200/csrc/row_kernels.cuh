@@ -85,8 +85,8 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 // Work partition shared by dispatch and combine.  A "unit" is one 512-byte
 // column slab of one token row (32 lanes x 16 bytes).  A row is cut into
 // items_per_row work items of `granule` units (the last may be shorter); the job
-// is T * items_per_row items.  Warps take items from an atomic counter, fetching
-// the next one while the current one is processed, so a warp that the memory
+// is T * items_per_row items.  Warps take items from an atomic counter (after two
+// fixed first items), fetching the next one while the current one is processed, so a warp that the memory
 // system serves slowly simply takes fewer items: no wave quantisation at prefill
 // sizes, full-GPU parallelism at decode sizes, no static tail.  Which warp moves
 // which bytes does not affect the result.  The counter is one of two used
@@ -100,10 +100,32 @@ __device__ __forceinline__ void begin_work(const RowArgs& a) {
   if (blockIdx.x == 0 && threadIdx.x == 0) *a.work_next = 0;
 }
 
-__device__ __forceinline__ int32_t fetch_item(const RowArgs& a) {
-  int32_t v = 0;
-  if ((threadIdx.x & 31) == 0) v = atomicAdd(a.work, 1);
-  return __shfl_sync(0xffffffffu, v, 0);
+// Hands a warp its work items: the first two are fixed (warp id, warp id + number of warps), so no
+// warp waits on an atomic before its first bytes move; every later one comes from the counter.
+struct ItemFeed {
+  int64_t gid, nwarps;
+  int32_t taken;
+};
+
+__device__ __forceinline__ ItemFeed begin_feed() {
+  ItemFeed f;
+  f.nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  f.gid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  f.taken = 0;
+  return f;
+}
+
+__device__ __forceinline__ int32_t fetch_item(const RowArgs& a, ItemFeed& f) {
+  int64_t item;
+  if (f.taken < 2) {
+    item = f.gid + f.taken * f.nwarps;
+  } else {
+    int32_t v = 0;
+    if ((threadIdx.x & 31) == 0) v = atomicAdd(a.work, 1);
+    item = 2 * f.nwarps + __shfl_sync(0xffffffffu, v, 0);
+  }
+  ++f.taken;
+  return (int32_t)min(item, (int64_t)a.n_items);
 }
 
 __device__ __forceinline__ WorkItem decode_item(const RowArgs& a, int32_t item) {
@@ -130,9 +152,10 @@ dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, c
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
 
-  int32_t item = fetch_item(a);
+  ItemFeed feed = begin_feed();
+  int32_t item = fetch_item(a, feed);
   while (item < a.n_items) {
-    const int32_t next_item = fetch_item(a);   // in flight while this item is processed
+    const int32_t next_item = fetch_item(a, feed);   // in flight while this item is processed
     const WorkItem w = decode_item(a, item);
     item = next_item;
     const int64_t slot = resolve_slot(a, map, w.t, lane, w.i0 == 0);   // the owner of the row start records delta
@@ -205,9 +228,10 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
 
-  int32_t item = fetch_item(a);
+  ItemFeed feed = begin_feed();
+  int32_t item = fetch_item(a, feed);
   while (item < a.n_items) {
-    const int32_t next_item = fetch_item(a);
+    const int32_t next_item = fetch_item(a, feed);
     const WorkItem wi = decode_item(a, item);
     item = next_item;
     const int64_t slot = resolve_slot(a, map, wi.t, lane, false);
