@@ -146,6 +146,14 @@ moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows /*DEVICE*/, int64_t
  * consumers).  slots DEVICE [T,K] int32; needs R * capacity_rows < 2^31. */
 moe_status_t moe_slots(moe_ctx_t* ctx, int64_t capacity_rows, int32_t* slots /*DEVICE*/, void* stream);
 
+/* Row range of every expert in the window allocation, for the expert side (Section 5.2, Expert
+ * computation: the FFNs consume the windows in place, with no further reordering, so the rows of one
+ * expert are one contiguous run -- exactly a grouped-GEMM problem list).  Works under both schedules.
+ *   row_start  DEVICE [E] int64   first window row of expert e ( = dst(e) * capacity_rows + o[e, 0] )
+ *   row_count  DEVICE [E] int32   rows received by expert e */
+moe_status_t moe_expert_ranges(moe_ctx_t* ctx, int64_t capacity_rows, int64_t* row_start /*DEVICE*/,
+                               int32_t* row_count /*DEVICE*/, void* stream);
+
 /* One whole layer call from HOST buffers, enqueued on `stream`:
  * host->device copies of x, topk_idx, topk_w; plan; dispatch; combine reading
  * the dispatched windows (identity experts); device->host copy of y.

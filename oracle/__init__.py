@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_dispatch.argtypes = [p, i32, i32, i32, p, p, i32]
         L.oracle_expert_scale.argtypes = [p, i32, i32, i32, i64, p, p]
         L.oracle_combine.argtypes = [p, i32, i32, i32, p, p, p, i32]
+        L.oracle_expert_ranges.argtypes = [i32, i32, i64, p, p, p]
+        L.oracle_expert_ranges.restype = ctypes.c_int
         L.oracle_dispatch_quant.argtypes = [p, i32, i32, i32, p, p, p, i32]
         L.oracle_dispatch_quant.restype = ctypes.c_int
         L.oracle_float_to_e4m3.argtypes = [ctypes.c_float]
@@ -113,6 +115,14 @@ def slots(topk_idx, E: int, R: int, pl: Plan, C: int, rank_tok_start=None):
     st = lib().oracle_slots(_ptr(topk_idx), T, K, E, R, _ptr(rts), _ptr(pl.s), _ptr(pl.o), _ptr(pl.n_recv),
                             int(C), _ptr(out))
     return st, out
+
+
+def expert_ranges(E: int, R: int, C: int, n_exp):
+    n_exp = _c(n_exp, np.int32)
+    start = np.full((E,), -1, np.int64)
+    count = np.full((E,), -1, np.int32)
+    st = lib().oracle_expert_ranges(E, R, int(C), _ptr(n_exp), _ptr(start), _ptr(count))
+    return st, start, count
 
 
 def dispatch(X_u16, slots_, windows_u16, n_threads: int = 1) -> int:

@@ -199,6 +199,21 @@ int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32
   return ORACLE_OK;
 }
 
+int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, const int32_t* n_exp,
+                         int64_t* row_start, int32_t* row_count) {
+  if (E < 1 || R < 1 || E % R != 0 || C < 0) return ORACLE_ERR_INVALID_ARG;
+  const int32_t E_r = E / R;
+  for (int32_t d = 0; d < R; ++d) {
+    int64_t row = (int64_t)d * C;
+    for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) {
+      row_start[e] = row;
+      row_count[e] = n_exp[e];
+      row += n_exp[e];
+    }
+  }
+  return ORACLE_OK;
+}
+
 int oracle_dispatch(const uint16_t* X, int32_t T, int32_t H, int32_t K,
                     const int64_t* slots, uint16_t* windows, int32_t n_threads) {
   if (T < 0 || H < 1 || K < 1) return ORACLE_ERR_INVALID_ARG;

@@ -57,6 +57,13 @@ int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32
                  const int32_t* rank_tok_start, const int32_t* s, const int32_t* o,
                  const int32_t* n_recv, int64_t C, int64_t* slots);
 
+/* Row range of every expert inside the window allocation: the expert FFNs consume the windows in
+ * place, without further reordering (Section 5.2, Expert computation), so each expert's rows are one
+ * contiguous run:  row_start[e] = dst(e) * C + (rows of earlier experts of the same rank),
+ * row_count[e] = n_exp[e]. */
+int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, const int32_t* n_exp,
+                         int64_t* row_start, int32_t* row_count);
+
 /* Dispatch (Algorithm 1, first loop): copy row X[t,:] to window row slot[t,j]
  * for every branch.  Rows no branch maps to are left as the caller set them.
  * n_threads > 1 splits the token range over std::thread workers (same result). */

@@ -24,7 +24,7 @@ MOE_SCHED_PREFILL, MOE_SCHED_DECODE = 0, 1
 EXPORTS = [
     "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
-    "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant",
+    "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE = 0, 1
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -66,6 +66,8 @@ def load() -> ctypes.CDLL:
     L.moe_plan_view.argtypes = [vp, ctypes.POINTER(MoePlanView)]
     L.moe_dispatch.argtypes = [vp, vp, vp, i64, vp]
     L.moe_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.moe_expert_ranges.argtypes = [vp, i64, vp, vp, vp]
+    L.moe_expert_ranges.restype = ctypes.c_int
     L.moe_dispatch_quant.argtypes = [vp, vp, vp, vp, i64, vp]
     L.moe_dispatch_quant.restype = ctypes.c_int
     L.moe_slots.argtypes = [vp, i64, vp, vp]
@@ -205,6 +207,15 @@ class MoeComm:
                                              _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_dispatch_quant")
+        return rc
+
+    def moe_expert_ranges(self, capacity_rows: int, row_start: torch.Tensor, row_count: torch.Tensor, stream=None,
+                          check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_expert_ranges(self._h, int(capacity_rows), _dev_ptr(row_start, torch.int64),
+                                            _dev_ptr(row_count, torch.int32), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_expert_ranges")
         return rc
 
     def moe_combine(self, windows: torch.Tensor, capacity_rows: int, topk_w: torch.Tensor, y: torch.Tensor,

@@ -479,6 +479,16 @@ moe_status_t moe_slots(moe_ctx_t* c, int64_t capacity_rows, int32_t* slots, void
   return launch_ok(ctx);
 }
 
+moe_status_t moe_expert_ranges(moe_ctx_t* ctx, int64_t capacity_rows, int64_t* row_start, int32_t* row_count,
+                               void* stream) {
+  if (ctx == nullptr || row_start == nullptr || row_count == nullptr || capacity_rows < 0) return MOE_ERR_INVALID_ARG;
+  if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  const int E = ctx->shape.E;
+  expert_ranges_kernel<<<(E + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      ctx->o, ctx->n_exp, E, ctx->shape.R, capacity_rows, row_start, row_count);
+  return launch_ok(ctx);
+}
+
 moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T, const int32_t* rank_tok_start,
                               const void* x_host, const int32_t* topk_idx_host, const float* topk_w_host,
                               void* x_dev, int32_t* topk_idx_dev, float* topk_w_dev, void* windows_dev,

@@ -324,4 +324,17 @@ slots_kernel(int32_t* __restrict__ slots, const RowArgs a, const __grid_constant
   }
 }
 
+// ---------------------------------------------------------------- expert ranges
+// Grouped-GEMM style descriptors for the expert side: expert e owns window rows
+// [row_start[e], row_start[e] + row_count[e]) -- the block of source rank 0 starts the expert's run.
+__global__ void __launch_bounds__(256)
+expert_ranges_kernel(const int32_t* __restrict__ large_off, const int32_t* __restrict__ n_exp, int32_t E, int32_t R,
+                     int64_t C, int64_t* __restrict__ row_start, int32_t* __restrict__ row_count) {
+  const int E_r = E / R;
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < E; e += gridDim.x * blockDim.x) {
+    row_start[e] = (int64_t)(e / E_r) * C + large_off[(size_t)e * R];
+    row_count[e] = n_exp[e];
+  }
+}
+
 }  // namespace moe

@@ -84,6 +84,8 @@ class GpuRun:
     windows: np.ndarray  # after dispatch, before the expert op
     Y: np.ndarray
     statuses: list
+    expert_start: np.ndarray = None
+    expert_count: np.ndarray = None
 
 
 def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Optional[binding.MoeComm] = None,
@@ -105,6 +107,9 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
     statuses.append(comm.moe_status())
     slots = torch.full((wl.T, wl.K), -5, dtype=torch.int32, device=dev)
     comm.moe_slots(C, slots)
+    e_start = torch.full((wl.E,), -5, dtype=torch.int64, device=dev)
+    e_count = torch.full((wl.E,), -5, dtype=torch.int32, device=dev)
+    comm.moe_expert_ranges(C, e_start, e_count)
     windows = torch.from_numpy(np.full((wl.R * C, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
     comm.moe_dispatch(X, windows, C)
     statuses.append(comm.moe_status())
@@ -115,7 +120,8 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
     Y = torch.from_numpy(np.full((wl.T, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
     comm.moe_combine(windows, C, w, Y)
     statuses.append(comm.moe_status())
-    out = GpuRun(view, slots.cpu().numpy(), win_host, Y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), statuses)
+    out = GpuRun(view, slots.cpu().numpy(), win_host, Y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), statuses,
+                 e_start.cpu().numpy(), e_count.cpu().numpy())
     if own:
         comm.close()
     return out
@@ -130,6 +136,9 @@ def assert_parity(g: GpuRun, o: OracleRun, schedule: int, combine_ulp: int = 1):
             continue
         assert np.array_equal(g.view[k], getattr(o.plan, on)), k          # bit-exact integers
     assert np.array_equal(g.slots.astype(np.int64), o.slots)
+    E, R = o.plan.o.shape
+    st, want_start, want_count = oracle.expert_ranges(E, R, g.windows.shape[0] // R, o.plan.n_exp)
+    assert st == oracle.OK and np.array_equal(g.expert_start, want_start) and np.array_equal(g.expert_count, want_count)
     assert np.array_equal(g.windows, o.windows)                           # bit-exact rows and canaries
     ulp = max_ulp_diff(g.Y, o.Y)
     assert ulp <= combine_ulp, ulp

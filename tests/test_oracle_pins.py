@@ -180,6 +180,16 @@ def test_plan_against_library_routines(case):
     before = np.concatenate([[0], np.cumsum(p.n_recv)])[dst]   # branches bound for earlier ranks
     assert np.array_equal(slots.reshape(-1), dst * C + pos - before)
 
+    # Expert row ranges: the rows of [start, start+count) hold exactly the branches routed to that expert.
+    st, e_start, e_count = oracle.expert_ranges(E, R, C, p.n_exp)
+    assert st == oracle.OK
+    owner = np.full(R * C, -1)
+    owner[slots.reshape(-1)] = idx.reshape(-1)
+    for e in range(E):
+        assert e_count[e] == (idx == e).sum()
+        assert (owner[e_start[e]:e_start[e] + e_count[e]] == e).all()
+    assert e_count.sum() == T * K
+
     # Bijection onto the used part of each segment; each expert's rows contiguous.
     used = np.sort(slots.reshape(-1))
     want = np.concatenate([d * C + np.arange(p.n_recv[d]) for d in range(R)]) if T else np.zeros(0)
