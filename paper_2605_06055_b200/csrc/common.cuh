@@ -33,7 +33,8 @@ struct RankMap {
 struct Control {
   int32_t status;       // first device-detected error (moe_status_t), 0 = none
   int32_t scan_ticket;  // "last block done" counter of the offset scan
-  int32_t work[2];      // work-item counters of the row kernels, used alternately (see row_kernels.cuh)
+  int32_t work;         // work-item counter of the running row kernel (see row_kernels.cuh); zero between launches
+  int32_t work_done;    // warps of the running row kernel that have finished; zero between launches
   int32_t pad[60];
 };
 

@@ -33,7 +33,6 @@ struct moe_ctx {
   const int32_t* topk_idx;  // device; routing indexes of the current plan, read again by dispatch/combine
   RankMap map;
   int64_t launches;
-  int32_t work_parity;      // which of the two work-item counters the next row-kernel launch uses
   int32_t dispatch_path;    // MOE_OPT_DISPATCH_PATH
   int32_t granule_override; // MOE_OPT_GRANULE
 };
@@ -116,7 +115,7 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.E_r = sh.E / sh.R;
   a.H16 = sh.H / 8;
   a.work = nullptr;
-  a.work_next = nullptr;
+  a.work_done = nullptr;
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
@@ -143,9 +142,8 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
   a.granule = (int32_t)g;
   a.items_per_row = (int32_t)((upr + g - 1) / g);
   a.n_items = (int32_t)((int64_t)ctx->T * a.items_per_row);
-  a.work = &ctx->ctl->work[ctx->work_parity];
-  a.work_next = &ctx->ctl->work[ctx->work_parity ^ 1];
-  ctx->work_parity ^= 1;
+  a.work = &ctx->ctl->work;
+  a.work_done = &ctx->ctl->work_done;
 }
 
 // One persistent wave: as many CTAs as fit on the device at once (from the occupancy calculator),
@@ -247,7 +245,6 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->compact_plan = false;
   ctx->launches = 0;
   ctx->topk_idx = nullptr;
-  ctx->work_parity = 0;
   ctx->dispatch_path = MOE_DISPATCH_AUTO;
   ctx->granule_override = 0;
 
@@ -682,7 +679,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.E_r = E / R;
   a.H16 = 0;
   a.work = nullptr;
-  a.work_next = nullptr;
+  a.work_done = nullptr;
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;

@@ -49,8 +49,10 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32)
 dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
                       float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
   extern __shared__ __align__(128) unsigned char smem[];
-  begin_work(a);
-  if (must_abort(a)) return;
+  if (must_abort(a)) {
+    end_work(a);
+    return;
+  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t row_bytes = (uint32_t)a.H16 * 16u;          // bf16 row
   const uint32_t code_bytes = (uint32_t)a.H16 * 8u;          // e4m3 row
@@ -151,6 +153,7 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
     ++it;
   }
   if (lane == 0) bulk_wait_all();
+  end_work(a);
 }
 
 }  // namespace moe

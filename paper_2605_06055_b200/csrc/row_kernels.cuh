@@ -24,8 +24,8 @@ struct RowArgs {
   int64_t C;                 // rows per window segment
   int32_t T, K, E, R, E_r;
   int32_t H16;               // 16-byte chunks per row
-  int32_t* work;             // this launch's work-item counter (zero on entry)
-  int32_t* work_next;        // the next launch's counter, zeroed by this launch
+  int32_t* work;             // work-item counter (zero on entry, zeroed again by the last warp to finish)
+  int32_t* work_done;        // finished-warp counter (same)
   int32_t granule;           // units (512-byte slabs) per work item
   int32_t items_per_row;     // ceil(units per row / granule)
   int32_t n_items;           // T * items_per_row
@@ -89,15 +89,25 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 // fixed first items), fetching the next one while the current one is processed, so a warp that the memory
 // system serves slowly simply takes fewer items: no wave quantisation at prefill
 // sizes, full-GPU parallelism at decode sizes, no static tail.  Which warp moves
-// which bytes does not affect the result.  The counter is one of two used
-// alternately: each launch zeroes the one the next launch will use.
+// which bytes does not affect the result.  The last warp of a launch to finish
+// puts the counters back to zero, so every launch (eager, or replayed from a
+// CUDA graph any number of times) starts from a clean state with no memset.
 struct WorkItem {
   int32_t t;       // token
   int32_t i0, i1;  // unit range inside the row
 };
 
-__device__ __forceinline__ void begin_work(const RowArgs& a) {
-  if (blockIdx.x == 0 && threadIdx.x == 0) *a.work_next = 0;
+// Called by every warp on every exit path of a row kernel.
+__device__ __forceinline__ void end_work(const RowArgs& a) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) {
+    const int32_t nwarps = (int32_t)(gridDim.x * (blockDim.x >> 5));
+    __threadfence();                                   // this warp's item fetches come before its sign-off
+    if (atomicAdd(a.work_done, 1) == nwarps - 1) {     // everyone else has signed off: nobody fetches any more
+      *a.work = 0;
+      *a.work_done = 0;
+    }
+  }
 }
 
 // Hands a warp its work items: the first two are fixed (warp id, warp id + number of warps), so no
@@ -146,8 +156,10 @@ template <int KT, int UNROLL>
 __global__ void __launch_bounds__(256, 1)
 dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, const RowArgs a,
                      const __grid_constant__ RankMap map) {
-  begin_work(a);
-  if (must_abort(a)) return;
+  if (must_abort(a)) {
+    end_work(a);
+    return;
+  }
   const int lane = threadIdx.x & 31;
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
@@ -196,6 +208,7 @@ dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, c
       }
     }
   }
+  end_work(a);
 }
 
 // ---------------------------------------------------------------- combine
@@ -222,8 +235,10 @@ template <int KT, int UNROLL, bool L1_ALLOC>
 __global__ void __launch_bounds__(256, 1)
 combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__ topk_w, uint4* __restrict__ Y,
                     const RowArgs a, const __grid_constant__ RankMap map) {
-  begin_work(a);
-  if (must_abort(a)) return;
+  if (must_abort(a)) {
+    end_work(a);
+    return;
+  }
   const int lane = threadIdx.x & 31;
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
@@ -303,6 +318,7 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
       }
     }
   }
+  end_work(a);
 }
 
 // ---------------------------------------------------------------- slots

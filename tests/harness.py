@@ -58,6 +58,7 @@ class OracleRun:
     slots: np.ndarray
     windows: np.ndarray
     Y: np.ndarray
+    windows_zero_init: np.ndarray = None   # the same dispatch into zero-filled windows
 
 
 def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4) -> OracleRun:
@@ -74,7 +75,12 @@ def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4) -> OracleRun:
         assert oracle.expert_scale(win, wl.H, wl.E, wl.R, C, p.n_exp, synth.bf16_to_u16(inp.scale)) == oracle.OK
     st, Y = oracle.combine(win, slots, inp.topk_w.numpy(), wl.H, n_threads)
     assert st == oracle.OK
-    return OracleRun(p, slots, win_after_dispatch, Y)
+    zero_init = np.where(win_after_dispatch == CANARY, np.uint16(0), win_after_dispatch)
+    used = np.zeros(wl.R * C, bool)
+    used[slots.reshape(-1)] = True
+    zero_init = win_after_dispatch.copy()
+    zero_init[~used] = 0
+    return OracleRun(p, slots, win_after_dispatch, Y, zero_init)
 
 
 @dataclass

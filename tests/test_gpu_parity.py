@@ -282,3 +282,56 @@ def test_forward_host_entry_point():
         o = harness.oracle_run(inp, C)
         assert harness.max_ulp_diff(synth.bf16_to_u16(y_host), o.Y) <= 1
     comm.close()
+
+
+def test_cuda_graph_replays_and_eager_calls_mix_freely():
+    """The path is capturable (no allocation, no synchronisation, host arrays passed by value), and a
+    captured call can be replayed any number of times between eager calls: every launch leaves the
+    work counters as it found them."""
+    dev = torch.device("cuda:0")
+    wl = synth.config(2)
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max())
+    o = harness.oracle_run(Workload_identity(inp), C)
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
+    win = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
+    Y = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    comm.moe_plan(wl.schedule, idx)
+    comm.moe_dispatch(X, win, C)                 # warm-up outside capture
+    torch.cuda.synchronize()
+    g_dispatch, g_step = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_dispatch):
+        comm.moe_dispatch(X, win, C)
+    with torch.cuda.graph(g_step):
+        comm.moe_plan(wl.schedule, idx)
+        comm.moe_dispatch(X, win, C)
+        comm.moe_combine(win, C, w, Y)
+    for n_replays in (1, 3):                     # odd counts of a single captured launch
+        win.zero_()
+        for _ in range(n_replays):
+            g_dispatch.replay()
+        comm.moe_combine(win, C, w, Y)           # eager call right after
+        assert comm.moe_status() == 0
+        assert np.array_equal(win.cpu().view(torch.int16).numpy().view(np.uint16), o.windows_zero_init)
+        assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), o.Y) <= 1
+    Y.zero_()
+    win.zero_()
+    g_step.replay()
+    g_dispatch.replay()
+    g_step.replay()
+    assert comm.moe_status() == 0
+    assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), o.Y) <= 1
+    comm.close()
+
+
+class Workload_identity:
+    """Inputs of a workload with the expert op forced to identity and zero-initialised windows (for graphs)."""
+
+    def __new__(cls, inp):
+        import copy
+        import dataclasses
+        out = copy.copy(inp)
+        out.wl = dataclasses.replace(inp.wl, expert_op="identity")
+        return out
