@@ -51,7 +51,8 @@ typedef enum {
 } moe_status_t;
 
 /* The two schedules of Section 4.  PREFILL runs Layout + Notify as separate
- * planning passes and keeps the whole planning table readable.  DECODE keeps
+ * planning passes (folded into one launch when every source rank holds at most
+ * 4096 branches) and keeps the whole planning table readable.  DECODE keeps
  * only the compact state (o_dec, delta, n_recv); delta is produced inside the
  * dispatch launch (Section 5.3, Decode Dispatch), or already by the single
  * planning launch when every source rank holds at most 4096 branches. */

@@ -26,7 +26,7 @@ struct moe_ctx {
   int32_t *M, *c_rank, *o, *n_exp, *n_recv, *s, *tile_rank, *tile_hist;
   // plan state (host)
   bool planned;
-  bool compact_plan;  // DECODE plan done by plan_rank_kernel: small offsets are final after moe_plan
+  bool compact_plan;  // plan done in one launch by plan_rank_kernel: small offsets are final after moe_plan
   moe_schedule_t schedule;
   int32_t T;
   int32_t n_tiles;
@@ -39,7 +39,7 @@ struct moe_ctx {
 
 namespace {
 
-// DECODE plans whose ranks each hold at most this many branches take the single-launch planner.
+// Plans (either schedule) whose ranks each hold at most this many branches take the single-launch planner.
 constexpr int64_t RANK_PLAN_MAX_BRANCHES = 4096;
 constexpr int RANK_PLAN_WIDE_MAX_E = 768;   // 32-warp CTAs while 33*E counters fit comfortably in shared memory
 
@@ -333,15 +333,15 @@ moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk
     const int64_t br = (int64_t)(map.tok_start[r + 1] - map.tok_start[r]) * sh.K;
     if (br > max_rank_branches) max_rank_branches = br;
   }
-  ctx->compact_plan = !full && max_rank_branches <= RANK_PLAN_MAX_BRANCHES;
+  ctx->compact_plan = max_rank_branches <= RANK_PLAN_MAX_BRANCHES;
   int n = 0;
   if (ctx->compact_plan) {
     if (sh.E <= RANK_PLAN_WIDE_MAX_E)
       plan_rank_kernel<32><<<sh.R, 32 * 32, 33 * sh.E * (int)sizeof(int32_t), st>>>(
-          topk_idx, map, sh.K, sh.E, ctx->s, ctx->M, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     else
       plan_rank_kernel<8><<<sh.R, 8 * 32, 9 * sh.E * (int)sizeof(int32_t), st>>>(
-          topk_idx, map, sh.K, sh.E, ctx->s, ctx->M, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     ++n;
   } else {
     if (tiles > 0) {

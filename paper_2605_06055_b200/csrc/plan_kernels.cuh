@@ -18,7 +18,8 @@
 //                      (exclusive scan in window order: expert, then source rank).
 //   plan_finalize_kernel  PREFILL only: s = in-tile rank + tile base.
 //                      (DECODE folds this step into the dispatch launch.)
-//   plan_rank_kernel   DECODE with few branches per rank: the whole plan in one launch.
+//   plan_rank_kernel   few branches per rank (decode steps, small prefill chunks): the whole
+//                      plan in one launch, small offsets final at once.
 #pragma once
 
 #include "common.cuh"
@@ -197,15 +198,15 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
   if (threadIdx.x == 0) ctl->scan_ticket = 0;  // ready for the next plan on this stream
 }
 
-// Compact planner of the DECODE schedule when every source rank holds few branches: ONE launch, one
-// CTA per source rank.  The CTA walks its rank's branches in passes of WARPS*32, carrying the running
+// Compact planner for batches in which every source rank holds few branches (every decode step,
+// small prefill chunks): ONE launch, one CTA per source rank.  The CTA walks its rank's branches in passes of WARPS*32, carrying the running
 // per-expert count in shared memory, so the small offsets come out final (no tile bases), row r of M
 // falls out at the end, and the last CTA to finish builds the large offsets.
 template <int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
-                 int32_t* __restrict__ s, int32_t* __restrict__ M, int32_t* __restrict__ o,
-                 int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
+                 int32_t full_table, int32_t* __restrict__ s, int32_t* __restrict__ M, int32_t* __restrict__ c_rank,
+                 int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
   extern __shared__ int32_t sm[];   // [WARPS][E] per-warp counts, [E] running base  (reused: 2E+1 scan area)
   __shared__ int is_last;
   int32_t* warp_hist = sm;
@@ -255,7 +256,7 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  build_large_offsets(M, E, R, 0, nullptr, o, n_exp, n_recv, sm);
+  build_large_offsets(M, E, R, full_table, c_rank, o, n_exp, n_recv, sm);
   if (threadIdx.x == 0) ctl->scan_ticket = 0;
 }
 
