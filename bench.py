@@ -455,6 +455,9 @@ def run_cuda(args, wl):
         dr = time_steps(dl, 100, 5, barrier, flush)
         gk = kernel_table(dwl, dr, peak)
         graph_us = time_graph_steps(dl, 100, flush)
+        wr = time_steps(dl, 100, 5, barrier, None)            # back-to-back: whatever fits stays in L2
+        wk = kernel_table(dwl, wr, peak)
+        warm_graph_us = time_graph_steps(dl, 100, None)
         line["decode"] = {
             "config": describe(dwl), "l2": "256 MB L2 flush between steps (untimed)",
             "timer": "CUDA events tick in 2.05 us steps on this GPU, so per-call figures are means over 100 steps",
@@ -463,6 +466,10 @@ def run_cuda(args, wl):
             "step_us_cuda_graph": sum(graph_us) / len(graph_us),
             "dispatch_GBps": gk["moe_dispatch"]["GBps"], "combine_GBps": gk["moe_combine"]["GBps"],
             "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3,
+            "warm": {"l2": "back-to-back steps, no flush", "plan_us": wk["moe_plan"]["us_mean"],
+                     "dispatch_us": wk["moe_dispatch"]["us_mean"], "combine_us": wk["moe_combine"]["us_mean"],
+                     "step_us_stream_launches": wr["ms_per_step"] * 1e3,
+                     "step_us_cuda_graph": sum(warm_graph_us) / len(warm_graph_us)},
         }
         del dl, flush
         torch.cuda.empty_cache()

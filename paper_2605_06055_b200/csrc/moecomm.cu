@@ -258,11 +258,17 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
     ok = cudaFuncSetAttribute(dispatch_quant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               BULK_SMEM_BUDGET + 1024) == cudaSuccess;
   if (ok) {
-    const int wide = 33 * shape->E * (int)sizeof(int32_t), narrow = 9 * shape->E * (int)sizeof(int32_t);
-    if (shape->E <= RANK_PLAN_WIDE_MAX_E && wide > 48 * 1024)
-      ok = cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide) == cudaSuccess;
-    if (ok && shape->E > RANK_PLAN_WIDE_MAX_E && narrow > 48 * 1024)
-      ok = cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, narrow) == cudaSuccess;
+    const int rank_smem =
+        rank_plan_smem_ints(shape->E, shape->R, shape->E <= RANK_PLAN_WIDE_MAX_E ? 32 : 8) * (int)sizeof(int32_t);
+    const int scan_smem = notify_smem_ints(shape->E, shape->R) * (int)sizeof(int32_t);
+    if (rank_smem > 48 * 1024)
+      ok = (shape->E <= RANK_PLAN_WIDE_MAX_E
+                ? cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)
+                : cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)) ==
+           cudaSuccess;
+    if (ok && scan_smem > 48 * 1024)
+      ok = cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) ==
+           cudaSuccess;
   }
   if (ok && tile_smem > 48 * 1024) {
     ok = cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_PREFILL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -326,7 +332,9 @@ moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int tile_smem = PLAN_WARPS * sh.E * (int)sizeof(int32_t);
-  const int scan_smem = (2 * sh.E + 1) * (int)sizeof(int32_t);
+  const int scan_smem = notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t);
+  const int rank_smem =
+      rank_plan_smem_ints(sh.E, sh.R, sh.E <= RANK_PLAN_WIDE_MAX_E ? 32 : 8) * (int)sizeof(int32_t);
   const int full = schedule == MOE_SCHED_PREFILL;
   int64_t max_rank_branches = 0;
   for (int r = 0; r < sh.R; ++r) {
@@ -337,10 +345,10 @@ moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk
   int n = 0;
   if (ctx->compact_plan) {
     if (sh.E <= RANK_PLAN_WIDE_MAX_E)
-      plan_rank_kernel<32><<<sh.R, 32 * 32, 33 * sh.E * (int)sizeof(int32_t), st>>>(
+      plan_rank_kernel<32><<<sh.R, 32 * 32, rank_smem, st>>>(
           topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     else
-      plan_rank_kernel<8><<<sh.R, 8 * 32, 9 * sh.E * (int)sizeof(int32_t), st>>>(
+      plan_rank_kernel<8><<<sh.R, 8 * 32, rank_smem, st>>>(
           topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     ++n;
   } else {
@@ -661,7 +669,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   if (tiles > 0)
     plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, PLAN_WARPS * E * (int)sizeof(int32_t), st>>>(
         topk_idx, map, K, E, sc->tile_rank, sc->tile_hist, status);
-  plan_scan_kernel<<<R, PLAN_THREADS, (2 * E + 1) * (int)sizeof(int32_t), st>>>(
+  plan_scan_kernel<<<R, PLAN_THREADS, notify_smem_ints(E, R) * (int)sizeof(int32_t), st>>>(
       sc->tile_hist, map, E, 0, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl);
   RowArgs a;
   a.topk_idx = topk_idx;

@@ -79,12 +79,14 @@ plan_tile_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
 
   // Exclusive scan over the warps (warp w holds earlier branches than warp w+1).
   for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
+    int32_t c[PLAN_WARPS];
+#pragma unroll
+    for (int w = 0; w < PLAN_WARPS; ++w) c[w] = warp_hist[w * E + e];   // all loads before the first store
     int32_t run = 0;
 #pragma unroll
     for (int w = 0; w < PLAN_WARPS; ++w) {
-      const int32_t c = warp_hist[w * E + e];
       warp_hist[w * E + e] = run;
-      run += c;
+      run += c[w];
     }
     tile_hist[(size_t)tile * E + e] = run;
   }
@@ -97,70 +99,138 @@ plan_tile_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   }
 }
 
-// Exclusive scan of n (<= blockDim-independent) ints held in shared memory,
-// done by warp 0: each lane owns a contiguous chunk.  out[i] = sum of in[0..i-1],
-// out[n] = total.  `in` and `out` may not alias.
-__device__ __forceinline__ void warp0_exclusive_scan(const int32_t* in, int32_t* out, int n) {
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    const int chunk = (n + 31) / 32;
-    const int lo = min(lane * chunk, n), hi = min(lo + chunk, n);
-    int32_t sum = 0;
-    for (int i = lo; i < hi; ++i) sum += in[i];
-    int32_t incl = sum;
+// Exclusive scan of n ints in shared memory by the whole CTA (blockDim.x a multiple of 32, <= 1024).
+// out[i] = in[0] + .. + in[i-1], out[n] = total.  `in` and `out` may not alias; `warp_sums` holds 33 ints.
+__device__ __forceinline__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n, int32_t* warp_sums) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  int32_t carry = 0;
+  for (int base = 0; base < n; base += blockDim.x) {   // uniform trip count
+    const int i = base + threadIdx.x;
+    const int32_t v = i < n ? in[i] : 0;
+    int32_t incl = v;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-      const int32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += v;
+      const int32_t u = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += u;
     }
-    int32_t run = incl - sum;
-    for (int i = lo; i < hi; ++i) {
-      out[i] = run;
-      run += in[i];
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int32_t w = lane < nwarps ? warp_sums[lane] : 0;
+      int32_t wi = w;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int32_t u = __shfl_up_sync(0xffffffffu, wi, d);
+        if (lane >= d) wi += u;
+      }
+      warp_sums[lane] = wi - w;              // exclusive prefix of the warp totals
+      if (lane == 31) warp_sums[32] = wi;    // chunk total
     }
-    if (lane == 31) out[n] = incl;
+    __syncthreads();
+    if (i < n) out[i] = carry + warp_sums[warp] + incl - v;
+    carry += warp_sums[32];
+    __syncthreads();
   }
+  if (threadIdx.x == 0) out[n] = carry;
+}
+
+// Shared memory the Notify step needs: n_exp [E], prefix [E+1], warp sums [33], and, when the count
+// matrix is small enough to stage, M transposed and padded as [E][R+1].
+constexpr int NOTIFY_STAGE_MAX = 8192;   // entries of M staged in shared memory
+__host__ __device__ constexpr int notify_smem_ints(int E, int R) {
+  return 2 * E + 1 + 33 + (R * E <= NOTIFY_STAGE_MAX ? E * (R + 1) : 0);
 }
 
 // Notify step proper: turns the complete count matrix M into receive counts and large offsets.
-// Run by ONE CTA (the last to finish counting).  sm: 2*E + 1 ints of shared memory.
+// Run by ONE CTA (the last to finish counting).  sm: notify_smem_ints(E, R) ints of shared memory.
+//
+// Staged path (R*E <= NOTIFY_STAGE_MAX): M is read from L2 once, in one batch of independent
+// coalesced loads, into a transposed [E][R+1] tile (the odd row pitch keeps both the column walk of
+// one thread per expert and the final row-major copy free of bank conflicts); the prefix over source
+// ranks is formed in place and o leaves the SM as one coalesced stream.  A thread that stored its own
+// 16 offsets of 4 bytes at a 64-byte pitch would instead occupy the store path for one cycle per
+// 32-byte sector, which measured 2.9 us for 4096 offsets.
+// Direct path (large R*E): loads first and in batches; no store sits between two loads, because the
+// compiler cannot know that o and M never overlap and would serialise them at one L2 round trip each.
 __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ M, int32_t E, int32_t R,
                                                     int32_t full_table, int32_t* __restrict__ c_rank,
                                                     int32_t* __restrict__ o, int32_t* __restrict__ n_exp,
                                                     int32_t* __restrict__ n_recv, int32_t* sm) {
   int32_t* nexp_s = sm;
   int32_t* pre_s = sm + E;
-  const int E_r = E / R;
+  int32_t* warp_sums = sm + 2 * E + 1;
+  int32_t* tile = sm + 2 * E + 1 + 33;   // [E][R+1], staged path only
+  const int E_r = E / R, P = R + 1;
+  const bool staged = R * E <= NOTIFY_STAGE_MAX;
+  if (staged) {
+    for (int i0 = 0; i0 < R * E; i0 += 4 * (int)blockDim.x) {   // batches of independent loads
+      int32_t v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + k * (int)blockDim.x + (int)threadIdx.x;
+        v[k] = i < R * E ? __ldcg(M + i) : 0;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + k * (int)blockDim.x + (int)threadIdx.x;   // i = r*E + e
+        if (i < R * E) tile[(i % E) * P + i / E] = v[k];
+      }
+    }
+    __syncthreads();
+  }
   for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
     int32_t acc = 0;
+    if (staged) {
+      for (int rr = 0; rr < R; ++rr) acc += tile[e * P + rr];
+    } else {
 #pragma unroll 16
-    for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);   // independent loads: keep many in flight
+      for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);
+    }
     nexp_s[e] = acc;
     n_exp[e] = acc;
   }
   __syncthreads();
-  warp0_exclusive_scan(nexp_s, pre_s, E);
+  block_exclusive_scan(nexp_s, pre_s, E, warp_sums);
   __syncthreads();
   // Window of rank d = experts d*E_r ..; offsets restart at 0 in every window.
-  for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
-    const int d = e / E_r;
-    int32_t run = pre_s[e] - pre_s[d * E_r];
-#pragma unroll 16
-    for (int rr = 0; rr < R; ++rr) {
-      o[(size_t)e * R + rr] = run;
-      run += __ldcg(M + (size_t)rr * E + e);
-    }
-  }
-  for (int d = threadIdx.x; d < R; d += (int)blockDim.x) n_recv[d] = pre_s[(d + 1) * E_r] - pre_s[d * E_r];
-  if (full_table) {
+  if (full_table) {   // per-rank branch counts, before the staged tile is overwritten by the offsets
     for (int i = threadIdx.x; i < R * R; i += (int)blockDim.x) {
       const int rr = i / R, d = i % R;
       int32_t acc = 0;
 #pragma unroll 16
-      for (int e = d * E_r; e < (d + 1) * E_r; ++e) acc += __ldcg(M + (size_t)rr * E + e);
+      for (int e = d * E_r; e < (d + 1) * E_r; ++e) acc += staged ? tile[e * P + rr] : __ldcg(M + (size_t)rr * E + e);
       c_rank[i] = acc;
     }
+    __syncthreads();
   }
+  if (staged) {
+    for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
+      int32_t run = pre_s[e] - pre_s[(e / E_r) * E_r];
+      for (int rr = 0; rr < R; ++rr) {
+        const int32_t m = tile[e * P + rr];
+        tile[e * P + rr] = run;
+        run += m;
+      }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < E * R; i += (int)blockDim.x) o[i] = tile[(i / R) * P + i % R];   // coalesced
+  } else {
+    for (int e = threadIdx.x; e < E; e += (int)blockDim.x) {
+      int32_t run = pre_s[e] - pre_s[(e / E_r) * E_r];
+      for (int r0 = 0; r0 < R; r0 += 16) {
+        int32_t m[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) m[k] = r0 + k < R ? __ldcg(M + (size_t)(r0 + k) * E + e) : 0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+          if (r0 + k < R) {
+            o[(size_t)e * R + r0 + k] = run;
+            run += m[k];
+          }
+      }
+    }
+  }
+  for (int d = threadIdx.x; d < R; d += (int)blockDim.x) n_recv[d] = pre_s[(d + 1) * E_r] - pre_s[d * E_r];
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS)
@@ -168,7 +238,7 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
                  const __grid_constant__ RankMap map, int32_t E, int32_t full_table,
                  int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
                  int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
-  extern __shared__ int32_t sm[];  // [E] n_exp, [E+1] prefix
+  extern __shared__ int32_t sm[];  // notify_smem_ints(E, R) ints
   __shared__ int is_last;
   const int r = blockIdx.x;
   const int R = map.R;
@@ -176,12 +246,16 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
 
   for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
     int32_t run = 0;
-#pragma unroll 16
-    for (int t = t0; t < t1; ++t) {
-      const size_t at = (size_t)t * E + e;
-      const int32_t c = tile_hist[at];
-      tile_hist[at] = run;
-      run += c;
+    for (int tb = t0; tb < t1; tb += 16) {   // loads first, then the in-place stores (see build_large_offsets)
+      int32_t c[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) c[k] = (tb + k < t1) ? tile_hist[(size_t)(tb + k) * E + e] : 0;
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        if (tb + k < t1) {
+          tile_hist[(size_t)(tb + k) * E + e] = run;
+          run += c[k];
+        }
     }
     M[(size_t)r * E + e] = run;
   }
@@ -199,18 +273,27 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
 }
 
 // Compact planner for batches in which every source rank holds few branches (every decode step,
-// small prefill chunks): ONE launch, one CTA per source rank.  The CTA walks its rank's branches in passes of WARPS*32, carrying the running
-// per-expert count in shared memory, so the small offsets come out final (no tile bases), row r of M
-// falls out at the end, and the last CTA to finish builds the large offsets.
+// small prefill chunks): ONE launch, one CTA per source rank.  The CTA walks its rank's branches in
+// passes of WARPS*32, carrying the running per-expert count in shared memory, so the small offsets
+// come out final (no tile bases), row r of M falls out at the end, and the last CTA to finish
+// builds the large offsets.
+// Shared memory: counts [E][WARPS+1] (expert-major with an odd pitch: neither the leaders' scattered
+// writes -- same warp column, different experts -- nor the scanning warp's row reads collide on a
+// bank), running base [E]; reused by the Notify step at the end.
+__host__ __device__ constexpr int rank_plan_smem_ints(int E, int R, int warps) {
+  return (warps + 2) * E > notify_smem_ints(E, R) ? (warps + 2) * E : notify_smem_ints(E, R);
+}
+
 template <int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
                  int32_t full_table, int32_t* __restrict__ s, int32_t* __restrict__ M, int32_t* __restrict__ c_rank,
                  int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
-  extern __shared__ int32_t sm[];   // [WARPS][E] per-warp counts, [E] running base  (reused: 2E+1 scan area)
+  extern __shared__ int32_t sm[];
   __shared__ int is_last;
-  int32_t* warp_hist = sm;
-  int32_t* rank_base = sm + WARPS * E;
+  constexpr int P = WARPS + 1;
+  int32_t* counts = sm;             // [E][P]
+  int32_t* rank_base = sm + P * E;  // [E]
   const int r = blockIdx.x, R = map.R;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int32_t b_begin = map.tok_start[r] * K, b_end = map.tok_start[r + 1] * K;
@@ -218,8 +301,7 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
 
   for (int e = threadIdx.x; e < E; e += WARPS * 32) rank_base[e] = 0;
   for (int32_t pass = b_begin; pass < b_end; pass += WARPS * 32) {
-    for (int i = threadIdx.x; i < WARPS * E; i += WARPS * 32) warp_hist[i] = 0;
-    __syncthreads();
+    for (int i = threadIdx.x; i < P * E; i += WARPS * 32) counts[i] = 0;
     const int32_t b = pass + warp * 32 + lane;
     int32_t e = -1;
     if (b < b_end) {
@@ -230,21 +312,41 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
       }
     }
     const unsigned peers = __match_any_sync(0xffffffffu, e);
-    const int ahead = __popc(peers & lt);
-    if (e >= 0 && ahead == 0) warp_hist[warp * E + e] = __popc(peers);   // one round per pass: no carry inside a warp
+    const int ahead = __popc(peers & lt);           // equal keys in lower lanes = earlier branches
     __syncthreads();
-    for (int x = threadIdx.x; x < E; x += WARPS * 32) {
-      int32_t run = rank_base[x];
-#pragma unroll 8
-      for (int w = 0; w < WARPS; ++w) {
-        const int32_t c = warp_hist[w * E + x];
-        warp_hist[w * E + x] = run;
-        run += c;
+    if (e >= 0 && ahead == 0) counts[e * P + warp] = __popc(peers);   // one round per pass: no carry inside a warp
+    __syncthreads();
+    // Exclusive scan across the warps of every expert's counts, by shuffles: lane w holds warp w's
+    // count.  Four experts at a time, so four independent shuffle chains are in flight per warp.
+    for (int x0 = warp; x0 < E; x0 += 4 * WARPS) {   // warp-uniform trip count
+      int32_t c[4], incl[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int x = x0 + k * WARPS;
+        c[k] = (x < E && lane < WARPS) ? counts[x * P + lane] : 0;
+        incl[k] = c[k];
       }
-      rank_base[x] = run;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int32_t u = __shfl_up_sync(0xffffffffu, incl[k], d);
+          if (lane >= d) incl[k] += u;
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int x = x0 + k * WARPS;
+        if (x < E) {
+          const int32_t base = rank_base[x];
+          if (lane < WARPS) counts[x * P + lane] = base + incl[k] - c[k];
+          __syncwarp();
+          if (lane == 31) rank_base[x] = base + incl[k];
+        }
+      }
     }
     __syncthreads();
-    if (b < b_end) s[b] = e >= 0 ? warp_hist[warp * E + e] + ahead : 0;
+    if (b < b_end) s[b] = e >= 0 ? counts[e * P + warp] + ahead : 0;
     __syncthreads();
   }
   __syncthreads();
