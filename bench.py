@@ -360,6 +360,57 @@ def time_e2e(layer: Layer, steps: int, barrier):
     return t0.elapsed_time(t1) / steps, wl.T * wl.H * 2 + wl.T * wl.K * 8, wl.T * wl.H * 2
 
 
+def time_repeated(fns, n: int) -> float:
+    """Microseconds per repetition of calling every function in `fns` once, n repetitions bracketed by
+    ONE pair of CUDA events (event pairs around single ~10 us calls tick in ~2 us steps on this GPU)."""
+    for _ in range(3):
+        for f in fns:
+            f()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(n):
+        for f in fns:
+            f()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e3 / n
+
+
+def decode_latency(dev, peak, n: int = 200) -> dict:
+    """Decode-step latency (config 2).  Per-call figures are differences of cumulative sequences
+    (flush | flush+plan | flush+plan+dispatch | ...), each timed over n repetitions."""
+    dwl = synth.config(2)
+    dl = Layer(dwl, dev)
+    c = dl.comm
+    flush_buf = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    flush = lambda: flush_buf.add_(1)
+    plan = lambda: c.moe_plan(dwl.schedule, dl.idx)
+    disp = lambda: c.moe_dispatch(dl.X, dl.windows, dl.C)
+    comb = lambda: c.moe_combine(dl.windows, dl.C, dl.w, dl.Y)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        dl.step()
+    replay = lambda: g.replay()
+    out = {"config": describe(dwl),
+           "method": f"cumulative sequences of calls, {n} repetitions per pair of CUDA events; per-call = difference",
+           "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3}
+    for name, pre in (("cold", [flush]), ("warm", [])):
+        base = time_repeated(pre, n) if pre else 0.0
+        t1 = time_repeated(pre + [plan], n)
+        t2 = time_repeated(pre + [plan, disp], n)
+        t3 = time_repeated(pre + [plan, disp, comb], n)
+        tg = time_repeated(pre + [replay], n)
+        out[name] = {"l2": "256 MB L2 flush before every step (its time subtracted)" if pre else
+                     "back-to-back steps, no flush",
+                     "plan_us": t1 - base, "dispatch_us": t2 - t1, "combine_us": t3 - t2,
+                     "step_us_stream_launches": t3 - base, "step_us_cuda_graph": tg - base,
+                     "dispatch_GBps": bytes_dispatch(dwl) / (t2 - t1) / 1e3,
+                     "combine_GBps": bytes_combine(dwl) / (t3 - t2) / 1e3}
+    assert c.moe_status() == 0
+    return out
+
+
 def kernel_table(wl, r, peak):
     med = statistics.median
     mean = lambda v: sum(v) / len(v)
@@ -448,30 +499,7 @@ def run_cuda(args, wl):
     torch.cuda.empty_cache()
 
     if world == 1 and not args.no_decode and wl.name != synth.config(2).name:
-        # decode-step latency (config 2) in the same line: stream launches and CUDA-graph replay
-        dwl = synth.config(2)
-        dl = Layer(dwl, dev)
-        flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-        dr = time_steps(dl, 100, 5, barrier, flush)
-        gk = kernel_table(dwl, dr, peak)
-        graph_us = time_graph_steps(dl, 100, flush)
-        wr = time_steps(dl, 100, 5, barrier, None)            # back-to-back: whatever fits stays in L2
-        wk = kernel_table(dwl, wr, peak)
-        warm_graph_us = time_graph_steps(dl, 100, None)
-        line["decode"] = {
-            "config": describe(dwl), "l2": "256 MB L2 flush between steps (untimed)",
-            "timer": "CUDA events tick in 2.05 us steps on this GPU, so per-call figures are means over 100 steps",
-            "plan_us": gk["moe_plan"]["us_mean"], "dispatch_us": gk["moe_dispatch"]["us_mean"],
-            "combine_us": gk["moe_combine"]["us_mean"], "step_us_stream_launches": dr["ms_per_step"] * 1e3,
-            "step_us_cuda_graph": sum(graph_us) / len(graph_us),
-            "dispatch_GBps": gk["moe_dispatch"]["GBps"], "combine_GBps": gk["moe_combine"]["GBps"],
-            "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3,
-            "warm": {"l2": "back-to-back steps, no flush", "plan_us": wk["moe_plan"]["us_mean"],
-                     "dispatch_us": wk["moe_dispatch"]["us_mean"], "combine_us": wk["moe_combine"]["us_mean"],
-                     "step_us_stream_launches": wr["ms_per_step"] * 1e3,
-                     "step_us_cuda_graph": sum(warm_graph_us) / len(warm_graph_us)},
-        }
-        del dl, flush
+        line["decode"] = decode_latency(dev, peak)
         torch.cuda.empty_cache()
 
     if world == 1 and args.workload == "c5" and not args.no_decode:
