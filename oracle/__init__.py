@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_dispatch.argtypes = [p, i32, i32, i32, p, p, i32]
         L.oracle_expert_scale.argtypes = [p, i32, i32, i32, i64, p, p]
         L.oracle_combine.argtypes = [p, i32, i32, i32, p, p, p, i32]
+        L.oracle_gate_topk.argtypes = [p, i32, i32, i32, p, p]
+        L.oracle_gate_topk.restype = ctypes.c_int
         L.oracle_expert_ranges.argtypes = [i32, i32, i64, p, p, p]
         L.oracle_expert_ranges.restype = ctypes.c_int
         L.oracle_dispatch_quant.argtypes = [p, i32, i32, i32, p, p, p, i32]
@@ -115,6 +117,15 @@ def slots(topk_idx, E: int, R: int, pl: Plan, C: int, rank_tok_start=None):
     st = lib().oracle_slots(_ptr(topk_idx), T, K, E, R, _ptr(rts), _ptr(pl.s), _ptr(pl.o), _ptr(pl.n_recv),
                             int(C), _ptr(out))
     return st, out
+
+
+def gate_topk(logits, K: int):
+    logits = _c(logits, np.float32)
+    T, E = logits.shape
+    idx = np.full((T, K), -1, np.int32)
+    w = np.full((T, K), -1.0, np.float32)
+    st = lib().oracle_gate_topk(_ptr(logits), T, E, K, _ptr(idx), _ptr(w))
+    return st, idx, w
 
 
 def expert_ranges(E: int, R: int, C: int, n_exp):

@@ -13,6 +13,7 @@
 
 #include "moe_oracle.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <thread>
@@ -119,6 +120,31 @@ int oracle_dispatch_quant(const uint16_t* X, int32_t T, int32_t H, int32_t K, co
       }
     }
   });
+  return ORACLE_OK;
+}
+
+int oracle_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* topk_idx, float* topk_w) {
+  if (T < 0 || E < 1 || K < 1 || K > E) return ORACLE_ERR_INVALID_ARG;
+  std::vector<char> taken((size_t)E);
+  for (int32_t t = 0; t < T; ++t) {
+    const float* l = logits + (int64_t)t * E;
+    std::fill(taken.begin(), taken.end(), 0);
+    for (int32_t j = 0; j < K; ++j) {          // K rounds of "largest remaining logit, lowest index on ties"
+      int32_t best = -1;
+      for (int32_t e = 0; e < E; ++e)
+        if (!taken[e] && (best < 0 || l[e] > l[best])) best = e;
+      taken[best] = 1;
+      topk_idx[(int64_t)t * K + j] = best;
+    }
+    const float top = l[topk_idx[(int64_t)t * K]];
+    float sum = 0.0f;
+    for (int32_t j = 0; j < K; ++j) {
+      const float ex = std::exp(l[topk_idx[(int64_t)t * K + j]] - top);   // float overload: fp32 exponential
+      topk_w[(int64_t)t * K + j] = ex;
+      sum += ex;
+    }
+    for (int32_t j = 0; j < K; ++j) topk_w[(int64_t)t * K + j] /= sum;
+  }
   return ORACLE_OK;
 }
 

@@ -34,6 +34,14 @@ enum {
   ORACLE_ERR_CAPACITY = 3
 };
 
+/* Top-k gating (the step before dispatch: "top-k gating produces routing indexes and weights",
+ * Figures 1 and 4).  The paper gives no formula; the reading taken is the common one that the
+ * benchmark configurations describe: the K largest router logits of every token, in descending
+ * order (equal logits: the lower expert index first), and the softmax over those K logits in fp32:
+ *   w_j = exp(l_j - l_0) / sum_{j'=0..K-1} exp(l_j' - l_0),   sum accumulated in ascending j.
+ *   logits [T,E] fp32 (finite)  ->  topk_idx [T,K] int32, topk_w [T,K] fp32. */
+int oracle_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* topk_idx, float* topk_w);
+
 /* Planning state of the prefill schedule (Layout + Notify, Section 5.2):
  *   M      [R,E]  M[r,e]  = #branches from source rank r to expert e      (gathered count matrix)
  *   c_rank [R,R]  c_rank[r,d] = #branches from source rank r to rank d    (per-rank branch counts)

@@ -518,3 +518,30 @@ def test_dispatch_quant_against_torch_pipeline_and_error_bound(T, K, E, R, H):
     assert bool((err <= bound).all())
     top = (wq[slots[:, 0]] & 0x7F).max(1)
     assert (top[amax.numpy() > 0] == 0x7E).all() and top[3] == 0
+
+
+# ----------------------------------------------------------------------------- gating
+@pytest.mark.parametrize("T,E,K", [(64, 16, 2), (200, 256, 8), (33, 8, 8), (50, 40, 1), (10, 4096, 32)])
+def test_gate_topk_against_torch(T, E, K):
+    rng = np.random.default_rng(E + K)
+    logits = rng.standard_normal((T, E)).astype(np.float32) * 3
+    st, idx, w = oracle.gate_topk(logits, K)
+    assert st == oracle.OK
+    top = torch.topk(torch.from_numpy(logits), K, dim=1)            # distinct values: the order is unique
+    assert np.array_equal(idx, top.indices.numpy())
+    ref = torch.softmax(top.values.double(), dim=1).numpy()
+    assert np.abs(w - ref).max() <= 2e-7 + 4e-7 * ref.max()
+    assert np.allclose(w.sum(1), 1.0, atol=3e-7)
+    assert (np.diff(w, axis=1) <= 0).all()                           # descending logits => descending weights
+
+
+def test_gate_topk_ties_take_the_lower_index_first():
+    logits = np.array([[1.0, 5.0, 5.0, 0.0, 5.0, 2.0],
+                       [0.0, 0.0, 0.0, 0.0, 0.0, 0.0],
+                       [-1.0, -1.0, 3.0, 3.0, -2.0, 3.0]], np.float32)
+    st, idx, w = oracle.gate_topk(logits, 4)
+    # the definition, literally: sort experts by (logit descending, index ascending)
+    want = [sorted(range(6), key=lambda e: (-row[e], e))[:4] for row in logits]
+    assert idx.tolist() == want == [[1, 2, 4, 5], [0, 1, 2, 3], [2, 3, 5, 0]]
+    assert np.allclose(w[1], 0.25) and w[0, 0] == w[0, 1] == w[0, 2]
+    assert oracle.gate_topk(logits, 7)[0] == oracle.ERR_INVALID_ARG   # K > E
