@@ -94,6 +94,22 @@ moe_status_t moe_destroy(moe_ctx_t* ctx);
 moe_status_t moe_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE*/,
                       int32_t T, const int32_t* rank_tok_start /*HOST*/, void* stream);
 
+/* Top-k gating, the step in front of the path (Figures 1 and 4: top-k gating produces routing indexes
+ * and weights).  The paper gives no formula; this library's definition is the K largest router logits
+ * of a token in descending order (equal logits: lower expert index first) and the fp32 softmax over
+ * those K logits, summed in ascending j.  Logits must be finite.
+ *   logits    DEVICE [T,E] fp32            topk_idx  DEVICE [T,K] int32, out
+ *                                          topk_w    DEVICE [T,K] fp32, out
+ * moe_gate_topk is the stand-alone kernel (no context).  moe_gate_plan gates and plans: when every
+ * source rank holds at most 4096 branches (every decode step) both happen in ONE launch -- each
+ * rank's CTA gates its tokens, keeps their indexes in shared memory and plans from there -- otherwise
+ * it is the gate kernel followed by moe_plan.  topk_idx must stay valid like moe_plan's input. */
+moe_status_t moe_gate_topk(const float* logits /*DEVICE*/, int32_t T, int32_t E, int32_t K,
+                           int32_t* topk_idx /*DEVICE*/, float* topk_w /*DEVICE*/, void* stream);
+moe_status_t moe_gate_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const float* logits /*DEVICE*/, int32_t T,
+                           const int32_t* rank_tok_start /*HOST*/, int32_t* topk_idx /*DEVICE*/,
+                           float* topk_w /*DEVICE*/, void* stream);
+
 /* DEVICE views into the workspace, valid until the next moe_plan on this
  * context.  Shapes: counts M [R,E], c_rank [R,R], small_off s|delta [T,K],
  * large_off o|o_dec [E,R] (window-local row), n_exp [E], n_recv [R].

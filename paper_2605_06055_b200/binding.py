@@ -25,6 +25,7 @@ EXPORTS = [
     "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
+    "moe_gate_topk", "moe_gate_plan",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE = 0, 1
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -66,6 +67,10 @@ def load() -> ctypes.CDLL:
     L.moe_plan_view.argtypes = [vp, ctypes.POINTER(MoePlanView)]
     L.moe_dispatch.argtypes = [vp, vp, vp, i64, vp]
     L.moe_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.moe_gate_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp]
+    L.moe_gate_topk.restype = ctypes.c_int
+    L.moe_gate_plan.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp, vp, vp]
+    L.moe_gate_plan.restype = ctypes.c_int
     L.moe_expert_ranges.argtypes = [vp, i64, vp, vp, vp]
     L.moe_expert_ranges.restype = ctypes.c_int
     L.moe_dispatch_quant.argtypes = [vp, vp, vp, vp, i64, vp]
@@ -168,6 +173,20 @@ class MoeComm:
             self.T, self.schedule, self._keep = T, schedule, topk_idx
         elif check:
             raise MoeError(rc, "moe_plan")
+        return rc
+
+    def moe_gate_plan(self, schedule: int, logits: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor,
+                      T: Optional[int] = None, rank_tok_start=None, stream=None, check: bool = True) -> int:
+        T = logits.shape[0] if T is None else T
+        rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_gate_plan(self._h, schedule, _dev_ptr(logits, torch.float32), T, _host_ptr(rts),
+                                        _dev_ptr(topk_idx, torch.int32), _dev_ptr(topk_w, torch.float32),
+                                        _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx
+        elif check:
+            raise MoeError(rc, "moe_gate_plan")
         return rc
 
     def moe_plan_view(self) -> dict:
@@ -280,3 +299,11 @@ def moe_slots_noalloc(topk_idx: torch.Tensor, E: int, R: int, capacity_rows: int
                                             int(capacity_rows), _dev_ptr(slots, torch.int32),
                                             _dev_ptr(n_recv, torch.int32), _dev_ptr(status, torch.int32),
                                             _stream_handle(stream)))
+
+
+def moe_gate_topk(logits: torch.Tensor, K: int, topk_idx: torch.Tensor, topk_w: torch.Tensor, stream=None) -> int:
+    """Stand-alone top-k gate (see include/moecomm.h): K largest logits + fp32 softmax over them."""
+    T, E = logits.shape
+    with torch.cuda.device(logits.device):
+        return int(load().moe_gate_topk(_dev_ptr(logits, torch.float32), T, E, K, _dev_ptr(topk_idx, torch.int32),
+                                        _dev_ptr(topk_w, torch.float32), _stream_handle(stream)))

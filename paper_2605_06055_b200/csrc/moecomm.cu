@@ -263,8 +263,14 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
     const int scan_smem = notify_smem_ints(shape->E, shape->R) * (int)sizeof(int32_t);
     if (rank_smem > 48 * 1024)
       ok = (shape->E <= RANK_PLAN_WIDE_MAX_E
-                ? cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)
-                : cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)) ==
+                ? cudaFuncSetAttribute(plan_rank_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)
+                : cudaFuncSetAttribute(plan_rank_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)) ==
+           cudaSuccess;
+    const bool wide = shape->E <= RANK_PLAN_WIDE_MAX_E;
+    const int gated_smem = rank_plan_gated_smem_ints(shape->E, shape->R, wide ? 32 : 8) * (int)sizeof(int32_t);
+    if (ok && gated_smem > 48 * 1024 && gated_smem <= 200 * 1024)
+      ok = (wide ? cudaFuncSetAttribute(plan_rank_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gated_smem)
+                 : cudaFuncSetAttribute(plan_rank_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gated_smem)) ==
            cudaSuccess;
     if (ok && scan_smem > 48 * 1024)
       ok = cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) ==
@@ -291,13 +297,30 @@ moe_status_t moe_destroy(moe_ctx_t* ctx) {
   return MOE_OK;
 }
 
-moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
-                      const int32_t* rank_tok_start, void* stream) {
-  moe_ctx* ctx = c;
+}  // extern "C"
+
+namespace {
+
+void launch_gate(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
+                 cudaStream_t st) {
+  int warps = 8;
+  while (warps > 1 && warps * E * (int)sizeof(float) > 96 * 1024) warps >>= 1;
+  const int smem = warps * E * (int)sizeof(float);
+  if (smem > 48 * 1024) cudaFuncSetAttribute(gate_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  int64_t grid = ((int64_t)T + warps - 1) / warps;
+  if (grid > (int64_t)num_sms * 8) grid = (int64_t)num_sms * 8;
+  if (grid < 1) grid = 1;
+  gate_topk_kernel<<<(int)grid, warps * 32, smem, st>>>(logits, T, E, K, idx, w);
+}
+
+// Planning, optionally with the gate in front (logits != nullptr: topk_idx and topk_w are OUTPUTS).
+moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                       const int32_t* rank_tok_start, void* stream, const float* logits, int32_t* idx_out,
+                       float* w_out) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   const moe_shape_t& sh = ctx->shape;
   if (schedule != MOE_SCHED_PREFILL && schedule != MOE_SCHED_DECODE) return MOE_ERR_INVALID_ARG;
-  if (T < 0 || T > sh.T_max || (T > 0 && topk_idx == nullptr)) return MOE_ERR_INVALID_ARG;
+  if (T < 0 || T > sh.T_max) return MOE_ERR_INVALID_ARG;
   if (rank_tok_start == nullptr && T % sh.R != 0) return MOE_ERR_INVALID_ARG;
   if (rank_tok_start != nullptr) {
     if (rank_tok_start[0] != 0 || rank_tok_start[sh.R] != T) return MOE_ERR_INVALID_ARG;
@@ -342,14 +365,33 @@ moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk
     if (br > max_rank_branches) max_rank_branches = br;
   }
   ctx->compact_plan = max_rank_branches <= RANK_PLAN_MAX_BRANCHES;
+  const bool wide = sh.E <= RANK_PLAN_WIDE_MAX_E;
+  const int gated_smem = rank_plan_gated_smem_ints(sh.E, sh.R, wide ? 32 : 8) * (int)sizeof(int32_t);
+  const bool fuse_gate = logits != nullptr && ctx->compact_plan && gated_smem <= 200 * 1024;
   int n = 0;
-  if (ctx->compact_plan) {
-    if (sh.E <= RANK_PLAN_WIDE_MAX_E)
-      plan_rank_kernel<32><<<sh.R, 32 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+  if (logits != nullptr && !fuse_gate) {   // gate as its own launch, then plan from the indexes it wrote
+    launch_gate(logits, T, sh.E, sh.K, idx_out, w_out, ctx->num_sms, st);
+    ++n;
+  }
+  if (fuse_gate) {
+    if (wide)
+      plan_rank_kernel<32, true><<<sh.R, 32 * 32, gated_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
+          logits, idx_out, w_out);
     else
-      plan_rank_kernel<8><<<sh.R, 8 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+      plan_rank_kernel<8, true><<<sh.R, 8 * 32, gated_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
+          logits, idx_out, w_out);
+    ++n;
+  } else if (ctx->compact_plan) {
+    if (wide)
+      plan_rank_kernel<32, false><<<sh.R, 32 * 32, rank_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
+          nullptr, nullptr, nullptr);
+    else
+      plan_rank_kernel<8, false><<<sh.R, 8 * 32, rank_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
+          nullptr, nullptr, nullptr);
     ++n;
   } else {
     if (tiles > 0) {
@@ -373,6 +415,36 @@ moe_status_t moe_plan(moe_ctx_t* c, moe_schedule_t schedule, const int32_t* topk
   const moe_status_t rc = launch_ok(ctx, n);
   if (rc == MOE_OK) ctx->planned = true;
   return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+moe_status_t moe_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                      const int32_t* rank_tok_start, void* stream) {
+  if (T > 0 && topk_idx == nullptr) return MOE_ERR_INVALID_ARG;
+  return plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, nullptr, nullptr, nullptr);
+}
+
+moe_status_t moe_gate_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const float* logits, int32_t T,
+                           const int32_t* rank_tok_start, int32_t* topk_idx, float* topk_w, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (ctx->shape.K > ctx->shape.E) return MOE_ERR_INVALID_ARG;
+  if (T > 0 && (logits == nullptr || topk_idx == nullptr || topk_w == nullptr)) return MOE_ERR_INVALID_ARG;
+  return plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, logits, topk_idx, topk_w);
+}
+
+moe_status_t moe_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* topk_idx, float* topk_w,
+                           void* stream) {
+  if (T < 0 || E < 1 || E > MOE_MAX_E || K < 1 || K > MOE_MAX_K || K > E) return MOE_ERR_INVALID_ARG;
+  if (T > 0 && (logits == nullptr || topk_idx == nullptr || topk_w == nullptr)) return MOE_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (T > 0) launch_gate(logits, T, E, K, topk_idx, topk_w, sms, static_cast<cudaStream_t>(stream));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 moe_status_t moe_plan_view(const moe_ctx_t* c, moe_plan_view_t* out) {

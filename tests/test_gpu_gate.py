@@ -1,0 +1,92 @@
+"""Top-k gating on the GPU (stand-alone and fused with the planner) against the CPU oracle.
+
+Indexes are compared bit for bit.  Weights are fp32 softmax values whose exponentials come from two
+different libms (device expf: <= 2 ulp, host expf: <= 1 ulp), followed by a K-term sum and a division:
+the relative budget is (2 + 1 + K/2 + 2) * 2^-24, below 1.3e-6 for K <= 32; the tests allow 2e-6.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06055_b200 import binding, synth
+from paper_2605_06055_b200.synth import DECODE, PREFILL
+
+pytestmark = pytest.mark.gpu
+RTOL = 2e-6
+
+
+def logits_for(T, E, seed, ties=False):
+    g = torch.Generator().manual_seed(seed)
+    l = torch.randn(T, E, generator=g) * 3
+    if ties:
+        l = torch.round(l)            # many equal logits: the lower index must win
+    return l.contiguous()
+
+
+@pytest.mark.parametrize("T,E,K,ties", [(256, 16, 2, False), (2048, 256, 8, False), (500, 256, 8, True),
+                                        (77, 8, 8, True), (300, 40, 1, False), (64, 4096, 32, False),
+                                        (1000, 1000, 6, True)])
+def test_gate_topk_kernel(T, E, K, ties):
+    dev = torch.device("cuda:0")
+    l = logits_for(T, E, T + E, ties)
+    st, want_idx, want_w = oracle.gate_topk(l.numpy(), K)
+    assert st == oracle.OK
+    idx = torch.full((T, K), -1, dtype=torch.int32, device=dev)
+    w = torch.full((T, K), -1.0, dtype=torch.float32, device=dev)
+    assert binding.moe_gate_topk(l.to(dev), K, idx, w) == binding.MOE_OK
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), want_idx)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+
+
+@pytest.mark.parametrize("case", [
+    ("decode_c2_fused", 2048, 256, 16, 8, DECODE, None),
+    ("prefill_small_fused", 1024, 64, 8, 4, PREFILL, None),
+    ("fused_ragged_empty_rank", 900, 32, 4, 6, DECODE, (400, 0, 137, 363)),
+    ("big_E_fused_8_warps", 256, 1024, 2, 8, DECODE, None),
+    ("unfused_large_ranks", 16384, 256, 2, 8, PREFILL, None),
+    ("unfused_large_E", 512, 4096, 4, 8, DECODE, None),
+], ids=lambda c: c[0])
+def test_gate_plan_matches_oracle_gate_then_oracle_plan(case):
+    name, T, E, R, K, sch, per = case
+    dev = torch.device("cuda:0")
+    l = logits_for(T, E, T * 7 + E, ties=(T % 2 == 0))
+    st, want_idx, want_w = oracle.gate_topk(l.numpy(), K)
+    rts = None if per is None else np.concatenate([[0], np.cumsum(per)]).astype(np.int32)
+    p = oracle.plan(want_idx, E, R, rts)
+    assert p.status == oracle.OK
+    C = int(p.n_recv.max()) + 1
+    _, want_slots = oracle.slots(want_idx, E, R, p, C, rts)
+
+    comm = binding.MoeComm(T, 64, E, R, K, dev)
+    idx = torch.full((T, K), -1, dtype=torch.int32, device=dev)
+    w = torch.full((T, K), -1.0, dtype=torch.float32, device=dev)
+    comm.moe_gate_plan(sch, l.to(dev), idx, w, T, rts)
+    slots = torch.empty((T, K), dtype=torch.int32, device=dev)
+    comm.moe_slots(C, slots)
+    assert comm.moe_status() == 0
+    assert np.array_equal(idx.cpu().numpy(), want_idx)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+    assert np.array_equal(slots.cpu().numpy().astype(np.int64), want_slots)
+    v = comm.moe_plan_view()
+    assert np.array_equal(v["large_off"].cpu().numpy(), p.o) and np.array_equal(v["n_recv"].cpu().numpy(), p.n_recv)
+    if sch == PREFILL:
+        assert np.array_equal(v["counts"].cpu().numpy(), p.M) and np.array_equal(v["small_off"].cpu().numpy(), p.s)
+    # the indexes and weights it wrote drive the rest of the path: identity experts give X back
+    x = torch.randn(T, 64, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16).to(dev)
+    win = torch.zeros((R * C, 64), dtype=torch.bfloat16, device=dev)
+    y = torch.empty_like(x)
+    comm.moe_dispatch(x, win, C)
+    comm.moe_combine(win, C, w, y)
+    assert comm.moe_status() == 0
+    assert torch.equal(y.view(torch.int16) & 0x7FFF, x.view(torch.int16) & 0x7FFF)
+    comm.close()
+
+
+def test_gate_argument_checks():
+    dev = torch.device("cuda:0")
+    l = torch.zeros((4, 8), device=dev)
+    idx = torch.zeros((4, 9), dtype=torch.int32, device=dev)
+    w = torch.zeros((4, 9), device=dev)
+    assert binding.moe_gate_topk(l, 9, idx, w) == binding.MOE_ERR_INVALID_ARG      # K > E
