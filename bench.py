@@ -395,18 +395,27 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
     out = {"config": describe(dwl),
            "method": f"cumulative sequences of calls, {n} repetitions per pair of CUDA events; per-call = difference",
            "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3}
+    from paper_2605_06055_b200 import binding
+    logits = torch.randn(dwl.T, dwl.E, generator=torch.Generator().manual_seed(7)).to(dev)
+    g_idx, g_w = torch.empty_like(dl.idx), torch.empty_like(dl.w)
+    gate = lambda: binding.moe_gate_topk(logits, dwl.K, g_idx, g_w)
+    gate_plan = lambda: c.moe_gate_plan(dwl.schedule, logits, g_idx, g_w)
     for name, pre in (("cold", [flush]), ("warm", [])):
         base = time_repeated(pre, n) if pre else 0.0
         t1 = time_repeated(pre + [plan], n)
         t2 = time_repeated(pre + [plan, disp], n)
         t3 = time_repeated(pre + [plan, disp, comb], n)
         tg = time_repeated(pre + [replay], n)
+        t_gate = time_repeated(pre + [gate], n)
+        t_gate_plan = time_repeated(pre + [gate_plan], n)
         out[name] = {"l2": "256 MB L2 flush before every step (its time subtracted)" if pre else
                      "back-to-back steps, no flush",
                      "plan_us": t1 - base, "dispatch_us": t2 - t1, "combine_us": t3 - t2,
                      "step_us_stream_launches": t3 - base, "step_us_cuda_graph": tg - base,
                      "dispatch_GBps": bytes_dispatch(dwl) / (t2 - t1) / 1e3,
-                     "combine_GBps": bytes_combine(dwl) / (t3 - t2) / 1e3}
+                     "combine_GBps": bytes_combine(dwl) / (t3 - t2) / 1e3,
+                     "gate_us": t_gate - base, "gate_plan_us": t_gate_plan - base}
+    plan()   # leave the context planned on dl.idx again
     assert c.moe_status() == 0
     return out
 
@@ -455,6 +464,13 @@ def run_cuda(args, wl):
     quant_us = None
     if wl.H % 16 == 0 and not args.no_decode:
         quant_us = time_dispatch_quant(layer, min(args.steps, 50), scratch)
+    gate_us = None
+    if not args.no_decode:
+        from paper_2605_06055_b200 import binding
+        logits = torch.randn(wl.T, wl.E, generator=torch.Generator().manual_seed(7)).to(dev)
+        g_idx, g_w = torch.empty_like(layer.idx), torch.empty_like(layer.w)
+        gate_us = time_repeated([lambda: binding.moe_gate_topk(logits, wl.K, g_idx, g_w)], 50)
+        del logits, g_idx, g_w
     e2e = None
     if not args.no_e2e:
         e2e_steps = max(3, min(args.steps, 10))
@@ -476,6 +492,11 @@ def run_cuda(args, wl):
                                          "bytes": bytes_dispatch_quant(wl), "GBps": gbps,
                                          "frac_of_measured_peak": gbps / peak, "frac_of_8TBps": gbps / NOMINAL_HBM_GBS,
                                          "note": "row-wise e4m3 + fp32 scale variant of dispatch; not part of the step"}
+    if gate_us is not None:
+        gb = wl.T * wl.E * 4 + wl.T * wl.K * 8
+        kernels["moe_gate_topk"] = {"us": gate_us, "bytes": gb, "GBps": gb / gate_us / 1e3,
+                                    "note": "top-k + softmax over fp32 router logits [T,E], back-to-back launches "
+                                            "(logits fit in L2); not part of the step"}
     dom = "moe_dispatch" if sum(r["dispatch_us"]) >= sum(r["combine_us"]) else "moe_combine"
     dom_kernel = "dispatch_bulk_kernel" if dom == "moe_dispatch" else "combine_rows_kernel"
     roofline = {"bound": "hbm", "kernel": dom_kernel, "achieved": kernels[dom]["GBps"], "peak": peak,

@@ -55,7 +55,74 @@ __device__ __forceinline__ void warp_gate_token(const float* __restrict__ logits
   idx_lane = sel_idx;
 }
 
-// Stand-alone gate: grid-stride over tokens, one warp per token.  Dynamic shared memory: warps * E floats.
+// Order-preserving map from fp32 to uint32 (larger float <=> larger key), so that the warp-wide
+// arg-max can use the single-instruction integer reductions (redux.sync).
+__device__ __forceinline__ uint32_t sortable_key(float f) {
+  const uint32_t u = __float_as_uint(f + 0.0f);   // -0 becomes +0: the two compare equal as floats
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// The same for E <= 32 * VPT with the row in registers: lane l holds experts l, l + 32, ... (coalesced
+// loads) as sortable keys; 0 marks "absent or retired" (no finite float maps to key 0).  A round is
+// VPT-1 integer max, one redux.max for the winning value, one redux.min for the lowest expert
+// index that holds it, and a predicated retire: about 45 instructions instead of about 110 with a
+// shuffle tree on (value, index) pairs.
+template <int VPT>
+__device__ __forceinline__ void warp_gate_token_regs(const float* __restrict__ logits_row, int E, int K, int lane,
+                                                     int32_t& idx_lane, float& w_lane) {
+  uint32_t v[VPT];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int e = lane + 32 * i;
+    v[i] = e < E ? sortable_key(__ldg(logits_row + e)) : 0u;
+  }
+  uint32_t sel_key = 0;
+  int32_t sel_idx = -1;
+  for (int j = 0; j < K; ++j) {
+    uint32_t local = v[0];
+#pragma unroll
+    for (int i = 1; i < VPT; ++i) local = max(local, v[i]);
+    const uint32_t best = __reduce_max_sync(0xffffffffu, local);
+    int32_t first = 0x7fffffff;                      // lowest expert index of mine that holds `best`
+#pragma unroll
+    for (int i = VPT - 1; i >= 0; --i) first = (v[i] == best) ? lane + 32 * i : first;
+    const int32_t be = (int32_t)__reduce_min_sync(0xffffffffu, (uint32_t)first);
+    if (lane == j) {
+      sel_key = best;
+      sel_idx = be;
+    }
+    // Retire the winner: a select on every register, so the array is never indexed dynamically.
+    const int32_t hit = (be & 31) == lane ? (be >> 5) : -1;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) v[i] = (i == hit) ? 0u : v[i];
+  }
+  const float sel_val = key_to_float(sel_key);
+  const float top = __shfl_sync(0xffffffffu, sel_val, 0);
+  const float ex = lane < K ? expf(sel_val - top) : 0.0f;
+  float sum = 0.0f;
+  for (int j = 0; j < K; ++j) sum += __shfl_sync(0xffffffffu, ex, j);
+  w_lane = __fdiv_rn(ex, sum);
+  idx_lane = sel_idx;
+}
+
+// Picks the register form when the row fits (E <= 1024), else the shared-memory form.
+__device__ __forceinline__ void warp_gate_any(const float* __restrict__ logits_row, float* row, int E, int K, int lane,
+                                              int32_t& idx_lane, float& w_lane) {
+  if (E <= 32) warp_gate_token_regs<1>(logits_row, E, K, lane, idx_lane, w_lane);
+  else if (E <= 64) warp_gate_token_regs<2>(logits_row, E, K, lane, idx_lane, w_lane);
+  else if (E <= 128) warp_gate_token_regs<4>(logits_row, E, K, lane, idx_lane, w_lane);
+  else if (E <= 256) warp_gate_token_regs<8>(logits_row, E, K, lane, idx_lane, w_lane);
+  else if (E <= 512) warp_gate_token_regs<16>(logits_row, E, K, lane, idx_lane, w_lane);
+  else if (E <= 1024) warp_gate_token_regs<32>(logits_row, E, K, lane, idx_lane, w_lane);
+  else warp_gate_token(logits_row, row, E, K, lane, idx_lane, w_lane);
+}
+
+// Stand-alone gate: grid-stride over tokens, one warp per token.  Dynamic shared memory: warps * E floats
+// (used only when E > 1024).
 __global__ void __launch_bounds__(256)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
                  float* __restrict__ topk_w) {
@@ -65,7 +132,7 @@ gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t
   for (int32_t t = blockIdx.x * wpc + warp; t < T; t += gridDim.x * wpc) {
     int32_t idx;
     float w;
-    warp_gate_token(logits + (size_t)t * E, row, E, K, lane, idx, w);
+    warp_gate_any(logits + (size_t)t * E, row, E, K, lane, idx, w);
     if (lane < K) {
       topk_idx[(size_t)t * K + lane] = idx;
       topk_w[(size_t)t * K + lane] = w;

@@ -9,6 +9,7 @@
 
 #include "common.cuh"
 #include "plan_kernels.cuh"
+#include "gate_kernels.cuh"
 #include "row_kernels.cuh"
 #include "bulk_kernels.cuh"
 #include "quant_kernels.cuh"
@@ -263,14 +264,8 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
     const int scan_smem = notify_smem_ints(shape->E, shape->R) * (int)sizeof(int32_t);
     if (rank_smem > 48 * 1024)
       ok = (shape->E <= RANK_PLAN_WIDE_MAX_E
-                ? cudaFuncSetAttribute(plan_rank_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)
-                : cudaFuncSetAttribute(plan_rank_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)) ==
-           cudaSuccess;
-    const bool wide = shape->E <= RANK_PLAN_WIDE_MAX_E;
-    const int gated_smem = rank_plan_gated_smem_ints(shape->E, shape->R, wide ? 32 : 8) * (int)sizeof(int32_t);
-    if (ok && gated_smem > 48 * 1024 && gated_smem <= 200 * 1024)
-      ok = (wide ? cudaFuncSetAttribute(plan_rank_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gated_smem)
-                 : cudaFuncSetAttribute(plan_rank_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gated_smem)) ==
+                ? cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)
+                : cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)) ==
            cudaSuccess;
     if (ok && scan_smem > 48 * 1024)
       ok = cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) ==
@@ -366,32 +361,18 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
   }
   ctx->compact_plan = max_rank_branches <= RANK_PLAN_MAX_BRANCHES;
   const bool wide = sh.E <= RANK_PLAN_WIDE_MAX_E;
-  const int gated_smem = rank_plan_gated_smem_ints(sh.E, sh.R, wide ? 32 : 8) * (int)sizeof(int32_t);
-  const bool fuse_gate = logits != nullptr && ctx->compact_plan && gated_smem <= 200 * 1024;
   int n = 0;
-  if (logits != nullptr && !fuse_gate) {   // gate as its own launch, then plan from the indexes it wrote
+  if (logits != nullptr) {   // gate first (its own launch, spread over all SMs), then plan from the indexes it wrote
     launch_gate(logits, T, sh.E, sh.K, idx_out, w_out, ctx->num_sms, st);
     ++n;
   }
-  if (fuse_gate) {
+  if (ctx->compact_plan) {
     if (wide)
-      plan_rank_kernel<32, true><<<sh.R, 32 * 32, gated_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
-          logits, idx_out, w_out);
+      plan_rank_kernel<32><<<sh.R, 32 * 32, rank_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     else
-      plan_rank_kernel<8, true><<<sh.R, 8 * 32, gated_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
-          logits, idx_out, w_out);
-    ++n;
-  } else if (ctx->compact_plan) {
-    if (wide)
-      plan_rank_kernel<32, false><<<sh.R, 32 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
-          nullptr, nullptr, nullptr);
-    else
-      plan_rank_kernel<8, false><<<sh.R, 8 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
-          nullptr, nullptr, nullptr);
+      plan_rank_kernel<8><<<sh.R, 8 * 32, rank_smem, st>>>(
+          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     ++n;
   } else {
     if (tiles > 0) {

@@ -23,7 +23,6 @@
 #pragma once
 
 #include "common.cuh"
-#include "gate_kernels.cuh"
 
 namespace moe {
 
@@ -285,20 +284,11 @@ __host__ __device__ constexpr int rank_plan_smem_ints(int E, int R, int warps) {
   return (warps + 2) * E > notify_smem_ints(E, R) ? (warps + 2) * E : notify_smem_ints(E, R);
 }
 
-// GATED: the routing indexes do not exist yet.  The CTA first gates its rank's tokens (one warp per
-// token, see gate_kernels.cuh), writes topk_idx / topk_w for dispatch and combine, keeps the indexes
-// in shared memory and plans from there: gate + plan in ONE launch.
-constexpr int RANK_PLAN_MAX_BRANCHES_I = 4096;
-__host__ __device__ constexpr int rank_plan_gated_smem_ints(int E, int R, int warps) {
-  return rank_plan_smem_ints(E, R, warps) + RANK_PLAN_MAX_BRANCHES_I + warps * E;
-}
-
-template <int WARPS, bool GATED>
+template <int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
                  int32_t full_table, int32_t* __restrict__ s, int32_t* __restrict__ M, int32_t* __restrict__ c_rank,
-                 int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl,
-                 const float* __restrict__ logits, int32_t* __restrict__ topk_idx_out, float* __restrict__ topk_w_out) {
+                 int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
   constexpr int P = WARPS + 1;
@@ -308,23 +298,6 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int32_t b_begin = map.tok_start[r] * K, b_end = map.tok_start[r + 1] * K;
   const unsigned lt = lanemask_lt();
-  int32_t* idx_s = sm + rank_plan_smem_ints(E, R, WARPS);   // GATED: this rank's routing indexes
-
-  if constexpr (GATED) {
-    float* row = reinterpret_cast<float*>(idx_s + RANK_PLAN_MAX_BRANCHES_I) + warp * E;
-    for (int32_t t = map.tok_start[r] + warp; t < map.tok_start[r + 1]; t += WARPS) {
-      int32_t gi;
-      float gw;
-      warp_gate_token(logits + (size_t)t * E, row, E, K, lane, gi, gw);
-      if (lane < K) {
-        topk_idx_out[(size_t)t * K + lane] = gi;
-        topk_w_out[(size_t)t * K + lane] = gw;
-        idx_s[(t - map.tok_start[r]) * K + lane] = gi;
-      }
-      __syncwarp();
-    }
-    __syncthreads();
-  }
 
   for (int e = threadIdx.x; e < E; e += WARPS * 32) rank_base[e] = 0;
   for (int32_t pass = b_begin; pass < b_end; pass += WARPS * 32) {
@@ -332,7 +305,7 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
     const int32_t b = pass + warp * 32 + lane;
     int32_t e = -1;
     if (b < b_end) {
-      e = GATED ? idx_s[b - b_begin] : __ldg(topk_idx + b);
+      e = __ldg(topk_idx + b);
       if (e < 0 || e >= E) {
         raise_status(&ctl->status, MOE_ERR_BAD_INDEX);
         e = -1;
