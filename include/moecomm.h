@@ -189,8 +189,13 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
  *                          REGISTERS (16-byte ld/st through registers, K-specialised), or
  *                          BULK (cp.async.bulk through shared-memory stages).  Same result.
  *   MOE_OPT_GRANULE        512-byte units per work item of dispatch/combine; 0 = chosen from the
- *                          job size.  Any value gives the same result. */
-typedef enum { MOE_OPT_DISPATCH_PATH = 0, MOE_OPT_GRANULE = 1 } moe_option_t;
+ *                          job size.  Any value gives the same result.
+ *   MOE_OPT_TEST_STARVE_WAIT_MS  failure-path test hook, 0 = off.  With value v > 0 the bulk-copy
+ *                          dispatch lets ONE warp wait for 16 bytes that are never sent and bounds
+ *                          every device-side wait by v milliseconds: that warp gives up, the status
+ *                          word becomes MOE_ERR_TIMEOUT, the kernel ends normally (no trap, nothing
+ *                          left in flight) and the windows are incomplete.  Normal bound: 2 s. */
+typedef enum { MOE_OPT_DISPATCH_PATH = 0, MOE_OPT_GRANULE = 1, MOE_OPT_TEST_STARVE_WAIT_MS = 2 } moe_option_t;
 enum { MOE_DISPATCH_AUTO = 0, MOE_DISPATCH_REGISTERS = 1, MOE_DISPATCH_BULK = 2 };
 moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);
 

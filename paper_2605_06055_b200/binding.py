@@ -27,7 +27,7 @@ EXPORTS = [
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
     "moe_gate_topk", "moe_gate_plan",
 ]
-MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE = 0, 1
+MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS = 0, 1, 2
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
 
 

@@ -9,8 +9,9 @@
 // HBM sees long sequential bursts per row, and the number of bytes in flight is
 // set by shared memory (about 170 KB per SM), not by registers or warp count.
 //
-// Every wait is bounded: an mbarrier that does not complete within WAIT_LIMIT
-// polls raises MOE_ERR_TIMEOUT and the warp stops taking work.
+// Every wait is bounded in time: an mbarrier that does not complete within the
+// limit (2 s by default) raises MOE_ERR_TIMEOUT and the warp stops taking work;
+// the kernel still ends normally and the context stays usable.
 #pragma once
 
 #include "row_kernels.cuh"
@@ -21,7 +22,7 @@ constexpr int BULK_MAX_WARPS = 8;      // warps per CTA: as many 3-stage rings a
 constexpr int BULK_SMEM_BUDGET = 200 * 1024;
 constexpr int BULK_STAGES = 3;
 constexpr int BULK_MAX_GRANULE = 32;   // a stage holds at most 16 KB of one row
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int32_t WAIT_LIMIT_MS_DEFAULT = 2000;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -43,11 +44,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait; false if the barrier did not complete.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait; false if the barrier did not complete within limit_ms milliseconds.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t limit_ms) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns(), limit = (uint64_t)limit_ms * 1000000ull;
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > limit) return false;
+  }
 }
 
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
@@ -100,7 +111,9 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
     const WorkItem w = decode_item(a, item);
     const uint32_t off = (uint32_t)w.i0 * 512u;
     const uint32_t bytes = min((uint32_t)w.i1 * 512u, row_bytes) - off;
-    mbar_expect_tx(bar0 + 8 * s, bytes);
+    // Test hook: one warp expects 16 bytes that never come, so its wait runs out (see MOE_OPT_TEST_STARVE_WAIT_MS).
+    const uint32_t starve = (a.test_starve && blockIdx.x == 0 && warp == 0 && item == 0) ? 16u : 0u;
+    mbar_expect_tx(bar0 + 8 * s, bytes + starve);
     bulk_load(buf0 + s * stage_bytes, X + (size_t)w.t * row_bytes + off, bytes, bar0 + 8 * s);
   };
 
@@ -126,7 +139,7 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
     const uint32_t bytes = min((uint32_t)w.i1 * 512u, row_bytes) - off;
 
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity, a.wait_limit_ms) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) {
       if (lane == 0) raise_status(a.status, MOE_ERR_TIMEOUT);

@@ -36,6 +36,7 @@ struct moe_ctx {
   int64_t launches;
   int32_t dispatch_path;    // MOE_OPT_DISPATCH_PATH
   int32_t granule_override; // MOE_OPT_GRANULE
+  int32_t starve_wait_ms;   // MOE_OPT_TEST_STARVE_WAIT_MS
 };
 
 namespace {
@@ -120,6 +121,8 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
+  a.wait_limit_ms = ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT;
+  a.test_starve = ctx->starve_wait_ms > 0;
   return a;
 }
 
@@ -248,6 +251,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->topk_idx = nullptr;
   ctx->dispatch_path = MOE_DISPATCH_AUTO;
   ctx->granule_override = 0;
+  ctx->starve_wait_ms = 0;
 
   // Shared memory of the planning kernels grows with E; opt in above 48 KB.
   const int tile_smem = PLAN_WARPS * shape->E * (int)sizeof(int32_t);
@@ -583,6 +587,10 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) 
         return MOE_ERR_INVALID_ARG;
       ctx->dispatch_path = (int32_t)value;
       return MOE_OK;
+    case MOE_OPT_TEST_STARVE_WAIT_MS:
+      if (value < 0 || value > 10000) return MOE_ERR_INVALID_ARG;
+      ctx->starve_wait_ms = (int32_t)value;
+      return MOE_OK;
     case MOE_OPT_GRANULE:
       if (value < 0 || value > (1 << 20)) return MOE_ERR_INVALID_ARG;
       ctx->granule_override = (int32_t)value;
@@ -744,6 +752,8 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
+  a.wait_limit_ms = WAIT_LIMIT_MS_DEFAULT;
+  a.test_starve = 0;
   int grid = (int)(((int64_t)T * K + 255) / 256);
   if (grid < 1) grid = 1;
   slots_kernel<<<grid, 256, 0, st>>>(slots, a, map);

@@ -94,7 +94,7 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
     const uint32_t in = buf0 + s * stage_stride, out = in + in_stride;
 
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity, a.wait_limit_ms) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) {
       if (lane == 0) raise_status(a.status, MOE_ERR_TIMEOUT);

@@ -29,6 +29,8 @@ struct RowArgs {
   int32_t granule;           // units (512-byte slabs) per work item
   int32_t items_per_row;     // ceil(units per row / granule)
   int32_t n_items;           // T * items_per_row
+  int32_t wait_limit_ms;     // bound of every device-side wait
+  int32_t test_starve;       // test hook of the bulk-copy dispatch: make one wait run out
 };
 
 // Window row of branch (t, lane) for lane < K, -1 otherwise.  Small offsets of

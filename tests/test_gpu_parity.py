@@ -339,3 +339,34 @@ class Workload_identity:
         out = copy.copy(inp)
         out.wl = dataclasses.replace(inp.wl, expert_op="identity")
         return out
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """Failure path without a fault: one warp of the bulk-copy dispatch waits for bytes that never
+    come; its bounded wait expires, the kernel ends normally with MOE_ERR_TIMEOUT in the status word,
+    and the next call on the same context is correct."""
+    dev = torch.device("cuda:0")
+    wl = Workload("starve", 1024, 2048, 32, 4, 4, PREFILL, "uniform", "identity", 61)
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max())
+    o = harness.oracle_run(inp, C)
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
+    win = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
+    Y = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    comm.moe_plan(PREFILL, idx)
+    comm.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 50)
+    comm.moe_dispatch(X, win, C)
+    assert comm.moe_status() == binding.MOE_ERR_TIMEOUT
+    assert comm.moe_status() == 0                                   # cleared by the read
+    comm.moe_combine(win, C, w, Y)                                  # runs (the status is clear), on incomplete windows
+    assert comm.moe_status() == 0
+    comm.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 0)
+    win.zero_()
+    comm.moe_dispatch(X, win, C)
+    comm.moe_combine(win, C, w, Y)
+    assert comm.moe_status() == 0
+    assert np.array_equal(win.cpu().view(torch.int16).numpy().view(np.uint16), o.windows_zero_init)
+    assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), o.Y) <= 1
+    comm.close()
