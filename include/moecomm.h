@@ -159,6 +159,27 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* 
 moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows /*DEVICE*/, int64_t capacity_rows,
                          const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
 
+/* Multi-rank decomposition of the same path (one process and one context per expert-parallel rank,
+ * Section 5.2: Layout is local, Notify exchanges count metadata only, Dispatch places rows directly
+ * into the destination ranks' windows, Combine reads them directly from there).
+ *   moe_layout   plans THIS rank's tokens only: small offsets s and the rank's row of the count matrix,
+ *                copied to counts_row (DEVICE [E] int32) for the caller to all-gather over the group.
+ *   moe_notify   takes the gathered matrix counts_all (DEVICE [R,E] int32, row r from rank r) and builds
+ *                the large offsets and receive counts; the context is then planned.
+ *   moe_dispatch_peers / moe_combine_peers
+ *                as moe_dispatch / moe_combine for the local tokens, with the window of rank d at
+ *                window_bases[d] (DEVICE array of R DEVICE pointers, each [capacity_rows, H] bf16,
+ *                16-byte aligned): peer-mapped windows of the other GPUs, or separate allocations.
+ * The library launches no collective and waits for no peer: the caller orders the phases (all-gather
+ * of the counts between layout and notify; a barrier after dispatch and after the experts). */
+moe_status_t moe_layout(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE [T_local,K]*/,
+                        int32_t T_local, int32_t my_rank, int32_t* counts_row /*DEVICE*/, void* stream);
+moe_status_t moe_notify(moe_ctx_t* ctx, const int32_t* counts_all /*DEVICE*/, void* stream);
+moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/, const void* const* window_bases /*DEVICE*/,
+                                int64_t capacity_rows, void* stream);
+moe_status_t moe_combine_peers(moe_ctx_t* ctx, const void* const* window_bases /*DEVICE*/, int64_t capacity_rows,
+                               const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
+
 /* Materialises slot(t,j) into caller memory (parity checks, expert-side
  * consumers).  slots DEVICE [T,K] int32; needs R * capacity_rows < 2^31. */
 moe_status_t moe_slots(moe_ctx_t* ctx, int64_t capacity_rows, int32_t* slots /*DEVICE*/, void* stream);

@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_dispatch.argtypes = [p, i32, i32, i32, p, p, i32]
         L.oracle_expert_scale.argtypes = [p, i32, i32, i32, i64, p, p]
         L.oracle_combine.argtypes = [p, i32, i32, i32, p, p, p, i32]
+        L.oracle_notify.argtypes = [p, i32, i32, p, p, p, p]
+        L.oracle_notify.restype = ctypes.c_int
         L.oracle_gate_topk.argtypes = [p, i32, i32, i32, p, p]
         L.oracle_gate_topk.restype = ctypes.c_int
         L.oracle_expert_ranges.argtypes = [i32, i32, i64, p, p, p]
@@ -117,6 +119,18 @@ def slots(topk_idx, E: int, R: int, pl: Plan, C: int, rank_tok_start=None):
     st = lib().oracle_slots(_ptr(topk_idx), T, K, E, R, _ptr(rts), _ptr(pl.s), _ptr(pl.o), _ptr(pl.n_recv),
                             int(C), _ptr(out))
     return st, out
+
+
+def notify(M):
+    """Large offsets and receive counts from a gathered count matrix M [R,E]."""
+    M = _c(M, np.int32)
+    R, E = M.shape
+    c_rank = np.full((R, R), -7, np.int32)
+    o = np.full((E, R), -7, np.int32)
+    n_exp = np.full((E,), -7, np.int32)
+    n_recv = np.full((R,), -7, np.int32)
+    st = lib().oracle_notify(_ptr(M), E, R, _ptr(c_rank), _ptr(o), _ptr(n_exp), _ptr(n_recv))
+    return st, c_rank, o, n_exp, n_recv
 
 
 def gate_topk(logits, K: int):

@@ -148,33 +148,10 @@ int oracle_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32
   return ORACLE_OK;
 }
 
-int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
-                const int32_t* rank_tok_start,
-                int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
-                int32_t* n_exp, int32_t* n_recv) {
-  if (!shape_ok(T, K, E, R, rank_tok_start)) return ORACLE_ERR_INVALID_ARG;
-  if (T > 0 && topk_idx == nullptr) return ORACLE_ERR_INVALID_ARG;
+int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t* c_rank, int32_t* o, int32_t* n_exp,
+                  int32_t* n_recv) {
+  if (E < 1 || R < 1 || E % R != 0) return ORACLE_ERR_INVALID_ARG;
   const int32_t E_r = E / R;
-  const int64_t B = (int64_t)T * K;
-
-  // Routing indexes lie in {0..E-1} (Section 5.1); anything else is an error.
-  for (int64_t b = 0; b < B; ++b)
-    if (topk_idx[b] < 0 || topk_idx[b] >= E) return ORACLE_ERR_BAD_INDEX;
-
-  // Layout: one pass over branches in flat order (t, j).  run[r][e] is the
-  // number of branches of source rank r seen so far that chose expert e, so the
-  // value read before the increment is s[t,j]; its final value is M[r,e].
-  std::vector<int32_t> run((size_t)R * E, 0);
-  for (int32_t t = 0; t < T; ++t) {
-    const int32_t r = src_rank(rank_tok_start, R, t);
-    for (int32_t j = 0; j < K; ++j) {
-      const int32_t e = topk_idx[(int64_t)t * K + j];
-      s[(int64_t)t * K + j] = run[(size_t)r * E + e]++;
-    }
-  }
-  for (int32_t r = 0; r < R; ++r)
-    for (int32_t e = 0; e < E; ++e) M[(size_t)r * E + e] = run[(size_t)r * E + e];
-
   // Per-rank branch counts: c_rank[r,d] = sum over experts of rank d of M[r,e].
   for (int32_t r = 0; r < R; ++r)
     for (int32_t d = 0; d < R; ++d) {
@@ -202,6 +179,35 @@ int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_
     n_recv[d] = acc;
   }
   return ORACLE_OK;
+}
+
+int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
+                const int32_t* rank_tok_start,
+                int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
+                int32_t* n_exp, int32_t* n_recv) {
+  if (!shape_ok(T, K, E, R, rank_tok_start)) return ORACLE_ERR_INVALID_ARG;
+  if (T > 0 && topk_idx == nullptr) return ORACLE_ERR_INVALID_ARG;
+  const int64_t B = (int64_t)T * K;
+
+  // Routing indexes lie in {0..E-1} (Section 5.1); anything else is an error.
+  for (int64_t b = 0; b < B; ++b)
+    if (topk_idx[b] < 0 || topk_idx[b] >= E) return ORACLE_ERR_BAD_INDEX;
+
+  // Layout: one pass over branches in flat order (t, j).  run[r][e] is the
+  // number of branches of source rank r seen so far that chose expert e, so the
+  // value read before the increment is s[t,j]; its final value is M[r,e].
+  std::vector<int32_t> run((size_t)R * E, 0);
+  for (int32_t t = 0; t < T; ++t) {
+    const int32_t r = src_rank(rank_tok_start, R, t);
+    for (int32_t j = 0; j < K; ++j) {
+      const int32_t e = topk_idx[(int64_t)t * K + j];
+      s[(int64_t)t * K + j] = run[(size_t)r * E + e]++;
+    }
+  }
+  for (int32_t r = 0; r < R; ++r)
+    for (int32_t e = 0; e < E; ++e) M[(size_t)r * E + e] = run[(size_t)r * E + e];
+
+  return oracle_notify(M, E, R, c_rank, o, n_exp, n_recv);
 }
 
 int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,

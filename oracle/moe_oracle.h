@@ -57,6 +57,12 @@ int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_
                 int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
                 int32_t* n_exp, int32_t* n_recv);
 
+/* Notify on its own (Section 5.2, Prefill Notify): from the gathered count matrix M [R,E] -- in a
+ * real expert-parallel group every rank contributes its row -- the large offsets o [E,R], the
+ * receive counts n_exp [E], n_recv [R] and c_rank [R,R].  oracle_plan is Layout followed by this. */
+int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t* c_rank, int32_t* o, int32_t* n_exp,
+                  int32_t* n_recv);
+
 /* Expert-window row of every branch (two-level offset rule, Section 5.1; Algorithm 1):
  *   slot[t,j] = dst(e) * C + o[e, src(t)] + s[t,j],  e = K[t,j].
  * The windows of the R ranks are R equal segments of C rows of one allocation.

@@ -25,7 +25,7 @@ EXPORTS = [
     "moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_plan_view", "moe_dispatch",
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
-    "moe_gate_topk", "moe_gate_plan",
+    "moe_gate_topk", "moe_gate_plan", "moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS = 0, 1, 2
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -67,6 +67,12 @@ def load() -> ctypes.CDLL:
     L.moe_plan_view.argtypes = [vp, ctypes.POINTER(MoePlanView)]
     L.moe_dispatch.argtypes = [vp, vp, vp, i64, vp]
     L.moe_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.moe_layout.argtypes = [vp, ctypes.c_int, vp, i32, i32, vp, vp]
+    L.moe_notify.argtypes = [vp, vp, vp]
+    L.moe_dispatch_peers.argtypes = [vp, vp, vp, i64, vp]
+    L.moe_combine_peers.argtypes = [vp, vp, i64, vp, vp, vp]
+    for _n in ("moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers"):
+        getattr(L, _n).restype = ctypes.c_int
     L.moe_gate_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     L.moe_gate_topk.restype = ctypes.c_int
     L.moe_gate_plan.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp, vp, vp]
@@ -187,6 +193,46 @@ class MoeComm:
             self.T, self.schedule, self._keep = T, schedule, topk_idx
         elif check:
             raise MoeError(rc, "moe_gate_plan")
+        return rc
+
+    # -- multi-rank decomposition ---------------------------------------------------
+    def moe_layout(self, schedule: int, topk_idx: torch.Tensor, my_rank: int, counts_row: torch.Tensor,
+                   stream=None, check: bool = True) -> int:
+        T = topk_idx.shape[0]
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_layout(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, my_rank,
+                                     _dev_ptr(counts_row, torch.int32), _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx
+        elif check:
+            raise MoeError(rc, "moe_layout")
+        return rc
+
+    def moe_notify(self, counts_all: torch.Tensor, stream=None, check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_notify(self._h, _dev_ptr(counts_all, torch.int32), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_notify")
+        return rc
+
+    def moe_dispatch_peers(self, x: torch.Tensor, window_bases: torch.Tensor, capacity_rows: int, stream=None,
+                           check: bool = True) -> int:
+        """window_bases: int64 CUDA tensor [R] holding the device address of every rank's window."""
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_dispatch_peers(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(window_bases, torch.int64),
+                                             int(capacity_rows), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_peers")
+        return rc
+
+    def moe_combine_peers(self, window_bases: torch.Tensor, capacity_rows: int, topk_w: torch.Tensor, y: torch.Tensor,
+                          stream=None, check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_combine_peers(self._h, _dev_ptr(window_bases, torch.int64), int(capacity_rows),
+                                            _dev_ptr(topk_w, torch.float32), _dev_ptr(y, torch.bfloat16),
+                                            _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_combine_peers")
         return rc
 
     def moe_plan_view(self) -> dict:

@@ -148,7 +148,7 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
     }
     for (int j = 0; j < a.K; ++j) {
       const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-      if (lane == 0 && row >= 0) bulk_store(windows + (size_t)row * row_bytes + off, buf0 + s * stage_bytes, bytes, evict_first);
+      if (lane == 0 && row >= 0) bulk_store(window_row(a, windows, row, row_bytes) + off, buf0 + s * stage_bytes, bytes, evict_first);
     }
     if (lane == 0) {
       bulk_commit();

@@ -27,6 +27,7 @@ struct moe_ctx {
   int32_t *M, *c_rank, *o, *n_exp, *n_recv, *s, *tile_rank, *tile_hist;
   // plan state (host)
   bool planned;
+  bool layout_done;   // moe_layout has run; moe_notify may complete the plan
   bool compact_plan;  // plan done in one launch by plan_rank_kernel: small offsets are final after moe_plan
   moe_schedule_t schedule;
   int32_t T;
@@ -121,6 +122,7 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
+  a.win_base = nullptr;
   a.wait_limit_ms = ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT;
   a.test_starve = ctx->starve_wait_ms > 0;
   return a;
@@ -246,6 +248,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->tile_rank = reinterpret_cast<int32_t*>(ctx->ws + L.tile_rank);
   ctx->tile_hist = reinterpret_cast<int32_t*>(ctx->ws + L.tile_hist);
   ctx->planned = false;
+  ctx->layout_done = false;
   ctx->compact_plan = false;
   ctx->launches = 0;
   ctx->topk_idx = nullptr;
@@ -273,7 +276,8 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
            cudaSuccess;
     if (ok && scan_smem > 48 * 1024)
       ok = cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) ==
-           cudaSuccess;
+               cudaSuccess &&
+           cudaFuncSetAttribute(notify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) == cudaSuccess;
   }
   if (ok && tile_smem > 48 * 1024) {
     ok = cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_PREFILL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -327,6 +331,7 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
       if (rank_tok_start[r + 1] < rank_tok_start[r]) return MOE_ERR_INVALID_ARG;
   }
   ctx->planned = false;
+  ctx->layout_done = false;
 
   const int rounds = schedule == MOE_SCHED_PREFILL ? ROUNDS_PREFILL : ROUNDS_DECODE;
   const int tile_branches = rounds * PLAN_THREADS;
@@ -445,13 +450,19 @@ moe_status_t moe_plan_view(const moe_ctx_t* c, moe_plan_view_t* out) {
   return MOE_OK;
 }
 
-moe_status_t moe_dispatch(moe_ctx_t* c, const void* x, void* windows, int64_t capacity_rows, void* stream) {
-  moe_ctx* ctx = c;
+}  // extern "C"
+
+namespace {
+
+moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const void* const* bases, int64_t capacity_rows,
+                           void* stream) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
-  if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || windows == nullptr))) return MOE_ERR_INVALID_ARG;
+  if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || (windows == nullptr && bases == nullptr))))
+    return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(windows)) return MOE_ERR_INVALID_ARG;
   RowArgs a = row_args(ctx, capacity_rows, true);
+  a.win_base = reinterpret_cast<const unsigned char* const*>(bases);
   a.topk_idx = ctx->topk_idx;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* xs = static_cast<const uint4*>(x);
@@ -469,6 +480,21 @@ moe_status_t moe_dispatch(moe_ctx_t* c, const void* x, void* windows, int64_t ca
     }
   }
   return launch_ok(ctx);
+}
+
+}  // namespace
+
+extern "C" {
+
+moe_status_t moe_dispatch(moe_ctx_t* ctx, const void* x, void* windows, int64_t capacity_rows, void* stream) {
+  if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
+  return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream);
+}
+
+moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x, const void* const* window_bases, int64_t capacity_rows,
+                                void* stream) {
+  if (window_bases == nullptr) return MOE_ERR_INVALID_ARG;
+  return dispatch_impl(ctx, x, nullptr, window_bases, capacity_rows, stream);
 }
 
 moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, float* scales, int64_t capacity_rows,
@@ -501,15 +527,20 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, fl
   return launch_ok(ctx);
 }
 
-moe_status_t moe_combine(moe_ctx_t* c, const void* windows, int64_t capacity_rows, const float* topk_w, void* y,
-                         void* stream) {
-  moe_ctx* ctx = c;
+}  // extern "C"
+
+namespace {
+
+moe_status_t combine_impl(moe_ctx* ctx, const void* windows, const void* const* bases, int64_t capacity_rows,
+                          const float* topk_w, void* y, void* stream) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
-  if (capacity_rows < 0 || (ctx->T > 0 && (windows == nullptr || topk_w == nullptr || y == nullptr)))
+  if (capacity_rows < 0 ||
+      (ctx->T > 0 && ((windows == nullptr && bases == nullptr) || topk_w == nullptr || y == nullptr)))
     return MOE_ERR_INVALID_ARG;
   if (!aligned16(windows) || !aligned16(y)) return MOE_ERR_INVALID_ARG;
   RowArgs a = row_args(ctx, capacity_rows, false);
+  a.win_base = reinterpret_cast<const unsigned char* const*>(bases);
   a.topk_idx = ctx->topk_idx;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* win = static_cast<const uint4*>(windows);
@@ -523,6 +554,50 @@ moe_status_t moe_combine(moe_ctx_t* c, const void* windows, int64_t capacity_row
     default: launch_combine<0>(ctx, a, win, topk_w, ys, st); break;
   }
   return launch_ok(ctx);
+}
+
+}  // namespace
+
+extern "C" {
+
+moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows, int64_t capacity_rows, const float* topk_w, void* y,
+                         void* stream) {
+  if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
+  return combine_impl(ctx, windows, nullptr, capacity_rows, topk_w, y, stream);
+}
+
+moe_status_t moe_combine_peers(moe_ctx_t* ctx, const void* const* window_bases, int64_t capacity_rows,
+                               const float* topk_w, void* y, void* stream) {
+  if (window_bases == nullptr) return MOE_ERR_INVALID_ARG;
+  return combine_impl(ctx, nullptr, window_bases, capacity_rows, topk_w, y, stream);
+}
+
+/* Multi-rank decomposition: Layout for one rank's tokens, Notify from the gathered counts. */
+moe_status_t moe_layout(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T_local,
+                        int32_t my_rank, int32_t* counts_row, void* stream) {
+  if (ctx == nullptr || my_rank < 0 || my_rank >= ctx->shape.R || counts_row == nullptr) return MOE_ERR_INVALID_ARG;
+  if (T_local > 0 && topk_idx == nullptr) return MOE_ERR_INVALID_ARG;
+  int32_t starts[MOE_MAX_R + 1];
+  for (int r = 0; r <= ctx->shape.R; ++r) starts[r] = r <= my_rank ? 0 : T_local;   // only my_rank owns tokens
+  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T_local, starts, stream, nullptr, nullptr, nullptr);
+  if (rc != MOE_OK) return rc;
+  ctx->planned = false;   // the offsets are not valid until moe_notify has seen every rank's counts
+  if (cudaMemcpyAsync(counts_row, ctx->M + (size_t)my_rank * ctx->shape.E, sizeof(int32_t) * ctx->shape.E,
+                      cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  ctx->layout_done = true;
+  return MOE_OK;
+}
+
+moe_status_t moe_notify(moe_ctx_t* ctx, const int32_t* counts_all, void* stream) {
+  if (ctx == nullptr || counts_all == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->layout_done) return MOE_ERR_NOT_PLANNED;
+  const moe_shape_t& sh = ctx->shape;
+  notify_kernel<<<1, 1024, notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t), static_cast<cudaStream_t>(stream)>>>(
+      counts_all, sh.E, sh.R, ctx->schedule == MOE_SCHED_PREFILL, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv);
+  const moe_status_t rc = launch_ok(ctx);
+  if (rc == MOE_OK) ctx->planned = true;
+  return rc;
 }
 
 moe_status_t moe_slots(moe_ctx_t* c, int64_t capacity_rows, int32_t* slots, void* stream) {
@@ -752,6 +827,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
+  a.win_base = nullptr;
   a.wait_limit_ms = WAIT_LIMIT_MS_DEFAULT;
   a.test_starve = 0;
   int grid = (int)(((int64_t)T * K + 255) / 256);

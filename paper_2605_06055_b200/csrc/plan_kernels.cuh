@@ -362,6 +362,19 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   if (threadIdx.x == 0) ctl->scan_ticket = 0;
 }
 
+// Notify from a count matrix gathered elsewhere (multi-rank use: every rank contributed its row):
+// installs it as M and rebuilds the large offsets and receive counts.  One CTA.
+__global__ void __launch_bounds__(1024)
+notify_kernel(const int32_t* __restrict__ counts_all, int32_t E, int32_t R, int32_t full_table,
+              int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+              int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
+  extern __shared__ int32_t sm[];
+  for (int i = threadIdx.x; i < R * E; i += blockDim.x) M[i] = counts_all[i];
+  __threadfence_block();
+  __syncthreads();
+  build_large_offsets(M, E, R, full_table, c_rank, o, n_exp, n_recv, sm);
+}
+
 template <int ROUNDS>
 __global__ void __launch_bounds__(PLAN_THREADS)
 plan_finalize_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,

@@ -29,6 +29,9 @@ struct RowArgs {
   int32_t granule;           // units (512-byte slabs) per work item
   int32_t items_per_row;     // ceil(units per row / granule)
   int32_t n_items;           // T * items_per_row
+  // Multi-rank use: window segment d starts at win_base[d] (device array of R device pointers, e.g. peer
+  // mappings of every rank's window); nullptr = one allocation of R consecutive segments of C rows.
+  const unsigned char* const* win_base;
   int32_t wait_limit_ms;     // bound of every device-side wait
   int32_t test_starve;       // test hook of the bulk-copy dispatch: make one wait run out
 };
@@ -48,6 +51,14 @@ __device__ __forceinline__ int64_t resolve_slot(const RowArgs& a, const RankMap&
     if (record) a.small_out[b] = so;
   }
   return (int64_t)(e / a.E_r) * a.C + __ldg(a.large_off + (size_t)e * a.R + r) + so;
+}
+
+// Address of window row `row` (global numbering d*C + local row).
+__device__ __forceinline__ unsigned char* window_row(const RowArgs& a, const void* windows, int64_t row,
+                                                     size_t row_bytes) {
+  if (a.win_base == nullptr) return (unsigned char*)windows + (size_t)row * row_bytes;
+  const int64_t d = row / a.C;
+  return (unsigned char*)a.win_base[d] + (size_t)(row - d * a.C) * row_bytes;
 }
 
 // True when the call must not touch payload memory: an earlier error is pending
@@ -179,7 +190,7 @@ dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, c
 #pragma unroll
       for (int j = 0; j < KT; ++j) {
         const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-        dst[j] = row >= 0 ? windows + (size_t)row * H16 : nullptr;
+        dst[j] = row >= 0 ? reinterpret_cast<uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
       }
       for (int i = w.i0; i < w.i1; i += UNROLL) {
         uint4 v[UNROLL];
@@ -205,7 +216,7 @@ dispatch_rows_kernel(const uint4* __restrict__ X, uint4* __restrict__ windows, c
         if (c < H16) v = ld_stream(src + c);
         for (int j = 0; j < K; ++j) {
           const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-          if (row >= 0 && c < H16) st_stream(windows + (size_t)row * H16 + c, v);
+          if (row >= 0 && c < H16) st_stream(reinterpret_cast<uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) + c, v);
         }
       }
     }
@@ -260,7 +271,7 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
 #pragma unroll
       for (int j = 0; j < KT; ++j) {
         const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-        src[j] = row >= 0 ? windows + (size_t)row * H16 : nullptr;
+        src[j] = row >= 0 ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
         w[j] = __shfl_sync(0xffffffffu, w_lane, j);
       }
       for (int i = wi.i0; i < wi.i1; i += UNROLL) {
@@ -302,7 +313,8 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
             const int j = jc + jj;
             const int64_t row = __shfl_sync(0xffffffffu, slot, j & 31);
             wv[jj] = __shfl_sync(0xffffffffu, w_lane, j & 31);
-            const uint4* src = (j < K && row >= 0) ? windows + (size_t)row * H16 : nullptr;
+            const uint4* src =
+                (j < K && row >= 0) ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u)
               v[u][jj] = (ok[u] && src != nullptr) ? ld_row<L1_ALLOC>(src + (i + u) * 32 + lane)

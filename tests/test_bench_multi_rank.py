@@ -45,3 +45,21 @@ def test_algorithmic_bytes_match_the_stated_formulas():
     assert bench.bytes_dispatch(wl) == 2 * 7168 * 32768 * 9 + 8 * 32768 * 8 + 4 * 256 * 8 == 4229963776
     assert bench.bytes_combine(wl) == 2 * 7168 * 32768 * 9 + 12 * 32768 * 8 + 4 * 256 * 8
     assert round(bench.bytes_dispatch(bench.WORKLOADS["c2"]()) / 1e6, 1) == 264.4
+
+
+def _gather_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    from paper_2605_06055_b200 import ep
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    row = torch.arange(6, dtype=torch.int32) + 100 * rank          # this rank's row of the count matrix
+    out[rank] = ep.all_gather_counts(row).tolist()
+    dist.destroy_process_group()
+
+
+def test_count_exchange_between_two_ranks_builds_the_same_matrix_everywhere():
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_gather_worker, args=(world, 31000 + os.getpid() % 2000, out), nprocs=world, join=True)
+        want = [[0, 1, 2, 3, 4, 5], [100, 101, 102, 103, 104, 105]]
+        assert out[0] == want and out[1] == want

@@ -1,0 +1,78 @@
+"""The multi-rank decomposition (moe_layout -> gather counts -> moe_notify -> moe_dispatch_peers ->
+experts -> moe_combine_peers) on ONE GPU: every expert-parallel rank gets its own context, its own
+token slice and its own window allocation, as R processes on R GPUs would have; the calls run one rank
+after the other (they never wait on one another).  The union of the windows and the outputs must be
+bit-identical to the oracle's single global result.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06055_b200 import binding, synth
+from paper_2605_06055_b200.synth import DECODE, PREFILL, Workload
+
+import harness
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    ("decode_like", 1024, 1024, 64, 8, 8, DECODE, "uniform", None),
+    ("prefill_ragged", 3000, 512, 32, 4, 4, PREFILL, "uniform", (1000, 0, 1500, 500)),
+    ("large_rank_tile_path", 6000, 64, 16, 2, 2, PREFILL, "replace", (5000, 1000)),
+    ("large_rank_tile_path_decode", 6000, 64, 16, 2, 2, DECODE, "replace", (5000, 1000)),
+    ("generic_k", 500, 264, 12, 3, 3, DECODE, "replace", (100, 150, 250)),
+]
+
+
+@pytest.mark.parametrize("path", [binding.MOE_DISPATCH_BULK, binding.MOE_DISPATCH_REGISTERS])
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_per_rank_contexts_and_separate_windows_reproduce_the_global_result(case, path):
+    name, T, H, E, R, K, sch, routing, per = case
+    dev = torch.device("cuda:0")
+    wl = Workload(name, T, H, E, R, K, sch, routing, "scale", 7000 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    rts = inp.rank_tok_start
+    p = oracle.plan(inp.topk_idx.numpy(), E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    want = harness.oracle_run(inp, C)
+
+    idx, w, X = inp.topk_idx.to(dev), inp.topk_w.to(dev), inp.X.to(dev)
+    comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
+    for c in comms:
+        c.moe_set_option(binding.MOE_OPT_DISPATCH_PATH, path)
+    # Layout on every rank, then the count "all-gather" (here: rows of one tensor), then Notify on every rank
+    counts = torch.full((R, E), -1, dtype=torch.int32, device=dev)
+    for r, c in enumerate(comms):
+        assert c.moe_dispatch_peers(X[:0], torch.zeros(R, dtype=torch.int64, device=dev), C, check=False) == \
+            binding.MOE_ERR_NOT_PLANNED
+        c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, counts[r])
+    assert np.array_equal(counts.cpu().numpy(), p.M)
+    for c in comms:
+        c.moe_notify(counts)
+    # one window allocation per rank, addressed through a base-pointer table
+    windows = [torch.from_numpy(np.full((C, H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+               for _ in range(R)]
+    bases = torch.tensor([wd.data_ptr() for wd in windows], dtype=torch.int64, device=dev)
+    for r, c in enumerate(comms):
+        c.moe_dispatch_peers(X[rts[r]:rts[r + 1]].contiguous(), bases, C)
+        assert c.moe_status() == 0
+        v = c.moe_plan_view()
+        assert np.array_equal(v["large_off"].cpu().numpy(), p.o) and np.array_equal(v["n_recv"].cpu().numpy(), p.n_recv)
+        assert np.array_equal(v["small_off"].cpu().numpy(), p.s[rts[r]:rts[r + 1]])
+    got = torch.cat(windows).cpu().view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(got, want.windows)
+    # experts (harness op on the concatenated view), then every rank combines its own tokens from all windows
+    allwin = torch.cat(windows)
+    harness.gpu_expert_scale(allwin, idx, E, R, C, inp.scale.to(dev))
+    for d in range(R):
+        windows[d].copy_(allwin[d * C:(d + 1) * C])
+    Y = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
+    for r, c in enumerate(comms):
+        y_r = torch.empty((int(rts[r + 1] - rts[r]), H), dtype=torch.bfloat16, device=dev)
+        c.moe_combine_peers(bases, C, w[rts[r]:rts[r + 1]].contiguous(), y_r)
+        assert c.moe_status() == 0
+        Y[rts[r]:rts[r + 1]] = y_r
+    assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
+    for c in comms:
+        c.close()

@@ -545,3 +545,27 @@ def test_gate_topk_ties_take_the_lower_index_first():
     assert idx.tolist() == want == [[1, 2, 4, 5], [0, 1, 2, 3], [2, 3, 5, 0]]
     assert np.allclose(w[1], 0.25) and w[0, 0] == w[0, 1] == w[0, 2]
     assert oracle.gate_topk(logits, 7)[0] == oracle.ERR_INVALID_ARG   # K > E
+
+
+# ----------------------------------------------------------------------------- multi-rank decomposition
+def test_layout_per_rank_plus_notify_equals_the_global_plan():
+    """Layout is local (Section 5.2): planning each rank's tokens alone gives that rank's row of M and
+    its small offsets; Notify on the gathered rows gives the global large offsets."""
+    rng = np.random.default_rng(12)
+    T, K, E, R = 300, 4, 12, 4
+    idx, rts = random_case(rng, T, K, E, R, replace=True)
+    whole = oracle.plan(idx, E, R, rts)
+    rows = []
+    for r in range(R):
+        local = idx[rts[r]:rts[r + 1]]
+        only_r = np.array([0] * (r + 1) + [len(local)] * (R - r), np.int32)     # rank r owns every local token
+        pr = oracle.plan(local, E, R, only_r)
+        assert pr.status == oracle.OK
+        assert np.array_equal(pr.s, whole.s[rts[r]:rts[r + 1]])
+        assert not np.delete(pr.M, r, axis=0).any()
+        rows.append(pr.M[r])
+    M = np.stack(rows)
+    st, c_rank, o, n_exp, n_recv = oracle.notify(M)
+    assert st == oracle.OK and np.array_equal(M, whole.M)
+    for a, b in ((c_rank, whole.c_rank), (o, whole.o), (n_exp, whole.n_exp), (n_recv, whole.n_recv)):
+        assert np.array_equal(a, b)
