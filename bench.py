@@ -316,26 +316,6 @@ def time_dispatch_quant(layer: Layer, steps: int, scratch=None):
     return [a.elapsed_time(b) * 1e3 for a, b in ev]
 
 
-def time_graph_steps(layer: Layer, steps: int, scratch=None):
-    """The same step captured once in a CUDA graph and replayed (what a decode loop would do)."""
-    g = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g):
-        layer.step()
-    for _ in range(3):
-        g.replay()
-    torch.cuda.synchronize()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in ev:
-        if scratch is not None:
-            scratch.add_(1)
-        a.record()
-        g.replay()
-        b.record()
-    torch.cuda.synchronize()
-    assert layer.comm.moe_status() == 0
-    return [a.elapsed_time(b) * 1e3 for a, b in ev]
-
-
 def time_e2e(layer: Layer, steps: int, barrier):
     """Whole layer through the C ABI from pinned HOST buffers: H2D of X, K, W and D2H of Y every step."""
     wl, c = layer.wl, layer.comm

@@ -4,9 +4,11 @@
 // Algorithm 1 / Algorithm 2 of the paper.  A warp works on (part of) one token
 // row at a time: lane j < K resolves branch (t, j) to its window row with the
 // two-level offset rule slot = dst(e)*C + o[e, src(t)] + s[t,j]; then the whole
-// warp moves its share of the row in 16-byte chunks.  Dispatch reads X[t,:] from HBM exactly once and
-// stores it K times; combine issues the K loads of a chunk before its
-// j-ordered fma chain.  There is no relay, permute or unpermute buffer.
+// warp moves its share of the row in 16-byte chunks.  Dispatch reads X[t,:] from
+// HBM exactly once and stores it K times; combine issues the K loads of a chunk
+// before its j-ordered fma chain.  There is no relay, permute or unpermute
+// buffer.  (The default dispatch is the bulk-copy kernel in bulk_kernels.cuh;
+// dispatch_rows_kernel here is the register path.)
 #pragma once
 
 #include "common.cuh"
@@ -15,9 +17,9 @@ namespace moe {
 
 struct RowArgs {
   const int32_t* topk_idx;   // [T,K]
-  const int32_t* small_off;  // PREFILL: s [T,K].  DECODE: in-tile rank [T,K]
-  int32_t* small_out;        // DECODE dispatch: where delta is recorded; else nullptr
-  const int32_t* tile_base;  // DECODE: [tiles,E] exclusive tile bases; PREFILL: nullptr
+  const int32_t* small_off;  // final small offsets s [T,K]; tile-planned DECODE: in-tile rank [T,K]
+  int32_t* small_out;        // tile-planned DECODE dispatch: where delta is recorded; else nullptr
+  const int32_t* tile_base;  // tile-planned DECODE: [tiles,E] exclusive tile bases; else nullptr
   const int32_t* large_off;  // o [E,R]
   const int32_t* n_recv;     // [R]
   int32_t* status;
