@@ -159,6 +159,15 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* 
 moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows /*DEVICE*/, int64_t capacity_rows,
                          const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
 
+/* Token sub-ranges of a plan: the same as moe_dispatch / moe_combine for tokens t_begin <= t < t_end
+ * only (x and y are still the full [T,H] tensors).  Chunks of a prefill batch can so be dispatched as
+ * they arrive and combined as their experts finish; any partition of [0,T) gives the same bytes. */
+moe_status_t moe_dispatch_range(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows /*DEVICE*/,
+                                int64_t capacity_rows, int32_t t_begin, int32_t t_end, void* stream);
+moe_status_t moe_combine_range(moe_ctx_t* ctx, const void* windows /*DEVICE*/, int64_t capacity_rows,
+                               const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, int32_t t_begin, int32_t t_end,
+                               void* stream);
+
 /* Multi-rank decomposition of the same path (one process and one context per expert-parallel rank,
  * Section 5.2: Layout is local, Notify exchanges count metadata only, Dispatch places rows directly
  * into the destination ranks' windows, Combine reads them directly from there).
@@ -193,8 +202,11 @@ moe_status_t moe_expert_ranges(moe_ctx_t* ctx, int64_t capacity_rows, int64_t* r
                                int32_t* row_count /*DEVICE*/, void* stream);
 
 /* One whole layer call from HOST buffers, enqueued on `stream`:
- * host->device copies of x, topk_idx, topk_w; plan; dispatch; combine reading
- * the dispatched windows (identity experts); device->host copy of y.
+ * host->device copies of topk_idx, topk_w; plan; then, in sixteen token chunks, host->device copy
+ * of the chunk of x (upload stream), dispatch and combine reading the dispatched windows (identity
+ * experts; caller's stream), and the device->host copy of the chunk of y (download stream), so both
+ * copy directions and the kernels overlap.  The two extra streams belong to the context and are
+ * created on first use.  `stream` finishes only after the last download.
  * The *_dev arguments are caller-owned DEVICE staging buffers of the shapes
  * given above.  Pass pinned host memory for the copies to be asynchronous.
  * rank_tok_start as in moe_plan.  Call moe_status() to wait for the result. */

@@ -26,6 +26,7 @@ EXPORTS = [
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
     "moe_gate_topk", "moe_gate_plan", "moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers",
+    "moe_dispatch_range", "moe_combine_range",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS = 0, 1, 2
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -67,6 +68,9 @@ def load() -> ctypes.CDLL:
     L.moe_plan_view.argtypes = [vp, ctypes.POINTER(MoePlanView)]
     L.moe_dispatch.argtypes = [vp, vp, vp, i64, vp]
     L.moe_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.moe_dispatch_range.argtypes = [vp, vp, vp, i64, i32, i32, vp]
+    L.moe_combine_range.argtypes = [vp, vp, i64, vp, vp, i32, i32, vp]
+    L.moe_dispatch_range.restype = L.moe_combine_range.restype = ctypes.c_int
     L.moe_layout.argtypes = [vp, ctypes.c_int, vp, i32, i32, vp, vp]
     L.moe_notify.argtypes = [vp, vp, vp]
     L.moe_dispatch_peers.argtypes = [vp, vp, vp, i64, vp]
@@ -193,6 +197,25 @@ class MoeComm:
             self.T, self.schedule, self._keep = T, schedule, topk_idx
         elif check:
             raise MoeError(rc, "moe_gate_plan")
+        return rc
+
+    def moe_dispatch_range(self, x, windows, capacity_rows: int, t_begin: int, t_end: int, stream=None,
+                           check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_dispatch_range(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(windows, torch.bfloat16),
+                                             int(capacity_rows), t_begin, t_end, _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_range")
+        return rc
+
+    def moe_combine_range(self, windows, capacity_rows: int, topk_w, y, t_begin: int, t_end: int, stream=None,
+                          check: bool = True) -> int:
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_combine_range(self._h, _dev_ptr(windows, torch.bfloat16), int(capacity_rows),
+                                            _dev_ptr(topk_w, torch.float32), _dev_ptr(y, torch.bfloat16),
+                                            t_begin, t_end, _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_combine_range")
         return rc
 
     # -- multi-rank decomposition ---------------------------------------------------

@@ -38,6 +38,9 @@ struct moe_ctx {
   int32_t dispatch_path;    // MOE_OPT_DISPATCH_PATH
   int32_t granule_override; // MOE_OPT_GRANULE
   int32_t starve_wait_ms;   // MOE_OPT_TEST_STARVE_WAIT_MS
+  cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
+  cudaStream_t in_stream;
+  cudaEvent_t fwd_events[2 * 16 + 2];
 };
 
 namespace {
@@ -46,6 +49,7 @@ namespace {
 constexpr int64_t RANK_PLAN_MAX_BRANCHES = 4096;
 constexpr int RANK_PLAN_WIDE_MAX_E = 768;   // 32-warp CTAs while 33*E counters fit comfortably in shared memory
 
+constexpr int FWD_CHUNKS = 16;  // token chunks of moe_forward_host's upload / compute / download pipeline
 constexpr size_t ALIGN = 256;
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
@@ -123,6 +127,8 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.items_per_row = 0;
   a.n_items = 0;
   a.win_base = nullptr;
+  a.t_begin = 0;
+  a.t_count = ctx->T;
   a.wait_limit_ms = ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT;
   a.test_starve = ctx->starve_wait_ms > 0;
   return a;
@@ -135,8 +141,9 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
   const int upr = (a.H16 + 31) / 32;
   int64_t g = upr < max_granule ? upr : max_granule;
   int64_t pieces = (upr + g - 1) / g;
-  if ((int64_t)ctx->T * pieces < nwarps && ctx->T > 0) {
-    pieces = (nwarps + ctx->T - 1) / ctx->T;
+  const int64_t tokens = a.t_count;
+  if (tokens * pieces < nwarps && tokens > 0) {
+    pieces = (nwarps + tokens - 1) / tokens;
     if (pieces > upr) pieces = upr;
     g = (upr + pieces - 1) / pieces;
   }
@@ -144,10 +151,10 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
   if (g > max_granule) g = max_granule;
   if (g > upr) g = upr;
   if (g < 1) g = 1;
-  while (((int64_t)ctx->T * ((upr + g - 1) / g)) > ((int64_t)1 << 30) && g < upr) ++g;   // n_items stays in int32
+  while ((tokens * ((upr + g - 1) / g)) > ((int64_t)1 << 30) && g < upr) ++g;   // n_items stays in int32
   a.granule = (int32_t)g;
   a.items_per_row = (int32_t)((upr + g - 1) / g);
-  a.n_items = (int32_t)((int64_t)ctx->T * a.items_per_row);
+  a.n_items = (int32_t)(tokens * a.items_per_row);
   a.work = &ctx->ctl->work;
   a.work_done = &ctx->ctl->work_done;
 }
@@ -155,13 +162,13 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
 // One persistent wave: as many CTAs as fit on the device at once (from the occupancy calculator),
 // but no more warps than there are 512-byte units of work.
 template <class Kernel>
-int row_grid(const moe_ctx* ctx, Kernel kernel) {
+int row_grid(const moe_ctx* ctx, Kernel kernel, int64_t tokens) {
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0) != cudaSuccess || per_sm < 1) {
     cudaGetLastError();
     per_sm = 2;
   }
-  const int64_t units = (int64_t)ctx->T * ((ctx->shape.H / 8 + 31) / 32);
+  const int64_t units = tokens * ((ctx->shape.H / 8 + 31) / 32);
   const int64_t need = (units + 7) / 8;
   const int64_t cap = (int64_t)ctx->num_sms * per_sm;
   return (int)(need < cap ? (need < 1 ? 1 : need) : cap);
@@ -176,7 +183,7 @@ constexpr int DISPATCH_UNROLL = 14;
 template <int KT>
 void launch_dispatch_regs(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
   auto kernel = dispatch_rows_kernel<KT, (KT > 0 ? DISPATCH_UNROLL : 1)>;
-  const int grid = row_grid(ctx, kernel);
+  const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
   kernel<<<grid, 256, 0, st>>>(x, win, b, ctx->map);
@@ -202,10 +209,10 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
 template <int KT>
 void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const float* w, uint4* y, cudaStream_t st) {
   // Jobs that read several times the L2 capacity take the L1-allocating loads (see ld_row).
-  const bool large = (int64_t)ctx->T * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
+  const bool large = (int64_t)a.t_count * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
   auto kernel = large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), true>
                       : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), false>;
-  const int grid = row_grid(ctx, kernel);
+  const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
   kernel<<<grid, 256, 0, st>>>(win, w, y, b, ctx->map);
@@ -255,6 +262,8 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->dispatch_path = MOE_DISPATCH_AUTO;
   ctx->granule_override = 0;
   ctx->starve_wait_ms = 0;
+  ctx->out_stream = nullptr;
+  ctx->in_stream = nullptr;
 
   // Shared memory of the planning kernels grows with E; opt in above 48 KB.
   const int tile_smem = PLAN_WARPS * shape->E * (int)sizeof(int32_t);
@@ -296,6 +305,13 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
 
 moe_status_t moe_destroy(moe_ctx_t* ctx) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (ctx->out_stream != nullptr) {
+    cudaStreamSynchronize(ctx->out_stream);
+    cudaStreamSynchronize(ctx->in_stream);
+    for (int i = 0; i < 2 * FWD_CHUNKS + 2; ++i) cudaEventDestroy(ctx->fwd_events[i]);
+    cudaStreamDestroy(ctx->out_stream);
+    cudaStreamDestroy(ctx->in_stream);
+  }
   delete ctx;
   return MOE_OK;
 }
@@ -455,14 +471,18 @@ moe_status_t moe_plan_view(const moe_ctx_t* c, moe_plan_view_t* out) {
 namespace {
 
 moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const void* const* bases, int64_t capacity_rows,
-                           void* stream) {
+                           void* stream, int32_t t_begin = 0, int32_t t_end = -1) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
   if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || (windows == nullptr && bases == nullptr))))
     return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(windows)) return MOE_ERR_INVALID_ARG;
+  if (t_end < 0) t_end = ctx->T;
+  if (t_begin < 0 || t_begin > t_end || t_end > ctx->T) return MOE_ERR_INVALID_ARG;
   RowArgs a = row_args(ctx, capacity_rows, true);
   a.win_base = reinterpret_cast<const unsigned char* const*>(bases);
+  a.t_begin = t_begin;
+  a.t_count = t_end - t_begin;
   a.topk_idx = ctx->topk_idx;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* xs = static_cast<const uint4*>(x);
@@ -489,6 +509,13 @@ extern "C" {
 moe_status_t moe_dispatch(moe_ctx_t* ctx, const void* x, void* windows, int64_t capacity_rows, void* stream) {
   if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
   return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream);
+}
+
+moe_status_t moe_dispatch_range(moe_ctx_t* ctx, const void* x, void* windows, int64_t capacity_rows, int32_t t_begin,
+                                int32_t t_end, void* stream) {
+  if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
+  if (t_end < 0) return MOE_ERR_INVALID_ARG;
+  return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream, t_begin, t_end);
 }
 
 moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x, const void* const* window_bases, int64_t capacity_rows,
@@ -532,15 +559,19 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, fl
 namespace {
 
 moe_status_t combine_impl(moe_ctx* ctx, const void* windows, const void* const* bases, int64_t capacity_rows,
-                          const float* topk_w, void* y, void* stream) {
+                          const float* topk_w, void* y, void* stream, int32_t t_begin = 0, int32_t t_end = -1) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
   if (capacity_rows < 0 ||
       (ctx->T > 0 && ((windows == nullptr && bases == nullptr) || topk_w == nullptr || y == nullptr)))
     return MOE_ERR_INVALID_ARG;
   if (!aligned16(windows) || !aligned16(y)) return MOE_ERR_INVALID_ARG;
+  if (t_end < 0) t_end = ctx->T;
+  if (t_begin < 0 || t_begin > t_end || t_end > ctx->T) return MOE_ERR_INVALID_ARG;
   RowArgs a = row_args(ctx, capacity_rows, false);
   a.win_base = reinterpret_cast<const unsigned char* const*>(bases);
+  a.t_begin = t_begin;
+  a.t_count = t_end - t_begin;
   a.topk_idx = ctx->topk_idx;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* win = static_cast<const uint4*>(windows);
@@ -564,6 +595,13 @@ moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows, int64_t capacity_r
                          void* stream) {
   if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
   return combine_impl(ctx, windows, nullptr, capacity_rows, topk_w, y, stream);
+}
+
+moe_status_t moe_combine_range(moe_ctx_t* ctx, const void* windows, int64_t capacity_rows, const float* topk_w, void* y,
+                               int32_t t_begin, int32_t t_end, void* stream) {
+  if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
+  if (t_end < 0) return MOE_ERR_INVALID_ARG;
+  return combine_impl(ctx, windows, nullptr, capacity_rows, topk_w, y, stream, t_begin, t_end);
 }
 
 moe_status_t moe_combine_peers(moe_ctx_t* ctx, const void* const* window_bases, int64_t capacity_rows,
@@ -639,17 +677,51 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
   const size_t row_bytes = (size_t)ctx->shape.H * 2, B = (size_t)T * ctx->shape.K;
   if (T > 0) {
     if (cudaMemcpyAsync(topk_idx_dev, topk_idx_host, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(topk_w_dev, topk_w_host, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(x_dev, x_host, (size_t)T * row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        cudaMemcpyAsync(topk_w_dev, topk_w_host, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
   moe_status_t rc = moe_plan(ctx, schedule, topk_idx_dev, T, rank_tok_start, stream);
-  if (rc != MOE_OK) return rc;
-  rc = moe_dispatch(ctx, x_dev, windows_dev, capacity_rows, stream);
-  if (rc != MOE_OK) return rc;
-  rc = moe_combine(ctx, windows_dev, capacity_rows, topk_w_dev, y_dev, stream);
-  if (rc != MOE_OK) return rc;
-  if (T > 0 && cudaMemcpyAsync(y_host, y_dev, (size_t)T * row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+  if (rc != MOE_OK || T == 0) return rc;
+
+  // Token chunks flow through a three-stream pipeline: an upload stream copies chunk c of x to the
+  // device, the caller's stream dispatches and combines it (identity experts: a token's output needs
+  // only its own rows), and a download stream copies its outputs back, so both copy directions and the
+  // kernels overlap.  Nothing here allocates device memory; streams and events are created on first use.
+  if (ctx->out_stream == nullptr) {
+    if (cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->in_stream, cudaStreamNonBlocking) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    for (int i = 0; i < 2 * FWD_CHUNKS + 2; ++i)
+      if (cudaEventCreateWithFlags(&ctx->fwd_events[i], cudaEventDisableTiming) != cudaSuccess) return MOE_ERR_CUDA;
+  }
+  cudaEvent_t* up = ctx->fwd_events;                      // [c]: chunk c uploaded
+  cudaEvent_t* done = ctx->fwd_events + FWD_CHUNKS;       // [c]: chunk c combined
+  cudaEvent_t start = ctx->fwd_events[2 * FWD_CHUNKS], finish = ctx->fwd_events[2 * FWD_CHUNKS + 1];
+  const int chunks = T >= 4 * FWD_CHUNKS ? FWD_CHUNKS : 1;
+  char* xd = static_cast<char*>(x_dev);
+  const char* xh = static_cast<const char*>(x_host);
+  char* yd = static_cast<char*>(y_dev);
+  char* yh = static_cast<char*>(y_host);
+  // Uploads may overwrite x_dev only after everything enqueued before this call has used it.
+  if (cudaEventRecord(start, st) != cudaSuccess || cudaStreamWaitEvent(ctx->in_stream, start, 0) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  for (int c = 0; c < chunks; ++c) {
+    const int32_t t0 = (int32_t)((int64_t)T * c / chunks), t1 = (int32_t)((int64_t)T * (c + 1) / chunks);
+    if (cudaMemcpyAsync(xd + t0 * row_bytes, xh + t0 * row_bytes, (size_t)(t1 - t0) * row_bytes, cudaMemcpyHostToDevice,
+                        ctx->in_stream) != cudaSuccess ||
+        cudaEventRecord(up[c], ctx->in_stream) != cudaSuccess || cudaStreamWaitEvent(st, up[c], 0) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    rc = moe_dispatch_range(ctx, x_dev, windows_dev, capacity_rows, t0, t1, stream);
+    if (rc != MOE_OK) return rc;
+    rc = moe_combine_range(ctx, windows_dev, capacity_rows, topk_w_dev, y_dev, t0, t1, stream);
+    if (rc != MOE_OK) return rc;
+    if (cudaEventRecord(done[c], st) != cudaSuccess || cudaStreamWaitEvent(ctx->out_stream, done[c], 0) != cudaSuccess ||
+        cudaMemcpyAsync(yh + t0 * row_bytes, yd + t0 * row_bytes, (size_t)(t1 - t0) * row_bytes, cudaMemcpyDeviceToHost,
+                        ctx->out_stream) != cudaSuccess)
+      return MOE_ERR_CUDA;
+  }
+  // The caller's stream finishes only after the last download, so synchronising it (moe_status) is enough.
+  if (cudaEventRecord(finish, ctx->out_stream) != cudaSuccess || cudaStreamWaitEvent(st, finish, 0) != cudaSuccess)
     return MOE_ERR_CUDA;
   return MOE_OK;
 }
@@ -828,6 +900,8 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.items_per_row = 0;
   a.n_items = 0;
   a.win_base = nullptr;
+  a.t_begin = 0;
+  a.t_count = T;
   a.wait_limit_ms = WAIT_LIMIT_MS_DEFAULT;
   a.test_starve = 0;
   int grid = (int)(((int64_t)T * K + 255) / 256);

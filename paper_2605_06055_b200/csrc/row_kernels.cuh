@@ -30,7 +30,8 @@ struct RowArgs {
   int32_t* work_done;        // finished-warp counter (same)
   int32_t granule;           // units (512-byte slabs) per work item
   int32_t items_per_row;     // ceil(units per row / granule)
-  int32_t n_items;           // T * items_per_row
+  int32_t n_items;           // t_count * items_per_row
+  int32_t t_begin, t_count;  // token range this launch covers (the whole batch unless a *_range call)
   // Multi-rank use: window segment d starts at win_base[d] (device array of R device pointers, e.g. peer
   // mappings of every rank's window); nullptr = one allocation of R consecutive segments of C rows.
   const unsigned char* const* win_base;
@@ -155,8 +156,9 @@ __device__ __forceinline__ int32_t fetch_item(const RowArgs& a, ItemFeed& f) {
 
 __device__ __forceinline__ WorkItem decode_item(const RowArgs& a, int32_t item) {
   WorkItem w;
-  w.t = item / a.items_per_row;
-  w.i0 = (item - w.t * a.items_per_row) * a.granule;
+  const int32_t q = item / a.items_per_row;
+  w.t = a.t_begin + q;
+  w.i0 = (item - q * a.items_per_row) * a.granule;
   w.i1 = min(w.i0 + a.granule, (a.H16 + 31) >> 5);
   return w;
 }

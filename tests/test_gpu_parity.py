@@ -370,3 +370,30 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
     assert np.array_equal(win.cpu().view(torch.int16).numpy().view(np.uint16), o.windows_zero_init)
     assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), o.Y) <= 1
     comm.close()
+
+
+def test_token_ranges_in_any_partition_give_the_same_bytes():
+    dev = torch.device("cuda:0")
+    wl = Workload("ranges", 1500, 1000, 32, 4, 6, PREFILL, "uniform", "identity", 88, rank_tokens=(400, 0, 600, 500))
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R, inp.rank_tok_start)
+    C = int(p.n_recv.max())
+    o = harness.oracle_run(inp, C)
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
+    comm.moe_plan(PREFILL, idx, wl.T, inp.rank_tok_start)
+    for path in PATHS:
+        comm.moe_set_option(binding.MOE_OPT_DISPATCH_PATH, path)
+        win = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
+        Y = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+        cuts = [0, 1, 2, 700, 700, 1499, 1500]
+        for a, b in reversed(list(zip(cuts[:-1], cuts[1:]))):            # any order, empty ranges included
+            comm.moe_dispatch_range(X, win, C, a, b)
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            comm.moe_combine_range(win, C, w, Y, a, b)
+        assert comm.moe_status() == 0
+        assert np.array_equal(win.cpu().view(torch.int16).numpy().view(np.uint16), o.windows_zero_init)
+        assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), o.Y) <= 1
+    assert comm.moe_dispatch_range(X, win, C, 5, 1501, check=False) == binding.MOE_ERR_INVALID_ARG
+    assert comm.moe_dispatch_range(X, win, C, 7, 3, check=False) == binding.MOE_ERR_INVALID_ARG
+    comm.close()
