@@ -84,7 +84,8 @@ moe_status_t moe_destroy(moe_ctx_t* ctx);
  * of Decode Dispatch): from the routing indexes computes the count matrix M,
  * the small offsets s and the large offsets o (exclusive scan of M in window
  * order), plus c_rank, n_exp, n_recv.
- *   topk_idx        DEVICE [T,K] int32, values in [0,E)
+ *   topk_idx        DEVICE [T,K] int32, values in [0,E).  The library reads it again in every
+ *                   dispatch / combine / slots call of this plan: keep it valid and unchanged.
  *   rank_tok_start  HOST   [R+1] int32, nondecreasing, [0]=0, [R]=T; NULL means
  *                   uniform T/R tokens per rank (T % R must be 0).  Read before
  *                   the call returns.

@@ -265,35 +265,24 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->out_stream = nullptr;
   ctx->in_stream = nullptr;
 
-  // Shared memory of the planning kernels grows with E; opt in above 48 KB.
-  const int tile_smem = PLAN_WARPS * shape->E * (int)sizeof(int32_t);
+  // Kernels whose dynamic shared memory can exceed 48 KB opt in to the device maximum.  The attribute
+  // belongs to the kernel, not to a context, so it is always set to the same (largest) value: contexts
+  // of different shapes can then be created and used in any order.
   bool ok = cudaMemset(ctx->ctl, 0, sizeof(Control)) == cudaSuccess;
-  if (ok)
-    ok = cudaFuncSetAttribute(dispatch_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              BULK_SMEM_BUDGET + 1024) == cudaSuccess;
-  if (ok)
-    ok = cudaFuncSetAttribute(dispatch_quant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              BULK_SMEM_BUDGET + 1024) == cudaSuccess;
-  if (ok) {
-    const int rank_smem =
-        rank_plan_smem_ints(shape->E, shape->R, shape->E <= RANK_PLAN_WIDE_MAX_E ? 32 : 8) * (int)sizeof(int32_t);
-    const int scan_smem = notify_smem_ints(shape->E, shape->R) * (int)sizeof(int32_t);
-    if (rank_smem > 48 * 1024)
-      ok = (shape->E <= RANK_PLAN_WIDE_MAX_E
-                ? cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)
-                : cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem)) ==
-           cudaSuccess;
-    if (ok && scan_smem > 48 * 1024)
-      ok = cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) ==
-               cudaSuccess &&
-           cudaFuncSetAttribute(notify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, scan_smem) == cudaSuccess;
-  }
-  if (ok && tile_smem > 48 * 1024) {
-    ok = cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_PREFILL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tile_smem) == cudaSuccess &&
-         cudaFuncSetAttribute(plan_tile_kernel<ROUNDS_DECODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tile_smem) == cudaSuccess;
-  }
+  int optin = 0;
+  ok = ok && cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) == cudaSuccess;
+  const int big = optin - 2048;   // leave room for the kernels' few static words
+  auto opt_in = [&](auto kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess;
+  };
+  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel) && opt_in(plan_rank_kernel<32>) &&
+       opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
+       opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel);
+  // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
+  const int rank_smem =
+      rank_plan_smem_ints(shape->E, shape->R, shape->E <= RANK_PLAN_WIDE_MAX_E ? 32 : 8) * (int)sizeof(int32_t);
+  ok = ok && PLAN_WARPS * shape->E * (int)sizeof(int32_t) <= big && rank_smem <= big &&
+       notify_smem_ints(shape->E, shape->R) * (int)sizeof(int32_t) <= big;
   if (!ok) {
     cudaGetLastError();
     delete ctx;
@@ -325,7 +314,6 @@ void launch_gate(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* 
   int warps = 8;
   while (warps > 1 && warps * E * (int)sizeof(float) > 96 * 1024) warps >>= 1;
   const int smem = warps * E * (int)sizeof(float);
-  if (smem > 48 * 1024) cudaFuncSetAttribute(gate_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   int64_t grid = ((int64_t)T + warps - 1) / warps;
   if (grid > (int64_t)num_sms * 8) grid = (int64_t)num_sms * 8;
   if (grid < 1) grid = 1;
@@ -449,6 +437,12 @@ moe_status_t moe_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K,
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return MOE_ERR_CUDA;
+  if (E > 1024) {   // the shared-memory form of the gate: opt in like moe_create does
+    int optin = 0;
+    if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaFuncSetAttribute(gate_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 2048) != cudaSuccess)
+      return MOE_ERR_CUDA;
+  }
   if (T > 0) launch_gate(logits, T, E, K, topk_idx, topk_w, sms, static_cast<cudaStream_t>(stream));
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -397,3 +397,22 @@ def test_token_ranges_in_any_partition_give_the_same_bytes():
     assert comm.moe_dispatch_range(X, win, C, 5, 1501, check=False) == binding.MOE_ERR_INVALID_ARG
     assert comm.moe_dispatch_range(X, win, C, 7, 3, check=False) == binding.MOE_ERR_INVALID_ARG
     comm.close()
+
+
+def test_contexts_of_different_shapes_coexist():
+    """Kernel attributes (opt-in shared memory) are per kernel, not per context: creating a small-E
+    context after a large-E one must not break the first."""
+    dev = torch.device("cuda:0")
+    big = Workload("bigE", 600, 64, 4096, 2, 8, PREFILL, "uniform", "identity", 5)       # 128 KB of planner counters
+    mid = Workload("midE", 600, 64, 2048, 2, 8, PREFILL, "uniform", "identity", 6)       # 64 KB
+    rank_big = Workload("bigE_tiles", 6000, 64, 4096, 2, 8, PREFILL, "uniform", "identity", 7, rank_tokens=(5000, 1000))
+    inps = [synth.make_inputs(w) for w in (big, mid, rank_big)]
+    comms = [binding.MoeComm(i.wl.T, i.wl.H, i.wl.E, i.wl.R, i.wl.K, dev) for i in inps]   # created in this order
+    for inp, comm in zip(inps, comms):                                                      # first one used last-created-first
+        p = oracle.plan(inp.topk_idx.numpy(), inp.wl.E, inp.wl.R, inp.rank_tok_start)
+        C = int(p.n_recv.max())
+        rts = None if inp.wl.rank_tokens is None else inp.rank_tok_start
+        g = harness.gpu_run(inp, C, PREFILL, comm=comm)
+        harness.assert_parity(g, harness.oracle_run(inp, C), PREFILL)
+    for c in comms:
+        c.close()
