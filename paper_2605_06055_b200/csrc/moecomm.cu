@@ -1,6 +1,8 @@
 // libmoecomm: host side of the C ABI declared in include/moecomm.h.
 // Argument validation, workspace layout, launch configuration.  Every step of
-// the path runs in the kernels of plan_kernels.cuh and row_kernels.cuh.
+// the path runs in the kernels of plan_kernels.cuh (planning), gate_kernels.cuh
+// (top-k gate), bulk_kernels.cuh / quant_kernels.cuh (bulk-copy dispatch, plain
+// and quantised) and row_kernels.cuh (register-path dispatch, combine, slots).
 
 #include <cstdio>
 #include <cstdlib>
@@ -41,6 +43,10 @@ struct moe_ctx {
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
   cudaEvent_t fwd_events[2 * 16 + 2];
+  // resident CTAs per SM of the row kernels this context has launched (occupancy calculator results)
+  const void* occ_kernel[16];
+  int occ_per_sm[16];
+  int occ_n;
 };
 
 namespace {
@@ -162,11 +168,20 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
 // One persistent wave: as many CTAs as fit on the device at once (from the occupancy calculator),
 // but no more warps than there are 512-byte units of work.
 template <class Kernel>
-int row_grid(const moe_ctx* ctx, Kernel kernel, int64_t tokens) {
+int row_grid(moe_ctx* ctx, Kernel kernel, int64_t tokens) {
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0) != cudaSuccess || per_sm < 1) {
-    cudaGetLastError();
-    per_sm = 2;
+  const void* key = reinterpret_cast<const void*>(kernel);
+  for (int i = 0; i < ctx->occ_n; ++i)
+    if (ctx->occ_kernel[i] == key) per_sm = ctx->occ_per_sm[i];
+  if (per_sm == 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0) != cudaSuccess || per_sm < 1) {
+      cudaGetLastError();
+      per_sm = 1;
+    }
+    if (ctx->occ_n < 16) {
+      ctx->occ_kernel[ctx->occ_n] = key;
+      ctx->occ_per_sm[ctx->occ_n++] = per_sm;
+    }
   }
   const int64_t units = tokens * ((ctx->shape.H / 8 + 31) / 32);
   const int64_t need = (units + 7) / 8;
@@ -264,6 +279,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->starve_wait_ms = 0;
   ctx->out_stream = nullptr;
   ctx->in_stream = nullptr;
+  ctx->occ_n = 0;
 
   // Kernels whose dynamic shared memory can exceed 48 KB opt in to the device maximum.  The attribute
   // belongs to the kernel, not to a context, so it is always set to the same (largest) value: contexts
