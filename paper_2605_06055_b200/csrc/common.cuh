@@ -14,7 +14,7 @@ namespace moe {
 // rounds of 32 branches.
 constexpr int PLAN_WARPS = 8;
 constexpr int PLAN_THREADS = PLAN_WARPS * 32;
-constexpr int ROUNDS_PREFILL = 8;  // 2048 branches per tile
+constexpr int ROUNDS_PREFILL = 4;  // 1024 branches per tile
 constexpr int ROUNDS_DECODE = 1;   //  256 branches per tile
 
 // Token ranges and tile ranges of the source ranks, passed by value as a

@@ -47,23 +47,26 @@ plan_tile_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   const int32_t b_begin = map.tok_start[r] * K + ((tile - map.tile_start[r]) << map.tile_shift);
   const int32_t b_end = min(b_begin + (ROUNDS * PLAN_THREADS), map.tok_start[r + 1] * K);
 
-  for (int i = threadIdx.x; i < PLAN_WARPS * E; i += PLAN_THREADS) warp_hist[i] = 0;
-  __syncthreads();
-
   int32_t* my_hist = warp_hist + warp * E;
   const int32_t warp_begin = b_begin + warp * (ROUNDS * 32);
   int32_t e_of[ROUNDS], rk[ROUNDS];
   const unsigned lt = lanemask_lt();
+  // All of the warp's routing indexes first (independent loads, one memory round trip that overlaps
+  // the clearing of the counters), then the rounds.
 #pragma unroll
   for (int i = 0; i < ROUNDS; ++i) {
     const int32_t b = warp_begin + i * 32 + lane;
-    int32_t e = -1;
-    if (b < b_end) {
-      e = __ldg(topk_idx + b);
-      if (e < 0 || e >= E) {
-        raise_status(status, MOE_ERR_BAD_INDEX);
-        e = -1;
-      }
+    e_of[i] = b < b_end ? __ldg(topk_idx + b) : -1;
+  }
+  for (int i = threadIdx.x; i < PLAN_WARPS * E; i += PLAN_THREADS) warp_hist[i] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < ROUNDS; ++i) {
+    const int32_t b = warp_begin + i * 32 + lane;
+    int32_t e = e_of[i];
+    if (b < b_end && (e < 0 || e >= E)) {
+      raise_status(status, MOE_ERR_BAD_INDEX);
+      e = -1;
     }
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     const int ahead = __popc(peers & lt);           // equal keys in lower lanes = earlier branches

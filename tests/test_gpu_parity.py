@@ -58,7 +58,7 @@ def test_config5_mixtral_sweep(T, schedule):
 
 
 def test_config3_shape_reduced_tokens():
-    # DeepSeek-V3-like prefill shape at 1/8 of the tokens: several 2048-branch tiles per rank plus a ragged tail.
+    # DeepSeek-V3-like prefill shape at 1/8 of the tokens: several 1024-branch tiles per rank plus a ragged tail.
     wl = Workload("c3_reduced", 8 * 517, 7168, 256, 8, 8, PREFILL, "uniform", "identity", 3003)
     run_and_check(wl)
 
@@ -88,7 +88,7 @@ EDGE = [
     ("empty_rank_ragged", 1000, 256, 32, 4, 8, "uniform", (0, 517, 0, 483)),
     ("many_ranks", 512, 64, 256, 64, 8, "uniform", None),
     ("big_E", 3000, 32, 2048, 2, 8, "uniform", None),
-    ("tile_boundary_exact", 2048, 32, 8, 2, 2, "uniform", None),   # 2048 branches per rank = exactly one tile
+    ("tile_boundary_exact", 2048, 32, 8, 2, 2, "uniform", None),   # 2048 branches per rank = exactly two tiles
     ("tile_boundary_plus1", 2050, 32, 8, 2, 2, "uniform", None),
     ("rank_above_compact_decode_limit", 6000, 16, 16, 2, 2, "uniform", (5000, 1000)),   # 10000 branches in rank 0
     ("compact_decode_several_passes", 1200, 16, 1024, 2, 6, "uniform", (682, 518)),     # E > 768: 8-warp planner
