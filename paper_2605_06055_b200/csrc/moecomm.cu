@@ -133,6 +133,8 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.items_per_row = 0;
   a.n_items = 0;
   a.win_base = nullptr;
+  a.prefetch_meta = 0;
+  a.static_first = 0;
   a.t_begin = 0;
   a.t_count = ctx->T;
   a.wait_limit_ms = ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT;
@@ -161,6 +163,7 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
   a.granule = (int32_t)g;
   a.items_per_row = (int32_t)((upr + g - 1) / g);
   a.n_items = (int32_t)(tokens * a.items_per_row);
+  a.static_first = a.n_items <= 4 * nwarps ? 2 : 0;
   a.work = &ctx->ctl->work;
   a.work_done = &ctx->ctl->work_done;
 }
@@ -230,6 +233,9 @@ void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const floa
   const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
+  // an item that is one or two batches of loads cannot hide its own metadata latency: prefetch it
+  constexpr int unroll = KT > 0 ? combine_unroll(KT) : 4;
+  b.prefetch_meta = (b.granule + unroll - 1) / unroll <= 2;
   kernel<<<grid, 256, 0, st>>>(win, w, y, b, ctx->map);
 }
 
@@ -910,6 +916,8 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.items_per_row = 0;
   a.n_items = 0;
   a.win_base = nullptr;
+  a.prefetch_meta = 0;
+  a.static_first = 0;
   a.t_begin = 0;
   a.t_count = T;
   a.wait_limit_ms = WAIT_LIMIT_MS_DEFAULT;

@@ -35,6 +35,8 @@ struct RowArgs {
   // Multi-rank use: window segment d starts at win_base[d] (device array of R device pointers, e.g. peer
   // mappings of every rank's window); nullptr = one allocation of R consecutive segments of C rows.
   const unsigned char* const* win_base;
+  int32_t static_first;      // work items per warp that are fixed (warp id + k * warps) before the counter is used
+  int32_t prefetch_meta;     // combine: fetch the next item's branch metadata while reducing the current one
   int32_t wait_limit_ms;     // bound of every device-side wait
   int32_t test_starve;       // test hook of the bulk-copy dispatch: make one wait run out
 };
@@ -54,6 +56,45 @@ __device__ __forceinline__ int64_t resolve_slot(const RowArgs& a, const RankMap&
     if (record) a.small_out[b] = so;
   }
   return (int64_t)(e / a.E_r) * a.C + __ldg(a.large_off + (size_t)e * a.R + r) + so;
+}
+
+// The same resolution in two phases, so that its memory latency can hide behind payload traffic:
+// load_meta issues the loads that depend only on the branch index (routing index, small offset,
+// weight) and finish_slot adds the large offset.  When a work item is a single batch of loads
+// (short rows, small K) combine calls load_meta for the NEXT item before it reduces the current
+// one; measured 274 -> 256 us at H=4096, K=2, and 618 -> 629 us at H=7168, K=8, where a row is seven
+// batches and the launcher therefore leaves the prefetch off.
+struct BranchMeta {
+  int32_t e, so;
+  float w;
+};
+
+__device__ __forceinline__ BranchMeta load_meta(const RowArgs& a, const float* __restrict__ topk_w, int32_t t,
+                                                int lane) {
+  BranchMeta m;
+  m.e = -1;
+  m.so = 0;
+  m.w = 0.0f;
+  if (lane < a.K) {
+    const int32_t b = t * a.K + lane;
+    m.e = __ldg(a.topk_idx + b);
+    m.so = __ldg(a.small_off + b);
+    if (topk_w != nullptr) m.w = __ldg(topk_w + b);
+  }
+  return m;
+}
+
+__device__ __forceinline__ int64_t finish_slot(const RowArgs& a, const RankMap& map, const BranchMeta& m, int32_t t,
+                                               int lane, bool record) {
+  if (lane >= a.K || m.e < 0 || m.e >= a.E) return -1;   // bad indexes were flagged by the plan; never dereferenced
+  const int32_t r = src_rank(map, t);
+  int32_t so = m.so;
+  if (a.tile_base != nullptr) {
+    const int32_t b = t * a.K + lane;
+    so += __ldg(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + m.e);
+    if (record) a.small_out[b] = so;
+  }
+  return (int64_t)(m.e / a.E_r) * a.C + __ldg(a.large_off + (size_t)m.e * a.R + r) + so;
 }
 
 // Address of window row `row` (global numbering d*C + local row).
@@ -126,8 +167,10 @@ __device__ __forceinline__ void end_work(const RowArgs& a) {
   }
 }
 
-// Hands a warp its work items: the first two are fixed (warp id, warp id + number of warps), so no
-// warp waits on an atomic before its first bytes move; every later one comes from the counter.
+// Hands a warp its work items.  In small jobs (a few items per warp: decode) the first two are fixed
+// (warp id, warp id + number of warps), so no warp waits on an atomic before its first bytes move
+// (2 us of a 48 us call); every later one comes from the counter.  Large jobs take every item from
+// the counter: fixed first items measured up to 6 % slower there.
 struct ItemFeed {
   int64_t gid, nwarps;
   int32_t taken;
@@ -143,12 +186,12 @@ __device__ __forceinline__ ItemFeed begin_feed() {
 
 __device__ __forceinline__ int32_t fetch_item(const RowArgs& a, ItemFeed& f) {
   int64_t item;
-  if (f.taken < 2) {
+  if (f.taken < a.static_first) {
     item = f.gid + f.taken * f.nwarps;
   } else {
     int32_t v = 0;
     if ((threadIdx.x & 31) == 0) v = atomicAdd(a.work, 1);
-    item = 2 * f.nwarps + __shfl_sync(0xffffffffu, v, 0);
+    item = a.static_first * f.nwarps + __shfl_sync(0xffffffffu, v, 0);
   }
   ++f.taken;
   return (int32_t)min(item, (int64_t)a.n_items);
@@ -262,12 +305,17 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
 
   ItemFeed feed = begin_feed();
   int32_t item = fetch_item(a, feed);
+  BranchMeta meta = {-1, 0, 0.0f};
+  if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item(a, item).t, lane);
   while (item < a.n_items) {
     const int32_t next_item = fetch_item(a, feed);
     const WorkItem wi = decode_item(a, item);
+    if (!a.prefetch_meta) meta = load_meta(a, topk_w, wi.t, lane);
+    const int64_t slot = finish_slot(a, map, meta, wi.t, lane, false);
+    const float w_lane = meta.w;
+    // short rows: the next item's routing index, small offset and weight travel while this item is reduced
+    if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item(a, next_item).t, lane);
     item = next_item;
-    const int64_t slot = resolve_slot(a, map, wi.t, lane, false);
-    const float w_lane = lane < K ? __ldg(topk_w + (size_t)wi.t * K + lane) : 0.0f;
     uint4* out = Y + (size_t)wi.t * H16;
     if constexpr (KT > 0) {
       const uint4* src[KT];
