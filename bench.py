@@ -173,9 +173,9 @@ def oracle_sample(wl, frac_den: int):
                           wl.routing, wl.expert_op, wl.seed, wl.zipf_s)
 
 
-def time_oracle(wl, steps: int, warmup: int, inp=None):
+def time_oracle(wl, steps: int, warmup: int, inp=None, cores=None):
     import oracle
-    cores = len(os.sched_getaffinity(0))
+    cores = len(os.sched_getaffinity(0)) if cores is None else cores
     inp = synth.make_inputs(wl) if inp is None else inp
     idx = inp.topk_idx.numpy()
     X = synth.bf16_to_u16(inp.X)
@@ -368,33 +368,60 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
     plan = lambda: c.moe_plan(dwl.schedule, dl.idx)
     disp = lambda: c.moe_dispatch(dl.X, dl.windows, dl.C)
     comb = lambda: c.moe_combine(dl.windows, dl.C, dl.w, dl.Y)
+    from paper_2605_06055_b200 import binding
+    fused = lambda: c.moe_plan_dispatch(dwl.schedule, dl.idx, dl.X, dl.windows, dl.C)
+    # three graphs of one step: separate calls with every kernel serialised, separate calls with the
+    # combine allowed to start behind the dispatch, and planning folded into the dispatch call
+    c.moe_set_option(binding.MOE_OPT_OVERLAP, 0)
+    g_serial = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_serial):
+        dl.step()
+    c.moe_set_option(binding.MOE_OPT_OVERLAP, 1)
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
         dl.step()
+    g_fused = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_fused):
+        fused()
+        comb()
     replay = lambda: g.replay()
+    replay_serial = lambda: g_serial.replay()
+    replay_fused = lambda: g_fused.replay()
     out = {"config": describe(dwl),
            "method": f"cumulative sequences of calls, {n} repetitions per pair of CUDA events; per-call = difference",
            "roofline_us_per_call_at_measured_peak": bytes_dispatch(dwl) / peak / 1e3}
-    from paper_2605_06055_b200 import binding
     logits = torch.randn(dwl.T, dwl.E, generator=torch.Generator().manual_seed(7)).to(dev)
     g_idx, g_w = torch.empty_like(dl.idx), torch.empty_like(dl.w)
     gate = lambda: binding.moe_gate_topk(logits, dwl.K, g_idx, g_w)
     gate_plan = lambda: c.moe_gate_plan(dwl.schedule, logits, g_idx, g_w)
+    # context for the per-call figures: a plain device-to-device copy that moves the same total bytes
+    half = bytes_dispatch(dwl) // 2
+    cp_src = torch.zeros(half, dtype=torch.uint8, device=dev)
+    cp_dst = torch.empty_like(cp_src)
+    copy = lambda: cp_dst.copy_(cp_src)
     for name, pre in (("cold", [flush]), ("warm", [])):
         base = time_repeated(pre, n) if pre else 0.0
+        t_copy = time_repeated(pre + [copy], n)
         t1 = time_repeated(pre + [plan], n)
         t2 = time_repeated(pre + [plan, disp], n)
         t3 = time_repeated(pre + [plan, disp, comb], n)
         tg = time_repeated(pre + [replay], n)
+        tgs = time_repeated(pre + [replay_serial], n)
+        tgf = time_repeated(pre + [replay_fused], n)
+        tf = time_repeated(pre + [fused, comb], n)
         t_gate = time_repeated(pre + [gate], n)
         t_gate_plan = time_repeated(pre + [gate_plan], n)
         out[name] = {"l2": "256 MB L2 flush before every step (its time subtracted)" if pre else
                      "back-to-back steps, no flush",
                      "plan_us": t1 - base, "dispatch_us": t2 - t1, "combine_us": t3 - t2,
                      "step_us_stream_launches": t3 - base, "step_us_cuda_graph": tg - base,
+                     "step_us_cuda_graph_no_overlap": tgs - base,
+                     "step_us_plan_dispatch_fused_stream_launches": tf - base,
+                     "step_us_plan_dispatch_fused_cuda_graph": tgf - base,
                      "dispatch_GBps": bytes_dispatch(dwl) / (t2 - t1) / 1e3,
                      "combine_GBps": bytes_combine(dwl) / (t3 - t2) / 1e3,
-                     "gate_us": t_gate - base, "gate_plan_us": t_gate_plan - base}
+                     "gate_us": t_gate - base, "gate_plan_us": t_gate_plan - base,
+                     "plain_copy_of_the_same_bytes_us": t_copy - base}
     plan()   # leave the context planned on dl.idx again
     assert c.moe_status() == 0
     return out
@@ -403,13 +430,17 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
 def kernel_table(wl, r, peak):
     med = statistics.median
     mean = lambda v: sum(v) / len(v)
+    p95 = lambda v: sorted(v)[min(len(v) - 1, int(0.95 * len(v)))]
     k = {
-        "moe_plan": {"us": med(r["plan_us"]), "us_mean": mean(r["plan_us"]), "bytes": bytes_plan(wl)},
+        "moe_plan": {"us": med(r["plan_us"]), "us_mean": mean(r["plan_us"]), "us_p95": p95(r["plan_us"]),
+                     "bytes": bytes_plan(wl)},
         "moe_dispatch": {"us": med(r["dispatch_us"]), "us_mean": mean(r["dispatch_us"]),
-                         "us_min": min(r["dispatch_us"]), "bytes": bytes_dispatch(wl),
+                         "us_min": min(r["dispatch_us"]), "us_p95": p95(r["dispatch_us"]),
+                         "bytes": bytes_dispatch(wl),
                          "GBps": bytes_dispatch(wl) / mean(r["dispatch_us"]) / 1e3},
         "moe_combine": {"us": med(r["combine_us"]), "us_mean": mean(r["combine_us"]),
-                        "us_min": min(r["combine_us"]), "bytes": bytes_combine(wl),
+                        "us_min": min(r["combine_us"]), "us_p95": p95(r["combine_us"]),
+                        "bytes": bytes_combine(wl),
                         "GBps": bytes_combine(wl) / mean(r["combine_us"]) / 1e3},
     }
     for name in ("moe_dispatch", "moe_combine"):
@@ -531,6 +562,12 @@ def run_cuda(args, wl):
                                 "sample": ("whole workload" if sample is wl else
                                            f"first half of every rank's tokens (T={sample.T})") +
                                           ", one timed pass after one warm-up pass, token-parallel over all cores"}
+        one = oracle_sample(wl, 16) if wl.T // wl.R >= 16 else wl
+        t1, _ = time_oracle(one, 1, 1, cores=1)
+        line["cpu_baseline"]["single_thread"] = {"value": bytes_step(one) / t1[0] / 1e9, "unit": "GB/s",
+                                                 "ms": t1[0] * 1e3,
+                                                 "sample": f"first 1/16 of every rank's tokens (T={one.T})"
+                                                           if one is not wl else "whole workload"}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

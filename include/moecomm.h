@@ -137,6 +137,18 @@ moe_status_t moe_plan_view(const moe_ctx_t* ctx, moe_plan_view_t* out /*HOST*/);
 moe_status_t moe_dispatch(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows /*DEVICE*/,
                           int64_t capacity_rows, void* stream);
 
+/* Planning folded into the dispatch call (Section 5.3, Decode Dispatch: the count and offset state is
+ * produced inside the dispatch procedure instead of by a separate Layout -> Notify sequence).
+ * Same result as moe_plan followed by moe_dispatch with the same arguments, for either schedule; the
+ * plan stays valid for moe_combine, moe_slots and the other consumers.  The dispatch kernel is
+ * launched with programmatic stream serialization behind the planner: it starts while the planner
+ * runs, moves the first payload loads of every warp (they depend on nothing the planner writes),
+ * and waits for the planner's completion before it reads any offset.  x and topk_idx need only be
+ * ready in stream order, as for the separate calls. */
+moe_status_t moe_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE*/,
+                               int32_t T, const int32_t* rank_tok_start /*HOST*/, const void* x /*DEVICE*/,
+                               void* windows /*DEVICE*/, int64_t capacity_rows, void* stream);
+
 /* Row-wise quantised dispatch (Section 5.2, Prefill Dispatch: with row-wise quantisation the scale
  * values go to a parallel scale tensor in the same row order).  The paper names no format; this
  * library's definition is fp8 e4m3 (1-4-3, bias 7, largest finite 448, no infinities) with one fp32
@@ -228,8 +240,17 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
  *                          dispatch lets ONE warp wait for 16 bytes that are never sent and bounds
  *                          every device-side wait by v milliseconds: that warp gives up, the status
  *                          word becomes MOE_ERR_TIMEOUT, the kernel ends normally (no trap, nothing
- *                          left in flight) and the windows are incomplete.  Normal bound: 2 s. */
-typedef enum { MOE_OPT_DISPATCH_PATH = 0, MOE_OPT_GRANULE = 1, MOE_OPT_TEST_STARVE_WAIT_MS = 2 } moe_option_t;
+ *                          left in flight) and the windows are incomplete.  Normal bound: 2 s.
+ *   MOE_OPT_OVERLAP        1 (default): moe_plan_dispatch starts its dispatch kernel while the planner
+ *                          runs (programmatic stream serialization; the early part of the kernel
+ *                          reads nothing the planner writes).  0: the dispatch kernel starts after the
+ *                          planner has ended.  Same result either way. */
+typedef enum {
+  MOE_OPT_DISPATCH_PATH = 0,
+  MOE_OPT_GRANULE = 1,
+  MOE_OPT_TEST_STARVE_WAIT_MS = 2,
+  MOE_OPT_OVERLAP = 3
+} moe_option_t;
 enum { MOE_DISPATCH_AUTO = 0, MOE_DISPATCH_REGISTERS = 1, MOE_DISPATCH_BULK = 2 };
 moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);
 

@@ -84,14 +84,10 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 // Dynamic shared memory: [warps][BULK_STAGES][stage_bytes] payload, then
 // [warps][BULK_STAGES] mbarriers.  stage_bytes = granule * 512; warps = blockDim.x / 32.
-__global__ void __launch_bounds__(BULK_MAX_WARPS * 32)
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1)
 dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows, const RowArgs a,
                      const __grid_constant__ RankMap map) {
   extern __shared__ __align__(128) unsigned char smem[];
-  if (must_abort(a)) {
-    end_work(a);
-    return;
-  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t stage_bytes = (uint32_t)a.granule * 512u;
   const uint32_t row_bytes = (uint32_t)a.H16 * 16u;
@@ -119,11 +115,38 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
 
   // Items in flight: q0 is consumed this iteration, q1 is loading, q2 is fetched now.
   ItemFeed feed = begin_feed();
-  int32_t q0 = fetch_item(a, feed);
-  int32_t q1 = fetch_item(a, feed);
-  if (lane == 0) {
-    if (q0 < a.n_items) issue_load(q0, 0);
-    if (q1 < a.n_items) issue_load(q1, 1);
+  int32_t q0 = a.n_items, q1 = a.n_items;
+  // Started early behind the planner (moe_plan_dispatch): the first two items of a small job are fixed
+  // and their payload depends on nothing the planner writes, so their loads travel while it runs.
+  // Nothing is taken from the work counter and no planner output is read before the wait.
+  const bool early = a.pdl && a.static_first >= 2;
+  if (early) {
+    q0 = fetch_item(a, feed);
+    q1 = fetch_item(a, feed);
+    if (lane == 0) {
+      if (q0 < a.n_items) issue_load(q0, 0);
+      if (q1 < a.n_items) issue_load(q1, 1);
+    }
+    if (q0 < a.n_items && lane < a.K) warm(a.topk_idx + (size_t)decode_item(a, q0).t * a.K + lane);
+  }
+  dependency_wait();      // returns at once unless this launch was allowed to start early
+  release_dependents();   // after the wait: whatever follows starts no earlier than the previous kernel's end
+  if (must_abort(a)) {
+    // loads already in flight must land before this CTA's shared memory is handed back
+    if (early && lane == 0) {
+      if (q0 < a.n_items) mbar_wait(bar0, 0, a.wait_limit_ms);
+      if (q1 < a.n_items) mbar_wait(bar0 + 8, 0, a.wait_limit_ms);
+    }
+    end_work(a);
+    return;
+  }
+  if (!early) {
+    q0 = fetch_item(a, feed);
+    q1 = fetch_item(a, feed);
+    if (lane == 0) {
+      if (q0 < a.n_items) issue_load(q0, 0);
+      if (q1 < a.n_items) issue_load(q1, 1);
+    }
   }
   uint64_t evict_first;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));

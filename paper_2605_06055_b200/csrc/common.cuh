@@ -60,6 +60,15 @@ __device__ __forceinline__ int32_t tile_of_branch(const RankMap& map, int32_t r,
   return map.tile_start[r] + ((b - map.tok_start[r] * K) >> map.tile_shift);
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may
+// start while the previous kernel of the stream still runs; dependency_wait() returns once that kernel
+// has completed and its writes are visible (at once when the launch carried no such attribute), and
+// release_dependents() lets the NEXT kernel of the stream start early in the same way.  The row kernels
+// release only after their own wait, so whatever completed before them has completed before any
+// kernel that follows them starts.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ unsigned lanemask_lt() {
   unsigned m;
   asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));

@@ -40,6 +40,7 @@ struct moe_ctx {
   int32_t dispatch_path;    // MOE_OPT_DISPATCH_PATH
   int32_t granule_override; // MOE_OPT_GRANULE
   int32_t starve_wait_ms;   // MOE_OPT_TEST_STARVE_WAIT_MS
+  int32_t overlap;          // MOE_OPT_OVERLAP
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
   cudaEvent_t fwd_events[2 * 16 + 2];
@@ -135,6 +136,7 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.win_base = nullptr;
   a.prefetch_meta = 0;
   a.static_first = 0;
+  a.pdl = 0;
   a.t_begin = 0;
   a.t_count = ctx->T;
   a.wait_limit_ms = ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT;
@@ -207,10 +209,27 @@ void launch_dispatch_regs(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   kernel<<<grid, 256, 0, st>>>(x, win, b, ctx->map);
 }
 
+// Launch with programmatic stream serialization when `pdl` is set: the kernel may then start while
+// the previous kernel of the stream is still running and orders itself with dependency_wait().
+template <class... KArgs, class... Args>
+void launch_kernel(void (*kernel)(KArgs...), int grid, int threads, int smem, cudaStream_t st, bool pdl, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Bulk-copy path: one CTA per SM; each warp drives a ring of BULK_STAGES stages, and the CTA has as
 // many warps (up to BULK_MAX_WARPS) as fit their rings into the shared-memory budget: 4 for 14 KB
 // rows, 8 for rows of 8 KB or less (short rows need more requests in flight to cover the latency).
-void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st) {
+void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4* win, cudaStream_t st, bool pdl) {
   const int upr = (a.H16 + 31) / 32;
   const int g_max = upr < BULK_MAX_GRANULE ? upr : BULK_MAX_GRANULE;
   int warps = BULK_SMEM_BUDGET / (BULK_STAGES * (g_max * 512 + 8));
@@ -220,8 +239,9 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * warps, g_max);
   const int smem = warps * BULK_STAGES * (b.granule * 512 + 8);
-  dispatch_bulk_kernel<<<grid, warps * 32, smem, st>>>(reinterpret_cast<const unsigned char*>(x),
-                                                     reinterpret_cast<unsigned char*>(win), b, ctx->map);
+  b.pdl = pdl;
+  launch_kernel(dispatch_bulk_kernel, grid, warps * 32, smem, st, pdl, reinterpret_cast<const unsigned char*>(x),
+                reinterpret_cast<unsigned char*>(win), b, ctx->map);
 }
 
 template <int KT>
@@ -283,6 +303,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->dispatch_path = MOE_DISPATCH_AUTO;
   ctx->granule_override = 0;
   ctx->starve_wait_ms = 0;
+  ctx->overlap = 1;
   ctx->out_stream = nullptr;
   ctx->in_stream = nullptr;
   ctx->occ_n = 0;
@@ -487,7 +508,7 @@ moe_status_t moe_plan_view(const moe_ctx_t* c, moe_plan_view_t* out) {
 namespace {
 
 moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const void* const* bases, int64_t capacity_rows,
-                           void* stream, int32_t t_begin = 0, int32_t t_end = -1) {
+                           void* stream, int32_t t_begin = 0, int32_t t_end = -1, bool behind_plan = false) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
   if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || (windows == nullptr && bases == nullptr))))
@@ -504,7 +525,7 @@ moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const voi
   const uint4* xs = static_cast<const uint4*>(x);
   uint4* win = static_cast<uint4*>(windows);
   if (ctx->dispatch_path != MOE_DISPATCH_REGISTERS) {
-    launch_dispatch_bulk(ctx, a, xs, win, st);
+    launch_dispatch_bulk(ctx, a, xs, win, st, behind_plan && ctx->overlap);
   } else {
     switch (ctx->shape.K) {
       case 1: launch_dispatch_regs<1>(ctx, a, xs, win, st); break;
@@ -525,6 +546,17 @@ extern "C" {
 moe_status_t moe_dispatch(moe_ctx_t* ctx, const void* x, void* windows, int64_t capacity_rows, void* stream) {
   if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;
   return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream);
+}
+
+moe_status_t moe_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                               const int32_t* rank_tok_start, const void* x, void* windows, int64_t capacity_rows,
+                               void* stream) {
+  if (ctx == nullptr || (T > 0 && (topk_idx == nullptr || x == nullptr || windows == nullptr)))
+    return MOE_ERR_INVALID_ARG;
+  if (capacity_rows < 0 || !aligned16(x) || !aligned16(windows)) return MOE_ERR_INVALID_ARG;
+  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, nullptr, nullptr, nullptr);
+  if (rc != MOE_OK) return rc;
+  return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream, 0, -1, true);
 }
 
 moe_status_t moe_dispatch_range(moe_ctx_t* ctx, const void* x, void* windows, int64_t capacity_rows, int32_t t_begin,
@@ -757,6 +789,10 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) 
     case MOE_OPT_GRANULE:
       if (value < 0 || value > (1 << 20)) return MOE_ERR_INVALID_ARG;
       ctx->granule_override = (int32_t)value;
+      return MOE_OK;
+    case MOE_OPT_OVERLAP:
+      if (value != 0 && value != 1) return MOE_ERR_INVALID_ARG;
+      ctx->overlap = (int32_t)value;
       return MOE_OK;
   }
   return MOE_ERR_INVALID_ARG;

@@ -294,6 +294,10 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
                  int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
+  // A dispatch launched behind this kernel with programmatic serialization (moe_plan_dispatch) may start
+  // now and move its first payload loads while the plan is computed; it waits for this kernel's
+  // completion before it reads anything written here.  Without such a dependent this does nothing.
+  release_dependents();
   constexpr int P = WARPS + 1;
   int32_t* counts = sm;             // [E][P]
   int32_t* rank_base = sm + P * E;  // [E]

@@ -37,6 +37,7 @@ struct RowArgs {
   const unsigned char* const* win_base;
   int32_t static_first;      // work items per warp that are fixed (warp id + k * warps) before the counter is used
   int32_t prefetch_meta;     // combine: fetch the next item's branch metadata while reducing the current one
+  int32_t pdl;               // dispatch launched behind the planner with programmatic stream serialization
   int32_t wait_limit_ms;     // bound of every device-side wait
   int32_t test_starve;       // test hook of the bulk-copy dispatch: make one wait run out
 };
@@ -95,6 +96,12 @@ __device__ __forceinline__ int64_t finish_slot(const RowArgs& a, const RankMap& 
     if (record) a.small_out[b] = so;
   }
   return (int64_t)(m.e / a.E_r) * a.C + __ldg(a.large_off + (size_t)m.e * a.R + r) + so;
+}
+
+// Pulls a word into the cache hierarchy ahead of its use; the value is discarded.
+__device__ __forceinline__ void warm(const int32_t* p) {
+  const int32_t v = __ldg(p);
+  asm volatile("" ::"r"(v));
 }
 
 // Address of window row `row` (global numbering d*C + local row).
@@ -295,14 +302,13 @@ template <int KT, int UNROLL, bool L1_ALLOC>
 __global__ void __launch_bounds__(256, 1)
 combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__ topk_w, uint4* __restrict__ Y,
                     const RowArgs a, const __grid_constant__ RankMap map) {
+  const int lane = threadIdx.x & 31;
+  const int K = KT > 0 ? KT : a.K;
+  const int H16 = a.H16;
   if (must_abort(a)) {
     end_work(a);
     return;
   }
-  const int lane = threadIdx.x & 31;
-  const int K = KT > 0 ? KT : a.K;
-  const int H16 = a.H16;
-
   ItemFeed feed = begin_feed();
   int32_t item = fetch_item(a, feed);
   BranchMeta meta = {-1, 0, 0.0f};
