@@ -43,16 +43,16 @@ def lib() -> ctypes.CDLL:
     if _lib is None:
         L = ctypes.CDLL(build())
         i32, i64, p = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
-        L.oracle_plan.argtypes = [p, i32, i32, i32, i32, p, p, p, p, p, p, p]
+        L.oracle_plan.argtypes = [p, i32, i32, i32, i32, p, i32, p, p, p, p, p, p]
         L.oracle_slots.argtypes = [p, i32, i32, i32, i32, p, p, p, p, i64, p]
         L.oracle_dispatch.argtypes = [p, i32, i32, i32, p, p, i32]
-        L.oracle_expert_scale.argtypes = [p, i32, i32, i32, i64, p, p]
+        L.oracle_expert_scale.argtypes = [p, i32, i32, i32, i64, i32, p, p]
         L.oracle_combine.argtypes = [p, i32, i32, i32, p, p, p, i32]
-        L.oracle_notify.argtypes = [p, i32, i32, p, p, p, p]
+        L.oracle_notify.argtypes = [p, i32, i32, i32, p, p, p, p]
         L.oracle_notify.restype = ctypes.c_int
         L.oracle_gate_topk.argtypes = [p, i32, i32, i32, p, p]
         L.oracle_gate_topk.restype = ctypes.c_int
-        L.oracle_expert_ranges.argtypes = [i32, i32, i64, p, p, p]
+        L.oracle_expert_ranges.argtypes = [i32, i32, i64, i32, p, p, p]
         L.oracle_expert_ranges.restype = ctypes.c_int
         L.oracle_dispatch_quant.argtypes = [p, i32, i32, i32, p, p, p, i32]
         L.oracle_dispatch_quant.restype = ctypes.c_int
@@ -95,7 +95,7 @@ class Plan:
     n_recv: np.ndarray   # [R]
 
 
-def plan(topk_idx, E: int, R: int, rank_tok_start=None) -> Plan:
+def plan(topk_idx, E: int, R: int, rank_tok_start=None, align: int = 1) -> Plan:
     topk_idx = _c(topk_idx, np.int32)
     T, K = topk_idx.shape
     rts = uniform_rank_tok_start(T, R) if rank_tok_start is None else _c(rank_tok_start, np.int32)
@@ -106,8 +106,8 @@ def plan(topk_idx, E: int, R: int, rank_tok_start=None) -> Plan:
     o = np.full((E, R), sentinel, np.int32)
     n_exp = np.full((E,), sentinel, np.int32)
     n_recv = np.full((R,), sentinel, np.int32)
-    st = lib().oracle_plan(_ptr(topk_idx), T, K, E, R, _ptr(rts), _ptr(M), _ptr(c_rank), _ptr(s), _ptr(o),
-                           _ptr(n_exp), _ptr(n_recv))
+    st = lib().oracle_plan(_ptr(topk_idx), T, K, E, R, _ptr(rts), int(align), _ptr(M), _ptr(c_rank), _ptr(s),
+                           _ptr(o), _ptr(n_exp), _ptr(n_recv))
     return Plan(st, M, c_rank, s, o, n_exp, n_recv)
 
 
@@ -121,7 +121,7 @@ def slots(topk_idx, E: int, R: int, pl: Plan, C: int, rank_tok_start=None):
     return st, out
 
 
-def notify(M):
+def notify(M, align: int = 1):
     """Large offsets and receive counts from a gathered count matrix M [R,E]."""
     M = _c(M, np.int32)
     R, E = M.shape
@@ -129,7 +129,7 @@ def notify(M):
     o = np.full((E, R), -7, np.int32)
     n_exp = np.full((E,), -7, np.int32)
     n_recv = np.full((R,), -7, np.int32)
-    st = lib().oracle_notify(_ptr(M), E, R, _ptr(c_rank), _ptr(o), _ptr(n_exp), _ptr(n_recv))
+    st = lib().oracle_notify(_ptr(M), E, R, int(align), _ptr(c_rank), _ptr(o), _ptr(n_exp), _ptr(n_recv))
     return st, c_rank, o, n_exp, n_recv
 
 
@@ -142,11 +142,11 @@ def gate_topk(logits, K: int):
     return st, idx, w
 
 
-def expert_ranges(E: int, R: int, C: int, n_exp):
+def expert_ranges(E: int, R: int, C: int, n_exp, align: int = 1):
     n_exp = _c(n_exp, np.int32)
     start = np.full((E,), -1, np.int64)
     count = np.full((E,), -1, np.int32)
-    st = lib().oracle_expert_ranges(E, R, int(C), _ptr(n_exp), _ptr(start), _ptr(count))
+    st = lib().oracle_expert_ranges(E, R, int(C), int(align), _ptr(n_exp), _ptr(start), _ptr(count))
     return st, start, count
 
 
@@ -179,11 +179,11 @@ def e4m3_to_float(c: int) -> float:
     return float(lib().oracle_e4m3_to_float(int(c)))
 
 
-def expert_scale(windows_u16, H: int, E: int, R: int, C: int, n_exp, scale_u16) -> int:
+def expert_scale(windows_u16, H: int, E: int, R: int, C: int, n_exp, scale_u16, align: int = 1) -> int:
     n_exp = _c(n_exp, np.int32)
     scale_u16 = _c(scale_u16, np.uint16)
     assert windows_u16.dtype == np.uint16 and windows_u16.flags["C_CONTIGUOUS"]
-    return lib().oracle_expert_scale(_ptr(windows_u16), H, E, R, int(C), _ptr(n_exp), _ptr(scale_u16))
+    return lib().oracle_expert_scale(_ptr(windows_u16), H, E, R, int(C), int(align), _ptr(n_exp), _ptr(scale_u16))
 
 
 def combine(windows_u16, slots_, W, H: int, n_threads: int = 1):

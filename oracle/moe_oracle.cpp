@@ -148,9 +148,12 @@ int oracle_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32
   return ORACLE_OK;
 }
 
-int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t* c_rank, int32_t* o, int32_t* n_exp,
-                  int32_t* n_recv) {
-  if (E < 1 || R < 1 || E % R != 0) return ORACLE_ERR_INVALID_ARG;
+// Smallest multiple of `align` that is >= rows.
+static int64_t round_up_rows(int64_t rows, int32_t align) { return (rows + align - 1) / align * align; }
+
+int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t align, int32_t* c_rank, int32_t* o,
+                  int32_t* n_exp, int32_t* n_recv) {
+  if (E < 1 || R < 1 || E % R != 0 || align < 1) return ORACLE_ERR_INVALID_ARG;
   const int32_t E_r = E / R;
   // Per-rank branch counts: c_rank[r,d] = sum over experts of rank d of M[r,e].
   for (int32_t r = 0; r < R; ++r)
@@ -163,7 +166,9 @@ int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t* c_rank, int32
   // Notify: receive counts, then large offsets.  Inside the window of rank d
   // the blocks follow each other expert by expert (ascending), and inside an
   // expert source rank by source rank (ascending); o[e,r] is where block
-  // (r -> e) begins, counted from the start of rank d's window.
+  // (r -> e) begins, counted from the start of rank d's window.  With
+  // align > 1 the run of every expert is padded to a whole number of
+  // `align`-row groups, so every expert starts on a multiple of align.
   for (int32_t e = 0; e < E; ++e) {
     int32_t acc = 0;
     for (int32_t r = 0; r < R; ++r) acc += M[(size_t)r * E + e];
@@ -171,21 +176,23 @@ int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t* c_rank, int32
   }
   for (int32_t d = 0; d < R; ++d) {
     int32_t acc = 0;
-    for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e)
+    for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) {
       for (int32_t r = 0; r < R; ++r) {
         o[(size_t)e * R + r] = acc;
         acc += M[(size_t)r * E + e];
       }
+      acc = (int32_t)round_up_rows(acc, align);
+    }
     n_recv[d] = acc;
   }
   return ORACLE_OK;
 }
 
 int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
-                const int32_t* rank_tok_start,
+                const int32_t* rank_tok_start, int32_t align,
                 int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
                 int32_t* n_exp, int32_t* n_recv) {
-  if (!shape_ok(T, K, E, R, rank_tok_start)) return ORACLE_ERR_INVALID_ARG;
+  if (!shape_ok(T, K, E, R, rank_tok_start) || align < 1) return ORACLE_ERR_INVALID_ARG;
   if (T > 0 && topk_idx == nullptr) return ORACLE_ERR_INVALID_ARG;
   const int64_t B = (int64_t)T * K;
 
@@ -207,7 +214,7 @@ int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_
   for (int32_t r = 0; r < R; ++r)
     for (int32_t e = 0; e < E; ++e) M[(size_t)r * E + e] = run[(size_t)r * E + e];
 
-  return oracle_notify(M, E, R, c_rank, o, n_exp, n_recv);
+  return oracle_notify(M, E, R, align, c_rank, o, n_exp, n_recv);
 }
 
 int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
@@ -231,16 +238,16 @@ int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32
   return ORACLE_OK;
 }
 
-int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, const int32_t* n_exp,
+int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, int32_t align, const int32_t* n_exp,
                          int64_t* row_start, int32_t* row_count) {
-  if (E < 1 || R < 1 || E % R != 0 || C < 0) return ORACLE_ERR_INVALID_ARG;
+  if (E < 1 || R < 1 || E % R != 0 || C < 0 || align < 1) return ORACLE_ERR_INVALID_ARG;
   const int32_t E_r = E / R;
   for (int32_t d = 0; d < R; ++d) {
-    int64_t row = (int64_t)d * C;
+    int64_t local = 0;   // row inside window d
     for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) {
-      row_start[e] = row;
+      row_start[e] = (int64_t)d * C + local;
       row_count[e] = n_exp[e];
-      row += n_exp[e];
+      local = round_up_rows(local + n_exp[e], align);
     }
   }
   return ORACLE_OK;
@@ -258,19 +265,22 @@ int oracle_dispatch(const uint16_t* X, int32_t T, int32_t H, int32_t K,
   return ORACLE_OK;
 }
 
-int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int64_t C,
+int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int64_t C, int32_t align,
                         const int32_t* n_exp, const uint16_t* scale) {
-  if (H < 1 || E < 1 || R < 1 || E % R != 0) return ORACLE_ERR_INVALID_ARG;
+  if (H < 1 || E < 1 || R < 1 || E % R != 0 || align < 1) return ORACLE_ERR_INVALID_ARG;
   const int32_t E_r = E / R;
   for (int32_t d = 0; d < R; ++d) {
-    int64_t row = (int64_t)d * C;
+    int64_t local = 0;   // row inside window d
     for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) {
       const float sc = oracle_bf16_to_float(scale[e]);
-      for (int32_t i = 0; i < n_exp[e]; ++i, ++row)
+      for (int32_t i = 0; i < n_exp[e]; ++i) {
+        const int64_t row = (int64_t)d * C + local + i;
         for (int32_t h = 0; h < H; ++h) {
           uint16_t* p = windows + row * H + h;
           *p = oracle_float_to_bf16(oracle_bf16_to_float(*p) * sc);
         }
+      }
+      local = round_up_rows(local + n_exp[e], align);   // padding rows are not the expert's
     }
   }
   return ORACLE_OK;

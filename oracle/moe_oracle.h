@@ -51,17 +51,26 @@ int oracle_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32
  *                 dst(e) = e / E_r, of the block (source rank r -> expert e);
  *                 blocks are laid out expert-major, then source rank       (Notify, definition of o)
  *   n_exp  [E]    rows received by expert e;  n_recv [R] rows received by rank d.
- * The decode schedule keeps only (o, s); its values are these same ones (Section 5.3). */
+ * The decode schedule keeps only (o, s); its values are these same ones (Section 5.3).
+ *
+ * align (>= 1) is this library's consumer-side extension; the paper has no counterpart and align = 1
+ * is its layout.  With align = A > 1 the run of every expert is padded to a whole number of A-row
+ * groups, so that every expert's first row is a multiple of A inside its window (a grouped GEMM
+ * that reads the window in place in tiles of A rows never sees two experts in one tile):
+ *   start_e = sum over earlier experts e' of the same rank of ceil(n_exp[e'] / A) * A,
+ *   o[e,r]  = start_e + sum_{r' < r} M[r',e],
+ *   n_recv[d] = sum over the experts of rank d of ceil(n_exp[e] / A) * A   (rows the window must hold);
+ * n_exp stays the true count, and the padding rows are never written nor read. */
 int oracle_plan(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32_t R,
-                const int32_t* rank_tok_start,
+                const int32_t* rank_tok_start, int32_t align,
                 int32_t* M, int32_t* c_rank, int32_t* s, int32_t* o,
                 int32_t* n_exp, int32_t* n_recv);
 
 /* Notify on its own (Section 5.2, Prefill Notify): from the gathered count matrix M [R,E] -- in a
  * real expert-parallel group every rank contributes its row -- the large offsets o [E,R], the
  * receive counts n_exp [E], n_recv [R] and c_rank [R,R].  oracle_plan is Layout followed by this. */
-int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t* c_rank, int32_t* o, int32_t* n_exp,
-                  int32_t* n_recv);
+int oracle_notify(const int32_t* M, int32_t E, int32_t R, int32_t align, int32_t* c_rank, int32_t* o,
+                  int32_t* n_exp, int32_t* n_recv);
 
 /* Expert-window row of every branch (two-level offset rule, Section 5.1; Algorithm 1):
  *   slot[t,j] = dst(e) * C + o[e, src(t)] + s[t,j],  e = K[t,j].
@@ -73,9 +82,9 @@ int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32
 
 /* Row range of every expert inside the window allocation: the expert FFNs consume the windows in
  * place, without further reordering (Section 5.2, Expert computation), so each expert's rows are one
- * contiguous run:  row_start[e] = dst(e) * C + (rows of earlier experts of the same rank),
- * row_count[e] = n_exp[e]. */
-int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, const int32_t* n_exp,
+ * contiguous run:  row_start[e] = dst(e) * C + (rows, padded to groups of `align`, of earlier experts
+ * of the same rank), row_count[e] = n_exp[e]. */
+int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, int32_t align, const int32_t* n_exp,
                          int64_t* row_start, int32_t* row_count);
 
 /* Dispatch (Algorithm 1, first loop): copy row X[t,:] to window row slot[t,j]
@@ -88,8 +97,9 @@ int oracle_dispatch(const uint16_t* X, int32_t T, int32_t H, int32_t K,
  * every received row of expert e by the bf16 scalar scale[e]:
  *   y = bf16_rne(float(x) * float(scale[e])).
  * Rows of expert e are rows start_e .. start_e + n_exp[e] - 1 of its rank's
- * segment, start_e = sum of n_exp over earlier experts of the same rank. */
-int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int64_t C,
+ * segment, start_e = sum of n_exp (each padded to a multiple of `align`) over earlier experts of the
+ * same rank. */
+int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int64_t C, int32_t align,
                         const int32_t* n_exp, const uint16_t* scale);
 
 /* Combine (Algorithm 1, second loop):

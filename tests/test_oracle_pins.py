@@ -569,3 +569,98 @@ def test_layout_per_rank_plus_notify_equals_the_global_plan():
     assert st == oracle.OK and np.array_equal(M, whole.M)
     for a, b in ((c_rank, whole.c_rank), (o, whole.o), (n_exp, whole.n_exp), (n_recv, whole.n_recv)):
         assert np.array_equal(a, b)
+
+
+# ----------------------------------------------------------------------------- aligned expert starts
+@pytest.mark.parametrize("align", [1, 2, 8, 128])
+@pytest.mark.parametrize("case", list(cases()), ids=lambda c: f"T{c[0]}K{c[1]}E{c[2]}R{c[3]}{'rep' if c[4] else ''}")
+def test_aligned_layout_against_library_routines(case, align):
+    """Expert runs padded to groups of `align` rows: counts and small offsets do not change, starts are
+    the exclusive cumulative sum (numpy) of the padded expert counts, restarting per window, and the
+    branches of an expert still fill [start, start + count) in stable order."""
+    T, K, E, R, _, idx, rts = case
+    base = oracle.plan(idx, E, R, rts)
+    p = oracle.plan(idx, E, R, rts, align=align)
+    assert p.status == oracle.OK
+    E_r = E // R
+    for name in ("M", "c_rank", "s", "n_exp"):
+        assert np.array_equal(getattr(p, name), getattr(base, name)), name
+    padded = -(-p.n_exp.astype(np.int64) // align) * align
+    per_window = padded.reshape(R, E_r)
+    start = (np.cumsum(per_window, 1) - per_window).reshape(-1)            # local first row of every expert
+    assert (start % align == 0).all()
+    within = np.cumsum(p.M.T, 1) - p.M.T                                    # [E,R]: rows of earlier source ranks
+    assert np.array_equal(p.o, start[:, None] + within)
+    assert np.array_equal(p.n_recv, per_window.sum(1))
+    if align == 1:
+        assert np.array_equal(p.o, base.o) and np.array_equal(p.n_recv, base.n_recv)
+
+    C = int(p.n_recv.max()) + align
+    st, slots = oracle.slots(idx, E, R, p, C, rts)
+    assert st == oracle.OK
+    st, e_start, e_count = oracle.expert_ranges(E, R, C, p.n_exp, align=align)
+    assert st == oracle.OK
+    assert np.array_equal(e_start, (np.arange(E) // E_r) * C + start) and np.array_equal(e_count, p.n_exp)
+    flat_e, flat_slot = idx.reshape(-1), slots.reshape(-1)
+    assert len(np.unique(flat_slot)) == T * K                               # no two branches share a row
+    for e in range(E):
+        rows = flat_slot[flat_e == e]                                       # flat (t, j) order = stable order
+        assert np.array_equal(rows, e_start[e] + np.arange(p.n_exp[e]))
+    # one row short of the padded need is a capacity error
+    if T:
+        assert oracle.slots(idx, E, R, p, int(p.n_recv.max()) - 1, rts)[0] == oracle.ERR_CAPACITY
+
+
+def test_aligned_layout_moves_rows_but_not_results():
+    """Dispatch + scale experts + combine give bit-identical Y for every alignment, and padding rows
+    keep the caller's bytes."""
+    rng = np.random.default_rng(77)
+    T, K, E, R, H = 150, 4, 12, 3, 24
+    idx, rts = random_case(rng, T, K, E, R, replace=True)
+    X = rand_bf16(rng, (T, H))
+    W = rng.random((T, K), dtype=np.float32)
+    scale = rand_bf16(rng, (E,))
+    outs = []
+    for align in (1, 4, 16):
+        p = oracle.plan(idx, E, R, rts, align=align)
+        C = int(p.n_recv.max())
+        st, slots = oracle.slots(idx, E, R, p, C, rts)
+        win = np.full((R * C, H), 0x7FC1, np.uint16)
+        assert oracle.dispatch(X, slots, win) == oracle.OK
+        used = np.zeros(R * C, bool)
+        used[slots.reshape(-1)] = True
+        assert (win[~used] == 0x7FC1).all() and used.sum() == T * K
+        assert oracle.expert_scale(win, H, E, R, C, p.n_exp, scale, align=align) == oracle.OK
+        assert (win[~used] == 0x7FC1).all()                                 # the expert op skips padding rows
+        st, Y = oracle.combine(win, slots, W, H)
+        outs.append(Y)
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+def test_aligned_notify_rejects_bad_alignment():
+    M = np.ones((2, 4), np.int32)
+    assert oracle.notify(M, align=0)[0] == oracle.ERR_INVALID_ARG
+    st, c_rank, o, n_exp, n_recv = oracle.notify(M, align=4)
+    assert st == oracle.OK and list(n_recv) == [8, 8] and list(o[:, 0]) == [0, 4, 0, 4] and list(o[:, 1]) == [1, 5, 1, 5]
+
+
+def test_brute_force_all_routings_tiny_aligned():
+    """The same 4^6 routings with expert runs padded to 4 rows, against the literal definition: an
+    expert starts after the padded runs of the earlier experts of its window, and inside the run the
+    blocks of lower source ranks come first."""
+    T, K, E, R, A = 3, 2, 4, 2, 4
+    rts = np.array([0, 2, 3], np.int32)
+    src = [0, 0, 1]
+    E_r = E // R
+    branches = [(t, j) for t in range(T) for j in range(K)]
+    for combo in itertools.product(range(E), repeat=T * K):
+        idx = np.array(combo, np.int32).reshape(T, K)
+        p = oracle.plan(idx, E, R, rts, align=A)
+        count = [sum(1 for (t, j) in branches if idx[t, j] == e) for e in range(E)]
+        for e in range(E):
+            start = sum(-(-count[e2] // A) * A for e2 in range((e // E_r) * E_r, e))
+            for r in range(R):
+                lower = sum(1 for (t, j) in branches if idx[t, j] == e and src[t] < r)
+                assert p.o[e, r] == start + lower
+        for d in range(R):
+            assert p.n_recv[d] == sum(-(-count[e] // A) * A for e in range(d * E_r, (d + 1) * E_r))
