@@ -244,12 +244,23 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
  *   MOE_OPT_OVERLAP        1 (default): moe_plan_dispatch starts its dispatch kernel while the planner
  *                          runs (programmatic stream serialization; the early part of the kernel
  *                          reads nothing the planner writes).  0: the dispatch kernel starts after the
- *                          planner has ended.  Same result either way. */
+ *                          planner has ended.  Same result either way.
+ *   MOE_OPT_EXPERT_ALIGN   A in [1, 4096], default 1 (the packed layout of Section 5.2).  With A > 1 later
+ *                          plans pad the run of every expert to a whole number of A-row groups, so that
+ *                          every expert's first row is a multiple of A inside its window and a grouped
+ *                          GEMM can read the window in place in tiles of A rows without two experts in
+ *                          one tile.  (No counterpart in the paper; an extension for the consumer of the
+ *                          windows.)  n_exp stays the true count; large_off includes the padding of
+ *                          earlier experts; n_recv[d] becomes the sum over the experts of rank d of
+ *                          ceil(n_exp[e] / A) * A, which is what capacity_rows is checked against.
+ *                          Padding rows are never written by dispatch nor read by combine.  Setting the
+ *                          option invalidates the current plan. */
 typedef enum {
   MOE_OPT_DISPATCH_PATH = 0,
   MOE_OPT_GRANULE = 1,
   MOE_OPT_TEST_STARVE_WAIT_MS = 2,
-  MOE_OPT_OVERLAP = 3
+  MOE_OPT_OVERLAP = 3,
+  MOE_OPT_EXPERT_ALIGN = 4
 } moe_option_t;
 enum { MOE_DISPATCH_AUTO = 0, MOE_DISPATCH_REGISTERS = 1, MOE_DISPATCH_BULK = 2 };
 moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);

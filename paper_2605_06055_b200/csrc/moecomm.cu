@@ -41,6 +41,7 @@ struct moe_ctx {
   int32_t granule_override; // MOE_OPT_GRANULE
   int32_t starve_wait_ms;   // MOE_OPT_TEST_STARVE_WAIT_MS
   int32_t overlap;          // MOE_OPT_OVERLAP
+  int32_t expert_align;     // MOE_OPT_EXPERT_ALIGN: every expert's run starts on a multiple of this many rows
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
   cudaEvent_t fwd_events[2 * 16 + 2];
@@ -304,6 +305,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->granule_override = 0;
   ctx->starve_wait_ms = 0;
   ctx->overlap = 1;
+  ctx->expert_align = 1;
   ctx->out_stream = nullptr;
   ctx->in_stream = nullptr;
   ctx->occ_n = 0;
@@ -425,10 +427,12 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
   if (ctx->compact_plan) {
     if (wide)
       plan_rank_kernel<32><<<sh.R, 32 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+          topk_idx, map, sh.K, sh.E, full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp,
+          ctx->n_recv, ctx->ctl);
     else
       plan_rank_kernel<8><<<sh.R, 8 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+          topk_idx, map, sh.K, sh.E, full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp,
+          ctx->n_recv, ctx->ctl);
     ++n;
   } else {
     if (tiles > 0) {
@@ -440,8 +444,8 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
             topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
       ++n;
     }
-    plan_scan_kernel<<<sh.R, PLAN_THREADS, scan_smem, st>>>(ctx->tile_hist, map, sh.E, full, ctx->M, ctx->c_rank,
-                                                            ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+    plan_scan_kernel<<<sh.R, PLAN_THREADS, scan_smem, st>>>(ctx->tile_hist, map, sh.E, full, ctx->expert_align, ctx->M,
+                                                            ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
     ++n;
     if (full && tiles > 0) {
       plan_finalize_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, 0, st>>>(topk_idx, map, sh.K, sh.E, ctx->tile_rank,
@@ -680,7 +684,8 @@ moe_status_t moe_notify(moe_ctx_t* ctx, const int32_t* counts_all, void* stream)
   if (!ctx->layout_done) return MOE_ERR_NOT_PLANNED;
   const moe_shape_t& sh = ctx->shape;
   notify_kernel<<<1, 1024, notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t), static_cast<cudaStream_t>(stream)>>>(
-      counts_all, sh.E, sh.R, ctx->schedule == MOE_SCHED_PREFILL, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv);
+      counts_all, sh.E, sh.R, ctx->schedule == MOE_SCHED_PREFILL, ctx->expert_align, ctx->M, ctx->c_rank, ctx->o,
+      ctx->n_exp, ctx->n_recv);
   const moe_status_t rc = launch_ok(ctx);
   if (rc == MOE_OK) ctx->planned = true;
   return rc;
@@ -789,6 +794,14 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) 
     case MOE_OPT_GRANULE:
       if (value < 0 || value > (1 << 20)) return MOE_ERR_INVALID_ARG;
       ctx->granule_override = (int32_t)value;
+      return MOE_OK;
+    case MOE_OPT_EXPERT_ALIGN:
+      if (value < 1 || value > 4096) return MOE_ERR_INVALID_ARG;
+      if ((int64_t)ctx->shape.T_max * ctx->shape.K + (int64_t)ctx->shape.E * (value - 1) >= ((int64_t)1 << 31))
+        return MOE_ERR_INVALID_ARG;   // padded row counts must stay in int32
+      ctx->expert_align = (int32_t)value;
+      ctx->planned = false;           // offsets of an earlier plan no longer describe the layout asked for
+      ctx->layout_done = false;
       return MOE_OK;
     case MOE_OPT_OVERLAP:
       if (value != 0 && value != 1) return MOE_ERR_INVALID_ARG;
@@ -930,7 +943,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
     plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, PLAN_WARPS * E * (int)sizeof(int32_t), st>>>(
         topk_idx, map, K, E, sc->tile_rank, sc->tile_hist, status);
   plan_scan_kernel<<<R, PLAN_THREADS, notify_smem_ints(E, R) * (int)sizeof(int32_t), st>>>(
-      sc->tile_hist, map, E, 0, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl);
+      sc->tile_hist, map, E, 0, 1, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl);
   RowArgs a;
   a.topk_idx = topk_idx;
   a.small_off = sc->tile_rank;

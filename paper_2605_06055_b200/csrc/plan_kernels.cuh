@@ -156,7 +156,7 @@ __host__ __device__ constexpr int notify_smem_ints(int E, int R) {
 // Direct path (large R*E): loads first and in batches; no store sits between two loads, because the
 // compiler cannot know that o and M never overlap and would serialise them at one L2 round trip each.
 __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ M, int32_t E, int32_t R,
-                                                    int32_t full_table, int32_t* __restrict__ c_rank,
+                                                    int32_t full_table, int32_t align, int32_t* __restrict__ c_rank,
                                                     int32_t* __restrict__ o, int32_t* __restrict__ n_exp,
                                                     int32_t* __restrict__ n_recv, int32_t* sm) {
   int32_t* nexp_s = sm;
@@ -189,7 +189,7 @@ __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ 
 #pragma unroll 16
       for (int rr = 0; rr < R; ++rr) acc += __ldcg(M + (size_t)rr * E + e);
     }
-    nexp_s[e] = acc;
+    nexp_s[e] = (acc + align - 1) / align * align;   // rows the expert's run occupies (align = 1: its count)
     n_exp[e] = acc;
   }
   __syncthreads();
@@ -238,7 +238,7 @@ __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ 
 
 __global__ void __launch_bounds__(PLAN_THREADS)
 plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusive bases */,
-                 const __grid_constant__ RankMap map, int32_t E, int32_t full_table,
+                 const __grid_constant__ RankMap map, int32_t E, int32_t full_table, int32_t align,
                  int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
                  int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
   extern __shared__ int32_t sm[];  // notify_smem_ints(E, R) ints
@@ -271,7 +271,7 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
   if (!is_last) return;
   __threadfence();
 
-  build_large_offsets(M, E, R, full_table, c_rank, o, n_exp, n_recv, sm);
+  build_large_offsets(M, E, R, full_table, align, c_rank, o, n_exp, n_recv, sm);
   if (threadIdx.x == 0) ctl->scan_ticket = 0;  // ready for the next plan on this stream
 }
 
@@ -290,7 +290,8 @@ __host__ __device__ constexpr int rank_plan_smem_ints(int E, int R, int warps) {
 template <int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
-                 int32_t full_table, int32_t* __restrict__ s, int32_t* __restrict__ M, int32_t* __restrict__ c_rank,
+                 int32_t full_table, int32_t align, int32_t* __restrict__ s, int32_t* __restrict__ M,
+                 int32_t* __restrict__ c_rank,
                  int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
@@ -365,21 +366,21 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  build_large_offsets(M, E, R, full_table, c_rank, o, n_exp, n_recv, sm);
+  build_large_offsets(M, E, R, full_table, align, c_rank, o, n_exp, n_recv, sm);
   if (threadIdx.x == 0) ctl->scan_ticket = 0;
 }
 
 // Notify from a count matrix gathered elsewhere (multi-rank use: every rank contributed its row):
 // installs it as M and rebuilds the large offsets and receive counts.  One CTA.
 __global__ void __launch_bounds__(1024)
-notify_kernel(const int32_t* __restrict__ counts_all, int32_t E, int32_t R, int32_t full_table,
+notify_kernel(const int32_t* __restrict__ counts_all, int32_t E, int32_t R, int32_t full_table, int32_t align,
               int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
               int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
   extern __shared__ int32_t sm[];
   for (int i = threadIdx.x; i < R * E; i += blockDim.x) M[i] = counts_all[i];
   __threadfence_block();
   __syncthreads();
-  build_large_offsets(M, E, R, full_table, c_rank, o, n_exp, n_recv, sm);
+  build_large_offsets(M, E, R, full_table, align, c_rank, o, n_exp, n_recv, sm);
 }
 
 template <int ROUNDS>

@@ -37,19 +37,24 @@ def max_ulp_diff(got_u16: np.ndarray, want_u16: np.ndarray) -> int:
 
 
 def gpu_expert_scale(windows: torch.Tensor, topk_idx: torch.Tensor, E: int, R: int, C: int,
-                     scale: torch.Tensor) -> None:
+                     scale: torch.Tensor, align: int = 1) -> None:
     """Stand-in expert op on the device (harness code, not the library):
-    every received row of expert e is multiplied by the bf16 scalar scale[e]."""
+    every received row of expert e is multiplied by the bf16 scalar scale[e]; with align > 1 the
+    padding rows behind an expert's run get the factor 1 (they stay as they are)."""
     n_exp = torch.bincount(topk_idx.reshape(-1).long(), minlength=E)
     E_r = E // R
     win = windows.view(R, C, -1)
     for d in range(R):
         cnt = n_exp[d * E_r:(d + 1) * E_r]
-        rows = int(cnt.sum())
+        pad = (cnt + align - 1) // align * align - cnt
+        rows = int((cnt + pad).sum())
         if rows == 0:
             continue
-        row_scale = torch.repeat_interleave(scale[d * E_r:(d + 1) * E_r], cnt)
-        win[d, :rows] = win[d, :rows] * row_scale[:, None]     # bf16*bf16: fp32 product, one RNE rounding
+        runs = torch.stack([cnt, pad], 1).reshape(-1)                       # count, padding, count, padding, ...
+        factors = torch.stack([scale[d * E_r:(d + 1) * E_r]] * 2, 1).reshape(-1)
+        real = torch.repeat_interleave(torch.tensor([True, False] * E_r, device=scale.device), runs)
+        row_scale = torch.repeat_interleave(factors, runs)
+        win[d, :rows][real] = win[d, :rows][real] * row_scale[real][:, None]   # bf16*bf16: fp32 product, one RNE rounding
 
 
 @dataclass
@@ -61,10 +66,10 @@ class OracleRun:
     windows_zero_init: np.ndarray = None   # the same dispatch into zero-filled windows
 
 
-def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4) -> OracleRun:
+def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4, align: int = 1) -> OracleRun:
     wl = inp.wl
     idx = inp.topk_idx.numpy()
-    p = oracle.plan(idx, wl.E, wl.R, inp.rank_tok_start)
+    p = oracle.plan(idx, wl.E, wl.R, inp.rank_tok_start, align=align)
     assert p.status == oracle.OK
     st, slots = oracle.slots(idx, wl.E, wl.R, p, C, inp.rank_tok_start)
     assert st == oracle.OK
@@ -72,7 +77,8 @@ def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4) -> OracleRun:
     assert oracle.dispatch(synth.bf16_to_u16(inp.X), slots, win, n_threads) == oracle.OK
     win_after_dispatch = win.copy()
     if wl.expert_op == "scale":
-        assert oracle.expert_scale(win, wl.H, wl.E, wl.R, C, p.n_exp, synth.bf16_to_u16(inp.scale)) == oracle.OK
+        assert oracle.expert_scale(win, wl.H, wl.E, wl.R, C, p.n_exp, synth.bf16_to_u16(inp.scale),
+                                   align=align) == oracle.OK
     st, Y = oracle.combine(win, slots, inp.topk_w.numpy(), wl.H, n_threads)
     assert st == oracle.OK
     zero_init = np.where(win_after_dispatch == CANARY, np.uint16(0), win_after_dispatch)
@@ -95,7 +101,8 @@ class GpuRun:
 
 
 def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Optional[binding.MoeComm] = None,
-            T_max: Optional[int] = None, dispatch_path: int = binding.MOE_DISPATCH_AUTO, granule: int = 0) -> GpuRun:
+            T_max: Optional[int] = None, dispatch_path: int = binding.MOE_DISPATCH_AUTO, granule: int = 0,
+            align: int = 1) -> GpuRun:
     wl = inp.wl
     dev = torch.device("cuda:0")
     schedule = wl.schedule if schedule is None else schedule
@@ -104,6 +111,7 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
         comm = binding.MoeComm(T_max or max(wl.T, 1), wl.H, wl.E, wl.R, wl.K, dev)
     comm.moe_set_option(binding.MOE_OPT_DISPATCH_PATH, dispatch_path)
     comm.moe_set_option(binding.MOE_OPT_GRANULE, granule)
+    comm.moe_set_option(binding.MOE_OPT_EXPERT_ALIGN, align)
     idx = inp.topk_idx.to(dev)
     w = inp.topk_w.to(dev)
     X = inp.X.to(dev)
@@ -122,7 +130,7 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
     view = {k: (None if v is None else v.cpu().numpy().copy()) for k, v in comm.moe_plan_view().items()}
     win_host = windows.cpu().view(torch.int16).numpy().view(np.uint16).copy()
     if wl.expert_op == "scale":
-        gpu_expert_scale(windows, idx, wl.E, wl.R, C, inp.scale.to(dev))
+        gpu_expert_scale(windows, idx, wl.E, wl.R, C, inp.scale.to(dev), align)
     Y = torch.from_numpy(np.full((wl.T, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
     comm.moe_combine(windows, C, w, Y)
     statuses.append(comm.moe_status())
@@ -133,7 +141,7 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
     return out
 
 
-def assert_parity(g: GpuRun, o: OracleRun, schedule: int, combine_ulp: int = 1):
+def assert_parity(g: GpuRun, o: OracleRun, schedule: int, combine_ulp: int = 1, align: int = 1):
     assert g.statuses == [0, 0, 0], g.statuses
     names = {"counts": "M", "c_rank": "c_rank", "small_off": "s", "large_off": "o", "n_exp": "n_exp", "n_recv": "n_recv"}
     for k, on in names.items():
@@ -143,7 +151,7 @@ def assert_parity(g: GpuRun, o: OracleRun, schedule: int, combine_ulp: int = 1):
         assert np.array_equal(g.view[k], getattr(o.plan, on)), k          # bit-exact integers
     assert np.array_equal(g.slots.astype(np.int64), o.slots)
     E, R = o.plan.o.shape
-    st, want_start, want_count = oracle.expert_ranges(E, R, g.windows.shape[0] // R, o.plan.n_exp)
+    st, want_start, want_count = oracle.expert_ranges(E, R, g.windows.shape[0] // R, o.plan.n_exp, align=align)
     assert st == oracle.OK and np.array_equal(g.expert_start, want_start) and np.array_equal(g.expert_count, want_count)
     assert np.array_equal(g.windows, o.windows)                           # bit-exact rows and canaries
     ulp = max_ulp_diff(g.Y, o.Y)

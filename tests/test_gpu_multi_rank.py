@@ -25,22 +25,24 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("align", [1, 16])
 @pytest.mark.parametrize("path", [binding.MOE_DISPATCH_BULK, binding.MOE_DISPATCH_REGISTERS])
 @pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
-def test_per_rank_contexts_and_separate_windows_reproduce_the_global_result(case, path):
+def test_per_rank_contexts_and_separate_windows_reproduce_the_global_result(case, path, align):
     name, T, H, E, R, K, sch, routing, per = case
     dev = torch.device("cuda:0")
     wl = Workload(name, T, H, E, R, K, sch, routing, "scale", 7000 + T, rank_tokens=per)
     inp = synth.make_inputs(wl)
     rts = inp.rank_tok_start
-    p = oracle.plan(inp.topk_idx.numpy(), E, R, rts)
+    p = oracle.plan(inp.topk_idx.numpy(), E, R, rts, align=align)
     C = int(p.n_recv.max()) + 1
-    want = harness.oracle_run(inp, C)
+    want = harness.oracle_run(inp, C, align=align)
 
     idx, w, X = inp.topk_idx.to(dev), inp.topk_w.to(dev), inp.X.to(dev)
     comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
     for c in comms:
         c.moe_set_option(binding.MOE_OPT_DISPATCH_PATH, path)
+        c.moe_set_option(binding.MOE_OPT_EXPERT_ALIGN, align)
     # Layout on every rank, then the count "all-gather" (here: rows of one tensor), then Notify on every rank
     counts = torch.full((R, E), -1, dtype=torch.int32, device=dev)
     for r, c in enumerate(comms):
@@ -64,7 +66,7 @@ def test_per_rank_contexts_and_separate_windows_reproduce_the_global_result(case
     assert np.array_equal(got, want.windows)
     # experts (harness op on the concatenated view), then every rank combines its own tokens from all windows
     allwin = torch.cat(windows)
-    harness.gpu_expert_scale(allwin, idx, E, R, C, inp.scale.to(dev))
+    harness.gpu_expert_scale(allwin, idx, E, R, C, inp.scale.to(dev), align)
     for d in range(R):
         windows[d].copy_(allwin[d * C:(d + 1) * C])
     Y = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
