@@ -357,6 +357,26 @@ def time_repeated(fns, n: int) -> float:
     return a.elapsed_time(b) * 1e3 / n
 
 
+def call_latency(layer: Layer, n: int, flush=None) -> dict:
+    """Per-call latency as differences of cumulative call sequences (plan | plan+dispatch | plan+dispatch+combine),
+    each timed over n repetitions between one pair of CUDA events; `flush` (an L2-flushing call) precedes every
+    repetition and its own time is subtracted."""
+    c, wl = layer.comm, layer.wl
+    plan = lambda: c.moe_plan(wl.schedule, layer.idx)
+    disp = lambda: c.moe_dispatch(layer.X, layer.windows, layer.C)
+    comb = lambda: c.moe_combine(layer.windows, layer.C, layer.w, layer.Y)
+    fused = lambda: c.moe_plan_dispatch(wl.schedule, layer.idx, layer.X, layer.windows, layer.C)
+    pre = [flush] if flush is not None else []
+    base = time_repeated(pre, n) if pre else 0.0
+    t1 = time_repeated(pre + [plan], n)
+    t2 = time_repeated(pre + [plan, disp], n)
+    t3 = time_repeated(pre + [plan, disp, comb], n)
+    tf = time_repeated(pre + [fused, comb], n)
+    assert c.moe_status() == 0
+    return {"plan_us": t1 - base, "dispatch_us": t2 - t1, "combine_us": t3 - t2, "step_us": t3 - base,
+            "step_us_plan_dispatch_fused": tf - base}
+
+
 def decode_latency(dev, peak, n: int = 200) -> dict:
     """Decode-step latency (config 2).  Per-call figures are differences of cumulative sequences
     (flush | flush+plan | flush+plan+dispatch | ...), each timed over n repetitions."""
@@ -535,23 +555,29 @@ def run_cuda(args, wl):
         torch.cuda.empty_cache()
 
     if world == 1 and args.workload == "c5" and not args.no_decode:
-        # config 5: both schedules timed at each T of the sweep (per-call medians, L2 flushed between steps)
+        # config 5: both schedules timed at each T of the sweep.  Calls of a few microseconds cannot be timed by
+        # one event pair each (the events tick in ~2 us steps), so every figure is a difference of cumulative
+        # call sequences; the L2 is flushed before every step while the windows are not far larger than it.
         line["sweep"] = []
-        flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+        flush_buf = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+        flush = lambda: flush_buf.add_(1)
         for T in (128, 1024, 8192, 65536):
             for sch in (synth.PREFILL, synth.DECODE):
                 swl = synth.config(5, T, sch)
                 sl = Layer(swl, dev)
-                sr = time_steps(sl, 50, 5, barrier, flush)
-                sk = kernel_table(swl, sr, peak)
-                line["sweep"].append({"T": T, "schedule": "prefill" if sch == synth.PREFILL else "decode",
-                                      "plan_us": sk["moe_plan"]["us"], "dispatch_us": sk["moe_dispatch"]["us"],
-                                      "combine_us": sk["moe_combine"]["us"],
-                                      "dispatch_GBps": sk["moe_dispatch"]["GBps"],
-                                      "combine_GBps": sk["moe_combine"]["GBps"],
-                                      "bytes_per_call": bytes_dispatch(swl)})
+                if T <= 8192:
+                    lat = call_latency(sl, 200, flush)
+                else:   # calls of hundreds of microseconds: one event pair per call attributes the time best
+                    sr = time_steps(sl, 50, 5, barrier)
+                    lat = {"plan_us": statistics.median(sr["plan_us"]), "dispatch_us": statistics.median(sr["dispatch_us"]),
+                           "combine_us": statistics.median(sr["combine_us"]), "step_us": sr["ms_per_step"] * 1e3}
+                line["sweep"].append(dict({"T": T, "schedule": "prefill" if sch == synth.PREFILL else "decode",
+                                           "l2": "flushed before every step" if T <= 8192 else "windows far larger than L2",
+                                           "dispatch_GBps": bytes_dispatch(swl) / lat["dispatch_us"] / 1e3,
+                                           "combine_GBps": bytes_combine(swl) / lat["combine_us"] / 1e3,
+                                           "bytes_per_call": bytes_dispatch(swl)}, **lat))
                 del sl
-        del flush
+        del flush_buf
         torch.cuda.empty_cache()
 
     if world == 1 and not args.no_cpu_baseline:
