@@ -141,6 +141,20 @@ def _stream_handle(stream) -> int:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
+class _NoSwitch:
+    """Stands in for torch.cuda.device(...) when the context's device is already current
+    (entering the real guard costs several microseconds per call)."""
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        return False
+
+
+_NO_SWITCH = _NoSwitch()
+
+
 class MoeComm:
     """One libmoecomm context (opaque handle + its torch-allocated workspace)."""
 
@@ -152,6 +166,7 @@ class MoeComm:
         nbytes = int(self.lib.moe_workspace_bytes(ctypes.byref(self._shape)))
         if nbytes == 0:
             raise MoeError(MOE_ERR_INVALID_ARG, "moe_workspace_bytes")
+        self._dev_index = self.device.index if self.device.index is not None else torch.cuda.current_device()
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
             h = ctypes.c_void_p()
@@ -162,6 +177,10 @@ class MoeComm:
         self.T = 0
         self.schedule = None
         self._keep = None  # routing tensor of the live plan (the library re-reads it)
+
+    def _on_device(self):
+        """Context manager that makes this context's device current (free when it already is)."""
+        return _NO_SWITCH if torch.cuda.current_device() == self._dev_index else torch.cuda.device(self.device)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -179,7 +198,7 @@ class MoeComm:
                  stream=None, check: bool = True) -> int:
         T = topk_idx.shape[0] if T is None else T
         rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_plan(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, _host_ptr(rts),
                                    _stream_handle(stream))
         if rc == MOE_OK:
@@ -193,7 +212,7 @@ class MoeComm:
                           check: bool = True) -> int:
         T = topk_idx.shape[0] if T is None else T
         rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_plan_dispatch(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, _host_ptr(rts),
                                             _dev_ptr(x, torch.bfloat16), _dev_ptr(windows, torch.bfloat16),
                                             int(capacity_rows), _stream_handle(stream))
@@ -207,7 +226,7 @@ class MoeComm:
                       T: Optional[int] = None, rank_tok_start=None, stream=None, check: bool = True) -> int:
         T = logits.shape[0] if T is None else T
         rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_gate_plan(self._h, schedule, _dev_ptr(logits, torch.float32), T, _host_ptr(rts),
                                         _dev_ptr(topk_idx, torch.int32), _dev_ptr(topk_w, torch.float32),
                                         _stream_handle(stream))
@@ -219,7 +238,7 @@ class MoeComm:
 
     def moe_dispatch_range(self, x, windows, capacity_rows: int, t_begin: int, t_end: int, stream=None,
                            check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_dispatch_range(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(windows, torch.bfloat16),
                                              int(capacity_rows), t_begin, t_end, _stream_handle(stream))
         if rc != MOE_OK and check:
@@ -228,7 +247,7 @@ class MoeComm:
 
     def moe_combine_range(self, windows, capacity_rows: int, topk_w, y, t_begin: int, t_end: int, stream=None,
                           check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_combine_range(self._h, _dev_ptr(windows, torch.bfloat16), int(capacity_rows),
                                             _dev_ptr(topk_w, torch.float32), _dev_ptr(y, torch.bfloat16),
                                             t_begin, t_end, _stream_handle(stream))
@@ -240,7 +259,7 @@ class MoeComm:
     def moe_layout(self, schedule: int, topk_idx: torch.Tensor, my_rank: int, counts_row: torch.Tensor,
                    stream=None, check: bool = True) -> int:
         T = topk_idx.shape[0]
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_layout(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, my_rank,
                                      _dev_ptr(counts_row, torch.int32), _stream_handle(stream))
         if rc == MOE_OK:
@@ -250,7 +269,7 @@ class MoeComm:
         return rc
 
     def moe_notify(self, counts_all: torch.Tensor, stream=None, check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_notify(self._h, _dev_ptr(counts_all, torch.int32), _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_notify")
@@ -259,7 +278,7 @@ class MoeComm:
     def moe_dispatch_peers(self, x: torch.Tensor, window_bases: torch.Tensor, capacity_rows: int, stream=None,
                            check: bool = True) -> int:
         """window_bases: int64 CUDA tensor [R] holding the device address of every rank's window."""
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_dispatch_peers(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(window_bases, torch.int64),
                                              int(capacity_rows), _stream_handle(stream))
         if rc != MOE_OK and check:
@@ -268,7 +287,7 @@ class MoeComm:
 
     def moe_combine_peers(self, window_bases: torch.Tensor, capacity_rows: int, topk_w: torch.Tensor, y: torch.Tensor,
                           stream=None, check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_combine_peers(self._h, _dev_ptr(window_bases, torch.int64), int(capacity_rows),
                                             _dev_ptr(topk_w, torch.float32), _dev_ptr(y, torch.bfloat16),
                                             _stream_handle(stream))
@@ -298,7 +317,7 @@ class MoeComm:
 
     def moe_dispatch(self, x: torch.Tensor, windows: torch.Tensor, capacity_rows: int, stream=None,
                      check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_dispatch(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(windows, torch.bfloat16),
                                        int(capacity_rows), _stream_handle(stream))
         if rc != MOE_OK and check:
@@ -307,7 +326,7 @@ class MoeComm:
 
     def moe_dispatch_quant(self, x: torch.Tensor, windows_q: torch.Tensor, scales: torch.Tensor, capacity_rows: int,
                            stream=None, check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_dispatch_quant(self._h, _dev_ptr(x, torch.bfloat16), _dev_ptr(windows_q, torch.uint8),
                                              _dev_ptr(scales, torch.float32), int(capacity_rows),
                                              _stream_handle(stream))
@@ -317,7 +336,7 @@ class MoeComm:
 
     def moe_expert_ranges(self, capacity_rows: int, row_start: torch.Tensor, row_count: torch.Tensor, stream=None,
                           check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_expert_ranges(self._h, int(capacity_rows), _dev_ptr(row_start, torch.int64),
                                             _dev_ptr(row_count, torch.int32), _stream_handle(stream))
         if rc != MOE_OK and check:
@@ -326,7 +345,7 @@ class MoeComm:
 
     def moe_combine(self, windows: torch.Tensor, capacity_rows: int, topk_w: torch.Tensor, y: torch.Tensor,
                     stream=None, check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_combine(self._h, _dev_ptr(windows, torch.bfloat16), int(capacity_rows),
                                       _dev_ptr(topk_w, torch.float32), _dev_ptr(y, torch.bfloat16),
                                       _stream_handle(stream))
@@ -335,7 +354,7 @@ class MoeComm:
         return rc
 
     def moe_slots(self, capacity_rows: int, slots: torch.Tensor, stream=None, check: bool = True) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_slots(self._h, int(capacity_rows), _dev_ptr(slots, torch.int32),
                                     _stream_handle(stream))
         if rc != MOE_OK and check:
@@ -346,7 +365,7 @@ class MoeComm:
                          x_dev, topk_idx_dev, topk_w_dev, windows_dev, capacity_rows: int, y_dev, y_host,
                          stream=None, check: bool = True) -> int:
         rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
-        with torch.cuda.device(self.device):
+        with self._on_device():
             rc = self.lib.moe_forward_host(
                 self._h, schedule, T, _host_ptr(rts), _host_ptr(x_host), _host_ptr(topk_idx_host),
                 _host_ptr(topk_w_host), _dev_ptr(x_dev), _dev_ptr(topk_idx_dev), _dev_ptr(topk_w_dev),
@@ -365,7 +384,7 @@ class MoeComm:
         return rc
 
     def moe_status(self, stream=None) -> int:
-        with torch.cuda.device(self.device):
+        with self._on_device():
             return int(self.lib.moe_status(self._h, _stream_handle(stream)))
 
     def moe_launch_count(self) -> int:
