@@ -198,7 +198,9 @@ int row_grid(moe_ctx* ctx, Kernel kernel, int64_t tokens) {
 // Loads in flight per lane before the dependent stores / fma chain.  Few fat warps (one 256-thread
 // CTA per SM with about 32 16-byte loads per lane) measured faster than many thin ones: every warp
 // then streams long contiguous runs of each row, which HBM serves with far fewer page switches.
-constexpr int combine_unroll(int K) { return K >= 8 ? 4 : K >= 6 ? 5 : K >= 4 ? 8 : 16; }
+constexpr int combine_unroll(int K) {
+  return K >= 16 ? 2 : K >= 9 ? 3 : K >= 7 ? 4 : K >= 6 ? 5 : K == 5 ? 6 : K == 4 ? 8 : K == 3 ? 10 : 16;
+}
 constexpr int DISPATCH_UNROLL = 14;
 
 template <int KT>
@@ -632,8 +634,14 @@ moe_status_t combine_impl(moe_ctx* ctx, const void* windows, const void* const* 
     case 1: launch_combine<1>(ctx, a, win, topk_w, ys, st); break;
     case 2: launch_combine<2>(ctx, a, win, topk_w, ys, st); break;
     case 4: launch_combine<4>(ctx, a, win, topk_w, ys, st); break;
+    case 3: launch_combine<3>(ctx, a, win, topk_w, ys, st); break;
+    case 5: launch_combine<5>(ctx, a, win, topk_w, ys, st); break;
     case 6: launch_combine<6>(ctx, a, win, topk_w, ys, st); break;
+    case 7: launch_combine<7>(ctx, a, win, topk_w, ys, st); break;
     case 8: launch_combine<8>(ctx, a, win, topk_w, ys, st); break;
+    case 10: launch_combine<10>(ctx, a, win, topk_w, ys, st); break;
+    case 12: launch_combine<12>(ctx, a, win, topk_w, ys, st); break;
+    case 16: launch_combine<16>(ctx, a, win, topk_w, ys, st); break;
     default: launch_combine<0>(ctx, a, win, topk_w, ys, st); break;
   }
   return launch_ok(ctx);

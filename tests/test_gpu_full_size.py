@@ -79,6 +79,15 @@ def test_full_size_prefill_sampled(n):
 
     # -- combine: identity experts and weights summing to 1 => Y == X at every element
     assert torch.equal(Y.view(torch.int16), X.view(torch.int16))
+    # -- planning folded into the dispatch call: the same bytes everywhere (padding rows included),
+    #    and the sampled rows once more against the host copy of X
+    windows2 = torch.empty_like(windows)
+    windows2.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+    comm.moe_plan_dispatch(wl.schedule, idx, X, windows2, C)
+    assert comm.moe_status() == 0
+    assert torch.equal(windows2.view(torch.int16), windows.view(torch.int16))
+    assert np.array_equal(as_u16(windows2.index_select(0, rows)), synth.bf16_to_u16(inp.X)[bt])
+    del windows2
     # -- and sampled tokens against the oracle run on their own rows (inputs come from the host copy of X)
     S = np.sort(rng.choice(wl.T, 256, replace=False))
     Xs = synth.bf16_to_u16(inp.X)[S]

@@ -83,6 +83,11 @@ EDGE = [
     ("H_not_mult_of_warp_row", 77, 1000, 16, 2, 6, "uniform", (30, 47)),
     ("K3_generic", 129, 264, 12, 3, 3, "replace", (40, 0, 89)),
     ("K5_generic_dups", 250, 520, 10, 5, 5, "replace", (1, 100, 49, 0, 100)),
+    ("K7", 300, 1032, 16, 4, 7, "uniform", None),
+    ("K10", 200, 2048, 64, 4, 10, "uniform", (50, 70, 0, 80)),
+    ("K12_dups", 150, 520, 24, 3, 12, "replace", None),
+    ("K16", 120, 4096, 32, 2, 16, "uniform", None),
+    ("K9_generic", 90, 264, 16, 2, 9, "uniform", None),
     ("K32_max", 40, 64, 64, 2, 32, "uniform", None),
     ("duplicates_in_token", 333, 72, 4, 2, 4, "replace", (300, 33)),
     ("empty_rank_ragged", 1000, 256, 32, 4, 8, "uniform", (0, 517, 0, 483)),
