@@ -419,9 +419,13 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
     cp_src = torch.zeros(half, dtype=torch.uint8, device=dev)
     cp_dst = torch.empty_like(cp_src)
     copy = lambda: cp_dst.copy_(cp_src)
+    wq = torch.empty((dwl.R * dl.C, dwl.H), dtype=torch.uint8, device=dev)
+    wscale = torch.empty((dwl.R * dl.C,), dtype=torch.float32, device=dev)
+    quant = lambda: c.moe_dispatch_quant(dl.X, wq, wscale, dl.C)
     for name, pre in (("cold", [flush]), ("warm", [])):
         base = time_repeated(pre, n) if pre else 0.0
         t_copy = time_repeated(pre + [copy], n)
+        t_quant = time_repeated(pre + [quant], n)
         t1 = time_repeated(pre + [plan], n)
         t2 = time_repeated(pre + [plan, disp], n)
         t3 = time_repeated(pre + [plan, disp, comb], n)
@@ -441,7 +445,9 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
                      "dispatch_GBps": bytes_dispatch(dwl) / (t2 - t1) / 1e3,
                      "combine_GBps": bytes_combine(dwl) / (t3 - t2) / 1e3,
                      "gate_us": t_gate - base, "gate_plan_us": t_gate_plan - base,
-                     "plain_copy_of_the_same_bytes_us": t_copy - base}
+                     "plain_copy_of_the_same_bytes_us": t_copy - base,
+                     "dispatch_quant_us": t_quant - base,
+                     "dispatch_quant_GBps": bytes_dispatch_quant(dwl) / (t_quant - base) / 1e3}
     plan()   # leave the context planned on dl.idx again
     assert c.moe_status() == 0
     return out

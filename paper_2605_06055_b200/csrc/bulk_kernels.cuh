@@ -165,7 +165,11 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
     if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity, a.wait_limit_ms) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) {
-      if (lane == 0) raise_status(a.status, MOE_ERR_TIMEOUT);
+      if (lane == 0) {
+        raise_status(a.status, MOE_ERR_TIMEOUT);
+        // the load of the next item is in flight: let it land (bounded) before the CTA's shared memory is handed back
+        if (q1 < a.n_items) mbar_wait(bar0 + 8 * ((it + 1) % BULK_STAGES), ((it + 1) / BULK_STAGES) & 1u, a.wait_limit_ms);
+      }
       alive = false;
       break;
     }

@@ -322,7 +322,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   auto opt_in = [&](auto kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess;
   };
-  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel) && opt_in(plan_rank_kernel<32>) &&
+  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2>) && opt_in(dispatch_quant_kernel<3>) && opt_in(plan_rank_kernel<32>) &&
        opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
        opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
@@ -593,17 +593,25 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, fl
   a.topk_idx = ctx->topk_idx;
   // One work item per token: the whole row is needed for its scale.
   const int upr = (a.H16 + 31) / 32;
-  const int stage = ((H * 2 + 127) / 128 + (H + 127) / 128) * 128;
-  int warps = BULK_SMEM_BUDGET / (QUANT_STAGES * (stage + 8));
-  if (warps > BULK_MAX_WARPS) warps = BULK_MAX_WARPS;
-  if (warps < 1) return MOE_ERR_INVALID_ARG;
+  const int stage = (H * 2 + 127) / 128 * 128;
   const int grid = ctx->num_sms;
+  auto warps_for = [&](int stages) {
+    int w = QUANT_SMEM_BUDGET / (stages * (stage + 8));
+    return w > QUANT_MAX_WARPS ? QUANT_MAX_WARPS : w;
+  };
+  // Three stages once every warp of the two-stage configuration would see eight rows or more.
+  const int stages = (warps_for(3) >= 1 && (int64_t)ctx->T >= (int64_t)8 * grid * warps_for(2)) ? 3 : 2;
+  int warps = warps_for(stages);
+  if (warps < 1) return MOE_ERR_INVALID_ARG;
+  const int64_t rows_per_sm = ((int64_t)ctx->T + grid - 1) / grid;
+  if (warps > rows_per_sm) warps = rows_per_sm < 1 ? 1 : (int)rows_per_sm;   // no warps without a row
   const int32_t keep = ctx->granule_override;
   ctx->granule_override = upr;
   set_work(ctx, a, (int64_t)grid * warps, upr);
   ctx->granule_override = keep;
-  const int smem = warps * QUANT_STAGES * (stage + 8);
-  dispatch_quant_kernel<<<grid, warps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+  const int smem = warps * stages * (stage + 8);
+  auto kernel = stages == 3 ? dispatch_quant_kernel<3> : dispatch_quant_kernel<2>;
+  kernel<<<grid, warps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
   return launch_ok(ctx);
 }

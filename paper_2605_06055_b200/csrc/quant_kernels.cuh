@@ -9,11 +9,17 @@
 // Each token is quantised once; its K branches receive the same code row and scale.
 //
 // Structure: the bulk-copy ring of dispatch_bulk_kernel with a compute step in
-// the middle.  A stage holds one whole row (needed for amax) plus its code row.
-// Lane 0 loads the row with cp.async.bulk; the warp reduces amax and converts
-// from shared memory into the stage's code buffer; lane 0 stores the code row K
-// times with cp.async.bulk while lanes j < K store the scale.  X is read from
-// HBM once and only H + 4 bytes per branch are written.
+// the middle.  A stage holds one whole row (needed for amax).  Lane 0 loads the
+// row with cp.async.bulk; the warp reduces amax from shared memory and converts
+// the row IN PLACE (codes are half as wide as the values, so the code of chunk c
+// lands on bytes that chunks <= c/2 occupied and have already been read); lane 0
+// stores the code row K times with cp.async.bulk while lanes j < K store the
+// scale.  X is read from HBM once and only H + 4 bytes per branch are written.
+//
+// What bounds the kernel at decode sizes is the latency of one warp walking its
+// row, so the number of rows in flight per SM matters: a stage without a
+// separate code buffer lets seven warps (instead of four or five) share an SM
+// at 14 KB rows.
 #pragma once
 
 #include <cuda_fp8.h>
@@ -22,8 +28,12 @@
 
 namespace moe {
 
-constexpr int QUANT_STAGES = 2;
+// Stages per warp: 2 for small batches (more warps, i.e. more rows in flight per SM, is what counts
+// when every warp sees only a few rows), 3 for large ones (two loads in flight per warp).  Measured:
+// decode shape (T=2048, 14 KB rows) 30.8 vs 32.7 us; T=65536 with 8 KB rows 235 vs 182 us.
 constexpr int QUANT_MAX_ROW_BYTES = 32 * 1024;
+constexpr int QUANT_MAX_WARPS = 16;
+constexpr int QUANT_SMEM_BUDGET = 220 * 1024;   // shared memory the warps' rings may fill
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -43,9 +53,10 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t two_bf16, float inv) {
   return (uint32_t)__nv_cvt_float2_to_fp8x2(f, __NV_SATFINITE, __NV_E4M3);
 }
 
-// Dynamic shared memory: [warps][QUANT_STAGES] stages of (in_stride + out_stride) bytes, then
-// [warps][QUANT_STAGES] mbarriers.  in_stride / out_stride: row bytes / code-row bytes rounded up to 128.
-__global__ void __launch_bounds__(BULK_MAX_WARPS * 32)
+// Dynamic shared memory: [warps][QUANT_STAGES] stages of in_stride bytes (row bytes rounded up to 128),
+// then [warps][QUANT_STAGES] mbarriers.
+template <int QUANT_STAGES>
+__global__ void __launch_bounds__(QUANT_MAX_WARPS * 32, 1)
 dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
                       float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -56,8 +67,7 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t row_bytes = (uint32_t)a.H16 * 16u;          // bf16 row
   const uint32_t code_bytes = (uint32_t)a.H16 * 8u;          // e4m3 row
-  const uint32_t in_stride = (row_bytes + 127u) & ~127u, out_stride = (code_bytes + 127u) & ~127u;
-  const uint32_t stage_stride = in_stride + out_stride;
+  const uint32_t stage_stride = (row_bytes + 127u) & ~127u;
   const uint32_t buf0 = smem_addr(smem) + warp * QUANT_STAGES * stage_stride;
   const uint32_t bar0 = smem_addr(smem) + n_warps * QUANT_STAGES * stage_stride + warp * QUANT_STAGES * 8;
 
@@ -77,27 +87,31 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   uint64_t evict_first;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
 
-  // One work item = one token row (items_per_row == 1).  q0 is consumed now, q1 is loading.
+  // One work item = one token row (items_per_row == 1).  q0 is consumed in this iteration; the load of
+  // q1 is issued at its start, into the stage whose code row was stored QUANT_STAGES - 1 iterations ago.
   ItemFeed feed = begin_feed();
   int32_t q0 = fetch_item(a, feed);
   int32_t q1 = fetch_item(a, feed);
-  if (lane == 0) {
-    if (q0 < a.n_items) issue_load(q0, 0);
-    if (q1 < a.n_items) issue_load(q1, 1 % QUANT_STAGES);
-  }
+  if (lane == 0 && q0 < a.n_items) issue_load(q0, 0);
   uint32_t it = 0;
+  bool timed_out = false;
   while (q0 < a.n_items) {
     const int32_t q2 = fetch_item(a, feed);
     const int s = it % QUANT_STAGES;
     const uint32_t parity = (it / QUANT_STAGES) & 1u;
-    const int64_t slot = resolve_slot(a, map, q0, lane, true);   // overlaps the load in flight
-    const uint32_t in = buf0 + s * stage_stride, out = in + in_stride;
+    if (lane == 0 && q1 < a.n_items) {
+      // the next stage still holds the code row of iteration it + 1 - QUANT_STAGES until its stores have read it
+      bulk_wait_read<QUANT_STAGES - 2>();
+      issue_load(q1, (it + 1) % QUANT_STAGES);
+    }
+    const int64_t slot = resolve_slot(a, map, q0, lane, true);   // overlaps the loads in flight
+    const uint32_t in = buf0 + s * stage_stride;
 
     int ok = 1;
     if (lane == 0) ok = mbar_wait(bar0 + 8 * s, parity, a.wait_limit_ms) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) {
-      if (lane == 0) raise_status(a.status, MOE_ERR_TIMEOUT);
+      timed_out = true;
       break;
     }
 
@@ -121,38 +135,39 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
       inv = __fdiv_rn(448.0f, amax);
     }
 
-    // The code buffer of this stage was last read by the stores of item it - QUANT_STAGES: allow only
-    // the QUANT_STAGES - 1 younger store groups to be still reading before it is overwritten.
-    if (lane == 0) bulk_wait_read<QUANT_STAGES - 1>();
-    __syncwarp();
-    for (int c = lane; c < a.H16; c += 32) {
-      const uint4 v = lds128(in + c * 16);
-      const uint32_t lo = quant_pair(v.x, inv) | (quant_pair(v.y, inv) << 16);
-      const uint32_t hi = quant_pair(v.z, inv) | (quant_pair(v.w, inv) << 16);
-      sts64(out + c * 8, lo, hi);
+    // In place: the pass over chunks c = 32 i + lane reads bytes [512 i, 512 i + 512) and writes bytes
+    // [256 i, 256 i + 256), which only earlier passes (and, for i = 0, this pass) have read; the warp
+    // barrier puts every lane's read of a pass in front of every lane's write of it.
+    for (int c = lane; c - lane < a.H16; c += 32) {   // warp-uniform trip count
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (c < a.H16) v = lds128(in + c * 16);
+      __syncwarp();
+      if (c < a.H16) {
+        const uint32_t lo = quant_pair(v.x, inv) | (quant_pair(v.y, inv) << 16);
+        const uint32_t hi = quant_pair(v.z, inv) | (quant_pair(v.w, inv) << 16);
+        sts64(in + c * 8, lo, hi);
+      }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // code row: generic writes -> bulk-copy reads
     __syncwarp();
 
     for (int j = 0; j < a.K; ++j) {
       const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-      if (lane == 0 && row >= 0) bulk_store(windows_q + (size_t)row * code_bytes, out, code_bytes, evict_first);
+      if (lane == 0 && row >= 0) bulk_store(windows_q + (size_t)row * code_bytes, in, code_bytes, evict_first);
     }
     if (lane < a.K && slot >= 0) scales[slot] = scale;
-    if (lane == 0) {
-      bulk_commit();
-      // The row buffer of this stage is free again (every lane has read it): refill it.
-      if (QUANT_STAGES == 2) {
-        if (q2 < a.n_items) issue_load(q2, s);
-      } else {
-        if (q2 < a.n_items) issue_load(q2, (it + 2) % QUANT_STAGES);
-      }
-    }
+    if (lane == 0) bulk_commit();   // one group per iteration
     q0 = q1;
     q1 = q2;
     ++it;
   }
-  if (lane == 0) bulk_wait_all();
+  if (lane == 0) {
+    if (timed_out) {   // report, and let the other load in flight land (bounded) before the CTA leaves
+      raise_status(a.status, MOE_ERR_TIMEOUT);
+      if (q1 < a.n_items) mbar_wait(bar0 + 8 * ((it + 1) % QUANT_STAGES), ((it + 1) / QUANT_STAGES) & 1u, a.wait_limit_ms);
+    }
+    bulk_wait_all();
+  }
   end_work(a);
 }
 

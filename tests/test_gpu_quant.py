@@ -23,6 +23,10 @@ CASES = [
     ("ragged_units", 123, 1008, 16, 2, 6, DECODE, "uniform", (23, 100)),
     ("K5_dups_empty_rank", 250, 528, 10, 5, 5, PREFILL, "replace", (1, 100, 49, 0, 100)),
     ("max_row", 64, 16384, 8, 2, 2, DECODE, "uniform", None),
+    ("tile_planned_decode", 6000, 64, 16, 2, 2, DECODE, "uniform", (5000, 1000)),
+    ("one_row", 2, 512, 4, 2, 2, DECODE, "uniform", None),
+    ("K32", 40, 64, 64, 2, 32, DECODE, "uniform", None),
+    ("many_rows_per_sm", 20000, 256, 32, 4, 4, PREFILL, "uniform", None),
 ]
 
 
@@ -49,7 +53,9 @@ def test_quantised_dispatch_bit_exact(case):
     comm.moe_plan(sch, inp.topk_idx.to(dev), T, rts)
     wq = torch.full((R * C, H), 0xAB, dtype=torch.uint8, device=dev)
     sc = torch.full((R * C,), -1.0, dtype=torch.float32, device=dev)
-    comm.moe_dispatch_quant(X.to(dev), wq, sc, C)
+    Xd = X.to(dev)
+    for _ in range(2):                                # twice: the second launch starts from the counters the first left
+        comm.moe_dispatch_quant(Xd, wq, sc, C)
     assert comm.moe_status() == 0
     assert np.array_equal(wq.cpu().numpy(), want_q)
     assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
