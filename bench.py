@@ -425,6 +425,7 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
     for name, pre in (("cold", [flush]), ("warm", [])):
         base = time_repeated(pre, n) if pre else 0.0
         t_copy = time_repeated(pre + [copy], n)
+        plan()   # the gate leg below leaves the context planned on other indexes
         t_quant = time_repeated(pre + [quant], n)
         t1 = time_repeated(pre + [plan], n)
         t2 = time_repeated(pre + [plan, disp], n)
@@ -450,6 +451,32 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
                      "dispatch_quant_GBps": bytes_dispatch_quant(dwl) / (t_quant - base) / 1e3}
     plan()   # leave the context planned on dl.idx again
     assert c.moe_status() == 0
+    del dl, wq, wscale, cp_src, cp_dst, logits
+    torch.cuda.empty_cache()
+
+    # The grid of the paper's decode table (Table 2): per-rank batch sizes 16..144, H = 4096 and 7168, plain and
+    # row-wise quantised dispatch, combine.  The paper does not state its rank count, expert count or top-k; this
+    # sweep takes the decode configuration's (16 ranks, 256 experts, top-8).  L2 flushed before every call.
+    sweep = []
+    for H in (4096, 7168):
+        for per_rank in (16, 32, 64, 80, 128, 144):
+            swl = synth.Workload(f"decode_b{per_rank}_H{H}", per_rank * dwl.R, H, dwl.E, dwl.R, dwl.K, synth.DECODE,
+                                 "uniform", "identity", 1200 + per_rank)
+            sl = Layer(swl, dev)
+            sq = torch.empty((swl.R * sl.C, swl.H), dtype=torch.uint8, device=dev)
+            ss = torch.empty((swl.R * sl.C,), dtype=torch.float32, device=dev)
+            sc = sl.comm
+            s_plan = lambda: sc.moe_plan(swl.schedule, sl.idx)
+            base = time_repeated([flush], n)
+            t_d = time_repeated([flush, lambda: sc.moe_dispatch(sl.X, sl.windows, sl.C)], n) - base
+            t_q = time_repeated([flush, lambda: sc.moe_dispatch_quant(sl.X, sq, ss, sl.C)], n) - base
+            t_c = time_repeated([flush, lambda: sc.moe_combine(sl.windows, sl.C, sl.w, sl.Y)], n) - base
+            t_p = time_repeated([flush, s_plan], n) - base
+            assert sc.moe_status() == 0
+            sweep.append({"tokens_per_rank": per_rank, "H": H, "plan_us": t_p, "dispatch_us": t_d,
+                          "dispatch_quant_us": t_q, "combine_us": t_c})
+            del sl, sq, ss
+    out["batch_sweep"] = {"ranks": dwl.R, "experts": dwl.E, "top_k": dwl.K, "rows": sweep}
     return out
 
 

@@ -134,6 +134,10 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
+  a.n_head = 0;
+  a.head_rows = 0;
+  a.tail_granule = 1;
+  a.tail_items_per_row = 1;
   a.win_base = nullptr;
   a.prefetch_meta = 0;
   a.static_first = 0;
@@ -148,7 +152,7 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
 // Chooses the work-item size and hands the launch its counter.  An item is a whole row (at most
 // max_granule units) whenever that still gives every warp an item -- whole rows measured best
 // even at decode sizes -- and an even fraction of a row for tiny batches.
-void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
+void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule, bool may_split_tail = true) {
   const int upr = (a.H16 + 31) / 32;
   int64_t g = upr < max_granule ? upr : max_granule;
   int64_t pieces = (upr + g - 1) / g;
@@ -166,6 +170,29 @@ void set_work(moe_ctx* ctx, RowArgs& a, int64_t nwarps, int max_granule) {
   a.granule = (int32_t)g;
   a.items_per_row = (int32_t)((upr + g - 1) / g);
   a.n_items = (int32_t)(tokens * a.items_per_row);
+  a.n_head = a.n_items;
+  a.head_rows = (int32_t)tokens;
+  a.tail_granule = a.granule;
+  a.tail_items_per_row = a.items_per_row;
+  // Whole-row items: after the last full round (one row per warp) fewer rows than warps are left.  When
+  // they would occupy at most a quarter of the warps, they are cut so that (nearly) every warp gets a
+  // piece, but no finer than MIN_TAIL_UNITS.  Measured at H=7168, K=8, T=1280 (96 rows left over):
+  // dispatch 38.5 -> 32.7 us, combine 45.0 -> 36.1 us.  Leftovers that fill more of the warps are not cut:
+  // at T=2048 (272 rows left for 592 dispatch warps) halving them measured 1.3 us slower.
+  constexpr int MIN_TAIL_UNITS = 4;
+  const int64_t left = tokens % nwarps;
+  if (may_split_tail && ctx->granule_override == 0 && a.items_per_row == 1 && tokens > nwarps && left > 0 &&
+      4 * left <= nwarps && upr >= 2 * MIN_TAIL_UNITS) {
+    int64_t pieces = nwarps / left;
+    if (pieces > upr / MIN_TAIL_UNITS) pieces = upr / MIN_TAIL_UNITS;
+    const int tg = (int)((upr + pieces - 1) / pieces);
+    const int tipr = (upr + tg - 1) / tg;
+    a.head_rows = (int32_t)(tokens - left);
+    a.n_head = a.head_rows;
+    a.tail_granule = tg;
+    a.tail_items_per_row = tipr;
+    a.n_items = (int32_t)(a.head_rows + left * tipr);
+  }
   a.static_first = a.n_items <= 4 * nwarps ? 2 : 0;
   a.work = &ctx->ctl->work;
   a.work_done = &ctx->ctl->work_done;
@@ -607,7 +634,7 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, fl
   if (warps > rows_per_sm) warps = rows_per_sm < 1 ? 1 : (int)rows_per_sm;   // no warps without a row
   const int32_t keep = ctx->granule_override;
   ctx->granule_override = upr;
-  set_work(ctx, a, (int64_t)grid * warps, upr);
+  set_work(ctx, a, (int64_t)grid * warps, upr, false);
   ctx->granule_override = keep;
   const int smem = warps * stages * (stage + 8);
   auto kernel = stages == 3 ? dispatch_quant_kernel<3> : dispatch_quant_kernel<2>;
@@ -980,6 +1007,10 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.granule = 1;
   a.items_per_row = 0;
   a.n_items = 0;
+  a.n_head = 0;
+  a.head_rows = 0;
+  a.tail_granule = 1;
+  a.tail_items_per_row = 1;
   a.win_base = nullptr;
   a.prefetch_meta = 0;
   a.static_first = 0;

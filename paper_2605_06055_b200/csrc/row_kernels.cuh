@@ -30,7 +30,12 @@ struct RowArgs {
   int32_t* work_done;        // finished-warp counter (same)
   int32_t granule;           // units (512-byte slabs) per work item
   int32_t items_per_row;     // ceil(units per row / granule)
-  int32_t n_items;           // t_count * items_per_row
+  int32_t n_items;           // head items + tail items
+  // The rows left over after the last full round of whole-row items (fewer rows than warps) are cut
+  // finer, tail_granule units per item, so that the launch does not end with a few warps each moving a
+  // whole row while the others idle.  Items [0, n_head) cover the first head_rows rows; without a tail
+  // n_head == n_items and head_rows == t_count.
+  int32_t n_head, head_rows, tail_granule, tail_items_per_row;
   int32_t t_begin, t_count;  // token range this launch covers (the whole batch unless a *_range call)
   // Multi-rank use: window segment d starts at win_base[d] (device array of R device pointers, e.g. peer
   // mappings of every rank's window); nullptr = one allocation of R consecutive segments of C rows.
@@ -206,10 +211,19 @@ __device__ __forceinline__ int32_t fetch_item(const RowArgs& a, ItemFeed& f) {
 
 __device__ __forceinline__ WorkItem decode_item(const RowArgs& a, int32_t item) {
   WorkItem w;
-  const int32_t q = item / a.items_per_row;
-  w.t = a.t_begin + q;
-  w.i0 = (item - q * a.items_per_row) * a.granule;
-  w.i1 = min(w.i0 + a.granule, (a.H16 + 31) >> 5);
+  const int32_t upr = (a.H16 + 31) >> 5;
+  if (item < a.n_head) {
+    const int32_t q = item / a.items_per_row;
+    w.t = a.t_begin + q;
+    w.i0 = (item - q * a.items_per_row) * a.granule;
+    w.i1 = min(w.i0 + a.granule, upr);
+  } else {
+    const int32_t rem = item - a.n_head;
+    const int32_t q = rem / a.tail_items_per_row;
+    w.t = a.t_begin + a.head_rows + q;
+    w.i0 = (rem - q * a.tail_items_per_row) * a.tail_granule;
+    w.i1 = min(w.i0 + a.tail_granule, upr);
+  }
   return w;
 }
 

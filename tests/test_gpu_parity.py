@@ -101,6 +101,8 @@ EDGE = [
     ("many_tiles", 200000, 32, 64, 8, 8, "uniform", None),                              # 1.6 M branches, 98 tiles per rank
     ("long_rows_two_items_per_row", 512, 16384, 16, 4, 4, "uniform", None),             # 32 KB rows
     ("row_of_three_units_and_a_tail", 700, 808, 8, 2, 2, "uniform", None),              # 1616-byte rows: 3 units + 80 B
+    ("leftover_rows_cut_finer", 1280, 7168, 256, 16, 8, "uniform", None),               # 1280 = 1184 warps + 96 rows
+    ("leftover_rows_cut_finer_ragged", 2500, 4104, 8, 4, 2, "uniform", (700, 600, 1100, 100)),   # 17 units per row
 ]
 
 
