@@ -1,0 +1,81 @@
+"""Seeded random shapes through the whole path on the GPU against the oracle: every integer, every
+window byte (canaries included) and the combined rows (<= 1 bf16 ulp), for random token counts,
+hidden sizes, expert / rank / top-k counts, ragged rank maps (empty ranks included), both
+schedules, both dispatch kernels, duplicate experts within a token, several work-item sizes and
+expert alignments."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06055_b200 import binding, synth
+from paper_2605_06055_b200.synth import DECODE, PREFILL, Workload
+
+import harness
+
+pytestmark = pytest.mark.gpu
+
+
+def random_workload(rng, i):
+    R = int(rng.choice([1, 2, 3, 4, 8, 16]))
+    E = R * int(rng.choice([1, 2, 3, 8, 32]))
+    K = int(rng.integers(1, min(E, 12) + 1))
+    replace = bool(rng.integers(0, 2))
+    if replace:
+        K = int(rng.integers(1, 13))
+    H = 8 * int(rng.choice([1, 2, 31, 32, 33, 64, 100, 128, 257, 512, 896]))
+    T = int(rng.choice([1, 2, 7, 33, 100, 257, 600, 1500, 2600]))
+    cuts = np.sort(rng.integers(0, T + 1, R - 1))
+    per = tuple(int(x) for x in np.diff(np.concatenate([[0], cuts, [T]])))
+    sch = PREFILL if rng.integers(0, 2) else DECODE
+    return Workload(f"fuzz{i}", T, H, E, R, K, sch, "replace" if replace else "uniform", "scale", 31000 + i,
+                    rank_tokens=per)
+
+
+@pytest.mark.parametrize("i", range(48))
+def test_random_shape(i):
+    rng = np.random.default_rng(77000 + i)
+    wl = random_workload(rng, i)
+    align = int(rng.choice([1, 1, 4, 16, 128]))
+    granule = int(rng.choice([0, 0, 0, 1, 3, 7]))
+    path = binding.MOE_DISPATCH_BULK if rng.integers(0, 2) else binding.MOE_DISPATCH_REGISTERS
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R, inp.rank_tok_start, align=align)
+    assert p.status == oracle.OK
+    C = int(p.n_recv.max()) + int(rng.integers(0, 3))
+    o = harness.oracle_run(inp, C, align=align)
+    g = harness.gpu_run(inp, C, wl.schedule, dispatch_path=path, granule=granule, align=align)
+    harness.assert_parity(g, o, wl.schedule, align=align)
+
+
+@pytest.mark.parametrize("i", range(12))
+def test_random_shape_fused_call_and_quantised_dispatch(i):
+    rng = np.random.default_rng(88000 + i)
+    wl = random_workload(rng, 100 + i)
+    if wl.H % 16:
+        wl = Workload(wl.name, wl.T, wl.H + 8, wl.E, wl.R, wl.K, wl.schedule, wl.routing, "identity", wl.seed,
+                      rank_tokens=wl.rank_tokens)
+    dev = torch.device("cuda:0")
+    inp = synth.make_inputs(wl)
+    idx_np = inp.topk_idx.numpy()
+    p = oracle.plan(idx_np, wl.E, wl.R, inp.rank_tok_start)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(idx_np, wl.E, wl.R, p, C, inp.rank_tok_start)
+    want = np.full((wl.R * C, wl.H), harness.CANARY, np.uint16)
+    assert oracle.dispatch(synth.bf16_to_u16(inp.X), slots, want) == oracle.OK
+    want_q = np.full((wl.R * C, wl.H), 0xAB, np.uint8)
+    want_s = np.full((wl.R * C,), -1.0, np.float32)
+    assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), slots, want_q, want_s, 4) == oracle.OK
+
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx = inp.X.to(dev), inp.topk_idx.to(dev)
+    win = torch.from_numpy(np.full((wl.R * C, wl.H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    wq = torch.full((wl.R * C, wl.H), 0xAB, dtype=torch.uint8, device=dev)
+    sc = torch.full((wl.R * C,), -1.0, dtype=torch.float32, device=dev)
+    comm.moe_plan_dispatch(wl.schedule, idx, X, win, C, wl.T, inp.rank_tok_start)
+    comm.moe_dispatch_quant(X, wq, sc, C)
+    assert comm.moe_status() == 0
+    assert np.array_equal(win.cpu().view(torch.int16).numpy().view(np.uint16), want)
+    assert np.array_equal(wq.cpu().numpy(), want_q)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+    comm.close()
