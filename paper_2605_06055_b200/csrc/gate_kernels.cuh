@@ -111,30 +111,22 @@ __device__ __forceinline__ void warp_gate_token_regs(const float* __restrict__ l
   idx_lane = sel_idx;
 }
 
-// Picks the register form when the row fits (E <= 1024), else the shared-memory form.
-__device__ __forceinline__ void warp_gate_any(const float* __restrict__ logits_row, float* row, int E, int K, int lane,
-                                              int32_t& idx_lane, float& w_lane) {
-  if (E <= 32) warp_gate_token_regs<1>(logits_row, E, K, lane, idx_lane, w_lane);
-  else if (E <= 64) warp_gate_token_regs<2>(logits_row, E, K, lane, idx_lane, w_lane);
-  else if (E <= 128) warp_gate_token_regs<4>(logits_row, E, K, lane, idx_lane, w_lane);
-  else if (E <= 256) warp_gate_token_regs<8>(logits_row, E, K, lane, idx_lane, w_lane);
-  else if (E <= 512) warp_gate_token_regs<16>(logits_row, E, K, lane, idx_lane, w_lane);
-  else if (E <= 1024) warp_gate_token_regs<32>(logits_row, E, K, lane, idx_lane, w_lane);
-  else warp_gate_token(logits_row, row, E, K, lane, idx_lane, w_lane);
-}
-
-// Stand-alone gate: grid-stride over tokens, one warp per token.  Dynamic shared memory: warps * E floats
-// (used only when E > 1024).
+// Stand-alone gate: grid-stride over tokens, one warp per token.  VPT > 0: register form for rows of at
+// most 32 * VPT logits (one instantiation per row length class, so that short rows keep few registers
+// and many warps per SM: 80 registers for a kernel holding every form, 3 CTAs per SM, against 6-8 CTAs
+// per SM for the 256-logit form on its own).  VPT == 0: shared-memory form for longer rows; dynamic shared
+// memory: warps * E floats.
+template <int VPT>
 __global__ void __launch_bounds__(256)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
                  float* __restrict__ topk_w) {
   extern __shared__ float gate_rows[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpc = blockDim.x >> 5;
-  float* row = gate_rows + warp * E;
   for (int32_t t = blockIdx.x * wpc + warp; t < T; t += gridDim.x * wpc) {
     int32_t idx;
     float w;
-    warp_gate_any(logits + (size_t)t * E, row, E, K, lane, idx, w);
+    if constexpr (VPT > 0) warp_gate_token_regs<VPT>(logits + (size_t)t * E, E, K, lane, idx, w);
+    else warp_gate_token(logits + (size_t)t * E, gate_rows + warp * E, E, K, lane, idx, w);
     if (lane < K) {
       topk_idx[(size_t)t * K + lane] = idx;
       topk_w[(size_t)t * K + lane] = w;

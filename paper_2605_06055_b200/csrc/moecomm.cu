@@ -351,7 +351,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   };
   ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2>) && opt_in(dispatch_quant_kernel<3>) && opt_in(plan_rank_kernel<32>) &&
        opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
-       opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel);
+       opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
   const int rank_smem =
       rank_plan_smem_ints(shape->E, shape->R, shape->E <= RANK_PLAN_WIDE_MAX_E ? 32 : 8) * (int)sizeof(int32_t);
@@ -383,15 +383,39 @@ moe_status_t moe_destroy(moe_ctx_t* ctx) {
 
 namespace {
 
+template <int VPT>
+void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
+                      cudaStream_t st) {
+  int warps = 8, smem = 0;
+  if (VPT == 0) {   // rows cached in shared memory
+    while (warps > 1 && warps * E * (int)sizeof(float) > 96 * 1024) warps >>= 1;
+    smem = warps * E * (int)sizeof(float);
+  }
+  static int cached = 0;   // resident CTAs per SM of a register form (one device kind per process)
+  int per_sm = VPT > 0 ? cached : 0;   // the shared-memory form's occupancy depends on E: asked every time
+  if (per_sm == 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gate_topk_kernel<VPT>, warps * 32, smem) != cudaSuccess ||
+        per_sm < 1) {
+      cudaGetLastError();
+      per_sm = 1;
+    }
+    if (VPT > 0) cached = per_sm;
+  }
+  int64_t grid = ((int64_t)T + warps - 1) / warps;
+  if (grid > (int64_t)num_sms * per_sm) grid = (int64_t)num_sms * per_sm;   // one resident wave, grid-stride over tokens
+  if (grid < 1) grid = 1;
+  gate_topk_kernel<VPT><<<(int)grid, warps * 32, smem, st>>>(logits, T, E, K, idx, w);
+}
+
 void launch_gate(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
                  cudaStream_t st) {
-  int warps = 8;
-  while (warps > 1 && warps * E * (int)sizeof(float) > 96 * 1024) warps >>= 1;
-  const int smem = warps * E * (int)sizeof(float);
-  int64_t grid = ((int64_t)T + warps - 1) / warps;
-  if (grid > (int64_t)num_sms * 8) grid = (int64_t)num_sms * 8;
-  if (grid < 1) grid = 1;
-  gate_topk_kernel<<<(int)grid, warps * 32, smem, st>>>(logits, T, E, K, idx, w);
+  if (E <= 32) launch_gate_form<1>(logits, T, E, K, idx, w, num_sms, st);
+  else if (E <= 64) launch_gate_form<2>(logits, T, E, K, idx, w, num_sms, st);
+  else if (E <= 128) launch_gate_form<4>(logits, T, E, K, idx, w, num_sms, st);
+  else if (E <= 256) launch_gate_form<8>(logits, T, E, K, idx, w, num_sms, st);
+  else if (E <= 512) launch_gate_form<16>(logits, T, E, K, idx, w, num_sms, st);
+  else if (E <= 1024) launch_gate_form<32>(logits, T, E, K, idx, w, num_sms, st);
+  else launch_gate_form<0>(logits, T, E, K, idx, w, num_sms, st);
 }
 
 // Planning, optionally with the gate in front (logits != nullptr: topk_idx and topk_w are OUTPUTS).
@@ -516,7 +540,7 @@ moe_status_t moe_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K,
   if (E > 1024) {   // the shared-memory form of the gate: opt in like moe_create does
     int optin = 0;
     if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
-        cudaFuncSetAttribute(gate_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 2048) != cudaSuccess)
+        cudaFuncSetAttribute(gate_topk_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 2048) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
   if (T > 0) launch_gate(logits, T, E, K, topk_idx, topk_w, sms, static_cast<cudaStream_t>(stream));
