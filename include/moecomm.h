@@ -254,13 +254,20 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
  *                          earlier experts; n_recv[d] becomes the sum over the experts of rank d of
  *                          ceil(n_exp[e] / A) * A, which is what capacity_rows is checked against.
  *                          Padding rows are never written by dispatch nor read by combine.  Setting the
- *                          option invalidates the current plan. */
+ *                          option invalidates the current plan.
+ *   MOE_OPT_CLUSTER_PLAN   1 (default): the single-launch planner of small batches (at most 4096 branches
+ *                          per source rank) runs its R CTAs as one thread-block cluster when R is 2, 4, 8 or
+ *                          16 and the device can co-schedule them: the count rows are exchanged through
+ *                          distributed shared memory and every CTA builds its own window's offsets.
+ *                          0: the last CTA to finish builds all offsets from the matrix in global memory.
+ *                          Same result. */
 typedef enum {
   MOE_OPT_DISPATCH_PATH = 0,
   MOE_OPT_GRANULE = 1,
   MOE_OPT_TEST_STARVE_WAIT_MS = 2,
   MOE_OPT_OVERLAP = 3,
-  MOE_OPT_EXPERT_ALIGN = 4
+  MOE_OPT_EXPERT_ALIGN = 4,
+  MOE_OPT_CLUSTER_PLAN = 5
 } moe_option_t;
 enum { MOE_DISPATCH_AUTO = 0, MOE_DISPATCH_REGISTERS = 1, MOE_DISPATCH_BULK = 2 };
 moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);

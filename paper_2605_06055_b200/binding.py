@@ -29,7 +29,7 @@ EXPORTS = [
     "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
-MOE_OPT_EXPERT_ALIGN = 4
+MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
 
 

@@ -41,6 +41,8 @@ struct moe_ctx {
   int32_t granule_override; // MOE_OPT_GRANULE
   int32_t starve_wait_ms;   // MOE_OPT_TEST_STARVE_WAIT_MS
   int32_t overlap;          // MOE_OPT_OVERLAP
+  int32_t cluster_plan;     // MOE_OPT_CLUSTER_PLAN
+  bool plan_cluster_ok;     // the compact planner of this shape can be launched as one cluster of R CTAs
   int32_t expert_align;     // MOE_OPT_EXPERT_ALIGN: every expert's run starts on a multiple of this many rows
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
@@ -334,6 +336,8 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->granule_override = 0;
   ctx->starve_wait_ms = 0;
   ctx->overlap = 1;
+  ctx->cluster_plan = 1;
+  ctx->plan_cluster_ok = false;
   ctx->expert_align = 1;
   ctx->out_stream = nullptr;
   ctx->in_stream = nullptr;
@@ -361,6 +365,32 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
     cudaGetLastError();
     delete ctx;
     return MOE_ERR_CUDA;
+  }
+  // Can the compact planner run as ONE cluster of R CTAs?  Sizes up to 8 are portable, 16 needs the opt-in.
+  if (shape->R == 2 || shape->R == 4 || shape->R == 8 || shape->R == 16) {
+    const bool wide = shape->E <= RANK_PLAN_WIDE_MAX_E;
+    const int smem = rank_smem + cluster_notify_smem_ints(shape->E, shape->R) * (int)sizeof(int32_t);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)shape->R);
+    cfg.blockDim = dim3((unsigned)((wide ? 32 : 8) * 32));
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)shape->R;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    bool fits = smem <= big;
+    if (fits && shape->R > 8)
+      fits = cudaFuncSetAttribute(plan_rank_kernel<32>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+             cudaFuncSetAttribute(plan_rank_kernel<8>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    if (fits)
+      fits = (wide ? cudaOccupancyMaxActiveClusters(&clusters, plan_rank_kernel<32>, &cfg)
+                   : cudaOccupancyMaxActiveClusters(&clusters, plan_rank_kernel<8>, &cfg)) == cudaSuccess && clusters >= 1;
+    cudaGetLastError();
+    ctx->plan_cluster_ok = fits;
   }
   *out = ctx;
   return MOE_OK;
@@ -478,14 +508,30 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
     ++n;
   }
   if (ctx->compact_plan) {
+    // One CTA per source rank.  When the R CTAs can run as one thread-block cluster, the Notify step reads
+    // the count rows from the CTAs' shared memory and every CTA builds its own window's offsets.
+    const bool as_cluster = ctx->cluster_plan && ctx->plan_cluster_ok;
+    const int threads = (wide ? 32 : 8) * 32;
+    const int smem = rank_smem + (as_cluster ? cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t) : 0);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)sh.R);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)sh.R;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = as_cluster ? 1 : 0;
+    const int32_t flag = as_cluster ? 1 : 0;
     if (wide)
-      plan_rank_kernel<32><<<sh.R, 32 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp,
-          ctx->n_recv, ctx->ctl);
+      cudaLaunchKernelEx(&cfg, plan_rank_kernel<32>, topk_idx, map, sh.K, sh.E, (int32_t)full, ctx->expert_align, ctx->s,
+                         ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl, flag);
     else
-      plan_rank_kernel<8><<<sh.R, 8 * 32, rank_smem, st>>>(
-          topk_idx, map, sh.K, sh.E, full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp,
-          ctx->n_recv, ctx->ctl);
+      cudaLaunchKernelEx(&cfg, plan_rank_kernel<8>, topk_idx, map, sh.K, sh.E, (int32_t)full, ctx->expert_align, ctx->s,
+                         ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl, flag);
     ++n;
   } else {
     if (tiles > 0) {
@@ -869,6 +915,10 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) 
       ctx->expert_align = (int32_t)value;
       ctx->planned = false;           // offsets of an earlier plan no longer describe the layout asked for
       ctx->layout_done = false;
+      return MOE_OK;
+    case MOE_OPT_CLUSTER_PLAN:
+      if (value != 0 && value != 1) return MOE_ERR_INVALID_ARG;
+      ctx->cluster_plan = (int32_t)value;
       return MOE_OK;
     case MOE_OPT_OVERLAP:
       if (value != 0 && value != 1) return MOE_ERR_INVALID_ARG;

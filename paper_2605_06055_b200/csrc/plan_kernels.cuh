@@ -22,6 +22,8 @@
 //                      plan in one launch, small offsets final at once.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace moe {
@@ -287,12 +289,68 @@ __host__ __device__ constexpr int rank_plan_smem_ints(int E, int R, int warps) {
   return (warps + 2) * E > notify_smem_ints(E, R) ? (warps + 2) * E : notify_smem_ints(E, R);
 }
 
+// Notify inside a thread-block cluster (the R CTAs of plan_rank_kernel launched as ONE cluster).
+// Every CTA keeps its row of M in shared memory; after a cluster barrier CTA d builds the offsets
+// of window d (its E/R experts x R source ranks) straight from the other CTAs' shared memory, so
+// the count matrix makes no trip through global memory, no CTA waits on a ticket, and the R windows
+// are scanned in parallel instead of by the last CTA alone.
+// Shared memory behind the planner's own: gathered tile [E/R][R+1], padded totals [E/R], their
+// prefix [E/R + 1], warp sums [33].
+__host__ __device__ constexpr int cluster_notify_smem_ints(int E, int R) {
+  return (E / R) * (R + 1) + 2 * (E / R) + 1 + 33;
+}
+
+__device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, [E] */, int32_t* scratch, int32_t E,
+                                               int32_t R, int32_t d, int32_t full_table, int32_t align,
+                                               int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+                                               int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int E_r = E / R, P = R + 1, nthreads = (int)blockDim.x, tid = (int)threadIdx.x;
+  int32_t* tile = scratch;            // [E_r][P]: entry (el, rr) = M[rr][d*E_r + el]
+  int32_t* tot = tile + E_r * P;      // [E_r] rows each expert's run occupies
+  int32_t* pre = tot + E_r;           // [E_r + 1]
+  int32_t* warp_sums = pre + E_r + 1;
+  cluster.sync();                     // every CTA's row of M is complete and visible
+  for (int q = tid; q < E_r * R; q += nthreads) {   // consecutive threads: consecutive experts of one remote row
+    const int el = q % E_r, rr = q / E_r;
+    const int32_t* remote = cluster.map_shared_rank(my_row, rr);
+    tile[el * P + rr] = remote[d * E_r + el];
+  }
+  __syncthreads();
+  if (full_table)
+    for (int rr = tid; rr < R; rr += nthreads) {     // branches from source rank rr to this rank
+      int32_t acc = 0;
+      for (int el = 0; el < E_r; ++el) acc += tile[el * P + rr];
+      c_rank[(size_t)rr * R + d] = acc;
+    }
+  __syncthreads();
+  for (int el = tid; el < E_r; el += nthreads) {     // exclusive prefix over source ranks, in place
+    int32_t run = 0;
+    for (int rr = 0; rr < R; ++rr) {
+      const int32_t m = tile[el * P + rr];
+      tile[el * P + rr] = run;
+      run += m;
+    }
+    n_exp[d * E_r + el] = run;
+    tot[el] = (run + align - 1) / align * align;
+  }
+  __syncthreads();
+  block_exclusive_scan(tot, pre, E_r, warp_sums);
+  __syncthreads();
+  for (int q = tid; q < E_r * R; q += nthreads)      // o[d*E_r + el][rr], one coalesced stream
+    o[(size_t)d * E_r * R + q] = pre[q / R] + tile[(q / R) * P + q % R];
+  if (tid == 0) n_recv[d] = pre[E_r];
+  cluster.sync();                     // no CTA leaves while its row may still be read
+}
+
 template <int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
                  int32_t full_table, int32_t align, int32_t* __restrict__ s, int32_t* __restrict__ M,
                  int32_t* __restrict__ c_rank,
-                 int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
+                 int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl,
+                 int32_t as_cluster /* the grid is one thread-block cluster of R CTAs */) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
   // A dispatch launched behind this kernel with programmatic serialization (moe_plan_dispatch) may start
@@ -359,6 +417,10 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += WARPS * 32) M[(size_t)r * E + e] = rank_base[e];
+  if (as_cluster) {
+    cluster_notify(rank_base, sm + (P + 1) * E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
+    return;
+  }
 
   __threadfence();
   __syncthreads();

@@ -199,3 +199,30 @@ def test_overlapped_step_is_capturable_and_replayable():
         assert np.array_equal(u16(win), o.windows_zero_init)
         assert harness.max_ulp_diff(u16(Y), o.Y) <= 1
     comm.close()
+
+
+@pytest.mark.parametrize("cluster", [1, 0])
+@pytest.mark.parametrize("schedule", [PREFILL, DECODE])
+@pytest.mark.parametrize("case", [
+    ("c2_shape", 2048, 7168, 256, 16, 8, None),
+    ("R8_ragged_empty_rank", 1500, 256, 64, 8, 6, (0, 400, 1, 99, 500, 0, 250, 250)),
+    ("R2_big_E", 900, 64, 2048, 2, 8, None),           # E above the wide planner's limit: 8-warp CTAs
+    ("R4_tiny", 8, 64, 4, 4, 1, None),
+    ("R16_E16", 320, 128, 16, 16, 4, None),            # one expert per rank
+], ids=lambda c: c[0])
+def test_single_launch_planner_as_a_cluster_and_with_the_last_cta(case, schedule, cluster):
+    """The small-batch planner gives the same table whether its CTAs exchange their count rows through
+    distributed shared memory (one cluster of R CTAs) or through global memory and a ticket."""
+    name, T, H, E, R, K, per = case
+    wl = Workload(name, T, H, E, R, K, schedule, "uniform", "scale", 6100 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    for align in (1, 8):
+        p = oracle.plan(inp.topk_idx.numpy(), E, R, inp.rank_tok_start, align=align)
+        C = int(p.n_recv.max()) + 1
+        o = harness.oracle_run(inp, C, align=align)
+        comm = binding.MoeComm(T, H, E, R, K, torch.device(DEV))
+        comm.moe_set_option(binding.MOE_OPT_CLUSTER_PLAN, cluster)
+        for _ in range(2):
+            g = harness.gpu_run(inp, C, schedule, comm=comm, align=align)
+            harness.assert_parity(g, o, schedule, align=align)
+        comm.close()
