@@ -43,6 +43,7 @@ struct moe_ctx {
   int32_t overlap;          // MOE_OPT_OVERLAP
   int32_t cluster_plan;     // MOE_OPT_CLUSTER_PLAN
   bool plan_cluster_ok;     // the compact planner of this shape can be launched as one cluster of R CTAs
+  bool scan_cluster_ok;     // the same for the scan kernel of the tile planner
   int32_t expert_align;     // MOE_OPT_EXPERT_ALIGN: every expert's run starts on a multiple of this many rows
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
@@ -241,20 +242,33 @@ void launch_dispatch_regs(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   kernel<<<grid, 256, 0, st>>>(x, win, b, ctx->map);
 }
 
-// Launch with programmatic stream serialization when `pdl` is set: the kernel may then start while
+// Launch with optional attributes.  `pdl`: programmatic stream serialization, i.e. the kernel may start while
 // the previous kernel of the stream is still running and orders itself with dependency_wait().
+// `cluster` > 0: the grid runs as thread-block clusters of that many CTAs.
 template <class... KArgs, class... Args>
-void launch_kernel(void (*kernel)(KArgs...), int grid, int threads, int smem, cudaStream_t st, bool pdl, Args... args) {
+void launch_kernel(void (*kernel)(KArgs...), int grid, int threads, int smem, cudaStream_t st, bool pdl, int cluster,
+                   Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3((unsigned)threads);
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster > 0) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.numAttrs = n;
   cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -272,7 +286,7 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   set_work(ctx, b, (int64_t)grid * warps, g_max);
   const int smem = warps * BULK_STAGES * (b.granule * 512 + 8);
   b.pdl = pdl;
-  launch_kernel(dispatch_bulk_kernel, grid, warps * 32, smem, st, pdl, reinterpret_cast<const unsigned char*>(x),
+  launch_kernel(dispatch_bulk_kernel, grid, warps * 32, smem, st, pdl, 0, reinterpret_cast<const unsigned char*>(x),
                 reinterpret_cast<unsigned char*>(win), b, ctx->map);
 }
 
@@ -284,7 +298,7 @@ void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const floa
                       : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), false>;
   const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
-  set_work(ctx, b, (int64_t)grid * 8, 1 << 20);
+  set_work(ctx, b, (int64_t)grid * 8, 1 << 20, !large);   // the large-job form has no tail items
   // an item that is one or two batches of loads cannot hide its own metadata latency: prefetch it
   constexpr int unroll = KT > 0 ? combine_unroll(KT) : 4;
   b.prefetch_meta = (b.granule + unroll - 1) / unroll <= 2;
@@ -338,6 +352,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->overlap = 1;
   ctx->cluster_plan = 1;
   ctx->plan_cluster_ok = false;
+  ctx->scan_cluster_ok = false;
   ctx->expert_align = 1;
   ctx->out_stream = nullptr;
   ctx->in_stream = nullptr;
@@ -391,6 +406,16 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
                    : cudaOccupancyMaxActiveClusters(&clusters, plan_rank_kernel<8>, &cfg)) == cudaSuccess && clusters >= 1;
     cudaGetLastError();
     ctx->plan_cluster_ok = fits;
+    // the scan kernel of the tile planner, same cluster shape
+    cfg.blockDim = dim3((unsigned)PLAN_THREADS);
+    cfg.dynamicSmemBytes = (size_t)(shape->E + cluster_notify_smem_ints(shape->E, shape->R)) * sizeof(int32_t);
+    clusters = 0;
+    fits = (int)cfg.dynamicSmemBytes <= big;
+    if (fits && shape->R > 8)
+      fits = cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    if (fits) fits = cudaOccupancyMaxActiveClusters(&clusters, plan_scan_kernel, &cfg) == cudaSuccess && clusters >= 1;
+    cudaGetLastError();
+    ctx->scan_cluster_ok = fits;
   }
   *out = ctx;
   return MOE_OK;
@@ -513,25 +538,15 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
     const bool as_cluster = ctx->cluster_plan && ctx->plan_cluster_ok;
     const int threads = (wide ? 32 : 8) * 32;
     const int smem = rank_smem + (as_cluster ? cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t) : 0);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)sh.R);
-    cfg.blockDim = dim3((unsigned)threads);
-    cfg.dynamicSmemBytes = (size_t)smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)sh.R;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = as_cluster ? 1 : 0;
     const int32_t flag = as_cluster ? 1 : 0;
     if (wide)
-      cudaLaunchKernelEx(&cfg, plan_rank_kernel<32>, topk_idx, map, sh.K, sh.E, (int32_t)full, ctx->expert_align, ctx->s,
-                         ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl, flag);
+      launch_kernel(plan_rank_kernel<32>, sh.R, threads, smem, st, false, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
+                    (int32_t)full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
+                    ctx->ctl, flag);
     else
-      cudaLaunchKernelEx(&cfg, plan_rank_kernel<8>, topk_idx, map, sh.K, sh.E, (int32_t)full, ctx->expert_align, ctx->s,
-                         ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl, flag);
+      launch_kernel(plan_rank_kernel<8>, sh.R, threads, smem, st, false, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
+                    (int32_t)full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
+                    ctx->ctl, flag);
     ++n;
   } else {
     if (tiles > 0) {
@@ -543,12 +558,21 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
             topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
       ++n;
     }
-    plan_scan_kernel<<<sh.R, PLAN_THREADS, scan_smem, st>>>(ctx->tile_hist, map, sh.E, full, ctx->expert_align, ctx->M,
-                                                            ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl);
+    // The three kernels are chained by programmatic stream serialization: each may be scheduled while the one
+    // in front still runs and waits for it before touching its output, so launch latencies (and the finalize
+    // kernel's index loads) overlap the kernel in front.  The scan kernel's R CTAs run as one cluster when
+    // the device can co-schedule them (see cluster_notify).
+    const bool chain = ctx->overlap != 0;
+    const bool scan_cluster = ctx->cluster_plan && ctx->scan_cluster_ok;
+    const int scan_bytes =
+        scan_cluster ? (sh.E + cluster_notify_smem_ints(sh.E, sh.R)) * (int)sizeof(int32_t) : scan_smem;
+    launch_kernel(plan_scan_kernel, sh.R, PLAN_THREADS, scan_bytes, st, chain && tiles > 0, scan_cluster ? sh.R : 0,
+                  ctx->tile_hist, map, sh.E, (int32_t)full, ctx->expert_align, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp,
+                  ctx->n_recv, ctx->ctl, (int32_t)(scan_cluster ? 1 : 0));
     ++n;
     if (full && tiles > 0) {
-      plan_finalize_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, 0, st>>>(topk_idx, map, sh.K, sh.E, ctx->tile_rank,
-                                                                          ctx->tile_hist, ctx->s);
+      launch_kernel(plan_finalize_kernel<ROUNDS_PREFILL>, tiles, PLAN_THREADS, 0, st, chain, 0, topk_idx, map, sh.K, sh.E,
+                    ctx->tile_rank, ctx->tile_hist, ctx->s);
       ++n;
     }
   }
@@ -1060,7 +1084,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
     plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, PLAN_WARPS * E * (int)sizeof(int32_t), st>>>(
         topk_idx, map, K, E, sc->tile_rank, sc->tile_hist, status);
   plan_scan_kernel<<<R, PLAN_THREADS, notify_smem_ints(E, R) * (int)sizeof(int32_t), st>>>(
-      sc->tile_hist, map, E, 0, 1, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl);
+      sc->tile_hist, map, E, 0, 1, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl, 0);
   RowArgs a;
   a.topk_idx = topk_idx;
   a.small_off = sc->tile_rank;

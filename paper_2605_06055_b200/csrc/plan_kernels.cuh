@@ -13,13 +13,18 @@
 //   plan_scan_kernel   one CTA per source rank: exclusive scan of the tile
 //                      histograms over that rank's tiles ("per-block counting
 //                      plus prefix accumulation over earlier blocks") -> tile
-//                      bases, row r of M.  The CTA that finishes last turns M
-//                      into n_exp, n_recv, c_rank and the large offsets o
-//                      (exclusive scan in window order: expert, then source rank).
+//                      bases, row r of M.  Then M becomes n_exp, n_recv, c_rank and the
+//                      large offsets o (exclusive scan in window order: expert, then
+//                      source rank): by every CTA for its own window when the R CTAs
+//                      run as one thread-block cluster (rows of M exchanged through
+//                      distributed shared memory), else by the CTA that finishes last.
 //   plan_finalize_kernel  PREFILL only: s = in-tile rank + tile base.
 //                      (DECODE folds this step into the dispatch launch.)
 //   plan_rank_kernel   few branches per rank (decode steps, small prefill chunks): the whole
 //                      plan in one launch, small offsets final at once.
+// The tile, scan and finalize kernels are chained by programmatic stream serialization: each lets
+// the next be scheduled at its start, and each waits for the one in front before it touches that
+// kernel's output.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -33,6 +38,7 @@ __global__ void __launch_bounds__(PLAN_THREADS)
 plan_tile_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
                  int32_t* __restrict__ tile_rank, int32_t* __restrict__ tile_hist, int32_t* status) {
   extern __shared__ int32_t warp_hist[];  // [PLAN_WARPS][E]
+  release_dependents();   // the scan kernel may be scheduled now; it waits for this kernel before reading anything
   const int tile = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -238,58 +244,8 @@ __device__ __forceinline__ void build_large_offsets(const int32_t* __restrict__ 
   for (int d = threadIdx.x; d < R; d += (int)blockDim.x) n_recv[d] = pre_s[(d + 1) * E_r] - pre_s[d * E_r];
 }
 
-__global__ void __launch_bounds__(PLAN_THREADS)
-plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusive bases */,
-                 const __grid_constant__ RankMap map, int32_t E, int32_t full_table, int32_t align,
-                 int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
-                 int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl) {
-  extern __shared__ int32_t sm[];  // notify_smem_ints(E, R) ints
-  __shared__ int is_last;
-  const int r = blockIdx.x;
-  const int R = map.R;
-  const int t0 = map.tile_start[r], t1 = map.tile_start[r + 1];
-
-  for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
-    int32_t run = 0;
-    for (int tb = t0; tb < t1; tb += 16) {   // loads first, then the in-place stores (see build_large_offsets)
-      int32_t c[16];
-#pragma unroll
-      for (int k = 0; k < 16; ++k) c[k] = (tb + k < t1) ? tile_hist[(size_t)(tb + k) * E + e] : 0;
-#pragma unroll
-      for (int k = 0; k < 16; ++k)
-        if (tb + k < t1) {
-          tile_hist[(size_t)(tb + k) * E + e] = run;
-          run += c[k];
-        }
-    }
-    M[(size_t)r * E + e] = run;
-  }
-
-  // Last block done: the final CTA to arrive sees every row of M.
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(&ctl->scan_ticket, 1) == R - 1);
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-
-  build_large_offsets(M, E, R, full_table, align, c_rank, o, n_exp, n_recv, sm);
-  if (threadIdx.x == 0) ctl->scan_ticket = 0;  // ready for the next plan on this stream
-}
-
-// Compact planner for batches in which every source rank holds few branches (every decode step,
-// small prefill chunks): ONE launch, one CTA per source rank.  The CTA walks its rank's branches in
-// passes of WARPS*32, carrying the running per-expert count in shared memory, so the small offsets
-// come out final (no tile bases), row r of M falls out at the end, and the last CTA to finish
-// builds the large offsets.
-// Shared memory: counts [E][WARPS+1] (expert-major with an odd pitch: neither the leaders' scattered
-// writes -- same warp column, different experts -- nor the scanning warp's row reads collide on a
-// bank), running base [E]; reused by the Notify step at the end.
-__host__ __device__ constexpr int rank_plan_smem_ints(int E, int R, int warps) {
-  return (warps + 2) * E > notify_smem_ints(E, R) ? (warps + 2) * E : notify_smem_ints(E, R);
-}
-
-// Notify inside a thread-block cluster (the R CTAs of plan_rank_kernel launched as ONE cluster).
+// Notify inside a thread-block cluster (the R CTAs of plan_rank_kernel or plan_scan_kernel launched as
+// ONE cluster).
 // Every CTA keeps its row of M in shared memory; after a cluster barrier CTA d builds the offsets
 // of window d (its E/R experts x R source ranks) straight from the other CTAs' shared memory, so
 // the count matrix makes no trip through global memory, no CTA waits on a ticket, and the R windows
@@ -342,6 +298,67 @@ __device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, 
     o[(size_t)d * E_r * R + q] = pre[q / R] + tile[(q / R) * P + q % R];
   if (tid == 0) n_recv[d] = pre[E_r];
   cluster.sync();                     // no CTA leaves while its row may still be read
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS)
+plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusive bases */,
+                 const __grid_constant__ RankMap map, int32_t E, int32_t full_table, int32_t align,
+                 int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+                 int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl,
+                 int32_t as_cluster /* the grid is one thread-block cluster of R CTAs */) {
+  // notify_smem_ints(E, R) ints, or (as a cluster) this CTA's row of M [E] followed by cluster_notify_smem_ints(E, R)
+  extern __shared__ int32_t sm[];
+  __shared__ int is_last;
+  release_dependents();   // lets the kernel behind (finalize, or a dispatch) be scheduled; it waits for this one
+  dependency_wait();      // the tile histograms are complete (returns at once under a plain launch)
+  const int r = blockIdx.x;
+  const int R = map.R;
+  const int t0 = map.tile_start[r], t1 = map.tile_start[r + 1];
+
+  for (int e = threadIdx.x; e < E; e += PLAN_THREADS) {
+    int32_t run = 0;
+    for (int tb = t0; tb < t1; tb += 16) {   // loads first, then the in-place stores (see build_large_offsets)
+      int32_t c[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) c[k] = (tb + k < t1) ? tile_hist[(size_t)(tb + k) * E + e] : 0;
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        if (tb + k < t1) {
+          tile_hist[(size_t)(tb + k) * E + e] = run;
+          run += c[k];
+        }
+    }
+    M[(size_t)r * E + e] = run;
+    if (as_cluster) sm[e] = run;
+  }
+  if (as_cluster) {   // see cluster_notify: every CTA builds its own window's offsets from the rows in shared memory
+    __syncthreads();
+    cluster_notify(sm, sm + E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
+    return;
+  }
+
+  // Last block done: the final CTA to arrive sees every row of M.
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(&ctl->scan_ticket, 1) == R - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+
+  build_large_offsets(M, E, R, full_table, align, c_rank, o, n_exp, n_recv, sm);
+  if (threadIdx.x == 0) ctl->scan_ticket = 0;  // ready for the next plan on this stream
+}
+
+// Compact planner for batches in which every source rank holds few branches (every decode step,
+// small prefill chunks): ONE launch, one CTA per source rank.  The CTA walks its rank's branches in
+// passes of WARPS*32, carrying the running per-expert count in shared memory, so the small offsets
+// come out final (no tile bases), row r of M falls out at the end, and the last CTA to finish
+// builds the large offsets.
+// Shared memory: counts [E][WARPS+1] (expert-major with an odd pitch: neither the leaders' scattered
+// writes -- same warp column, different experts -- nor the scanning warp's row reads collide on a
+// bank), running base [E]; reused by the Notify step at the end.
+__host__ __device__ constexpr int rank_plan_smem_ints(int E, int R, int warps) {
+  return (warps + 2) * E > notify_smem_ints(E, R) ? (warps + 2) * E : notify_smem_ints(E, R);
 }
 
 template <int WARPS>
@@ -450,6 +467,7 @@ __global__ void __launch_bounds__(PLAN_THREADS)
 plan_finalize_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
                      const int32_t* __restrict__ tile_rank, const int32_t* __restrict__ tile_base,
                      int32_t* __restrict__ s) {
+  release_dependents();   // a dispatch launched behind the plan may be scheduled; it waits for this kernel
   const int tile = blockIdx.x;
   int r = 0;
   {
@@ -462,11 +480,19 @@ plan_finalize_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant
   }
   const int32_t b_begin = map.tok_start[r] * K + ((tile - map.tile_start[r]) << map.tile_shift);
   const int32_t b_end = min(b_begin + (ROUNDS * PLAN_THREADS), map.tok_start[r + 1] * K);
+  // The routing indexes do not depend on the kernels in front: they travel while the scan kernel runs.
+  int32_t e_of[ROUNDS];
+#pragma unroll
+  for (int i = 0; i < ROUNDS; ++i) {
+    const int32_t b = b_begin + i * PLAN_THREADS + threadIdx.x;
+    e_of[i] = b < b_end ? __ldg(topk_idx + b) : -1;
+  }
+  dependency_wait();   // tile ranks and tile bases are complete (returns at once under a plain launch)
 #pragma unroll
   for (int i = 0; i < ROUNDS; ++i) {
     const int32_t b = b_begin + i * PLAN_THREADS + threadIdx.x;
     if (b < b_end) {
-      const int32_t e = __ldg(topk_idx + b);
+      const int32_t e = e_of[i];
       s[b] = (e >= 0 && e < E) ? tile_rank[b] + tile_base[(size_t)tile * E + e] : 0;
     }
   }

@@ -209,20 +209,26 @@ __device__ __forceinline__ int32_t fetch_item(const RowArgs& a, ItemFeed& f) {
   return (int32_t)min(item, (int64_t)a.n_items);
 }
 
+// TAIL = false: the launch has no finer-cut tail (n_head == n_items); saves the selects in kernels whose
+// registers are all spoken for (the large-job combine).
+template <bool TAIL = true>
 __device__ __forceinline__ WorkItem decode_item(const RowArgs& a, int32_t item) {
   WorkItem w;
-  const int32_t upr = (a.H16 + 31) >> 5;
-  if (item < a.n_head) {
+  if constexpr (TAIL) {
+    // head and tail items differ only in four launch constants: selects, then one division
+    const bool tail = item >= a.n_head;
+    const int32_t ipr = tail ? a.tail_items_per_row : a.items_per_row;
+    const int32_t g = tail ? a.tail_granule : a.granule;
+    const int32_t rem = tail ? item - a.n_head : item;
+    const int32_t q = rem / ipr;
+    w.t = a.t_begin + (tail ? a.head_rows : 0) + q;
+    w.i0 = (rem - q * ipr) * g;
+    w.i1 = min(w.i0 + g, (a.H16 + 31) >> 5);
+  } else {
     const int32_t q = item / a.items_per_row;
     w.t = a.t_begin + q;
     w.i0 = (item - q * a.items_per_row) * a.granule;
-    w.i1 = min(w.i0 + a.granule, upr);
-  } else {
-    const int32_t rem = item - a.n_head;
-    const int32_t q = rem / a.tail_items_per_row;
-    w.t = a.t_begin + a.head_rows + q;
-    w.i0 = (rem - q * a.tail_items_per_row) * a.tail_granule;
-    w.i1 = min(w.i0 + a.tail_granule, upr);
+    w.i1 = min(w.i0 + a.granule, (a.H16 + 31) >> 5);
   }
   return w;
 }
@@ -312,6 +318,7 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float (&acc)[8]) {
   return make_uint4(u[0], u[1], u[2], u[3]);
 }
 
+// L1_ALLOC selects the large-job form: L1-allocating loads (see ld_row) and no finer-cut tail items.
 template <int KT, int UNROLL, bool L1_ALLOC>
 __global__ void __launch_bounds__(256, 1)
 combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__ topk_w, uint4* __restrict__ Y,
@@ -326,15 +333,15 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
   ItemFeed feed = begin_feed();
   int32_t item = fetch_item(a, feed);
   BranchMeta meta = {-1, 0, 0.0f};
-  if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item(a, item).t, lane);
+  if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item<!L1_ALLOC>(a, item).t, lane);
   while (item < a.n_items) {
     const int32_t next_item = fetch_item(a, feed);
-    const WorkItem wi = decode_item(a, item);
+    const WorkItem wi = decode_item<!L1_ALLOC>(a, item);
     if (!a.prefetch_meta) meta = load_meta(a, topk_w, wi.t, lane);
     const int64_t slot = finish_slot(a, map, meta, wi.t, lane, false);
     const float w_lane = meta.w;
     // short rows: the next item's routing index, small offset and weight travel while this item is reduced
-    if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item(a, next_item).t, lane);
+    if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item<!L1_ALLOC>(a, next_item).t, lane);
     item = next_item;
     uint4* out = Y + (size_t)wi.t * H16;
     if constexpr (KT > 0) {
