@@ -241,10 +241,12 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
  *                          every device-side wait by v milliseconds: that warp gives up, the status
  *                          word becomes MOE_ERR_TIMEOUT, the kernel ends normally (no trap, nothing
  *                          left in flight) and the windows are incomplete.  Normal bound: 2 s.
- *   MOE_OPT_OVERLAP        1 (default): moe_plan_dispatch starts its dispatch kernel while the planner
- *                          runs (programmatic stream serialization; the early part of the kernel
- *                          reads nothing the planner writes).  0: the dispatch kernel starts after the
- *                          planner has ended.  Same result either way.
+ *   MOE_OPT_OVERLAP        1 (default): kernels that one call enqueues back to back are chained by programmatic
+ *                          stream serialization -- moe_plan_dispatch starts its dispatch kernel while the
+ *                          planner runs, the planner's own kernels and the planner behind the gate kernel
+ *                          (moe_gate_plan) are scheduled while the kernel in front still runs -- and each
+ *                          waits for the kernel in front before it reads anything that kernel writes.
+ *                          0: every kernel starts after the previous one has ended.  Same result either way.
  *   MOE_OPT_EXPERT_ALIGN   A in [1, 4096], default 1 (the packed layout of Section 5.2).  With A > 1 later
  *                          plans pad the run of every expert to a whole number of A-row groups, so that
  *                          every expert's first row is a multiple of A inside its window and a grouped

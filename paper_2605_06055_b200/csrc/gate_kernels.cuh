@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(256)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
                  float* __restrict__ topk_w) {
   extern __shared__ float gate_rows[];
+  release_dependents();   // a planner launched behind the gate (moe_gate_plan) may be scheduled; it waits for this kernel
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpc = blockDim.x >> 5;
   for (int32_t t = blockIdx.x * wpc + warp; t < T; t += gridDim.x * wpc) {
     int32_t idx;

@@ -539,23 +539,25 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
     const int threads = (wide ? 32 : 8) * 32;
     const int smem = rank_smem + (as_cluster ? cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t) : 0);
     const int32_t flag = as_cluster ? 1 : 0;
+    const bool behind_gate = logits != nullptr && ctx->overlap != 0;
     if (wide)
-      launch_kernel(plan_rank_kernel<32>, sh.R, threads, smem, st, false, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
+      launch_kernel(plan_rank_kernel<32>, sh.R, threads, smem, st, behind_gate, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
                     (int32_t)full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
                     ctx->ctl, flag);
     else
-      launch_kernel(plan_rank_kernel<8>, sh.R, threads, smem, st, false, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
+      launch_kernel(plan_rank_kernel<8>, sh.R, threads, smem, st, behind_gate, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
                     (int32_t)full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
                     ctx->ctl, flag);
     ++n;
   } else {
     if (tiles > 0) {
+      const bool behind_gate = logits != nullptr && ctx->overlap != 0;
       if (full)
-        plan_tile_kernel<ROUNDS_PREFILL><<<tiles, PLAN_THREADS, tile_smem, st>>>(
-            topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
+        launch_kernel(plan_tile_kernel<ROUNDS_PREFILL>, tiles, PLAN_THREADS, tile_smem, st, behind_gate, 0, topk_idx, map,
+                      sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
       else
-        plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, tile_smem, st>>>(
-            topk_idx, map, sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
+        launch_kernel(plan_tile_kernel<ROUNDS_DECODE>, tiles, PLAN_THREADS, tile_smem, st, behind_gate, 0, topk_idx, map,
+                      sh.K, sh.E, ctx->tile_rank, ctx->tile_hist, &ctx->ctl->status);
       ++n;
     }
     // The three kernels are chained by programmatic stream serialization: each may be scheduled while the one

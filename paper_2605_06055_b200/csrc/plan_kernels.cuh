@@ -38,6 +38,7 @@ __global__ void __launch_bounds__(PLAN_THREADS)
 plan_tile_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,
                  int32_t* __restrict__ tile_rank, int32_t* __restrict__ tile_hist, int32_t* status) {
   extern __shared__ int32_t warp_hist[];  // [PLAN_WARPS][E]
+  dependency_wait();      // behind the gate kernel (moe_gate_plan): its indexes are complete; else returns at once
   release_dependents();   // the scan kernel may be scheduled now; it waits for this kernel before reading anything
   const int tile = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -370,6 +371,9 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
                  int32_t as_cluster /* the grid is one thread-block cluster of R CTAs */) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
+  // Behind the gate kernel (moe_gate_plan) this kernel may have been scheduled early: the routing indexes
+  // are complete once the wait returns (at once under a plain launch).
+  dependency_wait();
   // A dispatch launched behind this kernel with programmatic serialization (moe_plan_dispatch) may start
   // now and move its first payload loads while the plan is computed; it waits for this kernel's
   // completion before it reads anything written here.  Without such a dependent this does nothing.
