@@ -149,6 +149,17 @@ moe_status_t moe_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, const in
                                int32_t T, const int32_t* rank_tok_start /*HOST*/, const void* x /*DEVICE*/,
                                void* windows /*DEVICE*/, int64_t capacity_rows, void* stream);
 
+/* The whole front of a layer in one call: moe_gate_topk, moe_plan and moe_dispatch enqueued back to
+ * back and chained like moe_plan_dispatch (the planner is scheduled behind the gate kernel and reads the
+ * indexes only after that kernel has completed; the dispatch kernel is scheduled behind the planner,
+ * releases nothing and reads no index before the planner has passed that point).  Same result as the
+ * three calls.  Arguments as in moe_gate_plan and moe_dispatch; topk_idx and topk_w are outputs. */
+moe_status_t moe_gate_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, const float* logits /*DEVICE*/,
+                                    int32_t T, const int32_t* rank_tok_start /*HOST*/,
+                                    int32_t* topk_idx /*DEVICE*/, float* topk_w /*DEVICE*/,
+                                    const void* x /*DEVICE*/, void* windows /*DEVICE*/, int64_t capacity_rows,
+                                    void* stream);
+
 /* Row-wise quantised dispatch (Section 5.2, Prefill Dispatch: with row-wise quantisation the scale
  * values go to a parallel scale tensor in the same row order).  The paper names no format; this
  * library's definition is fp8 e4m3 (1-4-3, bias 7, largest finite 448, no infinities) with one fp32

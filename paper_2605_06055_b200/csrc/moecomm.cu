@@ -688,6 +688,18 @@ moe_status_t moe_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, const in
   return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream, 0, -1, true);
 }
 
+moe_status_t moe_gate_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, const float* logits, int32_t T,
+                                    const int32_t* rank_tok_start, int32_t* topk_idx, float* topk_w, const void* x,
+                                    void* windows, int64_t capacity_rows, void* stream) {
+  if (ctx == nullptr || ctx->shape.K > ctx->shape.E) return MOE_ERR_INVALID_ARG;
+  if (T > 0 && (logits == nullptr || topk_idx == nullptr || topk_w == nullptr || x == nullptr || windows == nullptr))
+    return MOE_ERR_INVALID_ARG;
+  if (capacity_rows < 0 || !aligned16(x) || !aligned16(windows)) return MOE_ERR_INVALID_ARG;
+  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, logits, topk_idx, topk_w);
+  if (rc != MOE_OK) return rc;
+  return dispatch_impl(ctx, x, windows, nullptr, capacity_rows, stream, 0, -1, true);
+}
+
 moe_status_t moe_dispatch_range(moe_ctx_t* ctx, const void* x, void* windows, int64_t capacity_rows, int32_t t_begin,
                                 int32_t t_end, void* stream) {
   if (ctx != nullptr && ctx->T > 0 && windows == nullptr) return MOE_ERR_INVALID_ARG;

@@ -81,6 +81,20 @@ def test_gate_plan_matches_oracle_gate_then_oracle_plan(case):
     comm.moe_combine(win, C, w, y)
     assert comm.moe_status() == 0
     assert torch.equal(y.view(torch.int16) & 0x7FFF, x.view(torch.int16) & 0x7FFF)
+    # the same front of the layer as ONE call (gate, plan and dispatch chained), several times with nothing
+    # synchronised in between: same indexes, same window bytes as the separate calls just made
+    win_sep = win.clone()
+    for _ in range(3):
+        idx.fill_(-1)
+        w.fill_(-1.0)
+        win.zero_()
+        comm.moe_gate_plan_dispatch(sch, l.to(dev), idx, w, x, win, C, T, rts)
+        comm.moe_combine(win, C, w, y)
+    assert comm.moe_status() == 0
+    assert np.array_equal(idx.cpu().numpy(), want_idx)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+    assert torch.equal(win.view(torch.int16), win_sep.view(torch.int16))
+    assert torch.equal(y.view(torch.int16) & 0x7FFF, x.view(torch.int16) & 0x7FFF)
     comm.close()
 
 
