@@ -67,7 +67,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
 }
 
 // Window rows are written once and not read again by this kernel: an evict-first L2 policy on the
-// stores measured 1-8 % faster (653 vs 661 us at prefill size, 47 vs 51 us at decode size).
+// stores measured 1-8 % faster (653 vs 661 us at prefill size, 47 vs 51 us at decode size).  The same
+// policy on the row loads measured slower (664 vs 662 us, and the combine behind it 51 vs 49 us at
+// decode size), so they keep the default.
 __device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes, uint64_t policy) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
                ::"l"(dst), "r"(src_smem), "r"(bytes), "l"(policy) : "memory");
