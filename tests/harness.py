@@ -90,7 +90,7 @@ def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4, align: int = 1) ->
 
 
 @dataclass
-class GpuRun:
+class DeviceRun:
     view: dict          # plan tensors copied to host (numpy) after the run
     slots: np.ndarray
     windows: np.ndarray  # after dispatch, before the expert op
@@ -102,7 +102,7 @@ class GpuRun:
 
 def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Optional[binding.MoeComm] = None,
             T_max: Optional[int] = None, dispatch_path: int = binding.MOE_DISPATCH_AUTO, granule: int = 0,
-            align: int = 1) -> GpuRun:
+            align: int = 1) -> DeviceRun:
     wl = inp.wl
     dev = torch.device("cuda:0")
     schedule = wl.schedule if schedule is None else schedule
@@ -134,14 +134,14 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
     Y = torch.from_numpy(np.full((wl.T, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
     comm.moe_combine(windows, C, w, Y)
     statuses.append(comm.moe_status())
-    out = GpuRun(view, slots.cpu().numpy(), win_host, Y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), statuses,
+    out = DeviceRun(view, slots.cpu().numpy(), win_host, Y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), statuses,
                  e_start.cpu().numpy(), e_count.cpu().numpy())
     if own:
         comm.close()
     return out
 
 
-def assert_parity(g: GpuRun, o: OracleRun, schedule: int, combine_ulp: int = 1, align: int = 1):
+def assert_parity(g: DeviceRun, o: OracleRun, schedule: int, combine_ulp: int = 1, align: int = 1):
     assert g.statuses == [0, 0, 0], g.statuses
     names = {"counts": "M", "c_rank": "c_rank", "small_off": "s", "large_off": "o", "n_exp": "n_exp", "n_recv": "n_recv"}
     for k, on in names.items():
