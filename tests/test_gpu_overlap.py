@@ -226,3 +226,41 @@ def test_single_launch_planner_as_a_cluster_and_with_the_last_cta(case, schedule
             g = harness.gpu_run(inp, C, schedule, comm=comm, align=align)
             harness.assert_parity(g, o, schedule, align=align)
         comm.close()
+
+
+@pytest.mark.parametrize("schedule", [PREFILL, DECODE])
+def test_tile_planner_chain_is_capturable_and_replayable(schedule):
+    """The three chained planner kernels (the scan kernel as one cluster) inside a CUDA graph, with the
+    dispatch behind them, replayed several times and mixed with eager calls."""
+    dev = torch.device(DEV)
+    wl = Workload("tile_graph", 24000, 256, 32, 8, 4, schedule, "uniform", "identity", 6400)   # 12000 branches per rank
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R)
+    C = int(p.n_recv.max())
+    o = harness.oracle_run(inp, C)
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
+    win = torch.zeros((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
+    Y = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    comm.moe_plan_dispatch(schedule, idx, X, win, C)
+    comm.moe_combine(win, C, w, Y)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        comm.moe_plan_dispatch(schedule, idx, X, win, C)
+        comm.moe_combine(win, C, w, Y)
+    for n in (1, 3):
+        win.zero_()
+        Y.zero_()
+        for _ in range(n):
+            g.replay()
+        comm.moe_plan(schedule, idx)                   # eager calls right behind the replays
+        comm.moe_combine(win, C, w, Y)
+        assert comm.moe_status() == 0
+        assert np.array_equal(u16(win), o.windows_zero_init)
+        assert harness.max_ulp_diff(u16(Y), o.Y) <= 1
+        v = comm.moe_plan_view()
+        assert np.array_equal(v["large_off"].cpu().numpy(), o.plan.o)
+        if schedule == PREFILL:
+            assert np.array_equal(v["small_off"].cpu().numpy(), o.plan.s)
+    comm.close()
