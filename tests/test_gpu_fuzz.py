@@ -3,6 +3,8 @@ window byte (canaries included) and the combined rows (<= 1 bf16 ulp), for rando
 hidden sizes, expert / rank / top-k counts, ragged rank maps (empty ranks included), both
 schedules, both dispatch kernels, duplicate experts within a token, several work-item sizes and
 expert alignments."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -32,7 +34,10 @@ def random_workload(rng, i):
                     rank_tokens=per)
 
 
-@pytest.mark.parametrize("i", range(48))
+N_SHAPES = int(os.environ.get("MOE_FUZZ_SHAPES", "48"))     # a soak run sets this to hundreds
+
+
+@pytest.mark.parametrize("i", range(N_SHAPES))
 def test_random_shape(i):
     rng = np.random.default_rng(77000 + i)
     wl = random_workload(rng, i)
@@ -48,7 +53,7 @@ def test_random_shape(i):
     harness.assert_parity(g, o, wl.schedule, align=align)
 
 
-@pytest.mark.parametrize("i", range(12))
+@pytest.mark.parametrize("i", range(max(12, N_SHAPES // 4)))
 def test_random_shape_fused_call_and_quantised_dispatch(i):
     rng = np.random.default_rng(88000 + i)
     wl = random_workload(rng, 100 + i)
