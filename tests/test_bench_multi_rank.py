@@ -63,3 +63,48 @@ def test_count_exchange_between_two_ranks_builds_the_same_matrix_everywhere():
         mp.spawn(_gather_worker, args=(world, 31000 + os.getpid() % 2000, out), nprocs=world, join=True)
         want = [[0, 1, 2, 3, 4, 5], [100, 101, 102, 103, 104, 105]]
         assert out[0] == want and out[1] == want
+
+
+def _protocol_worker(rank, world, port, out):
+    """One expert-parallel rank on CPU: local Layout (the oracle on this rank's tokens), the count
+    exchange over the process group, Notify on the gathered matrix."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import numpy as np
+    import oracle
+    from paper_2605_06055_b200 import ep
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    E, K, align = 12, 3, 4
+    rng = np.random.default_rng(5)
+    counts = [37, 21]
+    idx_all = rng.integers(0, E, (sum(counts), K)).astype(np.int32)
+    lo = sum(counts[:rank])
+    local = idx_all[lo:lo + counts[rank]]
+    only_me = np.array([0] * (rank + 1) + [len(local)] * (world - rank), np.int32)
+    mine = oracle.plan(local, E, world, only_me, align=align)
+    gathered = ep.all_gather_counts(torch.from_numpy(mine.M[rank].copy())).numpy()
+    st, c_rank, o, n_exp, n_recv = oracle.notify(gathered, align=align)
+    out[rank] = (st, mine.s.tolist(), o.tolist(), n_recv.tolist(), gathered.tolist())
+    dist.destroy_process_group()
+
+
+def test_two_ranks_layout_exchange_notify_reproduce_the_global_plan():
+    import numpy as np
+    import oracle
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_protocol_worker, args=(world, 33000 + os.getpid() % 2000, out), nprocs=world, join=True)
+        results = dict(out)
+    E, K, align = 12, 3, 4
+    rng = np.random.default_rng(5)
+    counts = [37, 21]
+    idx_all = rng.integers(0, E, (sum(counts), K)).astype(np.int32)
+    whole = oracle.plan(idx_all, E, world, np.array([0, 37, 58], np.int32), align=align)
+    lo = 0
+    for rank in range(world):
+        st, s_local, o, n_recv, gathered = results[rank]
+        assert st == oracle.OK
+        assert gathered == whole.M.tolist()                       # every rank holds the same matrix
+        assert o == whole.o.tolist() and n_recv == whole.n_recv.tolist()
+        assert s_local == whole.s[lo:lo + counts[rank]].tolist()   # Layout is local
+        lo += counts[rank]
