@@ -264,3 +264,45 @@ def test_tile_planner_chain_is_capturable_and_replayable(schedule):
         if schedule == PREFILL:
             assert np.array_equal(v["small_off"].cpu().numpy(), o.plan.s)
     comm.close()
+
+
+@pytest.mark.parametrize("shape", [(2048, 1024, 256, 16, 8, DECODE), (24000, 64, 32, 8, 4, PREFILL),
+                                   (24000, 64, 32, 8, 4, DECODE), (96, 256, 16, 4, 2, PREFILL)],
+                         ids=["decode_cluster_planner", "tile_planner_prefill", "tile_planner_decode", "tiny"])
+def test_chained_front_equals_the_serialised_calls_on_fresh_random_routings(shape):
+    """gate -> plan -> dispatch as ONE chained call (+ combine) against the same steps enqueued one by one
+    on a context with every overlap switched off, on new logits and rows every iteration: the same
+    indexes, offsets, window bytes and outputs, bit for bit.  (The serialised path is the one the rest
+    of the suite checks against the oracle.)"""
+    T, H, E, R, K, sch = shape
+    dev = torch.device(DEV)
+    a = binding.MoeComm(T, H, E, R, K, dev)
+    b = binding.MoeComm(T, H, E, R, K, dev)
+    b.moe_set_option(binding.MOE_OPT_OVERLAP, 0)
+    b.moe_set_option(binding.MOE_OPT_CLUSTER_PLAN, 0)
+    C = (T * K // R) * 2 + 64
+    gen = torch.Generator(device=dev).manual_seed(4242)
+    for it in range(60):
+        logits = torch.randn(T, E, device=dev, generator=gen)
+        X = torch.randn(T, H, device=dev, generator=gen).bfloat16()
+        ia = torch.empty(T, K, dtype=torch.int32, device=dev)
+        wa = torch.empty(T, K, device=dev)
+        ib, wb = torch.empty_like(ia), torch.empty_like(wa)
+        wina = torch.zeros(R * C, H, dtype=torch.bfloat16, device=dev)
+        winb = torch.zeros_like(wina)
+        Ya, Yb = torch.empty_like(X), torch.empty_like(X)
+        a.moe_gate_plan_dispatch(sch, logits, ia, wa, X, wina, C)
+        a.moe_combine(wina, C, wa, Ya)
+        binding.moe_gate_topk(logits, K, ib, wb)
+        b.moe_plan(sch, ib)
+        b.moe_dispatch(X, winb, C)
+        b.moe_combine(winb, C, wb, Yb)
+        va, vb = a.moe_plan_view(), b.moe_plan_view()
+        assert torch.equal(ia, ib) and torch.equal(wa, wb)
+        assert torch.equal(va["large_off"], vb["large_off"]) and torch.equal(va["n_recv"], vb["n_recv"])
+        assert torch.equal(va["small_off"], vb["small_off"])
+        assert torch.equal(wina.view(torch.int16), winb.view(torch.int16))
+        assert torch.equal(Ya.view(torch.int16), Yb.view(torch.int16))
+    assert a.moe_status() == 0 and b.moe_status() == 0
+    a.close()
+    b.close()
