@@ -429,11 +429,13 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
     wq = torch.empty((dwl.R * dl.C, dwl.H), dtype=torch.uint8, device=dev)
     wscale = torch.empty((dwl.R * dl.C,), dtype=torch.float32, device=dev)
     quant = lambda: c.moe_dispatch_quant(dl.X, wq, wscale, dl.C)
+    quant_fused = lambda: c.moe_plan_dispatch_quant(dwl.schedule, dl.idx, dl.X, wq, wscale, dl.C)
     for name, pre in (("cold", [flush]), ("warm", [])):
         base = time_repeated(pre, n) if pre else 0.0
         t_copy = time_repeated(pre + [copy], n)
         plan()   # the gate leg below leaves the context planned on other indexes
         t_quant = time_repeated(pre + [quant], n)
+        t_quant_fused = time_repeated(pre + [quant_fused], n)
         t1 = time_repeated(pre + [plan], n)
         t2 = time_repeated(pre + [plan, disp], n)
         t3 = time_repeated(pre + [plan, disp, comb], n)
@@ -458,6 +460,7 @@ def decode_latency(dev, peak, n: int = 200) -> dict:
                      "step_us_gate_plan_dispatch_fused_then_combine": t_gate_step - base,
                      "plain_copy_of_the_same_bytes_us": t_copy - base,
                      "dispatch_quant_us": t_quant - base,
+                     "plan_dispatch_quant_fused_us": t_quant_fused - base,
                      "dispatch_quant_GBps": bytes_dispatch_quant(dwl) / (t_quant - base) / 1e3}
     plan()   # leave the context planned on dl.idx again
     assert c.moe_status() == 0

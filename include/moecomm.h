@@ -174,6 +174,14 @@ moe_status_t moe_gate_plan_dispatch(moe_ctx_t* ctx, moe_schedule_t schedule, con
 moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows_q /*DEVICE*/,
                                 float* scales /*DEVICE*/, int64_t capacity_rows, void* stream);
 
+/* moe_plan followed by moe_dispatch_quant as one chained call, like moe_plan_dispatch: the quantising
+ * dispatch kernel is scheduled while the planner runs and loads its first rows meanwhile.  Same result
+ * as the two calls. */
+moe_status_t moe_plan_dispatch_quant(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE*/,
+                                     int32_t T, const int32_t* rank_tok_start /*HOST*/, const void* x /*DEVICE*/,
+                                     void* windows_q /*DEVICE*/, float* scales /*DEVICE*/, int64_t capacity_rows,
+                                     void* stream);
+
 /* Combine (Algorithm 1 / Algorithm 2, second loop; Section 5.2 Prefill Combine):
  *   Y[t,h] = bf16_rne( sum_{j=0..K-1} W[t,j] * float(windows[slot(t,j), h]) )
  * accumulated in fp32 from +0 with one fused multiply-add per term, j ascending.

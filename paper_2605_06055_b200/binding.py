@@ -26,7 +26,7 @@ EXPORTS = [
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
     "moe_gate_topk", "moe_gate_plan", "moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers",
-    "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch",
+    "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
@@ -76,6 +76,8 @@ def load() -> ctypes.CDLL:
     L.moe_plan_dispatch.restype = ctypes.c_int
     L.moe_gate_plan_dispatch.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp, vp, vp, vp, i64, vp]
     L.moe_gate_plan_dispatch.restype = ctypes.c_int
+    L.moe_plan_dispatch_quant.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp, vp, vp, i64, vp]
+    L.moe_plan_dispatch_quant.restype = ctypes.c_int
     L.moe_layout.argtypes = [vp, ctypes.c_int, vp, i32, i32, vp, vp]
     L.moe_notify.argtypes = [vp, vp, vp]
     L.moe_dispatch_peers.argtypes = [vp, vp, vp, i64, vp]
@@ -222,6 +224,22 @@ class MoeComm:
             self.T, self.schedule, self._keep = T, schedule, topk_idx
         elif check:
             raise MoeError(rc, "moe_plan_dispatch")
+        return rc
+
+    def moe_plan_dispatch_quant(self, schedule: int, topk_idx: torch.Tensor, x: torch.Tensor, windows_q: torch.Tensor,
+                                scales: torch.Tensor, capacity_rows: int, T: Optional[int] = None, rank_tok_start=None,
+                                stream=None, check: bool = True) -> int:
+        T = topk_idx.shape[0] if T is None else T
+        rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
+        with self._on_device():
+            rc = self.lib.moe_plan_dispatch_quant(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, _host_ptr(rts),
+                                                  _dev_ptr(x, torch.bfloat16), _dev_ptr(windows_q, torch.uint8),
+                                                  _dev_ptr(scales, torch.float32), int(capacity_rows),
+                                                  _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx
+        elif check:
+            raise MoeError(rc, "moe_plan_dispatch_quant")
         return rc
 
     def moe_gate_plan_dispatch(self, schedule: int, logits: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor,

@@ -713,9 +713,8 @@ moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x, const void* const
   return dispatch_impl(ctx, x, nullptr, window_bases, capacity_rows, stream);
 }
 
-moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, float* scales, int64_t capacity_rows,
-                                void* stream) {
-  moe_ctx* ctx = c;
+static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windows_q, float* scales,
+                                        int64_t capacity_rows, void* stream, bool behind_plan) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
   const int H = ctx->shape.H;
@@ -745,10 +744,34 @@ moe_status_t moe_dispatch_quant(moe_ctx_t* c, const void* x, void* windows_q, fl
   set_work(ctx, a, (int64_t)grid * warps, upr, false);
   ctx->granule_override = keep;
   const int smem = warps * stages * (stage + 8);
-  auto kernel = stages == 3 ? dispatch_quant_kernel<3> : dispatch_quant_kernel<2>;
-  kernel<<<grid, warps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
+  const bool pdl = behind_plan && ctx->overlap != 0;
+  a.pdl = pdl;
+  if (stages == 3)
+    launch_kernel(dispatch_quant_kernel<3>, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
+                  static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
+  else
+    launch_kernel(dispatch_quant_kernel<2>, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
+                  static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
   return launch_ok(ctx);
+}
+
+moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x, void* windows_q, float* scales, int64_t capacity_rows,
+                                void* stream) {
+  return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, false);
+}
+
+moe_status_t moe_plan_dispatch_quant(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                                     const int32_t* rank_tok_start, const void* x, void* windows_q, float* scales,
+                                     int64_t capacity_rows, void* stream) {
+  if (ctx == nullptr || (T > 0 && (topk_idx == nullptr || x == nullptr || windows_q == nullptr || scales == nullptr)))
+    return MOE_ERR_INVALID_ARG;
+  const int H = ctx->shape.H;
+  if (H % 16 != 0 || H * 2 > QUANT_MAX_ROW_BYTES || capacity_rows < 0 || !aligned16(x) || !aligned16(windows_q) ||
+      (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)
+    return MOE_ERR_INVALID_ARG;   // before anything is enqueued
+  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, nullptr, nullptr, nullptr);
+  if (rc != MOE_OK) return rc;
+  return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, true);
 }
 
 }  // extern "C"

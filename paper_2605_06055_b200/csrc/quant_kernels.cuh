@@ -60,10 +60,6 @@ __global__ void __launch_bounds__(QUANT_MAX_WARPS * 32, 1)
 dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
                       float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
   extern __shared__ __align__(128) unsigned char smem[];
-  if (must_abort(a)) {
-    end_work(a);
-    return;
-  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t row_bytes = (uint32_t)a.H16 * 16u;          // bf16 row
   const uint32_t code_bytes = (uint32_t)a.H16 * 8u;          // e4m3 row
@@ -90,9 +86,28 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   // One work item = one token row (items_per_row == 1).  q0 is consumed in this iteration; the load of
   // q1 is issued at its start, into the stage whose code row was stored QUANT_STAGES - 1 iterations ago.
   ItemFeed feed = begin_feed();
-  int32_t q0 = fetch_item(a, feed);
-  int32_t q1 = fetch_item(a, feed);
-  if (lane == 0 && q0 < a.n_items) issue_load(q0, 0);
+  int32_t q0 = a.n_items, q1 = a.n_items;
+  // Started early behind the planner (moe_plan_dispatch_quant): the first two rows of a small job are fixed
+  // and depend on nothing the planner writes, so the first load travels while the plan is computed.
+  const bool early = a.pdl && a.static_first >= 2;
+  if (early) {
+    q0 = fetch_item(a, feed);
+    q1 = fetch_item(a, feed);
+    if (lane == 0 && q0 < a.n_items) issue_load(q0, 0);
+  }
+  dependency_wait();      // returns at once unless this launch was allowed to start early
+  release_dependents();
+  if (must_abort(a)) {
+    // a load already in flight must land before this CTA's shared memory is handed back
+    if (early && lane == 0 && q0 < a.n_items) mbar_wait(bar0, 0, a.wait_limit_ms);
+    end_work(a);
+    return;
+  }
+  if (!early) {
+    q0 = fetch_item(a, feed);
+    q1 = fetch_item(a, feed);
+    if (lane == 0 && q0 < a.n_items) issue_load(q0, 0);
+  }
   uint32_t it = 0;
   bool timed_out = false;
   while (q0 < a.n_items) {

@@ -59,6 +59,14 @@ def test_quantised_dispatch_bit_exact(case):
     assert comm.moe_status() == 0
     assert np.array_equal(wq.cpu().numpy(), want_q)
     assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+    # planning folded into the call (the kernel starts behind the planner): the same bytes
+    wq2 = torch.full((R * C, H), 0xAB, dtype=torch.uint8, device=dev)
+    sc2 = torch.full((R * C,), -1.0, dtype=torch.float32, device=dev)
+    for _ in range(2):
+        comm.moe_plan_dispatch_quant(sch, inp.topk_idx.to(dev), Xd, wq2, sc2, C, T, rts)
+    assert comm.moe_status() == 0
+    assert np.array_equal(wq2.cpu().numpy(), want_q)
+    assert np.array_equal(sc2.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
     if sch == DECODE:                                 # the launch also records delta, like moe_dispatch
         assert np.array_equal(comm.moe_plan_view()["small_off"].cpu().numpy(), p.s)
     # a consumer's view: dequantised rows are within the format's error of the bf16 rows
