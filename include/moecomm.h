@@ -102,8 +102,10 @@ moe_status_t moe_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* to
  *   logits    DEVICE [T,E] fp32            topk_idx  DEVICE [T,K] int32, out
  *                                          topk_w    DEVICE [T,K] fp32, out
  * moe_gate_topk is the stand-alone kernel (no context).  moe_gate_plan is the gate followed by
- * moe_plan on the indexes it wrote, enqueued back to back (a variant that gated inside the
- * one-CTA-per-rank planner measured slower: gating is instruction-bound and wants every SM).
+ * moe_plan on the indexes it wrote, enqueued back to back and chained (see MOE_OPT_OVERLAP): the planner
+ * is scheduled while the gate kernel runs and reads the indexes once that kernel has completed.  (A
+ * variant that gated inside the one-CTA-per-rank planner measured slower: gating is instruction-bound
+ * and wants every SM.)
  * topk_idx must stay valid like moe_plan's input. */
 moe_status_t moe_gate_topk(const float* logits /*DEVICE*/, int32_t T, int32_t E, int32_t K,
                            int32_t* topk_idx /*DEVICE*/, float* topk_w /*DEVICE*/, void* stream);
