@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_gate_topk.restype = ctypes.c_int
         L.oracle_expert_ranges.argtypes = [i32, i32, i64, i32, p, p, p]
         L.oracle_expert_ranges.restype = ctypes.c_int
+        L.oracle_expert_tiles.argtypes = [i32, i32, i64, i32, i32, p, i64, p, p, p, p]
+        L.oracle_expert_tiles.restype = ctypes.c_int
         L.oracle_dispatch_quant.argtypes = [p, i32, i32, i32, p, p, p, i32]
         L.oracle_dispatch_quant.restype = ctypes.c_int
         L.oracle_float_to_e4m3.argtypes = [ctypes.c_float]
@@ -148,6 +150,18 @@ def expert_ranges(E: int, R: int, C: int, n_exp, align: int = 1):
     count = np.full((E,), -1, np.int32)
     st = lib().oracle_expert_ranges(E, R, int(C), int(align), _ptr(n_exp), _ptr(start), _ptr(count))
     return st, start, count
+
+
+def expert_tiles(E: int, R: int, C: int, n_exp, tile_rows: int, max_tiles: int, align: int = 1):
+    """Tiles of at most tile_rows rows over every expert's run, in window order."""
+    n_exp = _c(n_exp, np.int32)
+    tile_expert = np.full((max_tiles,), -1, np.int32)
+    tile_row = np.full((max_tiles,), -1, np.int64)
+    tile_valid = np.full((max_tiles,), -1, np.int32)
+    n_tiles = np.zeros((1,), np.int64)
+    st = lib().oracle_expert_tiles(E, R, int(C), int(align), int(tile_rows), _ptr(n_exp), int(max_tiles),
+                                   _ptr(tile_expert), _ptr(tile_row), _ptr(tile_valid), _ptr(n_tiles))
+    return st, tile_expert, tile_row, tile_valid, int(n_tiles[0])
 
 
 def dispatch(X_u16, slots_, windows_u16, n_threads: int = 1) -> int:

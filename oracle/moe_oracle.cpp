@@ -253,6 +253,30 @@ int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, int32_t align, const i
   return ORACLE_OK;
 }
 
+int oracle_expert_tiles(int32_t E, int32_t R, int64_t C, int32_t align, int32_t tile_rows, const int32_t* n_exp,
+                        int64_t max_tiles, int32_t* tile_expert, int64_t* tile_row, int32_t* tile_valid,
+                        int64_t* n_tiles) {
+  if (E < 1 || R < 1 || E % R != 0 || C < 0 || align < 1 || tile_rows < 1 || max_tiles < 0) return ORACLE_ERR_INVALID_ARG;
+  const int32_t E_r = E / R;
+  int64_t k = 0;
+  for (int32_t d = 0; d < R; ++d) {
+    int64_t local = 0;   // row inside window d where the current expert's run starts
+    for (int32_t e = d * E_r; e < (d + 1) * E_r; ++e) {
+      for (int32_t r0 = 0; r0 < n_exp[e]; r0 += tile_rows) {   // the expert's run, tile_rows at a time
+        if (k < max_tiles) {
+          tile_expert[k] = e;
+          tile_row[k] = (int64_t)d * C + local + r0;
+          tile_valid[k] = n_exp[e] - r0 < tile_rows ? n_exp[e] - r0 : tile_rows;
+        }
+        ++k;
+      }
+      local = round_up_rows(local + n_exp[e], align);
+    }
+  }
+  *n_tiles = k;
+  return ORACLE_OK;
+}
+
 int oracle_dispatch(const uint16_t* X, int32_t T, int32_t H, int32_t K,
                     const int64_t* slots, uint16_t* windows, int32_t n_threads) {
   if (T < 0 || H < 1 || K < 1) return ORACLE_ERR_INVALID_ARG;

@@ -87,6 +87,15 @@ int oracle_slots(const int32_t* topk_idx, int32_t T, int32_t K, int32_t E, int32
 int oracle_expert_ranges(int32_t E, int32_t R, int64_t C, int32_t align, const int32_t* n_exp,
                          int64_t* row_start, int32_t* row_count);
 
+/* The same runs cut into tiles of at most tile_rows rows, in window order (rank, expert, position in the
+ * run): the work list of a grouped GEMM that reads the windows in place.  Tile k belongs to expert
+ * tile_expert[k], starts at window row tile_row[k] and holds tile_valid[k] rows (only the last tile of an
+ * expert can be short; an expert without rows has no tile).  At most max_tiles entries are written;
+ * *n_tiles is the number of tiles there are.  Consumer-side convenience, no counterpart in the paper. */
+int oracle_expert_tiles(int32_t E, int32_t R, int64_t C, int32_t align, int32_t tile_rows, const int32_t* n_exp,
+                        int64_t max_tiles, int32_t* tile_expert, int64_t* tile_row, int32_t* tile_valid,
+                        int64_t* n_tiles);
+
 /* Dispatch (Algorithm 1, first loop): copy row X[t,:] to window row slot[t,j]
  * for every branch.  Rows no branch maps to are left as the caller set them.
  * n_threads > 1 splits the token range over std::thread workers (same result). */

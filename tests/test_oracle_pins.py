@@ -664,3 +664,35 @@ def test_brute_force_all_routings_tiny_aligned():
                 assert p.o[e, r] == start + lower
         for d in range(R):
             assert p.n_recv[d] == sum(-(-count[e] // A) * A for e in range(d * E_r, (d + 1) * E_r))
+
+
+@pytest.mark.parametrize("align,tile_rows", [(1, 4), (8, 8), (16, 5), (1, 1000)])
+def test_expert_tiles_against_numpy(align, tile_rows):
+    """The tile list covers every expert's run exactly once, in window order, with only the last tile of an
+    expert short; its length is the sum of ceil(n_exp / tile_rows) (numpy)."""
+    rng = np.random.default_rng(321 + align + tile_rows)
+    T, K, E, R = 300, 4, 12, 3
+    idx, rts = random_case(rng, T, K, E, R, replace=True)
+    idx[idx == 5] = 4                                         # expert 5 receives nothing: it has no tile
+    p = oracle.plan(idx, E, R, rts, align=align)
+    C = int(p.n_recv.max()) + 3
+    _, e_start, e_count = oracle.expert_ranges(E, R, C, p.n_exp, align=align)
+    want_n = int(np.sum(-(-p.n_exp.astype(np.int64) // tile_rows)))
+    st, t_e, t_row, t_valid, n = oracle.expert_tiles(E, R, C, p.n_exp, tile_rows, want_n + 5, align=align)
+    assert st == oracle.OK and n == want_n
+    assert (t_e[n:] == -1).all() and (t_row[n:] == -1).all()                      # nothing beyond the list
+    assert (np.diff(t_e[:n]) >= 0).all() and 5 not in t_e[:n]                    # window order = expert order
+    covered = np.zeros(R * C, np.int32)
+    for k in range(n):
+        e = t_e[k]
+        off = t_row[k] - e_start[e]
+        assert off % tile_rows == 0 and 0 <= off < e_count[e]
+        assert t_valid[k] == min(tile_rows, e_count[e] - off)
+        covered[t_row[k]:t_row[k] + t_valid[k]] += 1
+    _, slots = oracle.slots(idx, E, R, p, C, rts)
+    used = np.zeros(R * C, np.int32)
+    used[slots.reshape(-1)] = 1
+    assert np.array_equal(covered, used)                                          # every received row in exactly one tile
+    # a short buffer: the count is still the full one, entries beyond the buffer are not written
+    st, t_e2, _, _, n2 = oracle.expert_tiles(E, R, C, p.n_exp, tile_rows, 3, align=align)
+    assert n2 == want_n and np.array_equal(t_e2, t_e[:3])
