@@ -235,6 +235,20 @@ moe_status_t moe_slots(moe_ctx_t* ctx, int64_t capacity_rows, int32_t* slots /*D
 moe_status_t moe_expert_ranges(moe_ctx_t* ctx, int64_t capacity_rows, int64_t* row_start /*DEVICE*/,
                                int32_t* row_count /*DEVICE*/, void* stream);
 
+/* The same runs cut into tiles of at most tile_rows rows, in window order (rank, expert, position in the
+ * run): the work list of a grouped GEMM that reads the windows in place.  (Consumer-side convenience, no
+ * counterpart in the paper.)  With MOE_OPT_EXPERT_ALIGN equal to tile_rows every tile also starts on a
+ * multiple of tile_rows inside its window.
+ *   tile_expert DEVICE [max_tiles] int32   expert of tile k
+ *   tile_row    DEVICE [max_tiles] int64   first window row of tile k
+ *   tile_valid  DEVICE [max_tiles] int32   rows of tile k that hold tokens (only an expert's last tile is short)
+ *   n_tiles     DEVICE [1] int32           number of tiles there are = sum over experts of ceil(n_exp / tile_rows);
+ *                                          entries beyond max_tiles are not written
+ * An upper bound for max_tiles that needs no device read: T*K / tile_rows + E. */
+moe_status_t moe_expert_tiles(moe_ctx_t* ctx, int64_t capacity_rows, int32_t tile_rows, int64_t max_tiles,
+                              int32_t* tile_expert /*DEVICE*/, int64_t* tile_row /*DEVICE*/,
+                              int32_t* tile_valid /*DEVICE*/, int32_t* n_tiles /*DEVICE*/, void* stream);
+
 /* One whole layer call from HOST buffers, enqueued on `stream`:
  * host->device copies of topk_idx, topk_w; plan; then, in sixteen token chunks, host->device copy
  * of the chunk of x (upload stream), dispatch and combine reading the dispatched windows (identity

@@ -891,6 +891,18 @@ moe_status_t moe_expert_ranges(moe_ctx_t* ctx, int64_t capacity_rows, int64_t* r
   return launch_ok(ctx);
 }
 
+moe_status_t moe_expert_tiles(moe_ctx_t* ctx, int64_t capacity_rows, int32_t tile_rows, int64_t max_tiles,
+                              int32_t* tile_expert, int64_t* tile_row, int32_t* tile_valid, int32_t* n_tiles,
+                              void* stream) {
+  if (ctx == nullptr || capacity_rows < 0 || tile_rows < 1 || max_tiles < 0 || n_tiles == nullptr) return MOE_ERR_INVALID_ARG;
+  if (max_tiles > 0 && (tile_expert == nullptr || tile_row == nullptr || tile_valid == nullptr)) return MOE_ERR_INVALID_ARG;
+  if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  const int E = ctx->shape.E;
+  expert_tiles_kernel<<<1, 1024, (2 * E + 1 + 33) * (int)sizeof(int32_t), static_cast<cudaStream_t>(stream)>>>(
+      ctx->o, ctx->n_exp, E, ctx->shape.R, capacity_rows, tile_rows, max_tiles, tile_expert, tile_row, tile_valid, n_tiles);
+  return launch_ok(ctx);
+}
+
 moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T, const int32_t* rank_tok_start,
                               const void* x_host, const int32_t* topk_idx_host, const float* topk_w_host,
                               void* x_dev, int32_t* topk_idx_dev, float* topk_w_dev, void* windows_dev,

@@ -502,4 +502,35 @@ plan_finalize_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant
   }
 }
 
+// Tile list over the experts' runs (work list of a grouped GEMM that reads the windows in place): tile k is
+// (expert, first window row, valid rows <= tile_rows), in window order.  ONE CTA; shared memory: tiles
+// per expert [E], their exclusive prefix [E + 1], warp sums [33].
+__global__ void __launch_bounds__(1024)
+expert_tiles_kernel(const int32_t* __restrict__ large_off, const int32_t* __restrict__ n_exp, int32_t E, int32_t R,
+                    int64_t C, int32_t tile_rows, int64_t max_tiles, int32_t* __restrict__ tile_expert,
+                    int64_t* __restrict__ tile_row, int32_t* __restrict__ tile_valid, int32_t* __restrict__ n_tiles) {
+  extern __shared__ int32_t tile_sm[];
+  int32_t* nt = tile_sm;
+  int32_t* pre = tile_sm + E;
+  int32_t* warp_sums = pre + E + 1;
+  const int E_r = E / R;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) nt[e] = (n_exp[e] + tile_rows - 1) / tile_rows;
+  __syncthreads();
+  block_exclusive_scan(nt, pre, E, warp_sums);   // window order is expert order
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    const int64_t start = (int64_t)(e / E_r) * C + large_off[(size_t)e * R];   // the block of source rank 0 starts the run
+    const int32_t count = n_exp[e];
+    for (int32_t i = 0; i < nt[e]; ++i) {
+      const int64_t k = (int64_t)pre[e] + i;
+      if (k < max_tiles) {
+        tile_expert[k] = e;
+        tile_row[k] = start + (int64_t)i * tile_rows;
+        tile_valid[k] = min(tile_rows, count - i * tile_rows);
+      }
+    }
+  }
+  if (threadIdx.x == 0) *n_tiles = pre[E];
+}
+
 }  // namespace moe

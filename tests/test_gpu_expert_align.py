@@ -78,3 +78,38 @@ def test_alignment_changes_need_a_new_plan_and_capacity_counts_padding():
     assert np.array_equal(comm.moe_plan_view()["n_recv"].cpu().numpy(), padded.n_recv)
     assert np.array_equal(Y.cpu().view(torch.int16).numpy().view(np.uint16), synth.bf16_to_u16(inp.X))
     comm.close()
+
+
+@pytest.mark.parametrize("align,tile_rows", [(1, 16), (128, 128), (8, 5), (1, 100000)])
+@pytest.mark.parametrize("schedule", [PREFILL, DECODE])
+def test_expert_tile_list_matches_the_oracle(schedule, align, tile_rows):
+    dev = torch.device("cuda:0")
+    for name, T, H, E, R, K, routing, per in CASES[:5]:
+        wl = Workload(name, T, H, E, R, K, schedule, routing, "identity", 5200 + T, rank_tokens=per)
+        inp = synth.make_inputs(wl)
+        p = oracle.plan(inp.topk_idx.numpy(), E, R, inp.rank_tok_start, align=align)
+        C = int(p.n_recv.max()) + 1
+        bound = T * K // tile_rows + E
+        st, w_e, w_row, w_valid, w_n = oracle.expert_tiles(E, R, C, p.n_exp, tile_rows, bound, align=align)
+        assert st == oracle.OK and w_n <= bound
+        comm = binding.MoeComm(max(T, 1), H, E, R, K, dev)
+        comm.moe_set_option(binding.MOE_OPT_EXPERT_ALIGN, align)
+        rts = None if per is None else inp.rank_tok_start
+        comm.moe_plan(schedule, inp.topk_idx.to(dev), T, rts)
+        t_e = torch.full((bound,), -1, dtype=torch.int32, device=dev)
+        t_row = torch.full((bound,), -1, dtype=torch.int64, device=dev)
+        t_valid = torch.full((bound,), -1, dtype=torch.int32, device=dev)
+        n = torch.full((1,), -1, dtype=torch.int32, device=dev)
+        comm.moe_expert_tiles(C, tile_rows, t_e, t_row, t_valid, n)
+        assert comm.moe_status() == 0
+        assert int(n.item()) == w_n
+        assert np.array_equal(t_e.cpu().numpy(), w_e) and np.array_equal(t_row.cpu().numpy(), w_row)
+        assert np.array_equal(t_valid.cpu().numpy(), w_valid)
+        if align == tile_rows:
+            assert ((t_row[:w_n] % C) % tile_rows == 0).all()          # tiles start on tile boundaries of their window
+        # a buffer that is too short: the count is the full one, nothing is written beyond the buffer
+        if w_n > 2:
+            short = torch.full((2,), -1, dtype=torch.int32, device=dev)
+            comm.moe_expert_tiles(C, tile_rows, short, t_row[:2].clone(), t_valid[:2].clone(), n)
+            assert comm.moe_status() == 0 and int(n.item()) == w_n and np.array_equal(short.cpu().numpy(), w_e[:2])
+        comm.close()
