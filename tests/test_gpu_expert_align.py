@@ -113,3 +113,42 @@ def test_expert_tile_list_matches_the_oracle(schedule, align, tile_rows):
             comm.moe_expert_tiles(C, tile_rows, short, t_row[:2].clone(), t_valid[:2].clone(), n)
             assert comm.moe_status() == 0 and int(n.item()) == w_n and np.array_equal(short.cpu().numpy(), w_e[:2])
         comm.close()
+
+
+def test_an_expert_op_driven_by_the_tile_list_gives_the_oracle_result():
+    """End to end with the expert side consuming the windows in place through the tile list alone
+    (no routing indexes, no counts): dispatch, scale every tile's rows by its expert's factor, combine."""
+    dev = torch.device("cuda:0")
+    tile = 64
+    wl = Workload("tiles_e2e", 3000, 512, 32, 4, 6, DECODE, "uniform", "scale", 5300, rank_tokens=(900, 0, 1300, 800))
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R, inp.rank_tok_start, align=tile)
+    C = int(p.n_recv.max())
+    want = harness.oracle_run(inp, C, align=tile)
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    comm.moe_set_option(binding.MOE_OPT_EXPERT_ALIGN, tile)
+    idx, w, X = inp.topk_idx.to(dev), inp.topk_w.to(dev), inp.X.to(dev)
+    win = torch.from_numpy(np.full((wl.R * C, wl.H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    comm.moe_plan_dispatch(wl.schedule, idx, X, win, C, wl.T, inp.rank_tok_start)
+    bound = wl.T * wl.K // tile + wl.E
+    t_e = torch.empty(bound, dtype=torch.int32, device=dev)
+    t_row = torch.empty(bound, dtype=torch.int64, device=dev)
+    t_valid = torch.empty(bound, dtype=torch.int32, device=dev)
+    n = torch.empty(1, dtype=torch.int32, device=dev)
+    comm.moe_expert_tiles(C, tile, t_e, t_row, t_valid, n)
+    assert comm.moe_status() == 0
+    k = int(n.item())
+    assert np.array_equal(win.cpu().view(torch.int16).numpy().view(np.uint16), want.windows)
+    # the stand-in expert op, tile by tile (harness code): rows [row, row + valid) of a tile belong to one expert
+    valid = t_valid[:k].long()
+    first = torch.repeat_interleave(t_row[:k], valid)
+    within = torch.arange(int(valid.sum()), device=dev) - torch.repeat_interleave(torch.cumsum(valid, 0) - valid, valid)
+    rows = first + within
+    factor = torch.repeat_interleave(inp.scale.to(dev)[t_e[:k].long()], valid)
+    assert rows.numel() == wl.T * wl.K and (t_row[:k] % C % tile == 0).all()
+    win[rows] = win[rows] * factor[:, None]
+    Y = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
+    comm.moe_combine(win, C, w, Y)
+    assert comm.moe_status() == 0
+    assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
+    comm.close()
