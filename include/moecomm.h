@@ -222,6 +222,12 @@ moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/, const 
                                 int64_t capacity_rows, void* stream);
 moe_status_t moe_combine_peers(moe_ctx_t* ctx, const void* const* window_bases /*DEVICE*/, int64_t capacity_rows,
                                const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
+/* Row-wise quantised dispatch in the same decomposition: code window and scale tensor of rank d start at
+ * window_q_bases[d] (uint8 [capacity_rows, H]) and scale_bases[d] (fp32 [capacity_rows]); both tables are
+ * DEVICE arrays of R device pointers. */
+moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/,
+                                      const void* const* window_q_bases /*DEVICE*/,
+                                      float* const* scale_bases /*DEVICE*/, int64_t capacity_rows, void* stream);
 
 /* Materialises slot(t,j) into caller memory (parity checks, expert-side
  * consumers).  slots DEVICE [T,K] int32; needs R * capacity_rows < 2^31. */

@@ -26,7 +26,7 @@ EXPORTS = [
     "moe_combine", "moe_slots", "moe_forward_host", "moe_status", "moe_status_string", "moe_launch_count",
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
     "moe_gate_topk", "moe_gate_plan", "moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers",
-    "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant", "moe_expert_tiles",
+    "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant", "moe_expert_tiles", "moe_dispatch_quant_peers",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
@@ -92,6 +92,8 @@ def load() -> ctypes.CDLL:
     L.moe_expert_ranges.restype = ctypes.c_int
     L.moe_expert_tiles.argtypes = [vp, i64, i32, i64, vp, vp, vp, vp, vp]
     L.moe_expert_tiles.restype = ctypes.c_int
+    L.moe_dispatch_quant_peers.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.moe_dispatch_quant_peers.restype = ctypes.c_int
     L.moe_dispatch_quant.argtypes = [vp, vp, vp, vp, i64, vp]
     L.moe_dispatch_quant.restype = ctypes.c_int
     L.moe_slots.argtypes = [vp, i64, vp, vp]
@@ -370,6 +372,17 @@ class MoeComm:
                                              _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_dispatch_quant")
+        return rc
+
+    def moe_dispatch_quant_peers(self, x: torch.Tensor, window_q_bases: torch.Tensor, scale_bases: torch.Tensor,
+                                 capacity_rows: int, stream=None, check: bool = True) -> int:
+        with self._on_device():
+            rc = self.lib.moe_dispatch_quant_peers(self._h, _dev_ptr(x, torch.bfloat16),
+                                                   _dev_ptr(window_q_bases, torch.int64),
+                                                   _dev_ptr(scale_bases, torch.int64), int(capacity_rows),
+                                                   _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_quant_peers")
         return rc
 
     def moe_expert_tiles(self, capacity_rows: int, tile_rows: int, tile_expert: torch.Tensor, tile_row: torch.Tensor,

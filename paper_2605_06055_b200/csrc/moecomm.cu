@@ -142,6 +142,7 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   a.tail_granule = 1;
   a.tail_items_per_row = 1;
   a.win_base = nullptr;
+  a.scale_base = nullptr;
   a.prefetch_meta = 0;
   a.static_first = 0;
   a.pdl = 0;
@@ -714,17 +715,21 @@ moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x, const void* const
 }
 
 static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windows_q, float* scales,
-                                        int64_t capacity_rows, void* stream, bool behind_plan) {
+                                        int64_t capacity_rows, void* stream, bool behind_plan,
+                                        const void* const* q_bases = nullptr, float* const* s_bases = nullptr) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
+  const bool peers = q_bases != nullptr;   // one code window and one scale tensor per rank, addressed through tables
   const int H = ctx->shape.H;
   if (H % 16 != 0 || H * 2 > QUANT_MAX_ROW_BYTES) return MOE_ERR_INVALID_ARG;
-  if (capacity_rows < 0 || (ctx->T > 0 && (x == nullptr || windows_q == nullptr || scales == nullptr)))
-    return MOE_ERR_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(windows_q) || (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)
+  if (capacity_rows < 0 || (peers && s_bases == nullptr)) return MOE_ERR_INVALID_ARG;
+  if (ctx->T > 0 && (x == nullptr || (!peers && (windows_q == nullptr || scales == nullptr)))) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || (!peers && (!aligned16(windows_q) || (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)))
     return MOE_ERR_INVALID_ARG;
   RowArgs a = row_args(ctx, capacity_rows, true);
   a.topk_idx = ctx->topk_idx;
+  a.win_base = reinterpret_cast<const unsigned char* const*>(q_bases);
+  a.scale_base = s_bases;
   // One work item per token: the whole row is needed for its scale.
   const int upr = (a.H16 + 31) / 32;
   const int stage = (H * 2 + 127) / 128 * 128;
@@ -758,6 +763,12 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
 moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x, void* windows_q, float* scales, int64_t capacity_rows,
                                 void* stream) {
   return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, false);
+}
+
+moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x, const void* const* window_q_bases,
+                                      float* const* scale_bases, int64_t capacity_rows, void* stream) {
+  if (window_q_bases == nullptr || scale_bases == nullptr) return MOE_ERR_INVALID_ARG;
+  return dispatch_quant_impl(ctx, x, nullptr, nullptr, capacity_rows, stream, false, window_q_bases, scale_bases);
 }
 
 moe_status_t moe_plan_dispatch_quant(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
@@ -1159,6 +1170,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.tail_granule = 1;
   a.tail_items_per_row = 1;
   a.win_base = nullptr;
+  a.scale_base = nullptr;
   a.prefetch_meta = 0;
   a.static_first = 0;
   a.t_begin = 0;

@@ -168,9 +168,12 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
 
     for (int j = 0; j < a.K; ++j) {
       const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-      if (lane == 0 && row >= 0) bulk_store(windows_q + (size_t)row * code_bytes, in, code_bytes, evict_first);
+      if (lane == 0 && row >= 0) bulk_store(window_row(a, windows_q, row, code_bytes), in, code_bytes, evict_first);
     }
-    if (lane < a.K && slot >= 0) scales[slot] = scale;
+    if (lane < a.K && slot >= 0) {
+      if (a.scale_base == nullptr) scales[slot] = scale;
+      else a.scale_base[slot / a.C][slot % a.C] = scale;   // one scale tensor per rank, same row order as its window
+    }
     if (lane == 0) bulk_commit();   // one group per iteration
     q0 = q1;
     q1 = q2;

@@ -40,6 +40,7 @@ struct RowArgs {
   // Multi-rank use: window segment d starts at win_base[d] (device array of R device pointers, e.g. peer
   // mappings of every rank's window); nullptr = one allocation of R consecutive segments of C rows.
   const unsigned char* const* win_base;
+  float* const* scale_base;  // quantised dispatch, multi-rank use: scales of segment d start at scale_base[d]; else nullptr
   int32_t static_first;      // work items per warp that are fixed (warp id + k * warps) before the counter is used
   int32_t prefetch_meta;     // combine: fetch the next item's branch metadata while reducing the current one
   int32_t pdl;               // dispatch launched behind the planner with programmatic stream serialization

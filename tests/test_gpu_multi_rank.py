@@ -78,3 +78,40 @@ def test_per_rank_contexts_and_separate_windows_reproduce_the_global_result(case
     assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
     for c in comms:
         c.close()
+
+
+@pytest.mark.parametrize("case", CASES[:3], ids=[c[0] for c in CASES[:3]])
+def test_quantised_dispatch_into_per_rank_windows(case):
+    """The quantising dispatch in the multi-rank decomposition: every rank quantises its own tokens and
+    writes codes and scales into every rank's own allocations; the union equals the oracle's global result."""
+    name, T, H, E, R, K, sch, routing, per = case
+    dev = torch.device("cuda:0")
+    wl = Workload(name, T, H, E, R, K, sch, routing, "identity", 7100 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    rts = inp.rank_tok_start
+    idx_np = inp.topk_idx.numpy()
+    p = oracle.plan(idx_np, E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(idx_np, E, R, p, C, rts)
+    want_q = np.full((R * C, H), 0xAB, np.uint8)
+    want_s = np.full((R * C,), -1.0, np.float32)
+    assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), slots, want_q, want_s, 4) == oracle.OK
+
+    idx, X = inp.topk_idx.to(dev), inp.X.to(dev)
+    comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
+    counts = torch.zeros((R, E), dtype=torch.int32, device=dev)
+    for r, c in enumerate(comms):
+        c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, counts[r])
+    for c in comms:
+        c.moe_notify(counts)
+    wq = [torch.full((C, H), 0xAB, dtype=torch.uint8, device=dev) for _ in range(R)]
+    sc = [torch.full((C,), -1.0, dtype=torch.float32, device=dev) for _ in range(R)]
+    q_bases = torch.tensor([t.data_ptr() for t in wq], dtype=torch.int64, device=dev)
+    s_bases = torch.tensor([t.data_ptr() for t in sc], dtype=torch.int64, device=dev)
+    for r, c in enumerate(comms):
+        c.moe_dispatch_quant_peers(X[rts[r]:rts[r + 1]].contiguous(), q_bases, s_bases, C)
+        assert c.moe_status() == 0
+    assert np.array_equal(torch.cat(wq).cpu().numpy(), want_q)
+    assert np.array_equal(torch.cat(sc).cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+    for c in comms:
+        c.close()
