@@ -62,6 +62,14 @@ class EpRank:
         torch.cuda.current_stream().synchronize()
         dist.barrier(self.group)                 # every rank's rows have landed before any expert reads its window
 
+    def dispatch_quant(self, x_local: torch.Tensor, window_q_bases: torch.Tensor, scale_bases: torch.Tensor,
+                       capacity_rows: int) -> None:
+        """Row-wise quantised dispatch: e4m3 codes into every rank's code window, one fp32 scale per row into
+        every rank's scale tensor (tables of R device addresses each)."""
+        self.comm.moe_dispatch_quant_peers(x_local, window_q_bases, scale_bases, capacity_rows)
+        torch.cuda.current_stream().synchronize()
+        dist.barrier(self.group)
+
     def combine(self, window_bases: torch.Tensor, capacity_rows: int, topk_w_local: torch.Tensor,
                 y_local: torch.Tensor) -> None:
         dist.barrier(self.group)                 # every expert has written its outputs
