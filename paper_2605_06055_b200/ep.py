@@ -8,8 +8,9 @@ module only exchanges the R x E count matrix with torch.distributed and keeps th
 The windows of the other ranks must be mapped into this process (a table of R device addresses):
 `symmetric_windows` obtains them from torch's symmetric memory where that is available.
 
-Only the single-GPU form (every rank a context of one process, separate window allocations) is
-exercised on a GPU by the test suite; the count exchange is tested with two gloo ranks on CPU.
+The test suite exercises this on ONE GPU: every rank a context of one process with separate window
+allocations, and two ranks as two processes whose windows are mapped into each other over CUDA IPC
+(counts over a gloo group).  The count exchange is also tested with two gloo ranks on CPU.
 """
 from __future__ import annotations
 
@@ -25,9 +26,12 @@ def all_gather_counts(counts_row: torch.Tensor, group=None) -> torch.Tensor:
     """Prefill Notify's metadata exchange: every rank contributes its row [E] of the count matrix and
     receives the whole matrix [R, E] (row r from rank r)."""
     world = dist.get_world_size(group)
-    flat = torch.empty(world * counts_row.numel(), dtype=counts_row.dtype, device=counts_row.device)
-    dist.all_gather_into_tensor(flat, counts_row.contiguous().view(-1), group=group)
-    return flat.view(world, counts_row.numel())
+    staged = counts_row.is_cuda and dist.get_backend(group) == "gloo"     # gloo moves host tensors only
+    src = counts_row.cpu() if staged else counts_row
+    flat = torch.empty(world * src.numel(), dtype=src.dtype, device=src.device)
+    dist.all_gather_into_tensor(flat, src.contiguous().view(-1), group=group)
+    out = flat.view(world, src.numel())
+    return out.to(counts_row.device) if staged else out
 
 
 def symmetric_windows(capacity_rows: int, H: int, device, group=None):

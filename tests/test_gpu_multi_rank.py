@@ -4,6 +4,8 @@ token slice and its own window allocation, as R processes on R GPUs would have; 
 after the other (they never wait on one another).  The union of the windows and the outputs must be
 bit-identical to the oracle's single global result.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -115,3 +117,78 @@ def test_quantised_dispatch_into_per_rank_windows(case):
     assert np.array_equal(torch.cat(sc).cpu().numpy().view(np.uint32), want_s.view(np.uint32))
     for c in comms:
         c.close()
+
+
+# ------------------------------------------------------------------ two processes, windows shared over CUDA IPC
+def _ipc_rank(rank, world, port, q_to, results):
+    """One expert-parallel rank as its own process on the one GPU: its window lives in its own
+    allocation, the other rank's window is mapped in over CUDA IPC, counts travel over a gloo group,
+    phases are ordered by host barriers (no kernel waits on another process's kernel)."""
+    import os
+    import torch.distributed as dist
+    from paper_2605_06055_b200 import ep
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    try:
+        dev = torch.device("cuda:0")
+        torch.cuda.set_device(dev)
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        T, H, E, K = 600, 512, 16, 4
+        wl = Workload("ipc", T, H, E, world, K, DECODE, "uniform", "identity", 7300, rank_tokens=(250, 350))
+        inp = synth.make_inputs(wl)
+        rts = inp.rank_tok_start
+        lo, hi = int(rts[rank]), int(rts[rank + 1])
+        me = ep.EpRank(hi - lo, H, E, K, dev)
+        me.plan(DECODE, inp.topk_idx[lo:hi].contiguous().to(dev))
+        C = int(me.comm.moe_plan_view()["n_recv"].max().item()) + 1
+        mine = torch.from_numpy(np.full((C, H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+        q_to[1 - rank].put(mine)                       # the other process maps this allocation (CUDA IPC)
+        other = q_to[rank].get(timeout=60)
+        wins = [mine, other] if rank == 0 else [other, mine]
+        bases = torch.tensor([w.data_ptr() for w in wins], dtype=torch.int64, device=dev)
+        me.dispatch(inp.X[lo:hi].contiguous().to(dev), bases, C)
+        y = torch.empty((hi - lo, H), dtype=torch.bfloat16, device=dev)
+        me.combine(bases, C, inp.topk_w[lo:hi].contiguous().to(dev), y)
+        st = me.status()
+        dist.barrier()                                 # nobody frees a window another rank may still read
+        results[rank] = ("ok", st, C, mine.cpu().view(torch.int16).numpy().view(np.uint16).copy(),
+                         y.cpu().view(torch.int16).numpy().view(np.uint16).copy())
+        dist.barrier()
+        dist.destroy_process_group()
+    except Exception as exc:                           # reported to the parent, which decides between skip and fail
+        results[rank] = ("error", repr(exc))
+
+
+def test_two_processes_exchange_rows_through_ipc_mapped_windows():
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    world = 2
+    with ctx.Manager() as m:
+        results = m.dict()
+        q_to = [ctx.Queue(), ctx.Queue()]
+        procs = [ctx.Process(target=_ipc_rank, args=(r, world, 35000 + os.getpid() % 2000, q_to, results))
+                 for r in range(world)]
+        for p_ in procs:
+            p_.start()
+        for p_ in procs:
+            p_.join(timeout=180)
+        alive = [p_ for p_ in procs if p_.is_alive()]
+        for p_ in alive:
+            p_.terminate()
+        assert not alive, "a rank did not finish"
+        res = dict(results)
+    errors = [v for v in res.values() if v[0] == "error"]
+    if errors and any("ipc" in e[1].lower() or "not supported" in e[1].lower() for e in errors):
+        pytest.skip("CUDA IPC is not available here: " + errors[0][1])
+    assert not errors and len(res) == world, res
+    T, H, E, K = 600, 512, 16, 4
+    wl = Workload("ipc", T, H, E, world, K, DECODE, "uniform", "identity", 7300, rank_tokens=(250, 350))
+    inp = synth.make_inputs(wl)
+    C = res[0][2]
+    assert res[1][2] == C
+    want = harness.oracle_run(inp, C)
+    rts = inp.rank_tok_start
+    for r in range(world):
+        _, st, _, win, y = res[r]
+        assert st == 0
+        assert np.array_equal(win, want.windows[r * C:(r + 1) * C])            # rows from both processes, bit-exact
+        assert harness.max_ulp_diff(y, want.Y[int(rts[r]):int(rts[r + 1])]) <= 1
