@@ -292,7 +292,8 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   // 14 KB rows, K=8: 4 warps 661.5 us, 3 warps 659.5 us, 2 warps 656.4 us, 1 warp 816 us; at 8 KB rows, K=2:
   // 8 warps 252 us, 4 warps 272 us; at 4 KB rows, K=8: 8 warps 381 us, 2 warps 668 us.  Small jobs keep every
   // warp: there the number of rows in flight decides (decode step 102.7 us with 4 warps, 115 us with 2).
-  if (BULK_STREAMS_TARGET > 0 && (int64_t)a.t_count >= (int64_t)16 * grid * warps) {
+  // "Large" = four rows or more per warp (T=4096 at 14 KB rows: 95.2 -> 93.6 us; T=2048 is slower with the rule).
+  if (BULK_STREAMS_TARGET > 0 && (int64_t)a.t_count >= (int64_t)4 * grid * warps) {
     int want = (BULK_STREAMS_TARGET + grid * ctx->shape.K / 2) / (grid * ctx->shape.K);
     const int floor_warps = (56 * 1024 + 2 * g_max * 512 - 1) / (2 * g_max * 512);
     if (want < floor_warps) want = floor_warps;
