@@ -43,12 +43,12 @@ L2_BYTES = 126 << 20
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; keyed by (kernel, workload).  Absent = not captured.
 NCU_TRAFFIC_BYTES = {
-    # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture at T=8192 (1049.7 MB / 999.4 MB per launch),
+    # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture at T=8192 (1049.7 MB / 998.8 MB per launch),
     # scaled by 4 for the full size: every token moves the same bytes
     ("combine_rows_kernel", "c3_prefill_dsv3"): 4 * 1049.7e6,
-    ("dispatch_bulk_kernel", "c3_prefill_dsv3"): 4 * 999.4e6,
+    ("dispatch_bulk_kernel", "c3_prefill_dsv3"): 4 * 998.8e6,
     ("combine_rows_kernel", "c3_prefill_dsv3_T8192"): 1049.7e6,
-    ("dispatch_bulk_kernel", "c3_prefill_dsv3_T8192"): 999.4e6,
+    ("dispatch_bulk_kernel", "c3_prefill_dsv3_T8192"): 998.8e6,
 }
 
 WORKLOADS = {
