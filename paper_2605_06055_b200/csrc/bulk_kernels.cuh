@@ -7,7 +7,10 @@
 // 14 KB row) into a stage, and when the stage's mbarrier completes, to store it
 // to the K destination rows.  One request covers the whole contiguous span, so
 // HBM sees long sequential bursts per row, and the number of bytes in flight is
-// set by shared memory (about 170 KB per SM), not by registers or warp count.
+// set by shared memory (up to about 170 KB per SM), not by registers.  How many
+// warps a CTA gets is the launcher's choice: as many rings as fit for small jobs,
+// for large ones only as many as keep about 2400 destination rows being written
+// at once across the device, which is what HBM serves best.
 //
 // Every wait is bounded in time: an mbarrier that does not complete within the
 // limit (2 s by default) raises MOE_ERR_TIMEOUT and the warp stops taking work;
