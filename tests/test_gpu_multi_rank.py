@@ -149,9 +149,21 @@ def _ipc_rank(rank, world, port, q_to, results):
         y = torch.empty((hi - lo, H), dtype=torch.bfloat16, device=dev)
         me.combine(bases, C, inp.topk_w[lo:hi].contiguous().to(dev), y)
         st = me.status()
+        # the quantising dispatch into per-process code windows and scale tensors, mapped the same way
+        my_q = torch.full((C, H), 0xAB, dtype=torch.uint8, device=dev)
+        my_s = torch.full((C,), -1.0, dtype=torch.float32, device=dev)
+        q_to[1 - rank].put((my_q, my_s))
+        other_q, other_s = q_to[rank].get(timeout=60)
+        qs = [my_q, other_q] if rank == 0 else [other_q, my_q]
+        ss = [my_s, other_s] if rank == 0 else [other_s, my_s]
+        q_bases = torch.tensor([t.data_ptr() for t in qs], dtype=torch.int64, device=dev)
+        s_bases = torch.tensor([t.data_ptr() for t in ss], dtype=torch.int64, device=dev)
+        me.dispatch_quant(inp.X[lo:hi].contiguous().to(dev), q_bases, s_bases, C)
+        st = st or me.status()
         dist.barrier()                                 # nobody frees a window another rank may still read
         results[rank] = ("ok", st, C, mine.cpu().view(torch.int16).numpy().view(np.uint16).copy(),
-                         y.cpu().view(torch.int16).numpy().view(np.uint16).copy())
+                         y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), my_q.cpu().numpy().copy(),
+                         my_s.cpu().numpy().copy())
         dist.barrier()
         dist.destroy_process_group()
     except Exception as exc:                           # reported to the parent, which decides between skip and fail
@@ -187,8 +199,13 @@ def test_two_processes_exchange_rows_through_ipc_mapped_windows():
     assert res[1][2] == C
     want = harness.oracle_run(inp, C)
     rts = inp.rank_tok_start
+    want_q = np.full((world * C, H), 0xAB, np.uint8)
+    want_s = np.full((world * C,), -1.0, np.float32)
+    assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 2) == oracle.OK
     for r in range(world):
-        _, st, _, win, y = res[r]
+        _, st, _, win, y, q, sc = res[r]
         assert st == 0
         assert np.array_equal(win, want.windows[r * C:(r + 1) * C])            # rows from both processes, bit-exact
         assert harness.max_ulp_diff(y, want.Y[int(rts[r]):int(rts[r + 1])]) <= 1
+        assert np.array_equal(q, want_q[r * C:(r + 1) * C])
+        assert np.array_equal(sc.view(np.uint32), want_s[r * C:(r + 1) * C].view(np.uint32))
