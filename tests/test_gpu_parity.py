@@ -423,3 +423,21 @@ def test_contexts_of_different_shapes_coexist():
         harness.assert_parity(g, harness.oracle_run(inp, C), PREFILL)
     for c in comms:
         c.close()
+
+
+def test_option_values_are_validated():
+    dev = torch.device("cuda:0")
+    comm = binding.MoeComm(64, 64, 8, 2, 2, dev)
+    bad = binding.MOE_ERR_INVALID_ARG
+    for opt, good, wrong in [(binding.MOE_OPT_DISPATCH_PATH, [0, 1, 2], [-1, 3]),
+                             (binding.MOE_OPT_GRANULE, [0, 1, 1 << 20], [-1, (1 << 20) + 1]),
+                             (binding.MOE_OPT_TEST_STARVE_WAIT_MS, [0], [-1, 10001]),
+                             (binding.MOE_OPT_OVERLAP, [0, 1], [-1, 2]),
+                             (binding.MOE_OPT_EXPERT_ALIGN, [1, 128, 4096], [0, -5, 4097]),
+                             (binding.MOE_OPT_CLUSTER_PLAN, [0, 1], [-1, 2])]:
+        for v in wrong:
+            assert comm.moe_set_option(opt, v, check=False) == bad, (opt, v)
+        for v in good:
+            assert comm.moe_set_option(opt, v, check=False) == binding.MOE_OK, (opt, v)
+    assert comm.moe_set_option(99, 0, check=False) == bad
+    comm.close()
