@@ -89,9 +89,11 @@ moe_status_t moe_destroy(moe_ctx_t* ctx);
  *   rank_tok_start  HOST   [R+1] int32, nondecreasing, [0]=0, [R]=T; NULL means
  *                   uniform T/R tokens per rank (T % R must be 0).  Read before
  *                   the call returns.
- * An index outside [0,E) sets the device status word to MOE_ERR_BAD_INDEX; the
- * offending branch is ignored by the counts and later calls write nothing
- * until moe_status() has cleared the word. */
+ * An index outside [0,E) sets the device status word to MOE_ERR_BAD_INDEX (the
+ * paper defines routing indexes in {0..E-1} only; there is no "dropped branch"
+ * value).  Calls enqueued behind such a plan write nothing, and when moe_status()
+ * reports the error it also discards the plan: dispatch / combine / slots then
+ * return MOE_ERR_NOT_PLANNED until a new plan has been made. */
 moe_status_t moe_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE*/,
                       int32_t T, const int32_t* rank_tok_start /*HOST*/, void* stream);
 
@@ -193,7 +195,8 @@ moe_status_t moe_plan_dispatch_quant(moe_ctx_t* ctx, moe_schedule_t schedule, co
 moe_status_t moe_combine(moe_ctx_t* ctx, const void* windows /*DEVICE*/, int64_t capacity_rows,
                          const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
 
-/* Token sub-ranges of a plan: the same as moe_dispatch / moe_combine for tokens t_begin <= t < t_end
+/* Token sub-ranges of a plan (a convenience of this library; the paper has no counterpart -- its kernels
+ * take a whole batch): the same as moe_dispatch / moe_combine for tokens t_begin <= t < t_end
  * only (x and y are still the full [T,H] tensors).  Chunks of a prefill batch can so be dispatched as
  * they arrive and combined as their experts finish; any partition of [0,T) gives the same bytes. */
 moe_status_t moe_dispatch_range(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows /*DEVICE*/,
@@ -255,7 +258,9 @@ moe_status_t moe_expert_tiles(moe_ctx_t* ctx, int64_t capacity_rows, int32_t til
                               int32_t* tile_expert /*DEVICE*/, int64_t* tile_row /*DEVICE*/,
                               int32_t* tile_valid /*DEVICE*/, int32_t* n_tiles /*DEVICE*/, void* stream);
 
-/* One whole layer call from HOST buffers, enqueued on `stream`:
+/* One whole layer call from HOST buffers, enqueued on `stream` (no counterpart in the paper, which starts
+ * and ends in device memory; this entry point exists so that an end-to-end number including the
+ * host<->device copies can be measured through the C ABI):
  * host->device copies of topk_idx, topk_w; plan; then, in sixteen token chunks, host->device copy
  * of the chunk of x (upload stream), dispatch and combine reading the dispatched windows (identity
  * experts; caller's stream), and the device->host copy of the chunk of y (download stream), so both
@@ -271,7 +276,8 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
                               void* windows_dev, int64_t capacity_rows, void* y_dev,
                               void* y_host, void* stream);
 
-/* Tuning knobs of a context (tests use them to reach every kernel; defaults are the measured best).
+/* Tuning knobs of a context (no counterpart in the paper; tests use them to reach every kernel, defaults
+ * are the measured best).
  *   MOE_OPT_DISPATCH_PATH  which dispatch kernel runs: AUTO (currently the bulk-copy kernel),
  *                          REGISTERS (16-byte ld/st through registers, K-specialised), or
  *                          BULK (cp.async.bulk through shared-memory stages).  Same result.
@@ -325,12 +331,14 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);
  *   topk_idx        DEVICE [T,K] int32          rank_tok_start  HOST [R+1] or NULL, as in moe_plan
  *   slots           DEVICE [T,K] int32, out     slot(t,j) as moe_plan(DECODE) + moe_slots gives it
  *   n_recv          DEVICE [R] int32, out       rows received per window
- *   status          DEVICE [1] int32, out       0, MOE_ERR_BAD_INDEX (that branch's slot is -1) or
- *                                               MOE_ERR_CAPACITY (no slot written)
+ *   status          DEVICE [1] int32, out       0, MOE_ERR_BAD_INDEX (some index outside [0, E)) or
+ *                                               MOE_ERR_CAPACITY (some n_recv[d] > capacity_rows); with
+ *                                               either error NO slot is written: `slots` keeps what it held
  * Limits: T*K <= 65536, E <= 512, R <= 64, K <= MOE_MAX_K, R*capacity_rows < 2^31; larger problems
  * are rejected with MOE_ERR_INVALID_ARG and a message on stderr -- use moe_plan with a workspace.
  * The first call on each device looks up the array's device address; make that call with the
- * device current and before any stream capture begins.  All calls on one device share the array
+ * device current and before any stream capture begins.  Host threads may make that first call at
+ * the same time (the address is kept in an atomic; every thread finds the same one).  All calls on one device share the array
  * (it keeps the previous call's contents; the words that must start at zero are cleared on the
  * stream each time), so two calls whose kernels may overlap on the GPU -- different streams with
  * no ordering between them -- race; order them on one stream or with events. */
@@ -340,12 +348,13 @@ moe_status_t moe_slots_noalloc(const int32_t* topk_idx /*DEVICE*/, int32_t T, in
                                void* stream);
 
 /* Synchronises `stream`, then returns and clears the device status word
- * (first device-detected error since the last call, or MOE_OK). */
+ * (first device-detected error since the last call, or MOE_OK).  Reporting MOE_ERR_BAD_INDEX also
+ * discards the context's plan (see moe_plan). */
 moe_status_t moe_status(moe_ctx_t* ctx, void* stream);
 
 const char* moe_status_string(moe_status_t status);
 
-/* Number of kernel launches this context has enqueued so far (for benchmarks). */
+/* Number of kernel launches this context has enqueued so far (for benchmarks; no counterpart in the paper). */
 int64_t moe_launch_count(const moe_ctx_t* ctx);
 
 #ifdef __cplusplus

@@ -15,7 +15,7 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("MOECOMM_LIB", os.path.join(_PKG, "libmoecomm.so"))   # override: tuning builds
+LIB_PATH = os.path.join(_PKG, "libmoecomm.so")
 
 MOE_OK, MOE_ERR_INVALID_ARG, MOE_ERR_BAD_INDEX, MOE_ERR_CAPACITY = 0, 1, 2, 3
 MOE_ERR_NOT_PLANNED, MOE_ERR_TIMEOUT, MOE_ERR_CUDA = 4, 5, 6

@@ -4,6 +4,7 @@
 // (top-k gate), bulk_kernels.cuh / quant_kernels.cuh (bulk-copy dispatch, plain
 // and quantised) and row_kernels.cuh (register-path dispatch, combine, slots).
 
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -283,9 +284,7 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   if (warps > BULK_MAX_WARPS) warps = BULK_MAX_WARPS;
   if (warps < 1) warps = 1;
   const int grid = ctx->num_sms;
-#ifndef BULK_STREAMS_TARGET
-#define BULK_STREAMS_TARGET 2400
-#endif
+  constexpr int BULK_STREAMS_TARGET = 2400;
   // Large jobs: HBM serves the writes best when about 2400 destination rows are being written at once
   // (every warp writes K rows at a time), so fewer warps than fit are used when K is large -- but never so
   // few that less than 56 KB of loads are in flight per SM (two stages per warp are loading).  Measured at
@@ -293,7 +292,7 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   // 8 warps 252 us, 4 warps 272 us; at 4 KB rows, K=8: 8 warps 381 us, 2 warps 668 us.  Small jobs keep every
   // warp: there the number of rows in flight decides (decode step 102.7 us with 4 warps, 115 us with 2).
   // "Large" = four rows or more per warp (T=4096 at 14 KB rows: 95.2 -> 93.6 us; T=2048 is slower with the rule).
-  if (BULK_STREAMS_TARGET > 0 && (int64_t)a.t_count >= (int64_t)4 * grid * warps) {
+  if ((int64_t)a.t_count >= (int64_t)4 * grid * warps) {
     int want = (BULK_STREAMS_TARGET + grid * ctx->shape.K / 2) / (grid * ctx->shape.K);
     const int floor_warps = (56 * 1024 + 2 * g_max * 512 - 1) / (2 * g_max * 512);
     if (want < floor_warps) want = floor_warps;
@@ -456,23 +455,28 @@ moe_status_t moe_destroy(moe_ctx_t* ctx) {
 
 namespace {
 
+constexpr int GATE_OCC_MAX_DEVICES = 64;
+
 template <int VPT>
 void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
-                      cudaStream_t st) {
+                      int dev, cudaStream_t st) {
   int warps = 8, smem = 0;
   if (VPT == 0) {   // rows cached in shared memory
     while (warps > 1 && warps * E * (int)sizeof(float) > 96 * 1024) warps >>= 1;
     smem = warps * E * (int)sizeof(float);
   }
-  static int cached = 0;   // resident CTAs per SM of a register form (one device kind per process)
-  int per_sm = VPT > 0 ? cached : 0;   // the shared-memory form's occupancy depends on E: asked every time
+  // Resident CTAs per SM.  The register forms' answer depends only on the device, so it is kept per device in
+  // a table of atomics (any thread may fill an entry; every writer stores the same value); the shared-memory
+  // form's answer depends on E and is asked every time.
+  static std::atomic<int> cached[GATE_OCC_MAX_DEVICES];
+  int per_sm = (VPT > 0 && dev >= 0 && dev < GATE_OCC_MAX_DEVICES) ? cached[dev].load(std::memory_order_relaxed) : 0;
   if (per_sm == 0) {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gate_topk_kernel<VPT>, warps * 32, smem) != cudaSuccess ||
         per_sm < 1) {
       cudaGetLastError();
       per_sm = 1;
     }
-    if (VPT > 0) cached = per_sm;
+    if (VPT > 0 && dev >= 0 && dev < GATE_OCC_MAX_DEVICES) cached[dev].store(per_sm, std::memory_order_relaxed);
   }
   int64_t grid = ((int64_t)T + warps - 1) / warps;
   if (grid > (int64_t)num_sms * per_sm) grid = (int64_t)num_sms * per_sm;   // one resident wave, grid-stride over tokens
@@ -481,14 +485,14 @@ void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int3
 }
 
 void launch_gate(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
-                 cudaStream_t st) {
-  if (E <= 32) launch_gate_form<1>(logits, T, E, K, idx, w, num_sms, st);
-  else if (E <= 64) launch_gate_form<2>(logits, T, E, K, idx, w, num_sms, st);
-  else if (E <= 128) launch_gate_form<4>(logits, T, E, K, idx, w, num_sms, st);
-  else if (E <= 256) launch_gate_form<8>(logits, T, E, K, idx, w, num_sms, st);
-  else if (E <= 512) launch_gate_form<16>(logits, T, E, K, idx, w, num_sms, st);
-  else if (E <= 1024) launch_gate_form<32>(logits, T, E, K, idx, w, num_sms, st);
-  else launch_gate_form<0>(logits, T, E, K, idx, w, num_sms, st);
+                 int dev, cudaStream_t st) {
+  if (E <= 32) launch_gate_form<1>(logits, T, E, K, idx, w, num_sms, dev, st);
+  else if (E <= 64) launch_gate_form<2>(logits, T, E, K, idx, w, num_sms, dev, st);
+  else if (E <= 128) launch_gate_form<4>(logits, T, E, K, idx, w, num_sms, dev, st);
+  else if (E <= 256) launch_gate_form<8>(logits, T, E, K, idx, w, num_sms, dev, st);
+  else if (E <= 512) launch_gate_form<16>(logits, T, E, K, idx, w, num_sms, dev, st);
+  else if (E <= 1024) launch_gate_form<32>(logits, T, E, K, idx, w, num_sms, dev, st);
+  else launch_gate_form<0>(logits, T, E, K, idx, w, num_sms, dev, st);
 }
 
 // Planning, optionally with the gate in front (logits != nullptr: topk_idx and topk_w are OUTPUTS).
@@ -547,7 +551,7 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
   const bool wide = sh.E <= RANK_PLAN_WIDE_MAX_E;
   int n = 0;
   if (logits != nullptr) {   // gate first (its own launch, spread over all SMs), then plan from the indexes it wrote
-    launch_gate(logits, T, sh.E, sh.K, idx_out, w_out, ctx->num_sms, st);
+    launch_gate(logits, T, sh.E, sh.K, idx_out, w_out, ctx->num_sms, ctx->device, st);
     ++n;
   }
   if (ctx->compact_plan) {
@@ -633,7 +637,7 @@ moe_status_t moe_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K,
         cudaFuncSetAttribute(gate_topk_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 2048) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
-  if (T > 0) launch_gate(logits, T, E, K, topk_idx, topk_w, sms, static_cast<cudaStream_t>(stream));
+  if (T > 0) launch_gate(logits, T, E, K, topk_idx, topk_w, sms, dev, static_cast<cudaStream_t>(stream));
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -1040,6 +1044,13 @@ moe_status_t moe_status(moe_ctx_t* ctx, void* stream) {
     if (cudaMemsetAsync(&ctx->ctl->status, 0, sizeof(word), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
       return MOE_ERR_CUDA;
+    // A plan that saw a routing index outside [0, E) left that branch out of its counts: it describes no
+    // valid layout, so it does not survive the report (a later dispatch returns MOE_ERR_NOT_PLANNED
+    // instead of silently skipping the branch).
+    if (word == MOE_ERR_BAD_INDEX) {
+      ctx->planned = false;
+      ctx->layout_done = false;
+    }
   }
   return (word >= 0 && word <= MOE_ERR_CUDA) ? static_cast<moe_status_t>(word) : MOE_ERR_CUDA;
 }
@@ -1090,23 +1101,35 @@ struct NoallocScratch {
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoallocScratch)];  // about 1.2 MB
 
+// The three launches below use the kernels' default (not opted-in) dynamic shared memory, so the largest
+// request an admitted shape can make must fit 48 KB: the Notify scratch with the count matrix staged
+// (R*E <= NOTIFY_STAGE_MAX entries plus one padding column per expert), and the per-warp counters of a tile.
+static_assert((2 * NOALLOC_MAX_E + 1 + 33 + NOTIFY_STAGE_MAX + NOALLOC_MAX_E) * sizeof(int32_t) <= 48 * 1024,
+              "Notify scratch of the no-alloc entry point exceeds the default shared-memory limit");
+static_assert(PLAN_WARPS * NOALLOC_MAX_E * sizeof(int32_t) <= 48 * 1024,
+              "tile counters of the no-alloc entry point exceed the default shared-memory limit");
+
 constexpr int NOALLOC_MAX_DEVICES = 64;
-NoallocScratch* g_noalloc_ptr[NOALLOC_MAX_DEVICES];  // device address of the array, per device; 0 = not set up
+// Device address of the array, per device; nullptr = not looked up yet.  Atomics: host threads that make
+// the first call on a device at the same time all store the same address.
+std::atomic<NoallocScratch*> g_noalloc_ptr[NOALLOC_MAX_DEVICES];
 
 // In host code g_noalloc_scratch is only a handle for the runtime, not a device address, so the
 // address each device uses is looked up once, with that device current.
 NoallocScratch* noalloc_scratch_for_current_device() {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return nullptr;
-  if (g_noalloc_ptr[dev] == nullptr) {
+  NoallocScratch* sc = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+  if (sc == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
       cudaGetLastError();
       return nullptr;
     }
-    g_noalloc_ptr[dev] = static_cast<NoallocScratch*>(p);
+    sc = static_cast<NoallocScratch*>(p);
+    g_noalloc_ptr[dev].store(sc, std::memory_order_release);
   }
-  return g_noalloc_ptr[dev];
+  return sc;
 }
 
 }  // namespace
@@ -1162,7 +1185,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
         topk_idx, map, K, E, sc->tile_rank, sc->tile_hist, status);
   plan_scan_kernel<<<R, PLAN_THREADS, notify_smem_ints(E, R) * (int)sizeof(int32_t), st>>>(
       sc->tile_hist, map, E, 0, 1, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl, 0);
-  RowArgs a;
+  RowArgs a = {};   // every field the kernel is handed has a defined value
   a.topk_idx = topk_idx;
   a.small_off = sc->tile_rank;
   a.small_out = nullptr;

@@ -11,9 +11,9 @@
 //                      counters in shared memory, exclusive scan across warps
 //                      -> in-tile rank of every branch, tile histogram [E]
 //   plan_scan_kernel   one CTA per source rank: exclusive scan of the tile
-//                      histograms over that rank's tiles ("per-block counting
-//                      plus prefix accumulation over earlier blocks") -> tile
-//                      bases, row r of M.  Then M becomes n_exp, n_recv, c_rank and the
+//                      histograms over that rank's tiles (counts per tile, then a
+//                      prefix over the earlier tiles of the same rank: Section 5.2,
+//                      Prefill Layout) -> tile bases, row r of M.  Then M becomes n_exp, n_recv, c_rank and the
 //                      large offsets o (exclusive scan in window order: expert, then
 //                      source rank): by every CTA for its own window when the R CTAs
 //                      run as one thread-block cluster (rows of M exchanged through

@@ -48,6 +48,17 @@ struct RowArgs {
   int32_t test_starve;       // test hook of the bulk-copy dispatch: make one wait run out
 };
 
+// Load of a word the planner wrote (small offsets, tile bases, large offsets).  A kernel chained behind the
+// planner by programmatic stream serialization is already running while the planner writes these arrays, so
+// they are not read-only for its lifetime and must not take the non-coherent path (ld.global.nc / __ldg);
+// a plain load issued after dependency_wait() sees the planner's writes.  Routing indexes, weights and payload
+// rows are inputs of the whole call and keep the non-coherent loads.
+__device__ __forceinline__ int32_t ld_plan(const int32_t* p) {
+  int32_t v;
+  asm volatile("ld.global.b32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
 // Window row of branch (t, lane) for lane < K, -1 otherwise.  Small offsets of
 // the DECODE schedule are finished here (in-tile rank + tile base).
 __device__ __forceinline__ int64_t resolve_slot(const RowArgs& a, const RankMap& map, int32_t t, int lane,
@@ -57,12 +68,12 @@ __device__ __forceinline__ int64_t resolve_slot(const RowArgs& a, const RankMap&
   const int32_t e = __ldg(a.topk_idx + b);
   if (e < 0 || e >= a.E) return -1;  // flagged by the plan; never dereferenced
   const int32_t r = src_rank(map, t);
-  int32_t so = __ldg(a.small_off + b);
+  int32_t so = ld_plan(a.small_off + b);
   if (a.tile_base != nullptr) {
-    so += __ldg(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + e);
+    so += ld_plan(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + e);
     if (record) a.small_out[b] = so;
   }
-  return (int64_t)(e / a.E_r) * a.C + __ldg(a.large_off + (size_t)e * a.R + r) + so;
+  return (int64_t)(e / a.E_r) * a.C + ld_plan(a.large_off + (size_t)e * a.R + r) + so;
 }
 
 // The same resolution in two phases, so that its memory latency can hide behind payload traffic:
@@ -85,7 +96,7 @@ __device__ __forceinline__ BranchMeta load_meta(const RowArgs& a, const float* _
   if (lane < a.K) {
     const int32_t b = t * a.K + lane;
     m.e = __ldg(a.topk_idx + b);
-    m.so = __ldg(a.small_off + b);
+    m.so = ld_plan(a.small_off + b);
     if (topk_w != nullptr) m.w = __ldg(topk_w + b);
   }
   return m;
@@ -98,10 +109,10 @@ __device__ __forceinline__ int64_t finish_slot(const RowArgs& a, const RankMap& 
   int32_t so = m.so;
   if (a.tile_base != nullptr) {
     const int32_t b = t * a.K + lane;
-    so += __ldg(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + m.e);
+    so += ld_plan(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + m.e);
     if (record) a.small_out[b] = so;
   }
-  return (int64_t)(m.e / a.E_r) * a.C + __ldg(a.large_off + (size_t)m.e * a.R + r) + so;
+  return (int64_t)(m.e / a.E_r) * a.C + ld_plan(a.large_off + (size_t)m.e * a.R + r) + so;
 }
 
 // Pulls a word into the cache hierarchy ahead of its use; the value is discarded.
@@ -428,9 +439,9 @@ slots_kernel(int32_t* __restrict__ slots, const RowArgs a, const __grid_constant
       continue;
     }
     const int32_t r = src_rank(map, t);
-    int32_t so = __ldg(a.small_off + b);
-    if (a.tile_base != nullptr) so += __ldg(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + e);
-    slots[b] = (int32_t)((int64_t)(e / a.E_r) * a.C + __ldg(a.large_off + (size_t)e * a.R + r) + so);
+    int32_t so = ld_plan(a.small_off + b);
+    if (a.tile_base != nullptr) so += ld_plan(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + e);
+    slots[b] = (int32_t)((int64_t)(e / a.E_r) * a.C + ld_plan(a.large_off + (size_t)e * a.R + r) + so);
   }
 }
 

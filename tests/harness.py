@@ -81,7 +81,6 @@ def oracle_run(inp: synth.Inputs, C: int, n_threads: int = 4, align: int = 1) ->
                                    align=align) == oracle.OK
     st, Y = oracle.combine(win, slots, inp.topk_w.numpy(), wl.H, n_threads)
     assert st == oracle.OK
-    zero_init = np.where(win_after_dispatch == CANARY, np.uint16(0), win_after_dispatch)
     used = np.zeros(wl.R * C, bool)
     used[slots.reshape(-1)] = True
     zero_init = win_after_dispatch.copy()

@@ -1,12 +1,15 @@
-"""Full benchmark sizes (configs 3 and 4) in the launch configuration bench.py times.
+"""Full benchmark sizes, in the launch configuration bench.py times, compared with the oracle whole tensor by
+whole tensor: every integer the plan produces, every byte of the expert windows after dispatch (padding rows
+and their canaries included), and every element of the combined output with a non-trivial expert stand-in
+(per-expert scaling) between dispatch and combine.  Covers configs 3 and 4, config 5 at T = 65536 under both
+schedules (the large-job combine with two branches), the top-7 shape of the benchmark (the large-job combine of
+the any-K family) and the row-wise quantised dispatch at config 3 (its three-stage form).
 
-The oracle cannot replay 4 GB of rows in seconds, so: every integer the plan
-produces is compared in full (the oracle's plan is cheap); dispatched rows and
-combined outputs are compared on sampled branches / tokens that the oracle
-computes one by one from the host inputs; and properties that hold at any size
-cover the rest (padding rows untouched, column checksums of the windows,
-identity round trip Y == X).
+The oracle runs token-parallel over all host cores (about half a second per pass at config 3); its windows are
+uploaded in chunks and compared on the device.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -18,91 +21,143 @@ import harness
 
 pytestmark = pytest.mark.gpu
 
+CORES = len(os.sched_getaffinity(0))
+CANARY_I16 = int(np.int16(np.uint16(harness.CANARY)))
+
 
 def as_u16(t: torch.Tensor) -> np.ndarray:
     return t.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("n", [3, 4])
-def test_full_size_prefill_sampled(n):
+def device_equals_host(dev_rows: torch.Tensor, host_rows: np.ndarray, chunk_rows: int = 1 << 16) -> bool:
+    """Element-wise comparison of a device tensor [rows, H] of 16-bit (or 8-bit) patterns with a host array of
+    the same shape, uploading the host side in chunks."""
+    assert tuple(dev_rows.shape) == host_rows.shape, (dev_rows.shape, host_rows.shape)
+    view = {2: torch.int16, 1: torch.uint8, 4: torch.int32}[host_rows.dtype.itemsize]
+    np_view = {2: np.int16, 1: np.uint8, 4: np.int32}[host_rows.dtype.itemsize]
+    for r0 in range(0, host_rows.shape[0], chunk_rows):
+        r1 = min(host_rows.shape[0], r0 + chunk_rows)
+        want = torch.from_numpy(host_rows[r0:r1].view(np_view)).to(dev_rows.device)
+        if not torch.equal(dev_rows[r0:r1].view(view), want):
+            return False
+    return True
+
+
+def full_windows(rows: int, H: int, dev) -> torch.Tensor:
+    win = torch.empty((rows, H), dtype=torch.bfloat16, device=dev)
+    win.view(torch.int16).fill_(CANARY_I16)
+    return win
+
+
+FULL_CASES = {
+    "c3": lambda: (synth.config(3), synth.PREFILL),
+    "c4": lambda: (synth.config(4), synth.PREFILL),
+    "c5_T65536_prefill": lambda: (synth.config(5, 65536, synth.PREFILL), synth.PREFILL),
+    "c5_T65536_decode": lambda: (synth.config(5, 65536, synth.DECODE), synth.DECODE),
+    # the benchmark's top-7 workload (no K-specialised dispatch; combine<7> in its large-job form)
+    "k7": lambda: (synth.Workload("k7_prefill", 16384, 7168, 256, 8, 7, synth.PREFILL, "uniform", "identity", 1007),
+                   synth.PREFILL),
+}
+
+
+@pytest.mark.parametrize("case", sorted(FULL_CASES))
+def test_full_size_whole_tensors_against_the_oracle(case):
     dev = torch.device("cuda:0")
-    wl = synth.config(n)
+    wl, schedule = FULL_CASES[case]()
     inp = synth.make_inputs(wl)
     idx_np = inp.topk_idx.numpy()
     p = oracle.plan(idx_np, wl.E, wl.R)
     assert p.status == oracle.OK
-    if n == 4:
-        assert p.n_exp.max() >= 10 * wl.B / wl.E
+    if case == "c4":
+        assert p.n_exp.max() >= 10 * wl.B / wl.E              # the premise of the skewed configuration
     C = (int(p.n_recv.max()) + 7) // 8 * 8                     # as bench.py sizes it
     st, slots = oracle.slots(idx_np, wl.E, wl.R, p, C)
     assert st == oracle.OK
+    # per-expert bf16 scale factors of the stand-in expert op (drawn apart from the inputs, so that X, K and W
+    # stay the benchmark's own)
+    scale = (0.5 + torch.rand(wl.E, generator=torch.Generator().manual_seed(4200 + wl.seed % 1000),
+                              dtype=torch.float32)).to(torch.bfloat16)
 
+    # ---- oracle: dispatch into canary-filled windows, scale, combine
+    X_u16 = synth.bf16_to_u16(inp.X)
+    win_ref = np.full((wl.R * C, wl.H), harness.CANARY, np.uint16)
+    assert oracle.dispatch(X_u16, slots, win_ref, CORES) == oracle.OK
+
+    # ---- device
     comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
     X, idx, w = inp.X.to(dev), inp.topk_idx.to(dev), inp.topk_w.to(dev)
-    windows = torch.empty((wl.R * C, wl.H), dtype=torch.bfloat16, device=dev)
-    windows.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+    windows = full_windows(wl.R * C, wl.H, dev)
     Y = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device=dev)
     got_slots = torch.empty((wl.T, wl.K), dtype=torch.int32, device=dev)
-    comm.moe_plan(wl.schedule, idx)
+    comm.moe_plan(schedule, idx)
     comm.moe_slots(C, got_slots)
     comm.moe_dispatch(X, windows, C)
-    comm.moe_combine(windows, C, w, Y)
     assert comm.moe_status() == 0
 
     # -- integers: everything, bit-exact
     v = comm.moe_plan_view()
     for k, name in {"counts": "M", "c_rank": "c_rank", "small_off": "s", "large_off": "o", "n_exp": "n_exp",
                     "n_recv": "n_recv"}.items():
+        if v[k] is None:
+            assert schedule == synth.DECODE and k in ("counts", "c_rank", "n_exp")
+            continue
         assert np.array_equal(v[k].cpu().numpy(), getattr(p, name)), k
     assert np.array_equal(got_slots.cpu().numpy().astype(np.int64), slots)
+    # -- dispatched bytes: the whole window allocation, padding rows (canaries) included
+    assert device_equals_host(windows, win_ref)
 
-    # -- dispatched rows: sampled branches against the host rows of X, bit-exact
-    rng = np.random.default_rng(n)
-    bt = rng.integers(0, wl.T, 3000)
-    bj = rng.integers(0, wl.K, 3000)
-    rows = torch.from_numpy(slots[bt, bj]).to(dev)
-    got = as_u16(windows.index_select(0, rows))
-    assert np.array_equal(got, synth.bf16_to_u16(inp.X)[bt])
-    # -- padding rows of every segment were never written
-    for d in range(wl.R):
-        pad = windows[d * C + int(p.n_recv[d]):(d + 1) * C]
-        if pad.numel():
-            assert bool((pad.view(torch.int16) == int(np.int16(np.uint16(harness.CANARY)))).all()), d
-    # -- any-size property: every token row sits in the windows exactly K times, so the column sums of the
-    #    bit patterns over the used rows equal K times the column sums over X (exact in int64)
-    used = torch.cat([windows[d * C:d * C + int(p.n_recv[d])] for d in range(wl.R)]) if n == 3 else None
-    if used is not None:
-        lhs = (used.view(torch.int16).to(torch.int64) & 0xFFFF).sum(0)
-        rhs = (X.view(torch.int16).to(torch.int64) & 0xFFFF).sum(0) * wl.K
-        assert torch.equal(lhs, rhs)
-        del used
-
-    # -- combine: identity experts and weights summing to 1 => Y == X at every element
-    assert torch.equal(Y.view(torch.int16), X.view(torch.int16))
-    # -- planning folded into the dispatch call: the same bytes everywhere (padding rows included),
-    #    and the sampled rows once more against the host copy of X
-    windows2 = torch.empty_like(windows)
-    windows2.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
-    comm.moe_plan_dispatch(wl.schedule, idx, X, windows2, C)
+    # -- planning folded into the dispatch call: the same bytes everywhere
+    windows2 = full_windows(wl.R * C, wl.H, dev)
+    comm.moe_plan_dispatch(schedule, idx, X, windows2, C)
     assert comm.moe_status() == 0
     assert torch.equal(windows2.view(torch.int16), windows.view(torch.int16))
-    assert np.array_equal(as_u16(windows2.index_select(0, rows)), synth.bf16_to_u16(inp.X)[bt])
     del windows2
-    # -- and sampled tokens against the oracle run on their own rows (inputs come from the host copy of X)
-    S = np.sort(rng.choice(wl.T, 256, replace=False))
-    Xs = synth.bf16_to_u16(inp.X)[S]
-    mini_slots = np.arange(len(S) * wl.K, dtype=np.int64).reshape(len(S), wl.K)
-    mini_win = np.zeros((len(S) * wl.K, wl.H), np.uint16)
-    assert oracle.dispatch(Xs, mini_slots, mini_win) == oracle.OK
-    # scale the mini windows and the device windows with per-row factors so the check is not the identity case
-    fac = torch.from_numpy(rng.uniform(0.5, 1.5, (len(S), wl.K)).astype(np.float32)).to(torch.bfloat16)
-    mw = synth.u16_to_bf16(mini_win).view(len(S), wl.K, wl.H) * fac[:, :, None]
-    mini_win = synth.bf16_to_u16(mw.reshape(len(S) * wl.K, wl.H).contiguous())
-    st, want = oracle.combine(mini_win, mini_slots, inp.topk_w.numpy()[S], wl.H)
-    srows = torch.from_numpy(slots[S].reshape(-1)).to(dev)
-    windows[srows] = (windows[srows].view(len(S), wl.K, wl.H) * fac.to(dev)[:, :, None]).reshape(-1, wl.H)
+
+    # -- combine, identity experts and weights summing to 1: Y == X at every element
     comm.moe_combine(windows, C, w, Y)
     assert comm.moe_status() == 0
-    got = as_u16(Y.index_select(0, torch.from_numpy(S).to(dev)))
-    assert harness.max_ulp_diff(got, want) <= 1
+    assert torch.equal(Y.view(torch.int16), X.view(torch.int16))
+
+    # -- combine behind the scaling expert op: all of Y against the oracle's, at most 1 bf16 ulp apart
+    assert oracle.expert_scale(win_ref, wl.H, wl.E, wl.R, C, p.n_exp, synth.bf16_to_u16(scale)) == oracle.OK
+    st, Y_ref = oracle.combine(win_ref, slots, inp.topk_w.numpy(), wl.H, CORES)
+    assert st == oracle.OK
+    harness.gpu_expert_scale(windows, idx, wl.E, wl.R, C, scale.to(dev))
+    assert device_equals_host(windows, win_ref)               # the harness op itself, so Y is compared on equal inputs
+    comm.moe_combine(windows, C, w, Y)
+    assert comm.moe_status() == 0
+    assert harness.max_ulp_diff(as_u16(Y), Y_ref) <= 1
+    comm.close()
+
+
+def test_full_size_quantised_dispatch_codes_and_scales():
+    """Row-wise quantised dispatch at config 3: every e4m3 code of the code windows and every fp32 scale,
+    bit-exact against the oracle (padding rows keep their fill)."""
+    dev = torch.device("cuda:0")
+    wl = synth.config(3)
+    inp = synth.make_inputs(wl)
+    idx_np = inp.topk_idx.numpy()
+    p = oracle.plan(idx_np, wl.E, wl.R)
+    C = (int(p.n_recv.max()) + 7) // 8 * 8
+    st, slots = oracle.slots(idx_np, wl.E, wl.R, p, C)
+    assert st == oracle.OK
+    want_q = np.full((wl.R * C, wl.H), 0xAB, np.uint8)
+    want_s = np.full((wl.R * C,), -1.0, np.float32)
+    assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), slots, want_q, want_s, CORES) == oracle.OK
+
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx = inp.X.to(dev), inp.topk_idx.to(dev)
+    wq = torch.full((wl.R * C, wl.H), 0xAB, dtype=torch.uint8, device=dev)
+    sc = torch.full((wl.R * C,), -1.0, dtype=torch.float32, device=dev)
+    comm.moe_plan(wl.schedule, idx)
+    comm.moe_dispatch_quant(X, wq, sc, C)
+    assert comm.moe_status() == 0
+    assert device_equals_host(wq, want_q)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+    # the chained form gives the same bytes
+    wq2 = torch.full_like(wq, 0xAB)
+    sc2 = torch.full_like(sc, -1.0)
+    comm.moe_plan_dispatch_quant(wl.schedule, idx, X, wq2, sc2, C)
+    assert comm.moe_status() == 0
+    assert torch.equal(wq2, wq) and torch.equal(sc2.view(torch.int32), sc.view(torch.int32))
     comm.close()

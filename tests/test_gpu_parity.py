@@ -262,6 +262,12 @@ def test_errors_leave_memory_untouched():
             assert comm.moe_status() == binding.MOE_ERR_BAD_INDEX
             assert comm.moe_status() == 0                      # cleared by the read
             assert canary_only(win) and canary_only(Y)
+            # the plan that saw the bad index does not survive the report: no call may go on to skip the branch
+            assert comm.moe_dispatch(X, win, C, check=False) == binding.MOE_ERR_NOT_PLANNED
+            assert comm.moe_combine(win, C, w, Y, check=False) == binding.MOE_ERR_NOT_PLANNED
+            assert comm.moe_slots(C, torch.empty((T, K), dtype=torch.int32, device=dev), check=False) == \
+                binding.MOE_ERR_NOT_PLANNED
+            assert canary_only(win) and canary_only(Y)
 
     # and the context still works afterwards
     comm.moe_plan(PREFILL, idx)
