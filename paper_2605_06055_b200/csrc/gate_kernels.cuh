@@ -5,8 +5,8 @@
 //   topk_w[t, j]        = exp(l_j - l_0) / sum_j' exp(l_j' - l_0)   (fp32, sum in ascending j)
 //
 // One warp per token, K rounds of "largest remaining logit"; the lane that owns the winner retires it.
-// Rows of up to 1024 logits live in registers (warp_gate_token_regs); longer rows are cached in
-// shared memory and scanned with a shuffle arg-max (warp_gate_token).
+// Rows of up to 1024 logits live in registers (warp_gate_load + warp_gate_select); longer rows are cached
+// in shared memory and scanned with a shuffle arg-max (warp_gate_token).
 #pragma once
 
 #include "common.cuh"
@@ -55,84 +55,242 @@ __device__ __forceinline__ void warp_gate_token(const float* __restrict__ logits
   idx_lane = sel_idx;
 }
 
-// Order-preserving map from fp32 to uint32 (larger float <=> larger key), so that the warp-wide
-// arg-max can use the single-instruction integer reductions (redux.sync).
-__device__ __forceinline__ uint32_t sortable_key(float f) {
-  const uint32_t u = __float_as_uint(f + 0.0f);   // -0 becomes +0: the two compare equal as floats
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+// Warp-wide max of fp32 values / min of unsigned values in one instruction each (redux.sync; the fp32 form
+// is an sm_100a instruction).  Inputs are finite or -inf, never NaN.
+__device__ __forceinline__ float warp_max_f32(float v) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+  return r;
 }
 
-__device__ __forceinline__ float key_to_float(uint32_t k) {
-  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
-
-// The same for E <= 32 * VPT with the row in registers: lane l holds experts l, l + 32, ... (coalesced
-// loads) as sortable keys; 0 marks "absent or retired" (no finite float maps to key 0).  A round is
-// VPT-1 integer max, one redux.max for the winning value, one redux.min for the lowest expert
-// index that holds it, and a predicated retire: about 45 instructions instead of about 110 with a
-// shuffle tree on (value, index) pairs.
+// The two largest of a lane's VPT logits with their expert indexes, lower index first among equals
+// (ascending walk, strict compares); i0, i1 are positions inside the lane.  `dead` bit i set: element i has been
+// selected already.
 template <int VPT>
-__device__ __forceinline__ void warp_gate_token_regs(const float* __restrict__ logits_row, int E, int K, int lane,
-                                                     int32_t& idx_lane, float& w_lane) {
-  uint32_t v[VPT];
+__device__ __forceinline__ void lane_top2(const float (&v)[VPT], uint32_t dead, float& h0, int32_t& i0, float& h1,
+                                          int32_t& i1) {
+  h0 = -INFINITY;
+  h1 = -INFINITY;
+  i0 = 0x7fffffff;
+  i1 = 0x7fffffff;
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
-    const int e = lane + 32 * i;
-    v[i] = e < E ? sortable_key(__ldg(logits_row + e)) : 0u;
+    const float x = ((dead >> i) & 1u) ? -INFINITY : v[i];
+    const bool p0 = x > h0, p1 = x > h1;
+    h1 = p0 ? h0 : (p1 ? x : h1);
+    i1 = p0 ? i0 : (p1 ? i : i1);
+    h0 = p0 ? x : h0;
+    i0 = p0 ? i : i0;
   }
-  uint32_t sel_key = 0;
+}
+
+// Rows of at most 32 * VPT logits, held in registers: lane l owns the VPT CONSECUTIVE experts l*VPT .. l*VPT+VPT-1
+// (two 16-byte loads per lane at 256 experts), so "lowest expert index" is "lowest lane, then lowest position".
+// Every lane keeps its two largest remaining logits cached.  A round is then: redux.max over the lane heads,
+// redux.min over the expert indexes of the lanes whose head equals it, and a pop on the one winning lane --
+// about a dozen instructions, none of which touches the VPT registers.  Only when a lane has been popped twice
+// is its cache rebuilt from its registers (a warp-uniform branch, taken well under once per token at 256 experts,
+// top-8).  -inf marks absent and selected entries (logits are finite); -0 and +0 compare equal in every
+// comparison made here, so either may be reported as the value (the weights do not depend on the sign of zero).
+template <int VPT>
+__device__ __forceinline__ void warp_gate_select(const float (&v)[VPT], int K, int lane, int32_t& idx_lane,
+                                                 float& w_lane) {
+  const int base = lane * VPT;
+  uint32_t dead = 0;
+  float h0, h1;
+  int32_t i0, i1;
+  lane_top2<VPT>(v, 0u, h0, i0, h1, i1);
+  float sel_val = 0.0f;
   int32_t sel_idx = -1;
   for (int j = 0; j < K; ++j) {
-    uint32_t local = v[0];
-#pragma unroll
-    for (int i = 1; i < VPT; ++i) local = max(local, v[i]);
-    const uint32_t best = __reduce_max_sync(0xffffffffu, local);
-    int32_t first = 0x7fffffff;                      // lowest expert index of mine that holds `best`
-#pragma unroll
-    for (int i = VPT - 1; i >= 0; --i) first = (v[i] == best) ? lane + 32 * i : first;
-    // (a vote for the holder plus a shuffle of its index instead of this second reduction measured
-    // slower: 35.2 vs 33.1 us at T=32768, E=256, K=8)
-    const int32_t be = (int32_t)__reduce_min_sync(0xffffffffu, (uint32_t)first);
+    const float best = warp_max_f32(h0);
+    const uint32_t cand = (h0 == best) ? (uint32_t)(base + i0) : 0x7fffffffu;
+    const uint32_t be = __reduce_min_sync(0xffffffffu, cand);   // lowest expert index that holds `best`
     if (lane == j) {
-      sel_key = best;
-      sel_idx = be;
+      sel_val = best;
+      sel_idx = (int32_t)be;
     }
-    // Retire the winner: a select on every register, so the array is never indexed dynamically.
-    const int32_t hit = (be & 31) == lane ? (be >> 5) : -1;
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) v[i] = (i == hit) ? 0u : v[i];
+    const bool win = cand == be;          // exactly one lane: expert indexes are unique
+    if (win) {
+      dead |= 1u << i0;
+      h0 = h1;
+      i0 = i1;
+      h1 = -INFINITY;
+      i1 = 0x7fffffff;
+    }
+    if constexpr (VPT > 2) {
+      // popped twice since the last rebuild: this lane's remaining logits are unknown to its cache
+      if (__any_sync(0xffffffffu, win && h0 == -INFINITY) && j + 1 < K) {
+        if (win) lane_top2<VPT>(v, dead, h0, i0, h1, i1);
+      }
+    }
   }
-  const float sel_val = key_to_float(sel_key);
-  const float top = __shfl_sync(0xffffffffu, sel_val, 0);
-  const float ex = lane < K ? expf(sel_val - top) : 0.0f;
-  float sum = 0.0f;
-  for (int j = 0; j < K; ++j) sum += __shfl_sync(0xffffffffu, ex, j);
-  w_lane = __fdiv_rn(ex, sum);
+  w_lane = sel_val;
   idx_lane = sel_idx;
 }
 
-// Stand-alone gate: grid-stride over tokens, one warp per token.  VPT > 0: register form for rows of at
-// most 32 * VPT logits (one instantiation per row length class, so that short rows keep few registers
-// and many warps per SM: 80 registers for a kernel holding every form, 3 CTAs per SM, against 6-8 CTAs
-// per SM for the 256-logit form on its own).  VPT == 0: shared-memory form for longer rows; dynamic shared
+// Selection by threshold and rank, for the common case.  theta, the K-th largest DISTINCT value among the 32
+// lane maxima (K rounds of "warp max, then drop the lanes that hold it": three instructions each, no index
+// tracking), is a lower bound of the K-th largest logit, because at least K entries are >= theta; so every
+// selected entry is >= theta, and only a few more are (about nine at 256 experts, top-8).  Those entries are
+// compacted, in ascending expert order, into one candidate per lane through shared memory; a candidate's place in
+// the output is the number of candidates with a larger logit plus the number of EARLIER candidates with an equal
+// one (equal logits: lower expert index first), counted directly.  More than 32 candidates (many equal logits, K
+// close to 32): the caller falls back to warp_gate_select.
+// On success lane j < K holds the j-th selected logit (in w_lane) and its expert.
+constexpr int GATE_RANK_WORDS = 132;
+
+template <int VPT>
+__device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int lane, float* sm, int32_t& idx_lane,
+                                               float& w_lane) {
+  float* cand_val = sm;                                          // [36]: up to 32 candidates + padding of the last group of four
+  int32_t* cand_idx = reinterpret_cast<int32_t*>(sm + 36);       // [32]
+  float* out_val = sm + 68;                                      // [32]
+  int32_t* out_idx = reinterpret_cast<int32_t*>(sm + 100);       // [32]
+  const int base = lane * VPT;
+  float m = v[0];
+#pragma unroll
+  for (int i = 1; i < VPT; ++i) m = fmaxf(m, v[i]);
+  float theta = 0.0f;
+  for (int j = 0; j < K; ++j) {
+    theta = warp_max_f32(m);
+    m = (m == theta) ? -INFINITY : m;
+  }
+  // absent entries are -inf and must never qualify; logits are finite, so -FLT_MAX admits every real entry
+  theta = fmaxf(theta, -3.402823466e+38f);
+  int c = 0;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) c += (v[i] >= theta) ? 1 : 0;
+  int incl = c;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int u = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += u;
+  }
+  const int C = __shfl_sync(0xffffffffu, incl, 31);
+  if (C > 32) return false;
+  // predicated stores, no branches: slot address advances by one word per candidate
+  uint32_t slot = (uint32_t)__cvta_generic_to_shared(cand_val) + 4u * (uint32_t)(incl - c);
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    uint32_t step;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ge.f32 p, %1, %2;\n\t"
+        "@p st.shared.f32 [%3], %1;\n\t"
+        "@p st.shared.u32 [%3+144], %4;\n\t"     // cand_idx = cand_val + 36 words
+        "selp.u32 %0, 4, 0, p;\n\t}"
+        : "=r"(step) : "f"(v[i]), "f"(theta), "r"(slot), "r"(base + i) : "memory");
+    slot += step;
+  }
+  __syncwarp();
+  if (lane < 3) cand_val[C + lane] = -INFINITY;   // the counting loop reads four candidates at a time
+  __syncwarp();
+  const float x = lane < C ? cand_val[lane] + 0.0f : -INFINITY;   // -0 becomes +0: equal logits get equal bit patterns
+  const int32_t xi = lane < C ? cand_idx[lane] : -1;
+  int rank = __popc(__match_any_sync(0xffffffffu, __float_as_uint(x)) & lanemask_lt());   // earlier equal candidates
+  for (int q = 0; q < C; q += 4) {
+    const float4 a = *reinterpret_cast<const float4*>(cand_val + q);   // broadcast read
+    rank += (a.x > x ? 1 : 0) + (a.y > x ? 1 : 0) + (a.z > x ? 1 : 0) + (a.w > x ? 1 : 0);
+  }
+  if (lane < C && rank < K) {
+    out_val[rank] = x;
+    out_idx[rank] = xi;
+  }
+  __syncwarp();
+  w_lane = lane < K ? out_val[lane] : 0.0f;
+  idx_lane = lane < K ? out_idx[lane] : -1;
+  __syncwarp();   // the next token of this warp reuses the buffers
+  return true;
+}
+
+// fp32 softmax over the K selected logits (lane j < K holds the j-th), summed in ascending j.
+__device__ __forceinline__ float warp_gate_softmax(float sel_val, int K, int lane) {
+  const float top = __shfl_sync(0xffffffffu, sel_val, 0);
+  const float ex = lane < K ? expf(sel_val - top) : 0.0f;
+  float sum = 0.0f;
+  // eight terms at a time; the lanes beyond K hold +0, which leaves the sum unchanged (K <= 32, so no index wraps)
+  for (int j0 = 0; j0 < K; j0 += 8) {
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) sum += __shfl_sync(0xffffffffu, ex, j0 + jj);
+  }
+  // the lanes beyond K divide 1 by the sum: a zero numerator would take the division's special-case path
+  return __fdiv_rn(lane < K ? ex : 1.0f, sum);
+}
+
+// Loads the row of one token into the lane-contiguous register layout.  `vec`: the row starts on a 16-byte
+// boundary and E is a multiple of 4, so a lane's run is read with 16-byte loads.
+template <int VPT>
+__device__ __forceinline__ void warp_gate_load(const float* __restrict__ row, int E, int lane, bool vec,
+                                               float (&v)[VPT]) {
+  const int base = lane * VPT;
+  if constexpr (VPT % 4 == 0) {
+    if (vec) {
+#pragma unroll
+      for (int q = 0; q < VPT / 4; ++q) {
+        float4 f = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (base + 4 * q < E) f = __ldg(reinterpret_cast<const float4*>(row + base) + q);
+        v[4 * q] = f.x;
+        v[4 * q + 1] = f.y;
+        v[4 * q + 2] = f.z;
+        v[4 * q + 3] = f.w;
+      }
+      return;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) v[i] = base + i < E ? __ldg(row + base + i) : -INFINITY;
+}
+
+// Stand-alone gate: grid-stride over tokens, one warp per token, the next token's row loaded while the current
+// one is selected.  VPT > 0: register form for rows of at most 32 * VPT logits (one instantiation per row
+// length class, so that short rows keep few registers and many warps per SM).  VPT == 0: shared-memory form for longer rows; dynamic shared
 // memory: warps * E floats.
 template <int VPT>
 __global__ void __launch_bounds__(256)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
                  float* __restrict__ topk_w) {
   extern __shared__ float gate_rows[];
+  __shared__ __align__(16) float gate_cand[8][GATE_RANK_WORDS];   // warp_gate_rank's buffers, one set per warp
   release_dependents();   // a planner launched behind the gate (moe_gate_plan) may be scheduled; it waits for this kernel
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpc = blockDim.x >> 5;
-  for (int32_t t = blockIdx.x * wpc + warp; t < T; t += gridDim.x * wpc) {
-    int32_t idx;
-    float w;
-    if constexpr (VPT > 0) warp_gate_token_regs<VPT>(logits + (size_t)t * E, E, K, lane, idx, w);
-    else warp_gate_token(logits + (size_t)t * E, gate_rows + warp * E, E, K, lane, idx, w);
-    if (lane < K) {
-      topk_idx[(size_t)t * K + lane] = idx;
-      topk_w[(size_t)t * K + lane] = w;
+  const int32_t stride = gridDim.x * wpc;
+  int32_t t = blockIdx.x * wpc + warp;
+  if constexpr (VPT > 0) {
+    const bool vec = (E % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0);
+    auto process = [&](const float (&v)[VPT], int32_t tok) {
+      int32_t idx;
+      float w;
+      if (!warp_gate_rank<VPT>(v, K, lane, gate_cand[warp], idx, w)) warp_gate_select<VPT>(v, K, lane, idx, w);
+      w = warp_gate_softmax(w, K, lane);
+      if (lane < K) {
+        topk_idx[(size_t)tok * K + lane] = idx;
+        topk_w[(size_t)tok * K + lane] = w;
+      }
+    };
+    // two row buffers used in turn: the next token's row travels while the current one is selected
+    float row_a[VPT], row_b[VPT];
+    if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row_a);
+    while (t < T) {
+      if (t + stride < T) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, row_b);
+      process(row_a, t);
+      t += stride;
+      if (t >= T) break;
+      if (t + stride < T) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, row_a);
+      process(row_b, t);
+      t += stride;
     }
-    __syncwarp();
+  } else {
+    for (; t < T; t += stride) {
+      int32_t idx;
+      float w;
+      warp_gate_token(logits + (size_t)t * E, gate_rows + warp * E, E, K, lane, idx, w);
+      if (lane < K) {
+        topk_idx[(size_t)t * K + lane] = idx;
+        topk_w[(size_t)t * K + lane] = w;
+      }
+      __syncwarp();
+    }
   }
 }
 

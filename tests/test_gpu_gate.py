@@ -26,10 +26,21 @@ def logits_for(T, E, seed, ties=False):
 
 @pytest.mark.parametrize("T,E,K,ties", [(256, 16, 2, False), (2048, 256, 8, False), (500, 256, 8, True),
                                         (77, 8, 8, True), (300, 40, 1, False), (64, 4096, 32, False),
-                                        (1000, 1000, 6, True)])
+                                        (1000, 1000, 6, True),
+                                        # every register form, full and partly filled lanes, K up to the limit
+                                        (333, 200, 8, True), (333, 40, 8, True), (257, 96, 4, True),
+                                        (129, 250, 8, True), (200, 512, 8, True), (96, 1024, 32, True),
+                                        (100, 32, 32, True), (5000, 256, 8, "few"), (300, 128, 32, "few"),
+                                        (64, 256, 8, "zeros")])
 def test_gate_topk_kernel(T, E, K, ties):
     dev = torch.device("cuda:0")
-    l = logits_for(T, E, T + E, ties)
+    l = logits_for(T, E, T + E, ties is True)
+    if ties == "few":       # three distinct values: nearly every selection is decided by the index, and lanes
+        l = torch.round(l / 6)   # are popped many times over (the cache rebuild runs in most rounds)
+    if ties == "zeros":     # -0 and +0 are equal: the lower index wins whatever the sign
+        l = torch.zeros(T, E)
+        l[torch.rand(T, E, generator=torch.Generator().manual_seed(3)) < 0.5] = -0.0
+        l[:, ::7] = -1.0
     st, want_idx, want_w = oracle.gate_topk(l.numpy(), K)
     assert st == oracle.OK
     idx = torch.full((T, K), -1, dtype=torch.int32, device=dev)
@@ -96,6 +107,24 @@ def test_gate_plan_matches_oracle_gate_then_oracle_plan(case):
     assert torch.equal(win.view(torch.int16), win_sep.view(torch.int16))
     assert torch.equal(y.view(torch.int16) & 0x7FFF, x.view(torch.int16) & 0x7FFF)
     comm.close()
+
+
+def test_gate_rows_that_do_not_start_on_16_bytes():
+    """The 16-byte row loads need an aligned row; any other pointer or row length takes scalar loads."""
+    dev = torch.device("cuda:0")
+    T, E, K = 300, 256, 8
+    l = logits_for(T, E, 99, True)
+    st, want_idx, want_w = oracle.gate_topk(l.numpy(), K)
+    buf = torch.zeros(T * E + 3, dtype=torch.float32, device=dev)
+    for off in (1, 2, 3):
+        shifted = buf[off:off + T * E].view(T, E)
+        shifted.copy_(l)
+        idx = torch.full((T, K), -1, dtype=torch.int32, device=dev)
+        w = torch.full((T, K), -1.0, dtype=torch.float32, device=dev)
+        assert binding.moe_gate_topk(shifted, K, idx, w) == binding.MOE_OK
+        torch.cuda.synchronize()
+        assert np.array_equal(idx.cpu().numpy(), want_idx)
+        assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
 
 
 def test_gate_argument_checks():
