@@ -47,7 +47,8 @@ typedef enum {
   MOE_ERR_CAPACITY = 3,    /* device-detected: some n_recv[d] > capacity_rows; nothing was written  */
   MOE_ERR_NOT_PLANNED = 4, /* dispatch / combine / slots / view before a successful moe_plan        */
   MOE_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired                                    */
-  MOE_ERR_CUDA = 6         /* a CUDA runtime call or kernel launch failed                           */
+  MOE_ERR_CUDA = 6,        /* a CUDA runtime call or kernel launch failed                           */
+  MOE_ERR_STALE_PEERS = 7  /* host-detected: the installed window address table is missing or out of date   */
 } moe_status_t;
 
 /* The two schedules of Section 4.  PREFILL runs Layout + Notify as separate
@@ -231,6 +232,58 @@ moe_status_t moe_combine_peers(moe_ctx_t* ctx, const void* const* window_bases /
 moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/,
                                       const void* const* window_q_bases /*DEVICE*/,
                                       float* const* scale_bases /*DEVICE*/, int64_t capacity_rows, void* stream);
+
+/* Window addresses of the expert-parallel group (Section 3.2: every rank's slice of the pooled memory is
+ * visible to every rank; Section 5.3, Decode Combine, and Section 6.1: remote window addresses are made
+ * available by an address handshake, or, in the cached-address mode, taken from an earlier exchange while
+ * that is still valid).  One process per rank; rank d's window is [capacity_rows, H] bf16 in its own GPU's
+ * memory.
+ *
+ *   moe_window_export   describes a window of THIS process for the other ranks: an inter-process handle of
+ *                       the allocation that holds it, the window's offset inside that allocation, the device,
+ *                       and a generation number chosen by the exporter, which must change whenever the rank
+ *                       exports a different window.  The result is plain bytes; the caller sends it to the
+ *                       other ranks over whatever channel it has (the binding uses the process group).
+ *   moe_peers_open      the address handshake: takes the R handles (entry my_rank is ignored; my_window is used
+ *                       for it), maps every other rank's window into this process (peer access over NVLink /
+ *                       PCIe is enabled by the mapping), and installs the R addresses and generations as the
+ *                       context's address table.  Mappings of an earlier handshake are released first.
+ *                       Synchronises `stream` before it releases or installs anything.
+ *   moe_peers_set       installs addresses the caller already has (separate allocations of one process, a
+ *                       symmetric-memory mapping, an earlier handshake of its own) without mapping anything:
+ *                       window_bases HOST [R] of DEVICE pointers, generations HOST [R] or NULL (all zero).
+ *   moe_peers_check     the cached-address test: MOE_OK if a table is installed and its generations equal
+ *                       `generations` (HOST [R], what the ranks announced for this call -- the binding sends each
+ *                       rank's generation along with its count row, so the test costs no exchange of its own);
+ *                       MOE_ERR_STALE_PEERS otherwise.
+ *   moe_dispatch_cached / moe_combine_cached
+ *                       as moe_dispatch_peers / moe_combine_peers with the installed table and its capacity.
+ *                       `generations` as in moe_peers_check (NULL: no test); with a stale or missing table they
+ *                       return MOE_ERR_STALE_PEERS and enqueue nothing -- no stale address is ever dereferenced.
+ *   moe_peers_close     synchronises `stream`, releases the mappings of moe_peers_open and forgets the table
+ *                       (also done by moe_destroy).
+ * Only this library's kernels touch the mapped windows: rows are stored to them with plain (non-multicast)
+ * bulk copies and read from them with ordinary loads.  The library still waits for no peer: the caller orders
+ * the phases (all ranks' dispatches complete before any expert reads; all experts complete before combine). */
+typedef struct {
+  unsigned char ipc[64]; /* inter-process memory handle of the allocation that holds the window */
+  int64_t offset;        /* first byte of the window inside that allocation                    */
+  int64_t bytes;         /* size of the window                                                 */
+  int32_t device;        /* device ordinal of the exporter                                     */
+  int32_t generation;    /* exporter's window generation                                       */
+} moe_window_handle_t;
+moe_status_t moe_window_export(const void* window /*DEVICE*/, int64_t bytes, int32_t generation,
+                               moe_window_handle_t* out /*HOST*/);
+moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles /*HOST [R]*/, int32_t my_rank,
+                            void* my_window /*DEVICE*/, int64_t capacity_rows, void* stream);
+moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases /*HOST [R]*/,
+                           const int32_t* generations /*HOST [R] or NULL*/, int64_t capacity_rows, void* stream);
+moe_status_t moe_peers_check(const moe_ctx_t* ctx, const int32_t* generations /*HOST [R]*/);
+moe_status_t moe_dispatch_cached(moe_ctx_t* ctx, const void* x /*DEVICE*/, const int32_t* generations /*HOST or NULL*/,
+                                 void* stream);
+moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations /*HOST or NULL*/,
+                                const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
+moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
 
 /* Materialises slot(t,j) into caller memory (parity checks, expert-side
  * consumers).  slots DEVICE [T,K] int32; needs R * capacity_rows < 2^31. */

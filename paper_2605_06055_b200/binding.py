@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmoecomm.so")
 
 MOE_OK, MOE_ERR_INVALID_ARG, MOE_ERR_BAD_INDEX, MOE_ERR_CAPACITY = 0, 1, 2, 3
-MOE_ERR_NOT_PLANNED, MOE_ERR_TIMEOUT, MOE_ERR_CUDA = 4, 5, 6
+MOE_ERR_NOT_PLANNED, MOE_ERR_TIMEOUT, MOE_ERR_CUDA, MOE_ERR_STALE_PEERS = 4, 5, 6, 7
 MOE_SCHED_PREFILL, MOE_SCHED_DECODE = 0, 1
 
 EXPORTS = [
@@ -27,6 +27,8 @@ EXPORTS = [
     "moe_slots_noalloc", "moe_set_option", "moe_dispatch_quant", "moe_expert_ranges",
     "moe_gate_topk", "moe_gate_plan", "moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers",
     "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant", "moe_expert_tiles", "moe_dispatch_quant_peers",
+    "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
+    "moe_dispatch_cached", "moe_combine_cached",
 ]
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
@@ -40,6 +42,15 @@ class MoeShape(ctypes.Structure):
 
 class MoePlanView(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("counts", "c_rank", "small_off", "large_off", "n_exp", "n_recv")]
+
+
+class MoeWindowHandle(ctypes.Structure):
+    """moe_window_handle_t: plain bytes describing one rank's window to the other ranks."""
+    _fields_ = [("ipc", ctypes.c_ubyte * 64), ("offset", ctypes.c_int64), ("bytes", ctypes.c_int64),
+                ("device", ctypes.c_int32), ("generation", ctypes.c_int32)]
+
+
+WINDOW_HANDLE_BYTES = ctypes.sizeof(MoeWindowHandle)
 
 
 class MoeError(RuntimeError):
@@ -96,6 +107,16 @@ def load() -> ctypes.CDLL:
     L.moe_dispatch_quant_peers.restype = ctypes.c_int
     L.moe_dispatch_quant.argtypes = [vp, vp, vp, vp, i64, vp]
     L.moe_dispatch_quant.restype = ctypes.c_int
+    L.moe_window_export.argtypes = [vp, i64, i32, ctypes.POINTER(MoeWindowHandle)]
+    L.moe_peers_open.argtypes = [vp, vp, i32, vp, i64, vp]
+    L.moe_peers_set.argtypes = [vp, vp, vp, i64, vp]
+    L.moe_peers_check.argtypes = [vp, vp]
+    L.moe_peers_close.argtypes = [vp, vp]
+    L.moe_dispatch_cached.argtypes = [vp, vp, vp, vp]
+    L.moe_combine_cached.argtypes = [vp, vp, vp, vp, vp]
+    for _n in ("moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
+               "moe_dispatch_cached", "moe_combine_cached"):
+        getattr(L, _n).restype = ctypes.c_int
     L.moe_slots.argtypes = [vp, i64, vp, vp]
     L.moe_forward_host.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     L.moe_status.argtypes = [vp, vp]
@@ -335,6 +356,60 @@ class MoeComm:
             raise MoeError(rc, "moe_combine_peers")
         return rc
 
+    # -- window addresses of the group: handshake and cached table ------------------------
+    def moe_peers_open(self, handles: bytes, my_rank: int, my_window: torch.Tensor, capacity_rows: int, stream=None,
+                       check: bool = True) -> int:
+        """handles: R exported handles back to back (R * WINDOW_HANDLE_BYTES bytes), entry r from rank r."""
+        assert len(handles) == self.R * WINDOW_HANDLE_BYTES
+        buf = ctypes.create_string_buffer(handles, len(handles))
+        with self._on_device():
+            rc = self.lib.moe_peers_open(self._h, ctypes.cast(buf, ctypes.c_void_p), my_rank,
+                                         _dev_ptr(my_window, torch.bfloat16), int(capacity_rows),
+                                         _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_peers_open")
+        return rc
+
+    def moe_peers_set(self, window_bases, generations, capacity_rows: int, stream=None, check: bool = True) -> int:
+        """window_bases: R device addresses (ints); generations: R ints or None."""
+        bases = np.ascontiguousarray(window_bases, dtype=np.uint64)
+        gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
+        assert bases.shape == (self.R,) and (gens is None or gens.shape == (self.R,))
+        with self._on_device():
+            rc = self.lib.moe_peers_set(self._h, _host_ptr(bases), _host_ptr(gens), int(capacity_rows),
+                                        _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_peers_set")
+        return rc
+
+    def moe_peers_check(self, generations) -> int:
+        gens = np.ascontiguousarray(generations, dtype=np.int32)
+        assert gens.shape == (self.R,)
+        return int(self.lib.moe_peers_check(self._h, _host_ptr(gens)))
+
+    def moe_peers_close(self, stream=None) -> int:
+        with self._on_device():
+            return int(self.lib.moe_peers_close(self._h, _stream_handle(stream)))
+
+    def moe_dispatch_cached(self, x: torch.Tensor, generations=None, stream=None, check: bool = True) -> int:
+        gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
+        with self._on_device():
+            rc = self.lib.moe_dispatch_cached(self._h, _dev_ptr(x, torch.bfloat16), _host_ptr(gens),
+                                              _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_cached")
+        return rc
+
+    def moe_combine_cached(self, generations, topk_w: torch.Tensor, y: torch.Tensor, stream=None,
+                           check: bool = True) -> int:
+        gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
+        with self._on_device():
+            rc = self.lib.moe_combine_cached(self._h, _host_ptr(gens), _dev_ptr(topk_w, torch.float32),
+                                             _dev_ptr(y, torch.bfloat16), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_combine_cached")
+        return rc
+
     def moe_plan_view(self) -> dict:
         """Zero-copy int32 tensors over the planning state in the workspace."""
         v = MoePlanView()
@@ -467,6 +542,17 @@ def moe_slots_noalloc(topk_idx: torch.Tensor, E: int, R: int, capacity_rows: int
                                             int(capacity_rows), _dev_ptr(slots, torch.int32),
                                             _dev_ptr(n_recv, torch.int32), _dev_ptr(status, torch.int32),
                                             _stream_handle(stream)))
+
+
+def moe_window_export(window: torch.Tensor, generation: int) -> bytes:
+    """Handle of one rank's window for the other ranks (see include/moecomm.h): WINDOW_HANDLE_BYTES plain bytes."""
+    h = MoeWindowHandle()
+    with torch.cuda.device(window.device):
+        rc = int(load().moe_window_export(_dev_ptr(window), window.numel() * window.element_size(), int(generation),
+                                          ctypes.byref(h)))
+    if rc != MOE_OK:
+        raise MoeError(rc, "moe_window_export")
+    return bytes(h)
 
 
 def moe_gate_topk(logits: torch.Tensor, K: int, topk_idx: torch.Tensor, topk_w: torch.Tensor, stream=None) -> int:

@@ -49,6 +49,13 @@ struct moe_ctx {
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
   cudaEvent_t fwd_events[2 * 16 + 2];
+  // window address table of the expert-parallel group (moe_peers_open / moe_peers_set)
+  const unsigned char** peer_table;   // device, [R] (inside the workspace)
+  void* peer_ptr[MOE_MAX_R];          // host copy of the installed addresses
+  void* peer_mapping[MOE_MAX_R];      // base of the inter-process mapping this context opened for rank d, or nullptr
+  int32_t peer_gen[MOE_MAX_R];
+  int64_t peer_capacity;
+  bool peers_installed;
   // resident CTAs per SM of the row kernels this context has launched (occupancy calculator results)
   const void* occ_kernel[16];
   int occ_per_sm[16];
@@ -80,7 +87,7 @@ int64_t max_tiles(const moe_shape_t* s) {
 }
 
 struct Layout {
-  size_t ctl, M, c_rank, o, n_exp, n_recv, s, tile_rank, tile_hist, total;
+  size_t ctl, M, c_rank, o, n_exp, n_recv, peers, s, tile_rank, tile_hist, total;
 };
 
 Layout layout_of(const moe_shape_t* s) {
@@ -98,6 +105,7 @@ Layout layout_of(const moe_shape_t* s) {
   L.o = take(sizeof(int32_t) * s->E * s->R);
   L.n_exp = take(sizeof(int32_t) * s->E);
   L.n_recv = take(sizeof(int32_t) * s->R);
+  L.peers = take(sizeof(void*) * s->R);
   L.s = take(sizeof(int32_t) * B);
   L.tile_rank = take(sizeof(int32_t) * B);
   L.tile_hist = take(sizeof(int32_t) * (size_t)max_tiles(s) * s->E);
@@ -310,9 +318,12 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
 template <int KT>
 void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const float* w, uint4* y, cudaStream_t st) {
   // Jobs that read several times the L2 capacity take the L1-allocating loads (see ld_row).
-  const bool large = (int64_t)a.t_count * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
-  auto kernel = large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), true>
-                      : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), false>;
+  // Windows addressed through a table of bases (other GPUs' memory) are read with coherent loads.
+  const bool peers = a.win_base != nullptr;
+  const bool large = !peers && (int64_t)a.t_count * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
+  auto kernel = peers ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_PEER>
+                : large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_L1>
+                        : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_STREAM>;
   const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * 8, 1 << 20, !large);   // the large-job form has no tail items
@@ -355,6 +366,14 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->o = reinterpret_cast<int32_t*>(ctx->ws + L.o);
   ctx->n_exp = reinterpret_cast<int32_t*>(ctx->ws + L.n_exp);
   ctx->n_recv = reinterpret_cast<int32_t*>(ctx->ws + L.n_recv);
+  ctx->peer_table = reinterpret_cast<const unsigned char**>(ctx->ws + L.peers);
+  ctx->peers_installed = false;
+  ctx->peer_capacity = 0;
+  for (int d = 0; d < MOE_MAX_R; ++d) {
+    ctx->peer_ptr[d] = nullptr;
+    ctx->peer_mapping[d] = nullptr;
+    ctx->peer_gen[d] = 0;
+  }
   ctx->s = reinterpret_cast<int32_t*>(ctx->ws + L.s);
   ctx->tile_rank = reinterpret_cast<int32_t*>(ctx->ws + L.tile_rank);
   ctx->tile_hist = reinterpret_cast<int32_t*>(ctx->ws + L.tile_hist);
@@ -440,6 +459,11 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
 
 moe_status_t moe_destroy(moe_ctx_t* ctx) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  for (int d = 0; d < ctx->shape.R; ++d)
+    if (ctx->peer_mapping[d] != nullptr) {
+      cudaIpcCloseMemHandle(ctx->peer_mapping[d]);
+      cudaGetLastError();
+    }
   if (ctx->out_stream != nullptr) {
     cudaStreamSynchronize(ctx->out_stream);
     cudaStreamSynchronize(ctx->in_stream);
@@ -897,6 +921,154 @@ moe_status_t moe_notify(moe_ctx_t* ctx, const int32_t* counts_all, void* stream)
   return rc;
 }
 
+/* ---------------------------------------------------------------------------------------------
+ * Window addresses of the expert-parallel group: export, handshake, cached table. */
+namespace {
+
+// Base and size of the device allocation that contains p.  The runtime API has no call for it, so the driver's
+// is looked up at run time (the library links no driver library and loads on a machine without one).
+bool allocation_range(const void* p, uintptr_t* base, size_t* size) {
+  typedef int (*range_fn)(unsigned long long*, size_t*, unsigned long long);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult found;
+  if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &fn, cudaEnableDefault, &found) != cudaSuccess || fn == nullptr ||
+      found != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  unsigned long long b = 0;
+  size_t n = 0;
+  if (reinterpret_cast<range_fn>(fn)(&b, &n, (unsigned long long)reinterpret_cast<uintptr_t>(p)) != 0) return false;
+  *base = (uintptr_t)b;
+  *size = n;
+  return true;
+}
+
+void release_mappings(moe_ctx* ctx) {
+  for (int d = 0; d < ctx->shape.R; ++d)
+    if (ctx->peer_mapping[d] != nullptr) {
+      cudaIpcCloseMemHandle(ctx->peer_mapping[d]);
+      cudaGetLastError();
+      ctx->peer_mapping[d] = nullptr;
+    }
+  ctx->peers_installed = false;
+}
+
+// Copies the host table to the device table on `stream` and marks it installed.
+moe_status_t install_table(moe_ctx* ctx, int64_t capacity_rows, cudaStream_t st) {
+  // pageable source: the runtime has staged the bytes by the time the call returns, so peer_ptr may change afterwards
+  if (cudaMemcpyAsync(ctx->peer_table, ctx->peer_ptr, sizeof(void*) * ctx->shape.R, cudaMemcpyHostToDevice, st) !=
+      cudaSuccess)
+    return MOE_ERR_CUDA;
+  ctx->peer_capacity = capacity_rows;
+  ctx->peers_installed = true;
+  return MOE_OK;
+}
+
+moe_status_t table_fresh(const moe_ctx* ctx, const int32_t* generations) {
+  if (!ctx->peers_installed) return MOE_ERR_STALE_PEERS;
+  if (generations != nullptr)
+    for (int d = 0; d < ctx->shape.R; ++d)
+      if (generations[d] != ctx->peer_gen[d]) return MOE_ERR_STALE_PEERS;
+  return MOE_OK;
+}
+
+}  // namespace
+
+moe_status_t moe_window_export(const void* window, int64_t bytes, int32_t generation, moe_window_handle_t* out) {
+  if (window == nullptr || out == nullptr || bytes <= 0 || !aligned16(window)) return MOE_ERR_INVALID_ARG;
+  static_assert(sizeof(cudaIpcMemHandle_t) == sizeof(out->ipc), "handle size");
+  uintptr_t base = 0;
+  size_t size = 0;
+  if (!allocation_range(window, &base, &size)) return MOE_ERR_CUDA;
+  const uintptr_t at = reinterpret_cast<uintptr_t>(window);
+  if (at < base || at + (uint64_t)bytes > base + size) return MOE_ERR_INVALID_ARG;   // the window spans allocations
+  cudaIpcMemHandle_t h;
+  if (cudaIpcGetMemHandle(&h, reinterpret_cast<void*>(base)) != cudaSuccess) {
+    cudaGetLastError();
+    return MOE_ERR_CUDA;
+  }
+  std::memcpy(out->ipc, &h, sizeof(h));
+  out->offset = (int64_t)(at - base);
+  out->bytes = bytes;
+  out->generation = generation;
+  if (cudaGetDevice(&out->device) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, int32_t my_rank, void* my_window,
+                            int64_t capacity_rows, void* stream) {
+  if (ctx == nullptr || handles == nullptr || my_window == nullptr || my_rank < 0 || my_rank >= ctx->shape.R ||
+      capacity_rows < 0 || !aligned16(my_window))
+    return MOE_ERR_INVALID_ARG;
+  const int64_t need = capacity_rows * ctx->shape.H * 2;
+  for (int d = 0; d < ctx->shape.R; ++d)
+    if (d != my_rank && (handles[d].bytes < need || (handles[d].offset & 15) != 0)) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;   // nothing in flight reads the old table
+  release_mappings(ctx);
+  for (int d = 0; d < ctx->shape.R; ++d) {
+    ctx->peer_gen[d] = handles[d].generation;
+    if (d == my_rank) {
+      ctx->peer_ptr[d] = my_window;
+      continue;
+    }
+    cudaIpcMemHandle_t h;
+    std::memcpy(&h, handles[d].ipc, sizeof(h));
+    void* base = nullptr;
+    if (cudaIpcOpenMemHandle(&base, h, cudaIpcMemLazyEnablePeerAccess) != cudaSuccess || base == nullptr) {
+      cudaGetLastError();
+      release_mappings(ctx);
+      return MOE_ERR_CUDA;
+    }
+    ctx->peer_mapping[d] = base;
+    ctx->peer_ptr[d] = static_cast<char*>(base) + handles[d].offset;
+  }
+  return install_table(ctx, capacity_rows, st);
+}
+
+moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, const int32_t* generations,
+                           int64_t capacity_rows, void* stream) {
+  if (ctx == nullptr || window_bases == nullptr || capacity_rows < 0) return MOE_ERR_INVALID_ARG;
+  for (int d = 0; d < ctx->shape.R; ++d)
+    if (window_bases[d] == nullptr || !aligned16(window_bases[d])) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
+  release_mappings(ctx);
+  for (int d = 0; d < ctx->shape.R; ++d) {
+    ctx->peer_ptr[d] = const_cast<void*>(window_bases[d]);
+    ctx->peer_gen[d] = generations != nullptr ? generations[d] : 0;
+  }
+  return install_table(ctx, capacity_rows, st);
+}
+
+moe_status_t moe_peers_check(const moe_ctx_t* ctx, const int32_t* generations) {
+  if (ctx == nullptr || generations == nullptr) return MOE_ERR_INVALID_ARG;
+  return table_fresh(ctx, generations);
+}
+
+moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return MOE_ERR_CUDA;
+  release_mappings(ctx);
+  return MOE_OK;
+}
+
+moe_status_t moe_dispatch_cached(moe_ctx_t* ctx, const void* x, const int32_t* generations, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  const moe_status_t fresh = table_fresh(ctx, generations);
+  if (fresh != MOE_OK) return fresh;
+  return dispatch_impl(ctx, x, nullptr, reinterpret_cast<const void* const*>(ctx->peer_table), ctx->peer_capacity, stream);
+}
+
+moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations, const float* topk_w, void* y, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  const moe_status_t fresh = table_fresh(ctx, generations);
+  if (fresh != MOE_OK) return fresh;
+  return combine_impl(ctx, nullptr, reinterpret_cast<const void* const*>(ctx->peer_table), ctx->peer_capacity, topk_w, y,
+                      stream);
+}
+
 moe_status_t moe_slots(moe_ctx_t* c, int64_t capacity_rows, int32_t* slots, void* stream) {
   moe_ctx* ctx = c;
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
@@ -1052,7 +1224,7 @@ moe_status_t moe_status(moe_ctx_t* ctx, void* stream) {
       ctx->layout_done = false;
     }
   }
-  return (word >= 0 && word <= MOE_ERR_CUDA) ? static_cast<moe_status_t>(word) : MOE_ERR_CUDA;
+  return (word >= 0 && word <= MOE_ERR_STALE_PEERS) ? static_cast<moe_status_t>(word) : MOE_ERR_CUDA;
 }
 
 const char* moe_status_string(moe_status_t status) {
@@ -1064,6 +1236,7 @@ const char* moe_status_string(moe_status_t status) {
     case MOE_ERR_NOT_PLANNED: return "no plan: call moe_plan first";
     case MOE_ERR_TIMEOUT: return "bounded device wait expired";
     case MOE_ERR_CUDA: return "CUDA error";
+    case MOE_ERR_STALE_PEERS: return "window address table missing or out of date";
   }
   return "unknown status";
 }

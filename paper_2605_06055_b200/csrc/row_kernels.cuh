@@ -140,23 +140,32 @@ __device__ __forceinline__ bool must_abort(const RowArgs& a) {
   return bad || over;
 }
 
-// 16-byte read-only load.  L1_ALLOC = false marks the line "no allocate" in L1 (streaming);
-// true lets it allocate.  Neither data is ever re-read, but measured on B200 the allocating form
-// is 3 % faster for combine at prefill sizes (617 vs 637 us) and 10 % slower at decode sizes
-// (55 vs 49 us), so the launcher picks by job size.
-template <bool L1_ALLOC>
+// 16-byte load of window / input rows, in three forms.
+// LD_STREAM, LD_L1: read-only (non-coherent) loads for rows of THIS GPU's memory, which nothing writes while the
+// kernel runs.  LD_STREAM marks the line "no allocate" in L1, LD_L1 lets it allocate.  Neither data is ever
+// re-read, but measured on B200 the allocating form is 3 % faster for combine at prefill sizes (617 vs 637 us)
+// and 10 % slower at decode sizes (55 vs 49 us), so the launcher picks by job size.
+// LD_PEER: ordinary (coherent) loads, for windows addressed through a table of bases -- other GPUs' memory that
+// other GPUs' kernels write.  They are valid whenever the reading kernel is ordered after the writers'
+// completion (a host barrier, or a preceding wait on arrival flags, followed by this launch), which the
+// non-coherent path does not promise once such ordering is established on the device.
+enum { LD_STREAM = 0, LD_L1 = 1, LD_PEER = 2 };
+template <int MODE>
 __device__ __forceinline__ uint4 ld_row(const uint4* p) {
   uint4 v;
-  if constexpr (L1_ALLOC)
+  if constexpr (MODE == LD_L1)
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  else if constexpr (MODE == LD_PEER)
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   else
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return ld_row<false>(p); }
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return ld_row<LD_STREAM>(p); }
 
 __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
   asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
@@ -330,8 +339,8 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float (&acc)[8]) {
   return make_uint4(u[0], u[1], u[2], u[3]);
 }
 
-// L1_ALLOC selects the large-job form: L1-allocating loads (see ld_row) and no finer-cut tail items.
-template <int KT, int UNROLL, bool L1_ALLOC>
+// MODE: how window rows are loaded (see ld_row).  LD_L1 is also the large-job form without finer-cut tail items.
+template <int KT, int UNROLL, int MODE>
 __global__ void __launch_bounds__(256, 1)
 combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__ topk_w, uint4* __restrict__ Y,
                     const RowArgs a, const __grid_constant__ RankMap map) {
@@ -345,15 +354,15 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
   ItemFeed feed = begin_feed();
   int32_t item = fetch_item(a, feed);
   BranchMeta meta = {-1, 0, 0.0f};
-  if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item<!L1_ALLOC>(a, item).t, lane);
+  if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item<MODE != LD_L1>(a, item).t, lane);
   while (item < a.n_items) {
     const int32_t next_item = fetch_item(a, feed);
-    const WorkItem wi = decode_item<!L1_ALLOC>(a, item);
+    const WorkItem wi = decode_item<MODE != LD_L1>(a, item);
     if (!a.prefetch_meta) meta = load_meta(a, topk_w, wi.t, lane);
     const int64_t slot = finish_slot(a, map, meta, wi.t, lane, false);
     const float w_lane = meta.w;
     // short rows: the next item's routing index, small offset and weight travel while this item is reduced
-    if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item<!L1_ALLOC>(a, next_item).t, lane);
+    if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item<MODE != LD_L1>(a, next_item).t, lane);
     item = next_item;
     uint4* out = Y + (size_t)wi.t * H16;
     if constexpr (KT > 0) {
@@ -374,7 +383,7 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
           ok[u] = (i + u < wi.i1) && (c < H16);
 #pragma unroll
           for (int j = 0; j < KT; ++j)
-            v[u][j] = (ok[u] && src[j] != nullptr) ? ld_row<L1_ALLOC>(src[j] + c) : make_uint4(0, 0, 0, 0);
+            v[u][j] = (ok[u] && src[j] != nullptr) ? ld_row<MODE>(src[j] + c) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -408,7 +417,7 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
                 (j < K && row >= 0) ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u)
-              v[u][jj] = (ok[u] && src != nullptr) ? ld_row<L1_ALLOC>(src + (i + u) * 32 + lane)
+              v[u][jj] = (ok[u] && src != nullptr) ? ld_row<MODE>(src + (i + u) * 32 + lane)
                                                    : make_uint4(0, 0, 0, 0);
           }
 #pragma unroll

@@ -1,83 +1,164 @@
-"""One expert-parallel rank per process: the host-side order of the multi-rank path.
+"""One expert-parallel rank per process (and per GPU): the host-side order of the multi-rank path.
 
-    layout (local)  ->  all-gather of the count rows  ->  notify  ->  dispatch into every rank's
-    window  ->  barrier  ->  experts  ->  barrier  ->  combine from every rank's window
+    layout (local)  ->  all-gather of the count rows (+ every rank's window generation)  ->  notify
+    ->  [address handshake, if the cached table is out of date]  ->  dispatch into every rank's window
+    ->  barrier  ->  experts  ->  barrier  ->  combine from every rank's window
 
-All compute is in libmoecomm (moe_layout, moe_notify, moe_dispatch_peers, moe_combine_peers); this
-module only exchanges the R x E count matrix with torch.distributed and keeps the phases in order.
-The windows of the other ranks must be mapped into this process (a table of R device addresses):
-`symmetric_windows` obtains them from torch's symmetric memory where that is available.
+All compute is in libmoecomm (moe_layout, moe_notify, moe_dispatch_cached, moe_combine_cached); this module
+exchanges the R x E count matrix and the window handles with torch.distributed and keeps the phases in order.
+Only the library's own kernels touch another rank's window; no torch op is ever given a peer address.
 
-The test suite exercises this on ONE GPU: every rank a context of one process with separate window
-allocations, and two ranks as two processes whose windows are mapped into each other over CUDA IPC
-(counts over a gloo group).  The count exchange is also tested with two gloo ranks on CPU.
+Window addresses (Section 5.3, Decode Combine; Section 6.1): every rank exports a handle of its window
+(moe_window_export); the handles are all-gathered and every rank maps the others' windows
+(moe_peers_open) -- the address handshake.  In the "cached" mode the handshake is repeated only when the
+cached table is out of date: every rank announces the generation of its window together with its count row,
+so the test rides on the exchange Notify needs anyway and costs no collective of its own.  In the "handshake"
+mode the addresses are exchanged before every dispatch.
+
+The test suite exercises this on ONE GPU (two processes whose windows are mapped into each other over CUDA
+inter-process handles, counts over a gloo group) and the exchange logic with two gloo ranks on CPU.
 """
 from __future__ import annotations
 
-from typing import Optional
-
+import numpy as np
 import torch
 import torch.distributed as dist
 
 from . import binding
 
 
-def all_gather_counts(counts_row: torch.Tensor, group=None) -> torch.Tensor:
-    """Prefill Notify's metadata exchange: every rank contributes its row [E] of the count matrix and
-    receives the whole matrix [R, E] (row r from rank r)."""
+def _staged(t: torch.Tensor, group) -> bool:
+    return t.is_cuda and dist.get_backend(group) == "gloo"     # gloo moves host tensors only
+
+
+def all_gather_rows(row: torch.Tensor, group=None) -> torch.Tensor:
+    """Every rank contributes one row and receives all of them, [R, len(row)], row r from rank r."""
     world = dist.get_world_size(group)
-    staged = counts_row.is_cuda and dist.get_backend(group) == "gloo"     # gloo moves host tensors only
-    src = counts_row.cpu() if staged else counts_row
+    staged = _staged(row, group)
+    src = row.cpu() if staged else row
     flat = torch.empty(world * src.numel(), dtype=src.dtype, device=src.device)
     dist.all_gather_into_tensor(flat, src.contiguous().view(-1), group=group)
     out = flat.view(world, src.numel())
-    return out.to(counts_row.device) if staged else out
+    return out.to(row.device) if staged else out
+
+
+def all_gather_counts(counts_row: torch.Tensor, group=None) -> torch.Tensor:
+    """Prefill Notify's metadata exchange: every rank contributes its row [E] of the count matrix and
+    receives the whole matrix [R, E] (row r from rank r)."""
+    return all_gather_rows(counts_row, group)
+
+
+def all_gather_bytes(mine: bytes, device, group=None) -> bytes:
+    """Every rank contributes len(mine) bytes (the same length everywhere) and receives all ranks' bytes back to
+    back in rank order.  `device`: where a device-only backend (NCCL) needs the staging tensor."""
+    src = torch.frombuffer(bytearray(mine), dtype=torch.uint8)
+    on_device = dist.get_backend(group) != "gloo"
+    if on_device:
+        src = src.to(device)
+    return bytes(all_gather_rows(src, group).cpu().reshape(-1).numpy().tobytes())
+
+
+def addresses_stale(table_generations, announced_generations) -> bool:
+    """The cached-address test: the table this rank holds was built from `table_generations`; the ranks have
+    just announced `announced_generations`.  None = no table yet."""
+    if table_generations is None:
+        return True
+    return not np.array_equal(np.asarray(table_generations, np.int32), np.asarray(announced_generations, np.int32))
 
 
 def symmetric_windows(capacity_rows: int, H: int, device, group=None):
-    """Allocates this rank's window in symmetric memory and returns (window, table of all ranks' window
-    addresses as an int64 CUDA tensor).  Needs torch's symmetric-memory support and peer access."""
+    """Alternative to the handle exchange where torch's symmetric memory is available: allocates this rank's
+    window there and returns (window, list of all ranks' window addresses) for moe_peers_set."""
     import torch.distributed._symmetric_memory as symm_mem
     win = symm_mem.empty((capacity_rows, H), dtype=torch.bfloat16, device=device)
     hdl = symm_mem.rendezvous(win, group if group is not None else dist.group.WORLD)
-    bases = torch.tensor([int(p) for p in hdl.buffer_ptrs], dtype=torch.int64, device=device)
-    return win, bases
+    return win, [int(p) for p in hdl.buffer_ptrs]
 
 
 class EpRank:
-    """The calls of one rank, in the order the schedules prescribe."""
+    """The calls of one rank, in the order the schedules prescribe.  mode: "cached" or "handshake"."""
 
-    def __init__(self, T_local_max: int, H: int, E: int, K: int, device, group=None):
-        self.group = group
+    def __init__(self, T_local_max: int, H: int, E: int, K: int, device, group=None, mode: str = "cached"):
+        assert mode in ("cached", "handshake")
+        self.group, self.mode, self.device = group, mode, device
         self.rank = dist.get_rank(group)
         self.R = dist.get_world_size(group)
+        self.E, self.H = E, H
         self.comm = binding.MoeComm(T_local_max, H, E, self.R, K, device)
-        self.counts_row = torch.zeros(E, dtype=torch.int32, device=device)
-        self.E = E
+        # what this rank sends in the metadata exchange: its count row [E], then its window generation [1]
+        self.message = torch.zeros(E + 1, dtype=torch.int32, device=device)
+        self.counts_row = self.message[:E]
+        self.window = None
+        self.capacity = 0
+        self.generation = 0                 # of this rank's own window; 0 = none attached
+        self.table_generations = None       # generations the installed address table was built from
+        self.announced = None               # generations gathered by the latest plan()
+        self.handshakes = 0
 
+    # -- windows -------------------------------------------------------------------------------------
+    def attach_window(self, window: torch.Tensor, capacity_rows: int) -> None:
+        """This rank's window from now on ([capacity_rows, H] bf16, the same capacity on every rank).  A new
+        window gets a new generation, which makes every rank's cached table stale at the next plan()."""
+        assert window.dtype == torch.bfloat16 and window.is_contiguous() and window.numel() >= capacity_rows * self.H
+        self.window, self.capacity = window, int(capacity_rows)
+        self.generation += 1
+        self.message[self.E:].fill_(self.generation)
+
+    def handshake(self) -> None:
+        """Collective: exchanges the window handles and maps every other rank's window."""
+        mine = binding.moe_window_export(self.window, self.generation)
+        handles = all_gather_bytes(mine, self.device, self.group)
+        gens = [binding.MoeWindowHandle.from_buffer_copy(handles, r * binding.WINDOW_HANDLE_BYTES).generation
+                for r in range(self.R)]
+        self.comm.moe_peers_open(handles, self.rank, self.window, self.capacity)
+        self.table_generations = np.asarray(gens, np.int32)
+        self.handshakes += 1
+
+    def install_addresses(self, window_bases, generations=None) -> None:
+        """Addresses obtained elsewhere (one process holding every window; symmetric memory)."""
+        gens = np.zeros(self.R, np.int32) if generations is None else np.asarray(generations, np.int32)
+        self.comm.moe_peers_set(window_bases, gens, self.capacity)
+        self.table_generations = gens
+
+    def _ensure_addresses(self) -> None:
+        # every rank holds the same table generations (handshakes are collective) and the same announcement,
+        # so every rank takes the same branch
+        if self.mode == "handshake" or addresses_stale(self.table_generations, self.announced):
+            self.handshake()
+
+    # -- the phases ------------------------------------------------------------------------------------
     def plan(self, schedule: int, topk_idx_local: torch.Tensor) -> torch.Tensor:
         self.comm.moe_layout(schedule, topk_idx_local, self.rank, self.counts_row)
-        counts_all = all_gather_counts(self.counts_row, self.group)      # metadata only, no payload
+        gathered = all_gather_rows(self.message, self.group)             # metadata only, no payload
+        counts_all = gathered[:, :self.E].contiguous()
+        self.announced = gathered[:, self.E].cpu().numpy().astype(np.int32)
         self.comm.moe_notify(counts_all)
         return counts_all
 
-    def dispatch(self, x_local: torch.Tensor, window_bases: torch.Tensor, capacity_rows: int) -> None:
-        self.comm.moe_dispatch_peers(x_local, window_bases, capacity_rows)
+    def dispatch(self, x_local: torch.Tensor) -> None:
+        self._ensure_addresses()
+        self.comm.moe_dispatch_cached(x_local, self.announced)
         torch.cuda.current_stream().synchronize()
         dist.barrier(self.group)                 # every rank's rows have landed before any expert reads its window
+
+    def combine(self, topk_w_local: torch.Tensor, y_local: torch.Tensor) -> None:
+        torch.cuda.current_stream().synchronize()
+        dist.barrier(self.group)                 # every expert has written its outputs
+        self.comm.moe_combine_cached(self.announced, topk_w_local, y_local)
 
     def dispatch_quant(self, x_local: torch.Tensor, window_q_bases: torch.Tensor, scale_bases: torch.Tensor,
                        capacity_rows: int) -> None:
         """Row-wise quantised dispatch: e4m3 codes into every rank's code window, one fp32 scale per row into
-        every rank's scale tensor (tables of R device addresses each)."""
+        every rank's scale tensor (tables of R device addresses each, supplied by the caller)."""
         self.comm.moe_dispatch_quant_peers(x_local, window_q_bases, scale_bases, capacity_rows)
         torch.cuda.current_stream().synchronize()
         dist.barrier(self.group)
 
-    def combine(self, window_bases: torch.Tensor, capacity_rows: int, topk_w_local: torch.Tensor,
-                y_local: torch.Tensor) -> None:
-        dist.barrier(self.group)                 # every expert has written its outputs
-        self.comm.moe_combine_peers(window_bases, capacity_rows, topk_w_local, y_local)
-
     def status(self) -> int:
         return self.comm.moe_status()
+
+    def close(self) -> None:
+        torch.cuda.current_stream().synchronize()
+        dist.barrier(self.group)                 # nobody unmaps a window another rank may still read
+        self.comm.moe_peers_close()
+        self.comm.close()

@@ -108,3 +108,48 @@ def test_two_ranks_layout_exchange_notify_reproduce_the_global_plan():
         assert o == whole.o.tolist() and n_recv == whole.n_recv.tolist()
         assert s_local == whole.s[lo:lo + counts[rank]].tolist()   # Layout is local
         lo += counts[rank]
+
+
+def _address_protocol_worker(rank, world, port, out):
+    """The address side of the multi-rank protocol on CPU: every step the ranks announce their window generation
+    along with their count row, decide from it whether the cached address table is still valid, and exchange
+    handles (plain bytes) only when it is not."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import numpy as np
+    from paper_2605_06055_b200 import ep
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    E = 5
+    generation, table, log = 1, None, []
+    for step in range(5):
+        if step == 3 and rank == 1:
+            generation += 1                                      # this rank moved its window
+        message = torch.cat([torch.full((E,), 10 * rank + step, dtype=torch.int32),
+                             torch.tensor([generation], dtype=torch.int32)])
+        gathered = ep.all_gather_rows(message)
+        counts, announced = gathered[:, :E], gathered[:, E].numpy()
+        assert counts.tolist() == [[10 * r + step] * E for r in range(world)]
+        stale = ep.addresses_stale(table, announced)
+        if stale:                                                # the handshake: handles are opaque bytes
+            mine = bytes([rank, generation]) + bytes(86)
+            handles = ep.all_gather_bytes(mine, torch.device("cpu"))
+            assert len(handles) == 88 * world
+            table = np.array([handles[88 * r + 1] for r in range(world)], np.int32)
+            assert [handles[88 * r] for r in range(world)] == list(range(world))
+        log.append((bool(stale), announced.tolist(), table.tolist()))
+    out[rank] = log
+    dist.destroy_process_group()
+
+
+def test_cached_addresses_are_re_exchanged_only_when_a_generation_changes():
+    from paper_2605_06055_b200 import ep
+    assert ep.addresses_stale(None, [1, 1])
+    assert not ep.addresses_stale([1, 2], [1, 2])
+    assert ep.addresses_stale([1, 2], [1, 3]) and ep.addresses_stale([1, 2], [2, 2])
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_address_protocol_worker, args=(world, 36000 + os.getpid() % 2000, out), nprocs=world, join=True)
+        logs = dict(out)
+    assert logs[0] == logs[1]                                    # every rank takes the same decisions
+    assert [s for s, _, _ in logs[0]] == [True, False, False, True, False]
+    assert logs[0][2][2] == [1, 1] and logs[0][4][2] == [1, 2]

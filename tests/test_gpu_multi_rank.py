@@ -119,11 +119,86 @@ def test_quantised_dispatch_into_per_rank_windows(case):
         c.close()
 
 
-# ------------------------------------------------------------------ two processes, windows shared over CUDA IPC
-def _ipc_rank(rank, world, port, q_to, results):
-    """One expert-parallel rank as its own process on the one GPU: its window lives in its own
-    allocation, the other rank's window is mapped in over CUDA IPC, counts travel over a gloo group,
-    phases are ordered by host barriers (no kernel waits on another process's kernel)."""
+def test_installed_address_table_and_generation_stamp_in_one_process():
+    """moe_peers_set / moe_dispatch_cached / moe_combine_cached with every rank a context of this process: the
+    installed table gives the same bytes as passing the table with every call; a stamp that does not match the
+    installed generations is refused before anything is enqueued; a re-installed table takes effect."""
+    name, T, H, E, R, K, sch, routing, per = CASES[1]
+    dev = torch.device("cuda:0")
+    wl = Workload(name, T, H, E, R, K, sch, routing, "scale", 7000 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    rts = inp.rank_tok_start
+    p = oracle.plan(inp.topk_idx.numpy(), E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    want = harness.oracle_run(inp, C)
+    idx, w, X = inp.topk_idx.to(dev), inp.topk_w.to(dev), inp.X.to(dev)
+    comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
+    counts = torch.zeros((R, E), dtype=torch.int32, device=dev)
+    for r, c in enumerate(comms):
+        c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, counts[r])
+    for c in comms:
+        c.moe_notify(counts)
+    fill = lambda: torch.from_numpy(np.full((C, H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    u16 = lambda ts: torch.cat(ts).cpu().view(torch.int16).numpy().view(np.uint16)
+    windows = [fill() for _ in range(R)]
+    gens = np.arange(1, R + 1, dtype=np.int32)
+    xs = [X[rts[r]:rts[r + 1]].contiguous() for r in range(R)]
+    for r, c in enumerate(comms):
+        assert c.moe_dispatch_cached(xs[r], gens, check=False) == binding.MOE_ERR_STALE_PEERS     # nothing installed
+        assert c.moe_peers_check(gens) == binding.MOE_ERR_STALE_PEERS
+        c.moe_peers_set([t.data_ptr() for t in windows], gens, C)
+        assert c.moe_peers_check(gens) == binding.MOE_OK
+        stale = gens.copy()
+        stale[(r + 1) % R] += 1
+        assert c.moe_dispatch_cached(xs[r], stale, check=False) == binding.MOE_ERR_STALE_PEERS
+        assert c.moe_status() == 0
+    assert (u16(windows) == harness.CANARY).all()               # every refusal left the windows alone
+    for r, c in enumerate(comms):
+        c.moe_dispatch_cached(xs[r], gens)
+        assert c.moe_status() == 0
+    assert np.array_equal(u16(windows), want.windows)
+    # the windows move to new allocations: new table, new generations; the old stamp is refused
+    windows2 = [fill() for _ in range(R)]
+    gens2 = gens + 10
+    for r, c in enumerate(comms):
+        c.moe_peers_set([t.data_ptr() for t in windows2], gens2, C)
+        assert c.moe_dispatch_cached(xs[r], gens, check=False) == binding.MOE_ERR_STALE_PEERS
+        c.moe_dispatch_cached(xs[r], gens2)
+        assert c.moe_status() == 0
+    assert np.array_equal(u16(windows2), want.windows)
+    allwin = torch.cat(windows2)
+    harness.gpu_expert_scale(allwin, idx, E, R, C, inp.scale.to(dev))
+    for d in range(R):
+        windows2[d].copy_(allwin[d * C:(d + 1) * C])
+    Y = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
+    for r, c in enumerate(comms):
+        y_r = torch.empty((int(rts[r + 1] - rts[r]), H), dtype=torch.bfloat16, device=dev)
+        assert c.moe_combine_cached(gens, w[rts[r]:rts[r + 1]].contiguous(), y_r, check=False) == binding.MOE_ERR_STALE_PEERS
+        c.moe_combine_cached(gens2, w[rts[r]:rts[r + 1]].contiguous(), y_r)
+        assert c.moe_status() == 0
+        Y[rts[r]:rts[r + 1]] = y_r
+    assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
+    for c in comms:
+        assert c.moe_peers_close() == binding.MOE_OK
+        assert c.moe_peers_check(gens2) == binding.MOE_ERR_STALE_PEERS
+        c.close()
+
+
+# ------------------------------------------------------------------ two processes, windows mapped into each other
+IPC_SHAPE = dict(T=600, H=512, E=16, K=4, per=(250, 350), seed=7300)
+
+
+def _ipc_workload(world):
+    c = IPC_SHAPE
+    return Workload("ipc", c["T"], c["H"], c["E"], world, c["K"], DECODE, "uniform", "identity", c["seed"],
+                    rank_tokens=c["per"])
+
+
+def _ipc_rank(rank, world, port, mode, q_to, results):
+    """One expert-parallel rank as its own process on the one GPU: its window lives in its own allocation, the
+    other rank's window is mapped in through the library's handle exchange (moe_window_export over a gloo group,
+    moe_peers_open), counts travel over the same group, phases are ordered by host barriers (no kernel waits on
+    another process's kernel)."""
     import os
     import torch.distributed as dist
     from paper_2605_06055_b200 import ep
@@ -132,24 +207,73 @@ def _ipc_rank(rank, world, port, q_to, results):
         dev = torch.device("cuda:0")
         torch.cuda.set_device(dev)
         dist.init_process_group("gloo", rank=rank, world_size=world)
-        T, H, E, K = 600, 512, 16, 4
-        wl = Workload("ipc", T, H, E, world, K, DECODE, "uniform", "identity", 7300, rank_tokens=(250, 350))
+        wl = _ipc_workload(world)
+        T, H, E, K = wl.T, wl.H, wl.E, wl.K
         inp = synth.make_inputs(wl)
         rts = inp.rank_tok_start
         lo, hi = int(rts[rank]), int(rts[rank + 1])
-        me = ep.EpRank(hi - lo, H, E, K, dev)
-        me.plan(DECODE, inp.topk_idx[lo:hi].contiguous().to(dev))
+        idx, x, w = (inp.topk_idx[lo:hi].contiguous().to(dev), inp.X[lo:hi].contiguous().to(dev),
+                     inp.topk_w[lo:hi].contiguous().to(dev))
+        me = ep.EpRank(hi - lo, H, E, K, dev, mode=mode)
+        me.plan(DECODE, idx)                               # first plan: learn the capacity the windows need
         C = int(me.comm.moe_plan_view()["n_recv"].max().item()) + 1
-        mine = torch.from_numpy(np.full((C, H), harness.CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
-        q_to[1 - rank].put(mine)                       # the other process maps this allocation (CUDA IPC)
-        other = q_to[rank].get(timeout=60)
-        wins = [mine, other] if rank == 0 else [other, mine]
-        bases = torch.tensor([w.data_ptr() for w in wins], dtype=torch.int64, device=dev)
-        me.dispatch(inp.X[lo:hi].contiguous().to(dev), bases, C)
+        log = {}
+        # nothing installed yet: the cached calls refuse instead of dereferencing anything
+        log["refused_without_table"] = me.comm.moe_dispatch_cached(x, me.announced, check=False)
+        # every window is a slice of a backing allocation of its own (large enough that the caching allocator
+        # gives it a device allocation to itself): the exported handle names that allocation, plus an offset
+        def new_window(offset_rows):
+            backing = torch.empty(12 << 20, dtype=torch.bfloat16, device=dev)
+            win = backing[offset_rows * H:(offset_rows + C) * H].view(C, H)
+            win.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+            return backing, win
+        backing, mine = new_window(0)
+        me.attach_window(mine, C)
         y = torch.empty((hi - lo, H), dtype=torch.bfloat16, device=dev)
-        me.combine(bases, C, inp.topk_w[lo:hi].contiguous().to(dev), y)
-        st = me.status()
-        # the quantising dispatch into per-process code windows and scale tensors, mapped the same way
+        u16 = lambda t: t.cpu().view(torch.int16).numpy().view(np.uint16).copy()
+
+        def step():
+            me.plan(DECODE, idx)
+            me.dispatch(x)
+            me.combine(w, y)
+            return me.status()
+
+        st = step()                                        # first step: the handshake happens here in both modes
+        log["handshakes_after_step_1"] = me.handshakes
+        win_1, y_1 = u16(mine), u16(y)
+        dist.barrier()                                     # both have read their windows before anyone refills
+        mine.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+        torch.cuda.synchronize()
+        dist.barrier()
+        st = st or step()                                  # same windows: the cached mode exchanges nothing
+        log["handshakes_after_step_2"] = me.handshakes
+        win_2, y_2 = u16(mine), u16(y)
+        # a stale stamp is refused and nothing is enqueued: rows stay as they are
+        wrong = me.announced.copy()
+        wrong[1 - rank] += 5
+        before = u16(mine)
+        log["refused_stale"] = me.comm.moe_dispatch_cached(x, wrong, check=False)
+        log["refused_stale_combine"] = me.comm.moe_combine_cached(wrong, w, y, check=False)
+        log["check_fresh"] = me.comm.moe_peers_check(me.announced)
+        log["check_stale"] = me.comm.moe_peers_check(wrong)
+        torch.cuda.synchronize()
+        dist.barrier()
+        log["untouched_after_refusal"] = bool(np.array_equal(u16(mine), before))
+        # rank 1 moves its window to a new allocation: every rank's table is stale at the next plan
+        dist.barrier()
+        if rank == 1:
+            keep_old = backing                         # stays mapped on the other rank until its next handshake
+            backing, mine = new_window(8)              # the new window starts 8 rows into its allocation
+            me.attach_window(mine, C)
+        else:
+            mine.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+        torch.cuda.synchronize()
+        dist.barrier()
+        st = st or step()
+        log["handshakes_after_step_3"] = me.handshakes
+        win_3, y_3 = u16(mine), u16(y)
+        # the quantising dispatch into per-process code windows and scale tensors, mapped through torch's own
+        # inter-process tensors (tables supplied by the caller)
         my_q = torch.full((C, H), 0xAB, dtype=torch.uint8, device=dev)
         my_s = torch.full((C,), -1.0, dtype=torch.float32, device=dev)
         q_to[1 - rank].put((my_q, my_s))
@@ -158,31 +282,33 @@ def _ipc_rank(rank, world, port, q_to, results):
         ss = [my_s, other_s] if rank == 0 else [other_s, my_s]
         q_bases = torch.tensor([t.data_ptr() for t in qs], dtype=torch.int64, device=dev)
         s_bases = torch.tensor([t.data_ptr() for t in ss], dtype=torch.int64, device=dev)
-        me.dispatch_quant(inp.X[lo:hi].contiguous().to(dev), q_bases, s_bases, C)
+        me.dispatch_quant(x, q_bases, s_bases, C)
         st = st or me.status()
         dist.barrier()                                 # nobody frees a window another rank may still read
-        results[rank] = ("ok", st, C, mine.cpu().view(torch.int16).numpy().view(np.uint16).copy(),
-                         y.cpu().view(torch.int16).numpy().view(np.uint16).copy(), my_q.cpu().numpy().copy(),
-                         my_s.cpu().numpy().copy())
+        results[rank] = ("ok", st, C, (win_1, y_1), (win_2, y_2), (win_3, y_3), my_q.cpu().numpy().copy(),
+                         my_s.cpu().numpy().copy(), log)
+        me.close()
         dist.barrier()
         dist.destroy_process_group()
     except Exception as exc:                           # reported to the parent, which decides between skip and fail
-        results[rank] = ("error", repr(exc))
+        import traceback
+        results[rank] = ("error", repr(exc) + "\n" + traceback.format_exc())
 
 
-def test_two_processes_exchange_rows_through_ipc_mapped_windows():
+@pytest.mark.parametrize("mode", ["cached", "handshake"])
+def test_two_processes_exchange_rows_through_mapped_windows(mode):
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     world = 2
     with ctx.Manager() as m:
         results = m.dict()
         q_to = [ctx.Queue(), ctx.Queue()]
-        procs = [ctx.Process(target=_ipc_rank, args=(r, world, 35000 + os.getpid() % 2000, q_to, results))
-                 for r in range(world)]
+        port = 35000 + (os.getpid() * 2 + (mode == "cached")) % 2000
+        procs = [ctx.Process(target=_ipc_rank, args=(r, world, port, mode, q_to, results)) for r in range(world)]
         for p_ in procs:
             p_.start()
         for p_ in procs:
-            p_.join(timeout=180)
+            p_.join(timeout=240)
         alive = [p_ for p_ in procs if p_.is_alive()]
         for p_ in alive:
             p_.terminate()
@@ -192,8 +318,8 @@ def test_two_processes_exchange_rows_through_ipc_mapped_windows():
     if errors and any("ipc" in e[1].lower() or "not supported" in e[1].lower() for e in errors):
         pytest.skip("CUDA IPC is not available here: " + errors[0][1])
     assert not errors and len(res) == world, res
-    T, H, E, K = 600, 512, 16, 4
-    wl = Workload("ipc", T, H, E, world, K, DECODE, "uniform", "identity", 7300, rank_tokens=(250, 350))
+    wl = _ipc_workload(world)
+    H = wl.H
     inp = synth.make_inputs(wl)
     C = res[0][2]
     assert res[1][2] == C
@@ -203,9 +329,19 @@ def test_two_processes_exchange_rows_through_ipc_mapped_windows():
     want_s = np.full((world * C,), -1.0, np.float32)
     assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 2) == oracle.OK
     for r in range(world):
-        _, st, _, win, y, q, sc = res[r]
+        _, st, _, s1, s2, s3, q, sc, log = res[r]
         assert st == 0
-        assert np.array_equal(win, want.windows[r * C:(r + 1) * C])            # rows from both processes, bit-exact
-        assert harness.max_ulp_diff(y, want.Y[int(rts[r]):int(rts[r + 1])]) <= 1
+        for (win, y) in (s1, s2, s3):
+            assert np.array_equal(win, want.windows[r * C:(r + 1) * C])        # rows from both processes, bit-exact
+            assert harness.max_ulp_diff(y, want.Y[int(rts[r]):int(rts[r + 1])]) <= 1
         assert np.array_equal(q, want_q[r * C:(r + 1) * C])
         assert np.array_equal(sc.view(np.uint32), want_s[r * C:(r + 1) * C].view(np.uint32))
+        assert log["refused_without_table"] == binding.MOE_ERR_STALE_PEERS
+        assert log["refused_stale"] == binding.MOE_ERR_STALE_PEERS
+        assert log["refused_stale_combine"] == binding.MOE_ERR_STALE_PEERS
+        assert log["check_fresh"] == binding.MOE_OK and log["check_stale"] == binding.MOE_ERR_STALE_PEERS
+        assert log["untouched_after_refusal"]
+        if mode == "cached":      # one handshake for the first step, none for the second, one after the move
+            assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 1, 2)
+        else:                     # the handshake mode exchanges addresses before every dispatch
+            assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 2, 3)
