@@ -516,6 +516,123 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
     return out
 
 
+# ----------------------------------------------------------------------------- expert-parallel leg (world > 1)
+def _group_reduce(value: float, op, dev, group=None) -> float:
+    import torch.distributed as dist
+    on_host = dist.get_backend(group) == "gloo"
+    t = torch.tensor([value], dtype=torch.float64, device="cpu" if on_host else dev)
+    dist.all_reduce(t, op=op, group=group)
+    return float(t.item())
+
+
+def ep_shape(key: str, R: int):
+    """The decode and prefill shapes with the ranks mapped to processes: 128 / 4096 tokens per rank."""
+    per_rank, sched = (128, synth.DECODE) if key == "decode" else (4096, synth.PREFILL)
+    return synth.Workload(f"ep_{key}_dsv3", per_rank * R, 7168, 256, R, 8, sched, "uniform", "identity", 1300 + R)
+
+
+def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"), modes=("cached", "handshake")) -> dict:
+    """The path with rank = process = GPU: every process plans its own tokens, the count rows (and window
+    generations) are all-gathered over the process group, every rank's window is mapped into every process
+    (moe_window_export / moe_peers_open), dispatch stores rows into the other GPUs' windows and combine loads
+    them from there.  Only the library's kernels touch peer memory.  Before anything is timed, every rank checks
+    its window against the single-GPU path run on the whole batch with R virtual ranks (the path the parity
+    tests compare with the CPU definition) and its output against the identity Y == X.  Phases are ordered by
+    host barriers; the step time is device time from the first to the last event of a step (idle gaps included),
+    max over ranks."""
+    import torch.distributed as dist
+    from paper_2605_06055_b200 import binding, ep
+    rank, R = dist.get_rank(group), dist.get_world_size(group)
+    out = {"ranks": R, "ordering": "host barriers between phases (stream synchronize + process-group barrier)",
+           "peer_access": "windows mapped through inter-process handles; plain bulk stores and coherent loads"}
+    if 256 % R != 0:
+        out["unavailable"] = f"256 experts do not divide over {R} ranks"
+        return out
+    for key in shapes:
+        wl = ep_shape(key, R)
+        inp = synth.make_inputs(wl)               # every rank draws the same batch from the seed and takes its slice
+        lo, hi = rank * (wl.T // R), (rank + 1) * (wl.T // R)
+        idx, w, X = (inp.topk_idx[lo:hi].contiguous().to(dev), inp.topk_w[lo:hi].contiguous().to(dev),
+                     inp.X[lo:hi].contiguous().to(dev))
+        Y = torch.empty_like(X)
+        res = {"config": describe(wl), "tokens_per_rank": wl.T // R}
+        # reference windows: the single-GPU path on the whole batch, R virtual ranks
+        ref = binding.MoeComm(wl.T, wl.H, wl.E, R, wl.K, dev)
+        g_idx, g_X = inp.topk_idx.to(dev), inp.X.to(dev)
+        ref.moe_plan(wl.schedule, g_idx)
+        assert ref.moe_status() == 0
+        C = (int(ref.moe_plan_view()["n_recv"].max().item()) + 7) // 8 * 8
+        ref_win = torch.zeros((R * C, wl.H), dtype=torch.bfloat16, device=dev)
+        ref.moe_dispatch(g_X, ref_win, C)
+        assert ref.moe_status() == 0
+        mine_ref = ref_win[rank * C:(rank + 1) * C].clone()
+        del ref_win, g_X, g_idx
+        ref.close()
+        for mode in modes:
+            me = ep.EpRank(wl.T // R, wl.H, wl.E, wl.K, dev, group, mode=mode)
+            window = torch.zeros((C, wl.H), dtype=torch.bfloat16, device=dev)
+            me.attach_window(window, C)
+            ok, why = 1.0, ""
+            try:
+                me.plan(wl.schedule, idx)
+                me.handshake()
+            except Exception as exc:      # e.g. no peer access between two of the GPUs
+                ok, why = 0.0, repr(exc)
+            if _group_reduce(ok, dist.ReduceOp.MIN, dev, group) < 1.0:
+                res[mode] = {"unavailable": why or "the address handshake failed on another rank"}
+                continue
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(steps)]
+
+            def step(e=None):
+                if e is not None:
+                    e[0].record()
+                me.plan(wl.schedule, idx)
+                if e is not None:
+                    e[1].record()
+                me._ensure_addresses()
+                if e is not None:
+                    e[2].record()
+                me.comm.moe_dispatch_cached(X, me.announced)
+                if e is not None:
+                    e[3].record()
+                torch.cuda.current_stream().synchronize()
+                dist.barrier(group)
+                if e is not None:
+                    e[4].record()
+                me.comm.moe_combine_cached(me.announced, w, Y)
+                if e is not None:
+                    e[5].record()
+                torch.cuda.current_stream().synchronize()
+                dist.barrier(group)        # nobody starts the next dispatch while a rank still reads
+
+            step()
+            assert me.status() == 0
+            same_window = bool(torch.equal(window.view(torch.int16), mine_ref.view(torch.int16)))
+            same_output = bool(torch.equal(Y.view(torch.int16), X.view(torch.int16)))
+            agreed = _group_reduce(1.0 if (same_window and same_output) else 0.0, dist.ReduceOp.MIN, dev, group)
+            assert agreed == 1.0, f"expert-parallel leg ({key}, {mode}): rank {rank} window {same_window}, output {same_output}"
+            for _ in range(2):
+                step()
+            handshakes0 = me.handshakes
+            for e in ev:
+                step(e)
+            assert me.status() == 0
+            mean = lambda a, b: sum(e[a].elapsed_time(e[b]) for e in ev) / steps * 1e3
+            red = lambda v: _group_reduce(v, dist.ReduceOp.MAX, dev, group)
+            res[mode] = {"verified": {"window_equals_single_gpu_path": True, "Y_equals_X": True},
+                         "step_us": red(mean(0, 5)), "plan_and_count_exchange_us": red(mean(0, 1)),
+                         "address_step_us": red(mean(1, 2)), "dispatch_kernel_us": red(mean(2, 3)),
+                         "barrier_after_dispatch_us": red(mean(3, 4)), "combine_kernel_us": red(mean(4, 5)),
+                         "handshakes_in_timed_steps": me.handshakes - handshakes0, "steps": steps,
+                         "dispatch_bytes_per_rank": bytes_dispatch(wl) // R}
+            me.close()
+            del window
+        out[key] = res
+        del inp, X, Y, idx, w, mine_ref
+        torch.cuda.empty_cache()
+    return out
+
+
 def kernel_table(wl, r, peak):
     med = statistics.median
     mean = lambda v: sum(v) / len(v)
@@ -613,6 +730,13 @@ def run_cuda(args, wl):
         e2e = {"value": aggregate_value(bytes_step(wl), world, e2e_ms), "unit": "GB/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
     clocks = sampler.stop()
+    ep_result = None
+    if world > 1:
+        # the replicas' buffers are not needed any more; every rank takes part in the expert-parallel leg
+        try:
+            ep_result = ep_leg(dev, min(args.steps, 20))
+        except Exception as exc:           # reported in the line, the replica numbers stand
+            ep_result = {"ranks": world, "error": repr(exc)}
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -648,6 +772,9 @@ def run_cuda(args, wl):
         "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": r["launches"], "e2e": e2e,
         "verified": verified,
     }
+    if ep_result is not None:
+        ep_result["note"] = ("rank = GPU; reported beside the replica figures above, which remain `value`")
+        line["ep"] = ep_result
 
     cpu_inp = layer.inp
     del layer, scratch

@@ -404,7 +404,9 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   auto opt_in = [&](auto kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess;
   };
-  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2>) && opt_in(dispatch_quant_kernel<3>) && opt_in(plan_rank_kernel<32>) &&
+  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2, 16>) && opt_in(dispatch_quant_kernel<3, 16>) &&
+       opt_in(dispatch_quant_kernel<2, 32>) && opt_in(dispatch_quant_kernel<3, 32>) &&
+       opt_in(dispatch_quant_kernel<2, 0>) && opt_in(dispatch_quant_kernel<3, 0>) && opt_in(plan_rank_kernel<32>) &&
        opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
        opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
@@ -779,9 +781,13 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   const int upr = (a.H16 + 31) / 32;
   const int stage = (H * 2 + 127) / 128 * 128;
   const int grid = ctx->num_sms;
+  // 16-byte chunks of a row per lane: rows of up to 16 (8 KB) or 32 (16 KB) are held in registers, longer ones
+  // take the two-pass form; the 32-chunk form has registers for eight warps.
+  const int cpl = upr <= 16 ? 16 : upr <= 32 ? 32 : 0;
+  const int max_warps = cpl == 32 ? 8 : QUANT_MAX_WARPS;
   auto warps_for = [&](int stages) {
     int w = QUANT_SMEM_BUDGET / (stages * (stage + 8));
-    return w > QUANT_MAX_WARPS ? QUANT_MAX_WARPS : w;
+    return w > max_warps ? max_warps : w;
   };
   // Three stages once every warp of the two-stage configuration would see eight rows or more.
   const int stages = (warps_for(3) >= 1 && (int64_t)ctx->T >= (int64_t)8 * grid * warps_for(2)) ? 3 : 2;
@@ -796,12 +802,19 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   const int smem = warps * stages * (stage + 8);
   const bool pdl = behind_plan && ctx->overlap != 0;
   a.pdl = pdl;
-  if (stages == 3)
-    launch_kernel(dispatch_quant_kernel<3>, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
+  auto launch = [&](auto kernel) {
+    launch_kernel(kernel, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
                   static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
-  else
-    launch_kernel(dispatch_quant_kernel<2>, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
-                  static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
+  };
+  if (stages == 3) {
+    if (cpl == 16) launch(dispatch_quant_kernel<3, 16>);
+    else if (cpl == 32) launch(dispatch_quant_kernel<3, 32>);
+    else launch(dispatch_quant_kernel<3, 0>);
+  } else {
+    if (cpl == 16) launch(dispatch_quant_kernel<2, 16>);
+    else if (cpl == 32) launch(dispatch_quant_kernel<2, 32>);
+    else launch(dispatch_quant_kernel<2, 0>);
+  }
   return launch_ok(ctx);
 }
 

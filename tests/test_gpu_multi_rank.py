@@ -345,3 +345,53 @@ def test_two_processes_exchange_rows_through_mapped_windows(mode):
             assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 1, 2)
         else:                     # the handshake mode exchanges addresses before every dispatch
             assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 2, 3)
+
+
+# ------------------------------------------------------------------ the benchmark's expert-parallel leg
+def _ep_leg_rank(rank, world, port, results):
+    import os
+    import torch.distributed as dist
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    try:
+        import bench
+        dev = torch.device("cuda:0")
+        torch.cuda.set_device(dev)
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        results[rank] = ("ok", bench.ep_leg(dev, 3, None, shapes=("decode",)))
+        dist.barrier()
+        dist.destroy_process_group()
+    except Exception as exc:
+        import traceback
+        results[rank] = ("error", repr(exc) + "\n" + traceback.format_exc())
+
+
+def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
+    """The code `bench.py --gpus N` runs for N > 1 (rank = process, windows mapped into each other), here as two
+    processes that share the one GPU and talk over gloo: it verifies its own windows and outputs before it times
+    anything, exchanges no addresses in the timed steps of the cached mode and one set per step in the handshake
+    mode."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    world = 2
+    with ctx.Manager() as m:
+        results = m.dict()
+        procs = [ctx.Process(target=_ep_leg_rank, args=(r, world, 37000 + os.getpid() % 2000, results))
+                 for r in range(world)]
+        for p_ in procs:
+            p_.start()
+        for p_ in procs:
+            p_.join(timeout=300)
+        alive = [p_ for p_ in procs if p_.is_alive()]
+        for p_ in alive:
+            p_.terminate()
+        assert not alive, "a rank did not finish"
+        res = dict(results)
+    assert all(v[0] == "ok" for v in res.values()) and len(res) == world, res
+    for r in range(world):
+        leg = res[r][1]
+        assert leg["ranks"] == 2 and "decode" in leg
+        for mode, want_handshakes in (("cached", 0), ("handshake", 3)):
+            got = leg["decode"][mode]
+            assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
+            assert got["handshakes_in_timed_steps"] == want_handshakes
+            assert got["step_us"] > 0 and got["dispatch_kernel_us"] > 0 and got["combine_kernel_us"] > 0

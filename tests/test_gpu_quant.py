@@ -27,6 +27,12 @@ CASES = [
     ("one_row", 2, 512, 4, 2, 2, DECODE, "uniform", None),
     ("K32", 40, 64, 64, 2, 32, DECODE, "uniform", None),
     ("many_rows_per_sm", 20000, 256, 32, 4, 4, PREFILL, "uniform", None),
+    # rows at the edges of the register forms: 16 chunks per lane (8 KB), one chunk more, 32 chunks (16 KB), one more
+    ("row_8k", 700, 4096, 8, 4, 2, DECODE, "uniform", None),
+    ("row_8k_plus", 300, 4096 + 16, 8, 4, 2, DECODE, "uniform", None),
+    ("row_16k", 300, 8192, 8, 4, 2, PREFILL, "uniform", None),
+    ("row_16k_plus", 200, 8192 + 16, 8, 2, 2, PREFILL, "uniform", None),
+    ("row_partial_last_chunk_group", 500, 3600, 16, 4, 4, DECODE, "uniform", None),
 ]
 
 
