@@ -531,19 +531,27 @@ def ep_shape(key: str, R: int):
     return synth.Workload(f"ep_{key}_dsv3", per_rank * R, 7168, 256, R, 8, sched, "uniform", "identity", 1300 + R)
 
 
-def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"), modes=("cached", "handshake")) -> dict:
+def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
+           variants=(("cached", "host"), ("handshake", "host"), ("cached", "device"))) -> dict:
     """The path with rank = process = GPU: every process plans its own tokens, the count rows (and window
     generations) are all-gathered over the process group, every rank's window is mapped into every process
     (moe_window_export / moe_peers_open), dispatch stores rows into the other GPUs' windows and combine loads
     them from there.  Only the library's kernels touch peer memory.  Before anything is timed, every rank checks
     its window against the single-GPU path run on the whole batch with R virtual ranks (the path the parity
-    tests compare with the CPU definition) and its output against the identity Y == X.  Phases are ordered by
-    host barriers; the step time is device time from the first to the last event of a step (idle gaps included),
-    max over ranks."""
+    tests compare with the CPU definition) and its output against the identity Y == X.
+    Variants: (address mode, phase order).  Address mode "cached" exchanges window addresses only when a rank's
+    window generation changes, "handshake" before every dispatch.  Phase order "host" separates the phases by a
+    stream synchronisation and a process-group barrier, "device" by arrival flags in the windows' state regions
+    (moe_signal_peers / moe_wait_peers) with no host synchronisation between the phases -- unless ranks share a
+    GPU, where a host barrier is placed between signal and wait (a wait kernel must not hold a GPU that the
+    signalling rank needs).  Times are device time between CUDA events (idle gaps included), max over ranks."""
     import torch.distributed as dist
     from paper_2605_06055_b200 import binding, ep
     rank, R = dist.get_rank(group), dist.get_world_size(group)
-    out = {"ranks": R, "ordering": "host barriers between phases (stream synchronize + process-group barrier)",
+    where = ep.all_gather_bytes(f"{os.uname().nodename}:{torch.cuda.get_device_properties(dev).uuid}".encode()
+                                .ljust(96)[:96], dev, group)
+    shared_gpu = len({where[96 * r:96 * (r + 1)] for r in range(R)}) < R
+    out = {"ranks": R, "ranks_share_a_gpu": shared_gpu,
            "peer_access": "windows mapped through inter-process handles; plain bulk stores and coherent loads"}
     if 256 % R != 0:
         out["unavailable"] = f"256 experts do not divide over {R} ranks"
@@ -568,10 +576,10 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"), modes=("ca
         mine_ref = ref_win[rank * C:(rank + 1) * C].clone()
         del ref_win, g_X, g_idx
         ref.close()
-        for mode in modes:
-            me = ep.EpRank(wl.T // R, wl.H, wl.E, wl.K, dev, group, mode=mode)
-            window = torch.zeros((C, wl.H), dtype=torch.bfloat16, device=dev)
-            me.attach_window(window, C)
+        for mode, sync in variants:
+            name = f"{mode}_addresses__{sync}_phase_order"
+            me = ep.EpRank(wl.T // R, wl.H, wl.E, wl.K, dev, group, mode=mode, sync=sync, host_fence=shared_gpu)
+            window = me.new_window(C)             # rows + zeroed state region, attached
             ok, why = 1.0, ""
             try:
                 me.plan(wl.schedule, idx)
@@ -579,9 +587,9 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"), modes=("ca
             except Exception as exc:      # e.g. no peer access between two of the GPUs
                 ok, why = 0.0, repr(exc)
             if _group_reduce(ok, dist.ReduceOp.MIN, dev, group) < 1.0:
-                res[mode] = {"unavailable": why or "the address handshake failed on another rank"}
+                res[name] = {"unavailable": why or "the address handshake failed on another rank"}
                 continue
-            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(steps)]
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
 
             def step(e=None):
                 if e is not None:
@@ -589,28 +597,21 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"), modes=("ca
                 me.plan(wl.schedule, idx)
                 if e is not None:
                     e[1].record()
-                me._ensure_addresses()
+                me.dispatch(X)             # addresses (if stale), rows into every window, then the phase boundary
                 if e is not None:
                     e[2].record()
-                me.comm.moe_dispatch_cached(X, me.announced)
+                me.combine(w, Y)           # identity experts: the phase boundary, then rows from every window
                 if e is not None:
                     e[3].record()
-                torch.cuda.current_stream().synchronize()
-                dist.barrier(group)
-                if e is not None:
-                    e[4].record()
-                me.comm.moe_combine_cached(me.announced, w, Y)
-                if e is not None:
-                    e[5].record()
-                torch.cuda.current_stream().synchronize()
-                dist.barrier(group)        # nobody starts the next dispatch while a rank still reads
+                if sync == "host":
+                    me._host_barrier()     # nobody starts the next dispatch while a rank still reads
 
             step()
             assert me.status() == 0
             same_window = bool(torch.equal(window.view(torch.int16), mine_ref.view(torch.int16)))
             same_output = bool(torch.equal(Y.view(torch.int16), X.view(torch.int16)))
             agreed = _group_reduce(1.0 if (same_window and same_output) else 0.0, dist.ReduceOp.MIN, dev, group)
-            assert agreed == 1.0, f"expert-parallel leg ({key}, {mode}): rank {rank} window {same_window}, output {same_output}"
+            assert agreed == 1.0, f"expert-parallel leg ({key}, {name}): rank {rank} window {same_window}, output {same_output}"
             for _ in range(2):
                 step()
             handshakes0 = me.handshakes
@@ -619,10 +620,9 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"), modes=("ca
             assert me.status() == 0
             mean = lambda a, b: sum(e[a].elapsed_time(e[b]) for e in ev) / steps * 1e3
             red = lambda v: _group_reduce(v, dist.ReduceOp.MAX, dev, group)
-            res[mode] = {"verified": {"window_equals_single_gpu_path": True, "Y_equals_X": True},
-                         "step_us": red(mean(0, 5)), "plan_and_count_exchange_us": red(mean(0, 1)),
-                         "address_step_us": red(mean(1, 2)), "dispatch_kernel_us": red(mean(2, 3)),
-                         "barrier_after_dispatch_us": red(mean(3, 4)), "combine_kernel_us": red(mean(4, 5)),
+            res[name] = {"verified": {"window_equals_single_gpu_path": True, "Y_equals_X": True},
+                         "step_us": red(mean(0, 3)), "plan_and_count_exchange_us": red(mean(0, 1)),
+                         "dispatch_phase_us": red(mean(1, 2)), "combine_phase_us": red(mean(2, 3)),
                          "handshakes_in_timed_steps": me.handshakes - handshakes0, "steps": steps,
                          "dispatch_bytes_per_rank": bytes_dispatch(wl) // R}
             me.close()

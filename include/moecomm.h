@@ -251,7 +251,8 @@ moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/,
  *                       Synchronises `stream` before it releases or installs anything.
  *   moe_peers_set       installs addresses the caller already has (separate allocations of one process, a
  *                       symmetric-memory mapping, an earlier handshake of its own) without mapping anything:
- *                       window_bases HOST [R] of DEVICE pointers, generations HOST [R] or NULL (all zero).
+ *                       window_bases HOST [R] of DEVICE pointers, generations HOST [R] or NULL (all zero);
+ *                       with_state != 0: every window is followed by its state region (see moe_signal_peers).
  *   moe_peers_check     the cached-address test: MOE_OK if a table is installed and its generations equal
  *                       `generations` (HOST [R], what the ranks announced for this call -- the binding sends each
  *                       rank's generation along with its count row, so the test costs no exchange of its own);
@@ -277,13 +278,41 @@ moe_status_t moe_window_export(const void* window /*DEVICE*/, int64_t bytes, int
 moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles /*HOST [R]*/, int32_t my_rank,
                             void* my_window /*DEVICE*/, int64_t capacity_rows, void* stream);
 moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases /*HOST [R]*/,
-                           const int32_t* generations /*HOST [R] or NULL*/, int64_t capacity_rows, void* stream);
+                           const int32_t* generations /*HOST [R] or NULL*/, int32_t my_rank, int64_t capacity_rows,
+                           int32_t with_state, void* stream);
 moe_status_t moe_peers_check(const moe_ctx_t* ctx, const int32_t* generations /*HOST [R]*/);
 moe_status_t moe_dispatch_cached(moe_ctx_t* ctx, const void* x /*DEVICE*/, const int32_t* generations /*HOST or NULL*/,
                                  void* stream);
 moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations /*HOST or NULL*/,
                                 const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
 moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
+
+/* Synchronisation metadata in the pooled memory (Section 3.2: every rank's slice carries communicator state
+ * beside its payload; Section 5.4: status flags and wait symbols order producers and consumers across ranks).
+ * A window allocation may be followed by a state region of moe_state_bytes(R) bytes -- allocate
+ * moe_window_bytes(shape, capacity_rows, 1), zero the state region once -- which the handshake maps together
+ * with the rows (moe_peers_open finds it from the exported size; moe_peers_set is told by with_state).  It
+ * holds MOE_SYNC_SLOTS arrays of R 32-bit epochs.
+ *   moe_signal_peers  enqueues, behind everything already on `stream`, a store of `epoch` into entry
+ *                     [slot][my_rank] of EVERY rank's state region (release, system scope): "what I enqueued
+ *                     before this -- my rows in your window, my experts' outputs -- is complete".
+ *   moe_wait_peers    enqueues a kernel that waits until entries [slot][0..R-1] of THIS rank's own state region
+ *                     have all reached `epoch` (acquire, system scope); whatever is enqueued behind it sees
+ *                     what the signalling ranks wrote before their signals.  The wait is bounded (2 s, or the
+ *                     MOE_OPT_TEST_STARVE_WAIT_MS value): when it runs out the status word becomes
+ *                     MOE_ERR_TIMEOUT, the kernel ends normally and later calls write nothing until
+ *                     moe_status() has reported it.
+ * Epochs must grow from call to call (compared as signed differences, so they may wrap).  A layer step uses
+ * three slots: rows dispatched (before the experts read their window), expert outputs ready (before combine
+ * reads), combine done (before the next step's dispatch overwrites a window).  With these no host
+ * synchronisation is needed between the phases.  MOE_ERR_STALE_PEERS if no table with state is installed.
+ * NOTE: a wait kernel occupies its GPU until the signals arrive, so the ranks must run on different GPUs (or the
+ * caller must know that the signals were sent before the wait is enqueued). */
+#define MOE_SYNC_SLOTS 4
+size_t moe_state_bytes(int32_t R);
+size_t moe_window_bytes(const moe_shape_t* shape /*HOST*/, int64_t capacity_rows, int32_t with_state);
+moe_status_t moe_signal_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream);
+moe_status_t moe_wait_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream);
 
 /* Materialises slot(t,j) into caller memory (parity checks, expert-side
  * consumers).  slots DEVICE [T,K] int32; needs R * capacity_rows < 2^31. */

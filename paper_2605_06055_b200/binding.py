@@ -28,8 +28,10 @@ EXPORTS = [
     "moe_gate_topk", "moe_gate_plan", "moe_layout", "moe_notify", "moe_dispatch_peers", "moe_combine_peers",
     "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant", "moe_expert_tiles", "moe_dispatch_quant_peers",
     "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
-    "moe_dispatch_cached", "moe_combine_cached",
+    "moe_dispatch_cached", "moe_combine_cached", "moe_state_bytes", "moe_window_bytes", "moe_signal_peers",
+    "moe_wait_peers",
 ]
+MOE_SYNC_SLOTS = 4
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -109,7 +111,14 @@ def load() -> ctypes.CDLL:
     L.moe_dispatch_quant.restype = ctypes.c_int
     L.moe_window_export.argtypes = [vp, i64, i32, ctypes.POINTER(MoeWindowHandle)]
     L.moe_peers_open.argtypes = [vp, vp, i32, vp, i64, vp]
-    L.moe_peers_set.argtypes = [vp, vp, vp, i64, vp]
+    L.moe_peers_set.argtypes = [vp, vp, vp, i32, i64, i32, vp]
+    L.moe_state_bytes.argtypes = [i32]
+    L.moe_state_bytes.restype = ctypes.c_size_t
+    L.moe_window_bytes.argtypes = [ctypes.POINTER(MoeShape), i64, i32]
+    L.moe_window_bytes.restype = ctypes.c_size_t
+    L.moe_signal_peers.argtypes = [vp, i32, ctypes.c_uint32, vp]
+    L.moe_wait_peers.argtypes = [vp, i32, ctypes.c_uint32, vp]
+    L.moe_signal_peers.restype = L.moe_wait_peers.restype = ctypes.c_int
     L.moe_peers_check.argtypes = [vp, vp]
     L.moe_peers_close.argtypes = [vp, vp]
     L.moe_dispatch_cached.argtypes = [vp, vp, vp, vp]
@@ -370,14 +379,16 @@ class MoeComm:
             raise MoeError(rc, "moe_peers_open")
         return rc
 
-    def moe_peers_set(self, window_bases, generations, capacity_rows: int, stream=None, check: bool = True) -> int:
-        """window_bases: R device addresses (ints); generations: R ints or None."""
+    def moe_peers_set(self, window_bases, generations, capacity_rows: int, my_rank: int = 0, with_state: bool = False,
+                      stream=None, check: bool = True) -> int:
+        """window_bases: R device addresses (ints); generations: R ints or None; with_state: every window is
+        followed by its state region (moe_window_bytes(..., with_state=True) bytes were allocated for it)."""
         bases = np.ascontiguousarray(window_bases, dtype=np.uint64)
         gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
         assert bases.shape == (self.R,) and (gens is None or gens.shape == (self.R,))
         with self._on_device():
-            rc = self.lib.moe_peers_set(self._h, _host_ptr(bases), _host_ptr(gens), int(capacity_rows),
-                                        _stream_handle(stream))
+            rc = self.lib.moe_peers_set(self._h, _host_ptr(bases), _host_ptr(gens), int(my_rank), int(capacity_rows),
+                                        int(bool(with_state)), _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_peers_set")
         return rc
@@ -408,6 +419,23 @@ class MoeComm:
                                              _dev_ptr(y, torch.bfloat16), _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_combine_cached")
+        return rc
+
+    def moe_window_bytes(self, capacity_rows: int, with_state: bool = True) -> int:
+        return int(self.lib.moe_window_bytes(ctypes.byref(self._shape), int(capacity_rows), int(bool(with_state))))
+
+    def moe_signal_peers(self, slot: int, epoch: int, stream=None, check: bool = True) -> int:
+        with self._on_device():
+            rc = self.lib.moe_signal_peers(self._h, int(slot), int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_signal_peers")
+        return rc
+
+    def moe_wait_peers(self, slot: int, epoch: int, stream=None, check: bool = True) -> int:
+        with self._on_device():
+            rc = self.lib.moe_wait_peers(self._h, int(slot), int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_wait_peers")
         return rc
 
     def moe_plan_view(self) -> dict:
@@ -542,6 +570,10 @@ def moe_slots_noalloc(topk_idx: torch.Tensor, E: int, R: int, capacity_rows: int
                                             int(capacity_rows), _dev_ptr(slots, torch.int32),
                                             _dev_ptr(n_recv, torch.int32), _dev_ptr(status, torch.int32),
                                             _stream_handle(stream)))
+
+
+def moe_state_bytes(R: int) -> int:
+    return int(load().moe_state_bytes(int(R)))
 
 
 def moe_window_export(window: torch.Tensor, generation: int) -> bytes:

@@ -56,6 +56,9 @@ struct moe_ctx {
   int32_t peer_gen[MOE_MAX_R];
   int64_t peer_capacity;
   bool peers_installed;
+  bool peers_have_state;              // every installed window is followed by its state region
+  int32_t my_rank;                    // this process's rank in the installed table
+  unsigned char** state_table;        // device, [R]: state region of every rank (inside the workspace)
   // resident CTAs per SM of the row kernels this context has launched (occupancy calculator results)
   const void* occ_kernel[16];
   int occ_per_sm[16];
@@ -105,7 +108,7 @@ Layout layout_of(const moe_shape_t* s) {
   L.o = take(sizeof(int32_t) * s->E * s->R);
   L.n_exp = take(sizeof(int32_t) * s->E);
   L.n_recv = take(sizeof(int32_t) * s->R);
-  L.peers = take(sizeof(void*) * s->R);
+  L.peers = take(sizeof(void*) * s->R * 2);   // window bases, then state-region bases
   L.s = take(sizeof(int32_t) * B);
   L.tile_rank = take(sizeof(int32_t) * B);
   L.tile_hist = take(sizeof(int32_t) * (size_t)max_tiles(s) * s->E);
@@ -367,7 +370,10 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->n_exp = reinterpret_cast<int32_t*>(ctx->ws + L.n_exp);
   ctx->n_recv = reinterpret_cast<int32_t*>(ctx->ws + L.n_recv);
   ctx->peer_table = reinterpret_cast<const unsigned char**>(ctx->ws + L.peers);
+  ctx->state_table = reinterpret_cast<unsigned char**>(ctx->ws + L.peers) + shape->R;
   ctx->peers_installed = false;
+  ctx->peers_have_state = false;
+  ctx->my_rank = 0;
   ctx->peer_capacity = 0;
   for (int d = 0; d < MOE_MAX_R; ++d) {
     ctx->peer_ptr[d] = nullptr;
@@ -967,13 +973,24 @@ void release_mappings(moe_ctx* ctx) {
   ctx->peers_installed = false;
 }
 
-// Copies the host table to the device table on `stream` and marks it installed.
-moe_status_t install_table(moe_ctx* ctx, int64_t capacity_rows, cudaStream_t st) {
-  // pageable source: the runtime has staged the bytes by the time the call returns, so peer_ptr may change afterwards
-  if (cudaMemcpyAsync(ctx->peer_table, ctx->peer_ptr, sizeof(void*) * ctx->shape.R, cudaMemcpyHostToDevice, st) !=
-      cudaSuccess)
+size_t state_bytes_for(int32_t R) { return align_up(sizeof(uint32_t) * MOE_SYNC_SLOTS * (size_t)R); }
+
+// Copies the host table (and the state-region addresses, which follow the rows of every window) to the device
+// tables on `stream` and marks them installed.
+moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows, bool with_state, cudaStream_t st) {
+  const int R = ctx->shape.R;
+  void* both[2 * MOE_MAX_R];
+  const size_t rows_bytes = align_up((size_t)capacity_rows * ctx->shape.H * 2);
+  for (int d = 0; d < R; ++d) {
+    both[d] = ctx->peer_ptr[d];
+    both[R + d] = with_state ? static_cast<char*>(ctx->peer_ptr[d]) + rows_bytes : nullptr;
+  }
+  // pageable source: the runtime has staged the bytes by the time the call returns
+  if (cudaMemcpyAsync(ctx->peer_table, both, sizeof(void*) * 2 * R, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   ctx->peer_capacity = capacity_rows;
+  ctx->my_rank = my_rank;
+  ctx->peers_have_state = with_state;
   ctx->peers_installed = true;
   return MOE_OK;
 }
@@ -1015,8 +1032,12 @@ moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, 
       capacity_rows < 0 || !aligned16(my_window))
     return MOE_ERR_INVALID_ARG;
   const int64_t need = capacity_rows * ctx->shape.H * 2;
-  for (int d = 0; d < ctx->shape.R; ++d)
+  const int64_t need_with_state = (int64_t)(align_up((size_t)need) + state_bytes_for(ctx->shape.R));
+  bool with_state = true;   // only if every rank exported its state region along with its rows
+  for (int d = 0; d < ctx->shape.R; ++d) {
     if (d != my_rank && (handles[d].bytes < need || (handles[d].offset & 15) != 0)) return MOE_ERR_INVALID_ARG;
+    if (handles[d].bytes < need_with_state) with_state = false;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;   // nothing in flight reads the old table
   release_mappings(ctx);
@@ -1037,12 +1058,13 @@ moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, 
     ctx->peer_mapping[d] = base;
     ctx->peer_ptr[d] = static_cast<char*>(base) + handles[d].offset;
   }
-  return install_table(ctx, capacity_rows, st);
+  return install_table(ctx, my_rank, capacity_rows, with_state, st);
 }
 
-moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, const int32_t* generations,
-                           int64_t capacity_rows, void* stream) {
-  if (ctx == nullptr || window_bases == nullptr || capacity_rows < 0) return MOE_ERR_INVALID_ARG;
+moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, const int32_t* generations, int32_t my_rank,
+                           int64_t capacity_rows, int32_t with_state, void* stream) {
+  if (ctx == nullptr || window_bases == nullptr || capacity_rows < 0 || my_rank < 0 || my_rank >= ctx->shape.R)
+    return MOE_ERR_INVALID_ARG;
   for (int d = 0; d < ctx->shape.R; ++d)
     if (window_bases[d] == nullptr || !aligned16(window_bases[d])) return MOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1052,7 +1074,35 @@ moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, cons
     ctx->peer_ptr[d] = const_cast<void*>(window_bases[d]);
     ctx->peer_gen[d] = generations != nullptr ? generations[d] : 0;
   }
-  return install_table(ctx, capacity_rows, st);
+  return install_table(ctx, my_rank, capacity_rows, with_state != 0, st);
+}
+
+size_t moe_state_bytes(int32_t R) { return (R < 1 || R > MOE_MAX_R) ? 0 : state_bytes_for(R); }
+
+size_t moe_window_bytes(const moe_shape_t* shape, int64_t capacity_rows, int32_t with_state) {
+  if (!shape_valid(shape) || capacity_rows < 0) return 0;
+  const size_t rows = (size_t)capacity_rows * shape->H * 2;
+  return with_state ? align_up(rows) + state_bytes_for(shape->R) : rows;
+}
+
+moe_status_t moe_signal_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream) {
+  if (ctx == nullptr || slot < 0 || slot >= MOE_SYNC_SLOTS) return MOE_ERR_INVALID_ARG;
+  if (!ctx->peers_installed || !ctx->peers_have_state) return MOE_ERR_STALE_PEERS;
+  const int R = ctx->shape.R;
+  signal_peers_kernel<<<1, R < 32 ? 32 : (R + 31) / 32 * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      ctx->state_table, R, ctx->my_rank, slot, epoch);
+  return launch_ok(ctx);
+}
+
+moe_status_t moe_wait_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream) {
+  if (ctx == nullptr || slot < 0 || slot >= MOE_SYNC_SLOTS) return MOE_ERR_INVALID_ARG;
+  if (!ctx->peers_installed || !ctx->peers_have_state) return MOE_ERR_STALE_PEERS;
+  const int R = ctx->shape.R;
+  const size_t rows_bytes = align_up((size_t)ctx->peer_capacity * ctx->shape.H * 2);
+  const unsigned char* mine = static_cast<const unsigned char*>(ctx->peer_ptr[ctx->my_rank]) + rows_bytes;
+  wait_peers_kernel<<<1, R < 32 ? 32 : (R + 31) / 32 * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      mine, R, slot, epoch, ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT, &ctx->ctl->status);
+  return launch_ok(ctx);
 }
 
 moe_status_t moe_peers_check(const moe_ctx_t* ctx, const int32_t* generations) {

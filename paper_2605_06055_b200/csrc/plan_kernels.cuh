@@ -502,6 +502,44 @@ plan_finalize_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Synchronisation metadata across ranks (Section 5.4): epochs in the state region behind every rank's window.
+// signal: thread d stores `epoch` into entry [slot][my_rank] of rank d's region with release semantics at system
+// scope, so that everything this stream completed before the launch (rows stored into rank d's window, expert
+// outputs) is visible to whoever acquires the entry.  Plain peer stores; nothing waits here.
+__global__ void signal_peers_kernel(unsigned char* const* __restrict__ state_of_rank, int32_t R, int32_t my_rank,
+                                    int32_t slot, uint32_t epoch) {
+  for (int d = threadIdx.x; d < R; d += blockDim.x) {
+    uint32_t* entry = reinterpret_cast<uint32_t*>(state_of_rank[d]) + (size_t)slot * R + my_rank;
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(entry), "r"(epoch) : "memory");
+  }
+}
+
+// wait: thread r polls entry [slot][r] of THIS rank's region (acquire, system scope) until it has reached `epoch`,
+// sleeping between polls, for at most limit_ms milliseconds; a wait that runs out raises MOE_ERR_TIMEOUT and the
+// kernel ends normally.
+__global__ void wait_peers_kernel(const unsigned char* __restrict__ my_state, int32_t R, int32_t slot, uint32_t epoch,
+                                  int32_t limit_ms, int32_t* status) {
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    const uint32_t* entry = reinterpret_cast<const uint32_t*>(my_state) + (size_t)slot * R + r;
+    uint64_t t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    const uint64_t limit = (uint64_t)limit_ms * 1000000ull;
+    for (;;) {
+      uint32_t seen;
+      asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(seen) : "l"(entry) : "memory");
+      if ((int32_t)(seen - epoch) >= 0) break;
+      uint64_t now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (now - t0 > limit) {
+        raise_status(status, MOE_ERR_TIMEOUT);
+        break;
+      }
+      __nanosleep(200);
+    }
+  }
+}
+
 // Tile list over the experts' runs (work list of a grouped GEMM that reads the windows in place): tile k is
 // (expert, first window row, valid rows <= tile_rows), in window order.  ONE CTA; shared memory: tiles
 // per expert [E], their exclusive prefix [E + 1], warp sums [33].

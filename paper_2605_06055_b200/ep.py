@@ -15,6 +15,14 @@ cached table is out of date: every rank announces the generation of its window t
 so the test rides on the exchange Notify needs anyway and costs no collective of its own.  In the "handshake"
 mode the addresses are exchanged before every dispatch.
 
+Phase order (Section 5.4): with sync="host" the phases are separated by a stream synchronisation and a
+process-group barrier.  With sync="device" they are ordered on the GPUs alone: every window allocation carries a
+state region behind its rows, a rank signals all ranks after its dispatch / its experts / its combine
+(moe_signal_peers) and waits for all ranks' signals before its experts read the window / before its combine /
+before its next dispatch (moe_wait_peers, bounded).  A wait kernel occupies its GPU until the signals arrive, so
+device ordering needs one GPU per rank; where ranks share a GPU (the tests) `host_fence=True` places a host barrier
+between signal and wait, so that every wait finds its signals already there.
+
 The test suite exercises this on ONE GPU (two processes whose windows are mapped into each other over CUDA
 inter-process handles, counts over a gloo group) and the exchange logic with two gloo ranks on CPU.
 """
@@ -78,9 +86,13 @@ def symmetric_windows(capacity_rows: int, H: int, device, group=None):
 class EpRank:
     """The calls of one rank, in the order the schedules prescribe.  mode: "cached" or "handshake"."""
 
-    def __init__(self, T_local_max: int, H: int, E: int, K: int, device, group=None, mode: str = "cached"):
-        assert mode in ("cached", "handshake")
+    SLOT_DISPATCHED, SLOT_EXPERTS_DONE, SLOT_COMBINED = 0, 1, 2
+
+    def __init__(self, T_local_max: int, H: int, E: int, K: int, device, group=None, mode: str = "cached",
+                 sync: str = "host", host_fence: bool = False):
+        assert mode in ("cached", "handshake") and sync in ("host", "device")
         self.group, self.mode, self.device = group, mode, device
+        self.sync, self.host_fence, self.epoch = sync, host_fence, 0
         self.rank = dist.get_rank(group)
         self.R = dist.get_world_size(group)
         self.E, self.H = E, H
@@ -96,13 +108,37 @@ class EpRank:
         self.handshakes = 0
 
     # -- windows -------------------------------------------------------------------------------------
+    def new_window(self, capacity_rows: int) -> torch.Tensor:
+        """Allocates this rank's window with its state region behind the rows (zeroed), attaches it and returns the
+        [capacity_rows, H] view of the rows."""
+        nbytes = self.comm.moe_window_bytes(capacity_rows, with_state=True)
+        backing = torch.zeros(nbytes // 2, dtype=torch.bfloat16, device=self.device)
+        self.attach_window(backing, capacity_rows)
+        return backing[:capacity_rows * self.H].view(capacity_rows, self.H)
+
     def attach_window(self, window: torch.Tensor, capacity_rows: int) -> None:
-        """This rank's window from now on ([capacity_rows, H] bf16, the same capacity on every rank).  A new
-        window gets a new generation, which makes every rank's cached table stale at the next plan()."""
+        """This rank's window from now on: a contiguous bf16 tensor whose first capacity_rows * H elements are the
+        rows (the same capacity on every rank); if it is moe_window_bytes(capacity_rows, with_state=True) bytes
+        long, what follows the rows is the state region of the device-side phase order.  A new window gets a
+        new generation, which makes every rank's cached table stale at the next plan()."""
         assert window.dtype == torch.bfloat16 and window.is_contiguous() and window.numel() >= capacity_rows * self.H
+        new_state = self._state_region(window, capacity_rows)
+        if self.sync == "device" and new_state is not None and self.window is not None and self.epoch > 0:
+            # The epochs move with the window: once every signal of the finished step has arrived in the old state
+            # region (the combine-done signals are a step's last), it is copied behind the new rows.
+            old_state = self._state_region(self.window, self.capacity)
+            if old_state is not None:
+                self.comm.moe_wait_peers(self.SLOT_COMBINED, self.epoch)
+                new_state.copy_(old_state)
         self.window, self.capacity = window, int(capacity_rows)
         self.generation += 1
         self.message[self.E:].fill_(self.generation)
+
+    def _state_region(self, window: torch.Tensor, capacity_rows: int):
+        """The state region behind the rows of a window allocation, or None if the allocation has none."""
+        state = binding.moe_state_bytes(self.R) // 2
+        start = self.comm.moe_window_bytes(capacity_rows, with_state=True) // 2 - state
+        return window[start:start + state] if window.numel() >= start + state else None
 
     def handshake(self) -> None:
         """Collective: exchanges the window handles and maps every other rank's window."""
@@ -117,7 +153,7 @@ class EpRank:
     def install_addresses(self, window_bases, generations=None) -> None:
         """Addresses obtained elsewhere (one process holding every window; symmetric memory)."""
         gens = np.zeros(self.R, np.int32) if generations is None else np.asarray(generations, np.int32)
-        self.comm.moe_peers_set(window_bases, gens, self.capacity)
+        self.comm.moe_peers_set(window_bases, gens, self.capacity, my_rank=self.rank)
         self.table_generations = gens
 
     def _ensure_addresses(self) -> None:
@@ -135,16 +171,40 @@ class EpRank:
         self.comm.moe_notify(counts_all)
         return counts_all
 
-    def dispatch(self, x_local: torch.Tensor) -> None:
-        self._ensure_addresses()
-        self.comm.moe_dispatch_cached(x_local, self.announced)
+    def _host_barrier(self) -> None:
         torch.cuda.current_stream().synchronize()
-        dist.barrier(self.group)                 # every rank's rows have landed before any expert reads its window
+        dist.barrier(self.group)
+
+    def _signal_then_wait(self, slot: int) -> None:
+        self.comm.moe_signal_peers(slot, self.epoch)
+        if self.host_fence:                      # ranks share a GPU: every signal is sent before any wait is enqueued
+            self._host_barrier()
+        self.comm.moe_wait_peers(slot, self.epoch)
+
+    def dispatch(self, x_local: torch.Tensor) -> None:
+        """Rows into every rank's window; returns once the experts of this rank may be enqueued."""
+        self._ensure_addresses()
+        if self.sync == "device":
+            self.epoch += 1
+            if self.epoch > 1:                   # every rank has finished reading the windows of the step before
+                self.comm.moe_wait_peers(self.SLOT_COMBINED, self.epoch - 1)
+            self.comm.moe_dispatch_cached(x_local, self.announced)
+            self._signal_then_wait(self.SLOT_DISPATCHED)
+        else:
+            self.comm.moe_dispatch_cached(x_local, self.announced)
+            self._host_barrier()                 # every rank's rows have landed before any expert reads its window
 
     def combine(self, topk_w_local: torch.Tensor, y_local: torch.Tensor) -> None:
-        torch.cuda.current_stream().synchronize()
-        dist.barrier(self.group)                 # every expert has written its outputs
-        self.comm.moe_combine_cached(self.announced, topk_w_local, y_local)
+        """Call after this rank's experts have been enqueued: waits for every rank's experts, then combines."""
+        if self.sync == "device":
+            self._signal_then_wait(self.SLOT_EXPERTS_DONE)
+            self.comm.moe_combine_cached(self.announced, topk_w_local, y_local)
+            self.comm.moe_signal_peers(self.SLOT_COMBINED, self.epoch)
+            if self.host_fence:
+                self._host_barrier()
+        else:
+            self._host_barrier()                 # every expert has written its outputs
+            self.comm.moe_combine_cached(self.announced, topk_w_local, y_local)
 
     def dispatch_quant(self, x_local: torch.Tensor, window_q_bases: torch.Tensor, scale_bases: torch.Tensor,
                        capacity_rows: int) -> None:

@@ -184,6 +184,80 @@ def test_installed_address_table_and_generation_stamp_in_one_process():
         c.close()
 
 
+def test_signals_and_bounded_waits_between_ranks_of_one_process():
+    """The device-side phase order with every rank a context of this process (all on the one GPU, so every signal
+    is enqueued before any wait): signals reach every rank's state region, waits pass once all R signals of the
+    epoch are there, and a wait nobody answers runs out after its bound, raises MOE_ERR_TIMEOUT without
+    trapping, and leaves the context usable."""
+    name, T, H, E, R, K, sch, routing, per = CASES[0]
+    dev = torch.device("cuda:0")
+    wl = Workload(name, T, H, E, R, K, sch, routing, "identity", 7000 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    rts = inp.rank_tok_start
+    p = oracle.plan(inp.topk_idx.numpy(), E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    want = harness.oracle_run(inp, C)
+    idx, w, X = inp.topk_idx.to(dev), inp.topk_w.to(dev), inp.X.to(dev)
+    comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
+    counts = torch.zeros((R, E), dtype=torch.int32, device=dev)
+    for r, c in enumerate(comms):
+        c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, counts[r])
+    for c in comms:
+        c.moe_notify(counts)
+    total = comms[0].moe_window_bytes(C, True) // 2
+    assert total * 2 >= C * H * 2 + binding.moe_state_bytes(R) > C * H * 2
+    backings = [torch.zeros(total, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+    rows = [b[:C * H].view(C, H) for b in backings]
+    for t in rows:
+        t.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+    bases = [b.data_ptr() for b in backings]
+    # without a state region the signals have nowhere to go
+    comms[0].moe_peers_set(bases, None, C, my_rank=0, with_state=False)
+    assert comms[0].moe_signal_peers(0, 1, check=False) == binding.MOE_ERR_STALE_PEERS
+    assert comms[0].moe_wait_peers(0, 1, check=False) == binding.MOE_ERR_STALE_PEERS
+    for r, c in enumerate(comms):
+        c.moe_peers_set(bases, None, C, my_rank=r, with_state=True)
+    state = lambda d: backings[d].view(torch.int32)[-(binding.moe_state_bytes(R) // 4):][:binding.MOE_SYNC_SLOTS * R].view(binding.MOE_SYNC_SLOTS, R)
+    for epoch in (1, 2):
+        for r, c in enumerate(comms):                      # every rank dispatches and signals ...
+            c.moe_dispatch_cached(X[rts[r]:rts[r + 1]].contiguous())
+            c.moe_signal_peers(0, epoch)
+        for c in comms:                                    # ... then every rank waits: all signals are there
+            c.moe_wait_peers(0, epoch)
+            assert c.moe_status() == 0
+        for d in range(R):
+            assert state(d)[0].tolist() == [epoch] * R and state(d)[1].tolist() == [epoch - 1] * R
+        assert np.array_equal(torch.cat(rows).cpu().view(torch.int16).numpy().view(np.uint16), want.windows)
+        for r, c in enumerate(comms):
+            c.moe_signal_peers(1, epoch)
+        Y = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
+        for r, c in enumerate(comms):
+            c.moe_wait_peers(1, epoch)
+            y_r = torch.empty((int(rts[r + 1] - rts[r]), H), dtype=torch.bfloat16, device=dev)
+            c.moe_combine_cached(None, w[rts[r]:rts[r + 1]].contiguous(), y_r)
+            assert c.moe_status() == 0
+            Y[rts[r]:rts[r + 1]] = y_r
+        assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
+    # only one of R signals arrives for epoch 3: the wait is bounded (50 ms here), reports, and nothing hangs
+    c = comms[1]
+    c.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 50)
+    comms[0].moe_signal_peers(0, 3)
+    c.moe_wait_peers(0, 3)
+    y_r = torch.full((int(rts[2] - rts[1]), H), 7.0, dtype=torch.bfloat16, device=dev)
+    c.moe_combine_cached(None, w[rts[1]:rts[2]].contiguous(), y_r)       # behind a failed wait: writes nothing
+    assert c.moe_status() == binding.MOE_ERR_TIMEOUT
+    assert bool((y_r == 7.0).all())
+    c.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 0)
+    for cc in comms[1:]:
+        cc.moe_signal_peers(0, 3)
+    c.moe_wait_peers(0, 3)                                               # now all R are there
+    c.moe_combine_cached(None, w[rts[1]:rts[2]].contiguous(), y_r)
+    assert c.moe_status() == 0
+    assert harness.max_ulp_diff(y_r.cpu().view(torch.int16).numpy().view(np.uint16), want.Y[int(rts[1]):int(rts[2])]) <= 1
+    for c in comms:
+        c.close()
+
+
 # ------------------------------------------------------------------ two processes, windows mapped into each other
 IPC_SHAPE = dict(T=600, H=512, E=16, K=4, per=(250, 350), seed=7300)
 
@@ -194,7 +268,7 @@ def _ipc_workload(world):
                     rank_tokens=c["per"])
 
 
-def _ipc_rank(rank, world, port, mode, q_to, results):
+def _ipc_rank(rank, world, port, mode, sync, q_to, results):
     """One expert-parallel rank as its own process on the one GPU: its window lives in its own allocation, the
     other rank's window is mapped in through the library's handle exchange (moe_window_export over a gloo group,
     moe_peers_open), counts travel over the same group, phases are ordered by host barriers (no kernel waits on
@@ -214,7 +288,8 @@ def _ipc_rank(rank, world, port, mode, q_to, results):
         lo, hi = int(rts[rank]), int(rts[rank + 1])
         idx, x, w = (inp.topk_idx[lo:hi].contiguous().to(dev), inp.X[lo:hi].contiguous().to(dev),
                      inp.topk_w[lo:hi].contiguous().to(dev))
-        me = ep.EpRank(hi - lo, H, E, K, dev, mode=mode)
+        # ranks share the GPU here: with the device-side phase order every signal is sent before any wait is enqueued
+        me = ep.EpRank(hi - lo, H, E, K, dev, mode=mode, sync=sync, host_fence=True)
         me.plan(DECODE, idx)                               # first plan: learn the capacity the windows need
         C = int(me.comm.moe_plan_view()["n_recv"].max().item()) + 1
         log = {}
@@ -222,13 +297,15 @@ def _ipc_rank(rank, world, port, mode, q_to, results):
         log["refused_without_table"] = me.comm.moe_dispatch_cached(x, me.announced, check=False)
         # every window is a slice of a backing allocation of its own (large enough that the caching allocator
         # gives it a device allocation to itself): the exported handle names that allocation, plus an offset
+        # (rows first, then the zeroed state region of the device-side phase order)
         def new_window(offset_rows):
-            backing = torch.empty(12 << 20, dtype=torch.bfloat16, device=dev)
-            win = backing[offset_rows * H:(offset_rows + C) * H].view(C, H)
+            backing = torch.zeros(12 << 20, dtype=torch.bfloat16, device=dev)
+            flat = backing[offset_rows * H:offset_rows * H + me.comm.moe_window_bytes(C, True) // 2]
+            win = flat[:C * H].view(C, H)
             win.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+            me.attach_window(flat, C)
             return backing, win
         backing, mine = new_window(0)
-        me.attach_window(mine, C)
         y = torch.empty((hi - lo, H), dtype=torch.bfloat16, device=dev)
         u16 = lambda t: t.cpu().view(torch.int16).numpy().view(np.uint16).copy()
 
@@ -264,7 +341,6 @@ def _ipc_rank(rank, world, port, mode, q_to, results):
         if rank == 1:
             keep_old = backing                         # stays mapped on the other rank until its next handshake
             backing, mine = new_window(8)              # the new window starts 8 rows into its allocation
-            me.attach_window(mine, C)
         else:
             mine.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
         torch.cuda.synchronize()
@@ -295,16 +371,16 @@ def _ipc_rank(rank, world, port, mode, q_to, results):
         results[rank] = ("error", repr(exc) + "\n" + traceback.format_exc())
 
 
-@pytest.mark.parametrize("mode", ["cached", "handshake"])
-def test_two_processes_exchange_rows_through_mapped_windows(mode):
+@pytest.mark.parametrize("mode,sync", [("cached", "host"), ("handshake", "host"), ("cached", "device")])
+def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     world = 2
     with ctx.Manager() as m:
         results = m.dict()
         q_to = [ctx.Queue(), ctx.Queue()]
-        port = 35000 + (os.getpid() * 2 + (mode == "cached")) % 2000
-        procs = [ctx.Process(target=_ipc_rank, args=(r, world, port, mode, q_to, results)) for r in range(world)]
+        port = 35000 + (os.getpid() * 4 + 2 * (mode == "cached") + (sync == "device")) % 2000
+        procs = [ctx.Process(target=_ipc_rank, args=(r, world, port, mode, sync, q_to, results)) for r in range(world)]
         for p_ in procs:
             p_.start()
         for p_ in procs:
@@ -369,7 +445,7 @@ def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
     """The code `bench.py --gpus N` runs for N > 1 (rank = process, windows mapped into each other), here as two
     processes that share the one GPU and talk over gloo: it verifies its own windows and outputs before it times
     anything, exchanges no addresses in the timed steps of the cached mode and one set per step in the handshake
-    mode."""
+    mode, and orders its phases by host barriers or by arrival flags."""
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     world = 2
@@ -390,8 +466,11 @@ def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
     for r in range(world):
         leg = res[r][1]
         assert leg["ranks"] == 2 and "decode" in leg
-        for mode, want_handshakes in (("cached", 0), ("handshake", 3)):
-            got = leg["decode"][mode]
+        assert leg["ranks_share_a_gpu"] is True
+        for variant, want_handshakes in (("cached_addresses__host_phase_order", 0),
+                                         ("handshake_addresses__host_phase_order", 3),
+                                         ("cached_addresses__device_phase_order", 0)):
+            got = leg["decode"][variant]
             assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
             assert got["handshakes_in_timed_steps"] == want_handshakes
-            assert got["step_us"] > 0 and got["dispatch_kernel_us"] > 0 and got["combine_kernel_us"] > 0
+            assert got["step_us"] > 0 and got["dispatch_phase_us"] > 0 and got["combine_phase_us"] > 0
