@@ -261,7 +261,10 @@ gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t
     auto process = [&](const float (&v)[VPT], int32_t tok) {
       int32_t idx;
       float w;
-      if (!warp_gate_rank<VPT>(v, K, lane, gate_cand[warp], idx, w)) warp_gate_select<VPT>(v, K, lane, idx, w);
+      // rows of one or two logits per lane: the rounds are already cheap (nothing to scan inside a lane)
+      bool done = false;
+      if constexpr (VPT >= 4) done = warp_gate_rank<VPT>(v, K, lane, gate_cand[warp], idx, w);
+      if (!done) warp_gate_select<VPT>(v, K, lane, idx, w);
       w = warp_gate_softmax(w, K, lane);
       if (lane < K) {
         topk_idx[(size_t)tok * K + lane] = idx;
