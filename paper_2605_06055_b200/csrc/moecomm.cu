@@ -410,9 +410,11 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   auto opt_in = [&](auto kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess;
   };
-  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2, 16>) && opt_in(dispatch_quant_kernel<3, 16>) &&
-       opt_in(dispatch_quant_kernel<2, 32>) && opt_in(dispatch_quant_kernel<3, 32>) &&
-       opt_in(dispatch_quant_kernel<2, 0>) && opt_in(dispatch_quant_kernel<3, 0>) && opt_in(plan_rank_kernel<32>) &&
+  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2, 16, true>) && opt_in(dispatch_quant_kernel<3, 16, true>) &&
+       opt_in(dispatch_quant_kernel<2, 32, true>) && opt_in(dispatch_quant_kernel<3, 32, true>) &&
+       opt_in(dispatch_quant_kernel<2, 16, false>) && opt_in(dispatch_quant_kernel<3, 16, false>) &&
+       opt_in(dispatch_quant_kernel<2, 32, false>) && opt_in(dispatch_quant_kernel<3, 32, false>) &&
+       opt_in(dispatch_quant_kernel<2, 0, false>) && opt_in(dispatch_quant_kernel<3, 0, false>) && opt_in(plan_rank_kernel<32>) &&
        opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
        opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
@@ -812,14 +814,15 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
     launch_kernel(kernel, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
                   static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
   };
+  const bool whole_slabs = a.H16 % 32 == 0;   // every chunk of a row is valid for all lanes or for none
   if (stages == 3) {
-    if (cpl == 16) launch(dispatch_quant_kernel<3, 16>);
-    else if (cpl == 32) launch(dispatch_quant_kernel<3, 32>);
-    else launch(dispatch_quant_kernel<3, 0>);
+    if (cpl == 16) whole_slabs ? launch(dispatch_quant_kernel<3, 16, true>) : launch(dispatch_quant_kernel<3, 16, false>);
+    else if (cpl == 32) whole_slabs ? launch(dispatch_quant_kernel<3, 32, true>) : launch(dispatch_quant_kernel<3, 32, false>);
+    else launch(dispatch_quant_kernel<3, 0, false>);
   } else {
-    if (cpl == 16) launch(dispatch_quant_kernel<2, 16>);
-    else if (cpl == 32) launch(dispatch_quant_kernel<2, 32>);
-    else launch(dispatch_quant_kernel<2, 0>);
+    if (cpl == 16) whole_slabs ? launch(dispatch_quant_kernel<2, 16, true>) : launch(dispatch_quant_kernel<2, 16, false>);
+    else if (cpl == 32) whole_slabs ? launch(dispatch_quant_kernel<2, 32, true>) : launch(dispatch_quant_kernel<2, 32, false>);
+    else launch(dispatch_quant_kernel<2, 0, false>);
   }
   return launch_ok(ctx);
 }

@@ -45,11 +45,18 @@ __device__ __forceinline__ void sts64(uint32_t addr, uint32_t lo, uint32_t hi) {
   asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(addr), "r"(lo), "r"(hi) : "memory");
 }
 
-// Two bf16 values packed in one word -> two e4m3 codes (low half first).
+// Two bf16 values packed in one word -> two e4m3 codes (low half first).  The two fp32 products come from one
+// packed multiply (mul.rn.f32x2, an sm_100 instruction: each half is the same round-to-nearest product as a
+// scalar multiply).
 __device__ __forceinline__ uint32_t quant_pair(uint32_t two_bf16, float inv) {
   float2 f;
-  f.x = __fmul_rn(__uint_as_float(two_bf16 << 16), inv);
-  f.y = __fmul_rn(__uint_as_float(two_bf16 & 0xffff0000u), inv);
+  asm("{\n\t.reg .b64 a, b, d;\n\t"
+      "mov.b64 a, {%2, %3};\n\t"
+      "mov.b64 b, {%4, %4};\n\t"
+      "mul.rn.f32x2 d, a, b;\n\t"
+      "mov.b64 {%0, %1}, d;\n\t}"
+      : "=f"(f.x), "=f"(f.y)
+      : "r"(two_bf16 << 16), "r"(two_bf16 & 0xffff0000u), "f"(inv));
   return (uint32_t)__nv_cvt_float2_to_fp8x2(f, __NV_SATFINITE, __NV_E4M3);
 }
 
@@ -61,7 +68,9 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t two_bf16, float inv) {
 // the stage twice and needs a warp barrier per chunk, which left a warp at about 0.15 instructions per cycle:
 // 3.8 us per 8 KB row, the whole run time at 49 rows per warp.  Registers decide how many warps a CTA may have:
 // 16 for CPL <= 16, 8 beyond.
-template <int QUANT_STAGES, int CPL>
+// FULL: the row is a whole number of 512-byte slabs (H % 256 == 0), so a chunk is valid for all lanes or for none
+// and the per-lane bounds checks (a possibly divergent branch per chunk) reduce to a warp-uniform one.
+template <int QUANT_STAGES, int CPL, bool FULL>
 __global__ void __launch_bounds__((CPL > 16 ? 8 : QUANT_MAX_WARPS) * 32, 1)
 dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
                       float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
@@ -151,30 +160,28 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
     if constexpr (CPL > 0) {
       uint4 v[CPL];
       uint32_t m[4] = {0u, 0u, 0u, 0u};
+      const int slabs = a.H16 >> 5;   // FULL: chunks per lane
+      auto mine = [&](int k) { return FULL ? k < slabs : lane + 32 * k < a.H16; };
 #pragma unroll
-      for (int k = 0; k < CPL; ++k) {
-        const int c = lane + 32 * k;
-        v[k] = make_uint4(0, 0, 0, 0);
-        if (c < a.H16) v[k] = lds128(in + c * 16);
-      }
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) v[k] = lds128(in + (lane + 32 * k) * 16);
 #pragma unroll
-      for (int k = 0; k < CPL; ++k) {
-        m[0] = __vmaxu2(m[0], v[k].x & 0x7fff7fffu);
-        m[1] = __vmaxu2(m[1], v[k].y & 0x7fff7fffu);
-        m[2] = __vmaxu2(m[2], v[k].z & 0x7fff7fffu);
-        m[3] = __vmaxu2(m[3], v[k].w & 0x7fff7fffu);
-      }
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) {
+          m[0] = __vmaxu2(m[0], v[k].x & 0x7fff7fffu);
+          m[1] = __vmaxu2(m[1], v[k].y & 0x7fff7fffu);
+          m[2] = __vmaxu2(m[2], v[k].z & 0x7fff7fffu);
+          m[3] = __vmaxu2(m[3], v[k].w & 0x7fff7fffu);
+        }
       scale_from(__vmaxu2(__vmaxu2(m[0], m[1]), __vmaxu2(m[2], m[3])));   // the shuffles inside order every lane's reads
       __syncwarp();                                                        // ... in front of every lane's writes
 #pragma unroll
-      for (int k = 0; k < CPL; ++k) {
-        const int c = lane + 32 * k;
-        if (c < a.H16) {
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) {
           const uint32_t lo = quant_pair(v[k].x, inv) | (quant_pair(v[k].y, inv) << 16);
           const uint32_t hi = quant_pair(v[k].z, inv) | (quant_pair(v[k].w, inv) << 16);
-          sts64(in + c * 8, lo, hi);
+          sts64(in + (lane + 32 * k) * 8, lo, hi);
         }
-      }
     } else {
       uint32_t m2 = 0;
       for (int c = lane; c < a.H16; c += 32) {
