@@ -152,9 +152,17 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
 #pragma unroll
   for (int i = 1; i < VPT; ++i) m = fmaxf(m, v[i]);
   float theta = 0.0f;
-  for (int j = 0; j < K; ++j) {
-    theta = warp_max_f32(m);
-    m = (m == theta) ? -INFINITY : m;
+  if (K == 8) {   // the common top-k degree, without the loop
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      theta = warp_max_f32(m);
+      m = (m == theta) ? -INFINITY : m;
+    }
+  } else {
+    for (int j = 0; j < K; ++j) {
+      theta = warp_max_f32(m);
+      m = (m == theta) ? -INFINITY : m;
+    }
   }
   // absent entries are -inf and must never qualify; logits are finite, so -FLT_MAX admits every real entry
   theta = fmaxf(theta, -3.402823466e+38f);
@@ -165,10 +173,11 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
     const int u = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += u;
+    incl += (lane >= d) ? u : 0;
   }
   const int C = __shfl_sync(0xffffffffu, incl, 31);
   if (C > 32) return false;
+  if (lane < 3) cand_val[C + lane] = -INFINITY;   // the counting loop reads four candidates at a time
   // predicated stores, no branches: slot address advances by one word per candidate
   uint32_t slot = (uint32_t)__cvta_generic_to_shared(cand_val) + 4u * (uint32_t)(incl - c);
 #pragma unroll
@@ -183,8 +192,6 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
         : "=r"(step) : "f"(v[i]), "f"(theta), "r"(slot), "r"(base + i) : "memory");
     slot += step;
   }
-  __syncwarp();
-  if (lane < 3) cand_val[C + lane] = -INFINITY;   // the counting loop reads four candidates at a time
   __syncwarp();
   const float x = lane < C ? cand_val[lane] + 0.0f : -INFINITY;   // -0 becomes +0: equal logits get equal bit patterns
   const int32_t xi = lane < C ? cand_idx[lane] : -1;
@@ -202,6 +209,114 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
   idx_lane = lane < K ? out_idx[lane] : -1;
   __syncwarp();   // the next token of this warp reuses the buffers
   return true;
+}
+
+// Two tokens per warp.  Everything a token costs whatever its row length -- the scan of the candidate counts, the
+// rank loop, the softmax and the stores -- is a good half of warp_gate_rank's instructions; here two tokens share
+// those instruction streams: the thresholds and the compaction still run over the whole warp for each token (the
+// two counts ride through ONE scan, packed in the halves of a word), then lanes 0-15 rank token A's candidates while
+// lanes 16-31 rank token B's, and the caller's epilogue works on half-warps.  Needs K <= 16; fails (nothing
+// written that matters) if a token has more than 16 candidates -- the caller then takes the tokens one by one.
+// On success lane j < K of half h holds the j-th selected logit and expert of token h.
+// sm: GATE_PAIR_WORDS words: candidate values [2][20], candidate experts [2][20], selected values [2][16], experts [2][16].
+constexpr int GATE_PAIR_WORDS = 144;
+
+template <int VPT>
+__device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], const float (&vb)[VPT], int K, int lane,
+                                                    float* sm, int32_t& idx_lane, float& w_lane) {
+  float* cand_val = sm;                                          // [2][20]: 16 candidates + padding of the last four
+  float* out_val = sm + 80;                                      // [2][16]
+  int32_t* out_idx = reinterpret_cast<int32_t*>(sm + 112);       // [2][16]
+  const int base = lane * VPT;
+  float ma = va[0], mb = vb[0];
+#pragma unroll
+  for (int i = 1; i < VPT; ++i) {
+    ma = fmaxf(ma, va[i]);
+    mb = fmaxf(mb, vb[i]);
+  }
+  float ta = 0.0f, tb = 0.0f;
+  auto round = [&]() {
+    ta = warp_max_f32(ma);
+    tb = warp_max_f32(mb);
+    ma = (ma == ta) ? -INFINITY : ma;
+    mb = (mb == tb) ? -INFINITY : mb;
+  };
+  if (K == 8) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) round();
+  } else {
+    for (int j = 0; j < K; ++j) round();
+  }
+  ta = fmaxf(ta, -3.402823466e+38f);   // absent entries (-inf) never qualify
+  tb = fmaxf(tb, -3.402823466e+38f);
+  int c = 0;   // candidates of this lane: token A in the low half of the word, token B in the high half
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) c += ((va[i] >= ta) ? 1 : 0) + ((vb[i] >= tb) ? 0x10000 : 0);
+  int incl = c;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int u = __shfl_up_sync(0xffffffffu, incl, d);
+    incl += (lane >= d) ? u : 0;
+  }
+  const int total = __shfl_sync(0xffffffffu, incl, 31);
+  const int Ca = total & 0xffff, Cb = total >> 16;
+  if (Ca > 16 || Cb > 16) return false;
+  const int half = lane >> 4, l = lane & 15;
+  const int Ch = half ? Cb : Ca;
+  if (l < 3) cand_val[half * 20 + Ch + l] = -INFINITY;   // the counting loop reads four candidates at a time
+  const int excl = incl - c;
+  const uint32_t sm_addr = (uint32_t)__cvta_generic_to_shared(cand_val);
+  uint32_t slot_a = sm_addr + 4u * (uint32_t)(excl & 0xffff), slot_b = sm_addr + 80u + 4u * (uint32_t)(excl >> 16);
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {   // predicated stores, no branches (see warp_gate_rank); experts 40 words behind the values
+    uint32_t step_a, step_b;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ge.f32 p, %2, %3;\n\t"
+        "setp.ge.f32 q, %6, %7;\n\t"
+        "@p st.shared.f32 [%4], %2;\n\t"
+        "@p st.shared.u32 [%4+160], %5;\n\t"
+        "@q st.shared.f32 [%8], %6;\n\t"
+        "@q st.shared.u32 [%8+160], %5;\n\t"
+        "selp.u32 %0, 4, 0, p;\n\t"
+        "selp.u32 %1, 4, 0, q;\n\t}"
+        : "=r"(step_a), "=r"(step_b)
+        : "f"(va[i]), "f"(ta), "r"(slot_a), "r"(base + i), "f"(vb[i]), "f"(tb), "r"(slot_b) : "memory");
+    slot_a += step_a;
+    slot_b += step_b;
+  }
+  __syncwarp();
+  const float* mine = cand_val + half * 20;
+  const float x = l < Ch ? mine[l] + 0.0f : -INFINITY;   // -0 becomes +0: equal logits get equal bit patterns
+  const int32_t xi = l < Ch ? reinterpret_cast<const int32_t*>(mine)[40 + l] : -1;
+  const unsigned same_half_before = lanemask_lt() & (half ? 0xffff0000u : 0x0000ffffu);
+  int rank = __popc(__match_any_sync(0xffffffffu, __float_as_uint(x)) & same_half_before);   // earlier equal candidates
+  for (int q = 0; q < Ch; q += 4) {
+    const float4 a = *reinterpret_cast<const float4*>(mine + q);
+    rank += (a.x > x ? 1 : 0) + (a.y > x ? 1 : 0) + (a.z > x ? 1 : 0) + (a.w > x ? 1 : 0);
+  }
+  if (l < Ch && rank < K) {
+    out_val[half * 16 + rank] = x;
+    out_idx[half * 16 + rank] = xi;
+  }
+  __syncwarp();
+  w_lane = l < K ? out_val[half * 16 + l] : 0.0f;
+  idx_lane = l < K ? out_idx[half * 16 + l] : -1;
+  __syncwarp();   // the next tokens of this warp reuse the buffers
+  return true;
+}
+
+// The softmax of warp_gate_softmax for two tokens at once: lane j < K of each half-warp holds its token's j-th logit.
+__device__ __forceinline__ float halfwarp_gate_softmax(float sel_val, int K, int lane) {
+  const int l = lane & 15;
+  const float top = __shfl_sync(0xffffffffu, sel_val, 0, 16);
+  const float ex = l < K ? expf(sel_val - top) : 0.0f;
+  float sum = 0.0f;
+  for (int j0 = 0; j0 < K; j0 += 8) {   // K <= 16: no index leaves the half-warp
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) sum += __shfl_sync(0xffffffffu, ex, j0 + jj, 16);
+  }
+  return __fdiv_rn(l < K ? ex : 1.0f, sum);
 }
 
 // fp32 softmax over the K selected logits (lane j < K holds the j-th), summed in ascending j.
@@ -247,11 +362,11 @@ __device__ __forceinline__ void warp_gate_load(const float* __restrict__ row, in
 // length class, so that short rows keep few registers and many warps per SM).  VPT == 0: shared-memory form for longer rows; dynamic shared
 // memory: warps * E floats.
 template <int VPT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, VPT == 8 ? 4 : 1)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
-                 float* __restrict__ topk_w) {
+                 float* __restrict__ topk_w, int32_t in_pairs /* launcher: enough tokens for two per warp */) {
   extern __shared__ float gate_rows[];
-  __shared__ __align__(16) float gate_cand[8][GATE_RANK_WORDS];   // warp_gate_rank's buffers, one set per warp
+  __shared__ __align__(16) float gate_cand[8][GATE_PAIR_WORDS];   // warp_gate_rank(_pair)'s buffers, one set per warp
   release_dependents();   // a planner launched behind the gate (moe_gate_plan) may be scheduled; it waits for this kernel
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpc = blockDim.x >> 5;
   const int32_t stride = gridDim.x * wpc;
@@ -271,7 +386,50 @@ gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t
         topk_w[(size_t)tok * K + lane] = w;
       }
     };
-    // two row buffers used in turn: the next token's row travels while the current one is selected
+    if (VPT >= 4 && K <= 16 && in_pairs) {   // (never taken for the short-row forms)
+      // Tokens in pairs (2p, 2p+1), two pairs of row buffers used in turn: the next pair's rows travel while the
+      // current pair is selected.  A last odd token, and pairs with too many candidates, go one by one.
+      float* pair_sm = gate_cand[warp];
+      const int32_t pairs = T >> 1, pstride = stride;
+      int32_t p = blockIdx.x * wpc + warp;
+      auto load_pair = [&](int32_t pp, float (&ra)[VPT], float (&rb)[VPT]) {
+        warp_gate_load<VPT>(logits + (size_t)(2 * pp) * E, E, lane, vec, ra);
+        warp_gate_load<VPT>(logits + (size_t)(2 * pp + 1) * E, E, lane, vec, rb);
+      };
+      auto process_pair = [&](const float (&ra)[VPT], const float (&rb)[VPT], int32_t pp) {
+        int32_t idx;
+        float w;
+        if (warp_gate_rank_pair<VPT>(ra, rb, K, lane, pair_sm, idx, w)) {
+          w = halfwarp_gate_softmax(w, K, lane);
+          const int l = lane & 15;
+          const size_t tok = (size_t)(2 * pp + (lane >> 4));
+          if (l < K) {
+            topk_idx[tok * K + l] = idx;
+            topk_w[tok * K + l] = w;
+          }
+        } else {
+          process(ra, 2 * pp);
+          process(rb, 2 * pp + 1);
+        }
+      };
+      float a0[VPT], b0[VPT], a1[VPT], b1[VPT];
+      if (p < pairs) load_pair(p, a0, b0);
+      while (p < pairs) {
+        if (p + pstride < pairs) load_pair(p + pstride, a1, b1);
+        process_pair(a0, b0, p);
+        p += pstride;
+        if (p >= pairs) break;
+        if (p + pstride < pairs) load_pair(p + pstride, a0, b0);
+        process_pair(a1, b1, p);
+        p += pstride;
+      }
+      if ((T & 1) && blockIdx.x == 0 && warp == 0) {
+        warp_gate_load<VPT>(logits + (size_t)(T - 1) * E, E, lane, vec, a0);
+        process(a0, T - 1);
+      }
+      return;
+    }
+    // one token at a time, two row buffers used in turn: the next token's row travels while the current one is selected
     float row_a[VPT], row_b[VPT];
     if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row_a);
     while (t < T) {

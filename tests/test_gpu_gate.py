@@ -31,7 +31,12 @@ def logits_for(T, E, seed, ties=False):
                                         (333, 200, 8, True), (333, 40, 8, True), (257, 96, 4, True),
                                         (129, 250, 8, True), (200, 512, 8, True), (96, 1024, 32, True),
                                         (100, 32, 32, True), (5000, 256, 8, "few"), (300, 128, 32, "few"),
-                                        (64, 256, 8, "zeros")])
+                                        (64, 256, 8, "zeros"),
+                                        # batches large enough for two tokens per warp: an odd token count, ties,
+                                        # every long-row form, K at the limit of that path and beyond it
+                                        (6001, 256, 8, False), (5000, 128, 8, True), (4097, 512, 16, True),
+                                        (3000, 1024, 8, False), (3001, 96, 4, True), (2600, 256, 17, True),
+                                        (4000, 256, 8, "zeros")])
 def test_gate_topk_kernel(T, E, K, ties):
     dev = torch.device("cuda:0")
     l = logits_for(T, E, T + E, ties is True)
@@ -112,7 +117,11 @@ def test_gate_plan_matches_oracle_gate_then_oracle_plan(case):
 def test_gate_rows_that_do_not_start_on_16_bytes():
     """The 16-byte row loads need an aligned row; any other pointer or row length takes scalar loads."""
     dev = torch.device("cuda:0")
-    T, E, K = 300, 256, 8
+    for T, E, K in ((300, 256, 8), (3001, 256, 8)):
+        _unaligned_rows(dev, T, E, K)
+
+
+def _unaligned_rows(dev, T, E, K):
     l = logits_for(T, E, 99, True)
     st, want_idx, want_w = oracle.gate_topk(l.numpy(), K)
     buf = torch.zeros(T * E + 3, dtype=torch.float32, device=dev)
