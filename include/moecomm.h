@@ -248,7 +248,9 @@ moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/,
  *                       for it), maps every other rank's window into this process (peer access over NVLink /
  *                       PCIe is enabled by the mapping), and installs the R addresses and generations as the
  *                       context's address table.  Mappings of an earlier handshake are released first.
- *                       Synchronises `stream` before it releases or installs anything.
+ *                       Synchronises `stream` before it releases or installs anything.  The handles must come
+ *                       from OTHER processes (a process cannot map its own export); windows that live in this
+ *                       process are installed with moe_peers_set.
  *   moe_peers_set       installs addresses the caller already has (separate allocations of one process, a
  *                       symmetric-memory mapping, an earlier handshake of its own) without mapping anything:
  *                       window_bases HOST [R] of DEVICE pointers, generations HOST [R] or NULL (all zero);

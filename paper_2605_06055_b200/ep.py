@@ -74,15 +74,6 @@ def addresses_stale(table_generations, announced_generations) -> bool:
     return not np.array_equal(np.asarray(table_generations, np.int32), np.asarray(announced_generations, np.int32))
 
 
-def symmetric_windows(capacity_rows: int, H: int, device, group=None):
-    """Alternative to the handle exchange where torch's symmetric memory is available: allocates this rank's
-    window there and returns (window, list of all ranks' window addresses) for moe_peers_set."""
-    import torch.distributed._symmetric_memory as symm_mem
-    win = symm_mem.empty((capacity_rows, H), dtype=torch.bfloat16, device=device)
-    hdl = symm_mem.rendezvous(win, group if group is not None else dist.group.WORLD)
-    return win, [int(p) for p in hdl.buffer_ptrs]
-
-
 class EpRank:
     """The calls of one rank, in the order the schedules prescribe.  mode: "cached" or "handshake"."""
 

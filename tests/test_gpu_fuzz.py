@@ -84,3 +84,38 @@ def test_random_shape_fused_call_and_quantised_dispatch(i):
     assert np.array_equal(wq.cpu().numpy(), want_q)
     assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
     comm.close()
+
+
+@pytest.mark.parametrize("i", range(max(16, N_SHAPES // 3)))
+def test_random_gate_shape(i):
+    """Top-k gating on random row lengths (every register form and the shared-memory form), top-k degrees up to
+    the limit, batches on both sides of the two-tokens-per-warp switch, with and without many equal logits, rows
+    that do and do not start on 16 bytes: indexes bit for bit, weights within the softmax budget."""
+    rng = np.random.default_rng(99000 + i)
+    E = int(rng.choice([1, 2, 7, 8, 31, 32, 33, 60, 64, 100, 128, 129, 200, 256, 257, 384, 512, 700, 1024, 1025, 2000]))
+    K = int(rng.integers(1, min(E, 32) + 1))
+    T = int(rng.choice([1, 2, 3, 50, 333, 1000, 2368, 2369, 3001, 5000]))
+    kind = int(rng.integers(0, 4))
+    g = torch.Generator().manual_seed(99000 + i)
+    l = torch.randn(T, E, generator=g) * 3
+    if kind == 1:
+        l = torch.round(l)                 # many equal logits
+    elif kind == 2:
+        l = torch.round(l / 6)             # three distinct values: the index decides nearly everything
+    elif kind == 3:
+        l[:, ::3] = -0.0                   # signed zeros among ordinary values
+        l[:, 1::3] = 0.0
+    st, want_idx, want_w = oracle.gate_topk(l.contiguous().numpy(), K)
+    assert st == oracle.OK
+    dev = torch.device("cuda:0")
+    off = int(rng.integers(0, 4))          # 0: aligned rows (if E % 4 == 0); else rows start off 16 bytes
+    buf = torch.zeros(T * E + 3, dtype=torch.float32, device=dev)
+    logits = buf[off:off + T * E].view(T, E)
+    logits.copy_(l)
+    idx = torch.full((T, K), -1, dtype=torch.int32, device=dev)
+    w = torch.full((T, K), -1.0, dtype=torch.float32, device=dev)
+    assert binding.moe_gate_topk(logits, K, idx, w) == binding.MOE_OK
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), want_idx), (E, K, T, kind, off)
+    rtol = (2 * K + 8) * 2.0 ** -24        # libm difference of the terms, two K-term sums, two divisions (see test_gpu_gate.py)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=rtol, atol=1e-12), (E, K, T, kind, off)

@@ -1,8 +1,12 @@
 """Top-k gating on the GPU (stand-alone and fused with the planner) against the CPU oracle.
 
 Indexes are compared bit for bit.  Weights are fp32 softmax values whose exponentials come from two
-different libms (device expf: <= 2 ulp, host expf: <= 1 ulp), followed by a K-term sum and a division:
-the relative budget is (2 + 1 + K/2 + 2) * 2^-24, below 1.3e-6 for K <= 32; the tests allow 2e-6.
+different libms (device expf: <= 2 ulp, host expf: <= 1 ulp: 3 ulp = 6 half-ulps between the two sides' terms),
+followed on each side by a K-term fp32 sum in ascending j -- each of its K-1 additions rounds by up to half an
+ulp of the running sum, and when many selected logits are equal those roundings all fall the same way, while a
+one-ulp difference in the addend can turn them the other way on the other side: up to 2(K-1) half-ulps between
+the sides -- and a division (one half-ulp each side).  Relative budget: (2K + 8) * 2^-24, e.g. 1.4e-6 at K = 8,
+4.3e-6 at K = 32 (a seeded case with K = 28 and two thirds of the logits equal reaches 2.3e-6).
 """
 import numpy as np
 import pytest
@@ -13,7 +17,10 @@ from paper_2605_06055_b200 import binding, synth
 from paper_2605_06055_b200.synth import DECODE, PREFILL
 
 pytestmark = pytest.mark.gpu
-RTOL = 2e-6
+
+
+def gate_rtol(K: int) -> float:
+    return (2 * K + 8) * 2.0 ** -24
 
 
 def logits_for(T, E, seed, ties=False):
@@ -53,7 +60,7 @@ def test_gate_topk_kernel(T, E, K, ties):
     assert binding.moe_gate_topk(l.to(dev), K, idx, w) == binding.MOE_OK
     torch.cuda.synchronize()
     assert np.array_equal(idx.cpu().numpy(), want_idx)
-    assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=gate_rtol(K), atol=1e-12)
 
 
 @pytest.mark.parametrize("case", [
@@ -83,7 +90,7 @@ def test_gate_plan_matches_oracle_gate_then_oracle_plan(case):
     comm.moe_slots(C, slots)
     assert comm.moe_status() == 0
     assert np.array_equal(idx.cpu().numpy(), want_idx)
-    assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=gate_rtol(K), atol=1e-12)
     assert np.array_equal(slots.cpu().numpy().astype(np.int64), want_slots)
     v = comm.moe_plan_view()
     assert np.array_equal(v["large_off"].cpu().numpy(), p.o) and np.array_equal(v["n_recv"].cpu().numpy(), p.n_recv)
@@ -108,7 +115,7 @@ def test_gate_plan_matches_oracle_gate_then_oracle_plan(case):
         comm.moe_combine(win, C, w, y)
     assert comm.moe_status() == 0
     assert np.array_equal(idx.cpu().numpy(), want_idx)
-    assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+    assert np.allclose(w.cpu().numpy(), want_w, rtol=gate_rtol(K), atol=1e-12)
     assert torch.equal(win.view(torch.int16), win_sep.view(torch.int16))
     assert torch.equal(y.view(torch.int16) & 0x7FFF, x.view(torch.int16) & 0x7FFF)
     comm.close()
@@ -133,7 +140,7 @@ def _unaligned_rows(dev, T, E, K):
         assert binding.moe_gate_topk(shifted, K, idx, w) == binding.MOE_OK
         torch.cuda.synchronize()
         assert np.array_equal(idx.cpu().numpy(), want_idx)
-        assert np.allclose(w.cpu().numpy(), want_w, rtol=RTOL, atol=1e-12)
+        assert np.allclose(w.cpu().numpy(), want_w, rtol=gate_rtol(K), atol=1e-12)
 
 
 def test_gate_argument_checks():
