@@ -474,3 +474,44 @@ def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
             assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
             assert got["handshakes_in_timed_steps"] == want_handshakes
             assert got["step_us"] > 0 and got["dispatch_phase_us"] > 0 and got["combine_phase_us"] > 0
+
+
+def _ep_leg_nccl_single_rank(port, results):
+    import os
+    import torch.distributed as dist
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK="0", WORLD_SIZE="1")
+    try:
+        import bench
+        dev = torch.device("cuda:0")
+        torch.cuda.set_device(dev)
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+        results[0] = ("ok", bench.ep_leg(dev, 3, None, shapes=("decode",)))
+        dist.destroy_process_group()
+    except Exception as exc:
+        import traceback
+        results[0] = ("error", repr(exc) + "\n" + traceback.format_exc())
+
+
+def test_benchmark_expert_parallel_leg_over_nccl_with_one_rank():
+    """The same leg over the backend a multi-GPU run uses (NCCL: device tensors in every exchange), with the one
+    rank this machine can give it: the exchanges, the handshake with no peer to map, and the device-side phase order
+    WITHOUT the host barrier between signal and wait (one rank per GPU), which a single rank satisfies by itself."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as m:
+        results = m.dict()
+        p_ = ctx.Process(target=_ep_leg_nccl_single_rank, args=(38000 + os.getpid() % 2000, results))
+        p_.start()
+        p_.join(timeout=300)
+        if p_.is_alive():
+            p_.terminate()
+            raise AssertionError("the rank did not finish")
+        res = dict(results)
+    assert res[0][0] == "ok", res
+    leg = res[0][1]
+    assert leg["ranks"] == 1 and leg["ranks_share_a_gpu"] is False
+    for variant in ("cached_addresses__host_phase_order", "handshake_addresses__host_phase_order",
+                    "cached_addresses__device_phase_order"):
+        got = leg["decode"][variant]
+        assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
+        assert got["step_us"] > 0
