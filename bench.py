@@ -662,6 +662,43 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
     return out
 
 
+def spawn_ep_child(cmd, env, timeout_s: float) -> dict:
+    """Runs the expert-parallel leg of this rank as a child process (its own process group over MASTER_PORT + 17)
+    and returns what its rank 0 printed.  The leg touches other GPUs' memory and waits for other ranks; run apart
+    from the replica figures, a failure there -- an address handshake that is refused, a rank that dies, a wait
+    that never returns -- ends with the child (killed by exact PID after timeout_s) and an `error` entry, never with
+    the loss of the benchmark's line."""
+    try:
+        done = subprocess.run(cmd, env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=timeout_s)
+    except subprocess.TimeoutExpired:
+        return {"error": f"the expert-parallel leg did not finish within {timeout_s:.0f} s; its process was ended"}
+    if done.returncode != 0:
+        return {"error": f"the expert-parallel leg exited with code {done.returncode}",
+                "stderr_tail": done.stderr[-400:]}
+    for ln in reversed(done.stdout.splitlines()):
+        if ln.startswith("{"):
+            return json.loads(ln)
+    return {}
+
+
+def run_ep_child(args) -> None:
+    """`--ep-child`: one rank of the expert-parallel leg; rank 0 prints the leg's JSON object."""
+    import torch.distributed as dist
+    local = int(os.environ.get("LOCAL_RANK", "0")) if args.ep_device < 0 else args.ep_device
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    if args.ep_backend == "nccl":
+        dist.init_process_group("nccl", device_id=dev)
+    else:
+        dist.init_process_group(args.ep_backend)
+    shapes = tuple(args.ep_shapes.split(","))
+    out = ep_leg(dev, args.steps or 20, None, shapes=shapes)
+    if dist.get_rank() == 0:
+        print(json.dumps(out), flush=True)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def kernel_table(wl, r, peak):
     med = statistics.median
     mean = lambda v: sum(v) / len(v)
@@ -761,11 +798,14 @@ def run_cuda(args, wl):
     clocks = sampler.stop()
     ep_result = None
     if world > 1:
-        # the replicas' buffers are not needed any more; every rank takes part in the expert-parallel leg
-        try:
-            ep_result = ep_leg(dev, min(args.steps, 20))
-        except Exception as exc:           # reported in the line, the replica numbers stand
-            ep_result = {"ranks": world, "error": repr(exc)}
+        # every rank starts its part of the expert-parallel leg as a child process (see spawn_ep_child)
+        # (its own store on another port: the launcher's store holds this process group's keys)
+        env = dict(os.environ, MASTER_PORT=str(int(os.environ.get("MASTER_PORT", "29500")) + 17),
+                   TORCHELASTIC_USE_AGENT_STORE="False")
+        cmd = [sys.executable, os.path.abspath(__file__), "--ep-child", "--steps", str(min(args.steps, 20))]
+        ep_result = spawn_ep_child(cmd, env, timeout_s=420.0)
+        ep_result.setdefault("ranks", world)
+        barrier()
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -876,9 +916,16 @@ def main():
     ap.add_argument("--no-decode", action="store_true", help="skip the decode-latency leg (profiling runs)")
     ap.add_argument("--no-prefill-sizes", action="store_true",
                     help="skip the other prefill sizes the roofline target is stated on (c4, c5 at T=65536)")
+    ap.add_argument("--ep-child", action="store_true", help=argparse.SUPPRESS)      # one rank of the expert-parallel leg
+    ap.add_argument("--ep-backend", default="nccl", help=argparse.SUPPRESS)
+    ap.add_argument("--ep-device", type=int, default=-1, help=argparse.SUPPRESS)    # tests: every rank on this GPU
+    ap.add_argument("--ep-shapes", default="decode,prefill", help=argparse.SUPPRESS)
     ap.add_argument("--decode-grid", action="store_true",
                     help="also time the batch-size x hidden-size grid of the paper's decode table (off by default)")
     args = ap.parse_args()
+    if args.ep_child:
+        run_ep_child(args)
+        return
     wl = WORKLOADS[args.workload]()
     if args.impl == "reference":                 # the oracle takes ~0.3 s per step on its 1/8 sample
         args.steps = 10 if args.steps is None else args.steps

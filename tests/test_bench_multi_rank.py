@@ -153,3 +153,19 @@ def test_cached_addresses_are_re_exchanged_only_when_a_generation_changes():
     assert logs[0] == logs[1]                                    # every rank takes the same decisions
     assert [s for s, _, _ in logs[0]] == [True, False, False, True, False]
     assert logs[0][2][2] == [1, 1] and logs[0][4][2] == [1, 2]
+
+
+def test_expert_parallel_child_that_fails_or_hangs_costs_only_its_own_entry():
+    """bench.py runs the expert-parallel leg of a multi-GPU run in child processes; a child that exits badly, prints
+    nothing or never returns becomes an `error` entry (the child is ended after the timeout), a good one's last
+    JSON line is returned."""
+    import sys
+    import bench
+    env = dict(os.environ)
+    ok = bench.spawn_ep_child([sys.executable, "-c", "print('noise'); print('{\"ranks\": 2, \"decode\": {}}')"], env, 30)
+    assert ok == {"ranks": 2, "decode": {}}
+    bad = bench.spawn_ep_child([sys.executable, "-c", "import sys; sys.stderr.write('boom'); sys.exit(3)"], env, 30)
+    assert "error" in bad and "3" in bad["error"] and "boom" in bad["stderr_tail"]
+    hung = bench.spawn_ep_child([sys.executable, "-c", "import time; time.sleep(60)"], env, 1.5)
+    assert "error" in hung and "did not finish" in hung["error"]
+    assert bench.spawn_ep_child([sys.executable, "-c", "pass"], env, 30) == {}

@@ -515,3 +515,28 @@ def test_benchmark_expert_parallel_leg_over_nccl_with_one_rank():
         got = leg["decode"][variant]
         assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
         assert got["step_us"] > 0
+
+
+def test_expert_parallel_child_mode_of_the_benchmark_two_ranks_on_one_gpu():
+    """`bench.py --ep-child`, which a multi-GPU run of the benchmark starts once per rank, here as two processes on
+    the one GPU over gloo: rank 0 prints the leg's JSON object."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    port = 39000 + os.getpid() % 2000
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.join(root, "bench.py"), "--ep-child", "--ep-backend", "gloo",
+                                       "--ep-device", "0", "--ep-shapes", "decode", "--steps", "3"], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = [p_.communicate(timeout=300) for p_ in procs]
+    assert all(p_.returncode == 0 for p_ in procs), [o[1][-600:] for o in outs]
+    leg = json.loads([ln for ln in outs[0][0].splitlines() if ln.startswith("{")][-1])
+    assert leg["ranks"] == 2 and leg["ranks_share_a_gpu"] is True
+    for variant in ("cached_addresses__host_phase_order", "handshake_addresses__host_phase_order",
+                    "cached_addresses__device_phase_order"):
+        assert leg["decode"][variant]["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
+    assert not [ln for ln in outs[1][0].splitlines() if ln.startswith("{")]       # only rank 0 prints
