@@ -60,3 +60,23 @@ def test_null_handles_and_strings(lib):
     for code in range(7):
         assert binding.status_string(code)
     assert binding.status_string(binding.MOE_ERR_CAPACITY) != binding.status_string(binding.MOE_OK)
+
+
+def test_window_and_state_sizes_host_logic(lib):
+    """Sizes of a window allocation with the state region of the device-side phase order behind its rows."""
+    assert binding.moe_state_bytes(1) == 256 and binding.moe_state_bytes(16) == 256      # 4 slots x R epochs, 256-byte units
+    assert binding.moe_state_bytes(64) == 1024 and binding.moe_state_bytes(256) == 4096
+    assert binding.moe_state_bytes(0) == 0 and binding.moe_state_bytes(257) == 0
+    shape = binding.MoeShape(2048, 7168, 256, 16, 8)
+    rows = 1300 * 7168 * 2
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 0) == rows
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 1) == (rows + 255) // 256 * 256 + 256
+    assert lib.moe_window_bytes(ctypes.byref(shape), -1, 1) == 0 and lib.moe_window_bytes(None, 8, 1) == 0
+    assert ctypes.sizeof(binding.MoeWindowHandle) == 88
+    # calls that need a context reject a missing one before touching anything
+    assert lib.moe_peers_check(None, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_signal_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_wait_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_dispatch_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_window_export(None, 16, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert binding.status_string(binding.MOE_ERR_STALE_PEERS) != binding.status_string(binding.MOE_ERR_CUDA)
