@@ -490,7 +490,6 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
         tgs = time_repeated(pre + [replay_serial], n)
         tgf = time_repeated(pre + [replay_fused], n)
         tf = time_repeated(pre + [fused, comb], n)
-        t_gate = time_repeated(pre + [gate], n)
         t_gate_plan = time_repeated(pre + [gate_plan], n)
         t_gate_step = time_repeated(pre + gate_step, n)
         assert c.moe_status() == 0
@@ -503,7 +502,7 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
                      "step_us_plan_dispatch_fused_cuda_graph": tgf - base,
                      "dispatch_GBps": bytes_dispatch(dwl) / (t2 - t1) / 1e3,
                      "combine_GBps": bytes_combine(dwl) / (t3 - t2) / 1e3,
-                     "gate_us": t_gate - base, "gate_plan_us": t_gate_plan - base,
+                     "gate_plan_us": t_gate_plan - base,
                      "step_us_gate_plan_dispatch_fused_then_combine": t_gate_step - base,
                      "plain_copy_of_the_same_bytes_us": t_copy - base,
                      "dispatch_quant_us": t_quant - base,
