@@ -602,12 +602,19 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
         ref.moe_dispatch(g_X, ref_win, C)
         assert ref.moe_status() == 0
         mine_ref = ref_win[rank * C:(rank + 1) * C].clone()
-        del ref_win, g_X, g_idx
+        del ref_win
+        ref_q = torch.zeros((R * C, wl.H), dtype=torch.uint8, device=dev)
+        ref_s = torch.zeros((R * C,), dtype=torch.float32, device=dev)
+        ref.moe_dispatch_quant(g_X, ref_q, ref_s, C)
+        assert ref.moe_status() == 0
+        mine_ref_q, mine_ref_s = ref_q[rank * C:(rank + 1) * C].clone(), ref_s[rank * C:(rank + 1) * C].clone()
+        del ref_q, ref_s, g_X, g_idx
         ref.close()
         for mode, sync in variants:
             name = f"{mode}_addresses__{sync}_phase_order"
             me = ep.EpRank(wl.T // R, wl.H, wl.E, wl.K, dev, group, mode=mode, sync=sync, host_fence=shared_gpu)
-            window = me.new_window(C)             # rows + zeroed state region, attached
+            with_quant = (mode, sync) == ("cached", "host")   # this variant also times the quantised dispatch
+            window = me.new_window(C, quant=with_quant)       # rows + zeroed state region (+ codes, scales), attached
             ok, why = 1.0, ""
             try:
                 me.plan(wl.schedule, idx)
@@ -653,10 +660,30 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
                          "dispatch_phase_us": red(mean(1, 2)), "combine_phase_us": red(mean(2, 3)),
                          "handshakes_in_timed_steps": me.handshakes - handshakes0, "steps": steps,
                          "dispatch_bytes_per_rank": bytes_dispatch(wl) // R}
+            if with_quant:
+                # row-wise quantised dispatch through the same address table: codes and scales of this rank against
+                # the single-GPU path's, then timed like the dispatch phase above
+                me.plan(wl.schedule, idx)
+                me.dispatch_quant(X)
+                assert me.status() == 0
+                codes, scales = me.quant_views()
+                same = bool(torch.equal(codes, mine_ref_q)) and bool(torch.equal(scales.view(torch.int32),
+                                                                                 mine_ref_s.view(torch.int32)))
+                assert _group_reduce(1.0 if same else 0.0, dist.ReduceOp.MIN, dev, group) == 1.0, \
+                    f"expert-parallel leg ({key}): quantised dispatch differs on rank {rank}"
+                qe = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+                for a, b in qe:
+                    me.plan(wl.schedule, idx)
+                    a.record()
+                    me.dispatch_quant(X)
+                    b.record()
+                    me._host_barrier()
+                res[name]["quantised_dispatch_phase_us"] = red(sum(a.elapsed_time(b) for a, b in qe) / steps * 1e3)
+                res[name]["verified"]["quantised_codes_and_scales_equal_single_gpu_path"] = True
             me.close()
             del window
         out[key] = res
-        del inp, X, Y, idx, w, mine_ref
+        del inp, X, Y, idx, w, mine_ref, mine_ref_q, mine_ref_s
         torch.cuda.empty_cache()
     return out
 

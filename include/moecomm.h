@@ -254,13 +254,15 @@ moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/,
  *   moe_peers_set       installs addresses the caller already has (separate allocations of one process, a
  *                       symmetric-memory mapping, an earlier handshake of its own) without mapping anything:
  *                       window_bases HOST [R] of DEVICE pointers, generations HOST [R] or NULL (all zero);
- *                       with_state != 0: every window is followed by its state region (see moe_signal_peers).
+ *                       flags: MOE_WINDOW_* bits saying what follows the rows of EVERY window.
  *   moe_peers_check     the cached-address test: MOE_OK if a table is installed and its generations equal
  *                       `generations` (HOST [R], what the ranks announced for this call -- the binding sends each
  *                       rank's generation along with its count row, so the test costs no exchange of its own);
  *                       MOE_ERR_STALE_PEERS otherwise.
- *   moe_dispatch_cached / moe_combine_cached
- *                       as moe_dispatch_peers / moe_combine_peers with the installed table and its capacity.
+ *   moe_dispatch_cached / moe_combine_cached / moe_dispatch_quant_cached
+ *                       as moe_dispatch_peers / moe_combine_peers / moe_dispatch_quant_peers with the installed
+ *                       table and its capacity (the quantised form needs windows exported with MOE_WINDOW_QUANT:
+ *                       codes and scales land in the parts of every rank's allocation that flag reserves).
  *                       `generations` as in moe_peers_check (NULL: no test); with a stale or missing table they
  *                       return MOE_ERR_STALE_PEERS and enqueue nothing -- no stale address is ever dereferenced.
  *   moe_peers_close     synchronises `stream`, releases the mappings of moe_peers_open and forgets the table
@@ -274,27 +276,36 @@ typedef struct {
   int64_t bytes;         /* size of the window                                                 */
   int32_t device;        /* device ordinal of the exporter                                     */
   int32_t generation;    /* exporter's window generation                                       */
+  int32_t flags;         /* MOE_WINDOW_*: what follows the rows inside the exported range      */
+  int32_t reserved;
 } moe_window_handle_t;
-moe_status_t moe_window_export(const void* window /*DEVICE*/, int64_t bytes, int32_t generation,
+/* What a window allocation holds behind its [capacity_rows, H] bf16 rows (each part starts on a 256-byte boundary,
+ * in this order; moe_window_bytes gives the total): */
+#define MOE_WINDOW_STATE 1 /* the state region of the device-side phase order (moe_signal_peers), zeroed once   */
+#define MOE_WINDOW_QUANT 2 /* the e4m3 code window [capacity_rows, H] uint8 and the scale tensor [capacity_rows]
+                              fp32 of the row-wise quantised dispatch (moe_dispatch_quant_cached)               */
+moe_status_t moe_window_export(const void* window /*DEVICE*/, int64_t bytes, int32_t generation, int32_t flags,
                                moe_window_handle_t* out /*HOST*/);
 moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles /*HOST [R]*/, int32_t my_rank,
                             void* my_window /*DEVICE*/, int64_t capacity_rows, void* stream);
 moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases /*HOST [R]*/,
                            const int32_t* generations /*HOST [R] or NULL*/, int32_t my_rank, int64_t capacity_rows,
-                           int32_t with_state, void* stream);
+                           int32_t flags, void* stream);
 moe_status_t moe_peers_check(const moe_ctx_t* ctx, const int32_t* generations /*HOST [R]*/);
 moe_status_t moe_dispatch_cached(moe_ctx_t* ctx, const void* x /*DEVICE*/, const int32_t* generations /*HOST or NULL*/,
                                  void* stream);
 moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations /*HOST or NULL*/,
                                 const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
+moe_status_t moe_dispatch_quant_cached(moe_ctx_t* ctx, const void* x /*DEVICE*/,
+                                       const int32_t* generations /*HOST or NULL*/, void* stream);
 moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
 
 /* Synchronisation metadata in the pooled memory (Section 3.2: every rank's slice carries communicator state
  * beside its payload; Section 5.4: status flags and wait symbols order producers and consumers across ranks).
  * A window allocation may be followed by a state region of moe_state_bytes(R) bytes -- allocate
- * moe_window_bytes(shape, capacity_rows, 1), zero the state region once -- which the handshake maps together
- * with the rows (moe_peers_open finds it from the exported size; moe_peers_set is told by with_state).  It
- * holds MOE_SYNC_SLOTS arrays of R 32-bit epochs.
+ * moe_window_bytes(shape, capacity_rows, MOE_WINDOW_STATE), zero the state region once, export with that flag --
+ * which the handshake maps together with the rows (every rank must export the same flags).  It holds
+ * MOE_SYNC_SLOTS arrays of R 32-bit epochs.
  *   moe_signal_peers  enqueues, behind everything already on `stream`, a store of `epoch` into entry
  *                     [slot][my_rank] of EVERY rank's state region (release, system scope): "what I enqueued
  *                     before this -- my rows in your window, my experts' outputs -- is complete".
@@ -312,7 +323,7 @@ moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
  * caller must know that the signals were sent before the wait is enqueued). */
 #define MOE_SYNC_SLOTS 4
 size_t moe_state_bytes(int32_t R);
-size_t moe_window_bytes(const moe_shape_t* shape /*HOST*/, int64_t capacity_rows, int32_t with_state);
+size_t moe_window_bytes(const moe_shape_t* shape /*HOST*/, int64_t capacity_rows, int32_t flags);
 moe_status_t moe_signal_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream);
 moe_status_t moe_wait_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream);
 

@@ -29,9 +29,10 @@ EXPORTS = [
     "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant", "moe_expert_tiles", "moe_dispatch_quant_peers",
     "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
     "moe_dispatch_cached", "moe_combine_cached", "moe_state_bytes", "moe_window_bytes", "moe_signal_peers",
-    "moe_wait_peers",
+    "moe_wait_peers", "moe_dispatch_quant_cached",
 ]
 MOE_SYNC_SLOTS = 4
+MOE_WINDOW_STATE, MOE_WINDOW_QUANT = 1, 2
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -49,7 +50,8 @@ class MoePlanView(ctypes.Structure):
 class MoeWindowHandle(ctypes.Structure):
     """moe_window_handle_t: plain bytes describing one rank's window to the other ranks."""
     _fields_ = [("ipc", ctypes.c_ubyte * 64), ("offset", ctypes.c_int64), ("bytes", ctypes.c_int64),
-                ("device", ctypes.c_int32), ("generation", ctypes.c_int32)]
+                ("device", ctypes.c_int32), ("generation", ctypes.c_int32), ("flags", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
 
 
 WINDOW_HANDLE_BYTES = ctypes.sizeof(MoeWindowHandle)
@@ -109,7 +111,9 @@ def load() -> ctypes.CDLL:
     L.moe_dispatch_quant_peers.restype = ctypes.c_int
     L.moe_dispatch_quant.argtypes = [vp, vp, vp, vp, i64, vp]
     L.moe_dispatch_quant.restype = ctypes.c_int
-    L.moe_window_export.argtypes = [vp, i64, i32, ctypes.POINTER(MoeWindowHandle)]
+    L.moe_window_export.argtypes = [vp, i64, i32, i32, ctypes.POINTER(MoeWindowHandle)]
+    L.moe_dispatch_quant_cached.argtypes = [vp, vp, vp, vp]
+    L.moe_dispatch_quant_cached.restype = ctypes.c_int
     L.moe_peers_open.argtypes = [vp, vp, i32, vp, i64, vp]
     L.moe_peers_set.argtypes = [vp, vp, vp, i32, i64, i32, vp]
     L.moe_state_bytes.argtypes = [i32]
@@ -379,16 +383,16 @@ class MoeComm:
             raise MoeError(rc, "moe_peers_open")
         return rc
 
-    def moe_peers_set(self, window_bases, generations, capacity_rows: int, my_rank: int = 0, with_state: bool = False,
+    def moe_peers_set(self, window_bases, generations, capacity_rows: int, my_rank: int = 0, flags: int = 0,
                       stream=None, check: bool = True) -> int:
-        """window_bases: R device addresses (ints); generations: R ints or None; with_state: every window is
-        followed by its state region (moe_window_bytes(..., with_state=True) bytes were allocated for it)."""
+        """window_bases: R device addresses (ints); generations: R ints or None; flags: MOE_WINDOW_* bits saying
+        what follows the rows of every window (moe_window_bytes(capacity_rows, flags) bytes were allocated)."""
         bases = np.ascontiguousarray(window_bases, dtype=np.uint64)
         gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
         assert bases.shape == (self.R,) and (gens is None or gens.shape == (self.R,))
         with self._on_device():
             rc = self.lib.moe_peers_set(self._h, _host_ptr(bases), _host_ptr(gens), int(my_rank), int(capacity_rows),
-                                        int(bool(with_state)), _stream_handle(stream))
+                                        int(flags), _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_peers_set")
         return rc
@@ -421,8 +425,17 @@ class MoeComm:
             raise MoeError(rc, "moe_combine_cached")
         return rc
 
-    def moe_window_bytes(self, capacity_rows: int, with_state: bool = True) -> int:
-        return int(self.lib.moe_window_bytes(ctypes.byref(self._shape), int(capacity_rows), int(bool(with_state))))
+    def moe_window_bytes(self, capacity_rows: int, flags: int = MOE_WINDOW_STATE) -> int:
+        return int(self.lib.moe_window_bytes(ctypes.byref(self._shape), int(capacity_rows), int(flags)))
+
+    def moe_dispatch_quant_cached(self, x: torch.Tensor, generations=None, stream=None, check: bool = True) -> int:
+        gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
+        with self._on_device():
+            rc = self.lib.moe_dispatch_quant_cached(self._h, _dev_ptr(x, torch.bfloat16), _host_ptr(gens),
+                                                    _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_quant_cached")
+        return rc
 
     def moe_signal_peers(self, slot: int, epoch: int, stream=None, check: bool = True) -> int:
         with self._on_device():
@@ -576,12 +589,13 @@ def moe_state_bytes(R: int) -> int:
     return int(load().moe_state_bytes(int(R)))
 
 
-def moe_window_export(window: torch.Tensor, generation: int) -> bytes:
-    """Handle of one rank's window for the other ranks (see include/moecomm.h): WINDOW_HANDLE_BYTES plain bytes."""
+def moe_window_export(window: torch.Tensor, generation: int, flags: int = 0) -> bytes:
+    """Handle of one rank's window allocation for the other ranks (see include/moecomm.h): WINDOW_HANDLE_BYTES plain
+    bytes.  flags: MOE_WINDOW_* bits saying what the allocation holds behind its rows."""
     h = MoeWindowHandle()
     with torch.cuda.device(window.device):
         rc = int(load().moe_window_export(_dev_ptr(window), window.numel() * window.element_size(), int(generation),
-                                          ctypes.byref(h)))
+                                          int(flags), ctypes.byref(h)))
     if rc != MOE_OK:
         raise MoeError(rc, "moe_window_export")
     return bytes(h)

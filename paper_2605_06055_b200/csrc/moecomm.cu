@@ -57,6 +57,9 @@ struct moe_ctx {
   int64_t peer_capacity;
   bool peers_installed;
   bool peers_have_state;              // every installed window is followed by its state region
+  bool peers_have_quant;              // ... and by a code window and a scale tensor
+  unsigned char** code_table;         // device, [R]: e4m3 code window of every rank
+  float** scale_table;                // device, [R]: scale tensor of every rank
   int32_t my_rank;                    // this process's rank in the installed table
   unsigned char** state_table;        // device, [R]: state region of every rank (inside the workspace)
   // resident CTAs per SM of the row kernels this context has launched (occupancy calculator results)
@@ -108,7 +111,7 @@ Layout layout_of(const moe_shape_t* s) {
   L.o = take(sizeof(int32_t) * s->E * s->R);
   L.n_exp = take(sizeof(int32_t) * s->E);
   L.n_recv = take(sizeof(int32_t) * s->R);
-  L.peers = take(sizeof(void*) * s->R * 2);   // window bases, then state-region bases
+  L.peers = take(sizeof(void*) * s->R * 4);   // window bases, state regions, code windows, scale tensors
   L.s = take(sizeof(int32_t) * B);
   L.tile_rank = take(sizeof(int32_t) * B);
   L.tile_hist = take(sizeof(int32_t) * (size_t)max_tiles(s) * s->E);
@@ -372,7 +375,10 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->peer_table = reinterpret_cast<const unsigned char**>(ctx->ws + L.peers);
   ctx->state_table = reinterpret_cast<unsigned char**>(ctx->ws + L.peers) + shape->R;
   ctx->peers_installed = false;
+  ctx->code_table = ctx->state_table + shape->R;
+  ctx->scale_table = reinterpret_cast<float**>(ctx->code_table + shape->R);
   ctx->peers_have_state = false;
+  ctx->peers_have_quant = false;
   ctx->my_rank = 0;
   ctx->peer_capacity = 0;
   for (int d = 0; d < MOE_MAX_R; ++d) {
@@ -983,22 +989,44 @@ void release_mappings(moe_ctx* ctx) {
 
 size_t state_bytes_for(int32_t R) { return align_up(sizeof(uint32_t) * MOE_SYNC_SLOTS * (size_t)R); }
 
-// Copies the host table (and the state-region addresses, which follow the rows of every window) to the device
-// tables on `stream` and marks them installed.
-moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows, bool with_state, cudaStream_t st) {
+// Parts of a window allocation, byte offsets from its first row (see MOE_WINDOW_* in the header).
+struct WindowParts {
+  size_t state, codes, scales, total;
+};
+WindowParts window_parts(const moe_shape_t& sh, int64_t capacity_rows, int32_t flags) {
+  WindowParts p;
+  const size_t rows = (size_t)capacity_rows * sh.H * 2;
+  size_t at = flags != 0 ? align_up(rows) : rows;
+  p.state = at;
+  if (flags & MOE_WINDOW_STATE) at += state_bytes_for(sh.R);
+  p.codes = at;
+  if (flags & MOE_WINDOW_QUANT) at += align_up((size_t)capacity_rows * sh.H);
+  p.scales = at;
+  if (flags & MOE_WINDOW_QUANT) at += align_up((size_t)capacity_rows * sizeof(float));
+  p.total = at;
+  return p;
+}
+
+// Copies the addresses of every rank's rows, state region, code window and scale tensor to the device tables on
+// `stream` and marks them installed.
+moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows, int32_t flags, cudaStream_t st) {
   const int R = ctx->shape.R;
-  void* both[2 * MOE_MAX_R];
-  const size_t rows_bytes = align_up((size_t)capacity_rows * ctx->shape.H * 2);
+  void* all[4 * MOE_MAX_R];
+  const WindowParts parts = window_parts(ctx->shape, capacity_rows, flags);
   for (int d = 0; d < R; ++d) {
-    both[d] = ctx->peer_ptr[d];
-    both[R + d] = with_state ? static_cast<char*>(ctx->peer_ptr[d]) + rows_bytes : nullptr;
+    char* base = static_cast<char*>(ctx->peer_ptr[d]);
+    all[d] = base;
+    all[R + d] = (flags & MOE_WINDOW_STATE) ? base + parts.state : nullptr;
+    all[2 * R + d] = (flags & MOE_WINDOW_QUANT) ? base + parts.codes : nullptr;
+    all[3 * R + d] = (flags & MOE_WINDOW_QUANT) ? base + parts.scales : nullptr;
   }
   // pageable source: the runtime has staged the bytes by the time the call returns
-  if (cudaMemcpyAsync(ctx->peer_table, both, sizeof(void*) * 2 * R, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  if (cudaMemcpyAsync(ctx->peer_table, all, sizeof(void*) * 4 * R, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   ctx->peer_capacity = capacity_rows;
   ctx->my_rank = my_rank;
-  ctx->peers_have_state = with_state;
+  ctx->peers_have_state = (flags & MOE_WINDOW_STATE) != 0;
+  ctx->peers_have_quant = (flags & MOE_WINDOW_QUANT) != 0;
   ctx->peers_installed = true;
   return MOE_OK;
 }
@@ -1013,8 +1041,11 @@ moe_status_t table_fresh(const moe_ctx* ctx, const int32_t* generations) {
 
 }  // namespace
 
-moe_status_t moe_window_export(const void* window, int64_t bytes, int32_t generation, moe_window_handle_t* out) {
-  if (window == nullptr || out == nullptr || bytes <= 0 || !aligned16(window)) return MOE_ERR_INVALID_ARG;
+moe_status_t moe_window_export(const void* window, int64_t bytes, int32_t generation, int32_t flags,
+                               moe_window_handle_t* out) {
+  if (window == nullptr || out == nullptr || bytes <= 0 || !aligned16(window) ||
+      (flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0)
+    return MOE_ERR_INVALID_ARG;
   static_assert(sizeof(cudaIpcMemHandle_t) == sizeof(out->ipc), "handle size");
   uintptr_t base = 0;
   size_t size = 0;
@@ -1030,6 +1061,8 @@ moe_status_t moe_window_export(const void* window, int64_t bytes, int32_t genera
   out->offset = (int64_t)(at - base);
   out->bytes = bytes;
   out->generation = generation;
+  out->flags = flags;
+  out->reserved = 0;
   if (cudaGetDevice(&out->device) != cudaSuccess) return MOE_ERR_CUDA;
   return MOE_OK;
 }
@@ -1039,13 +1072,12 @@ moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, 
   if (ctx == nullptr || handles == nullptr || my_window == nullptr || my_rank < 0 || my_rank >= ctx->shape.R ||
       capacity_rows < 0 || !aligned16(my_window))
     return MOE_ERR_INVALID_ARG;
-  const int64_t need = capacity_rows * ctx->shape.H * 2;
-  const int64_t need_with_state = (int64_t)(align_up((size_t)need) + state_bytes_for(ctx->shape.R));
-  bool with_state = true;   // only if every rank exported its state region along with its rows
-  for (int d = 0; d < ctx->shape.R; ++d) {
-    if (d != my_rank && (handles[d].bytes < need || (handles[d].offset & 15) != 0)) return MOE_ERR_INVALID_ARG;
-    if (handles[d].bytes < need_with_state) with_state = false;
-  }
+  // every rank exports the same parts, and enough bytes for them at this capacity
+  const int32_t flags = handles[my_rank].flags;
+  if ((flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0) return MOE_ERR_INVALID_ARG;
+  const int64_t need = (int64_t)window_parts(ctx->shape, capacity_rows, flags).total;
+  for (int d = 0; d < ctx->shape.R; ++d)
+    if (handles[d].flags != flags || handles[d].bytes < need || (handles[d].offset & 15) != 0) return MOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;   // nothing in flight reads the old table
   release_mappings(ctx);
@@ -1066,12 +1098,13 @@ moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, 
     ctx->peer_mapping[d] = base;
     ctx->peer_ptr[d] = static_cast<char*>(base) + handles[d].offset;
   }
-  return install_table(ctx, my_rank, capacity_rows, with_state, st);
+  return install_table(ctx, my_rank, capacity_rows, flags, st);
 }
 
 moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, const int32_t* generations, int32_t my_rank,
-                           int64_t capacity_rows, int32_t with_state, void* stream) {
-  if (ctx == nullptr || window_bases == nullptr || capacity_rows < 0 || my_rank < 0 || my_rank >= ctx->shape.R)
+                           int64_t capacity_rows, int32_t flags, void* stream) {
+  if (ctx == nullptr || window_bases == nullptr || capacity_rows < 0 || my_rank < 0 || my_rank >= ctx->shape.R ||
+      (flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0)
     return MOE_ERR_INVALID_ARG;
   for (int d = 0; d < ctx->shape.R; ++d)
     if (window_bases[d] == nullptr || !aligned16(window_bases[d])) return MOE_ERR_INVALID_ARG;
@@ -1082,15 +1115,14 @@ moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, cons
     ctx->peer_ptr[d] = const_cast<void*>(window_bases[d]);
     ctx->peer_gen[d] = generations != nullptr ? generations[d] : 0;
   }
-  return install_table(ctx, my_rank, capacity_rows, with_state != 0, st);
+  return install_table(ctx, my_rank, capacity_rows, flags, st);
 }
 
 size_t moe_state_bytes(int32_t R) { return (R < 1 || R > MOE_MAX_R) ? 0 : state_bytes_for(R); }
 
-size_t moe_window_bytes(const moe_shape_t* shape, int64_t capacity_rows, int32_t with_state) {
-  if (!shape_valid(shape) || capacity_rows < 0) return 0;
-  const size_t rows = (size_t)capacity_rows * shape->H * 2;
-  return with_state ? align_up(rows) + state_bytes_for(shape->R) : rows;
+size_t moe_window_bytes(const moe_shape_t* shape, int64_t capacity_rows, int32_t flags) {
+  if (!shape_valid(shape) || capacity_rows < 0 || (flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0) return 0;
+  return window_parts(*shape, capacity_rows, flags).total;
 }
 
 moe_status_t moe_signal_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream) {
@@ -1106,8 +1138,8 @@ moe_status_t moe_wait_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* 
   if (ctx == nullptr || slot < 0 || slot >= MOE_SYNC_SLOTS) return MOE_ERR_INVALID_ARG;
   if (!ctx->peers_installed || !ctx->peers_have_state) return MOE_ERR_STALE_PEERS;
   const int R = ctx->shape.R;
-  const size_t rows_bytes = align_up((size_t)ctx->peer_capacity * ctx->shape.H * 2);
-  const unsigned char* mine = static_cast<const unsigned char*>(ctx->peer_ptr[ctx->my_rank]) + rows_bytes;
+  const unsigned char* mine = static_cast<const unsigned char*>(ctx->peer_ptr[ctx->my_rank]) +
+                              window_parts(ctx->shape, ctx->peer_capacity, MOE_WINDOW_STATE).state;
   wait_peers_kernel<<<1, R < 32 ? 32 : (R + 31) / 32 * 32, 0, static_cast<cudaStream_t>(stream)>>>(
       mine, R, slot, epoch, ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT, &ctx->ctl->status);
   return launch_ok(ctx);
@@ -1130,6 +1162,15 @@ moe_status_t moe_dispatch_cached(moe_ctx_t* ctx, const void* x, const int32_t* g
   const moe_status_t fresh = table_fresh(ctx, generations);
   if (fresh != MOE_OK) return fresh;
   return dispatch_impl(ctx, x, nullptr, reinterpret_cast<const void* const*>(ctx->peer_table), ctx->peer_capacity, stream);
+}
+
+moe_status_t moe_dispatch_quant_cached(moe_ctx_t* ctx, const void* x, const int32_t* generations, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  const moe_status_t fresh = table_fresh(ctx, generations);
+  if (fresh != MOE_OK) return fresh;
+  if (!ctx->peers_have_quant) return MOE_ERR_STALE_PEERS;   // the installed windows reserve no room for codes and scales
+  return dispatch_quant_impl(ctx, x, nullptr, nullptr, ctx->peer_capacity, stream, false,
+                             reinterpret_cast<const void* const*>(ctx->code_table), ctx->scale_table);
 }
 
 moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations, const float* topk_w, void* y, void* stream) {

@@ -92,48 +92,61 @@ class EpRank:
         self.message = torch.zeros(E + 1, dtype=torch.int32, device=device)
         self.counts_row = self.message[:E]
         self.window = None
-        self.capacity = 0
+        self.capacity, self.flags = 0, 0
         self.generation = 0                 # of this rank's own window; 0 = none attached
         self.table_generations = None       # generations the installed address table was built from
         self.announced = None               # generations gathered by the latest plan()
         self.handshakes = 0
 
     # -- windows -------------------------------------------------------------------------------------
-    def new_window(self, capacity_rows: int) -> torch.Tensor:
-        """Allocates this rank's window with its state region behind the rows (zeroed), attaches it and returns the
+    def new_window(self, capacity_rows: int, quant: bool = False) -> torch.Tensor:
+        """Allocates this rank's window with its state region behind the rows (zeroed) and, with quant=True, the code
+        window and scale tensor of the quantised dispatch behind that; attaches it and returns the
         [capacity_rows, H] view of the rows."""
-        nbytes = self.comm.moe_window_bytes(capacity_rows, with_state=True)
+        flags = binding.MOE_WINDOW_STATE | (binding.MOE_WINDOW_QUANT if quant else 0)
+        nbytes = self.comm.moe_window_bytes(capacity_rows, flags)
         backing = torch.zeros(nbytes // 2, dtype=torch.bfloat16, device=self.device)
-        self.attach_window(backing, capacity_rows)
+        self.attach_window(backing, capacity_rows, flags)
         return backing[:capacity_rows * self.H].view(capacity_rows, self.H)
 
-    def attach_window(self, window: torch.Tensor, capacity_rows: int) -> None:
+    def quant_views(self):
+        """(codes [capacity_rows, H] uint8, scales [capacity_rows] fp32) of this rank's window allocation."""
+        assert self.flags & binding.MOE_WINDOW_QUANT
+        raw = self.window.view(torch.uint8)
+        scales_at = self.comm.moe_window_bytes(self.capacity, self.flags) - (self.capacity * 4 + 255) // 256 * 256
+        codes_at = scales_at - (self.capacity * self.H + 255) // 256 * 256
+        codes = raw[codes_at:codes_at + self.capacity * self.H].view(self.capacity, self.H)
+        scales = raw[scales_at:scales_at + self.capacity * 4].view(torch.float32)
+        return codes, scales
+
+    def attach_window(self, window: torch.Tensor, capacity_rows: int, flags: int = 0) -> None:
         """This rank's window from now on: a contiguous bf16 tensor whose first capacity_rows * H elements are the
-        rows (the same capacity on every rank); if it is moe_window_bytes(capacity_rows, with_state=True) bytes
-        long, what follows the rows is the state region of the device-side phase order.  A new window gets a
-        new generation, which makes every rank's cached table stale at the next plan()."""
-        assert window.dtype == torch.bfloat16 and window.is_contiguous() and window.numel() >= capacity_rows * self.H
-        new_state = self._state_region(window, capacity_rows)
+        rows (the same capacity on every rank) and which holds, behind them, the parts that `flags` (MOE_WINDOW_*)
+        names: moe_window_bytes(capacity_rows, flags) bytes in all, every rank with the same flags.  A new window
+        gets a new generation, which makes every rank's cached table stale at the next plan()."""
+        assert window.dtype == torch.bfloat16 and window.is_contiguous()
+        assert window.numel() * 2 >= self.comm.moe_window_bytes(capacity_rows, flags)
+        new_state = self._state_region(window, capacity_rows) if flags & binding.MOE_WINDOW_STATE else None
         if self.sync == "device" and new_state is not None and self.window is not None and self.epoch > 0:
             # The epochs move with the window: once every signal of the finished step has arrived in the old state
             # region (the combine-done signals are a step's last), it is copied behind the new rows.
-            old_state = self._state_region(self.window, self.capacity)
+            old_state = self._state_region(self.window, self.capacity) if self.flags & binding.MOE_WINDOW_STATE else None
             if old_state is not None:
                 self.comm.moe_wait_peers(self.SLOT_COMBINED, self.epoch)
                 new_state.copy_(old_state)
-        self.window, self.capacity = window, int(capacity_rows)
+        self.window, self.capacity, self.flags = window, int(capacity_rows), int(flags)
         self.generation += 1
         self.message[self.E:].fill_(self.generation)
 
     def _state_region(self, window: torch.Tensor, capacity_rows: int):
-        """The state region behind the rows of a window allocation, or None if the allocation has none."""
+        """The state region behind the rows of a window allocation that has one."""
         state = binding.moe_state_bytes(self.R) // 2
-        start = self.comm.moe_window_bytes(capacity_rows, with_state=True) // 2 - state
-        return window[start:start + state] if window.numel() >= start + state else None
+        start = self.comm.moe_window_bytes(capacity_rows, binding.MOE_WINDOW_STATE) // 2 - state
+        return window[start:start + state]
 
     def handshake(self) -> None:
         """Collective: exchanges the window handles and maps every other rank's window."""
-        mine = binding.moe_window_export(self.window, self.generation)
+        mine = binding.moe_window_export(self.window, self.generation, self.flags)
         handles = all_gather_bytes(mine, self.device, self.group)
         gens = [binding.MoeWindowHandle.from_buffer_copy(handles, r * binding.WINDOW_HANDLE_BYTES).generation
                 for r in range(self.R)]
@@ -144,7 +157,7 @@ class EpRank:
     def install_addresses(self, window_bases, generations=None) -> None:
         """Addresses obtained elsewhere (one process holding every window; symmetric memory)."""
         gens = np.zeros(self.R, np.int32) if generations is None else np.asarray(generations, np.int32)
-        self.comm.moe_peers_set(window_bases, gens, self.capacity, my_rank=self.rank)
+        self.comm.moe_peers_set(window_bases, gens, self.capacity, my_rank=self.rank, flags=self.flags)
         self.table_generations = gens
 
     def _ensure_addresses(self) -> None:
@@ -197,13 +210,20 @@ class EpRank:
             self._host_barrier()                 # every expert has written its outputs
             self.comm.moe_combine_cached(self.announced, topk_w_local, y_local)
 
-    def dispatch_quant(self, x_local: torch.Tensor, window_q_bases: torch.Tensor, scale_bases: torch.Tensor,
-                       capacity_rows: int) -> None:
-        """Row-wise quantised dispatch: e4m3 codes into every rank's code window, one fp32 scale per row into
-        every rank's scale tensor (tables of R device addresses each, supplied by the caller)."""
-        self.comm.moe_dispatch_quant_peers(x_local, window_q_bases, scale_bases, capacity_rows)
-        torch.cuda.current_stream().synchronize()
-        dist.barrier(self.group)
+    def dispatch_quant(self, x_local: torch.Tensor) -> None:
+        """Row-wise quantised dispatch: e4m3 codes into every rank's code window, one fp32 scale per row into every
+        rank's scale tensor -- the parts of the window allocations that MOE_WINDOW_QUANT reserves, reached through
+        the same address table as the rows.  Returns once this rank's experts may read its codes."""
+        self._ensure_addresses()
+        if self.sync == "device":
+            self.epoch += 1
+            if self.epoch > 1:
+                self.comm.moe_wait_peers(self.SLOT_COMBINED, self.epoch - 1)
+            self.comm.moe_dispatch_quant_cached(x_local, self.announced)
+            self._signal_then_wait(self.SLOT_DISPATCHED)
+        else:
+            self.comm.moe_dispatch_quant_cached(x_local, self.announced)
+            self._host_barrier()
 
     def status(self) -> int:
         return self.comm.moe_status()

@@ -130,11 +130,11 @@ def _address_protocol_worker(rank, world, port, out):
         assert counts.tolist() == [[10 * r + step] * E for r in range(world)]
         stale = ep.addresses_stale(table, announced)
         if stale:                                                # the handshake: handles are opaque bytes
-            mine = bytes([rank, generation]) + bytes(86)
+            mine = bytes([rank, generation]) + bytes(94)
             handles = ep.all_gather_bytes(mine, torch.device("cpu"))
-            assert len(handles) == 88 * world
-            table = np.array([handles[88 * r + 1] for r in range(world)], np.int32)
-            assert [handles[88 * r] for r in range(world)] == list(range(world))
+            assert len(handles) == 96 * world
+            table = np.array([handles[96 * r + 1] for r in range(world)], np.int32)
+            assert [handles[96 * r] for r in range(world)] == list(range(world))
         log.append((bool(stale), announced.tolist(), table.tolist()))
     out[rank] = log
     dist.destroy_process_group()

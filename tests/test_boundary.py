@@ -69,14 +69,21 @@ def test_window_and_state_sizes_host_logic(lib):
     assert binding.moe_state_bytes(0) == 0 and binding.moe_state_bytes(257) == 0
     shape = binding.MoeShape(2048, 7168, 256, 16, 8)
     rows = 1300 * 7168 * 2
+    up = lambda n: (n + 255) // 256 * 256
     assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 0) == rows
-    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 1) == (rows + 255) // 256 * 256 + 256
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_STATE) == up(rows) + 256
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_QUANT) == \
+        up(rows) + up(1300 * 7168) + up(1300 * 4)
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT) == \
+        up(rows) + 256 + up(1300 * 7168) + up(1300 * 4)
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 4) == 0                       # unknown flag
     assert lib.moe_window_bytes(ctypes.byref(shape), -1, 1) == 0 and lib.moe_window_bytes(None, 8, 1) == 0
-    assert ctypes.sizeof(binding.MoeWindowHandle) == 88
+    assert ctypes.sizeof(binding.MoeWindowHandle) == 96
     # calls that need a context reject a missing one before touching anything
     assert lib.moe_peers_check(None, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_signal_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_wait_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_dispatch_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG
-    assert lib.moe_window_export(None, 16, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_window_export(None, 16, 1, 0, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_dispatch_quant_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG
     assert binding.status_string(binding.MOE_ERR_STALE_PEERS) != binding.status_string(binding.MOE_ERR_CUDA)

@@ -204,20 +204,22 @@ def test_signals_and_bounded_waits_between_ranks_of_one_process():
         c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, counts[r])
     for c in comms:
         c.moe_notify(counts)
-    total = comms[0].moe_window_bytes(C, True) // 2
-    assert total * 2 >= C * H * 2 + binding.moe_state_bytes(R) > C * H * 2
+    FLAGS = binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT
+    total = comms[0].moe_window_bytes(C, FLAGS) // 2
+    state_at = (comms[0].moe_window_bytes(C, binding.MOE_WINDOW_STATE) - binding.moe_state_bytes(R)) // 4
+    assert total * 2 >= C * H * 2 + binding.moe_state_bytes(R) + C * H + 4 * C
     backings = [torch.zeros(total, dtype=torch.bfloat16, device=dev) for _ in range(R)]
     rows = [b[:C * H].view(C, H) for b in backings]
     for t in rows:
         t.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
     bases = [b.data_ptr() for b in backings]
     # without a state region the signals have nowhere to go
-    comms[0].moe_peers_set(bases, None, C, my_rank=0, with_state=False)
+    comms[0].moe_peers_set(bases, None, C, my_rank=0, flags=0)
     assert comms[0].moe_signal_peers(0, 1, check=False) == binding.MOE_ERR_STALE_PEERS
     assert comms[0].moe_wait_peers(0, 1, check=False) == binding.MOE_ERR_STALE_PEERS
     for r, c in enumerate(comms):
-        c.moe_peers_set(bases, None, C, my_rank=r, with_state=True)
-    state = lambda d: backings[d].view(torch.int32)[-(binding.moe_state_bytes(R) // 4):][:binding.MOE_SYNC_SLOTS * R].view(binding.MOE_SYNC_SLOTS, R)
+        c.moe_peers_set(bases, None, C, my_rank=r, flags=FLAGS)
+    state = lambda d: backings[d].view(torch.int32)[state_at:state_at + binding.MOE_SYNC_SLOTS * R].view(binding.MOE_SYNC_SLOTS, R)
     for epoch in (1, 2):
         for r, c in enumerate(comms):                      # every rank dispatches and signals ...
             c.moe_dispatch_cached(X[rts[r]:rts[r + 1]].contiguous())
@@ -238,6 +240,23 @@ def test_signals_and_bounded_waits_between_ranks_of_one_process():
             assert c.moe_status() == 0
             Y[rts[r]:rts[r + 1]] = y_r
         assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
+    # the quantised dispatch through the same table: codes and scales land in the parts of every allocation that
+    # MOE_WINDOW_QUANT reserves; a table installed without that flag refuses the call
+    want_q = np.full((R * C, H), 0, np.uint8)
+    want_s = np.full((R * C,), 0.0, np.float32)
+    assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 4) == oracle.OK
+    for r, c in enumerate(comms):
+        c.moe_dispatch_quant_cached(X[rts[r]:rts[r + 1]].contiguous())
+        assert c.moe_status() == 0
+    up = lambda n: (n + 255) // 256 * 256
+    codes_at = up(C * H * 2) + binding.moe_state_bytes(R)
+    scales_at = codes_at + up(C * H)
+    got_q = np.concatenate([b.view(torch.uint8)[codes_at:codes_at + C * H].view(C, H).cpu().numpy() for b in backings])
+    got_s = np.concatenate([b.view(torch.uint8)[scales_at:scales_at + 4 * C].view(torch.float32).cpu().numpy() for b in backings])
+    assert np.array_equal(got_q, want_q) and np.array_equal(got_s.view(np.uint32), want_s.view(np.uint32))
+    comms[0].moe_peers_set(bases, None, C, my_rank=0, flags=binding.MOE_WINDOW_STATE)
+    assert comms[0].moe_dispatch_quant_cached(X[:int(rts[1])].contiguous(), check=False) == binding.MOE_ERR_STALE_PEERS
+    comms[0].moe_peers_set(bases, None, C, my_rank=0, flags=FLAGS)
     # only one of R signals arrives for epoch 3: the wait is bounded (50 ms here), reports, and nothing hangs
     c = comms[1]
     c.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 50)
@@ -268,7 +287,7 @@ def _ipc_workload(world):
                     rank_tokens=c["per"])
 
 
-def _ipc_rank(rank, world, port, mode, sync, q_to, results):
+def _ipc_rank(rank, world, port, mode, sync, results):
     """One expert-parallel rank as its own process on the one GPU: its window lives in its own allocation, the
     other rank's window is mapped in through the library's handle exchange (moe_window_export over a gloo group,
     moe_peers_open), counts travel over the same group, phases are ordered by host barriers (no kernel waits on
@@ -300,10 +319,11 @@ def _ipc_rank(rank, world, port, mode, sync, q_to, results):
         # (rows first, then the zeroed state region of the device-side phase order)
         def new_window(offset_rows):
             backing = torch.zeros(12 << 20, dtype=torch.bfloat16, device=dev)
-            flat = backing[offset_rows * H:offset_rows * H + me.comm.moe_window_bytes(C, True) // 2]
+            flags = binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT
+            flat = backing[offset_rows * H:offset_rows * H + me.comm.moe_window_bytes(C, flags) // 2]
             win = flat[:C * H].view(C, H)
             win.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
-            me.attach_window(flat, C)
+            me.attach_window(flat, C, flags)
             return backing, win
         backing, mine = new_window(0)
         y = torch.empty((hi - lo, H), dtype=torch.bfloat16, device=dev)
@@ -348,18 +368,12 @@ def _ipc_rank(rank, world, port, mode, sync, q_to, results):
         st = st or step()
         log["handshakes_after_step_3"] = me.handshakes
         win_3, y_3 = u16(mine), u16(y)
-        # the quantising dispatch into per-process code windows and scale tensors, mapped through torch's own
-        # inter-process tensors (tables supplied by the caller)
-        my_q = torch.full((C, H), 0xAB, dtype=torch.uint8, device=dev)
-        my_s = torch.full((C,), -1.0, dtype=torch.float32, device=dev)
-        q_to[1 - rank].put((my_q, my_s))
-        other_q, other_s = q_to[rank].get(timeout=60)
-        qs = [my_q, other_q] if rank == 0 else [other_q, my_q]
-        ss = [my_s, other_s] if rank == 0 else [other_s, my_s]
-        q_bases = torch.tensor([t.data_ptr() for t in qs], dtype=torch.int64, device=dev)
-        s_bases = torch.tensor([t.data_ptr() for t in ss], dtype=torch.int64, device=dev)
-        me.dispatch_quant(x, q_bases, s_bases, C)
+        # the quantising dispatch: codes and scales go into the parts of every rank's window allocation that
+        # MOE_WINDOW_QUANT reserves, through the same address table as the rows
+        me.plan(DECODE, idx)
+        me.dispatch_quant(x)
         st = st or me.status()
+        my_q, my_s = me.quant_views()
         dist.barrier()                                 # nobody frees a window another rank may still read
         results[rank] = ("ok", st, C, (win_1, y_1), (win_2, y_2), (win_3, y_3), my_q.cpu().numpy().copy(),
                          my_s.cpu().numpy().copy(), log)
@@ -378,9 +392,8 @@ def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
     world = 2
     with ctx.Manager() as m:
         results = m.dict()
-        q_to = [ctx.Queue(), ctx.Queue()]
         port = 35000 + (os.getpid() * 4 + 2 * (mode == "cached") + (sync == "device")) % 2000
-        procs = [ctx.Process(target=_ipc_rank, args=(r, world, port, mode, sync, q_to, results)) for r in range(world)]
+        procs = [ctx.Process(target=_ipc_rank, args=(r, world, port, mode, sync, results)) for r in range(world)]
         for p_ in procs:
             p_.start()
         for p_ in procs:
@@ -401,8 +414,8 @@ def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
     assert res[1][2] == C
     want = harness.oracle_run(inp, C)
     rts = inp.rank_tok_start
-    want_q = np.full((world * C, H), 0xAB, np.uint8)
-    want_s = np.full((world * C,), -1.0, np.float32)
+    want_q = np.full((world * C, H), 0, np.uint8)          # the allocations start zeroed
+    want_s = np.full((world * C,), 0.0, np.float32)
     assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 2) == oracle.OK
     for r in range(world):
         _, st, _, s1, s2, s3, q, sc, log = res[r]
@@ -471,7 +484,7 @@ def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
                                          ("handshake_addresses__host_phase_order", 3),
                                          ("cached_addresses__device_phase_order", 0)):
             got = leg["decode"][variant]
-            assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
+            assert got["verified"]["window_equals_single_gpu_path"] and got["verified"]["Y_equals_X"]
             assert got["handshakes_in_timed_steps"] == want_handshakes
             assert got["step_us"] > 0 and got["dispatch_phase_us"] > 0 and got["combine_phase_us"] > 0
 
@@ -513,8 +526,10 @@ def test_benchmark_expert_parallel_leg_over_nccl_with_one_rank():
     for variant in ("cached_addresses__host_phase_order", "handshake_addresses__host_phase_order",
                     "cached_addresses__device_phase_order"):
         got = leg["decode"][variant]
-        assert got["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
+        assert got["verified"]["window_equals_single_gpu_path"] and got["verified"]["Y_equals_X"]
         assert got["step_us"] > 0
+    first = leg["decode"]["cached_addresses__host_phase_order"]
+    assert first["verified"]["quantised_codes_and_scales_equal_single_gpu_path"] and first["quantised_dispatch_phase_us"] > 0
 
 
 def test_expert_parallel_child_mode_of_the_benchmark_two_ranks_on_one_gpu():
@@ -538,5 +553,6 @@ def test_expert_parallel_child_mode_of_the_benchmark_two_ranks_on_one_gpu():
     assert leg["ranks"] == 2 and leg["ranks_share_a_gpu"] is True
     for variant in ("cached_addresses__host_phase_order", "handshake_addresses__host_phase_order",
                     "cached_addresses__device_phase_order"):
-        assert leg["decode"][variant]["verified"] == {"window_equals_single_gpu_path": True, "Y_equals_X": True}
+        assert leg["decode"][variant]["verified"]["window_equals_single_gpu_path"]
+        assert leg["decode"][variant]["verified"]["Y_equals_X"]
     assert not [ln for ln in outs[1][0].splitlines() if ln.startswith("{")]       # only rank 0 prints
