@@ -560,7 +560,7 @@ def ep_shape(key: str, R: int):
 
 
 def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
-           variants=(("cached", "host"), ("handshake", "host"), ("cached", "device"))) -> dict:
+           variants=(("cached", "host"), ("handshake", "host"), ("cached", "device"), ("static", "device"))) -> dict:
     """The path with rank = process = GPU: every process plans its own tokens, the count rows (and window
     generations) are all-gathered over the process group, every rank's window is mapped into every process
     (moe_window_export / moe_peers_open), dispatch stores rows into the other GPUs' windows and combine loads
@@ -568,7 +568,9 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
     its window against the single-GPU path run on the whole batch with R virtual ranks (the path the parity
     tests compare with the CPU definition) and its output against the identity Y == X.
     Variants: (address mode, phase order).  Address mode "cached" exchanges window addresses only when a rank's
-    window generation changes, "handshake" before every dispatch.  Phase order "host" separates the phases by a
+    window generation changes (the generations are read on the host every step), "handshake" before every dispatch,
+    "static" once (no validity test; with the device phase order a step has no host synchronisation beyond the count
+    exchange itself).  Phase order "host" separates the phases by a
     stream synchronisation and a process-group barrier, "device" by arrival flags in the windows' state regions
     (moe_signal_peers / moe_wait_peers) with no host synchronisation between the phases -- unless ranks share a
     GPU, where a host barrier is placed between signal and wait (a wait kernel must not hold a GPU that the

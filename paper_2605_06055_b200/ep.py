@@ -75,13 +75,18 @@ def addresses_stale(table_generations, announced_generations) -> bool:
 
 
 class EpRank:
-    """The calls of one rank, in the order the schedules prescribe.  mode: "cached" or "handshake"."""
+    """The calls of one rank, in the order the schedules prescribe.
+    mode: "handshake" exchanges the window addresses before every dispatch; "cached" tests every step whether the
+    cached table is still valid (the generations that came with the count rows are read on the host: one stream
+    synchronisation per step) and exchanges them only when it is not; "static" exchanges them once and takes the
+    caller's word that no window moves afterwards -- with sync="device" a step then contains no host
+    synchronisation at all (call handshake() yourself, on every rank, after attaching a different window)."""
 
     SLOT_DISPATCHED, SLOT_EXPERTS_DONE, SLOT_COMBINED = 0, 1, 2
 
     def __init__(self, T_local_max: int, H: int, E: int, K: int, device, group=None, mode: str = "cached",
                  sync: str = "host", host_fence: bool = False):
-        assert mode in ("cached", "handshake") and sync in ("host", "device")
+        assert mode in ("cached", "handshake", "static") and sync in ("host", "device")
         self.group, self.mode, self.device = group, mode, device
         self.sync, self.host_fence, self.epoch = sync, host_fence, 0
         self.rank = dist.get_rank(group)
@@ -163,7 +168,10 @@ class EpRank:
     def _ensure_addresses(self) -> None:
         # every rank holds the same table generations (handshakes are collective) and the same announcement,
         # so every rank takes the same branch
-        if self.mode == "handshake" or addresses_stale(self.table_generations, self.announced):
+        if self.mode == "static":
+            if self.table_generations is None:
+                self.handshake()
+        elif self.mode == "handshake" or addresses_stale(self.table_generations, self.announced):
             self.handshake()
 
     # -- the phases ------------------------------------------------------------------------------------
@@ -171,7 +179,8 @@ class EpRank:
         self.comm.moe_layout(schedule, topk_idx_local, self.rank, self.counts_row)
         gathered = all_gather_rows(self.message, self.group)             # metadata only, no payload
         counts_all = gathered[:, :self.E].contiguous()
-        self.announced = gathered[:, self.E].cpu().numpy().astype(np.int32)
+        # "static": nothing is read back, so nothing waits for the stream; the calls run without a validity test
+        self.announced = None if self.mode == "static" else gathered[:, self.E].cpu().numpy().astype(np.int32)
         self.comm.moe_notify(counts_all)
         return counts_all
 

@@ -346,19 +346,19 @@ def _ipc_rank(rank, world, port, mode, sync, results):
         log["handshakes_after_step_2"] = me.handshakes
         win_2, y_2 = u16(mine), u16(y)
         # a stale stamp is refused and nothing is enqueued: rows stay as they are
-        wrong = me.announced.copy()
+        wrong = (me.announced if me.announced is not None else me.table_generations).copy()
         wrong[1 - rank] += 5
         before = u16(mine)
         log["refused_stale"] = me.comm.moe_dispatch_cached(x, wrong, check=False)
         log["refused_stale_combine"] = me.comm.moe_combine_cached(wrong, w, y, check=False)
-        log["check_fresh"] = me.comm.moe_peers_check(me.announced)
+        log["check_fresh"] = me.comm.moe_peers_check(me.announced if me.announced is not None else me.table_generations)
         log["check_stale"] = me.comm.moe_peers_check(wrong)
         torch.cuda.synchronize()
         dist.barrier()
         log["untouched_after_refusal"] = bool(np.array_equal(u16(mine), before))
         # rank 1 moves its window to a new allocation: every rank's table is stale at the next plan
         dist.barrier()
-        if rank == 1:
+        if rank == 1 and mode != "static":             # ("static": the caller promises that no window moves)
             keep_old = backing                         # stays mapped on the other rank until its next handshake
             backing, mine = new_window(8)              # the new window starts 8 rows into its allocation
         else:
@@ -385,14 +385,15 @@ def _ipc_rank(rank, world, port, mode, sync, results):
         results[rank] = ("error", repr(exc) + "\n" + traceback.format_exc())
 
 
-@pytest.mark.parametrize("mode,sync", [("cached", "host"), ("handshake", "host"), ("cached", "device")])
+@pytest.mark.parametrize("mode,sync", [("cached", "host"), ("handshake", "host"), ("cached", "device"),
+                                       ("static", "device")])
 def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     world = 2
     with ctx.Manager() as m:
         results = m.dict()
-        port = 35000 + (os.getpid() * 4 + 2 * (mode == "cached") + (sync == "device")) % 2000
+        port = 35000 + (os.getpid() * 8 + 4 * (mode == "static") + 2 * (mode == "cached") + (sync == "device")) % 2000
         procs = [ctx.Process(target=_ipc_rank, args=(r, world, port, mode, sync, results)) for r in range(world)]
         for p_ in procs:
             p_.start()
@@ -432,6 +433,8 @@ def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
         assert log["untouched_after_refusal"]
         if mode == "cached":      # one handshake for the first step, none for the second, one after the move
             assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 1, 2)
+        elif mode == "static":    # exchanged once
+            assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 1, 1)
         else:                     # the handshake mode exchanges addresses before every dispatch
             assert (log["handshakes_after_step_1"], log["handshakes_after_step_2"], log["handshakes_after_step_3"]) == (1, 2, 3)
 
@@ -482,7 +485,8 @@ def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
         assert leg["ranks_share_a_gpu"] is True
         for variant, want_handshakes in (("cached_addresses__host_phase_order", 0),
                                          ("handshake_addresses__host_phase_order", 3),
-                                         ("cached_addresses__device_phase_order", 0)):
+                                         ("cached_addresses__device_phase_order", 0),
+                                         ("static_addresses__device_phase_order", 0)):
             got = leg["decode"][variant]
             assert got["verified"]["window_equals_single_gpu_path"] and got["verified"]["Y_equals_X"]
             assert got["handshakes_in_timed_steps"] == want_handshakes
@@ -524,7 +528,7 @@ def test_benchmark_expert_parallel_leg_over_nccl_with_one_rank():
     leg = res[0][1]
     assert leg["ranks"] == 1 and leg["ranks_share_a_gpu"] is False
     for variant in ("cached_addresses__host_phase_order", "handshake_addresses__host_phase_order",
-                    "cached_addresses__device_phase_order"):
+                    "cached_addresses__device_phase_order", "static_addresses__device_phase_order"):
         got = leg["decode"][variant]
         assert got["verified"]["window_equals_single_gpu_path"] and got["verified"]["Y_equals_X"]
         assert got["step_us"] > 0
