@@ -547,6 +547,36 @@ def test_gate_topk_ties_take_the_lower_index_first():
     assert oracle.gate_topk(logits, 7)[0] == oracle.ERR_INVALID_ARG   # K > E
 
 
+@pytest.mark.parametrize("K", [2, 8, 28, 32])
+def test_gate_weights_within_the_fp32_budget_of_the_exact_softmax(K):
+    """One side's share of the gate-weight tolerance the GPU tests use, (2K + 8) * 2^-24 between the two sides:
+    against the softmax of the same fp32 differences l_j - l_0 evaluated in fp64, the oracle's fp32 weights are off by
+    at most (K + 2) half-ulps -- the
+    exponentials (<= 1 ulp each), the K - 1 roundings of the ascending sum, the division.  The adversarial case is
+    many EQUAL selected logits: every addition of the sum then rounds the same way (a random case stays near
+    sqrt(K) half-ulps), which is why the budget is linear in K."""
+    E, T = 48, 4000
+    rng = np.random.default_rng(K)
+    worst = 0.0
+    for equal_share in (0.0, 0.7):
+        logits = (rng.standard_normal((T, E)) * 3).astype(np.float32)
+        n_eq = int(E * equal_share)
+        if n_eq:
+            logits[:, :n_eq] = (rng.standard_normal((T, 1)) * 2).astype(np.float32)    # one value, repeated
+        st, idx, w = oracle.gate_topk(logits, K)
+        assert st == oracle.OK
+        sel = np.take_along_axis(logits, idx.astype(np.int64), axis=1)
+        # the fp32 differences l_j - l_0 are part of the definition (both sides form the same ones); everything
+        # after them is evaluated exactly here
+        ex = np.exp((sel - sel[:, :1]).astype(np.float32).astype(np.float64))
+        exact = ex / ex.sum(1, keepdims=True)
+        rel = np.abs(w.astype(np.float64) - exact) / exact
+        assert rel.max() <= (K + 2) * 2.0 ** -24, (K, equal_share, rel.max())
+        worst = max(worst, rel.max())
+    if K >= 28:          # the linear term is really there: the equal-logit case gets well past a sqrt(K) budget
+        assert worst > 2.5 * np.sqrt(K) * 2.0 ** -25, worst
+
+
 # ----------------------------------------------------------------------------- multi-rank decomposition
 def test_layout_per_rank_plus_notify_equals_the_global_plan():
     """Layout is local (Section 5.2): planning each rank's tokens alone gives that rank's row of M and
