@@ -387,59 +387,59 @@ gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t
       }
     };
     if (VPT >= 4 && K <= 16 && in_pairs) {   // (never taken for the short-row forms)
-      // Tokens in pairs (2p, 2p+1), two pairs of row buffers used in turn: the next pair's rows travel while the
-      // current pair is selected.  A last odd token, and pairs with too many candidates, go one by one.
+      // Tokens in pairs (2p, 2p+1): the next pair's rows travel while the current pair is selected.  Pairs with
+      // too many candidates go one by one; a last odd token is left to the loop below.
       float* pair_sm = gate_cand[warp];
-      const int32_t pairs = T >> 1, pstride = stride;
+      const int32_t pairs = T >> 1;
       int32_t p = blockIdx.x * wpc + warp;
       auto load_pair = [&](int32_t pp, float (&ra)[VPT], float (&rb)[VPT]) {
         warp_gate_load<VPT>(logits + (size_t)(2 * pp) * E, E, lane, vec, ra);
         warp_gate_load<VPT>(logits + (size_t)(2 * pp + 1) * E, E, lane, vec, rb);
       };
-      auto process_pair = [&](const float (&ra)[VPT], const float (&rb)[VPT], int32_t pp) {
+      float a[VPT], b[VPT], na[VPT], nb[VPT];
+      if (p < pairs) load_pair(p, a, b);
+      for (; p < pairs; p += stride) {
+        const bool more = p + stride < pairs;
+        if (more) load_pair(p + stride, na, nb);
         int32_t idx;
         float w;
-        if (warp_gate_rank_pair<VPT>(ra, rb, K, lane, pair_sm, idx, w)) {
+        if (warp_gate_rank_pair<VPT>(a, b, K, lane, pair_sm, idx, w)) {
           w = halfwarp_gate_softmax(w, K, lane);
           const int l = lane & 15;
-          const size_t tok = (size_t)(2 * pp + (lane >> 4));
+          const size_t tok = (size_t)(2 * p + (lane >> 4));
           if (l < K) {
             topk_idx[tok * K + l] = idx;
             topk_w[tok * K + l] = w;
           }
         } else {
-          process(ra, 2 * pp);
-          process(rb, 2 * pp + 1);
+          for (int h = 0; h < 2; ++h) {   // one instance of the single-token code for both
+            float one[VPT];
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) one[i] = h ? b[i] : a[i];
+            process(one, 2 * p + h);
+          }
         }
-      };
-      float a0[VPT], b0[VPT], a1[VPT], b1[VPT];
-      if (p < pairs) load_pair(p, a0, b0);
-      while (p < pairs) {
-        if (p + pstride < pairs) load_pair(p + pstride, a1, b1);
-        process_pair(a0, b0, p);
-        p += pstride;
-        if (p >= pairs) break;
-        if (p + pstride < pairs) load_pair(p + pstride, a0, b0);
-        process_pair(a1, b1, p);
-        p += pstride;
+        if (more) {
+#pragma unroll
+          for (int i = 0; i < VPT; ++i) {
+            a[i] = na[i];
+            b[i] = nb[i];
+          }
+        }
       }
-      if ((T & 1) && blockIdx.x == 0 && warp == 0) {
-        warp_gate_load<VPT>(logits + (size_t)(T - 1) * E, E, lane, vec, a0);
-        process(a0, T - 1);
-      }
-      return;
+      t = ((T & 1) && blockIdx.x == 0 && warp == 0) ? T - 1 : T;   // the odd token, by the loop below
     }
-    // one token at a time, two row buffers used in turn: the next token's row travels while the current one is selected
-    float row_a[VPT], row_b[VPT];
-    if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row_a);
-    while (t < T) {
-      if (t + stride < T) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, row_b);
-      process(row_a, t);
-      t += stride;
-      if (t >= T) break;
-      if (t + stride < T) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, row_a);
-      process(row_b, t);
-      t += stride;
+    // one token at a time: the next token's row travels while the current one is selected
+    float row[VPT], next_row[VPT];
+    if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row);
+    for (; t < T; t += stride) {
+      const bool more = t + stride < T;
+      if (more) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, next_row);
+      process(row, t);
+      if (more) {
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) row[i] = next_row[i];
+      }
     }
   } else {
     for (; t < T; t += stride) {
