@@ -357,14 +357,35 @@ __device__ __forceinline__ void warp_gate_load(const float* __restrict__ row, in
   for (int i = 0; i < VPT; ++i) v[i] = base + i < E ? __ldg(row + base + i) : -INFINITY;
 }
 
-// Stand-alone gate: grid-stride over tokens, one warp per token, the next token's row loaded while the current
-// one is selected.  VPT > 0: register form for rows of at most 32 * VPT logits (one instantiation per row
-// length class, so that short rows keep few registers and many warps per SM).  VPT == 0: shared-memory form for longer rows; dynamic shared
-// memory: warps * E floats.
+// One token, start to finish: threshold-and-rank selection (long rows), the rounds when that gives up or for short
+// rows, softmax, stores.  sm: GATE_RANK_WORDS words of this warp.
 template <int VPT>
+__device__ __forceinline__ void warp_gate_one(const float (&v)[VPT], int32_t tok, int K, int lane, float* sm,
+                                              int32_t* __restrict__ topk_idx, float* __restrict__ topk_w) {
+  int32_t idx;
+  float w;
+  // rows of one or two logits per lane: the rounds are already cheap (nothing to scan inside a lane)
+  bool done = false;
+  if constexpr (VPT >= 4) done = warp_gate_rank<VPT>(v, K, lane, sm, idx, w);
+  if (!done) warp_gate_select<VPT>(v, K, lane, idx, w);
+  w = warp_gate_softmax(w, K, lane);
+  if (lane < K) {
+    topk_idx[(size_t)tok * K + lane] = idx;
+    topk_w[(size_t)tok * K + lane] = w;
+  }
+}
+
+// Stand-alone gate: grid-stride over tokens, the next rows loaded while the current ones are selected (two sets of
+// row buffers used in turn).  VPT > 0: register form for rows of at most 32 * VPT logits (one instantiation per
+// row length class, so that short rows keep few registers and many warps per SM).  PAIRS: two tokens per warp
+// (tokens 2p and 2p+1; needs VPT >= 4 and K <= 16), else one.  VPT == 0: shared-memory form for longer rows;
+// dynamic shared memory: warps * E floats.
+// Every selection form appears at most twice in a kernel: with more inlined copies the code outgrew the
+// instruction caches and a call chained behind others started 2 us later.
+template <int VPT, bool PAIRS>
 __global__ void __launch_bounds__(256, VPT == 8 ? 4 : 1)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
-                 float* __restrict__ topk_w, int32_t in_pairs /* launcher: enough tokens for two per warp */) {
+                 float* __restrict__ topk_w) {
   extern __shared__ float gate_rows[];
   __shared__ __align__(16) float gate_cand[8][GATE_PAIR_WORDS];   // warp_gate_rank(_pair)'s buffers, one set per warp
   release_dependents();   // a planner launched behind the gate (moe_gate_plan) may be scheduled; it waits for this kernel
@@ -374,71 +395,59 @@ gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t
   if constexpr (VPT > 0) {
     const bool vec = (E % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0);
     auto process = [&](const float (&v)[VPT], int32_t tok) {
-      int32_t idx;
-      float w;
-      // rows of one or two logits per lane: the rounds are already cheap (nothing to scan inside a lane)
-      bool done = false;
-      if constexpr (VPT >= 4) done = warp_gate_rank<VPT>(v, K, lane, gate_cand[warp], idx, w);
-      if (!done) warp_gate_select<VPT>(v, K, lane, idx, w);
-      w = warp_gate_softmax(w, K, lane);
-      if (lane < K) {
-        topk_idx[(size_t)tok * K + lane] = idx;
-        topk_w[(size_t)tok * K + lane] = w;
-      }
+      warp_gate_one<VPT>(v, tok, K, lane, gate_cand[warp], topk_idx, topk_w);
     };
-    if (VPT >= 4 && K <= 16 && in_pairs) {   // (never taken for the short-row forms)
-      // Tokens in pairs (2p, 2p+1): the next pair's rows travel while the current pair is selected.  Pairs with
-      // too many candidates go one by one; a last odd token is left to the loop below.
-      float* pair_sm = gate_cand[warp];
-      const int32_t pairs = T >> 1;
-      int32_t p = blockIdx.x * wpc + warp;
+    if constexpr (PAIRS) {
+      // t counts pairs here.  An odd T ends in a pair whose second token does not exist: its row is read from
+      // the last token again and nothing is stored for it.
+      const int32_t pairs = (T + 1) >> 1;
       auto load_pair = [&](int32_t pp, float (&ra)[VPT], float (&rb)[VPT]) {
+        const int32_t second = min(2 * pp + 1, T - 1);
         warp_gate_load<VPT>(logits + (size_t)(2 * pp) * E, E, lane, vec, ra);
-        warp_gate_load<VPT>(logits + (size_t)(2 * pp + 1) * E, E, lane, vec, rb);
+        warp_gate_load<VPT>(logits + (size_t)second * E, E, lane, vec, rb);
       };
-      float a[VPT], b[VPT], na[VPT], nb[VPT];
-      if (p < pairs) load_pair(p, a, b);
-      for (; p < pairs; p += stride) {
-        const bool more = p + stride < pairs;
-        if (more) load_pair(p + stride, na, nb);
+      auto process_pair = [&](const float (&ra)[VPT], const float (&rb)[VPT], int32_t pp) {
         int32_t idx;
         float w;
-        if (warp_gate_rank_pair<VPT>(a, b, K, lane, pair_sm, idx, w)) {
+        if (warp_gate_rank_pair<VPT>(ra, rb, K, lane, gate_cand[warp], idx, w)) {
           w = halfwarp_gate_softmax(w, K, lane);
           const int l = lane & 15;
-          const size_t tok = (size_t)(2 * p + (lane >> 4));
-          if (l < K) {
-            topk_idx[tok * K + l] = idx;
-            topk_w[tok * K + l] = w;
+          const int32_t tok = 2 * pp + (lane >> 4);
+          if (l < K && tok < T) {
+            topk_idx[(size_t)tok * K + l] = idx;
+            topk_w[(size_t)tok * K + l] = w;
           }
-        } else {
-          for (int h = 0; h < 2; ++h) {   // one instance of the single-token code for both
+        } else {   // too many candidates for a half-warp: one by one (a single copy of that code for both)
+          for (int h = 0; h < 2 && 2 * pp + h < T; ++h) {
             float one[VPT];
 #pragma unroll
-            for (int i = 0; i < VPT; ++i) one[i] = h ? b[i] : a[i];
-            process(one, 2 * p + h);
+            for (int i = 0; i < VPT; ++i) one[i] = h ? rb[i] : ra[i];
+            process(one, 2 * pp + h);
           }
         }
-        if (more) {
-#pragma unroll
-          for (int i = 0; i < VPT; ++i) {
-            a[i] = na[i];
-            b[i] = nb[i];
-          }
-        }
+      };
+      float a0[VPT], b0[VPT], a1[VPT], b1[VPT];
+      if (t < pairs) load_pair(t, a0, b0);
+      while (t < pairs) {
+        if (t + stride < pairs) load_pair(t + stride, a1, b1);
+        process_pair(a0, b0, t);
+        t += stride;
+        if (t >= pairs) break;
+        if (t + stride < pairs) load_pair(t + stride, a0, b0);
+        process_pair(a1, b1, t);
+        t += stride;
       }
-      t = ((T & 1) && blockIdx.x == 0 && warp == 0) ? T - 1 : T;   // the odd token, by the loop below
-    }
-    // one token at a time: the next token's row travels while the current one is selected
-    float row[VPT], next_row[VPT];
-    if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row);
-    for (; t < T; t += stride) {
-      const bool more = t + stride < T;
-      if (more) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, next_row);
-      process(row, t);
-      if (more) {
-#pragma unroll
-        for (int i = 0; i < VPT; ++i) row[i] = next_row[i];
+    } else {
+      float row_a[VPT], row_b[VPT];
+      if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row_a);
+      while (t < T) {
+        if (t + stride < T) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, row_b);
+        process(row_a, t);
+        t += stride;
+        if (t >= T) break;
+        if (t + stride < T) warp_gate_load<VPT>(logits + (size_t)(t + stride) * E, E, lane, vec, row_a);
+        process(row_b, t);
+        t += stride;
       }
     }
   } else {

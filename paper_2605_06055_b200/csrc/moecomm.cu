@@ -422,7 +422,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
        opt_in(dispatch_quant_kernel<2, 32, false>) && opt_in(dispatch_quant_kernel<3, 32, false>) &&
        opt_in(dispatch_quant_kernel<2, 0, false>) && opt_in(dispatch_quant_kernel<3, 0, false>) && opt_in(plan_rank_kernel<32>) &&
        opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
-       opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0>);
+       opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0, false>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
   const int rank_smem =
       rank_plan_smem_ints(shape->E, shape->R, shape->E <= RANK_PLAN_WIDE_MAX_E ? 32 : 8) * (int)sizeof(int32_t);
@@ -497,9 +497,9 @@ namespace {
 
 constexpr int GATE_OCC_MAX_DEVICES = 64;
 
-template <int VPT>
-void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
-                      int dev, cudaStream_t st) {
+template <int VPT, bool PAIRS>
+void launch_gate_kernel(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
+                        int dev, cudaStream_t st) {
   int warps = 8, smem = 0;
   if (VPT == 0) {   // rows cached in shared memory
     while (warps > 1 && warps * E * (int)sizeof(float) > 96 * 1024) warps >>= 1;
@@ -511,22 +511,34 @@ void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int3
   static std::atomic<int> cached[GATE_OCC_MAX_DEVICES];
   int per_sm = (VPT > 0 && dev >= 0 && dev < GATE_OCC_MAX_DEVICES) ? cached[dev].load(std::memory_order_relaxed) : 0;
   if (per_sm == 0) {
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gate_topk_kernel<VPT>, warps * 32, smem) != cudaSuccess ||
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gate_topk_kernel<VPT, PAIRS>, warps * 32, smem) !=
+            cudaSuccess ||
         per_sm < 1) {
       cudaGetLastError();
       per_sm = 1;
     }
     if (VPT > 0 && dev >= 0 && dev < GATE_OCC_MAX_DEVICES) cached[dev].store(per_sm, std::memory_order_relaxed);
   }
-  // Two tokens per warp (they share the rank / softmax / store instructions) once that still leaves every SM a
-  // full CTA of pairs; small batches keep one token per warp and so more warps.  3.0 against 2.7 us at T=2048,
-  // 4.7 against 5.1 us at T=8192, 12.3 against 14.3 us at T=32768 (256 logits, top-8).
-  const int32_t in_pairs = (VPT >= 4 && K <= 16 && (int64_t)T / 2 >= (int64_t)num_sms * warps) ? 1 : 0;
-  const int64_t units = in_pairs ? ((int64_t)T + 1) / 2 : (int64_t)T;
+  const int64_t units = PAIRS ? ((int64_t)T + 1) / 2 : (int64_t)T;
   int64_t grid = (units + warps - 1) / warps;
   if (grid > (int64_t)num_sms * per_sm) grid = (int64_t)num_sms * per_sm;   // one resident wave, grid-stride over tokens
   if (grid < 1) grid = 1;
-  gate_topk_kernel<VPT><<<(int)grid, warps * 32, smem, st>>>(logits, T, E, K, idx, w, in_pairs);
+  gate_topk_kernel<VPT, PAIRS><<<(int)grid, warps * 32, smem, st>>>(logits, T, E, K, idx, w);
+}
+
+template <int VPT>
+void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
+                      int dev, cudaStream_t st) {
+  // Two tokens per warp (they share the rank / softmax / store instructions) once that still leaves every SM a
+  // full CTA of pairs; small batches keep one token per warp and so more warps.  3.0 against 2.7 us at T=2048,
+  // 4.7 against 5.1 us at T=8192, 12.3 against 14.3 us at T=32768 (256 logits, top-8).
+  if constexpr (VPT >= 4) {
+    if (K <= 16 && (int64_t)T / 2 >= (int64_t)num_sms * 8) {
+      launch_gate_kernel<VPT, true>(logits, T, E, K, idx, w, num_sms, dev, st);
+      return;
+    }
+  }
+  launch_gate_kernel<VPT, false>(logits, T, E, K, idx, w, num_sms, dev, st);
 }
 
 void launch_gate(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* idx, float* w, int num_sms,
@@ -679,7 +691,7 @@ moe_status_t moe_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K,
   if (E > 1024) {   // the shared-memory form of the gate: opt in like moe_create does
     int optin = 0;
     if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
-        cudaFuncSetAttribute(gate_topk_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 2048) != cudaSuccess)
+        cudaFuncSetAttribute(gate_topk_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 2048) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
   if (T > 0) launch_gate(logits, T, E, K, topk_idx, topk_w, sms, dev, static_cast<cudaStream_t>(stream));

@@ -55,12 +55,15 @@ def test_gate_topk_kernel(T, E, K, ties):
         l[:, ::7] = -1.0
     st, want_idx, want_w = oracle.gate_topk(l.numpy(), K)
     assert st == oracle.OK
-    idx = torch.full((T, K), -1, dtype=torch.int32, device=dev)
-    w = torch.full((T, K), -1.0, dtype=torch.float32, device=dev)
+    # two guard rows behind the outputs: an odd token count must not be rounded up to a pair
+    idx_all = torch.full((T + 2, K), -1, dtype=torch.int32, device=dev)
+    w_all = torch.full((T + 2, K), -1.0, dtype=torch.float32, device=dev)
+    idx, w = idx_all[:T], w_all[:T]
     assert binding.moe_gate_topk(l.to(dev), K, idx, w) == binding.MOE_OK
     torch.cuda.synchronize()
     assert np.array_equal(idx.cpu().numpy(), want_idx)
     assert np.allclose(w.cpu().numpy(), want_w, rtol=gate_rtol(K), atol=1e-12)
+    assert bool((idx_all[T:] == -1).all()) and bool((w_all[T:] == -1.0).all())
 
 
 @pytest.mark.parametrize("case", [
