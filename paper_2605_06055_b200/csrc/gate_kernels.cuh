@@ -138,15 +138,14 @@ __device__ __forceinline__ void warp_gate_select(const float (&v)[VPT], int K, i
 // one (equal logits: lower expert index first), counted directly.  More than 32 candidates (many equal logits, K
 // close to 32): the caller falls back to warp_gate_select.
 // On success lane j < K holds the j-th selected logit (in w_lane) and its expert.
-constexpr int GATE_RANK_WORDS = 132;
+constexpr int GATE_RANK_WORDS = 136;
 
 template <int VPT>
 __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int lane, float* sm, int32_t& idx_lane,
                                                float& w_lane) {
-  float* cand_val = sm;                                          // [36]: up to 32 candidates + padding of the last group of four
-  int32_t* cand_idx = reinterpret_cast<int32_t*>(sm + 36);       // [32]
-  float* out_val = sm + 68;                                      // [32]
-  int32_t* out_idx = reinterpret_cast<int32_t*>(sm + 100);       // [32]
+  float2* cand = reinterpret_cast<float2*>(sm);                  // [36] (value, expert): 32 candidates + padding of the last four
+  float* out_val = sm + 72;                                      // [32]
+  int32_t* out_idx = reinterpret_cast<int32_t*>(sm + 104);       // [32]
   const int base = lane * VPT;
   float m = v[0];
 #pragma unroll
@@ -177,28 +176,31 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
   }
   const int C = __shfl_sync(0xffffffffu, incl, 31);
   if (C > 32) return false;
-  if (lane < 3) cand_val[C + lane] = -INFINITY;   // the counting loop reads four candidates at a time
-  // predicated stores, no branches: slot address advances by one word per candidate
-  uint32_t slot = (uint32_t)__cvta_generic_to_shared(cand_val) + 4u * (uint32_t)(incl - c);
+  if (lane < 3) cand[C + lane].x = -INFINITY;   // the counting loop reads four candidates at a time
+  // predicated stores and address steps, no branches: one 8-byte (value, expert) store per candidate
+  uint32_t slot = (uint32_t)__cvta_generic_to_shared(cand) + 8u * (uint32_t)(incl - c);
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
-    uint32_t step;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ge.f32 p, %1, %2;\n\t"
-        "@p st.shared.f32 [%3], %1;\n\t"
-        "@p st.shared.u32 [%3+144], %4;\n\t"     // cand_idx = cand_val + 36 words
-        "selp.u32 %0, 4, 0, p;\n\t}"
-        : "=r"(step) : "f"(v[i]), "f"(theta), "r"(slot), "r"(base + i) : "memory");
-    slot += step;
+        "@p st.shared.v2.b32 [%0], {%3, %4};\n\t"
+        "@p add.u32 %0, %0, 8;\n\t}"
+        : "+r"(slot) : "f"(v[i]), "f"(theta), "r"(__float_as_uint(v[i])), "r"(base + i) : "memory");
   }
   __syncwarp();
-  const float x = lane < C ? cand_val[lane] + 0.0f : -INFINITY;   // -0 becomes +0: equal logits get equal bit patterns
-  const int32_t xi = lane < C ? cand_idx[lane] : -1;
+  float x = -INFINITY;
+  int32_t xi = -1;
+  if (lane < C) {
+    const float2 me = cand[lane];
+    x = me.x + 0.0f;   // -0 becomes +0: equal logits get equal bit patterns
+    xi = __float_as_int(me.y);
+  }
   int rank = __popc(__match_any_sync(0xffffffffu, __float_as_uint(x)) & lanemask_lt());   // earlier equal candidates
   for (int q = 0; q < C; q += 4) {
-    const float4 a = *reinterpret_cast<const float4*>(cand_val + q);   // broadcast read
-    rank += (a.x > x ? 1 : 0) + (a.y > x ? 1 : 0) + (a.z > x ? 1 : 0) + (a.w > x ? 1 : 0);
+    const float4 c01 = *reinterpret_cast<const float4*>(cand + q);   // broadcast reads
+    const float4 c23 = *reinterpret_cast<const float4*>(cand + q + 2);
+    rank += (c01.x > x ? 1 : 0) + (c01.z > x ? 1 : 0) + (c23.x > x ? 1 : 0) + (c23.z > x ? 1 : 0);
   }
   if (lane < C && rank < K) {
     out_val[rank] = x;
@@ -218,13 +220,13 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
 // lanes 16-31 rank token B's, and the caller's epilogue works on half-warps.  Needs K <= 16; fails (nothing
 // written that matters) if a token has more than 16 candidates -- the caller then takes the tokens one by one.
 // On success lane j < K of half h holds the j-th selected logit and expert of token h.
-// sm: GATE_PAIR_WORDS words: candidate values [2][20], candidate experts [2][20], selected values [2][16], experts [2][16].
+// sm: GATE_PAIR_WORDS words: candidates [2][20] as (value, expert) pairs, selected values [2][16], experts [2][16].
 constexpr int GATE_PAIR_WORDS = 144;
 
 template <int VPT>
 __device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], const float (&vb)[VPT], int K, int lane,
                                                     float* sm, int32_t& idx_lane, float& w_lane) {
-  float* cand_val = sm;                                          // [2][20]: 16 candidates + padding of the last four
+  float2* cand = reinterpret_cast<float2*>(sm);                  // [2][20]: 16 candidates + padding of the last four
   float* out_val = sm + 80;                                      // [2][16]
   int32_t* out_idx = reinterpret_cast<int32_t*>(sm + 112);       // [2][16]
   const int base = lane * VPT;
@@ -249,9 +251,13 @@ __device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], cons
   }
   ta = fmaxf(ta, -3.402823466e+38f);   // absent entries (-inf) never qualify
   tb = fmaxf(tb, -3.402823466e+38f);
-  int c = 0;   // candidates of this lane: token A in the low half of the word, token B in the high half
+  int na = 0, nb = 0;   // minus this lane's candidate counts
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) c += ((va[i] >= ta) ? 1 : 0) + ((vb[i] >= tb) ? 0x10000 : 0);
+  for (int i = 0; i < VPT; ++i) {
+    na += (va[i] >= ta) ? -1 : 0;
+    nb += (vb[i] >= tb) ? -1 : 0;
+  }
+  const int c = -(na + (nb << 16));   // token A's count in the low half of the word, token B's in the high half
   int incl = c;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
@@ -263,37 +269,40 @@ __device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], cons
   if (Ca > 16 || Cb > 16) return false;
   const int half = lane >> 4, l = lane & 15;
   const int Ch = half ? Cb : Ca;
-  if (l < 3) cand_val[half * 20 + Ch + l] = -INFINITY;   // the counting loop reads four candidates at a time
+  if (l < 3) cand[half * 20 + Ch + l].x = -INFINITY;   // the counting loop reads four candidates at a time
   const int excl = incl - c;
-  const uint32_t sm_addr = (uint32_t)__cvta_generic_to_shared(cand_val);
-  uint32_t slot_a = sm_addr + 4u * (uint32_t)(excl & 0xffff), slot_b = sm_addr + 80u + 4u * (uint32_t)(excl >> 16);
+  const uint32_t sm_addr = (uint32_t)__cvta_generic_to_shared(cand);
+  uint32_t slot_a = sm_addr + 8u * (uint32_t)(excl & 0xffff), slot_b = sm_addr + 160u + 8u * (uint32_t)(excl >> 16);
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) {   // predicated stores, no branches (see warp_gate_rank); experts 40 words behind the values
-    uint32_t step_a, step_b;
+  for (int i = 0; i < VPT; ++i) {   // predicated stores and address steps, no branches
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ge.f32 p, %2, %3;\n\t"
         "setp.ge.f32 q, %6, %7;\n\t"
-        "@p st.shared.f32 [%4], %2;\n\t"
-        "@p st.shared.u32 [%4+160], %5;\n\t"
-        "@q st.shared.f32 [%8], %6;\n\t"
-        "@q st.shared.u32 [%8+160], %5;\n\t"
-        "selp.u32 %0, 4, 0, p;\n\t"
-        "selp.u32 %1, 4, 0, q;\n\t}"
-        : "=r"(step_a), "=r"(step_b)
-        : "f"(va[i]), "f"(ta), "r"(slot_a), "r"(base + i), "f"(vb[i]), "f"(tb), "r"(slot_b) : "memory");
-    slot_a += step_a;
-    slot_b += step_b;
+        "@p st.shared.v2.b32 [%0], {%4, %5};\n\t"
+        "@q st.shared.v2.b32 [%1], {%8, %5};\n\t"
+        "@p add.u32 %0, %0, 8;\n\t"
+        "@q add.u32 %1, %1, 8;\n\t}"
+        : "+r"(slot_a), "+r"(slot_b)
+        : "f"(va[i]), "f"(ta), "r"(__float_as_uint(va[i])), "r"(base + i), "f"(vb[i]), "f"(tb),
+          "r"(__float_as_uint(vb[i]))
+        : "memory");
   }
   __syncwarp();
-  const float* mine = cand_val + half * 20;
-  const float x = l < Ch ? mine[l] + 0.0f : -INFINITY;   // -0 becomes +0: equal logits get equal bit patterns
-  const int32_t xi = l < Ch ? reinterpret_cast<const int32_t*>(mine)[40 + l] : -1;
+  const float2* mine = cand + half * 20;
+  float x = -INFINITY;
+  int32_t xi = -1;
+  if (l < Ch) {
+    const float2 me = mine[l];
+    x = me.x + 0.0f;   // -0 becomes +0: equal logits get equal bit patterns
+    xi = __float_as_int(me.y);
+  }
   const unsigned same_half_before = lanemask_lt() & (half ? 0xffff0000u : 0x0000ffffu);
   int rank = __popc(__match_any_sync(0xffffffffu, __float_as_uint(x)) & same_half_before);   // earlier equal candidates
   for (int q = 0; q < Ch; q += 4) {
-    const float4 a = *reinterpret_cast<const float4*>(mine + q);
-    rank += (a.x > x ? 1 : 0) + (a.y > x ? 1 : 0) + (a.z > x ? 1 : 0) + (a.w > x ? 1 : 0);
+    const float4 c01 = *reinterpret_cast<const float4*>(mine + q);   // broadcast reads inside the half-warp
+    const float4 c23 = *reinterpret_cast<const float4*>(mine + q + 2);
+    rank += (c01.x > x ? 1 : 0) + (c01.z > x ? 1 : 0) + (c23.x > x ? 1 : 0) + (c23.z > x ? 1 : 0);
   }
   if (l < Ch && rank < K) {
     out_val[half * 16 + rank] = x;
@@ -375,13 +384,14 @@ __device__ __forceinline__ void warp_gate_one(const float (&v)[VPT], int32_t tok
   }
 }
 
-// Stand-alone gate: grid-stride over tokens, the next rows loaded while the current ones are selected (two sets of
-// row buffers used in turn).  VPT > 0: register form for rows of at most 32 * VPT logits (one instantiation per
-// row length class, so that short rows keep few registers and many warps per SM).  PAIRS: two tokens per warp
-// (tokens 2p and 2p+1; needs VPT >= 4 and K <= 16), else one.  VPT == 0: shared-memory form for longer rows;
-// dynamic shared memory: warps * E floats.
-// Every selection form appears at most twice in a kernel: with more inlined copies the code outgrew the
-// instruction caches and a call chained behind others started 2 us later.
+// Stand-alone gate: grid-stride over tokens.  VPT > 0: register form for rows of at most 32 * VPT logits (one
+// instantiation per row length class, so that short rows keep few registers and many warps per SM).  PAIRS: two
+// tokens per warp (tokens 2p and 2p+1; needs VPT >= 4 and K <= 16), else one.  VPT == 0: shared-memory form for
+// longer rows; dynamic shared memory: warps * E floats.
+// The pair form loads its rows when it needs them: 32 resident warps per SM cover the latency, and loading the
+// next pair ahead cost 32 registers, moves and spills (13.2 against 12.3 us at 32768 tokens of 256 logits).  No
+// kernel inlines a selection form more than twice: with more copies the code outgrew the instruction caches
+// (231 KB) and a planner chained behind the gate started 2 us later.
 template <int VPT, bool PAIRS>
 __global__ void __launch_bounds__(256, VPT == 8 ? 4 : 1)
 gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t K, int32_t* __restrict__ topk_idx,
@@ -426,18 +436,14 @@ gate_topk_kernel(const float* __restrict__ logits, int32_t T, int32_t E, int32_t
           }
         }
       };
-      float a0[VPT], b0[VPT], a1[VPT], b1[VPT];
-      if (t < pairs) load_pair(t, a0, b0);
-      while (t < pairs) {
-        if (t + stride < pairs) load_pair(t + stride, a1, b1);
-        process_pair(a0, b0, t);
-        t += stride;
-        if (t >= pairs) break;
-        if (t + stride < pairs) load_pair(t + stride, a0, b0);
-        process_pair(a1, b1, t);
-        t += stride;
+      float a[VPT], b[VPT];
+      for (; t < pairs; t += stride) {
+        load_pair(t, a, b);
+        process_pair(a, b, t);
       }
     } else {
+      // two row buffers used in turn, the next token's row travelling while the current one is selected: the short
+      // rows' few instructions per token do not cover a load from DRAM (11.2 against 12.2 us, 32768 tokens of 64)
       float row_a[VPT], row_b[VPT];
       if (t < T) warp_gate_load<VPT>(logits + (size_t)t * E, E, lane, vec, row_a);
       while (t < T) {
