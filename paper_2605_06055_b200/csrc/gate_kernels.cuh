@@ -129,6 +129,19 @@ __device__ __forceinline__ void warp_gate_select(const float (&v)[VPT], int K, i
   idx_lane = sel_idx;
 }
 
+// -1 where a >= b (a > b), else 0.  Written as `set`: the compiler turns the plain conditional into a longer
+// sequence (50 more instructions per pair of tokens when the candidate counts were written that way).
+__device__ __forceinline__ int32_t ge_mask_f32(float a, float b) {
+  int32_t m;
+  asm("set.ge.s32.f32 %0, %1, %2;" : "=r"(m) : "f"(a), "f"(b));
+  return m;
+}
+__device__ __forceinline__ int32_t gt_mask_f32(float a, float b) {
+  int32_t m;
+  asm("set.gt.s32.f32 %0, %1, %2;" : "=r"(m) : "f"(a), "f"(b));
+  return m;
+}
+
 // Selection by threshold and rank, for the common case.  theta, the K-th largest DISTINCT value among the 32
 // lane maxima (K rounds of "warp max, then drop the lanes that hold it": three instructions each, no index
 // tracking), is a lower bound of the K-th largest logit, because at least K entries are >= theta; so every
@@ -167,7 +180,7 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
   theta = fmaxf(theta, -3.402823466e+38f);
   int c = 0;
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) c += (v[i] >= theta) ? 1 : 0;
+  for (int i = 0; i < VPT; ++i) c -= ge_mask_f32(v[i], theta);
   int incl = c;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
@@ -200,7 +213,7 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
   for (int q = 0; q < C; q += 4) {
     const float4 c01 = *reinterpret_cast<const float4*>(cand + q);   // broadcast reads
     const float4 c23 = *reinterpret_cast<const float4*>(cand + q + 2);
-    rank += (c01.x > x ? 1 : 0) + (c01.z > x ? 1 : 0) + (c23.x > x ? 1 : 0) + (c23.z > x ? 1 : 0);
+    rank -= gt_mask_f32(c01.x, x) + gt_mask_f32(c01.z, x) + gt_mask_f32(c23.x, x) + gt_mask_f32(c23.z, x);
   }
   if (lane < C && rank < K) {
     out_val[rank] = x;
@@ -254,8 +267,8 @@ __device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], cons
   int na = 0, nb = 0;   // minus this lane's candidate counts
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
-    na += (va[i] >= ta) ? -1 : 0;
-    nb += (vb[i] >= tb) ? -1 : 0;
+    na += ge_mask_f32(va[i], ta);
+    nb += ge_mask_f32(vb[i], tb);
   }
   const int c = -(na + (nb << 16));   // token A's count in the low half of the word, token B's in the high half
   int incl = c;
@@ -302,7 +315,7 @@ __device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], cons
   for (int q = 0; q < Ch; q += 4) {
     const float4 c01 = *reinterpret_cast<const float4*>(mine + q);   // broadcast reads inside the half-warp
     const float4 c23 = *reinterpret_cast<const float4*>(mine + q + 2);
-    rank += (c01.x > x ? 1 : 0) + (c01.z > x ? 1 : 0) + (c23.x > x ? 1 : 0) + (c23.z > x ? 1 : 0);
+    rank -= gt_mask_f32(c01.x, x) + gt_mask_f32(c01.z, x) + gt_mask_f32(c23.x, x) + gt_mask_f32(c23.z, x);
   }
   if (l < Ch && rank < K) {
     out_val[half * 16 + rank] = x;
