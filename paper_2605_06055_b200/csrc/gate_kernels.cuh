@@ -197,9 +197,9 @@ __device__ __forceinline__ bool warp_gate_rank(const float (&v)[VPT], int K, int
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ge.f32 p, %1, %2;\n\t"
-        "@p st.shared.v2.b32 [%0], {%3, %4};\n\t"
+        "@p st.shared.v2.b32 [%0], {%1, %3};\n\t"
         "@p add.u32 %0, %0, 8;\n\t}"
-        : "+r"(slot) : "f"(v[i]), "f"(theta), "r"(__float_as_uint(v[i])), "r"(base + i) : "memory");
+        : "+r"(slot) : "f"(v[i]), "f"(theta), "r"(base + i) : "memory");
   }
   __syncwarp();
   float x = -INFINITY;
@@ -291,14 +291,13 @@ __device__ __forceinline__ bool warp_gate_rank_pair(const float (&va)[VPT], cons
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ge.f32 p, %2, %3;\n\t"
-        "setp.ge.f32 q, %6, %7;\n\t"
-        "@p st.shared.v2.b32 [%0], {%4, %5};\n\t"
-        "@q st.shared.v2.b32 [%1], {%8, %5};\n\t"
+        "setp.ge.f32 q, %5, %6;\n\t"
+        "@p st.shared.v2.b32 [%0], {%2, %4};\n\t"
+        "@q st.shared.v2.b32 [%1], {%5, %4};\n\t"
         "@p add.u32 %0, %0, 8;\n\t"
         "@q add.u32 %1, %1, 8;\n\t}"
         : "+r"(slot_a), "+r"(slot_b)
-        : "f"(va[i]), "f"(ta), "r"(__float_as_uint(va[i])), "r"(base + i), "f"(vb[i]), "f"(tb),
-          "r"(__float_as_uint(vb[i]))
+        : "f"(va[i]), "f"(ta), "r"(base + i), "f"(vb[i]), "f"(tb)
         : "memory");
   }
   __syncwarp();
