@@ -34,8 +34,8 @@ enum {
   ORACLE_ERR_CAPACITY = 3
 };
 
-/* Top-k gating (the step before dispatch: "top-k gating produces routing indexes and weights",
- * Figures 1 and 4).  The paper gives no formula; the reading taken is the common one that the
+/* Top-k gating (the step before dispatch: both workflow figures, Figures 1 and 4, start from a gate
+ * that turns hidden states into routing indexes and routing weights).  The paper gives no formula; the reading taken is the common one that the
  * benchmark configurations describe: the K largest router logits of every token, in descending
  * order (equal logits: the lower expert index first), and the softmax over those K logits in fp32:
  *   w_j = exp(l_j - l_0) / sum_{j'=0..K-1} exp(l_j' - l_0),   sum accumulated in ascending j.
@@ -118,8 +118,8 @@ int oracle_expert_scale(uint16_t* windows, int32_t H, int32_t E, int32_t R, int6
 int oracle_combine(const uint16_t* windows, int32_t T, int32_t H, int32_t K,
                    const int64_t* slots, const float* W, uint16_t* Y, int32_t n_threads);
 
-/* Row-wise quantised dispatch (Section 5.2, Prefill Dispatch: "if row-wise quantization is enabled,
- * the corresponding scale values are written into a parallel scale tensor in the same row order").
+/* Row-wise quantised dispatch (Section 5.2, Prefill Dispatch: with row-wise quantisation switched on,
+ * the scales go to a second tensor laid out row for row like the expert window).
  * The paper fixes no format; the reading taken here is fp8 e4m3 (1-4-3, bias 7, largest finite value
  * 448, no infinities) with one fp32 scale per row:
  *   amax  = max_h |float(X[t,h])|
