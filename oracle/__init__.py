@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_expert_tiles.restype = ctypes.c_int
         L.oracle_dispatch_quant.argtypes = [p, i32, i32, i32, p, p, p, i32]
         L.oracle_dispatch_quant.restype = ctypes.c_int
+        L.oracle_dispatch_quant_group.argtypes = [p, i32, i32, i32, p, p, p, i32, i32]
+        L.oracle_dispatch_quant_group.restype = ctypes.c_int
         L.oracle_float_to_e4m3.argtypes = [ctypes.c_float]
         L.oracle_float_to_e4m3.restype = ctypes.c_uint8
         L.oracle_e4m3_to_float.argtypes = [ctypes.c_uint8]
@@ -183,6 +185,18 @@ def dispatch_quant(X_u16, slots_, windows_q, scales, n_threads: int = 1) -> int:
     assert windows_q.dtype == np.uint8 and windows_q.flags["C_CONTIGUOUS"]
     assert scales.dtype == np.float32 and scales.flags["C_CONTIGUOUS"]
     return lib().oracle_dispatch_quant(_ptr(X_u16), T, H, K, _ptr(slots_), _ptr(windows_q), _ptr(scales), n_threads)
+
+
+def dispatch_quant_group(X_u16, slots_, windows_q, scales, group: int, n_threads: int = 1) -> int:
+    """As dispatch_quant with one fp32 scale per `group` consecutive elements: scales is [rows, H // group]."""
+    X_u16 = _c(X_u16, np.uint16)
+    slots_ = _c(slots_, np.int64)
+    T, H = X_u16.shape
+    K = slots_.shape[1]
+    assert windows_q.dtype == np.uint8 and windows_q.flags["C_CONTIGUOUS"]
+    assert scales.dtype == np.float32 and scales.flags["C_CONTIGUOUS"]
+    return lib().oracle_dispatch_quant_group(_ptr(X_u16), T, H, K, _ptr(slots_), _ptr(windows_q), _ptr(scales),
+                                             int(group), n_threads)
 
 
 def float_to_e4m3(x: float) -> int:

@@ -123,6 +123,36 @@ int oracle_dispatch_quant(const uint16_t* X, int32_t T, int32_t H, int32_t K, co
   return ORACLE_OK;
 }
 
+int oracle_dispatch_quant_group(const uint16_t* X, int32_t T, int32_t H, int32_t K, const int64_t* slots,
+                                uint8_t* windows_q, float* scales, int32_t group, int32_t n_threads) {
+  if (T < 0 || H < 1 || K < 1 || group < 1 || H % group != 0) return ORACLE_ERR_INVALID_ARG;
+  const int32_t G = H / group;
+  for_token_ranges(T, n_threads, [=](int32_t lo, int32_t hi) {
+    std::vector<uint8_t> code((size_t)H);
+    std::vector<float> scale((size_t)G);
+    for (int32_t t = lo; t < hi; ++t) {
+      const uint16_t* x = X + (int64_t)t * H;
+      for (int32_t g = 0; g < G; ++g) {      // every group of `group` consecutive elements is a little row of its own
+        float amax = 0.0f;
+        for (int32_t h = g * group; h < (g + 1) * group; ++h) amax = std::fmax(amax, std::fabs(oracle_bf16_to_float(x[h])));
+        float inv = 1.0f;
+        scale[g] = 1.0f;
+        if (amax > 0.0f) {
+          scale[g] = amax / 448.0f;
+          inv = 448.0f / amax;
+        }
+        for (int32_t h = g * group; h < (g + 1) * group; ++h) code[h] = oracle_float_to_e4m3(oracle_bf16_to_float(x[h]) * inv);
+      }
+      for (int32_t j = 0; j < K; ++j) {
+        const int64_t row = slots[(int64_t)t * K + j];
+        std::memcpy(windows_q + row * H, code.data(), (size_t)H);
+        std::memcpy(scales + row * G, scale.data(), (size_t)G * sizeof(float));
+      }
+    }
+  });
+  return ORACLE_OK;
+}
+
 int oracle_gate_topk(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* topk_idx, float* topk_w) {
   if (T < 0 || E < 1 || K < 1 || K > E) return ORACLE_ERR_INVALID_ARG;
   std::vector<char> taken((size_t)E);

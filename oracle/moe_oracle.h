@@ -130,6 +130,13 @@ int oracle_combine(const uint16_t* windows, int32_t T, int32_t H, int32_t K,
 int oracle_dispatch_quant(const uint16_t* X, int32_t T, int32_t H, int32_t K, const int64_t* slots,
                           uint8_t* windows_q, float* scales, int32_t n_threads);
 
+/* The same with one scale per GROUP of `group` consecutive elements of a row instead of one per row (the
+ * paper names no granularity; 128 is the group the fp8 expert GEMMs of the benchmark's model family consume):
+ * each group is quantised exactly like a row of its own by the rule above.  H % group == 0.
+ *   windows_q [rows, H] uint8,  scales [rows, H / group] fp32 (group g of row r at scales[r * (H/group) + g]). */
+int oracle_dispatch_quant_group(const uint16_t* X, int32_t T, int32_t H, int32_t K, const int64_t* slots,
+                                uint8_t* windows_q, float* scales, int32_t group, int32_t n_threads);
+
 /* e4m3 conversions used above, exported so that tests can pin them against a library conversion. */
 uint8_t oracle_float_to_e4m3(float f);
 float oracle_e4m3_to_float(uint8_t c);

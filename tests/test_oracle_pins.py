@@ -520,6 +520,68 @@ def test_dispatch_quant_against_torch_pipeline_and_error_bound(T, K, E, R, H):
     assert (top[amax.numpy() > 0] == 0x7E).all() and top[3] == 0
 
 
+@pytest.mark.parametrize("T,K,E,R,H,group", [(40, 2, 8, 4, 256, 128), (33, 8, 16, 2, 384, 128), (20, 4, 8, 2, 96, 32)])
+def test_dispatch_quant_group_against_torch_pipeline_rowwise_slices_and_error_bound(T, K, E, R, H, group):
+    rng = np.random.default_rng(T + H)
+    idx, rts = random_case(rng, T, K, E, R)
+    X = rand_bf16(rng, (T, H))
+    X[3] = 0                                          # an all-zero row: every scale 1, codes 0
+    X[4, group:2 * group] = 0                         # one all-zero group inside a live row
+    X[5, 7] = synth.bf16_to_u16(torch.tensor([300.0]).to(torch.bfloat16))[0]     # an outlier: only ITS group's scale grows
+    X[:, :group] = (u16_to_float(X[:, :group]) * 64).astype(np.float32).view(np.uint32) >> 16   # groups of very different magnitude
+    G = H // group
+    p = oracle.plan(idx, E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(idx, E, R, p, C, rts)
+    wq = np.full((R * C, H), 0xAB, np.uint8)
+    sc = np.full((R * C, G), -1.0, np.float32)
+    assert oracle.dispatch_quant_group(X, slots, wq, sc, group) == oracle.OK
+
+    # (1) library ops: fp32 amax per group, two fp32 divisions, fp32 product, torch's e4m3 rounding
+    xf = torch.from_numpy(u16_to_float(X)).view(T, G, group)
+    amax = xf.abs().amax(dim=2)
+    scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+    inv = torch.where(amax > 0, torch.full_like(amax, 448.0) / amax, torch.ones_like(amax))
+    codes = (xf * inv[:, :, None]).to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(T, H)
+    owner = np.full(R * C, -1)
+    owner[slots.reshape(-1)] = np.repeat(np.arange(T), K)
+    for row in range(R * C):
+        t = owner[row]
+        if t < 0:
+            assert (wq[row] == 0xAB).all() and (sc[row] == -1.0).all()          # untouched
+        else:
+            nz = codes[t] & 0x7F != 0
+            assert np.array_equal(wq[row] & 0x7F != 0, nz)
+            assert np.array_equal(wq[row][nz], codes[t][nz]) and np.array_equal(sc[row], scale[t].numpy())
+
+    # (2) every group is a row of its own for the row-wise function: X viewed as [T*G, group], one slot per little row
+    little = np.ascontiguousarray(X.reshape(T * G, group))
+    lw = np.zeros((T * G, group), np.uint8)
+    ls = np.zeros((T * G,), np.float32)
+    assert oracle.dispatch_quant(little, np.arange(T * G, dtype=np.int64)[:, None], lw, ls) == oracle.OK
+    first = slots[:, 0]
+    assert np.array_equal(wq[first], lw.reshape(T, H)) and np.array_equal(sc[first], ls.reshape(T, G))
+    # ... and one group spanning the row IS the row-wise function
+    wq1 = np.zeros((R * C, H), np.uint8)
+    sc1 = np.zeros((R * C, 1), np.float32)
+    wq2 = np.zeros((R * C, H), np.uint8)
+    sc2 = np.zeros((R * C,), np.float32)
+    assert oracle.dispatch_quant_group(X, slots, wq1, sc1, H) == oracle.OK
+    assert oracle.dispatch_quant(X, slots, wq2, sc2) == oracle.OK
+    assert np.array_equal(wq1, wq2) and np.array_equal(sc1[:, 0], sc2)
+
+    # (3) round trip within the format's error, group by group; the largest element of a live group takes the top code
+    deq = (torch.from_numpy(wq[first]).view(torch.float8_e4m3fn).float().view(T, G, group) *
+           torch.from_numpy(sc[first])[:, :, None])
+    err = (deq - xf).abs()
+    bound = xf.abs() * 2.0 ** -4 * (1 + 1e-5) + scale[:, :, None] * 2.0 ** -10 * (1 + 1e-5)
+    assert bool((err <= bound).all())
+    top = (wq[first] & 0x7F).reshape(T, G, group).max(2)
+    assert (top[amax.numpy() > 0] == 0x7E).all() and (top[3] == 0).all() and top[4, 1] == 0
+    # H not a multiple of the group is refused
+    assert oracle.dispatch_quant_group(X, slots, wq, sc, group - 1 if H % (group - 1) else group + 1) != oracle.OK
+
+
 # ----------------------------------------------------------------------------- gating
 @pytest.mark.parametrize("T,E,K", [(64, 16, 2), (200, 256, 8), (33, 8, 8), (50, 40, 1), (10, 4096, 32)])
 def test_gate_topk_against_torch(T, E, K):
