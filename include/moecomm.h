@@ -187,6 +187,25 @@ moe_status_t moe_plan_dispatch_quant(moe_ctx_t* ctx, moe_schedule_t schedule, co
                                      void* windows_q /*DEVICE*/, float* scales /*DEVICE*/, int64_t capacity_rows,
                                      void* stream);
 
+/* The quantised dispatch with one scale per GROUP of group_size consecutive elements of a row instead of
+ * one per row (same passage; the paper names no granularity either, and 128 is what fp8 expert GEMMs with
+ * 1 x 128 activation scales consume).  Every group is quantised by the rule of moe_dispatch_quant as if it
+ * were a row of its own.
+ *   group_size must be 128 and H % 128 == 0 (else MOE_ERR_INVALID_ARG); H <= 16384
+ *   windows_q  DEVICE [R, capacity_rows, H] uint8, 16-byte aligned
+ *   scales     DEVICE [R, capacity_rows, H / 128] fp32: group g of window row r at scales[r * (H/128) + g]
+ * Otherwise as moe_dispatch_quant. */
+moe_status_t moe_dispatch_quant_group(moe_ctx_t* ctx, const void* x /*DEVICE*/, void* windows_q /*DEVICE*/,
+                                      float* scales /*DEVICE*/, int64_t capacity_rows, int32_t group_size,
+                                      void* stream);
+
+/* moe_plan followed by moe_dispatch_quant_group as one chained call (see moe_plan_dispatch_quant). */
+moe_status_t moe_plan_dispatch_quant_group(moe_ctx_t* ctx, moe_schedule_t schedule,
+                                           const int32_t* topk_idx /*DEVICE*/, int32_t T,
+                                           const int32_t* rank_tok_start /*HOST*/, const void* x /*DEVICE*/,
+                                           void* windows_q /*DEVICE*/, float* scales /*DEVICE*/,
+                                           int64_t capacity_rows, int32_t group_size, void* stream);
+
 /* Combine (Algorithm 1 / Algorithm 2, second loop; Section 5.2 Prefill Combine):
  *   Y[t,h] = bf16_rne( sum_{j=0..K-1} W[t,j] * float(windows[slot(t,j), h]) )
  * accumulated in fp32 from +0 with one fused multiply-add per term, j ascending.

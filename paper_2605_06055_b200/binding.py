@@ -29,7 +29,7 @@ EXPORTS = [
     "moe_dispatch_range", "moe_combine_range", "moe_plan_dispatch", "moe_gate_plan_dispatch", "moe_plan_dispatch_quant", "moe_expert_tiles", "moe_dispatch_quant_peers",
     "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
     "moe_dispatch_cached", "moe_combine_cached", "moe_state_bytes", "moe_window_bytes", "moe_signal_peers",
-    "moe_wait_peers", "moe_dispatch_quant_cached",
+    "moe_wait_peers", "moe_dispatch_quant_cached", "moe_dispatch_quant_group", "moe_plan_dispatch_quant_group",
 ]
 MOE_SYNC_SLOTS = 4
 MOE_WINDOW_STATE, MOE_WINDOW_QUANT = 1, 2
@@ -93,6 +93,10 @@ def load() -> ctypes.CDLL:
     L.moe_gate_plan_dispatch.restype = ctypes.c_int
     L.moe_plan_dispatch_quant.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp, vp, vp, i64, vp]
     L.moe_plan_dispatch_quant.restype = ctypes.c_int
+    L.moe_plan_dispatch_quant_group.argtypes = [vp, ctypes.c_int, vp, i32, vp, vp, vp, vp, i64, i32, vp]
+    L.moe_plan_dispatch_quant_group.restype = ctypes.c_int
+    L.moe_dispatch_quant_group.argtypes = [vp, vp, vp, vp, i64, i32, vp]
+    L.moe_dispatch_quant_group.restype = ctypes.c_int
     L.moe_layout.argtypes = [vp, ctypes.c_int, vp, i32, i32, vp, vp]
     L.moe_notify.argtypes = [vp, vp, vp]
     L.moe_dispatch_peers.argtypes = [vp, vp, vp, i64, vp]
@@ -278,6 +282,24 @@ class MoeComm:
             self.T, self.schedule, self._keep = T, schedule, topk_idx
         elif check:
             raise MoeError(rc, "moe_plan_dispatch_quant")
+        return rc
+
+    def moe_plan_dispatch_quant_group(self, schedule: int, topk_idx: torch.Tensor, x: torch.Tensor,
+                                      windows_q: torch.Tensor, scales: torch.Tensor, capacity_rows: int,
+                                      group_size: int = 128, T: Optional[int] = None, rank_tok_start=None,
+                                      stream=None, check: bool = True) -> int:
+        T = topk_idx.shape[0] if T is None else T
+        rts = None if rank_tok_start is None else np.ascontiguousarray(rank_tok_start, dtype=np.int32)
+        with self._on_device():
+            rc = self.lib.moe_plan_dispatch_quant_group(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T,
+                                                        _host_ptr(rts), _dev_ptr(x, torch.bfloat16),
+                                                        _dev_ptr(windows_q, torch.uint8),
+                                                        _dev_ptr(scales, torch.float32), int(capacity_rows),
+                                                        int(group_size), _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx
+        elif check:
+            raise MoeError(rc, "moe_plan_dispatch_quant_group")
         return rc
 
     def moe_gate_plan_dispatch(self, schedule: int, logits: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor,
@@ -488,6 +510,16 @@ class MoeComm:
                                              _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_dispatch_quant")
+        return rc
+
+    def moe_dispatch_quant_group(self, x: torch.Tensor, windows_q: torch.Tensor, scales: torch.Tensor,
+                                 capacity_rows: int, group_size: int = 128, stream=None, check: bool = True) -> int:
+        with self._on_device():
+            rc = self.lib.moe_dispatch_quant_group(self._h, _dev_ptr(x, torch.bfloat16),
+                                                   _dev_ptr(windows_q, torch.uint8), _dev_ptr(scales, torch.float32),
+                                                   int(capacity_rows), int(group_size), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_quant_group")
         return rc
 
     def moe_dispatch_quant_peers(self, x: torch.Tensor, window_q_bases: torch.Tensor, scale_bases: torch.Tensor,

@@ -2,7 +2,7 @@
 
     python -m paper_2605_06055_b200.cases <call> <workload> [--reps N] [--flush]
 
-  call      gate | plan | dispatch | combine | dispatch_quant | step
+  call      gate | plan | dispatch | combine | dispatch_quant | dispatch_quant_group | step
   workload  c1 c2 c3 c4 c3s (config 3 at a quarter of the tokens) c5 (T=65536) c5m (T=8192) k7
 
 Every repetition is preceded by a 256 MB write when --flush is given, so that a workload smaller than the L2
@@ -32,7 +32,7 @@ WORKLOADS = {
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("call", choices=["gate", "plan", "dispatch", "combine", "dispatch_quant", "step"])
+    ap.add_argument("call", choices=["gate", "plan", "dispatch", "combine", "dispatch_quant", "dispatch_quant_group", "step"])
     ap.add_argument("workload", choices=sorted(WORKLOADS))
     ap.add_argument("--reps", type=int, default=4)
     ap.add_argument("--flush", action="store_true")
@@ -63,6 +63,10 @@ def main() -> None:
         wq = torch.zeros((wl.R * C, wl.H), dtype=torch.uint8, device=dev)
         sc = torch.zeros((wl.R * C,), dtype=torch.float32, device=dev)
         call = lambda: comm.moe_dispatch_quant(X, wq, sc, C)
+    elif args.call == "dispatch_quant_group":
+        wq = torch.zeros((wl.R * C, wl.H), dtype=torch.uint8, device=dev)
+        sc = torch.zeros((wl.R * C, wl.H // 128), dtype=torch.float32, device=dev)
+        call = lambda: comm.moe_dispatch_quant_group(X, wq, sc, C)
     else:
         def call():
             comm.moe_plan(wl.schedule, idx)

@@ -416,11 +416,17 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   auto opt_in = [&](auto kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess;
   };
-  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<2, 16, true>) && opt_in(dispatch_quant_kernel<3, 16, true>) &&
-       opt_in(dispatch_quant_kernel<2, 32, true>) && opt_in(dispatch_quant_kernel<3, 32, true>) &&
-       opt_in(dispatch_quant_kernel<2, 16, false>) && opt_in(dispatch_quant_kernel<3, 16, false>) &&
-       opt_in(dispatch_quant_kernel<2, 32, false>) && opt_in(dispatch_quant_kernel<3, 32, false>) &&
-       opt_in(dispatch_quant_kernel<2, 0, false>) && opt_in(dispatch_quant_kernel<3, 0, false>) && opt_in(plan_rank_kernel<32>) &&
+  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<3, 16, true>) &&
+       opt_in(dispatch_quant_kernel<3, 32, true>) &&
+       opt_in(dispatch_quant_kernel<3, 16, false>) &&
+       opt_in(dispatch_quant_kernel<3, 32, false>) &&
+       opt_in(dispatch_quant_kernel<2, 0, false>) && opt_in(dispatch_quant_kernel<3, 0, false>) &&
+       opt_in(dispatch_quant_kernel<2, 0, false, true>) && opt_in(dispatch_quant_kernel<3, 0, false, true>) &&
+       opt_in(dispatch_quant_reg_kernel<16, true, true>) && opt_in(dispatch_quant_reg_kernel<16, false, true>) &&
+       opt_in(dispatch_quant_reg_kernel<16, true, false>) && opt_in(dispatch_quant_reg_kernel<16, false, false>) &&
+       opt_in(dispatch_quant_reg_kernel<32, true, true>) && opt_in(dispatch_quant_reg_kernel<32, false, true>) &&
+       opt_in(dispatch_quant_reg_kernel<32, true, false>) && opt_in(dispatch_quant_reg_kernel<32, false, false>) &&
+       opt_in(plan_rank_kernel<32>) &&
        opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
        opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0, false>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
@@ -792,14 +798,22 @@ moe_status_t moe_dispatch_peers(moe_ctx_t* ctx, const void* x, const void* const
   return dispatch_impl(ctx, x, nullptr, window_bases, capacity_rows, stream);
 }
 
+// group: 0 = one scale per row, QUANT_GROUP = one per 128 elements.
+static bool quant_shape_ok(int H, int group) {
+  if (H % 16 != 0 || H * 2 > QUANT_MAX_ROW_BYTES) return false;
+  return group == 0 || (group == QUANT_GROUP && H % QUANT_GROUP == 0);
+}
+
 static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windows_q, float* scales,
                                         int64_t capacity_rows, void* stream, bool behind_plan,
-                                        const void* const* q_bases = nullptr, float* const* s_bases = nullptr) {
+                                        const void* const* q_bases = nullptr, float* const* s_bases = nullptr,
+                                        int group = 0) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->planned) return MOE_ERR_NOT_PLANNED;
   const bool peers = q_bases != nullptr;   // one code window and one scale tensor per rank, addressed through tables
   const int H = ctx->shape.H;
-  if (H % 16 != 0 || H * 2 > QUANT_MAX_ROW_BYTES) return MOE_ERR_INVALID_ARG;
+  if (!quant_shape_ok(H, group)) return MOE_ERR_INVALID_ARG;
+  const bool grouped = group != 0;
   if (capacity_rows < 0 || (peers && s_bases == nullptr)) return MOE_ERR_INVALID_ARG;
   if (ctx->T > 0 && (x == nullptr || (!peers && (windows_q == nullptr || scales == nullptr)))) return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || (!peers && (!aligned16(windows_q) || (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)))
@@ -815,44 +829,96 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   // 16-byte chunks of a row per lane: rows of up to 16 (8 KB) or 32 (16 KB) are held in registers, longer ones
   // take the two-pass form; the 32-chunk form has registers for eight warps.
   const int cpl = upr <= 16 ? 16 : upr <= 32 ? 32 : 0;
-  const int max_warps = cpl == 32 ? 8 : QUANT_MAX_WARPS;
-  auto warps_for = [&](int stages) {
-    int w = QUANT_SMEM_BUDGET / (stages * (stage + 8));
-    return w > max_warps ? max_warps : w;
-  };
-  // Three stages once every warp of the two-stage configuration would see eight rows or more.
-  const int stages = (warps_for(3) >= 1 && (int64_t)ctx->T >= (int64_t)8 * grid * warps_for(2)) ? 3 : 2;
-  int warps = warps_for(stages);
-  if (warps < 1) return MOE_ERR_INVALID_ARG;
   const int64_t rows_per_sm = ((int64_t)ctx->T + grid - 1) / grid;
-  if (warps > rows_per_sm) warps = rows_per_sm < 1 ? 1 : (int)rows_per_sm;   // no warps without a row
+  const bool pdl = behind_plan && ctx->overlap != 0;
+  a.pdl = pdl;
+  const bool whole_slabs = a.H16 % 32 == 0;   // every chunk of a row is valid for all lanes or for none
   const int32_t keep = ctx->granule_override;
+  // The ring of whole-row stages: two or three stages per warp; the two-pass form also stages the row's group scales.
+  const int ring_warps_max = cpl == 32 ? 8 : QUANT_MAX_WARPS;
+  const int per_warp_extra = (grouped && cpl == 0) ? QUANT_MAX_GROUPS * (int)sizeof(float) : 0;
+  auto ring_warps = [&](int stages) {
+    int w = QUANT_SMEM_BUDGET / (stages * (stage + 8) + per_warp_extra);
+    return w > ring_warps_max ? ring_warps_max : w;
+  };
+  // A large job: every warp of the two-stage ring would see eight rows or more.
+  const bool large = ring_warps(3) >= 1 && (int64_t)ctx->T >= (int64_t)8 * grid * ring_warps(2);
+  // Rows short enough for registers take the register kernel (a load buffer and a code buffer per warp, the group
+  // scales and reciprocals behind the codes) when the job is small or the scales are group-wise: more rows in
+  // flight per SM is what both need.  Large row-wise jobs stay on the three-stage ring, which runs at the copy rate
+  // with five to nine warps; the register kernel with ten warps or more dropped to 0.74 of that at 8 KB rows
+  // (T=65536: 237 against 175 us).  Measured, register kernel against ring: decode shape 31.9 against 33.8 us
+  // row-wise and 40.0 against 44.1 us group-wise; group-wise at 32768 rows of 14 KB 398 against 419 us.
+  if (cpl > 0 && (grouped || !large)) {
+    const int sc_bytes = grouped ? ((H / QUANT_GROUP) * 4 + 15) / 16 * 16 : 0;
+    const int per_warp = stage + (H + 2 * sc_bytes + 127) / 128 * 128 + 8;
+    int warps = QUANT_SMEM_BUDGET / per_warp;
+    const int cap = cpl == 32 ? QUANT_REG_WARPS_LONG : QUANT_REG_WARPS_SHORT;
+    if (warps > cap) warps = cap;
+    // the fewest warps that still finish in the same number of rounds (14 rows per SM: 7 warps, not 10)
+    const int64_t rounds = rows_per_sm < 1 ? 1 : (rows_per_sm + warps - 1) / warps;
+    warps = rows_per_sm < 1 ? 1 : (int)((rows_per_sm + rounds - 1) / rounds);
+    ctx->granule_override = upr;
+    set_work(ctx, a, (int64_t)grid * warps, upr, false);
+    ctx->granule_override = keep;
+    auto launch = [&](auto kernel) {
+      launch_kernel(kernel, grid, warps * 32, warps * per_warp, static_cast<cudaStream_t>(stream), pdl, 0,
+                    static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
+    };
+    if (cpl == 16) {
+      if (grouped) whole_slabs ? launch(dispatch_quant_reg_kernel<16, true, true>) : launch(dispatch_quant_reg_kernel<16, false, true>);
+      else whole_slabs ? launch(dispatch_quant_reg_kernel<16, true, false>) : launch(dispatch_quant_reg_kernel<16, false, false>);
+    } else {
+      if (grouped) whole_slabs ? launch(dispatch_quant_reg_kernel<32, true, true>) : launch(dispatch_quant_reg_kernel<32, false, true>);
+      else whole_slabs ? launch(dispatch_quant_reg_kernel<32, true, false>) : launch(dispatch_quant_reg_kernel<32, false, false>);
+    }
+    return launch_ok(ctx);
+  }
+  const int stages = large ? 3 : 2;
+  int warps = ring_warps(stages);
+  if (warps < 1) return MOE_ERR_INVALID_ARG;
+  if (warps > rows_per_sm) warps = rows_per_sm < 1 ? 1 : (int)rows_per_sm;   // no warps without a row
   ctx->granule_override = upr;
   set_work(ctx, a, (int64_t)grid * warps, upr, false);
   ctx->granule_override = keep;
-  const int smem = warps * stages * (stage + 8);
-  const bool pdl = behind_plan && ctx->overlap != 0;
-  a.pdl = pdl;
+  const int smem = warps * (stages * (stage + 8) + per_warp_extra);
   auto launch = [&](auto kernel) {
     launch_kernel(kernel, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
                   static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
   };
-  const bool whole_slabs = a.H16 % 32 == 0;   // every chunk of a row is valid for all lanes or for none
-  if (stages == 3) {
+  if (grouped) {   // rows beyond 16 KB
+    stages == 3 ? launch(dispatch_quant_kernel<3, 0, false, true>) : launch(dispatch_quant_kernel<2, 0, false, true>);
+  } else if (stages == 3) {
     if (cpl == 16) whole_slabs ? launch(dispatch_quant_kernel<3, 16, true>) : launch(dispatch_quant_kernel<3, 16, false>);
     else if (cpl == 32) whole_slabs ? launch(dispatch_quant_kernel<3, 32, true>) : launch(dispatch_quant_kernel<3, 32, false>);
     else launch(dispatch_quant_kernel<3, 0, false>);
-  } else {
-    if (cpl == 16) whole_slabs ? launch(dispatch_quant_kernel<2, 16, true>) : launch(dispatch_quant_kernel<2, 16, false>);
-    else if (cpl == 32) whole_slabs ? launch(dispatch_quant_kernel<2, 32, true>) : launch(dispatch_quant_kernel<2, 32, false>);
-    else launch(dispatch_quant_kernel<2, 0, false>);
+  } else {   // (rows beyond 16 KB only: shorter rows of small jobs went to the register kernel)
+    launch(dispatch_quant_kernel<2, 0, false>);
   }
   return launch_ok(ctx);
+}
+
+// moe_plan followed by the quantising dispatch, chained; every host-side check comes before anything is enqueued.
+static moe_status_t plan_dispatch_quant_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                                             const int32_t* rank_tok_start, const void* x, void* windows_q,
+                                             float* scales, int64_t capacity_rows, int group, void* stream) {
+  if (!quant_shape_ok(ctx->shape.H, group) || capacity_rows < 0 || !aligned16(x) || !aligned16(windows_q) ||
+      (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)
+    return MOE_ERR_INVALID_ARG;
+  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, nullptr, nullptr, nullptr);
+  if (rc != MOE_OK) return rc;
+  return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, true, nullptr, nullptr, group);
 }
 
 moe_status_t moe_dispatch_quant(moe_ctx_t* ctx, const void* x, void* windows_q, float* scales, int64_t capacity_rows,
                                 void* stream) {
   return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, false);
+}
+
+moe_status_t moe_dispatch_quant_group(moe_ctx_t* ctx, const void* x, void* windows_q, float* scales,
+                                      int64_t capacity_rows, int32_t group_size, void* stream) {
+  if (group_size != QUANT_GROUP) return MOE_ERR_INVALID_ARG;
+  return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, false, nullptr, nullptr, group_size);
 }
 
 moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x, const void* const* window_q_bases,
@@ -866,13 +932,17 @@ moe_status_t moe_plan_dispatch_quant(moe_ctx_t* ctx, moe_schedule_t schedule, co
                                      int64_t capacity_rows, void* stream) {
   if (ctx == nullptr || (T > 0 && (topk_idx == nullptr || x == nullptr || windows_q == nullptr || scales == nullptr)))
     return MOE_ERR_INVALID_ARG;
-  const int H = ctx->shape.H;
-  if (H % 16 != 0 || H * 2 > QUANT_MAX_ROW_BYTES || capacity_rows < 0 || !aligned16(x) || !aligned16(windows_q) ||
-      (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)
-    return MOE_ERR_INVALID_ARG;   // before anything is enqueued
-  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T, rank_tok_start, stream, nullptr, nullptr, nullptr);
-  if (rc != MOE_OK) return rc;
-  return dispatch_quant_impl(ctx, x, windows_q, scales, capacity_rows, stream, true);
+  return plan_dispatch_quant_impl(ctx, schedule, topk_idx, T, rank_tok_start, x, windows_q, scales, capacity_rows, 0, stream);
+}
+
+moe_status_t moe_plan_dispatch_quant_group(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
+                                           const int32_t* rank_tok_start, const void* x, void* windows_q,
+                                           float* scales, int64_t capacity_rows, int32_t group_size, void* stream) {
+  if (ctx == nullptr || group_size != QUANT_GROUP ||
+      (T > 0 && (topk_idx == nullptr || x == nullptr || windows_q == nullptr || scales == nullptr)))
+    return MOE_ERR_INVALID_ARG;
+  return plan_dispatch_quant_impl(ctx, schedule, topk_idx, T, rank_tok_start, x, windows_q, scales, capacity_rows,
+                                  group_size, stream);
 }
 
 }  // extern "C"

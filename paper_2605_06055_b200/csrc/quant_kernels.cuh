@@ -7,6 +7,9 @@
 //   scale = amax / 448, inv = 448 / amax         (fp32, round to nearest; 1 and 1 when amax == 0)
 //   code[h] = e4m3( x[h] * inv )                 (fp32 product, round to nearest even, clamped to +-448)
 // Each token is quantised once; its K branches receive the same code row and scale.
+// Group-wise form (GROUPED): the same rule applied to every group of 128 consecutive elements of a row on its
+// own -- H / 128 scales per row, [rows, H / 128] fp32 in the same row order.  A group is the 16 chunks of 16 bytes
+// that one half-warp reads side by side, so its maximum is one half-warp reduction.
 //
 // Structure: the bulk-copy ring of dispatch_bulk_kernel with a compute step in
 // the middle.  A stage holds one whole row (needed for amax).  Lane 0 loads the
@@ -33,12 +36,26 @@ namespace moe {
 // decode shape (T=2048, 14 KB rows) 30.8 vs 32.7 us; T=65536 with 8 KB rows 235 vs 182 us.
 constexpr int QUANT_MAX_ROW_BYTES = 32 * 1024;
 constexpr int QUANT_MAX_WARPS = 16;
+constexpr int QUANT_REG_WARPS_LONG = 10;        // register kernel, rows beyond 8 KB: 204 registers per thread at most
+constexpr int QUANT_REG_WARPS_SHORT = 14;       // register kernel, rows up to 8 KB (16 warps measured slower than 14)
 constexpr int QUANT_SMEM_BUDGET = 220 * 1024;   // shared memory the warps' rings may fill
+constexpr int QUANT_GROUP = 128;                 // elements per scale of the group-wise form
+constexpr int QUANT_MAX_GROUPS = QUANT_MAX_ROW_BYTES / 2 / QUANT_GROUP;
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 
 __device__ __forceinline__ void sts64(uint32_t addr, uint32_t lo, uint32_t hi) {
@@ -70,10 +87,14 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t two_bf16, float inv) {
 // 16 for CPL <= 16, 8 beyond.
 // FULL: the row is a whole number of 512-byte slabs (H % 256 == 0), so a chunk is valid for all lanes or for none
 // and the per-lane bounds checks (a possibly divergent branch per chunk) reduce to a warp-uniform one.
-template <int QUANT_STAGES, int CPL, bool FULL>
+// GROUPED (two-pass form only; shorter rows take dispatch_quant_reg_kernel): one scale per 128 elements
+// (H % 128 == 0); dynamic shared memory then ends with [warps][QUANT_MAX_GROUPS] floats, the scales of the row a
+// warp is working on.
+template <int QUANT_STAGES, int CPL, bool FULL, bool GROUPED = false>
 __global__ void __launch_bounds__((CPL > 16 ? 8 : QUANT_MAX_WARPS) * 32, 1)
 dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
                       float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
+  static_assert(!GROUPED || CPL == 0, "group-wise scales of rows held in registers: dispatch_quant_reg_kernel");
   extern __shared__ __align__(128) unsigned char smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t row_bytes = (uint32_t)a.H16 * 16u;          // bf16 row
@@ -81,6 +102,16 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   const uint32_t stage_stride = (row_bytes + 127u) & ~127u;
   const uint32_t buf0 = smem_addr(smem) + warp * QUANT_STAGES * stage_stride;
   const uint32_t bar0 = smem_addr(smem) + n_warps * QUANT_STAGES * stage_stride + warp * QUANT_STAGES * 8;
+  // GROUPED: the scales of the row in hand
+  float* group_scale = reinterpret_cast<float*>(smem + (size_t)n_warps * QUANT_STAGES * (stage_stride + 8)) +
+                       warp * QUANT_MAX_GROUPS;
+  const int n_groups = a.H16 >> 4;                                      // GROUPED: scales per row
+  const unsigned half_mask = lane < 16 ? 0x0000ffffu : 0xffff0000u;
+  // Which half-warp, through an opaque instruction: with `lane >> 4` the compiler (12.9) simplified the byte
+  // offset (lane >> 4) * 4 to lane >> 2 under the store's guard (lane & 15) == 0 and then reused that address
+  // for the unguarded loads of every lane -- a misaligned address on the device.
+  int half;
+  asm("shr.u32 %0, %1, 4;" : "=r"(half) : "r"(lane));
 
   if (lane == 0) {
 #pragma unroll
@@ -157,6 +188,24 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
         inv = __fdiv_rn(448.0f, amax);
       }
     };
+    // Group-wise: chunk c = lane + 32 k of a row holds elements 8c .. 8c+7, so the sixteen lanes of a half-warp hold
+    // group 2k + half between them.  Converts this lane's chunk and leaves the group's scale in group_scale.
+    // Called by whole half-warps only (a row is a whole number of groups).
+    auto convert_group = [&](const uint4& v, int k, uint32_t dst) {
+      uint32_t m2 = __vmaxu2(__vmaxu2(v.x & 0x7fff7fffu, v.y & 0x7fff7fffu), __vmaxu2(v.z & 0x7fff7fffu, v.w & 0x7fff7fffu));
+      uint32_t mbits = max(m2 & 0xffffu, m2 >> 16);
+      mbits = __reduce_max_sync(half_mask, mbits);
+      const float amax = __uint_as_float(mbits << 16);
+      float g_scale = 1.0f, g_inv = 1.0f;
+      if (amax > 0.0f) {
+        g_scale = __fdiv_rn(amax, 448.0f);
+        g_inv = __fdiv_rn(448.0f, amax);
+      }
+      const uint32_t lo = quant_pair(v.x, g_inv) | (quant_pair(v.y, g_inv) << 16);
+      const uint32_t hi = quant_pair(v.z, g_inv) | (quant_pair(v.w, g_inv) << 16);
+      sts64(dst, lo, hi);
+      if ((lane & 15) == 0) group_scale[2 * k + half] = g_scale;
+    };
     if constexpr (CPL > 0) {
       uint4 v[CPL];
       uint32_t m[4] = {0u, 0u, 0u, 0u};
@@ -182,6 +231,14 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
           const uint32_t hi = quant_pair(v[k].z, inv) | (quant_pair(v[k].w, inv) << 16);
           sts64(in + (lane + 32 * k) * 8, lo, hi);
         }
+    } else if constexpr (GROUPED) {
+      // any row length: one pass, a chunk per lane at a time (in place as in the row-wise two-pass form below)
+      for (int c = lane, k = 0; c - lane < a.H16; c += 32, ++k) {   // warp-uniform trip count
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (c < a.H16) v = lds128(in + c * 16);
+        __syncwarp();
+        if (c < a.H16) convert_group(v, k, in + c * 8);
+      }
     } else {
       uint32_t m2 = 0;
       for (int c = lane; c < a.H16; c += 32) {
@@ -213,7 +270,14 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
       const int64_t row = __shfl_sync(0xffffffffu, slot, j);
       if (lane == 0 && row >= 0) bulk_store(window_row(a, windows_q, row, code_bytes), in, code_bytes, evict_first);
     }
-    if (lane < a.K && slot >= 0) {
+    if constexpr (GROUPED) {   // group_scale was written in front of the warp barrier above
+      for (int j = 0; j < a.K; ++j) {
+        const int64_t row = __shfl_sync(0xffffffffu, slot, j);
+        if (row < 0) continue;
+        float* dst = a.scale_base == nullptr ? scales + row * n_groups : a.scale_base[row / a.C] + (row % a.C) * n_groups;
+        for (int g = lane; g < n_groups; g += 32) dst[g] = group_scale[g];
+      }
+    } else if (lane < a.K && slot >= 0) {
       if (a.scale_base == nullptr) scales[slot] = scale;
       else a.scale_base[slot / a.C][slot % a.C] = scale;   // one scale tensor per rank, same row order as its window
     }
@@ -227,6 +291,191 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
       raise_status(a.status, MOE_ERR_TIMEOUT);
       if (q1 < a.n_items) mbar_wait(bar0 + 8 * ((it + 1) % QUANT_STAGES), ((it + 1) / QUANT_STAGES) & 1u, a.wait_limit_ms);
     }
+    bulk_wait_all();
+  }
+  end_work(a);
+}
+
+// The register forms as a kernel of their own: once a row of at most CPL * 512 bytes sits in a warp's registers its
+// load buffer is free again, so the NEXT row's load is issued right then and travels while this row is converted
+// and stored; the codes go to a separate buffer half as wide.  A warp needs 3H bytes of shared memory (2H load
+// buffer + H code buffer) instead of the 4H or 6H of a ring of whole-row stages, so more warps -- more rows in
+// flight -- share an SM: 10 instead of 5-7 at 14 KB rows.  One load and one group of stores are in flight per warp.
+// Dynamic shared memory: [warps] load buffers of l_stride bytes (row bytes rounded up to 128), [warps] code buffers
+// of c_stride bytes (codes, then for GROUPED the row's scales and their reciprocals, rounded up to 128), [warps]
+// mbarriers.
+template <int CPL, bool FULL, bool GROUPED>
+__global__ void __launch_bounds__((CPL > 16 ? QUANT_REG_WARPS_LONG : QUANT_REG_WARPS_SHORT) * 32, 1)
+dispatch_quant_reg_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
+                          float* __restrict__ scales, const RowArgs a, const __grid_constant__ RankMap map) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  const uint32_t row_bytes = (uint32_t)a.H16 * 16u;          // bf16 row
+  const uint32_t code_bytes = (uint32_t)a.H16 * 8u;          // e4m3 row
+  const int n_groups = a.H16 >> 4;                            // GROUPED: scales per row
+  const uint32_t sc_bytes = GROUPED ? (((uint32_t)n_groups * 4u + 15u) & ~15u) : 0u;
+  const uint32_t l_stride = (row_bytes + 127u) & ~127u;
+  const uint32_t c_stride = (code_bytes + 2u * sc_bytes + 127u) & ~127u;
+  const uint32_t in = smem_addr(smem) + warp * l_stride;
+  const uint32_t out = smem_addr(smem) + n_warps * l_stride + warp * c_stride;
+  const uint32_t bar = smem_addr(smem) + n_warps * (l_stride + c_stride) + warp * 8;
+  const unsigned half_mask = lane < 16 ? 0x0000ffffu : 0xffff0000u;
+  int half;   // lane >> 4 through an opaque instruction (see dispatch_quant_kernel)
+  asm("shr.u32 %0, %1, 4;" : "=r"(half) : "r"(lane));
+
+  if (lane == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  auto issue_load = [&](int32_t token) {   // lane 0 only
+    mbar_expect_tx(bar, row_bytes);
+    bulk_load(in, X + (size_t)token * row_bytes, row_bytes, bar);
+  };
+
+  uint64_t evict_first;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
+
+  // One work item = one token row.  q0 is consumed in this iteration; the load of q1 is issued in the middle of
+  // it, as soon as every lane holds its part of q0.
+  ItemFeed feed = begin_feed();
+  int32_t q0 = a.n_items, q1 = a.n_items;
+  // Started early behind the planner: the first rows of a small job are fixed and depend on nothing the planner
+  // writes, so the first load travels while the plan is computed.
+  const bool early = a.pdl && a.static_first >= 2;
+  if (early) {
+    q0 = fetch_item(a, feed);
+    q1 = fetch_item(a, feed);
+    if (lane == 0 && q0 < a.n_items) issue_load(q0);
+  }
+  dependency_wait();      // returns at once unless this launch was allowed to start early
+  release_dependents();
+  if (must_abort(a)) {
+    // a load already in flight must land before this CTA's shared memory is handed back
+    if (early && lane == 0 && q0 < a.n_items) mbar_wait(bar, 0, a.wait_limit_ms);
+    end_work(a);
+    return;
+  }
+  if (!early) {
+    q0 = fetch_item(a, feed);
+    q1 = fetch_item(a, feed);
+    if (lane == 0 && q0 < a.n_items) issue_load(q0);
+  }
+  const int slabs = a.H16 >> 5;   // FULL: chunks per lane
+  auto mine = [&](int k) { return FULL ? k < slabs : lane + 32 * k < a.H16; };
+  uint32_t it = 0;
+  bool timed_out = false;
+  while (q0 < a.n_items) {
+    const int32_t q2 = fetch_item(a, feed);
+    const int64_t slot = resolve_slot(a, map, q0, lane, true);   // overlaps the load in flight
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, it & 1u, a.wait_limit_ms) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) {
+      timed_out = true;   // the only load in flight is the one that did not land
+      break;
+    }
+    uint4 v[CPL];
+#pragma unroll
+    for (int k = 0; k < CPL; ++k)
+      if (mine(k)) v[k] = lds128(in + (lane + 32 * k) * 16);
+
+    float scale = 1.0f, inv = 1.0f;
+    if constexpr (GROUPED) {
+      const uint32_t sc = out + code_bytes, rc = sc + sc_bytes;
+      if (lane == 0) bulk_wait_read<0>();   // the previous row's stores have read the code buffer
+      __syncwarp();
+      // group maxima: one half-warp reduction per chunk (its sixteen lanes store the same word)
+#pragma unroll
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) {
+          const uint32_t m2 = __vmaxu2(__vmaxu2(v[k].x & 0x7fff7fffu, v[k].y & 0x7fff7fffu),
+                                       __vmaxu2(v[k].z & 0x7fff7fffu, v[k].w & 0x7fff7fffu));
+          const uint32_t mbits = __reduce_max_sync(half_mask, max(m2 & 0xffffu, m2 >> 16));
+          sts_f32(sc + 4 * (2 * k + half), __uint_as_float(mbits << 16));
+        }
+      __syncwarp();   // every reduction has consumed every lane's chunk: the load buffer is free
+      if (lane == 0 && q1 < a.n_items) issue_load(q1);
+      for (int g = lane; g < n_groups; g += 32) {   // lane g: scale and reciprocal of group g
+        const float amax = lds_f32(sc + 4 * g);
+        const float den = amax > 0.0f ? amax : 448.0f;   // an all-zero group: scale and reciprocal 1
+        sts_f32(sc + 4 * g, __fdiv_rn(den, 448.0f));
+        sts_f32(rc + 4 * g, __fdiv_rn(448.0f, den));
+      }
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) {
+          const float g_inv = lds_f32(rc + 4 * (2 * k + half));
+          const uint32_t lo = quant_pair(v[k].x, g_inv) | (quant_pair(v[k].y, g_inv) << 16);
+          const uint32_t hi = quant_pair(v[k].z, g_inv) | (quant_pair(v[k].w, g_inv) << 16);
+          sts64(out + (lane + 32 * k) * 8, lo, hi);
+        }
+    } else {
+      // amax: |bf16| patterns order like the values, so a per-halfword unsigned max of the sign-cleared words is
+      // the maximum magnitude.
+      uint32_t m[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) {
+          m[0] = __vmaxu2(m[0], v[k].x & 0x7fff7fffu);
+          m[1] = __vmaxu2(m[1], v[k].y & 0x7fff7fffu);
+          m[2] = __vmaxu2(m[2], v[k].z & 0x7fff7fffu);
+          m[3] = __vmaxu2(m[3], v[k].w & 0x7fff7fffu);
+        }
+      const uint32_t m2 = __vmaxu2(__vmaxu2(m[0], m[1]), __vmaxu2(m[2], m[3]));
+      const uint32_t mbits = __reduce_max_sync(0xffffffffu, max(m2 & 0xffffu, m2 >> 16));
+      // the reduction has consumed every lane's chunks: the load buffer is free
+      if (lane == 0) {
+        if (q1 < a.n_items) issue_load(q1);
+        bulk_wait_read<0>();   // the previous row's stores have read the code buffer
+      }
+      const float amax = __uint_as_float(mbits << 16);
+      if (amax > 0.0f) {
+        scale = __fdiv_rn(amax, 448.0f);
+        inv = __fdiv_rn(448.0f, amax);
+      }
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < CPL; ++k)
+        if (mine(k)) {
+          const uint32_t lo = quant_pair(v[k].x, inv) | (quant_pair(v[k].y, inv) << 16);
+          const uint32_t hi = quant_pair(v[k].z, inv) | (quant_pair(v[k].w, inv) << 16);
+          sts64(out + (lane + 32 * k) * 8, lo, hi);
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> bulk-copy reads
+    __syncwarp();
+
+    for (int j = 0; j < a.K; ++j) {
+      const int64_t row = __shfl_sync(0xffffffffu, slot, j);
+      if (row < 0) continue;
+      if (lane == 0) bulk_store(window_row(a, windows_q, row, code_bytes), out, code_bytes, evict_first);
+      if constexpr (GROUPED) {
+        // a bulk copy where the row of scales starts on a 16-byte boundary and is a multiple of 16 bytes long
+        float* dst = a.scale_base == nullptr ? scales + row * n_groups : a.scale_base[row / a.C] + (row % a.C) * n_groups;
+        if ((n_groups & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+          if (lane == 0) bulk_store(dst, out + code_bytes, (uint32_t)n_groups * 4u, evict_first);
+        } else {
+          for (int g = lane; g < n_groups; g += 32) dst[g] = lds_f32(out + code_bytes + 4 * g);
+        }
+      }
+    }
+    if constexpr (!GROUPED) {
+      if (lane < a.K && slot >= 0) {
+        if (a.scale_base == nullptr) scales[slot] = scale;
+        else a.scale_base[slot / a.C][slot % a.C] = scale;   // one scale tensor per rank, same row order as its window
+      }
+    }
+    if (lane == 0) bulk_commit();   // one group per row
+    q0 = q1;
+    q1 = q2;
+    ++it;
+  }
+  if (lane == 0) {
+    if (timed_out) raise_status(a.status, MOE_ERR_TIMEOUT);
     bulk_wait_all();
   }
   end_work(a);
