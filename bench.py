@@ -84,9 +84,11 @@ def bytes_plan(wl) -> int:
     return 8 * wl.T * wl.K + 8 * wl.E * wl.R
 
 
-def bytes_dispatch_quant(wl) -> int:
-    # read each bf16 row once; per branch write H e4m3 codes and one fp32 scale; same metadata as dispatch
-    return 2 * wl.H * wl.T + wl.K * wl.T * (wl.H + 4) + 8 * wl.T * wl.K + 4 * wl.E * wl.R
+def bytes_dispatch_quant(wl, group: int = 0) -> int:
+    # read each bf16 row once; per branch write H e4m3 codes and one fp32 scale per row (per `group` elements);
+    # same metadata as dispatch
+    scales = 1 if group == 0 else wl.H // group
+    return 2 * wl.H * wl.T + wl.K * wl.T * (wl.H + 4 * scales) + 8 * wl.T * wl.K + 4 * wl.E * wl.R
 
 
 def bytes_step(wl) -> int:
@@ -319,19 +321,24 @@ def time_steps(layer: Layer, steps: int, warmup: int, barrier, scratch=None):
     }
 
 
-def time_dispatch_quant(layer: Layer, steps: int, scratch=None):
-    """The row-wise quantised variant of dispatch (e4m3 codes + fp32 scale per row), same plan."""
+def time_dispatch_quant(layer: Layer, steps: int, scratch=None, group: int = 0):
+    """The quantised variant of dispatch (e4m3 codes + one fp32 scale per row, or per `group` elements), same plan."""
     wl = layer.wl
     wq = torch.zeros((wl.R * layer.C, wl.H), dtype=torch.uint8, device=layer.dev)
-    sc = torch.zeros((wl.R * layer.C,), dtype=torch.float32, device=layer.dev)
+    if group == 0:
+        sc = torch.zeros((wl.R * layer.C,), dtype=torch.float32, device=layer.dev)
+        call = lambda: layer.comm.moe_dispatch_quant(layer.X, wq, sc, layer.C)
+    else:
+        sc = torch.zeros((wl.R * layer.C, wl.H // group), dtype=torch.float32, device=layer.dev)
+        call = lambda: layer.comm.moe_dispatch_quant_group(layer.X, wq, sc, layer.C, group)
     for _ in range(3):
-        layer.comm.moe_dispatch_quant(layer.X, wq, sc, layer.C)
+        call()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for a, b in ev:
         if scratch is not None:
             scratch.add_(1)
         a.record()
-        layer.comm.moe_dispatch_quant(layer.X, wq, sc, layer.C)
+        call()
         b.record()
     torch.cuda.synchronize()
     assert layer.comm.moe_status() == 0
@@ -476,6 +483,8 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
     wscale = torch.empty((dwl.R * dl.C,), dtype=torch.float32, device=dev)
     quant = lambda: c.moe_dispatch_quant(dl.X, wq, wscale, dl.C)
     quant_fused = lambda: c.moe_plan_dispatch_quant(dwl.schedule, dl.idx, dl.X, wq, wscale, dl.C)
+    gscale = torch.empty((dwl.R * dl.C, dwl.H // 128), dtype=torch.float32, device=dev) if dwl.H % 128 == 0 else None
+    quant_group = (lambda: c.moe_dispatch_quant_group(dl.X, wq, gscale, dl.C, 128)) if gscale is not None else None
     out["gate_us_in_a_cuda_graph"] = time_graphed(gate)      # a 3 us kernel: launches from Python are slower than it
     for name, pre in (("cold", [flush]), ("warm", [])):
         base = time_repeated(pre, n) if pre else 0.0
@@ -483,6 +492,7 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
         plan()   # the gate leg below leaves the context planned on other indexes
         t_quant = time_repeated(pre + [quant], n)
         t_quant_fused = time_repeated(pre + [quant_fused], n)
+        t_quant_group = time_repeated(pre + [quant_group], n) if quant_group is not None else None
         t1 = time_repeated(pre + [plan], n)
         t2 = time_repeated(pre + [plan, disp], n)
         t3 = time_repeated(pre + [plan, disp, comb], n)
@@ -508,6 +518,9 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
                      "dispatch_quant_us": t_quant - base,
                      "plan_dispatch_quant_fused_us": t_quant_fused - base,
                      "dispatch_quant_GBps": bytes_dispatch_quant(dwl) / (t_quant - base) / 1e3}
+        if t_quant_group is not None:
+            out[name]["dispatch_quant_group128_us"] = t_quant_group - base
+            out[name]["dispatch_quant_group128_GBps"] = bytes_dispatch_quant(dwl, 128) / (t_quant_group - base) / 1e3
     plan()   # leave the context planned on dl.idx again
     assert c.moe_status() == 0
     del dl, wq, wscale, cp_src, cp_dst, logits, g_win, flush_buf
@@ -806,9 +819,11 @@ def run_cuda(args, wl):
     r = time_steps(layer, args.steps, args.warmup, barrier, scratch)
     ms_per_step = reduce_max_over_ranks(r["ms_per_step"], dist, dev)
     verified = verify(layer)            # bench steps use identity experts whatever the workload names
-    quant_us = None
+    quant_us = quant_group_us = None
     if wl.H % 16 == 0 and not args.no_decode:
         quant_us = time_dispatch_quant(layer, min(args.steps, 50), scratch)
+        if wl.H % 128 == 0:
+            quant_group_us = time_dispatch_quant(layer, min(args.steps, 50), scratch, 128)
     gate_us = None
     if not args.no_decode:
         from paper_2605_06055_b200 import binding
@@ -847,6 +862,13 @@ def run_cuda(args, wl):
                                          "bytes": bytes_dispatch_quant(wl), "GBps": gbps,
                                          "frac_of_measured_peak": gbps / peak, "frac_of_8TBps": gbps / NOMINAL_HBM_GBS,
                                          "note": "row-wise e4m3 + fp32 scale variant of dispatch; not part of the step"}
+    if quant_group_us is not None:
+        gb = bytes_dispatch_quant(wl, 128)
+        gbps = gb / (sum(quant_group_us) / len(quant_group_us)) / 1e3
+        kernels["moe_dispatch_quant_group"] = {"us": statistics.median(quant_group_us), "us_min": min(quant_group_us),
+                                               "bytes": gb, "GBps": gbps, "frac_of_measured_peak": gbps / peak,
+                                               "frac_of_8TBps": gbps / NOMINAL_HBM_GBS,
+                                               "note": "e4m3 + one fp32 scale per 128 elements; not part of the step"}
     if gate_us is not None:
         gb = wl.T * wl.E * 4 + wl.T * wl.K * 8
         kernels["moe_gate_topk"] = {"us": gate_us, "bytes": gb, "GBps": gb / gate_us / 1e3,

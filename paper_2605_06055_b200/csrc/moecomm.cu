@@ -416,9 +416,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   auto opt_in = [&](auto kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess;
   };
-  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<3, 16, true>) &&
-       opt_in(dispatch_quant_kernel<3, 32, true>) &&
-       opt_in(dispatch_quant_kernel<3, 16, false>) &&
+  ok = ok && opt_in(dispatch_bulk_kernel) && opt_in(dispatch_quant_kernel<3, 32, true>) &&
        opt_in(dispatch_quant_kernel<3, 32, false>) &&
        opt_in(dispatch_quant_kernel<2, 0, false>) && opt_in(dispatch_quant_kernel<3, 0, false>) &&
        opt_in(dispatch_quant_kernel<2, 0, false, true>) && opt_in(dispatch_quant_kernel<3, 0, false, true>) &&
@@ -844,16 +842,19 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   // A large job: every warp of the two-stage ring would see eight rows or more.
   const bool large = ring_warps(3) >= 1 && (int64_t)ctx->T >= (int64_t)8 * grid * ring_warps(2);
   // Rows short enough for registers take the register kernel (a load buffer and a code buffer per warp, the group
-  // scales and reciprocals behind the codes) when the job is small or the scales are group-wise: more rows in
-  // flight per SM is what both need.  Large row-wise jobs stay on the three-stage ring, which runs at the copy rate
-  // with five to nine warps; the register kernel with ten warps or more dropped to 0.74 of that at 8 KB rows
-  // (T=65536: 237 against 175 us).  Measured, register kernel against ring: decode shape 31.9 against 33.8 us
-  // row-wise and 40.0 against 44.1 us group-wise; group-wise at 32768 rows of 14 KB 398 against 419 us.
-  if (cpl > 0 && (grouped || !large)) {
+  // scales and reciprocals behind the codes): more rows in flight per SM.  Only large row-wise jobs of rows beyond
+  // 8 KB stay on the three-stage ring, which runs them at the copy rate with five warps (32768 rows of 14 KB: 371
+  // against 376 us).  Measured, register kernel against ring: decode shape 31.9 against 33.8 us row-wise and 33.8
+  // against 44.1 us group-wise; 65536 rows of 4 KB 170 against 203 us; 65536 rows of 8 KB 179 against 176 us.
+  // Warps per CTA: as many as fit, but for large jobs of short rows at most 9.  At 65536 rows of 8 KB ten or eleven
+  // warps reach 169-172 us in one run and 237-240 us (the rate of six warps) in the next, and twelve or more are
+  // always at 237-240: past about 2700 window rows being written at once HBM serves the writes badly (the bulk-copy
+  // dispatch bounds its warps for the same reason), and where exactly that sets in changes from run to run.
+  if (cpl == 16 || (cpl == 32 && (grouped || !large))) {
     const int sc_bytes = grouped ? ((H / QUANT_GROUP) * 4 + 15) / 16 * 16 : 0;
     const int per_warp = stage + (H + 2 * sc_bytes + 127) / 128 * 128 + 8;
     int warps = QUANT_SMEM_BUDGET / per_warp;
-    const int cap = cpl == 32 ? QUANT_REG_WARPS_LONG : QUANT_REG_WARPS_SHORT;
+    const int cap = cpl == 32 ? QUANT_REG_WARPS_LONG : large ? QUANT_REG_WARPS_SHORT_LARGE_JOB : QUANT_REG_WARPS_SHORT;
     if (warps > cap) warps = cap;
     // the fewest warps that still finish in the same number of rounds (14 rows per SM: 7 warps, not 10)
     const int64_t rounds = rows_per_sm < 1 ? 1 : (rows_per_sm + warps - 1) / warps;
@@ -889,8 +890,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   if (grouped) {   // rows beyond 16 KB
     stages == 3 ? launch(dispatch_quant_kernel<3, 0, false, true>) : launch(dispatch_quant_kernel<2, 0, false, true>);
   } else if (stages == 3) {
-    if (cpl == 16) whole_slabs ? launch(dispatch_quant_kernel<3, 16, true>) : launch(dispatch_quant_kernel<3, 16, false>);
-    else if (cpl == 32) whole_slabs ? launch(dispatch_quant_kernel<3, 32, true>) : launch(dispatch_quant_kernel<3, 32, false>);
+    if (cpl == 32) whole_slabs ? launch(dispatch_quant_kernel<3, 32, true>) : launch(dispatch_quant_kernel<3, 32, false>);
     else launch(dispatch_quant_kernel<3, 0, false>);
   } else {   // (rows beyond 16 KB only: shorter rows of small jobs went to the register kernel)
     launch(dispatch_quant_kernel<2, 0, false>);

@@ -38,6 +38,7 @@ constexpr int QUANT_MAX_ROW_BYTES = 32 * 1024;
 constexpr int QUANT_MAX_WARPS = 16;
 constexpr int QUANT_REG_WARPS_LONG = 10;        // register kernel, rows beyond 8 KB: 204 registers per thread at most
 constexpr int QUANT_REG_WARPS_SHORT = 14;       // register kernel, rows up to 8 KB (16 warps measured slower than 14)
+constexpr int QUANT_REG_WARPS_SHORT_LARGE_JOB = 9;
 constexpr int QUANT_SMEM_BUDGET = 220 * 1024;   // shared memory the warps' rings may fill
 constexpr int QUANT_GROUP = 128;                 // elements per scale of the group-wise form
 constexpr int QUANT_MAX_GROUPS = QUANT_MAX_ROW_BYTES / 2 / QUANT_GROUP;
@@ -319,7 +320,6 @@ dispatch_quant_reg_kernel(const unsigned char* __restrict__ X, unsigned char* __
   const uint32_t in = smem_addr(smem) + warp * l_stride;
   const uint32_t out = smem_addr(smem) + n_warps * l_stride + warp * c_stride;
   const uint32_t bar = smem_addr(smem) + n_warps * (l_stride + c_stride) + warp * 8;
-  const unsigned half_mask = lane < 16 ? 0x0000ffffu : 0xffff0000u;
   int half;   // lane >> 4 through an opaque instruction (see dispatch_quant_kernel)
   asm("shr.u32 %0, %1, 4;" : "=r"(half) : "r"(lane));
 
@@ -385,24 +385,64 @@ dispatch_quant_reg_kernel(const unsigned char* __restrict__ X, unsigned char* __
     float scale = 1.0f, inv = 1.0f;
     if constexpr (GROUPED) {
       const uint32_t sc = out + code_bytes, rc = sc + sc_bytes;
-      if (lane == 0) bulk_wait_read<0>();   // the previous row's stores have read the code buffer
-      __syncwarp();
-      // group maxima: one half-warp reduction per chunk (its sixteen lanes store the same word)
+      // Group maxima.  Chunk k of a lane belongs to group 2k + half, whose other fifteen chunks sit in the other
+      // lanes of the half-warp.  (A sub-warp redux per chunk compiles into a 35-instruction collective: 1000
+      // instructions per 14 KB row.)  Instead the maxima of chunks 2i and 2i+1 share a word, and a transposing
+      // butterfly -- at every step a lane hands half of its words to its partner and reduces the other half with
+      // what it receives -- leaves lane l of each half-warp with the finished maxima of one word: 15 shuffles and
+      // packed maxima for 32 chunks.  That lane turns them into scale and reciprocal, so the divisions of all the
+      // row's groups run side by side.
+      constexpr int P = CPL / 2;   // words per lane: 16 or 8
+      uint32_t w[P];
 #pragma unroll
-      for (int k = 0; k < CPL; ++k)
-        if (mine(k)) {
-          const uint32_t m2 = __vmaxu2(__vmaxu2(v[k].x & 0x7fff7fffu, v[k].y & 0x7fff7fffu),
-                                       __vmaxu2(v[k].z & 0x7fff7fffu, v[k].w & 0x7fff7fffu));
-          const uint32_t mbits = __reduce_max_sync(half_mask, max(m2 & 0xffffu, m2 >> 16));
-          sts_f32(sc + 4 * (2 * k + half), __uint_as_float(mbits << 16));
+      for (int i = 0; i < P; ++i) {
+        uint32_t e = 0u, o = 0u;   // per-halfword maxima of chunk 2i and of chunk 2i+1
+        if (mine(2 * i))
+          e = __vmaxu2(__vmaxu2(v[2 * i].x & 0x7fff7fffu, v[2 * i].y & 0x7fff7fffu),
+                       __vmaxu2(v[2 * i].z & 0x7fff7fffu, v[2 * i].w & 0x7fff7fffu));
+        if (mine(2 * i + 1))
+          o = __vmaxu2(__vmaxu2(v[2 * i + 1].x & 0x7fff7fffu, v[2 * i + 1].y & 0x7fff7fffu),
+                       __vmaxu2(v[2 * i + 1].z & 0x7fff7fffu, v[2 * i + 1].w & 0x7fff7fffu));
+        // (max of e's halves, max of o's halves)
+        w[i] = __vmaxu2(__byte_perm(e, o, 0x5410), __byte_perm(e, o, 0x7632));
+      }
+      if (lane == 0) bulk_wait_read<0>();   // the previous row's stores have read the code buffer (the shuffles
+                                            // below keep every other lane behind this wait)
+      int held = P;
+#pragma unroll
+      for (int bit = 8; bit >= 1; bit >>= 1) {
+        const bool up = (lane & bit) != 0;
+        if (held > 1) {
+          held >>= 1;
+#pragma unroll
+          for (int j = 0; j < P / 2; ++j)
+            if (j < held) {
+              const uint32_t send = up ? w[j] : w[j + held];
+              const uint32_t keep = up ? w[j + held] : w[j];
+              w[j] = __vmaxu2(keep, __shfl_xor_sync(0xffffffffu, send, bit));
+            }
+        } else {   // one word left (rows of at most 8 KB): both partners finish with the same word
+          w[0] = __vmaxu2(w[0], __shfl_xor_sync(0xffffffffu, w[0], bit));
         }
-      __syncwarp();   // every reduction has consumed every lane's chunk: the load buffer is free
+      }
+      // every lane has handed over all of its chunks' maxima: the load buffer is free
       if (lane == 0 && q1 < a.n_items) issue_load(q1);
-      for (int g = lane; g < n_groups; g += 32) {   // lane g: scale and reciprocal of group g
-        const float amax = lds_f32(sc + 4 * g);
-        const float den = amax > 0.0f ? amax : 448.0f;   // an all-zero group: scale and reciprocal 1
-        sts_f32(sc + 4 * g, __fdiv_rn(den, 448.0f));
-        sts_f32(rc + 4 * g, __fdiv_rn(448.0f, den));
+      {
+        // P == 16: lane l of a half-warp holds word l = chunks 2l and 2l+1; P == 8: word l >> 1, of which it takes
+        // chunk 2 (l >> 1) + (l & 1)
+        const int l = lane & 15;
+#pragma unroll
+        for (int part = 0; part < (P == 16 ? 2 : 1); ++part) {
+          const int k = P == 16 ? 2 * l + part : l;
+          const uint32_t bits = (P == 16 ? part : (l & 1)) ? (w[0] >> 16) : (w[0] & 0xffffu);
+          const int g = 2 * k + half;
+          if (g < n_groups) {
+            const float amax = __uint_as_float(bits << 16);
+            const float den = amax > 0.0f ? amax : 448.0f;   // an all-zero group: scale and reciprocal 1
+            sts_f32(sc + 4 * g, __fdiv_rn(den, 448.0f));
+            sts_f32(rc + 4 * g, __fdiv_rn(448.0f, den));
+          }
+        }
       }
       __syncwarp();
 #pragma unroll
