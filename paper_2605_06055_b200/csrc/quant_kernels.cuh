@@ -1,6 +1,6 @@
-// Row-wise quantised dispatch: bf16 rows in, fp8 e4m3 codes + one fp32 scale per
-// row out, written straight into the destination expert windows and a parallel
-// scale tensor in the same row order (Section 5.2, Prefill Dispatch).
+// Quantised dispatch: bf16 rows in, fp8 e4m3 codes + fp32 scales out, written
+// straight into the destination expert windows and a parallel scale tensor in
+// the same row order (Section 5.2, Prefill Dispatch).
 //
 // Format (the paper names none; this is the library's definition):
 //   amax  = max_h |x[h]|                         (inputs are finite)
@@ -9,20 +9,21 @@
 // Each token is quantised once; its K branches receive the same code row and scale.
 // Group-wise form (GROUPED): the same rule applied to every group of 128 consecutive elements of a row on its
 // own -- H / 128 scales per row, [rows, H / 128] fp32 in the same row order.  A group is the 16 chunks of 16 bytes
-// that one half-warp reads side by side, so its maximum is one half-warp reduction.
+// that one half-warp reads side by side.
 //
-// Structure: the bulk-copy ring of dispatch_bulk_kernel with a compute step in
-// the middle.  A stage holds one whole row (needed for amax).  Lane 0 loads the
-// row with cp.async.bulk; the warp reduces amax from shared memory and converts
-// the row IN PLACE (codes are half as wide as the values, so the code of chunk c
-// lands on bytes that chunks <= c/2 occupied and have already been read); lane 0
-// stores the code row K times with cp.async.bulk while lanes j < K store the
-// scale.  X is read from HBM once and only H + 4 bytes per branch are written.
-//
-// What bounds the kernel at decode sizes is the latency of one warp walking its
-// row, so the number of rows in flight per SM matters: a stage without a
-// separate code buffer lets seven warps (instead of four or five) share an SM
-// at 14 KB rows.
+// Two kernels.  Both load a whole row (needed for amax) into shared memory with one cp.async.bulk, store the code
+// row K times with cp.async.bulk, read X from HBM once and write only H + 4 bytes (group-wise: H + H/32) per
+// branch; what bounds them below the copy rate is the latency of one warp walking its row, so the number of rows
+// in flight per SM -- the number of warps shared memory admits -- is what counts.
+//   dispatch_quant_reg_kernel  rows of at most 16 KB, held in registers: a load buffer (2H bytes) and a code
+//                              buffer (H bytes) per warp; the next row's load is issued as soon as the current
+//                              row is in registers.  3H bytes per warp.
+//   dispatch_quant_kernel      a ring of two or three whole-row stages per warp, the codes written IN PLACE over
+//                              the first half of the row's stage (they are half as wide, so the code of chunk c
+//                              lands on bytes that chunks <= c/2 occupied and have already been read).  4H or 6H
+//                              bytes per warp.  Kept for large row-wise jobs of rows beyond 8 KB (two loads in
+//                              flight per warp, five warps: the copy rate at 14 KB rows) and, in a two-pass form
+//                              that needs no registers for the row, for rows beyond 16 KB.
 #pragma once
 
 #include <cuda_fp8.h>
@@ -31,9 +32,7 @@
 
 namespace moe {
 
-// Stages per warp: 2 for small batches (more warps, i.e. more rows in flight per SM, is what counts
-// when every warp sees only a few rows), 3 for large ones (two loads in flight per warp).  Measured:
-// decode shape (T=2048, 14 KB rows) 30.8 vs 32.7 us; T=65536 with 8 KB rows 235 vs 182 us.
+// Ring kernel, stages per warp: 3 for large jobs (two loads in flight per warp), 2 otherwise.
 constexpr int QUANT_MAX_ROW_BYTES = 32 * 1024;
 constexpr int QUANT_MAX_WARPS = 16;
 constexpr int QUANT_REG_WARPS_LONG = 10;        // register kernel, rows beyond 8 KB: 204 registers per thread at most
