@@ -3,7 +3,8 @@ whole tensor: every integer the plan produces, every byte of the expert windows 
 and their canaries included), and every element of the combined output with a non-trivial expert stand-in
 (per-expert scaling) between dispatch and combine.  Covers configs 3 and 4, config 5 at T = 65536 under both
 schedules (the large-job combine with two branches), the top-7 shape of the benchmark (the large-job combine of
-the any-K family) and the row-wise quantised dispatch at config 3 (its three-stage form).
+the any-K family) and the quantised dispatch at config 3, row-wise (the three-stage ring) and with one scale per
+128 elements (the register kernel).
 
 The oracle runs token-parallel over all host cores (about half a second per pass at config 3); its windows are
 uploaded in chunks and compared on the device.
@@ -158,6 +159,40 @@ def test_full_size_quantised_dispatch_codes_and_scales():
     wq2 = torch.full_like(wq, 0xAB)
     sc2 = torch.full_like(sc, -1.0)
     comm.moe_plan_dispatch_quant(wl.schedule, idx, X, wq2, sc2, C)
+    assert comm.moe_status() == 0
+    assert torch.equal(wq2, wq) and torch.equal(sc2.view(torch.int32), sc.view(torch.int32))
+    comm.close()
+
+
+def test_full_size_group_quantised_dispatch_codes_and_scales():
+    """One scale per 128 elements at config 3 (the register kernel with ten warps per SM): every e4m3 code and
+    every one of the 56 fp32 scales of every window row, bit-exact against the oracle; padding rows keep their fill."""
+    dev = torch.device("cuda:0")
+    wl = synth.config(3)
+    G = wl.H // 128
+    inp = synth.make_inputs(wl)
+    idx_np = inp.topk_idx.numpy()
+    p = oracle.plan(idx_np, wl.E, wl.R)
+    C = (int(p.n_recv.max()) + 7) // 8 * 8
+    st, slots = oracle.slots(idx_np, wl.E, wl.R, p, C)
+    assert st == oracle.OK
+    want_q = np.full((wl.R * C, wl.H), 0xAB, np.uint8)
+    want_s = np.full((wl.R * C, G), -1.0, np.float32)
+    assert oracle.dispatch_quant_group(synth.bf16_to_u16(inp.X), slots, want_q, want_s, 128, CORES) == oracle.OK
+
+    comm = binding.MoeComm(wl.T, wl.H, wl.E, wl.R, wl.K, dev)
+    X, idx = inp.X.to(dev), inp.topk_idx.to(dev)
+    wq = torch.full((wl.R * C, wl.H), 0xAB, dtype=torch.uint8, device=dev)
+    sc = torch.full((wl.R * C, G), -1.0, dtype=torch.float32, device=dev)
+    comm.moe_plan(wl.schedule, idx)
+    comm.moe_dispatch_quant_group(X, wq, sc, C)
+    assert comm.moe_status() == 0
+    assert device_equals_host(wq, want_q)
+    assert device_equals_host(sc.view(torch.int32), want_s.view(np.int32))
+    # the chained form gives the same bytes
+    wq2 = torch.full_like(wq, 0xAB)
+    sc2 = torch.full_like(sc, -1.0)
+    comm.moe_plan_dispatch_quant_group(wl.schedule, idx, X, wq2, sc2, C)
     assert comm.moe_status() == 0
     assert torch.equal(wq2, wq) and torch.equal(sc2.view(torch.int32), sc.view(torch.int32))
     comm.close()
