@@ -280,8 +280,9 @@ moe_status_t moe_dispatch_quant_peers(moe_ctx_t* ctx, const void* x /*DEVICE*/,
  *                       MOE_ERR_STALE_PEERS otherwise.
  *   moe_dispatch_cached / moe_combine_cached / moe_dispatch_quant_cached
  *                       as moe_dispatch_peers / moe_combine_peers / moe_dispatch_quant_peers with the installed
- *                       table and its capacity (the quantised form needs windows exported with MOE_WINDOW_QUANT:
- *                       codes and scales land in the parts of every rank's allocation that flag reserves).
+ *                       table and its capacity (the quantised forms need windows exported with MOE_WINDOW_QUANT
+ *                       or MOE_WINDOW_QUANT_GROUP: codes and scales land in the parts of every rank's allocation
+ *                       that flag reserves).
  *                       `generations` as in moe_peers_check (NULL: no test); with a stale or missing table they
  *                       return MOE_ERR_STALE_PEERS and enqueue nothing -- no stale address is ever dereferenced.
  *   moe_peers_close     synchronises `stream`, releases the mappings of moe_peers_open and forgets the table
@@ -303,6 +304,9 @@ typedef struct {
 #define MOE_WINDOW_STATE 1 /* the state region of the device-side phase order (moe_signal_peers), zeroed once   */
 #define MOE_WINDOW_QUANT 2 /* the e4m3 code window [capacity_rows, H] uint8 and the scale tensor [capacity_rows]
                               fp32 of the row-wise quantised dispatch (moe_dispatch_quant_cached)               */
+#define MOE_WINDOW_QUANT_GROUP 4 /* the code window and the scale tensor [capacity_rows, H / 128] fp32 of the
+                              group-wise quantised dispatch (moe_dispatch_quant_group_cached); not together with
+                              MOE_WINDOW_QUANT, and H % 128 == 0                                                */
 moe_status_t moe_window_export(const void* window /*DEVICE*/, int64_t bytes, int32_t generation, int32_t flags,
                                moe_window_handle_t* out /*HOST*/);
 moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles /*HOST [R]*/, int32_t my_rank,
@@ -317,6 +321,10 @@ moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations /*HOS
                                 const float* topk_w /*DEVICE*/, void* y /*DEVICE*/, void* stream);
 moe_status_t moe_dispatch_quant_cached(moe_ctx_t* ctx, const void* x /*DEVICE*/,
                                        const int32_t* generations /*HOST or NULL*/, void* stream);
+/* moe_dispatch_quant_group through the installed table: windows exported with MOE_WINDOW_QUANT_GROUP. */
+moe_status_t moe_dispatch_quant_group_cached(moe_ctx_t* ctx, const void* x /*DEVICE*/,
+                                             const int32_t* generations /*HOST or NULL*/, int32_t group_size,
+                                             void* stream);
 moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
 
 /* Synchronisation metadata in the pooled memory (Section 3.2: every rank's slice carries communicator state

@@ -30,9 +30,10 @@ EXPORTS = [
     "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
     "moe_dispatch_cached", "moe_combine_cached", "moe_state_bytes", "moe_window_bytes", "moe_signal_peers",
     "moe_wait_peers", "moe_dispatch_quant_cached", "moe_dispatch_quant_group", "moe_plan_dispatch_quant_group",
+    "moe_dispatch_quant_group_cached",
 ]
 MOE_SYNC_SLOTS = 4
-MOE_WINDOW_STATE, MOE_WINDOW_QUANT = 1, 2
+MOE_WINDOW_STATE, MOE_WINDOW_QUANT, MOE_WINDOW_QUANT_GROUP = 1, 2, 4
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -118,6 +119,8 @@ def load() -> ctypes.CDLL:
     L.moe_window_export.argtypes = [vp, i64, i32, i32, ctypes.POINTER(MoeWindowHandle)]
     L.moe_dispatch_quant_cached.argtypes = [vp, vp, vp, vp]
     L.moe_dispatch_quant_cached.restype = ctypes.c_int
+    L.moe_dispatch_quant_group_cached.argtypes = [vp, vp, vp, i32, vp]
+    L.moe_dispatch_quant_group_cached.restype = ctypes.c_int
     L.moe_peers_open.argtypes = [vp, vp, i32, vp, i64, vp]
     L.moe_peers_set.argtypes = [vp, vp, vp, i32, i64, i32, vp]
     L.moe_state_bytes.argtypes = [i32]
@@ -457,6 +460,16 @@ class MoeComm:
                                                     _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_dispatch_quant_cached")
+        return rc
+
+    def moe_dispatch_quant_group_cached(self, x: torch.Tensor, generations=None, group_size: int = 128, stream=None,
+                                        check: bool = True) -> int:
+        gens = None if generations is None else np.ascontiguousarray(generations, dtype=np.int32)
+        with self._on_device():
+            rc = self.lib.moe_dispatch_quant_group_cached(self._h, _dev_ptr(x, torch.bfloat16), _host_ptr(gens),
+                                                          int(group_size), _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_dispatch_quant_group_cached")
         return rc
 
     def moe_signal_peers(self, slot: int, epoch: int, stream=None, check: bool = True) -> int:

@@ -57,7 +57,8 @@ struct moe_ctx {
   int64_t peer_capacity;
   bool peers_installed;
   bool peers_have_state;              // every installed window is followed by its state region
-  bool peers_have_quant;              // ... and by a code window and a scale tensor
+  bool peers_have_quant;              // ... and by a code window and a scale tensor (one scale per row)
+  bool peers_have_quant_group;        // ... or by a code window and a tensor of group scales
   unsigned char** code_table;         // device, [R]: e4m3 code window of every rank
   float** scale_table;                // device, [R]: scale tensor of every rank
   int32_t my_rank;                    // this process's rank in the installed table
@@ -379,6 +380,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->scale_table = reinterpret_cast<float**>(ctx->code_table + shape->R);
   ctx->peers_have_state = false;
   ctx->peers_have_quant = false;
+  ctx->peers_have_quant_group = false;
   ctx->my_rank = 0;
   ctx->peer_capacity = 0;
   for (int d = 0; d < MOE_MAX_R; ++d) {
@@ -1082,11 +1084,22 @@ WindowParts window_parts(const moe_shape_t& sh, int64_t capacity_rows, int32_t f
   p.state = at;
   if (flags & MOE_WINDOW_STATE) at += state_bytes_for(sh.R);
   p.codes = at;
-  if (flags & MOE_WINDOW_QUANT) at += align_up((size_t)capacity_rows * sh.H);
+  if (flags & (MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP)) at += align_up((size_t)capacity_rows * sh.H);
   p.scales = at;
   if (flags & MOE_WINDOW_QUANT) at += align_up((size_t)capacity_rows * sizeof(float));
+  if (flags & MOE_WINDOW_QUANT_GROUP) at += align_up((size_t)capacity_rows * (sh.H / QUANT_GROUP) * sizeof(float));
   p.total = at;
   return p;
+}
+
+// Known bits only, and at most one form of quantised parts.
+bool window_flags_ok(int32_t flags) {
+  if ((flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP)) != 0) return false;
+  return (flags & MOE_WINDOW_QUANT) == 0 || (flags & MOE_WINDOW_QUANT_GROUP) == 0;
+}
+// ... and a shape the group-wise parts exist for.
+bool window_flags_fit(int32_t flags, const moe_shape_t& sh) {
+  return window_flags_ok(flags) && ((flags & MOE_WINDOW_QUANT_GROUP) == 0 || sh.H % QUANT_GROUP == 0);
 }
 
 // Copies the addresses of every rank's rows, state region, code window and scale tensor to the device tables on
@@ -1099,8 +1112,9 @@ moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows,
     char* base = static_cast<char*>(ctx->peer_ptr[d]);
     all[d] = base;
     all[R + d] = (flags & MOE_WINDOW_STATE) ? base + parts.state : nullptr;
-    all[2 * R + d] = (flags & MOE_WINDOW_QUANT) ? base + parts.codes : nullptr;
-    all[3 * R + d] = (flags & MOE_WINDOW_QUANT) ? base + parts.scales : nullptr;
+    const bool quant = (flags & (MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP)) != 0;
+    all[2 * R + d] = quant ? base + parts.codes : nullptr;
+    all[3 * R + d] = quant ? base + parts.scales : nullptr;
   }
   // pageable source: the runtime has staged the bytes by the time the call returns
   if (cudaMemcpyAsync(ctx->peer_table, all, sizeof(void*) * 4 * R, cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -1109,6 +1123,7 @@ moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows,
   ctx->my_rank = my_rank;
   ctx->peers_have_state = (flags & MOE_WINDOW_STATE) != 0;
   ctx->peers_have_quant = (flags & MOE_WINDOW_QUANT) != 0;
+  ctx->peers_have_quant_group = (flags & MOE_WINDOW_QUANT_GROUP) != 0;
   ctx->peers_installed = true;
   return MOE_OK;
 }
@@ -1125,8 +1140,7 @@ moe_status_t table_fresh(const moe_ctx* ctx, const int32_t* generations) {
 
 moe_status_t moe_window_export(const void* window, int64_t bytes, int32_t generation, int32_t flags,
                                moe_window_handle_t* out) {
-  if (window == nullptr || out == nullptr || bytes <= 0 || !aligned16(window) ||
-      (flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0)
+  if (window == nullptr || out == nullptr || bytes <= 0 || !aligned16(window) || !window_flags_ok(flags))
     return MOE_ERR_INVALID_ARG;
   static_assert(sizeof(cudaIpcMemHandle_t) == sizeof(out->ipc), "handle size");
   uintptr_t base = 0;
@@ -1156,7 +1170,7 @@ moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, 
     return MOE_ERR_INVALID_ARG;
   // every rank exports the same parts, and enough bytes for them at this capacity
   const int32_t flags = handles[my_rank].flags;
-  if ((flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0) return MOE_ERR_INVALID_ARG;
+  if (!window_flags_fit(flags, ctx->shape)) return MOE_ERR_INVALID_ARG;
   const int64_t need = (int64_t)window_parts(ctx->shape, capacity_rows, flags).total;
   for (int d = 0; d < ctx->shape.R; ++d)
     if (handles[d].flags != flags || handles[d].bytes < need || (handles[d].offset & 15) != 0) return MOE_ERR_INVALID_ARG;
@@ -1186,7 +1200,7 @@ moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles, 
 moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, const int32_t* generations, int32_t my_rank,
                            int64_t capacity_rows, int32_t flags, void* stream) {
   if (ctx == nullptr || window_bases == nullptr || capacity_rows < 0 || my_rank < 0 || my_rank >= ctx->shape.R ||
-      (flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0)
+      !window_flags_fit(flags, ctx->shape))
     return MOE_ERR_INVALID_ARG;
   for (int d = 0; d < ctx->shape.R; ++d)
     if (window_bases[d] == nullptr || !aligned16(window_bases[d])) return MOE_ERR_INVALID_ARG;
@@ -1203,7 +1217,7 @@ moe_status_t moe_peers_set(moe_ctx_t* ctx, const void* const* window_bases, cons
 size_t moe_state_bytes(int32_t R) { return (R < 1 || R > MOE_MAX_R) ? 0 : state_bytes_for(R); }
 
 size_t moe_window_bytes(const moe_shape_t* shape, int64_t capacity_rows, int32_t flags) {
-  if (!shape_valid(shape) || capacity_rows < 0 || (flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT)) != 0) return 0;
+  if (!shape_valid(shape) || capacity_rows < 0 || !window_flags_fit(flags, *shape)) return 0;
   return window_parts(*shape, capacity_rows, flags).total;
 }
 
@@ -1253,6 +1267,16 @@ moe_status_t moe_dispatch_quant_cached(moe_ctx_t* ctx, const void* x, const int3
   if (!ctx->peers_have_quant) return MOE_ERR_STALE_PEERS;   // the installed windows reserve no room for codes and scales
   return dispatch_quant_impl(ctx, x, nullptr, nullptr, ctx->peer_capacity, stream, false,
                              reinterpret_cast<const void* const*>(ctx->code_table), ctx->scale_table);
+}
+
+moe_status_t moe_dispatch_quant_group_cached(moe_ctx_t* ctx, const void* x, const int32_t* generations,
+                                             int32_t group_size, void* stream) {
+  if (ctx == nullptr || group_size != QUANT_GROUP) return MOE_ERR_INVALID_ARG;
+  const moe_status_t fresh = table_fresh(ctx, generations);
+  if (fresh != MOE_OK) return fresh;
+  if (!ctx->peers_have_quant_group) return MOE_ERR_STALE_PEERS;   // no room for codes and group scales in the installed windows
+  return dispatch_quant_impl(ctx, x, nullptr, nullptr, ctx->peer_capacity, stream, false,
+                             reinterpret_cast<const void* const*>(ctx->code_table), ctx->scale_table, group_size);
 }
 
 moe_status_t moe_combine_cached(moe_ctx_t* ctx, const int32_t* generations, const float* topk_w, void* y, void* stream) {

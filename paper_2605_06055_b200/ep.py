@@ -104,25 +104,31 @@ class EpRank:
         self.handshakes = 0
 
     # -- windows -------------------------------------------------------------------------------------
-    def new_window(self, capacity_rows: int, quant: bool = False) -> torch.Tensor:
-        """Allocates this rank's window with its state region behind the rows (zeroed) and, with quant=True, the code
-        window and scale tensor of the quantised dispatch behind that; attaches it and returns the
-        [capacity_rows, H] view of the rows."""
-        flags = binding.MOE_WINDOW_STATE | (binding.MOE_WINDOW_QUANT if quant else 0)
+    def new_window(self, capacity_rows: int, quant: bool = False, quant_group: bool = False) -> torch.Tensor:
+        """Allocates this rank's window with its state region behind the rows (zeroed) and, with quant=True
+        (one scale per row) or quant_group=True (one per 128 elements), the code window and scale tensor of the
+        quantised dispatch behind that; attaches it and returns the [capacity_rows, H] view of the rows."""
+        assert not (quant and quant_group)
+        flags = binding.MOE_WINDOW_STATE | (binding.MOE_WINDOW_QUANT if quant else 0) | \
+            (binding.MOE_WINDOW_QUANT_GROUP if quant_group else 0)
         nbytes = self.comm.moe_window_bytes(capacity_rows, flags)
         backing = torch.zeros(nbytes // 2, dtype=torch.bfloat16, device=self.device)
         self.attach_window(backing, capacity_rows, flags)
         return backing[:capacity_rows * self.H].view(capacity_rows, self.H)
 
     def quant_views(self):
-        """(codes [capacity_rows, H] uint8, scales [capacity_rows] fp32) of this rank's window allocation."""
-        assert self.flags & binding.MOE_WINDOW_QUANT
+        """(codes [capacity_rows, H] uint8, scales fp32) of this rank's window allocation; scales are [capacity_rows]
+        with MOE_WINDOW_QUANT, [capacity_rows, H // 128] with MOE_WINDOW_QUANT_GROUP."""
+        assert self.flags & (binding.MOE_WINDOW_QUANT | binding.MOE_WINDOW_QUANT_GROUP)
+        per_row = self.H // 128 if self.flags & binding.MOE_WINDOW_QUANT_GROUP else 1
         raw = self.window.view(torch.uint8)
-        scales_at = self.comm.moe_window_bytes(self.capacity, self.flags) - (self.capacity * 4 + 255) // 256 * 256
+        scale_bytes = self.capacity * per_row * 4
+        scales_at = self.comm.moe_window_bytes(self.capacity, self.flags) - (scale_bytes + 255) // 256 * 256
         codes_at = scales_at - (self.capacity * self.H + 255) // 256 * 256
         codes = raw[codes_at:codes_at + self.capacity * self.H].view(self.capacity, self.H)
-        scales = raw[scales_at:scales_at + self.capacity * 4].view(torch.float32)
-        return codes, scales
+        scales = raw[scales_at:scales_at + scale_bytes].view(torch.float32)
+        return codes, (scales.view(self.capacity, per_row) if per_row > 1 or self.flags & binding.MOE_WINDOW_QUANT_GROUP
+                       else scales)
 
     def attach_window(self, window: torch.Tensor, capacity_rows: int, flags: int = 0) -> None:
         """This rank's window from now on: a contiguous bf16 tensor whose first capacity_rows * H elements are the
@@ -220,18 +226,23 @@ class EpRank:
             self.comm.moe_combine_cached(self.announced, topk_w_local, y_local)
 
     def dispatch_quant(self, x_local: torch.Tensor) -> None:
-        """Row-wise quantised dispatch: e4m3 codes into every rank's code window, one fp32 scale per row into every
-        rank's scale tensor -- the parts of the window allocations that MOE_WINDOW_QUANT reserves, reached through
-        the same address table as the rows.  Returns once this rank's experts may read its codes."""
+        """Quantised dispatch: e4m3 codes into every rank's code window, fp32 scales (one per row, or one per 128
+        elements if the windows were made with quant_group) into every rank's scale tensor -- the parts of the
+        window allocations that MOE_WINDOW_QUANT / MOE_WINDOW_QUANT_GROUP reserve, reached through the same address
+        table as the rows.  Returns once this rank's experts may read its codes."""
         self._ensure_addresses()
+        if self.flags & binding.MOE_WINDOW_QUANT_GROUP:
+            call = lambda: self.comm.moe_dispatch_quant_group_cached(x_local, self.announced)
+        else:
+            call = lambda: self.comm.moe_dispatch_quant_cached(x_local, self.announced)
         if self.sync == "device":
             self.epoch += 1
             if self.epoch > 1:
                 self.comm.moe_wait_peers(self.SLOT_COMBINED, self.epoch - 1)
-            self.comm.moe_dispatch_quant_cached(x_local, self.announced)
+            call()
             self._signal_then_wait(self.SLOT_DISPATCHED)
         else:
-            self.comm.moe_dispatch_quant_cached(x_local, self.announced)
+            call()
             self._host_barrier()
 
     def status(self) -> int:

@@ -76,7 +76,12 @@ def test_window_and_state_sizes_host_logic(lib):
         up(rows) + up(1300 * 7168) + up(1300 * 4)
     assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT) == \
         up(rows) + 256 + up(1300 * 7168) + up(1300 * 4)
-    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 4) == 0                       # unknown flag
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT_GROUP) == \
+        up(rows) + 256 + up(1300 * 7168) + up(1300 * 56 * 4)                           # one scale per 128 elements
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_QUANT | binding.MOE_WINDOW_QUANT_GROUP) == 0
+    odd = binding.MoeShape(2048, 7168 + 64, 256, 16, 8)                                # H % 128 != 0: no group-wise parts
+    assert lib.moe_window_bytes(ctypes.byref(odd), 1300, binding.MOE_WINDOW_QUANT_GROUP) == 0
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 8) == 0                       # unknown flag
     assert lib.moe_window_bytes(ctypes.byref(shape), -1, 1) == 0 and lib.moe_window_bytes(None, 8, 1) == 0
     assert ctypes.sizeof(binding.MoeWindowHandle) == 96
     # calls that need a context reject a missing one before touching anything

@@ -184,6 +184,62 @@ def test_installed_address_table_and_generation_stamp_in_one_process():
         c.close()
 
 
+@pytest.mark.parametrize("case", [c for c in CASES if c[2] % 128 == 0], ids=[c[0] for c in CASES if c[2] % 128 == 0])
+def test_group_quantised_dispatch_through_the_installed_table(case):
+    """Windows made with MOE_WINDOW_QUANT_GROUP: every rank's codes and its [C, H/128] group scales land in the
+    parts of its allocation that the flag reserves, bit-identical to the oracle's single global result; the sizes
+    and flags the library accepts are the documented ones."""
+    name, T, H, E, R, K, sch, routing, per = case
+    dev = torch.device("cuda:0")
+    G = H // 128
+    wl = Workload(name, T, H, E, R, K, sch, routing, "identity", 7300 + T, rank_tokens=per)
+    inp = synth.make_inputs(wl)
+    rts = inp.rank_tok_start
+    p = oracle.plan(inp.topk_idx.numpy(), E, R, rts)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(inp.topk_idx.numpy(), E, R, p, C, rts)
+    want_q = np.full((R * C, H), 0, np.uint8)
+    want_s = np.full((R * C, G), 0.0, np.float32)
+    assert oracle.dispatch_quant_group(synth.bf16_to_u16(inp.X), slots, want_q, want_s, 128, 4) == oracle.OK
+
+    idx, X = inp.topk_idx.to(dev), inp.X.to(dev)
+    comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
+    counts = torch.zeros((R, E), dtype=torch.int32, device=dev)
+    for r, c in enumerate(comms):
+        c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, counts[r])
+    for c in comms:
+        c.moe_notify(counts)
+    FLAGS = binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT_GROUP
+    up = lambda n: (n + 255) // 256 * 256
+    total = comms[0].moe_window_bytes(C, FLAGS)
+    assert total == up(C * H * 2) + binding.moe_state_bytes(R) + up(C * H) + up(C * G * 4)
+    # both quantised forms at once, or an unknown bit, are refused (size 0)
+    assert comms[0].moe_window_bytes(C, FLAGS | binding.MOE_WINDOW_QUANT) == 0
+    assert comms[0].moe_window_bytes(C, 8) == 0
+    backings = [torch.zeros(total // 2, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+    bases = [b.data_ptr() for b in backings]
+    for r, c in enumerate(comms):
+        c.moe_peers_set(bases, None, C, my_rank=r, flags=FLAGS)
+    for r, c in enumerate(comms):
+        x_r = X[rts[r]:rts[r + 1]].contiguous()
+        # the row-wise call needs windows with row-wise parts
+        assert c.moe_dispatch_quant_cached(x_r, check=False) == binding.MOE_ERR_STALE_PEERS
+        assert c.moe_dispatch_quant_group_cached(x_r, group_size=64, check=False) == binding.MOE_ERR_INVALID_ARG
+        c.moe_dispatch_quant_group_cached(x_r)
+        assert c.moe_status() == 0
+    codes_at = up(C * H * 2) + binding.moe_state_bytes(R)
+    scales_at = codes_at + up(C * H)
+    got_q = np.concatenate([b.view(torch.uint8)[codes_at:codes_at + C * H].view(C, H).cpu().numpy() for b in backings])
+    got_s = np.concatenate([b.view(torch.uint8)[scales_at:scales_at + 4 * C * G].view(torch.float32).view(C, G).cpu().numpy()
+                            for b in backings])
+    assert np.array_equal(got_q, want_q) and np.array_equal(got_s.view(np.uint32), want_s.view(np.uint32))
+    # a table installed with the row-wise parts refuses the group-wise call
+    comms[0].moe_peers_set(bases, None, C, my_rank=0, flags=binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT)
+    assert comms[0].moe_dispatch_quant_group_cached(X[:int(rts[1])].contiguous(), check=False) == binding.MOE_ERR_STALE_PEERS
+    for c in comms:
+        c.close()
+
+
 def test_signals_and_bounded_waits_between_ranks_of_one_process():
     """The device-side phase order with every rank a context of this process (all on the one GPU, so every signal
     is enqueued before any wait): signals reach every rank's state region, waits pass once all R signals of the
@@ -319,7 +375,9 @@ def _ipc_rank(rank, world, port, mode, sync, results):
         # (rows first, then the zeroed state region of the device-side phase order)
         def new_window(offset_rows):
             backing = torch.zeros(12 << 20, dtype=torch.bfloat16, device=dev)
-            flags = binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_QUANT
+            # (the handshake mode carries the group-wise quantised parts, the other modes the row-wise ones)
+            flags = binding.MOE_WINDOW_STATE | (binding.MOE_WINDOW_QUANT_GROUP if mode == "handshake"
+                                                else binding.MOE_WINDOW_QUANT)
             flat = backing[offset_rows * H:offset_rows * H + me.comm.moe_window_bytes(C, flags) // 2]
             win = flat[:C * H].view(C, H)
             win.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
@@ -416,8 +474,12 @@ def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
     want = harness.oracle_run(inp, C)
     rts = inp.rank_tok_start
     want_q = np.full((world * C, H), 0, np.uint8)          # the allocations start zeroed
-    want_s = np.full((world * C,), 0.0, np.float32)
-    assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 2) == oracle.OK
+    if mode == "handshake":                                # windows with one scale per 128 elements
+        want_s = np.full((world * C, H // 128), 0.0, np.float32)
+        assert oracle.dispatch_quant_group(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 128, 2) == oracle.OK
+    else:
+        want_s = np.full((world * C,), 0.0, np.float32)
+        assert oracle.dispatch_quant(synth.bf16_to_u16(inp.X), want.slots, want_q, want_s, 2) == oracle.OK
     for r in range(world):
         _, st, _, s1, s2, s3, q, sc, log = res[r]
         assert st == 0
@@ -425,6 +487,7 @@ def test_two_processes_exchange_rows_through_mapped_windows(mode, sync):
             assert np.array_equal(win, want.windows[r * C:(r + 1) * C])        # rows from both processes, bit-exact
             assert harness.max_ulp_diff(y, want.Y[int(rts[r]):int(rts[r + 1])]) <= 1
         assert np.array_equal(q, want_q[r * C:(r + 1) * C])
+        assert sc.shape == want_s[r * C:(r + 1) * C].shape
         assert np.array_equal(sc.view(np.uint32), want_s[r * C:(r + 1) * C].view(np.uint32))
         assert log["refused_without_table"] == binding.MOE_ERR_STALE_PEERS
         assert log["refused_stale"] == binding.MOE_ERR_STALE_PEERS
