@@ -4,9 +4,11 @@
 //                         expert index first)
 //   topk_w[t, j]        = exp(l_j - l_0) / sum_j' exp(l_j' - l_0)   (fp32, sum in ascending j)
 //
-// One warp per token, K rounds of "largest remaining logit"; the lane that owns the winner retires it.
-// Rows of up to 1024 logits live in registers (warp_gate_load + warp_gate_select); longer rows are cached
-// in shared memory and scanned with a shuffle arg-max (warp_gate_token).
+// Rows of up to 1024 logits live in registers, a lane owning consecutive experts (warp_gate_load).  Rows of four
+// logits per lane or more are selected by threshold and rank (warp_gate_rank; two tokens per warp for large
+// batches: warp_gate_rank_pair); shorter rows, and tokens with too many equal logits for that, by K rounds of
+// "largest remaining logit" over cached lane maxima (warp_gate_select).  Rows beyond 1024 logits are cached in
+// shared memory and scanned with a shuffle arg-max, one warp per token (warp_gate_token).
 #pragma once
 
 #include "common.cuh"
