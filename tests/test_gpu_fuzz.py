@@ -87,6 +87,55 @@ def test_random_shape_fused_call_and_quantised_dispatch(i):
 
 
 @pytest.mark.parametrize("i", range(max(16, N_SHAPES // 3)))
+def test_random_quantised_dispatch_shape(i):
+    """Row lengths on both sides of every kernel form of the quantising dispatch (16 / 32 chunks per lane in
+    registers, the two-pass form beyond 16 KB, whole and partial 512-byte slabs), batch sizes on both sides of the
+    large-job rule, one scale per row and one per 128 elements: codes and scales bit-exact, padding untouched."""
+    rng = np.random.default_rng(99000 + i)
+    R = int(rng.choice([1, 2, 4, 8]))
+    E = R * int(rng.choice([1, 2, 8]))
+    K = int(rng.integers(1, min(E, 8) + 1))
+    H = 128 * int(rng.choice([1, 2, 3, 7, 16, 28, 31, 32, 33, 56, 63, 64, 65, 100, 128]))
+    # few long rows, many short ones: the largest cases stay near 100 MB of rows
+    T = int(rng.choice([1, 5, 40, 300, 1500] if H > 4096 else [1, 5, 40, 300, 1500, 6000, 20000 if H <= 512 else 9000]))
+    cuts = np.sort(rng.integers(0, T + 1, R - 1))
+    per = tuple(int(x) for x in np.diff(np.concatenate([[0], cuts, [T]])))
+    sch = PREFILL if rng.integers(0, 2) else DECODE
+    wl = Workload(f"qfuzz{i}", T, H, E, R, K, sch, "replace" if rng.integers(0, 2) else "uniform", "identity", 41000 + i,
+                  rank_tokens=per)
+    dev = torch.device("cuda:0")
+    inp = synth.make_inputs(wl)
+    X = inp.X.clone()
+    X[rng.integers(0, T)] = 0                                  # an all-zero row
+    X[rng.integers(0, T), rng.integers(0, H)] = 2.0e4          # an outlier
+    X[:, :128] *= 2.0 ** -7                                    # a group far smaller than the others
+    idx_np = inp.topk_idx.numpy()
+    p = oracle.plan(idx_np, E, R, inp.rank_tok_start)
+    C = int(p.n_recv.max()) + 1
+    _, slots = oracle.slots(idx_np, E, R, p, C, inp.rank_tok_start)
+    x_u16 = synth.bf16_to_u16(X)
+    comm = binding.MoeComm(T, H, E, R, K, dev)
+    Xd, idx = X.to(dev), inp.topk_idx.to(dev)
+    comm.moe_plan(sch, idx, T, inp.rank_tok_start)
+    for group in (0, 128):
+        G = 1 if group == 0 else H // group
+        want_q = np.full((R * C, H), 0xAB, np.uint8)
+        want_s = np.full((R * C, G), -1.0, np.float32)
+        wq = torch.full((R * C, H), 0xAB, dtype=torch.uint8, device=dev)
+        sc = torch.full((R * C, G), -1.0, dtype=torch.float32, device=dev)
+        if group == 0:
+            assert oracle.dispatch_quant(x_u16, slots, want_q, want_s.reshape(-1), 4) == oracle.OK
+            comm.moe_dispatch_quant(Xd, wq, sc.view(-1), C)
+        else:
+            assert oracle.dispatch_quant_group(x_u16, slots, want_q, want_s, group, 4) == oracle.OK
+            comm.moe_dispatch_quant_group(Xd, wq, sc, C, group)
+        assert comm.moe_status() == 0
+        assert np.array_equal(wq.cpu().numpy(), want_q), (group, T, H, K)
+        assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_s.view(np.uint32)), (group, T, H, K)
+    comm.close()
+
+
+@pytest.mark.parametrize("i", range(max(16, N_SHAPES // 3)))
 def test_random_gate_shape(i):
     """Top-k gating on random row lengths (every register form and the shared-memory form), top-k degrees up to
     the limit, batches on both sides of the two-tokens-per-warp switch, with and without many equal logits, rows
