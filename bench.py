@@ -552,9 +552,22 @@ def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
             t_g = best([flush, lambda: sc.moe_dispatch_quant_group(sl.X, sq, sg, sl.C, 128)]) - base
             t_c = best([flush, lambda: sc.moe_combine(sl.windows, sl.C, sl.w, sl.Y)]) - base
             t_p = best([flush, s_plan]) - base
+            # the same calls back to back (no flush): what a decode loop sees when the windows fit in L2
+            # (captured in CUDA graphs: launches from Python cannot feed calls this short fast enough)
+            fused_step = lambda: (sc.moe_plan_dispatch(swl.schedule, sl.idx, sl.X, sl.windows, sl.C),
+                                  sc.moe_combine(sl.windows, sl.C, sl.w, sl.Y))
+            warm = {"dispatch_us": time_graphed(lambda: sc.moe_dispatch(sl.X, sl.windows, sl.C)),
+                    "dispatch_quant_us": time_graphed(lambda: sc.moe_dispatch_quant(sl.X, sq, ss, sl.C)),
+                    "dispatch_quant_group128_us": time_graphed(lambda: sc.moe_dispatch_quant_group(sl.X, sq, sg, sl.C, 128)),
+                    "combine_us": time_graphed(lambda: sc.moe_combine(sl.windows, sl.C, sl.w, sl.Y)),
+                    "plan_us": time_graphed(s_plan),
+                    "plan_dispatch_fused_then_combine_us": time_graphed(fused_step)}
+            t_step = best([flush, lambda: sc.moe_plan_dispatch(swl.schedule, sl.idx, sl.X, sl.windows, sl.C),
+                           lambda: sc.moe_combine(sl.windows, sl.C, sl.w, sl.Y)]) - base
             assert sc.moe_status() == 0
             sweep.append({"tokens_per_rank": per_rank, "H": H, "plan_us": t_p, "dispatch_us": t_d,
-                          "dispatch_quant_us": t_q, "dispatch_quant_group128_us": t_g, "combine_us": t_c})
+                          "dispatch_quant_us": t_q, "dispatch_quant_group128_us": t_g, "combine_us": t_c,
+                          "plan_dispatch_fused_then_combine_us": t_step, "back_to_back": warm})
             del sl, sq, ss, sg
     out["batch_sweep"] = {"ranks": dwl.R, "experts": dwl.E, "top_k": dwl.K, "rows": sweep}
     return out
