@@ -257,6 +257,13 @@ __host__ __device__ constexpr int cluster_notify_smem_ints(int E, int R) {
   return (E / R) * (R + 1) + 2 * (E / R) + 1 + 33;
 }
 
+// The two halves of a cluster barrier.  Between them a CTA does what needs nobody else's data (arrive has release,
+// wait has acquire semantics: what a CTA wrote to its shared memory before arriving is visible to the others after
+// their wait).  Every thread of every CTA of the cluster executes each of them once per phase.
+__device__ __forceinline__ void cluster_arrive() { __cluster_barrier_arrive(); }
+__device__ __forceinline__ void cluster_wait() { __cluster_barrier_wait(); }
+
+// On entry every thread of the CTA has ARRIVED at the cluster barrier that says "my row of M is complete".
 __device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, [E] */, int32_t* scratch, int32_t E,
                                                int32_t R, int32_t d, int32_t full_table, int32_t align,
                                                int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
@@ -268,12 +275,13 @@ __device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, 
   int32_t* tot = tile + E_r * P;      // [E_r] rows each expert's run occupies
   int32_t* pre = tot + E_r;           // [E_r + 1]
   int32_t* warp_sums = pre + E_r + 1;
-  cluster.sync();                     // every CTA's row of M is complete and visible
+  cluster_wait();                     // every CTA's row of M is complete and visible
   for (int q = tid; q < E_r * R; q += nthreads) {   // consecutive threads: consecutive experts of one remote row
     const int el = q % E_r, rr = q / E_r;
     const int32_t* remote = cluster.map_shared_rank(my_row, rr);
     tile[el * P + rr] = remote[d * E_r + el];
   }
+  cluster_arrive();                   // this thread reads no other CTA's shared memory from here on
   __syncthreads();
   if (full_table)
     for (int rr = tid; rr < R; rr += nthreads) {     // branches from source rank rr to this rank
@@ -298,7 +306,7 @@ __device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, 
   for (int q = tid; q < E_r * R; q += nthreads)      // o[d*E_r + el][rr], one coalesced stream
     o[(size_t)d * E_r * R + q] = pre[q / R] + tile[(q / R) * P + q % R];
   if (tid == 0) n_recv[d] = pre[E_r];
-  cluster.sync();                     // no CTA leaves while its row may still be read
+  cluster_wait();                     // no CTA leaves while its row may still be read
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS)
@@ -334,6 +342,7 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
   }
   if (as_cluster) {   // see cluster_notify: every CTA builds its own window's offsets from the rows in shared memory
     __syncthreads();
+    cluster_arrive();   // this CTA's row is complete
     cluster_notify(sm, sm + E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
     return;
   }
@@ -387,16 +396,15 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   const unsigned lt = lanemask_lt();
 
   for (int e = threadIdx.x; e < E; e += WARPS * 32) rank_base[e] = 0;
+  bool arrived = false;   // as_cluster: at the barrier that says "my row of M is complete"
   for (int32_t pass = b_begin; pass < b_end; pass += WARPS * 32) {
-    for (int i = threadIdx.x; i < P * E; i += WARPS * 32) counts[i] = 0;
     const int32_t b = pass + warp * 32 + lane;
     int32_t e = -1;
-    if (b < b_end) {
-      e = __ldg(topk_idx + b);
-      if (e < 0 || e >= E) {
-        raise_status(&ctl->status, MOE_ERR_BAD_INDEX);
-        e = -1;
-      }
+    if (b < b_end) e = __ldg(topk_idx + b);   // on its way while the counters are cleared
+    for (int i = threadIdx.x; i < P * E; i += WARPS * 32) counts[i] = 0;
+    if (b < b_end && (e < 0 || e >= E)) {
+      raise_status(&ctl->status, MOE_ERR_BAD_INDEX);
+      e = -1;
     }
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     const int ahead = __popc(peers & lt);           // equal keys in lower lanes = earlier branches
@@ -433,10 +441,18 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
       }
     }
     __syncthreads();
+    const bool last_pass = pass + WARPS * 32 >= b_end;
+    if (as_cluster && last_pass) {   // rank_base is final: the other CTAs may read it while s and M go out
+      cluster_arrive();
+      arrived = true;
+    }
     if (b < b_end) s[b] = e >= 0 ? counts[e * P + warp] + ahead : 0;
-    __syncthreads();
+    if (!last_pass) __syncthreads();   // the next pass clears the counters
   }
-  __syncthreads();
+  if (as_cluster && !arrived) {   // a rank without tokens
+    __syncthreads();
+    cluster_arrive();
+  }
   for (int e = threadIdx.x; e < E; e += WARPS * 32) M[(size_t)r * E + e] = rank_base[e];
   if (as_cluster) {
     cluster_notify(rank_base, sm + (P + 1) * E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
