@@ -97,6 +97,7 @@ EDGE = [
     ("tile_boundary_plus1", 2050, 32, 8, 2, 2, "uniform", None),
     ("rank_above_compact_decode_limit", 6000, 16, 16, 2, 2, "uniform", (5000, 1000)),   # 10000 branches in rank 0
     ("compact_decode_several_passes", 1200, 16, 1024, 2, 6, "uniform", (682, 518)),     # E > 768: 8-warp planner
+    ("compact_several_passes_empty_ranks", 900, 64, 32, 4, 8, "uniform", (0, 500, 0, 400)),   # 4 passes of the 32-warp planner beside ranks that arrive at once
     ("max_ranks_max_experts", 4096, 64, 4096, 256, 8, "uniform", None),                 # R = MOE_MAX_R, E = MOE_MAX_E
     ("many_tiles", 200000, 32, 64, 8, 8, "uniform", None),                              # 1.6 M branches, 98 tiles per rank
     ("long_rows_two_items_per_row", 512, 16384, 16, 4, 4, "uniform", None),             # 32 KB rows
