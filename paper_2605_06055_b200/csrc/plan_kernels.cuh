@@ -283,26 +283,58 @@ __device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, 
   }
   cluster_arrive();                   // this thread reads no other CTA's shared memory from here on
   __syncthreads();
-  if (full_table)
+  if (full_table) {
     for (int rr = tid; rr < R; rr += nthreads) {     // branches from source rank rr to this rank
       int32_t acc = 0;
       for (int el = 0; el < E_r; ++el) acc += tile[el * P + rr];
       c_rank[(size_t)rr * R + d] = acc;
     }
-  __syncthreads();
-  for (int el = tid; el < E_r; el += nthreads) {     // exclusive prefix over source ranks, in place
-    int32_t run = 0;
-    for (int rr = 0; rr < R; ++rr) {
-      const int32_t m = tile[el * P + rr];
-      tile[el * P + rr] = run;
-      run += m;
-    }
-    n_exp[d * E_r + el] = run;
-    tot[el] = (run + align - 1) / align * align;
+    __syncthreads();
   }
-  __syncthreads();
-  block_exclusive_scan(tot, pre, E_r, warp_sums);
-  __syncthreads();
+  if (E_r <= 32 && R <= 16) {
+    // Few experts per window (every decode configuration): one warp does both prefixes from registers -- lane el
+    // loads its expert's R counts at once, writes their running sums back, and the padded totals are scanned
+    // across the lanes by shuffles.  (With a dependent load-store chain per source rank and a block-wide scan
+    // behind it these two steps took 1.0 us.)
+    if (tid < 32) {
+      const int el = tid;
+      const bool live = el < E_r;
+      int32_t m[16];
+#pragma unroll
+      for (int rr = 0; rr < 16; ++rr) m[rr] = (live && rr < R) ? tile[el * P + rr] : 0;
+      int32_t run = 0;
+#pragma unroll
+      for (int rr = 0; rr < 16; ++rr) {
+        if (live && rr < R) tile[el * P + rr] = run;
+        run += m[rr];
+      }
+      if (live) n_exp[d * E_r + el] = run;
+      const int32_t padded = live ? (run + align - 1) / align * align : 0;
+      int32_t incl = padded;
+#pragma unroll
+      for (int dd = 1; dd < 32; dd <<= 1) {
+        const int32_t u = __shfl_up_sync(0xffffffffu, incl, dd);
+        if (tid >= dd) incl += u;
+      }
+      if (live) pre[el] = incl - padded;
+      if (tid == 31) pre[E_r] = incl;
+    }
+    __syncthreads();
+  } else {
+    for (int el = tid; el < E_r; el += nthreads) {     // exclusive prefix over source ranks, in place
+      int32_t run = 0;
+      for (int rr = 0; rr < R; ++rr) {
+        const int32_t m = tile[el * P + rr];
+        tile[el * P + rr] = run;
+        run += m;
+      }
+      n_exp[d * E_r + el] = run;
+      tot[el] = (run + align - 1) / align * align;
+    }
+    __syncthreads();
+    block_exclusive_scan(tot, pre, E_r, warp_sums);
+    __syncthreads();
+  }
   for (int q = tid; q < E_r * R; q += nthreads)      // o[d*E_r + el][rr], one coalesced stream
     o[(size_t)d * E_r * R + q] = pre[q / R] + tile[(q / R) * P + q % R];
   if (tid == 0) n_recv[d] = pre[E_r];
