@@ -121,10 +121,12 @@ dispatch_bulk_kernel(const unsigned char* __restrict__ X, unsigned char* __restr
   // Items in flight: q0 is consumed this iteration, q1 is loading, q2 is fetched now.
   ItemFeed feed = begin_feed();
   int32_t q0 = a.n_items, q1 = a.n_items;
-  // Started early behind the planner (moe_plan_dispatch): the first two items of a small job are fixed
-  // and their payload depends on nothing the planner writes, so their loads travel while it runs.
-  // Nothing is taken from the work counter and no planner output is read before the wait.
-  const bool early = a.pdl && a.static_first >= 2;
+  // The first two items of a small job are fixed and their payload depends on nothing a planner writes, so
+  // their loads are issued before anything else: before the wait for a planner this launch was chained behind
+  // (moe_plan_dispatch: they travel while it runs), and before the status and capacity checks, whose loads
+  // otherwise stand in front of the first payload byte (1 us of a flushed call).  Nothing is taken from the
+  // work counter and no planner output is read before the wait; a call that must abort lets them land first.
+  const bool early = a.static_first >= 2;
   if (early) {
     q0 = fetch_item(a, feed);
     q1 = fetch_item(a, feed);

@@ -133,9 +133,9 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   // q1 is issued at its start, into the stage whose code row was stored QUANT_STAGES - 1 iterations ago.
   ItemFeed feed = begin_feed();
   int32_t q0 = a.n_items, q1 = a.n_items;
-  // Started early behind the planner (moe_plan_dispatch_quant): the first two rows of a small job are fixed
-  // and depend on nothing the planner writes, so the first load travels while the plan is computed.
-  const bool early = a.pdl && a.static_first >= 2;
+  // The first two rows of a small job are fixed and depend on nothing a planner writes, so the first load is
+  // issued before the wait for a planner in front (moe_plan_dispatch_quant) and before the status checks.
+  const bool early = a.static_first >= 2;
   if (early) {
     q0 = fetch_item(a, feed);
     q1 = fetch_item(a, feed);
@@ -341,9 +341,9 @@ dispatch_quant_reg_kernel(const unsigned char* __restrict__ X, unsigned char* __
   // it, as soon as every lane holds its part of q0.
   ItemFeed feed = begin_feed();
   int32_t q0 = a.n_items, q1 = a.n_items;
-  // Started early behind the planner: the first rows of a small job are fixed and depend on nothing the planner
-  // writes, so the first load travels while the plan is computed.
-  const bool early = a.pdl && a.static_first >= 2;
+  // The first rows of a small job are fixed and depend on nothing a planner writes, so the first load is issued
+  // before the wait for a planner in front and before the status checks.
+  const bool early = a.static_first >= 2;
   if (early) {
     q0 = fetch_item(a, feed);
     q1 = fetch_item(a, feed);
