@@ -347,18 +347,34 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
   const int lane = threadIdx.x & 31;
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
+  ItemFeed feed = begin_feed();
+  int32_t item = a.n_items;
+  BranchMeta meta = {-1, 0, 0.0f};
+  // Small jobs: the first item is fixed (no counter), and the plan it reads is complete before this launch, so its
+  // routing index, small offset and weight are asked for before the status and capacity checks and travel
+  // while those are evaluated -- one round trip to memory less in front of the first row.
+  bool meta_ready = false;
+  if constexpr (MODE != LD_L1) {
+    if (a.static_first >= 2) {
+      item = fetch_item(a, feed);
+      if (item < a.n_items) meta = load_meta(a, topk_w, decode_item<true>(a, item).t, lane);
+      meta_ready = true;
+    }
+  }
   if (must_abort(a)) {
     end_work(a);
     return;
   }
-  ItemFeed feed = begin_feed();
-  int32_t item = fetch_item(a, feed);
-  BranchMeta meta = {-1, 0, 0.0f};
-  if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item<MODE != LD_L1>(a, item).t, lane);
+  if (!meta_ready) {
+    item = fetch_item(a, feed);
+    if (a.prefetch_meta && item < a.n_items) meta = load_meta(a, topk_w, decode_item<MODE != LD_L1>(a, item).t, lane);
+    meta_ready = a.prefetch_meta != 0;
+  }
   while (item < a.n_items) {
     const int32_t next_item = fetch_item(a, feed);
     const WorkItem wi = decode_item<MODE != LD_L1>(a, item);
-    if (!a.prefetch_meta) meta = load_meta(a, topk_w, wi.t, lane);
+    if (!meta_ready) meta = load_meta(a, topk_w, wi.t, lane);
+    meta_ready = a.prefetch_meta != 0;   // from the second item on, only the prefetching form has it in hand
     const int64_t slot = finish_slot(a, map, meta, wi.t, lane, false);
     const float w_lane = meta.w;
     // short rows: the next item's routing index, small offset and weight travel while this item is reduced
