@@ -321,6 +321,23 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
   }
   RowArgs b = a;
   set_work(ctx, b, (int64_t)grid * warps, g_max);
+  // Small and medium jobs: the fewest warps that still finish in the same number of rounds.  2048 rows of 8 KB are
+  // 13.8 rows per SM: two rounds with eight warps, of which the second is only three quarters full, and two full
+  // rounds with seven (32.1 -> 30.4 us flushed, 27.6 -> 25.6 us back to back; 1024 rows: 19.5 -> 18.4 us).
+  if (b.static_first >= 2 && b.n_items > 0 && ctx->granule_override == 0) {
+    const int64_t rounds = ((int64_t)b.n_items + (int64_t)grid * warps - 1) / ((int64_t)grid * warps);
+    const int fewer = (int)(((int64_t)b.n_items + grid * rounds - 1) / (grid * rounds));
+    if (fewer >= 1 && fewer < warps) {
+      RowArgs c = a;
+      set_work(ctx, c, (int64_t)grid * fewer, g_max);
+      // (the cut of the rows changes with the warp count: taken only if the rounds come out at least nine tenths
+      // full -- 1280 rows of 8 KB are better off with eight warps and their leftover rows cut finer)
+      if ((int64_t)c.n_items <= rounds * grid * fewer && (int64_t)c.n_items * 10 >= rounds * grid * fewer * 9) {
+        b = c;
+        warps = fewer;
+      }
+    }
+  }
   const int smem = warps * BULK_STAGES * (b.granule * 512 + 8);
   b.pdl = pdl;
   launch_kernel(dispatch_bulk_kernel, grid, warps * 32, smem, st, pdl, 0, reinterpret_cast<const unsigned char*>(x),
@@ -338,11 +355,26 @@ void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const floa
                         : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_STREAM>;
   const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
-  set_work(ctx, b, (int64_t)grid * 8, 1 << 20, !large);   // the large-job form has no tail items
+  int warps = 8;
+  set_work(ctx, b, (int64_t)grid * warps, 1 << 20, !large);   // the large-job form has no tail items
+  // Small and medium jobs: the fewest warps that finish in the same number of (nearly full) rounds, as in
+  // launch_dispatch_bulk.
+  if (b.static_first >= 2 && b.n_items > 0 && ctx->granule_override == 0) {
+    const int64_t rounds = ((int64_t)b.n_items + (int64_t)grid * warps - 1) / ((int64_t)grid * warps);
+    const int fewer = (int)(((int64_t)b.n_items + grid * rounds - 1) / (grid * rounds));
+    if (fewer >= 1 && fewer < warps) {
+      RowArgs c = a;
+      set_work(ctx, c, (int64_t)grid * fewer, 1 << 20, !large);
+      if ((int64_t)c.n_items <= rounds * grid * fewer && (int64_t)c.n_items * 10 >= rounds * grid * fewer * 9) {
+        b = c;
+        warps = fewer;
+      }
+    }
+  }
   // an item that is one or two batches of loads cannot hide its own metadata latency: prefetch it
   constexpr int unroll = KT > 0 ? combine_unroll(KT) : 4;
   b.prefetch_meta = (b.granule + unroll - 1) / unroll <= 2;
-  kernel<<<grid, 256, 0, st>>>(win, w, y, b, ctx->map);
+  kernel<<<grid, warps * 32, 0, st>>>(win, w, y, b, ctx->map);
 }
 
 }  // namespace
