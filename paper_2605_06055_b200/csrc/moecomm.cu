@@ -332,7 +332,13 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
       set_work(ctx, c, (int64_t)grid * fewer, g_max);
       // (the cut of the rows changes with the warp count: taken only if the rounds come out at least nine tenths
       // full -- 1280 rows of 8 KB are better off with eight warps and their leftover rows cut finer)
-      if ((int64_t)c.n_items <= rounds * grid * fewer && (int64_t)c.n_items * 10 >= rounds * grid * fewer * 9) {
+      // Behind the planner the rule is left alone for CTAs small enough to fit two per SM: the planner's CTAs
+      // still hold their SMs when the dispatch CTAs are placed, so some SMs get two of them, and with the
+      // full warp count the CTAs placed last are the idle ones (plan + dispatch + combine at 16 / 32 tokens
+      // per rank of 8 KB rows: 17.2 / 23.1 us back to back without the rule, 18.9 / 25.7 us with it).
+      const bool doubles_up = pdl && 2 * fewer * BULK_STAGES * (c.granule * 512 + 8) <= BULK_SMEM_BUDGET;
+      if (!doubles_up && (int64_t)c.n_items <= rounds * grid * fewer &&
+          (int64_t)c.n_items * 10 >= rounds * grid * fewer * 9) {
         b = c;
         warps = fewer;
       }
