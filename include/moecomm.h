@@ -122,7 +122,11 @@ moe_status_t moe_gate_plan(moe_ctx_t* ctx, moe_schedule_t schedule, const float*
  * PREFILL fills every field.  DECODE leaves counts, c_rank and n_exp NULL, and
  * small_off is guaranteed to hold delta only after moe_dispatch has run (small
  * decode batches, at most 4096 branches per source rank, are planned in a single
- * launch that already leaves it final after moe_plan). */
+ * launch that already leaves it final after moe_plan).
+ * rows [T,K] is what the last dispatch over the whole batch recorded for this plan (see MOE_OPT_SLOT_REUSE):
+ * the window row d*capacity_rows + large_off + small_off of every branch, the same numbers moe_slots writes,
+ * for the capacity_rows given in rows_capacity; NULL and -1 when nothing is recorded (no such dispatch since
+ * the plan, or an error was reported since).  Its contents are final once that dispatch has completed. */
 typedef struct {
   const int32_t* counts;
   const int32_t* c_rank;
@@ -130,6 +134,8 @@ typedef struct {
   const int32_t* large_off;
   const int32_t* n_exp;
   const int32_t* n_recv;
+  const int32_t* rows;
+  int64_t rows_capacity;
 } moe_plan_view_t;
 moe_status_t moe_plan_view(const moe_ctx_t* ctx, moe_plan_view_t* out /*HOST*/);
 
@@ -431,14 +437,26 @@ moe_status_t moe_forward_host(moe_ctx_t* ctx, moe_schedule_t schedule, int32_t T
  *                          16 and the device can co-schedule them: the count rows are exchanged through
  *                          distributed shared memory and every CTA builds its own window's offsets.
  *                          0: the last CTA to finish builds all offsets from the matrix in global memory.
- *                          Same result. */
+ *                          Same result.
+ *   MOE_OPT_SLOT_REUSE     1 (default): a dispatch over the whole batch (any form, not the *_range calls) also
+ *                          records every branch's window row (the sum of Section 5.2's two offsets and the
+ *                          window start) in the workspace, and a combine of the same plan with the same
+ *                          capacity_rows reads that row back instead of resolving routing index -> large
+ *                          offset again: one dependent load less before its first payload loads.  The record
+ *                          is dropped by every new plan, by MOE_OPT_EXPERT_ALIGN and by a moe_status that
+ *                          reports an error; a recorded row outside [0, R * capacity_rows) is never used as
+ *                          an address (the branch is skipped and the status becomes MOE_ERR_NOT_PLANNED).
+ *                          It assumes that the kernels run in the order of the calls (calls recorded into
+ *                          a graph count from when the graph runs).  0: combine always resolves the branch
+ *                          from the plan.  Same result. */
 typedef enum {
   MOE_OPT_DISPATCH_PATH = 0,
   MOE_OPT_GRANULE = 1,
   MOE_OPT_TEST_STARVE_WAIT_MS = 2,
   MOE_OPT_OVERLAP = 3,
   MOE_OPT_EXPERT_ALIGN = 4,
-  MOE_OPT_CLUSTER_PLAN = 5
+  MOE_OPT_CLUSTER_PLAN = 5,
+  MOE_OPT_SLOT_REUSE = 6
 } moe_option_t;
 enum { MOE_DISPATCH_AUTO = 0, MOE_DISPATCH_REGISTERS = 1, MOE_DISPATCH_BULK = 2 };
 moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value);

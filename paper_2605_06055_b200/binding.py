@@ -35,7 +35,7 @@ EXPORTS = [
 MOE_SYNC_SLOTS = 4
 MOE_WINDOW_STATE, MOE_WINDOW_QUANT, MOE_WINDOW_QUANT_GROUP = 1, 2, 4
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
-MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN = 4, 5
+MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN, MOE_OPT_SLOT_REUSE = 4, 5, 6
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
 
 
@@ -45,7 +45,8 @@ class MoeShape(ctypes.Structure):
 
 
 class MoePlanView(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("counts", "c_rank", "small_off", "large_off", "n_exp", "n_recv")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("counts", "c_rank", "small_off", "large_off", "n_exp", "n_recv",
+                                               "rows")] + [("rows_capacity", ctypes.c_int64)]
 
 
 class MoeWindowHandle(ctypes.Structure):
@@ -494,7 +495,7 @@ class MoeComm:
             raise MoeError(rc, "moe_plan_view")
         base = self.workspace.data_ptr()
         shapes = {"counts": (self.R, self.E), "c_rank": (self.R, self.R), "small_off": (self.T, self.K),
-                  "large_off": (self.E, self.R), "n_exp": (self.E,), "n_recv": (self.R,)}
+                  "large_off": (self.E, self.R), "n_exp": (self.E,), "n_recv": (self.R,), "rows": (self.T, self.K)}
         out = {}
         for name, shp in shapes.items():
             p = getattr(v, name)
@@ -504,6 +505,7 @@ class MoeComm:
             n = int(np.prod(shp))
             off = p - base
             out[name] = self.workspace[off:off + 4 * n].view(torch.int32).view(*shp)
+        out["rows_capacity"] = int(v.rows_capacity)
         return out
 
     def moe_dispatch(self, x: torch.Tensor, windows: torch.Tensor, capacity_rows: int, stream=None,

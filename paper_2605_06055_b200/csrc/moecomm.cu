@@ -43,9 +43,14 @@ struct moe_ctx {
   int32_t starve_wait_ms;   // MOE_OPT_TEST_STARVE_WAIT_MS
   int32_t overlap;          // MOE_OPT_OVERLAP
   int32_t cluster_plan;     // MOE_OPT_CLUSTER_PLAN
+  int32_t slot_reuse;       // MOE_OPT_SLOT_REUSE
   bool plan_cluster_ok;     // the compact planner of this shape can be launched as one cluster of R CTAs
   bool scan_cluster_ok;     // the same for the scan kernel of the tile planner
   int32_t expert_align;     // MOE_OPT_EXPERT_ALIGN: every expert's run starts on a multiple of this many rows
+  // Window rows of every branch as the last whole-batch dispatch of the current plan recorded them, and the capacity
+  // they were computed for (-1: none); a combine with that capacity reads them instead of resolving the branch again.
+  int32_t* slot_table;      // device, [T_max * K] (inside the workspace)
+  int64_t slots_for_C;
   cudaStream_t out_stream;  // moe_forward_host: download and upload streams, created on first use (no device memory)
   cudaStream_t in_stream;
   cudaEvent_t fwd_events[2 * 16 + 2];
@@ -94,7 +99,7 @@ int64_t max_tiles(const moe_shape_t* s) {
 }
 
 struct Layout {
-  size_t ctl, M, c_rank, o, n_exp, n_recv, peers, s, tile_rank, tile_hist, total;
+  size_t ctl, M, c_rank, o, n_exp, n_recv, peers, s, slot, tile_rank, tile_hist, total;
 };
 
 Layout layout_of(const moe_shape_t* s) {
@@ -114,6 +119,7 @@ Layout layout_of(const moe_shape_t* s) {
   L.n_recv = take(sizeof(int32_t) * s->R);
   L.peers = take(sizeof(void*) * s->R * 4);   // window bases, state regions, code windows, scale tensors
   L.s = take(sizeof(int32_t) * B);
+  L.slot = take(sizeof(int32_t) * B);
   L.tile_rank = take(sizeof(int32_t) * B);
   L.tile_hist = take(sizeof(int32_t) * (size_t)max_tiles(s) * s->E);
   L.total = at;
@@ -137,6 +143,8 @@ RowArgs row_args(const moe_ctx* ctx, int64_t C, bool dispatching) {
   const bool finish_delta = ctx->schedule == MOE_SCHED_DECODE && !ctx->compact_plan;
   a.small_off = finish_delta ? ctx->tile_rank : ctx->s;
   a.small_out = (finish_delta && dispatching) ? ctx->s : nullptr;
+  a.slot_out = nullptr;
+  a.slot_in = nullptr;
   a.tile_base = finish_delta ? ctx->tile_hist : nullptr;
   a.large_off = ctx->o;
   a.n_recv = ctx->n_recv;
@@ -432,9 +440,12 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
     ctx->peer_gen[d] = 0;
   }
   ctx->s = reinterpret_cast<int32_t*>(ctx->ws + L.s);
+  ctx->slot_table = reinterpret_cast<int32_t*>(ctx->ws + L.slot);
+  ctx->slots_for_C = -1;
   ctx->tile_rank = reinterpret_cast<int32_t*>(ctx->ws + L.tile_rank);
   ctx->tile_hist = reinterpret_cast<int32_t*>(ctx->ws + L.tile_hist);
   ctx->planned = false;
+  ctx->slots_for_C = -1;
   ctx->layout_done = false;
   ctx->compact_plan = false;
   ctx->launches = 0;
@@ -444,6 +455,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->starve_wait_ms = 0;
   ctx->overlap = 1;
   ctx->cluster_plan = 1;
+  ctx->slot_reuse = 1;
   ctx->plan_cluster_ok = false;
   ctx->scan_cluster_ok = false;
   ctx->expert_align = 1;
@@ -616,6 +628,7 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
       if (rank_tok_start[r + 1] < rank_tok_start[r]) return MOE_ERR_INVALID_ARG;
   }
   ctx->planned = false;
+  ctx->slots_for_C = -1;
   ctx->layout_done = false;
 
   const int rounds = schedule == MOE_SCHED_PREFILL ? ROUNDS_PREFILL : ROUNDS_DECODE;
@@ -757,12 +770,20 @@ moe_status_t moe_plan_view(const moe_ctx_t* c, moe_plan_view_t* out) {
   out->large_off = c->o;
   out->n_exp = full ? c->n_exp : nullptr;
   out->n_recv = c->n_recv;
+  out->rows = c->slots_for_C >= 0 ? c->slot_table : nullptr;
+  out->rows_capacity = c->slots_for_C;
   return MOE_OK;
 }
 
 }  // extern "C"
 
 namespace {
+
+// A dispatch over the whole batch records every branch's window row for the combine that follows (rows are kept
+// as 32-bit words: not for windows of 2^31 rows or more).
+bool records_slots(const moe_ctx* ctx, const RowArgs& a) {
+  return a.t_begin == 0 && a.t_count == ctx->T && ctx->T > 0 && (int64_t)ctx->shape.R * a.C < ((int64_t)1 << 31);
+}
 
 moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const void* const* bases, int64_t capacity_rows,
                            void* stream, int32_t t_begin = 0, int32_t t_end = -1, bool behind_plan = false) {
@@ -778,6 +799,8 @@ moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const voi
   a.t_begin = t_begin;
   a.t_count = t_end - t_begin;
   a.topk_idx = ctx->topk_idx;
+  const bool records = records_slots(ctx, a);
+  if (records) a.slot_out = ctx->slot_table;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* xs = static_cast<const uint4*>(x);
   uint4* win = static_cast<uint4*>(windows);
@@ -793,7 +816,9 @@ moe_status_t dispatch_impl(moe_ctx* ctx, const void* x, void* windows, const voi
       default: launch_dispatch_regs<0>(ctx, a, xs, win, st); break;
     }
   }
-  return launch_ok(ctx);
+  const moe_status_t rc = launch_ok(ctx);
+  if (records && rc == MOE_OK) ctx->slots_for_C = capacity_rows;
+  return rc;
 }
 
 }  // namespace
@@ -865,6 +890,13 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   a.topk_idx = ctx->topk_idx;
   a.win_base = reinterpret_cast<const unsigned char* const*>(q_bases);
   a.scale_base = s_bases;
+  const bool records = records_slots(ctx, a);
+  if (records) a.slot_out = ctx->slot_table;
+  auto launched = [&]() {
+    const moe_status_t rc = launch_ok(ctx);
+    if (records && rc == MOE_OK) ctx->slots_for_C = capacity_rows;
+    return rc;
+  };
   // One work item per token: the whole row is needed for its scale.
   const int upr = (a.H16 + 31) / 32;
   const int stage = (H * 2 + 127) / 128 * 128;
@@ -918,7 +950,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
       if (grouped) whole_slabs ? launch(dispatch_quant_reg_kernel<32, true, true>) : launch(dispatch_quant_reg_kernel<32, false, true>);
       else whole_slabs ? launch(dispatch_quant_reg_kernel<32, true, false>) : launch(dispatch_quant_reg_kernel<32, false, false>);
     }
-    return launch_ok(ctx);
+    return launched();
   }
   const int stages = large ? 3 : 2;
   int warps = ring_warps(stages);
@@ -940,7 +972,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   } else {   // (rows beyond 16 KB only: shorter rows of small jobs went to the register kernel)
     launch(dispatch_quant_kernel<2, 0, false>);
   }
-  return launch_ok(ctx);
+  return launched();
 }
 
 // moe_plan followed by the quantising dispatch, chained; every host-side check comes before anything is enqueued.
@@ -1009,6 +1041,7 @@ moe_status_t combine_impl(moe_ctx* ctx, const void* windows, const void* const* 
   a.t_begin = t_begin;
   a.t_count = t_end - t_begin;
   a.topk_idx = ctx->topk_idx;
+  if (ctx->slots_for_C == capacity_rows && ctx->slot_reuse) a.slot_in = ctx->slot_table;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const uint4* win = static_cast<const uint4*>(windows);
   uint4* ys = static_cast<uint4*>(y);
@@ -1062,6 +1095,7 @@ moe_status_t moe_layout(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* 
   const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T_local, starts, stream, nullptr, nullptr, nullptr);
   if (rc != MOE_OK) return rc;
   ctx->planned = false;   // the offsets are not valid until moe_notify has seen every rank's counts
+  ctx->slots_for_C = -1;
   if (cudaMemcpyAsync(counts_row, ctx->M + (size_t)my_rank * ctx->shape.E, sizeof(int32_t) * ctx->shape.E,
                       cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MOE_ERR_CUDA;
@@ -1452,6 +1486,7 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) 
         return MOE_ERR_INVALID_ARG;   // padded row counts must stay in int32
       ctx->expert_align = (int32_t)value;
       ctx->planned = false;           // offsets of an earlier plan no longer describe the layout asked for
+      ctx->slots_for_C = -1;
       ctx->layout_done = false;
       return MOE_OK;
     case MOE_OPT_CLUSTER_PLAN:
@@ -1461,6 +1496,10 @@ moe_status_t moe_set_option(moe_ctx_t* ctx, moe_option_t option, int64_t value) 
     case MOE_OPT_OVERLAP:
       if (value != 0 && value != 1) return MOE_ERR_INVALID_ARG;
       ctx->overlap = (int32_t)value;
+      return MOE_OK;
+    case MOE_OPT_SLOT_REUSE:
+      if (value != 0 && value != 1) return MOE_ERR_INVALID_ARG;
+      ctx->slot_reuse = (int32_t)value;
       return MOE_OK;
   }
   return MOE_ERR_INVALID_ARG;
@@ -1480,6 +1519,7 @@ moe_status_t moe_status(moe_ctx_t* ctx, void* stream) {
     // A plan that saw a routing index outside [0, E) left that branch out of its counts: it describes no
     // valid layout, so it does not survive the report (a later dispatch returns MOE_ERR_NOT_PLANNED
     // instead of silently skipping the branch).
+    ctx->slots_for_C = -1;   // a dispatch that stopped early has not recorded every row
     if (word == MOE_ERR_BAD_INDEX) {
       ctx->planned = false;
       ctx->layout_done = false;
@@ -1623,6 +1663,8 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
   a.topk_idx = topk_idx;
   a.small_off = sc->tile_rank;
   a.small_out = nullptr;
+  a.slot_out = nullptr;
+  a.slot_in = nullptr;
   a.tile_base = sc->tile_hist;
   a.large_off = sc->o;
   a.n_recv = n_recv;

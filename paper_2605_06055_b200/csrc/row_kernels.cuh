@@ -19,6 +19,11 @@ struct RowArgs {
   const int32_t* topk_idx;   // [T,K]
   const int32_t* small_off;  // final small offsets s [T,K]; tile-planned DECODE: in-tile rank [T,K]
   int32_t* small_out;        // tile-planned DECODE dispatch: where delta is recorded; else nullptr
+  // Finished window rows (dst*C + row in window) of every branch: a dispatch over the whole batch records them
+  // (slot_out), and a combine with the same plan and capacity reads them back (slot_in) instead of walking
+  // routing index -> large offset: one dependent load less in front of its first payload loads.  Else nullptr.
+  int32_t* slot_out;
+  const int32_t* slot_in;
   const int32_t* tile_base;  // tile-planned DECODE: [tiles,E] exclusive tile bases; else nullptr
   const int32_t* large_off;  // o [E,R]
   const int32_t* n_recv;     // [R]
@@ -73,7 +78,9 @@ __device__ __forceinline__ int64_t resolve_slot(const RowArgs& a, const RankMap&
     so += ld_plan(a.tile_base + (size_t)tile_of_branch(map, r, b, a.K) * a.E + e);
     if (record) a.small_out[b] = so;
   }
-  return (int64_t)(e / a.E_r) * a.C + ld_plan(a.large_off + (size_t)e * a.R + r) + so;
+  const int64_t slot = (int64_t)(e / a.E_r) * a.C + ld_plan(a.large_off + (size_t)e * a.R + r) + so;
+  if (record && a.slot_out != nullptr) a.slot_out[b] = (int32_t)slot;
+  return slot;
 }
 
 // The same resolution in two phases, so that its memory latency can hide behind payload traffic:
@@ -95,8 +102,12 @@ __device__ __forceinline__ BranchMeta load_meta(const RowArgs& a, const float* _
   m.w = 0.0f;
   if (lane < a.K) {
     const int32_t b = t * a.K + lane;
-    m.e = __ldg(a.topk_idx + b);
-    m.so = ld_plan(a.small_off + b);
+    if (a.slot_in != nullptr) {
+      m.so = ld_plan(a.slot_in + b);   // the finished row; the routing index is not needed
+    } else {
+      m.e = __ldg(a.topk_idx + b);
+      m.so = ld_plan(a.small_off + b);
+    }
     if (topk_w != nullptr) m.w = __ldg(topk_w + b);
   }
   return m;
@@ -104,6 +115,16 @@ __device__ __forceinline__ BranchMeta load_meta(const RowArgs& a, const float* _
 
 __device__ __forceinline__ int64_t finish_slot(const RowArgs& a, const RankMap& map, const BranchMeta& m, int32_t t,
                                                int lane, bool record) {
+  if (a.slot_in != nullptr) {
+    // A recorded row is trusted only inside the windows: a table that no dispatch has filled (calls recorded into a
+    // graph that never ran) must not become an address.
+    if (lane >= a.K) return -1;
+    if ((uint32_t)m.so >= (uint32_t)(a.R * a.C)) {
+      raise_status(a.status, MOE_ERR_NOT_PLANNED);
+      return -1;
+    }
+    return (int64_t)m.so;
+  }
   if (lane >= a.K || m.e < 0 || m.e >= a.E) return -1;   // bad indexes were flagged by the plan; never dereferenced
   const int32_t r = src_rank(map, t);
   int32_t so = m.so;

@@ -126,7 +126,7 @@ def gpu_run(inp: synth.Inputs, C: int, schedule: Optional[int] = None, comm: Opt
     windows = torch.from_numpy(np.full((wl.R * C, wl.H), CANARY, np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
     comm.moe_dispatch(X, windows, C)
     statuses.append(comm.moe_status())
-    view = {k: (None if v is None else v.cpu().numpy().copy()) for k, v in comm.moe_plan_view().items()}
+    view = {k: (v.cpu().numpy().copy() if torch.is_tensor(v) else v) for k, v in comm.moe_plan_view().items()}
     win_host = windows.cpu().view(torch.int16).numpy().view(np.uint16).copy()
     if wl.expert_op == "scale":
         gpu_expert_scale(windows, idx, wl.E, wl.R, C, inp.scale.to(dev), align)
@@ -149,6 +149,12 @@ def assert_parity(g: DeviceRun, o: OracleRun, schedule: int, combine_ulp: int = 
             continue
         assert np.array_equal(g.view[k], getattr(o.plan, on)), k          # bit-exact integers
     assert np.array_equal(g.slots.astype(np.int64), o.slots)
+    # the rows the whole-batch dispatch recorded for the combine behind it: the same numbers, for the same capacity
+    if g.slots.size:
+        assert g.view["rows_capacity"] == g.windows.shape[0] // o.plan.o.shape[1]
+        assert np.array_equal(g.view["rows"].astype(np.int64), o.slots)
+    else:
+        assert g.view["rows"] is None and g.view["rows_capacity"] == -1
     E, R = o.plan.o.shape
     st, want_start, want_count = oracle.expert_ranges(E, R, g.windows.shape[0] // R, o.plan.n_exp, align=align)
     assert st == oracle.OK and np.array_equal(g.expert_start, want_start) and np.array_equal(g.expert_count, want_count)

@@ -441,7 +441,8 @@ def test_option_values_are_validated():
                              (binding.MOE_OPT_TEST_STARVE_WAIT_MS, [0], [-1, 10001]),
                              (binding.MOE_OPT_OVERLAP, [0, 1], [-1, 2]),
                              (binding.MOE_OPT_EXPERT_ALIGN, [1, 128, 4096], [0, -5, 4097]),
-                             (binding.MOE_OPT_CLUSTER_PLAN, [0, 1], [-1, 2])]:
+                             (binding.MOE_OPT_CLUSTER_PLAN, [0, 1], [-1, 2]),
+                             (binding.MOE_OPT_SLOT_REUSE, [0, 1], [-1, 2])]:
         for v in wrong:
             assert comm.moe_set_option(opt, v, check=False) == bad, (opt, v)
         for v in good:
