@@ -52,6 +52,9 @@ NCU_TRAFFIC_BYTES = {
     # 201 MB workloads, L2 flushed before the launch: part of what the kernel writes is still dirty in L2 at its end
     ("dispatch_bulk_kernel", "c5_mixtral_T8192_prefill"): 67.3e6 + 76.0e6,
     ("combine_rows_kernel", "c5_mixtral_T8192_prefill"): 134.4e6 + 12.4e6,
+    # full size, one launch each (read + write)
+    ("dispatch_bulk_kernel", "c5_mixtral_T65536_prefill"): 538.0e6 + 1015.1e6,
+    ("combine_rows_kernel", "c5_mixtral_T65536_prefill"): 1074.8e6 + 504.7e6,
 }
 
 WORKLOADS = {
