@@ -64,6 +64,10 @@ def test_per_rank_contexts_and_separate_windows_reproduce_the_global_result(case
         v = c.moe_plan_view()
         assert np.array_equal(v["large_off"].cpu().numpy(), p.o) and np.array_equal(v["n_recv"].cpu().numpy(), p.n_recv)
         assert np.array_equal(v["small_off"].cpu().numpy(), p.s[rts[r]:rts[r + 1]])
+        # the rows this rank's dispatch recorded for its combine: the global numbering d*C + row in window d
+        if rts[r + 1] > rts[r]:
+            assert v["rows_capacity"] == C
+            assert np.array_equal(v["rows"].cpu().numpy().astype(np.int64), want.slots[rts[r]:rts[r + 1]])
     got = torch.cat(windows).cpu().view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(got, want.windows)
     # experts (harness op on the concatenated view), then every rank combines its own tokens from all windows
