@@ -302,6 +302,16 @@ void launch_kernel(void (*kernel)(KArgs...), int grid, int threads, int smem, cu
   cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Dynamic shared memory to ask for when a one-CTA-per-SM kernel is launched behind a planner with programmatic
+// stream serialization.  Its CTAs are placed while the planner's CTAs still hold their SMs, and CTAs that are small
+// enough to fit two per SM then double up on some SMs and leave others without any for the whole launch: with
+// the two-warp CTAs (86 KB) of a large job of 14 KB rows, plan + dispatch as one call took 870 us against 663 us
+// as two calls at 32768 tokens (229 against 181 us at 8192, 79.7 against 72.4 us at 3072).  Asking for more
+// than half an SM's shared memory keeps it at one CTA per SM (661, 179 and 71.6 us); the kernels take their layout
+// from the warp count, not from the size of the allocation.
+constexpr int SOLO_SMEM_BYTES = 120 * 1024;
+int solo_smem(int smem, bool pdl) { return (pdl && smem < SOLO_SMEM_BYTES) ? SOLO_SMEM_BYTES : smem; }
+
 // Bulk-copy path: one CTA per SM; each warp drives a ring of BULK_STAGES stages, and the CTA has as
 // many warps (up to BULK_MAX_WARPS) as fit their rings into the shared-memory budget: 4 for 14 KB
 // rows, 8 for rows of 8 KB or less (short rows need more requests in flight to cover the latency).
@@ -340,19 +350,13 @@ void launch_dispatch_bulk(moe_ctx* ctx, const RowArgs& a, const uint4* x, uint4*
       set_work(ctx, c, (int64_t)grid * fewer, g_max);
       // (the cut of the rows changes with the warp count: taken only if the rounds come out at least nine tenths
       // full -- 1280 rows of 8 KB are better off with eight warps and their leftover rows cut finer)
-      // Behind the planner the rule is left alone for CTAs small enough to fit two per SM: the planner's CTAs
-      // still hold their SMs when the dispatch CTAs are placed, so some SMs get two of them, and with the
-      // full warp count the CTAs placed last are the idle ones (plan + dispatch + combine at 16 / 32 tokens
-      // per rank of 8 KB rows: 17.2 / 23.1 us back to back without the rule, 18.9 / 25.7 us with it).
-      const bool doubles_up = pdl && 2 * fewer * BULK_STAGES * (c.granule * 512 + 8) <= BULK_SMEM_BUDGET;
-      if (!doubles_up && (int64_t)c.n_items <= rounds * grid * fewer &&
-          (int64_t)c.n_items * 10 >= rounds * grid * fewer * 9) {
+      if ((int64_t)c.n_items <= rounds * grid * fewer && (int64_t)c.n_items * 10 >= rounds * grid * fewer * 9) {
         b = c;
         warps = fewer;
       }
     }
   }
-  const int smem = warps * BULK_STAGES * (b.granule * 512 + 8);
+  const int smem = solo_smem(warps * BULK_STAGES * (b.granule * 512 + 8), pdl);
   b.pdl = pdl;
   launch_kernel(dispatch_bulk_kernel, grid, warps * 32, smem, st, pdl, 0, reinterpret_cast<const unsigned char*>(x),
                 reinterpret_cast<unsigned char*>(win), b, ctx->map);
@@ -940,7 +944,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
     set_work(ctx, a, (int64_t)grid * warps, upr, false);
     ctx->granule_override = keep;
     auto launch = [&](auto kernel) {
-      launch_kernel(kernel, grid, warps * 32, warps * per_warp, static_cast<cudaStream_t>(stream), pdl, 0,
+      launch_kernel(kernel, grid, warps * 32, solo_smem(warps * per_warp, pdl), static_cast<cudaStream_t>(stream), pdl, 0,
                     static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
     };
     if (cpl == 16) {
@@ -959,7 +963,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   ctx->granule_override = upr;
   set_work(ctx, a, (int64_t)grid * warps, upr, false);
   ctx->granule_override = keep;
-  const int smem = warps * (stages * (stage + 8) + per_warp_extra);
+  const int smem = solo_smem(warps * (stages * (stage + 8) + per_warp_extra), pdl);
   auto launch = [&](auto kernel) {
     launch_kernel(kernel, grid, warps * 32, smem, static_cast<cudaStream_t>(stream), pdl, 0,
                   static_cast<const unsigned char*>(x), static_cast<unsigned char*>(windows_q), scales, a, ctx->map);
