@@ -367,8 +367,10 @@ void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const floa
   // Jobs that read several times the L2 capacity take the L1-allocating loads (see ld_row).
   // Windows addressed through a table of bases (other GPUs' memory) are read with coherent loads.
   const bool peers = a.win_base != nullptr;
-  const bool large = !peers && (int64_t)a.t_count * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
-  auto kernel = peers ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_PEER>
+  const bool many_bytes = (int64_t)a.t_count * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
+  const bool large = !peers && many_bytes;
+  auto kernel = peers ? (many_bytes ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_PEER_L1>
+                                    : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_PEER>)
                 : large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_L1>
                         : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_STREAM>;
   const int grid = row_grid(ctx, kernel, a.t_count);

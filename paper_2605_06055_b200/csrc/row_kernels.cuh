@@ -146,7 +146,8 @@ __device__ __forceinline__ void warm(const int32_t* p) {
 __device__ __forceinline__ unsigned char* window_row(const RowArgs& a, const void* windows, int64_t row,
                                                      size_t row_bytes) {
   if (a.win_base == nullptr) return (unsigned char*)windows + (size_t)row * row_bytes;
-  const int64_t d = row / a.C;
+  // (rows below 2^32 -- every realistic window -- take the 32-bit division: the 64-bit one is a long subroutine)
+  const int64_t d = (uint64_t)(row | a.C) >> 32 ? row / a.C : (int64_t)((uint32_t)row / (uint32_t)a.C);
   return (unsigned char*)a.win_base[d] + (size_t)(row - d * a.C) * row_bytes;
 }
 
@@ -166,11 +167,13 @@ __device__ __forceinline__ bool must_abort(const RowArgs& a) {
 // kernel runs.  LD_STREAM marks the line "no allocate" in L1, LD_L1 lets it allocate.  Neither data is ever
 // re-read, but measured on B200 the allocating form is 3 % faster for combine at prefill sizes (617 vs 637 us)
 // and 10 % slower at decode sizes (55 vs 49 us), so the launcher picks by job size.
-// LD_PEER: ordinary (coherent) loads, for windows addressed through a table of bases -- other GPUs' memory that
-// other GPUs' kernels write.  They are valid whenever the reading kernel is ordered after the writers'
+// LD_PEER, LD_PEER_L1: ordinary (coherent) loads, for windows addressed through a table of bases -- other GPUs'
+// memory that other GPUs' kernels write.  They are valid whenever the reading kernel is ordered after the writers'
 // completion (a host barrier, or a preceding wait on arrival flags, followed by this launch), which the
-// non-coherent path does not promise once such ordering is established on the device.
-enum { LD_STREAM = 0, LD_L1 = 1, LD_PEER = 2 };
+// non-coherent path does not promise once such ordering is established on the device.  The same choice by job
+// size: LD_PEER does not allocate in L1, LD_PEER_L1 does (one GPU, every window behind the table: 51.3 against
+// 55.1 us at the decode shape, 637 against 613 us at 32768 tokens).
+enum { LD_STREAM = 0, LD_L1 = 1, LD_PEER = 2, LD_PEER_L1 = 3 };
 template <int MODE>
 __device__ __forceinline__ uint4 ld_row(const uint4* p) {
   uint4 v;
@@ -178,6 +181,9 @@ __device__ __forceinline__ uint4 ld_row(const uint4* p) {
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   else if constexpr (MODE == LD_PEER)
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  else if constexpr (MODE == LD_PEER_L1)
     asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   else
@@ -398,6 +404,13 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
     meta_ready = a.prefetch_meta != 0;   // from the second item on, only the prefetching form has it in hand
     const int64_t slot = finish_slot(a, map, meta, wi.t, lane, false);
     const float w_lane = meta.w;
+    // Lane j turns its own branch's row into an address once (with a table of bases: one division and one table
+    // entry per lane, side by side, instead of K of each one after the other in every lane); the addresses are
+    // what the lanes exchange.
+    // (lanes without a branch resolve row 0 and drop the result: no divergent path in front of the loads)
+    const unsigned long long any_addr =
+        reinterpret_cast<unsigned long long>(window_row(a, windows, slot >= 0 ? slot : 0, (size_t)H16 * 16));
+    const unsigned long long row_addr = slot >= 0 ? any_addr : 0ull;
     // short rows: the next item's routing index, small offset and weight travel while this item is reduced
     if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item<MODE != LD_L1>(a, next_item).t, lane);
     item = next_item;
@@ -407,8 +420,12 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
       float w[KT];
 #pragma unroll
       for (int j = 0; j < KT; ++j) {
-        const int64_t row = __shfl_sync(0xffffffffu, slot, j);
-        src[j] = row >= 0 ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
+        if constexpr (KT <= 2) {   // one or two rows: every lane resolving them itself measured 1-3 % faster
+          const int64_t row = __shfl_sync(0xffffffffu, slot, j);
+          src[j] = row >= 0 ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
+        } else {
+          src[j] = reinterpret_cast<const uint4*>(__shfl_sync(0xffffffffu, row_addr, j));
+        }
         w[j] = __shfl_sync(0xffffffffu, w_lane, j);
       }
       for (int i = wi.i0; i < wi.i1; i += UNROLL) {
@@ -448,10 +465,9 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
 #pragma unroll
           for (int jj = 0; jj < 8; ++jj) {
             const int j = jc + jj;
-            const int64_t row = __shfl_sync(0xffffffffu, slot, j & 31);
+            const unsigned long long addr = __shfl_sync(0xffffffffu, row_addr, j & 31);
             wv[jj] = __shfl_sync(0xffffffffu, w_lane, j & 31);
-            const uint4* src =
-                (j < K && row >= 0) ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
+            const uint4* src = j < K ? reinterpret_cast<const uint4*>(addr) : nullptr;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u)
               v[u][jj] = (ok[u] && src != nullptr) ? ld_row<MODE>(src + (i + u) * 32 + lane)
