@@ -488,7 +488,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
        opt_in(dispatch_quant_reg_kernel<32, true, true>) && opt_in(dispatch_quant_reg_kernel<32, false, true>) &&
        opt_in(dispatch_quant_reg_kernel<32, true, false>) && opt_in(dispatch_quant_reg_kernel<32, false, false>) &&
        opt_in(plan_rank_kernel<32>) &&
-       opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_kernel) &&
+       opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_rank_kernel) &&
        opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0, false>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
   const int rank_smem =
@@ -620,9 +620,11 @@ void launch_gate(const float* logits, int32_t T, int32_t E, int32_t K, int32_t* 
 }
 
 // Planning, optionally with the gate in front (logits != nullptr: topk_idx and topk_w are OUTPUTS).
+// local_rank >= 0: only that rank owns tokens and only its local part is wanted (its small offsets and its row of
+// M; moe_layout) -- one CTA instead of R and no Notify step.
 moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* topk_idx, int32_t T,
                        const int32_t* rank_tok_start, void* stream, const float* logits, int32_t* idx_out,
-                       float* w_out) {
+                       float* w_out, int32_t local_rank = -1) {
   if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
   const moe_shape_t& sh = ctx->shape;
   if (schedule != MOE_SCHED_PREFILL && schedule != MOE_SCHED_DECODE) return MOE_ERR_INVALID_ARG;
@@ -674,6 +676,7 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
   }
   ctx->compact_plan = max_rank_branches <= RANK_PLAN_MAX_BRANCHES;
   const bool wide = sh.E <= RANK_PLAN_WIDE_MAX_E;
+  bool split_notify = false;
   int n = 0;
   if (logits != nullptr) {   // gate first (its own launch, spread over all SMs), then plan from the indexes it wrote
     launch_gate(logits, T, sh.E, sh.K, idx_out, w_out, ctx->num_sms, ctx->device, st);
@@ -682,19 +685,25 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
   if (ctx->compact_plan) {
     // One CTA per source rank.  When the R CTAs can run as one thread-block cluster, the Notify step reads
     // the count rows from the CTAs' shared memory and every CTA builds its own window's offsets.
-    const bool as_cluster = ctx->cluster_plan && ctx->plan_cluster_ok;
+    const bool local = local_rank >= 0;
+    const bool as_cluster = !local && ctx->cluster_plan && ctx->plan_cluster_ok;
     const int threads = (wide ? 32 : 8) * 32;
     const int smem = rank_smem + (as_cluster ? cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t) : 0);
-    const int32_t flag = as_cluster ? 1 : 0;
+    // More ranks than a cluster holds: the last CTA alone would build E x R offsets (20 us at R = 64), so the
+    // CTAs only count and a second launch builds every window's offsets side by side.
+    split_notify = !local && !as_cluster && sh.R > 16;
+    const int32_t mode = (local || split_notify) ? PLAN_LOCAL : as_cluster ? PLAN_CLUSTER : PLAN_TICKET;
+    const int ctas = local ? 1 : sh.R;
+    const int32_t first = local ? local_rank : 0;
     const bool behind_gate = logits != nullptr && ctx->overlap != 0;
     if (wide)
-      launch_kernel(plan_rank_kernel<32>, sh.R, threads, smem, st, behind_gate, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
+      launch_kernel(plan_rank_kernel<32>, ctas, threads, smem, st, behind_gate, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
                     (int32_t)full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
-                    ctx->ctl, flag);
+                    ctx->ctl, mode, first);
     else
-      launch_kernel(plan_rank_kernel<8>, sh.R, threads, smem, st, behind_gate, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
+      launch_kernel(plan_rank_kernel<8>, ctas, threads, smem, st, behind_gate, as_cluster ? sh.R : 0, topk_idx, map, sh.K, sh.E,
                     (int32_t)full, ctx->expert_align, ctx->s, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
-                    ctx->ctl, flag);
+                    ctx->ctl, mode, first);
     ++n;
   } else {
     if (tiles > 0) {
@@ -712,18 +721,27 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
     // kernel's index loads) overlap the kernel in front.  The scan kernel's R CTAs run as one cluster when
     // the device can co-schedule them (see cluster_notify).
     const bool chain = ctx->overlap != 0;
-    const bool scan_cluster = ctx->cluster_plan && ctx->scan_cluster_ok;
+    const bool local = local_rank >= 0;
+    const bool scan_cluster = !local && ctx->cluster_plan && ctx->scan_cluster_ok;
+    split_notify = !local && !scan_cluster && sh.R > 16;
     const int scan_bytes =
         scan_cluster ? (sh.E + cluster_notify_smem_ints(sh.E, sh.R)) * (int)sizeof(int32_t) : scan_smem;
-    launch_kernel(plan_scan_kernel, sh.R, PLAN_THREADS, scan_bytes, st, chain && tiles > 0, scan_cluster ? sh.R : 0,
-                  ctx->tile_hist, map, sh.E, (int32_t)full, ctx->expert_align, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp,
-                  ctx->n_recv, ctx->ctl, (int32_t)(scan_cluster ? 1 : 0));
+    launch_kernel(plan_scan_kernel, local ? 1 : sh.R, PLAN_THREADS, scan_bytes, st, chain && tiles > 0,
+                  scan_cluster ? sh.R : 0, ctx->tile_hist, map, sh.E, (int32_t)full, ctx->expert_align, ctx->M,
+                  ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv, ctx->ctl,
+                  (int32_t)((local || split_notify) ? PLAN_LOCAL : scan_cluster ? PLAN_CLUSTER : PLAN_TICKET),
+                  (int32_t)(local ? local_rank : 0));
     ++n;
     if (full && tiles > 0) {
       launch_kernel(plan_finalize_kernel<ROUNDS_PREFILL>, tiles, PLAN_THREADS, 0, st, chain, 0, topk_idx, map, sh.K, sh.E,
                     ctx->tile_rank, ctx->tile_hist, ctx->s);
       ++n;
     }
+  }
+  if (split_notify) {
+    notify_rank_kernel<<<sh.R, 256, cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t), st>>>(
+        ctx->M, sh.E, sh.R, (int32_t)full, ctx->expert_align, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv);
+    ++n;
   }
   const moe_status_t rc = launch_ok(ctx, n);
   if (rc == MOE_OK) ctx->planned = true;
@@ -1098,7 +1116,7 @@ moe_status_t moe_layout(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* 
   if (T_local > 0 && topk_idx == nullptr) return MOE_ERR_INVALID_ARG;
   int32_t starts[MOE_MAX_R + 1];
   for (int r = 0; r <= ctx->shape.R; ++r) starts[r] = r <= my_rank ? 0 : T_local;   // only my_rank owns tokens
-  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T_local, starts, stream, nullptr, nullptr, nullptr);
+  const moe_status_t rc = plan_impl(ctx, schedule, topk_idx, T_local, starts, stream, nullptr, nullptr, nullptr, my_rank);
   if (rc != MOE_OK) return rc;
   ctx->planned = false;   // the offsets are not valid until moe_notify has seen every rank's counts
   ctx->slots_for_C = -1;
@@ -1113,7 +1131,8 @@ moe_status_t moe_notify(moe_ctx_t* ctx, const int32_t* counts_all, void* stream)
   if (ctx == nullptr || counts_all == nullptr) return MOE_ERR_INVALID_ARG;
   if (!ctx->layout_done) return MOE_ERR_NOT_PLANNED;
   const moe_shape_t& sh = ctx->shape;
-  notify_kernel<<<1, 1024, notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t), static_cast<cudaStream_t>(stream)>>>(
+  notify_rank_kernel<<<sh.R, 256, cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t),
+                       static_cast<cudaStream_t>(stream)>>>(
       counts_all, sh.E, sh.R, ctx->schedule == MOE_SCHED_PREFILL, ctx->expert_align, ctx->M, ctx->c_rank, ctx->o,
       ctx->n_exp, ctx->n_recv);
   const moe_status_t rc = launch_ok(ctx);
@@ -1664,7 +1683,7 @@ extern "C" moe_status_t moe_slots_noalloc(const int32_t* topk_idx, int32_t T, in
     plan_tile_kernel<ROUNDS_DECODE><<<tiles, PLAN_THREADS, PLAN_WARPS * E * (int)sizeof(int32_t), st>>>(
         topk_idx, map, K, E, sc->tile_rank, sc->tile_hist, status);
   plan_scan_kernel<<<R, PLAN_THREADS, notify_smem_ints(E, R) * (int)sizeof(int32_t), st>>>(
-      sc->tile_hist, map, E, 0, 1, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl, 0);
+      sc->tile_hist, map, E, 0, 1, sc->M, sc->c_rank, sc->o, sc->n_exp, n_recv, &sc->ctl, PLAN_TICKET, 0);
   RowArgs a = {};   // every field the kernel is handed has a defined value
   a.topk_idx = topk_idx;
   a.small_off = sc->tile_rank;

@@ -257,6 +257,10 @@ __host__ __device__ constexpr int cluster_notify_smem_ints(int E, int R) {
   return (E / R) * (R + 1) + 2 * (E / R) + 1 + 33;
 }
 
+// How the planners' Notify step runs: by the last CTA to finish (a ticket), by every CTA of a cluster for its own
+// window, or not at all (one rank's local part of a multi-rank plan: moe_layout).
+enum { PLAN_TICKET = 0, PLAN_CLUSTER = 1, PLAN_LOCAL = 2 };
+
 // The two halves of a cluster barrier.  Between them a CTA does what needs nobody else's data (arrive has release,
 // wait has acquire semantics: what a CTA wrote to its shared memory before arriving is visible to the others after
 // their wait).  Every thread of every CTA of the cluster executes each of them once per phase.
@@ -266,29 +270,18 @@ __device__ __forceinline__ void cluster_wait() { __cluster_barrier_wait(); }
 // (The releasing form waits until this thread's earlier global stores are visible, which is not wanted there.)
 __device__ __forceinline__ void cluster_arrive_relaxed() { __cluster_barrier_arrive_relaxed(); }
 
-// On entry every thread of the CTA has ARRIVED at the cluster barrier that says "my row of M is complete".
-__device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, [E] */, int32_t* scratch, int32_t E,
-                                               int32_t R, int32_t d, int32_t full_table, int32_t align,
-                                               int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+// Offsets of ONE window (rank d: its E/R experts x R source ranks) from the gathered tile of counts; every thread
+// of the CTA calls it after the tile is complete (a __syncthreads behind the gather).
+// scratch: cluster_notify_smem_ints(E, R) ints: tile [E/R][R+1] with entry (el, rr) = M[rr][d*E/R + el], padded
+// totals [E/R], their prefix [E/R + 1], warp sums [33].
+__device__ __forceinline__ void window_offsets(int32_t* scratch, int32_t E, int32_t R, int32_t d, int32_t full_table,
+                                               int32_t align, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
                                                int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
-  namespace cg = cooperative_groups;
-  cg::cluster_group cluster = cg::this_cluster();
   const int E_r = E / R, P = R + 1, nthreads = (int)blockDim.x, tid = (int)threadIdx.x;
-  int32_t* tile = scratch;            // [E_r][P]: entry (el, rr) = M[rr][d*E_r + el]
+  int32_t* tile = scratch;
   int32_t* tot = tile + E_r * P;      // [E_r] rows each expert's run occupies
   int32_t* pre = tot + E_r;           // [E_r + 1]
   int32_t* warp_sums = pre + E_r + 1;
-  cluster_wait();                     // every CTA's row of M is complete and visible
-  for (int q = tid; q < E_r * R; q += nthreads) {   // consecutive threads: consecutive experts of one remote row
-    const int el = q % E_r, rr = q / E_r;
-    const int32_t* remote = cluster.map_shared_rank(my_row, rr);
-    tile[el * P + rr] = remote[d * E_r + el];
-  }
-  // This thread reads no other CTA's shared memory from here on.  Its remote loads have returned -- the stores
-  // above carry their values -- and the barrier orders nothing else, so the arrival need not release anything
-  // (a releasing arrival here waits for the s and M stores to drain: 0.3 us).
-  cluster_arrive_relaxed();
-  __syncthreads();
   if (full_table) {
     for (int rr = tid; rr < R; rr += nthreads) {     // branches from source rank rr to this rank
       int32_t acc = 0;
@@ -344,6 +337,29 @@ __device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, 
   for (int q = tid; q < E_r * R; q += nthreads)      // o[d*E_r + el][rr], one coalesced stream
     o[(size_t)d * E_r * R + q] = pre[q / R] + tile[(q / R) * P + q % R];
   if (tid == 0) n_recv[d] = pre[E_r];
+}
+
+// On entry every thread of the CTA has ARRIVED at the cluster barrier that says "my row of M is complete".
+__device__ __forceinline__ void cluster_notify(const int32_t* my_row /* shared, [E] */, int32_t* scratch, int32_t E,
+                                               int32_t R, int32_t d, int32_t full_table, int32_t align,
+                                               int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+                                               int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int E_r = E / R, P = R + 1, nthreads = (int)blockDim.x, tid = (int)threadIdx.x;
+  int32_t* tile = scratch;            // [E_r][P]: entry (el, rr) = M[rr][d*E_r + el]
+  cluster_wait();                     // every CTA's row of M is complete and visible
+  for (int q = tid; q < E_r * R; q += nthreads) {   // consecutive threads: consecutive experts of one remote row
+    const int el = q % E_r, rr = q / E_r;
+    const int32_t* remote = cluster.map_shared_rank(my_row, rr);
+    tile[el * P + rr] = remote[d * E_r + el];
+  }
+  // This thread reads no other CTA's shared memory from here on.  Its remote loads have returned -- the stores
+  // above carry their values -- and the barrier orders nothing else, so the arrival need not release anything
+  // (a releasing arrival here waits for the s and M stores to drain: 0.3 us).
+  cluster_arrive_relaxed();
+  __syncthreads();
+  window_offsets(scratch, E, R, d, full_table, align, c_rank, o, n_exp, n_recv);
   cluster_wait();                     // no CTA leaves while its row may still be read
 }
 
@@ -352,13 +368,15 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
                  const __grid_constant__ RankMap map, int32_t E, int32_t full_table, int32_t align,
                  int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
                  int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl,
-                 int32_t as_cluster /* the grid is one thread-block cluster of R CTAs */) {
+                 int32_t mode /* PLAN_TICKET, PLAN_CLUSTER (the grid is one cluster of R CTAs) or PLAN_LOCAL */,
+                 int32_t first_rank /* rank of CTA 0 (PLAN_LOCAL: the grid is the one CTA of the rank that owns tokens) */) {
   // notify_smem_ints(E, R) ints, or (as a cluster) this CTA's row of M [E] followed by cluster_notify_smem_ints(E, R)
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
   release_dependents();   // lets the kernel behind (finalize, or a dispatch) be scheduled; it waits for this one
   dependency_wait();      // the tile histograms are complete (returns at once under a plain launch)
-  const int r = blockIdx.x;
+  const bool as_cluster = mode == PLAN_CLUSTER;
+  const int r = blockIdx.x + first_rank;
   const int R = map.R;
   const int t0 = map.tile_start[r], t1 = map.tile_start[r + 1];
 
@@ -384,6 +402,7 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
     cluster_notify(sm, sm + E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
     return;
   }
+  if (mode == PLAN_LOCAL) return;   // this rank's row of M and its tile bases are all that was asked for
 
   // Last block done: the final CTA to arrive sees every row of M.
   __threadfence();
@@ -415,9 +434,10 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
                  int32_t full_table, int32_t align, int32_t* __restrict__ s, int32_t* __restrict__ M,
                  int32_t* __restrict__ c_rank,
                  int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl,
-                 int32_t as_cluster /* the grid is one thread-block cluster of R CTAs */) {
+                 int32_t mode /* PLAN_TICKET, PLAN_CLUSTER or PLAN_LOCAL, see plan_scan_kernel */, int32_t first_rank) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
+  const bool as_cluster = mode == PLAN_CLUSTER;
   // Behind the gate kernel (moe_gate_plan) this kernel may have been scheduled early: the routing indexes
   // are complete once the wait returns (at once under a plain launch).
   dependency_wait();
@@ -428,7 +448,7 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   constexpr int P = WARPS + 1;
   int32_t* counts = sm;             // [E][P]
   int32_t* rank_base = sm + P * E;  // [E]
-  const int r = blockIdx.x, R = map.R;
+  const int r = blockIdx.x + first_rank, R = map.R;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int32_t b_begin = map.tok_start[r] * K, b_end = map.tok_start[r + 1] * K;
   const unsigned lt = lanemask_lt();
@@ -483,6 +503,7 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
     cluster_notify(rank_base, sm + (P + 1) * E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
     return;
   }
+  if (mode == PLAN_LOCAL) return;   // s and this rank's row of M: the offsets come from moe_notify
 
   __threadfence();
   __syncthreads();
@@ -494,17 +515,26 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
   if (threadIdx.x == 0) ctl->scan_ticket = 0;
 }
 
-// Notify from a count matrix gathered elsewhere (multi-rank use: every rank contributed its row):
-// installs it as M and rebuilds the large offsets and receive counts.  One CTA.
-__global__ void __launch_bounds__(1024)
-notify_kernel(const int32_t* __restrict__ counts_all, int32_t E, int32_t R, int32_t full_table, int32_t align,
-              int32_t* __restrict__ M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
-              int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
+// Notify from a count matrix gathered elsewhere (multi-rank use: every rank contributed its row): installs it as M
+// and rebuilds the large offsets and receive counts.  R CTAs, one per window: the gathered matrix is complete in
+// global memory before the launch, so CTA d takes its E/R columns of every row straight from there (and copies
+// row d into M) -- no CTA waits for another and the time does not grow with R (a single CTA building every window
+// took 4.2 us at R = 8 and 16.5 us at R = 64).
+// Dynamic shared memory: cluster_notify_smem_ints(E, R) ints.
+__global__ void __launch_bounds__(256)
+notify_rank_kernel(const int32_t* counts_all, int32_t E, int32_t R, int32_t full_table, int32_t align,
+                   int32_t* M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+                   int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv) {
   extern __shared__ int32_t sm[];
-  for (int i = threadIdx.x; i < R * E; i += blockDim.x) M[i] = counts_all[i];
-  __threadfence_block();
+  const int d = blockIdx.x, E_r = E / R, P = R + 1;
+  for (int q = threadIdx.x; q < E_r * R; q += (int)blockDim.x) {   // consecutive threads: consecutive experts of one row
+    const int el = q % E_r, rr = q / E_r;
+    sm[el * P + rr] = counts_all[(size_t)rr * E + d * E_r + el];
+  }
+  if (counts_all != M)   // (the planners of one GPU call this on M itself when R is too large for a cluster)
+    for (int e = threadIdx.x; e < E; e += (int)blockDim.x) M[(size_t)d * E + e] = counts_all[(size_t)d * E + e];
   __syncthreads();
-  build_large_offsets(M, E, R, full_table, align, c_rank, o, n_exp, n_recv, sm);
+  window_offsets(sm, E, R, d, full_table, align, c_rank, o, n_exp, n_recv);
 }
 
 template <int ROUNDS>

@@ -92,6 +92,10 @@ EDGE = [
     ("duplicates_in_token", 333, 72, 4, 2, 4, "replace", (300, 33)),
     ("empty_rank_ragged", 1000, 256, 32, 4, 8, "uniform", (0, 517, 0, 483)),
     ("many_ranks", 512, 64, 256, 64, 8, "uniform", None),
+    # more ranks than a cluster holds: the counting CTAs are followed by a launch that builds every window's offsets
+    ("many_ranks_tiles", 19200, 32, 64, 32, 8, "uniform", None),           # 4800 branches per rank: tile planner
+    ("max_ranks", 768, 64, 256, 256, 2, "uniform", None),                  # R = 256, one expert per rank
+    ("many_ranks_ragged", 3000, 40, 96, 48, 4, "zipf", tuple([0, 125] * 24)),
     ("big_E", 3000, 32, 2048, 2, 8, "uniform", None),
     ("tile_boundary_exact", 2048, 32, 8, 2, 2, "uniform", None),   # 2048 branches per rank = exactly two tiles
     ("tile_boundary_plus1", 2050, 32, 8, 2, 2, "uniform", None),
