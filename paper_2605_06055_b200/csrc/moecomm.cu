@@ -259,7 +259,7 @@ int row_grid(moe_ctx* ctx, Kernel kernel, int64_t tokens) {
 // CTA per SM with about 32 16-byte loads per lane) measured faster than many thin ones: every warp
 // then streams long contiguous runs of each row, which HBM serves with far fewer page switches.
 constexpr int combine_unroll(int K) {
-  return K >= 16 ? 2 : K >= 9 ? 3 : K >= 7 ? 4 : K >= 6 ? 5 : K == 5 ? 6 : K == 4 ? 8 : K == 3 ? 10 : 16;
+  return K >= 17 ? 1 : K >= 16 ? 2 : K >= 9 ? 3 : K >= 7 ? 4 : K >= 6 ? 5 : K == 5 ? 6 : K == 4 ? 8 : K == 3 ? 10 : 16;
 }
 constexpr int DISPATCH_UNROLL = 14;
 
@@ -369,10 +369,10 @@ void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const floa
   const bool peers = a.win_base != nullptr;
   const bool many_bytes = (int64_t)a.t_count * ctx->shape.K * ctx->shape.H * 2 >= ((int64_t)512 << 20);
   const bool large = !peers && many_bytes;
-  auto kernel = peers ? (many_bytes ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_PEER_L1>
-                                    : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_PEER>)
-                : large ? combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_L1>
-                        : combine_rows_kernel<KT, (KT > 0 ? combine_unroll(KT) : 4), LD_STREAM>;
+  auto kernel = peers ? (many_bytes ? combine_rows_kernel<KT, combine_unroll(KT > 0 ? KT : -KT), LD_PEER_L1>
+                                    : combine_rows_kernel<KT, combine_unroll(KT > 0 ? KT : -KT), LD_PEER>)
+                : large ? combine_rows_kernel<KT, combine_unroll(KT > 0 ? KT : -KT), LD_L1>
+                        : combine_rows_kernel<KT, combine_unroll(KT > 0 ? KT : -KT), LD_STREAM>;
   const int grid = row_grid(ctx, kernel, a.t_count);
   RowArgs b = a;
   int warps = 8;
@@ -392,7 +392,7 @@ void launch_combine(moe_ctx* ctx, const RowArgs& a, const uint4* win, const floa
     }
   }
   // an item that is one or two batches of loads cannot hide its own metadata latency: prefetch it
-  constexpr int unroll = KT > 0 ? combine_unroll(KT) : 4;
+  constexpr int unroll = combine_unroll(KT > 0 ? KT : -KT);
   b.prefetch_meta = (b.granule + unroll - 1) / unroll <= 2;
   kernel<<<grid, warps * 32, 0, st>>>(win, w, y, b, ctx->map);
 }
@@ -1081,7 +1081,11 @@ moe_status_t combine_impl(moe_ctx* ctx, const void* windows, const void* const* 
     case 10: launch_combine<10>(ctx, a, win, topk_w, ys, st); break;
     case 12: launch_combine<12>(ctx, a, win, topk_w, ys, st); break;
     case 16: launch_combine<16>(ctx, a, win, topk_w, ys, st); break;
-    default: launch_combine<0>(ctx, a, win, topk_w, ys, st); break;
+    default:   // the other degrees share three kernels: up to 16, 24 or 32 branches, K of them live
+      if (ctx->shape.K <= 16) launch_combine<-16>(ctx, a, win, topk_w, ys, st);
+      else if (ctx->shape.K <= 24) launch_combine<-24>(ctx, a, win, topk_w, ys, st);
+      else launch_combine<-32>(ctx, a, win, topk_w, ys, st);
+      break;
   }
   return launch_ok(ctx);
 }

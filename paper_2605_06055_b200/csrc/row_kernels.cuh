@@ -372,6 +372,7 @@ __global__ void __launch_bounds__(256, 1)
 combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__ topk_w, uint4* __restrict__ Y,
                     const RowArgs a, const __grid_constant__ RankMap map) {
   const int lane = threadIdx.x & 31;
+  constexpr int KMAX = KT > 0 ? KT : -KT;
   const int K = KT > 0 ? KT : a.K;
   const int H16 = a.H16;
   ItemFeed feed = begin_feed();
@@ -415,73 +416,43 @@ combine_rows_kernel(const uint4* __restrict__ windows, const float* __restrict__
     if (a.prefetch_meta && next_item < a.n_items) meta = load_meta(a, topk_w, decode_item<MODE != LD_L1>(a, next_item).t, lane);
     item = next_item;
     uint4* out = Y + (size_t)wi.t * H16;
-    if constexpr (KT > 0) {
-      const uint4* src[KT];
-      float w[KT];
+    {
+      // KT > 0: exactly KT branches.  KT < 0: up to KMAX = -KT branches, K of them live (the degrees without a kernel
+      // of their own); the others hold a null address and are skipped, loads and fma alike, so the chain of the
+      // live ones is the same.  (A form that fetched addresses and weights by shuffles inside the row loop, eight
+      // branches at a time, ran at 1.6-1.75 TB/s whatever K: 417 us against 110 us for K = 9 at 8192 rows of 8 KB.)
+      const uint4* src[KMAX];
+      float w[KMAX];
 #pragma unroll
-      for (int j = 0; j < KT; ++j) {
-        if constexpr (KT <= 2) {   // one or two rows: every lane resolving them itself measured 1-3 % faster
+      for (int j = 0; j < KMAX; ++j) {
+        if constexpr (KT > 0 && KT <= 2) {   // one or two rows: every lane resolving them itself measured 1-3 % faster
           const int64_t row = __shfl_sync(0xffffffffu, slot, j);
           src[j] = row >= 0 ? reinterpret_cast<const uint4*>(window_row(a, windows, row, (size_t)H16 * 16)) : nullptr;
         } else {
           src[j] = reinterpret_cast<const uint4*>(__shfl_sync(0xffffffffu, row_addr, j));
         }
         w[j] = __shfl_sync(0xffffffffu, w_lane, j);
+        if (KT < 0 && j >= K) src[j] = nullptr;
       }
       for (int i = wi.i0; i < wi.i1; i += UNROLL) {
-        uint4 v[UNROLL][KT];
+        uint4 v[UNROLL][KMAX];
         bool ok[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
           const int c = (i + u) * 32 + lane;
           ok[u] = (i + u < wi.i1) && (c < H16);
 #pragma unroll
-          for (int j = 0; j < KT; ++j)
+          for (int j = 0; j < KMAX; ++j)
             v[u][j] = (ok[u] && src[j] != nullptr) ? ld_row<MODE>(src[j] + c) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
           float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int j = 0; j < KT; ++j) fma_bf16x8(acc, w[j], v[u][j]);   // j ascending, one fma per term
+          for (int j = 0; j < KMAX; ++j)
+            if (KT > 0 || j < K) fma_bf16x8(acc, w[j], v[u][j]);   // j ascending, one fma per term
           if (ok[u]) out[(i + u) * 32 + lane] = pack_bf16x8(acc);
         }
-      }
-    } else {
-      // Any K <= 32: branches are taken eight at a time, still in ascending j, so the fma chain
-      // is the same; UNROLL x 8 loads are in flight per lane.
-      for (int i = wi.i0; i < wi.i1; i += UNROLL) {   // warp-uniform trip counts: shuffles stay convergent
-        float acc[UNROLL][8];
-        bool ok[UNROLL];
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          ok[u] = (i + u < wi.i1) && ((i + u) * 32 + lane < H16);
-#pragma unroll
-          for (int x = 0; x < 8; ++x) acc[u][x] = 0.f;
-        }
-        for (int jc = 0; jc < K; jc += 8) {
-          uint4 v[UNROLL][8];
-          float wv[8];
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            const int j = jc + jj;
-            const unsigned long long addr = __shfl_sync(0xffffffffu, row_addr, j & 31);
-            wv[jj] = __shfl_sync(0xffffffffu, w_lane, j & 31);
-            const uint4* src = j < K ? reinterpret_cast<const uint4*>(addr) : nullptr;
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u)
-              v[u][jj] = (ok[u] && src != nullptr) ? ld_row<MODE>(src + (i + u) * 32 + lane)
-                                                   : make_uint4(0, 0, 0, 0);
-          }
-#pragma unroll
-          for (int u = 0; u < UNROLL; ++u)
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj)
-              if (jc + jj < K) fma_bf16x8(acc[u], wv[jj], v[u][jj]);
-        }
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u)
-          if (ok[u]) out[(i + u) * 32 + lane] = pack_bf16x8(acc[u]);
       }
     }
   }
