@@ -935,7 +935,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   const int32_t keep = ctx->granule_override;
   // The ring of whole-row stages: two or three stages per warp; the two-pass form also stages the row's group scales.
   const int ring_warps_max = cpl == 32 ? 8 : QUANT_MAX_WARPS;
-  const int per_warp_extra = (grouped && cpl == 0) ? QUANT_MAX_GROUPS * (int)sizeof(float) : 0;
+  const int per_warp_extra = (grouped && cpl == 0) ? 2 * QUANT_MAX_GROUPS * (int)sizeof(float) : 0;   // scales, reciprocals
   auto ring_warps = [&](int stages) {
     int w = QUANT_SMEM_BUDGET / (stages * (stage + 8) + per_warp_extra);
     return w > ring_warps_max ? ring_warps_max : w;

@@ -88,8 +88,8 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t two_bf16, float inv) {
 // FULL: the row is a whole number of 512-byte slabs (H % 256 == 0), so a chunk is valid for all lanes or for none
 // and the per-lane bounds checks (a possibly divergent branch per chunk) reduce to a warp-uniform one.
 // GROUPED (two-pass form only; shorter rows take dispatch_quant_reg_kernel): one scale per 128 elements
-// (H % 128 == 0); dynamic shared memory then ends with [warps][QUANT_MAX_GROUPS] floats, the scales of the row a
-// warp is working on.
+// (H % 128 == 0); dynamic shared memory then ends with [warps][2][QUANT_MAX_GROUPS] floats, the scales and the
+// reciprocals of the row a warp is working on.
 template <int QUANT_STAGES, int CPL, bool FULL, bool GROUPED = false>
 __global__ void __launch_bounds__((CPL > 16 ? 8 : QUANT_MAX_WARPS) * 32, 1)
 dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __restrict__ windows_q,
@@ -104,9 +104,9 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
   const uint32_t bar0 = smem_addr(smem) + n_warps * QUANT_STAGES * stage_stride + warp * QUANT_STAGES * 8;
   // GROUPED: the scales of the row in hand
   float* group_scale = reinterpret_cast<float*>(smem + (size_t)n_warps * QUANT_STAGES * (stage_stride + 8)) +
-                       warp * QUANT_MAX_GROUPS;
+                       warp * 2 * QUANT_MAX_GROUPS;                     // [QUANT_MAX_GROUPS] scales, then reciprocals
+  float* group_inv = group_scale + QUANT_MAX_GROUPS;
   const int n_groups = a.H16 >> 4;                                      // GROUPED: scales per row
-  const unsigned half_mask = lane < 16 ? 0x0000ffffu : 0xffff0000u;
   // Which half-warp, through an opaque instruction: with `lane >> 4` the compiler (12.9) simplified the byte
   // offset (lane >> 4) * 4 to lane >> 2 under the store's guard (lane & 15) == 0 and then reused that address
   // for the unguarded loads of every lane -- a misaligned address on the device.
@@ -188,24 +188,6 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
         inv = __fdiv_rn(448.0f, amax);
       }
     };
-    // Group-wise: chunk c = lane + 32 k of a row holds elements 8c .. 8c+7, so the sixteen lanes of a half-warp hold
-    // group 2k + half between them.  Converts this lane's chunk and leaves the group's scale in group_scale.
-    // Called by whole half-warps only (a row is a whole number of groups).
-    auto convert_group = [&](const uint4& v, int k, uint32_t dst) {
-      uint32_t m2 = __vmaxu2(__vmaxu2(v.x & 0x7fff7fffu, v.y & 0x7fff7fffu), __vmaxu2(v.z & 0x7fff7fffu, v.w & 0x7fff7fffu));
-      uint32_t mbits = max(m2 & 0xffffu, m2 >> 16);
-      mbits = __reduce_max_sync(half_mask, mbits);
-      const float amax = __uint_as_float(mbits << 16);
-      float g_scale = 1.0f, g_inv = 1.0f;
-      if (amax > 0.0f) {
-        g_scale = __fdiv_rn(amax, 448.0f);
-        g_inv = __fdiv_rn(448.0f, amax);
-      }
-      const uint32_t lo = quant_pair(v.x, g_inv) | (quant_pair(v.y, g_inv) << 16);
-      const uint32_t hi = quant_pair(v.z, g_inv) | (quant_pair(v.w, g_inv) << 16);
-      sts64(dst, lo, hi);
-      if ((lane & 15) == 0) group_scale[2 * k + half] = g_scale;
-    };
     if constexpr (CPL > 0) {
       uint4 v[CPL];
       uint32_t m[4] = {0u, 0u, 0u, 0u};
@@ -232,12 +214,69 @@ dispatch_quant_kernel(const unsigned char* __restrict__ X, unsigned char* __rest
           sts64(in + (lane + 32 * k) * 8, lo, hi);
         }
     } else if constexpr (GROUPED) {
-      // any row length: one pass, a chunk per lane at a time (in place as in the row-wise two-pass form below)
-      for (int c = lane, k = 0; c - lane < a.H16; c += 32, ++k) {   // warp-uniform trip count
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (c < a.H16) v = lds128(in + c * 16);
-        __syncwarp();
-        if (c < a.H16) convert_group(v, k, in + c * 8);
+      // Any row length, in batches of 16 chunks per lane (8 KB of the row, 32 groups), in place like the row-wise
+      // two-pass form below: a batch is read into registers, its group maxima come from the transposing butterfly
+      // of dispatch_quant_reg_kernel (packed maxima of two chunks per word, 7 shuffles for the batch), one lane per
+      // group turns them into scale and reciprocal, and the batch is converted.  (One chunk at a time with a
+      // sub-warp reduction and two divisions per lane and chunk ran at 2.3 TB/s on 32 KB rows against 6.1 TB/s for
+      // the row-wise form.)  Batch b writes bytes [4096 b, 4096 b + 4096) of the stage, which only batches <= b
+      // have read.
+      for (int c0 = 0; c0 < a.H16; c0 += 512) {   // warp-uniform trip count; a.H16 is a multiple of 16
+        uint4 v[16];
+        uint32_t w[8];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int c = c0 + lane + 32 * k;
+          v[k] = c < a.H16 ? lds128(in + c * 16) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {   // per-halfword maxima of chunks 2i and 2i+1 share a word
+          const uint32_t e = __vmaxu2(__vmaxu2(v[2 * i].x & 0x7fff7fffu, v[2 * i].y & 0x7fff7fffu),
+                                      __vmaxu2(v[2 * i].z & 0x7fff7fffu, v[2 * i].w & 0x7fff7fffu));
+          const uint32_t o = __vmaxu2(__vmaxu2(v[2 * i + 1].x & 0x7fff7fffu, v[2 * i + 1].y & 0x7fff7fffu),
+                                      __vmaxu2(v[2 * i + 1].z & 0x7fff7fffu, v[2 * i + 1].w & 0x7fff7fffu));
+          w[i] = __vmaxu2(__byte_perm(e, o, 0x5410), __byte_perm(e, o, 0x7632));
+        }
+        int held = 8;
+#pragma unroll
+        for (int bit = 8; bit >= 1; bit >>= 1) {
+          const bool up = (lane & bit) != 0;
+          if (held > 1) {
+            held >>= 1;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (j < held) {
+                const uint32_t send = up ? w[j] : w[j + held];
+                const uint32_t keep = up ? w[j + held] : w[j];
+                w[j] = __vmaxu2(keep, __shfl_xor_sync(0xffffffffu, send, bit));
+              }
+          } else {   // one word left: both partners finish with the same word
+            w[0] = __vmaxu2(w[0], __shfl_xor_sync(0xffffffffu, w[0], bit));
+          }
+        }
+        {
+          // lane l of a half-warp holds word l >> 1 (chunks 2 (l >> 1) and 2 (l >> 1) + 1) and takes chunk k = l
+          const int l = lane & 15;
+          const uint32_t bits = (l & 1) ? (w[0] >> 16) : (w[0] & 0xffffu);
+          const int g = (c0 >> 4) + 2 * l + half;
+          if (g < n_groups) {
+            const float amax = __uint_as_float(bits << 16);
+            const float den = amax > 0.0f ? amax : 448.0f;   // an all-zero group: scale and reciprocal 1
+            group_scale[g] = __fdiv_rn(den, 448.0f);
+            group_inv[g] = __fdiv_rn(448.0f, den);
+          }
+        }
+        __syncwarp();   // the reciprocals are visible; every lane's reads of the batch are in registers
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int c = c0 + lane + 32 * k;
+          if (c < a.H16) {
+            const float g_inv = group_inv[(c0 >> 4) + 2 * k + half];
+            const uint32_t lo = quant_pair(v[k].x, g_inv) | (quant_pair(v[k].y, g_inv) << 16);
+            const uint32_t hi = quant_pair(v[k].z, g_inv) | (quant_pair(v[k].w, g_inv) << 16);
+            sts64(in + c * 8, lo, hi);
+          }
+        }
       }
     } else {
       uint32_t m2 = 0;
