@@ -1078,6 +1078,7 @@ moe_status_t combine_impl(moe_ctx* ctx, const void* windows, const void* const* 
     case 6: launch_combine<6>(ctx, a, win, topk_w, ys, st); break;
     case 7: launch_combine<7>(ctx, a, win, topk_w, ys, st); break;
     case 8: launch_combine<8>(ctx, a, win, topk_w, ys, st); break;
+    case 9: launch_combine<9>(ctx, a, win, topk_w, ys, st); break;   // eight routed experts and a shared one
     case 10: launch_combine<10>(ctx, a, win, topk_w, ys, st); break;
     case 12: launch_combine<12>(ctx, a, win, topk_w, ys, st); break;
     case 16: launch_combine<16>(ctx, a, win, topk_w, ys, st); break;
