@@ -434,6 +434,95 @@ def call_latency(layer: Layer, n: int, flush=None) -> dict:
             "step_us_plan_dispatch_fused": tf - base}
 
 
+def sweeps(dev, n: int = 20) -> dict:
+    """Opt-in (--sweeps): one call each of plan, dispatch, combine, the quantised dispatch and the chained
+    moe_plan_dispatch over sweeps of the top-k degree, the row length, the rank count and the shapes of published
+    MoE models, in microseconds with the TB/s of algorithmic bytes beside them; small jobs start from a flushed L2.
+    Every cell checks Y == X.  A paper-independent health check of the kernels away from the benchmark shapes:
+    the generic-K combine, the chained launch behind the planner, the table-addressed combine and the long-row
+    group-wise quantisation were each found several times below their neighbours by these tables."""
+    from paper_2605_06055_b200 import binding
+    flush_buf = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+
+    def cell(name, T, H, E, R, K, sch, peers=False):
+        wl = synth.Workload(name, T, H, E, R, K, sch, "uniform", "identity", 1002)
+        l = Layer(wl, dev)
+        c = l.comm
+        nb = 2 * wl.H * wl.T * (1 + wl.K)
+        pre = [lambda: flush_buf.add_(1)] if nb < (400 << 20) else []
+        base = min(time_repeated(pre, n) for _ in range(2)) if pre else 0.0
+        t = lambda fns: min(time_repeated(pre + fns, n) for _ in range(2)) - base
+        plan = lambda: c.moe_plan(wl.schedule, l.idx)
+        disp = lambda: c.moe_dispatch(l.X, l.windows, l.C)
+        comb = lambda: c.moe_combine(l.windows, l.C, l.w, l.Y)
+        out = {"T": T, "H": H, "E": E, "R": R, "K": K, "plan_us": t([plan])}
+        out["dispatch_us"] = t([disp])
+        out["combine_us"] = t([comb])
+        out["plan_then_dispatch_us"] = t([plan, disp])
+        out["plan_dispatch_chained_us"] = t([lambda: c.moe_plan_dispatch(wl.schedule, l.idx, l.X, l.windows, l.C)])
+        if H % 16 == 0:
+            wq = torch.zeros((wl.R * l.C, wl.H), dtype=torch.uint8, device=dev)
+            sc = torch.zeros((wl.R * l.C,), dtype=torch.float32, device=dev)
+            out["dispatch_quant_us"] = t([lambda: c.moe_dispatch_quant(l.X, wq, sc, l.C)])
+            if H % 128 == 0:
+                scg = torch.zeros((wl.R * l.C, wl.H // 128), dtype=torch.float32, device=dev)
+                out["dispatch_quant_group128_us"] = t([lambda: c.moe_dispatch_quant_group(l.X, wq, scg, l.C)])
+                del scg
+            del wq, sc
+        if peers:   # the same windows addressed through a table of bases (the multi-rank calls on one GPU)
+            bases = torch.tensor([l.windows.data_ptr() + d * l.C * wl.H * 2 for d in range(wl.R)], dtype=torch.int64,
+                                 device=dev)
+            out["dispatch_peers_us"] = t([lambda: c.moe_dispatch_peers(l.X, bases, l.C)])
+            out["combine_peers_us"] = t([lambda: c.moe_combine_peers(bases, l.C, l.w, l.Y)])
+        c.moe_dispatch(l.X, l.windows, l.C)
+        c.moe_combine(l.windows, l.C, l.w, l.Y)
+        assert c.moe_status() == 0
+        assert torch.equal(l.Y.view(torch.int16), l.X.view(torch.int16)), name
+        out["dispatch_TBps"] = nb / out["dispatch_us"] / 1e6
+        out["combine_TBps"] = nb / out["combine_us"] / 1e6
+        c.close()
+        del l
+        torch.cuda.empty_cache()
+        return out
+
+    P, D = synth.PREFILL, synth.DECODE
+    res = {"method": f"{n} repetitions per pair of CUDA events, better of two; 256 MB L2 flush in front of jobs below "
+                     "400 MB (its time subtracted)"}
+    res["top_k"] = {f"K{K}": cell(f"K{K}", 8192, 4096, 64, 8, K, P) for K in (1, 2, 3, 4, 6, 8, 9, 11, 16, 20, 24, 32)}
+    res["row_length"] = {f"H{H}": cell(f"H{H}", 16384 if H <= 8192 else 8192, H, 64, 8, 8, P)
+                         for H in (256, 512, 1024, 2048, 2880, 4096, 5120, 7168, 8192, 12288, 16384)}
+    res["ranks"] = {f"R{R}": cell(f"R{R}", 2048, 7168, 256, R, 8, D, peers=True) for R in (1, 2, 4, 8, 16, 32, 64)}
+    res["tokens"] = {f"T{T}": cell(f"T{T}", T, 7168, 256, 8 if T >= 8192 else 16, 8, P if T >= 8192 else D, peers=True)
+                     for T in (512, 1024, 3072, 4096, 8192, 32768)}
+    models = {"H4096_E128_K8": (4096, 128, 8, 8), "H2048_E128_K8": (2048, 128, 8, 8), "H2880_E128_K4": (2880, 128, 8, 4),
+              "H5120_E128_K1": (5120, 128, 8, 1), "H6144_E8_K2": (6144, 8, 8, 2), "H5120_E160_K6": (5120, 160, 8, 6),
+              "H7168_E384_K8": (7168, 384, 16, 8)}
+    res["model_shapes_T32768"] = {k: cell(k, 32768, H, E, R, K, P) for k, (H, E, R, K) in models.items()}
+    res["model_shapes_T1024"] = {k: cell(k, 1024, H, E, R, K, D) for k, (H, E, R, K) in models.items()}
+    # one rank's part of a multi-rank plan (moe_layout) and the offsets from the gathered counts (moe_notify)
+    res["layout_notify"] = {}
+    for R in (8, 16, 64):
+        for per in (128, 4096):
+            E, K, H = 256, 8, 7168
+            wl = synth.Workload(f"R{R}_per{per}", per * R, H, E, R, K, D if per == 128 else P, "uniform", "identity", 1002)
+            idx = synth.make_inputs(wl).topk_idx.to(dev)
+            whole = binding.MoeComm(wl.T, H, E, R, K, dev)
+            whole.moe_plan(P, idx)
+            counts = whole.moe_plan_view()["counts"].clone()
+            whole.close()
+            mine = idx[:per].contiguous()
+            c = binding.MoeComm(per, H, E, R, K, dev)
+            lay = lambda: c.moe_layout(wl.schedule, mine, 0, counts[0])
+            noti = lambda: c.moe_notify(counts)
+            lay(), noti()
+            assert c.moe_status() == 0
+            res["layout_notify"][f"R{R}_{per}_tokens_per_rank"] = {
+                "layout_us": time_graphed(lay), "notify_us": time_graphed(noti),
+                "both_us": time_graphed(lambda: (lay(), noti())), "note": "back to back inside a CUDA graph"}
+            c.close()
+    return res
+
+
 def decode_latency(dev, peak, n: int = 200, grid: bool = False) -> dict:
     """Decode-step latency (config 2).  Per-call figures are differences of cumulative sequences
     (flush | flush+plan | flush+plan+dispatch | ...), each timed over n repetitions."""
@@ -941,6 +1030,9 @@ def run_cuda(args, wl):
     if world == 1 and not args.no_decode and wl.name != synth.config(2).name:
         line["decode"] = decode_latency(dev, peak, grid=args.decode_grid)
         torch.cuda.empty_cache()
+    if world == 1 and args.sweeps:
+        line["sweeps"] = sweeps(dev)
+        torch.cuda.empty_cache()
 
     if world == 1 and args.workload == "c5" and not args.no_decode:
         # config 5: both schedules timed at each T of the sweep.  Calls of a few microseconds cannot be timed by
@@ -1005,6 +1097,8 @@ def main():
     ap.add_argument("--ep-backend", default="nccl", help=argparse.SUPPRESS)
     ap.add_argument("--ep-device", type=int, default=-1, help=argparse.SUPPRESS)    # tests: every rank on this GPU
     ap.add_argument("--ep-shapes", default="decode,prefill", help=argparse.SUPPRESS)
+    ap.add_argument("--sweeps", action="store_true",
+                    help="also time single calls over sweeps of top-k, row length, rank count and model shapes")
     ap.add_argument("--decode-grid", action="store_true",
                     help="also time the batch-size x hidden-size grid of the paper's decode table (off by default)")
     args = ap.parse_args()

@@ -906,6 +906,7 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   const int H = ctx->shape.H;
   if (!quant_shape_ok(H, group)) return MOE_ERR_INVALID_ARG;
   const bool grouped = group != 0;
+  const int sh_K = ctx->shape.K;
   if (capacity_rows < 0 || (peers && s_bases == nullptr)) return MOE_ERR_INVALID_ARG;
   if (ctx->T > 0 && (x == nullptr || (!peers && (windows_q == nullptr || scales == nullptr)))) return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || (!peers && (!aligned16(windows_q) || (reinterpret_cast<uintptr_t>(scales) & 3u) != 0)))
@@ -944,14 +945,15 @@ static moe_status_t dispatch_quant_impl(moe_ctx* ctx, const void* x, void* windo
   const bool large = ring_warps(3) >= 1 && (int64_t)ctx->T >= (int64_t)8 * grid * ring_warps(2);
   // Rows short enough for registers take the register kernel (a load buffer and a code buffer per warp, the group
   // scales and reciprocals behind the codes): more rows in flight per SM.  Only large row-wise jobs of rows beyond
-  // 8 KB stay on the three-stage ring, which runs them at the copy rate with five warps (32768 rows of 14 KB: 371
-  // against 376 us).  Measured, register kernel against ring: decode shape 31.9 against 33.8 us row-wise and 33.8
+  // 8 KB with five or more branches per token stay on the three-stage ring, which runs them at the copy rate with
+  // five warps (32768 rows of 14 KB, K=8: 368 against 373 us); with fewer branches the job is read-dominated and the
+  // register kernel's ten warps are ahead (K=1: 116 against 172 us, K=2: 150 against 182, K=3: 186 against 199).  Measured, register kernel against ring: decode shape 31.9 against 33.8 us row-wise and 33.8
   // against 44.1 us group-wise; 65536 rows of 4 KB 170 against 203 us; 65536 rows of 8 KB 179 against 176 us.
   // Warps per CTA: as many as fit, but for large jobs of short rows at most 9.  At 65536 rows of 8 KB ten or eleven
   // warps reach 169-172 us in one run and 237-240 us (the rate of six warps) in the next, and twelve or more are
   // always at 237-240: past about 2700 window rows being written at once HBM serves the writes badly (the bulk-copy
   // dispatch bounds its warps for the same reason), and where exactly that sets in changes from run to run.
-  if (cpl == 16 || (cpl == 32 && (grouped || !large))) {
+  if (cpl == 16 || (cpl == 32 && (grouped || !large || sh_K < 5))) {
     const int sc_bytes = grouped ? ((H / QUANT_GROUP) * 4 + 15) / 16 * 16 : 0;
     const int per_warp = stage + (H + 2 * sc_bytes + 127) / 128 * 128 + 8;
     int warps = QUANT_SMEM_BUDGET / per_warp;
