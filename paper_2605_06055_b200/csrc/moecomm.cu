@@ -258,8 +258,11 @@ int row_grid(moe_ctx* ctx, Kernel kernel, int64_t tokens) {
 // Loads in flight per lane before the dependent stores / fma chain.  Few fat warps (one 256-thread
 // CTA per SM with about 32 16-byte loads per lane) measured faster than many thin ones: every warp
 // then streams long contiguous runs of each row, which HBM serves with far fewer page switches.
+// More than 32 where it measured ahead: K=4 with 48 (a row of 10-12 units is then one phase of loads instead of
+// a long and a short one: 179 -> 147 us at 32768 rows of 5760 bytes), K=9 and 10 with 36-40 (3-4 % at every size
+// tried); 48 loads measured behind for K=1, 2, 8 and mixed for K=6.
 constexpr int combine_unroll(int K) {
-  return K >= 17 ? 1 : K >= 16 ? 2 : K >= 9 ? 3 : K >= 7 ? 4 : K >= 6 ? 5 : K == 5 ? 6 : K == 4 ? 8 : K == 3 ? 10 : 16;
+  return K >= 17 ? 1 : K >= 16 ? 2 : K >= 11 ? 3 : K >= 7 ? 4 : K >= 6 ? 5 : K == 5 ? 6 : K == 4 ? 12 : K == 3 ? 10 : 16;
 }
 constexpr int DISPATCH_UNROLL = 14;
 
