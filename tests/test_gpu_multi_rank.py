@@ -24,6 +24,10 @@ CASES = [
     ("large_rank_tile_path", 6000, 64, 16, 2, 2, PREFILL, "replace", (5000, 1000)),
     ("large_rank_tile_path_decode", 6000, 64, 16, 2, 2, DECODE, "replace", (5000, 1000)),
     ("generic_k", 500, 264, 12, 3, 3, DECODE, "replace", (100, 150, 250)),
+    # Notify from the gathered counts at the ends of its range: 2048 experts per window, and 64 windows of two
+    ("many_experts_per_rank", 400, 64, 4096, 2, 8, PREFILL, "uniform", (150, 250)),
+    ("many_ranks", 640, 64, 128, 64, 4, DECODE, "uniform", None),
+    ("k11_masked_combine", 300, 512, 32, 4, 11, PREFILL, "uniform", (100, 50, 0, 150)),
 ]
 
 
