@@ -89,6 +89,9 @@ EDGE = [
     ("K16", 120, 4096, 32, 2, 16, "uniform", None),
     ("K9_generic", 90, 264, 16, 2, 9, "uniform", None),
     ("K32_max", 40, 64, 64, 2, 32, "uniform", None),
+    ("K20_of_24", 100, 264, 64, 2, 20, "uniform", None),                   # combine forms with spare branches
+    ("K27_of_32", 90, 136, 64, 4, 27, "uniform", (30, 0, 40, 20)),
+    ("K13_of_16", 150, 4096, 32, 2, 13, "uniform", None),
     ("duplicates_in_token", 333, 72, 4, 2, 4, "replace", (300, 33)),
     ("empty_rank_ragged", 1000, 256, 32, 4, 8, "uniform", (0, 517, 0, 483)),
     ("many_ranks", 512, 64, 256, 64, 8, "uniform", None),
