@@ -53,6 +53,30 @@ def test_random_shape(i):
     harness.assert_parity(g, o, wl.schedule, align=align)
 
 
+@pytest.mark.parametrize("i", range(max(24, N_SHAPES // 4)))
+def test_random_shape_many_ranks_and_high_degrees(i):
+    """More ranks than a thread-block cluster holds (the planners' Notify step runs as a launch of its own) and
+    degrees up to the maximum (the combine forms with spare branches)."""
+    rng = np.random.default_rng(99000 + i)
+    R = int(rng.choice([24, 32, 48, 64, 256]))
+    E = R * int(rng.choice([1, 2, 4]))
+    K = int(rng.integers(1, min(E, 32) + 1))
+    H = 8 * int(rng.choice([1, 17, 32, 64, 129, 512]))
+    T = int(rng.choice([1, 50, 257, 1000, 3000, 9000]))
+    cuts = np.sort(rng.integers(0, T + 1, R - 1))
+    per = tuple(int(x) for x in np.diff(np.concatenate([[0], cuts, [T]])))
+    sch = PREFILL if rng.integers(0, 2) else DECODE
+    wl = Workload(f"wide{i}", T, H, E, R, K, sch, "uniform", "scale", 41000 + i, rank_tokens=per)
+    align = int(rng.choice([1, 1, 8]))
+    inp = synth.make_inputs(wl)
+    p = oracle.plan(inp.topk_idx.numpy(), wl.E, wl.R, inp.rank_tok_start, align=align)
+    assert p.status == oracle.OK
+    C = int(p.n_recv.max()) + int(rng.integers(0, 3))
+    o = harness.oracle_run(inp, C, align=align)
+    g = harness.gpu_run(inp, C, wl.schedule, align=align)
+    harness.assert_parity(g, o, wl.schedule, align=align)
+
+
 @pytest.mark.parametrize("i", range(max(12, N_SHAPES // 4)))
 def test_random_shape_fused_call_and_quantised_dispatch(i):
     rng = np.random.default_rng(88000 + i)
