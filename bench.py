@@ -681,7 +681,8 @@ def ep_shape(key: str, R: int):
 
 
 def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
-           variants=(("cached", "host"), ("handshake", "host"), ("cached", "device"), ("static", "device"))) -> dict:
+           variants=(("cached", "host"), ("handshake", "host"), ("cached", "device"), ("static", "device"),
+                     ("static", "device", "device"))) -> dict:
     """The path with rank = process = GPU: every process plans its own tokens, the count rows (and window
     generations) are all-gathered over the process group, every rank's window is mapped into every process
     (moe_window_export / moe_peers_open), dispatch stores rows into the other GPUs' windows and combine loads
@@ -695,7 +696,10 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
     stream synchronisation and a process-group barrier, "device" by arrival flags in the windows' state regions
     (moe_signal_peers / moe_wait_peers) with no host synchronisation between the phases -- unless ranks share a
     GPU, where a host barrier is placed between signal and wait (a wait kernel must not hold a GPU that the
-    signalling rank needs).  Times are device time between CUDA events (idle gaps included), max over ranks."""
+    signalling rank needs).  A third entry "device" sends the count rows through the mailboxes behind the state
+    regions (moe_push_counts / moe_notify_peers) instead of an all-gather of the process group: with static
+    addresses and the device phase order a step then contains no collective and no host synchronisation at all.
+    Times are device time between CUDA events (idle gaps included), max over ranks."""
     import torch.distributed as dist
     from paper_2605_06055_b200 import binding, ep
     rank, R = dist.get_rank(group), dist.get_world_size(group)
@@ -733,15 +737,19 @@ def ep_leg(dev, steps: int, group=None, shapes=("decode", "prefill"),
         mine_ref_q, mine_ref_s = ref_q[rank * C:(rank + 1) * C].clone(), ref_s[rank * C:(rank + 1) * C].clone()
         del ref_q, ref_s, g_X, g_idx
         ref.close()
-        for mode, sync in variants:
-            name = f"{mode}_addresses__{sync}_phase_order"
-            me = ep.EpRank(wl.T // R, wl.H, wl.E, wl.K, dev, group, mode=mode, sync=sync, host_fence=shared_gpu)
+        for variant in variants:
+            mode, sync = variant[0], variant[1]
+            counts = variant[2] if len(variant) > 2 else "collective"
+            name = f"{mode}_addresses__{sync}_phase_order" + ("__counts_through_mailboxes" if counts == "device" else "")
+            me = ep.EpRank(wl.T // R, wl.H, wl.E, wl.K, dev, group, mode=mode, sync=sync, host_fence=shared_gpu,
+                           counts=counts)
             with_quant = (mode, sync) == ("cached", "host")   # this variant also times the quantised dispatch
             window = me.new_window(C, quant=with_quant)       # rows + zeroed state region (+ codes, scales), attached
             ok, why = 1.0, ""
             try:
-                me.plan(wl.schedule, idx)
-                me.handshake()
+                me.plan(wl.schedule, idx)     # (with the mailboxes: exchanges the addresses first, they carry the counts)
+                if counts != "device":
+                    me.handshake()
             except Exception as exc:      # e.g. no peer access between two of the GPUs
                 ok, why = 0.0, repr(exc)
             if _group_reduce(ok, dist.ReduceOp.MIN, dev, group) < 1.0:

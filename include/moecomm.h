@@ -313,6 +313,8 @@ typedef struct {
 #define MOE_WINDOW_QUANT_GROUP 4 /* the code window and the scale tensor [capacity_rows, H / 128] fp32 of the
                               group-wise quantised dispatch (moe_dispatch_quant_group_cached); not together with
                               MOE_WINDOW_QUANT, and H % 128 == 0                                                */
+#define MOE_WINDOW_COUNTS 8 /* the mailbox of the count exchange (moe_push_counts), directly behind the state region:
+                              only together with MOE_WINDOW_STATE; zeroed once with it                        */
 moe_status_t moe_window_export(const void* window /*DEVICE*/, int64_t bytes, int32_t generation, int32_t flags,
                                moe_window_handle_t* out /*HOST*/);
 moe_status_t moe_peers_open(moe_ctx_t* ctx, const moe_window_handle_t* handles /*HOST [R]*/, int32_t my_rank,
@@ -355,6 +357,25 @@ moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
  * NOTE: a wait kernel occupies its GPU until the signals arrive, so the ranks must run on different GPUs (or the
  * caller must know that the signals were sent before the wait is enqueued). */
 #define MOE_SYNC_SLOTS 4
+/* Count exchange through the pooled memory (Section 5.2, Notify: count metadata is the only thing the ranks exchange
+ * before payload moves; here it moves by the library's own peer stores instead of a collective of the caller's).
+ * Windows exported with MOE_WINDOW_STATE | MOE_WINDOW_COUNTS carry, behind the arrival flags, a mailbox of two
+ * buffers of [R][E] counts and [R] epoch words, zeroed once together with the state region.
+ *   moe_push_counts   after moe_layout: stores this rank's row of counts into entry [my_rank] of EVERY rank's
+ *                     mailbox (buffer epoch & 1) and publishes it with the epoch word (release, system scope).
+ *                     Waits for nobody.
+ *   moe_notify_peers  moe_notify from this rank's own mailbox: enqueues a kernel that waits until all R epoch words
+ *                     of buffer epoch & 1 have reached `epoch` (acquire, system scope; bounded like moe_wait_peers:
+ *                     MOE_ERR_TIMEOUT in the status word, a normal end, and no plan once moe_status has reported
+ *                     it) and then builds the large offsets and receive counts; the context is then planned.
+ * Epochs of successive exchanges must grow by one (the two buffers alternate); a rank may run one exchange ahead
+ * of the slowest rank, which the phase order of a layer step guarantees (nobody starts step e + 2 before every
+ * rank has combined step e + 1, hence consumed the counts of step e).  The NOTE on moe_wait_peers applies:
+ * with several ranks on one GPU every rank's push must have been enqueued before any rank's notify.
+ * MOE_ERR_STALE_PEERS without an installed table whose windows have the mailbox; MOE_ERR_NOT_PLANNED before
+ * moe_layout.  (No counterpart call in the paper: its Notify kernel does both halves.) */
+moe_status_t moe_push_counts(moe_ctx_t* ctx, uint32_t epoch, void* stream);
+moe_status_t moe_notify_peers(moe_ctx_t* ctx, uint32_t epoch, void* stream);
 size_t moe_state_bytes(int32_t R);
 size_t moe_window_bytes(const moe_shape_t* shape /*HOST*/, int64_t capacity_rows, int32_t flags);
 moe_status_t moe_signal_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* stream);

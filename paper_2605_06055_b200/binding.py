@@ -30,10 +30,10 @@ EXPORTS = [
     "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
     "moe_dispatch_cached", "moe_combine_cached", "moe_state_bytes", "moe_window_bytes", "moe_signal_peers",
     "moe_wait_peers", "moe_dispatch_quant_cached", "moe_dispatch_quant_group", "moe_plan_dispatch_quant_group",
-    "moe_dispatch_quant_group_cached",
+    "moe_dispatch_quant_group_cached", "moe_push_counts", "moe_notify_peers",
 ]
 MOE_SYNC_SLOTS = 4
-MOE_WINDOW_STATE, MOE_WINDOW_QUANT, MOE_WINDOW_QUANT_GROUP = 1, 2, 4
+MOE_WINDOW_STATE, MOE_WINDOW_QUANT, MOE_WINDOW_QUANT_GROUP, MOE_WINDOW_COUNTS = 1, 2, 4, 8
 MOE_OPT_DISPATCH_PATH, MOE_OPT_GRANULE, MOE_OPT_TEST_STARVE_WAIT_MS, MOE_OPT_OVERLAP = 0, 1, 2, 3
 MOE_OPT_EXPERT_ALIGN, MOE_OPT_CLUSTER_PLAN, MOE_OPT_SLOT_REUSE = 4, 5, 6
 MOE_DISPATCH_AUTO, MOE_DISPATCH_REGISTERS, MOE_DISPATCH_BULK = 0, 1, 2
@@ -131,6 +131,8 @@ def load() -> ctypes.CDLL:
     L.moe_signal_peers.argtypes = [vp, i32, ctypes.c_uint32, vp]
     L.moe_wait_peers.argtypes = [vp, i32, ctypes.c_uint32, vp]
     L.moe_signal_peers.restype = L.moe_wait_peers.restype = ctypes.c_int
+    L.moe_push_counts.argtypes = L.moe_notify_peers.argtypes = [vp, ctypes.c_uint32, vp]
+    L.moe_push_counts.restype = L.moe_notify_peers.restype = ctypes.c_int
     L.moe_peers_check.argtypes = [vp, vp]
     L.moe_peers_close.argtypes = [vp, vp]
     L.moe_dispatch_cached.argtypes = [vp, vp, vp, vp]
@@ -485,6 +487,20 @@ class MoeComm:
             rc = self.lib.moe_wait_peers(self._h, int(slot), int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_wait_peers")
+        return rc
+
+    def moe_push_counts(self, epoch: int, stream=None, check: bool = True) -> int:
+        with self._on_device():
+            rc = self.lib.moe_push_counts(self._h, int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_push_counts")
+        return rc
+
+    def moe_notify_peers(self, epoch: int, stream=None, check: bool = True) -> int:
+        with self._on_device():
+            rc = self.lib.moe_notify_peers(self._h, int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
+        if rc != MOE_OK and check:
+            raise MoeError(rc, "moe_notify_peers")
         return rc
 
     def moe_plan_view(self) -> dict:

@@ -64,6 +64,9 @@ struct moe_ctx {
   bool peers_have_state;              // every installed window is followed by its state region
   bool peers_have_quant;              // ... and by a code window and a scale tensor (one scale per row)
   bool peers_have_quant_group;        // ... or by a code window and a tensor of group scales
+  bool peers_have_counts;             // ... and the state region by the mailbox of the count exchange
+  unsigned char** box_table;          // device, [R]: count mailbox of every rank
+  bool notified_by_box;               // the current plan's offsets came from moe_notify_peers
   unsigned char** code_table;         // device, [R]: e4m3 code window of every rank
   float** scale_table;                // device, [R]: scale tensor of every rank
   int32_t my_rank;                    // this process's rank in the installed table
@@ -117,7 +120,7 @@ Layout layout_of(const moe_shape_t* s) {
   L.o = take(sizeof(int32_t) * s->E * s->R);
   L.n_exp = take(sizeof(int32_t) * s->E);
   L.n_recv = take(sizeof(int32_t) * s->R);
-  L.peers = take(sizeof(void*) * s->R * 4);   // window bases, state regions, code windows, scale tensors
+  L.peers = take(sizeof(void*) * s->R * 5);   // window bases, state regions, code windows, scale tensors, count mailboxes
   L.s = take(sizeof(int32_t) * B);
   L.slot = take(sizeof(int32_t) * B);
   L.tile_rank = take(sizeof(int32_t) * B);
@@ -438,6 +441,9 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
   ctx->peers_installed = false;
   ctx->code_table = ctx->state_table + shape->R;
   ctx->scale_table = reinterpret_cast<float**>(ctx->code_table + shape->R);
+  ctx->box_table = ctx->code_table + 2 * shape->R;
+  ctx->peers_have_counts = false;
+  ctx->notified_by_box = false;
   ctx->peers_have_state = false;
   ctx->peers_have_quant = false;
   ctx->peers_have_quant_group = false;
@@ -491,7 +497,7 @@ moe_status_t moe_create(const moe_shape_t* shape, void* workspace, size_t worksp
        opt_in(dispatch_quant_reg_kernel<32, true, true>) && opt_in(dispatch_quant_reg_kernel<32, false, true>) &&
        opt_in(dispatch_quant_reg_kernel<32, true, false>) && opt_in(dispatch_quant_reg_kernel<32, false, false>) &&
        opt_in(plan_rank_kernel<32>) &&
-       opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_rank_kernel) &&
+       opt_in(plan_rank_kernel<8>) && opt_in(plan_scan_kernel) && opt_in(notify_rank_kernel) && opt_in(notify_box_kernel) &&
        opt_in(plan_tile_kernel<ROUNDS_PREFILL>) && opt_in(plan_tile_kernel<ROUNDS_DECODE>) && opt_in(gate_topk_kernel<0, false>);
   // The shape must fit: per-warp expert counters of the planners, the Notify scratch.
   const int rank_smem =
@@ -641,6 +647,7 @@ moe_status_t plan_impl(moe_ctx* ctx, moe_schedule_t schedule, const int32_t* top
   ctx->planned = false;
   ctx->slots_for_C = -1;
   ctx->layout_done = false;
+  ctx->notified_by_box = false;
 
   const int rounds = schedule == MOE_SCHED_PREFILL ? ROUNDS_PREFILL : ROUNDS_DECODE;
   const int tile_branches = rounds * PLAN_THREADS;
@@ -1187,7 +1194,7 @@ size_t state_bytes_for(int32_t R) { return align_up(sizeof(uint32_t) * MOE_SYNC_
 
 // Parts of a window allocation, byte offsets from its first row (see MOE_WINDOW_* in the header).
 struct WindowParts {
-  size_t state, codes, scales, total;
+  size_t state, box, codes, scales, total;
 };
 WindowParts window_parts(const moe_shape_t& sh, int64_t capacity_rows, int32_t flags) {
   WindowParts p;
@@ -1195,6 +1202,8 @@ WindowParts window_parts(const moe_shape_t& sh, int64_t capacity_rows, int32_t f
   size_t at = flags != 0 ? align_up(rows) : rows;
   p.state = at;
   if (flags & MOE_WINDOW_STATE) at += state_bytes_for(sh.R);
+  p.box = at;
+  if (flags & MOE_WINDOW_COUNTS) at += align_up(counts_box_bytes(sh.E, sh.R));
   p.codes = at;
   if (flags & (MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP)) at += align_up((size_t)capacity_rows * sh.H);
   p.scales = at;
@@ -1206,7 +1215,8 @@ WindowParts window_parts(const moe_shape_t& sh, int64_t capacity_rows, int32_t f
 
 // Known bits only, and at most one form of quantised parts.
 bool window_flags_ok(int32_t flags) {
-  if ((flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP)) != 0) return false;
+  if ((flags & ~(MOE_WINDOW_STATE | MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP | MOE_WINDOW_COUNTS)) != 0) return false;
+  if ((flags & MOE_WINDOW_COUNTS) != 0 && (flags & MOE_WINDOW_STATE) == 0) return false;   // the mailbox follows the flags
   return (flags & MOE_WINDOW_QUANT) == 0 || (flags & MOE_WINDOW_QUANT_GROUP) == 0;
 }
 // ... and a shape the group-wise parts exist for.
@@ -1218,7 +1228,7 @@ bool window_flags_fit(int32_t flags, const moe_shape_t& sh) {
 // `stream` and marks them installed.
 moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows, int32_t flags, cudaStream_t st) {
   const int R = ctx->shape.R;
-  void* all[4 * MOE_MAX_R];
+  void* all[5 * MOE_MAX_R];
   const WindowParts parts = window_parts(ctx->shape, capacity_rows, flags);
   for (int d = 0; d < R; ++d) {
     char* base = static_cast<char*>(ctx->peer_ptr[d]);
@@ -1227,15 +1237,17 @@ moe_status_t install_table(moe_ctx* ctx, int32_t my_rank, int64_t capacity_rows,
     const bool quant = (flags & (MOE_WINDOW_QUANT | MOE_WINDOW_QUANT_GROUP)) != 0;
     all[2 * R + d] = quant ? base + parts.codes : nullptr;
     all[3 * R + d] = quant ? base + parts.scales : nullptr;
+    all[4 * R + d] = (flags & MOE_WINDOW_COUNTS) ? base + parts.box : nullptr;
   }
   // pageable source: the runtime has staged the bytes by the time the call returns
-  if (cudaMemcpyAsync(ctx->peer_table, all, sizeof(void*) * 4 * R, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  if (cudaMemcpyAsync(ctx->peer_table, all, sizeof(void*) * 5 * R, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   ctx->peer_capacity = capacity_rows;
   ctx->my_rank = my_rank;
   ctx->peers_have_state = (flags & MOE_WINDOW_STATE) != 0;
   ctx->peers_have_quant = (flags & MOE_WINDOW_QUANT) != 0;
   ctx->peers_have_quant_group = (flags & MOE_WINDOW_QUANT_GROUP) != 0;
+  ctx->peers_have_counts = (flags & MOE_WINDOW_COUNTS) != 0;
   ctx->peers_installed = true;
   return MOE_OK;
 }
@@ -1351,6 +1363,36 @@ moe_status_t moe_wait_peers(moe_ctx_t* ctx, int32_t slot, uint32_t epoch, void* 
   wait_peers_kernel<<<1, R < 32 ? 32 : (R + 31) / 32 * 32, 0, static_cast<cudaStream_t>(stream)>>>(
       mine, R, slot, epoch, ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT, &ctx->ctl->status);
   return launch_ok(ctx);
+}
+
+moe_status_t moe_push_counts(moe_ctx_t* ctx, uint32_t epoch, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->layout_done) return MOE_ERR_NOT_PLANNED;
+  if (!ctx->peers_installed || !ctx->peers_have_counts) return MOE_ERR_STALE_PEERS;
+  const moe_shape_t& sh = ctx->shape;
+  push_counts_kernel<<<sh.R, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      ctx->box_table, ctx->M + (size_t)ctx->my_rank * sh.E, sh.E, sh.R, ctx->my_rank, epoch);
+  return launch_ok(ctx);
+}
+
+moe_status_t moe_notify_peers(moe_ctx_t* ctx, uint32_t epoch, void* stream) {
+  if (ctx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!ctx->layout_done) return MOE_ERR_NOT_PLANNED;
+  if (!ctx->peers_installed || !ctx->peers_have_counts) return MOE_ERR_STALE_PEERS;
+  const moe_shape_t& sh = ctx->shape;
+  unsigned char* mine = static_cast<unsigned char*>(ctx->peer_ptr[ctx->my_rank]) +
+                        window_parts(sh, ctx->peer_capacity, MOE_WINDOW_STATE | MOE_WINDOW_COUNTS).box;
+  notify_box_kernel<<<sh.R, 256, cluster_notify_smem_ints(sh.E, sh.R) * (int)sizeof(int32_t),
+                      static_cast<cudaStream_t>(stream)>>>(
+      mine, sh.E, sh.R, epoch, ctx->starve_wait_ms > 0 ? ctx->starve_wait_ms : WAIT_LIMIT_MS_DEFAULT,
+      ctx->schedule == MOE_SCHED_PREFILL, ctx->expert_align, ctx->M, ctx->c_rank, ctx->o, ctx->n_exp, ctx->n_recv,
+      &ctx->ctl->status);
+  const moe_status_t rc = launch_ok(ctx);
+  if (rc == MOE_OK) {
+    ctx->planned = true;
+    ctx->notified_by_box = true;
+  }
+  return rc;
 }
 
 moe_status_t moe_peers_check(const moe_ctx_t* ctx, const int32_t* generations) {
@@ -1555,7 +1597,7 @@ moe_status_t moe_status(moe_ctx_t* ctx, void* stream) {
     // valid layout, so it does not survive the report (a later dispatch returns MOE_ERR_NOT_PLANNED
     // instead of silently skipping the branch).
     ctx->slots_for_C = -1;   // a dispatch that stopped early has not recorded every row
-    if (word == MOE_ERR_BAD_INDEX) {
+    if (word == MOE_ERR_BAD_INDEX || (word == MOE_ERR_TIMEOUT && ctx->notified_by_box)) {
       ctx->planned = false;
       ctx->layout_done = false;
     }

@@ -537,6 +537,78 @@ notify_rank_kernel(const int32_t* counts_all, int32_t E, int32_t R, int32_t full
   window_offsets(sm, E, R, d, full_table, align, c_rank, o, n_exp, n_recv);
 }
 
+// Count exchange through the pooled memory (Section 5.2, Notify: the ranks exchange count metadata only).  Behind
+// the arrival flags of a rank's state region lies a mailbox of two buffers, each [R][E] counts and [R] epoch
+// words; an exchange with epoch e uses buffer e & 1.
+__host__ __device__ constexpr size_t counts_box_bytes(int E, int R) {
+  return 2 * ((size_t)R * E + R) * sizeof(int32_t);
+}
+__device__ __forceinline__ int32_t* box_counts(unsigned char* box, int E, int R, uint32_t epoch) {
+  return reinterpret_cast<int32_t*>(box) + (size_t)(epoch & 1u) * ((size_t)R * E + R);
+}
+
+// push: CTA d stores this rank's row of counts into entry [my_rank] of rank d's mailbox (plain peer stores), then
+// one thread publishes it with the epoch word (release, system scope, behind a CTA barrier and a system fence, so
+// the row is visible to whoever acquires the word).  Nothing waits here.
+__global__ void __launch_bounds__(256)
+push_counts_kernel(unsigned char* const* __restrict__ box_of_rank, const int32_t* __restrict__ my_row, int32_t E,
+                   int32_t R, int32_t my_rank, uint32_t epoch) {
+  int32_t* buf = box_counts(box_of_rank[blockIdx.x], E, R, epoch);
+  int32_t* dst = buf + (size_t)my_rank * E;
+  for (int e = threadIdx.x; e < E; e += (int)blockDim.x) dst[e] = my_row[e];
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence_system();
+    uint32_t* word = reinterpret_cast<uint32_t*>(buf + (size_t)R * E) + my_rank;
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(word), "r"(epoch) : "memory");
+  }
+}
+
+// notify from the mailbox: CTA d waits until every rank's epoch word in THIS rank's mailbox has reached `epoch`
+// (acquire, system scope; at most limit_ms milliseconds, then MOE_ERR_TIMEOUT and a normal end with nothing
+// written), then builds window d's offsets from the gathered rows like notify_rank_kernel.
+// Dynamic shared memory: cluster_notify_smem_ints(E, R) ints.
+__global__ void __launch_bounds__(256)
+notify_box_kernel(unsigned char* my_box, int32_t E, int32_t R, uint32_t epoch, int32_t limit_ms, int32_t full_table,
+                  int32_t align, int32_t* M, int32_t* __restrict__ c_rank, int32_t* __restrict__ o,
+                  int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, int32_t* status) {
+  extern __shared__ int32_t sm[];
+  __shared__ int gave_up;
+  if (threadIdx.x == 0) gave_up = 0;
+  __syncthreads();
+  const int32_t* buf = box_counts(my_box, E, R, epoch);
+  const uint32_t* words = reinterpret_cast<const uint32_t*>(buf + (size_t)R * E);
+  for (int r = threadIdx.x; r < R; r += (int)blockDim.x) {
+    uint64_t t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    const uint64_t limit = (uint64_t)limit_ms * 1000000ull;
+    for (;;) {
+      uint32_t seen;
+      asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(seen) : "l"(words + r) : "memory");
+      if ((int32_t)(seen - epoch) >= 0) break;
+      uint64_t now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (now - t0 > limit) {
+        raise_status(status, MOE_ERR_TIMEOUT);
+        gave_up = 1;
+        break;
+      }
+      __nanosleep(200);
+    }
+  }
+  __syncthreads();   // every row this CTA reads was acquired by one of its threads in front of this barrier
+  if (gave_up) return;
+  const int d = blockIdx.x, E_r = E / R, P = R + 1;
+  const volatile int32_t* rows = buf;   // written by other GPUs during this kernel's lifetime: no cached copies
+  for (int q = threadIdx.x; q < E_r * R; q += (int)blockDim.x) {
+    const int el = q % E_r, rr = q / E_r;
+    sm[el * P + rr] = rows[(size_t)rr * E + d * E_r + el];
+  }
+  for (int e = threadIdx.x; e < E; e += (int)blockDim.x) M[(size_t)d * E + e] = rows[(size_t)d * E + e];
+  __syncthreads();
+  window_offsets(sm, E, R, d, full_table, align, c_rank, o, n_exp, n_recv);
+}
+
 template <int ROUNDS>
 __global__ void __launch_bounds__(PLAN_THREADS)
 plan_finalize_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ RankMap map, int32_t K, int32_t E,

@@ -85,8 +85,13 @@ class EpRank:
     SLOT_DISPATCHED, SLOT_EXPERTS_DONE, SLOT_COMBINED = 0, 1, 2
 
     def __init__(self, T_local_max: int, H: int, E: int, K: int, device, group=None, mode: str = "cached",
-                 sync: str = "host", host_fence: bool = False):
+                 sync: str = "host", host_fence: bool = False, counts: str = "collective"):
         assert mode in ("cached", "handshake", "static") and sync in ("host", "device")
+        # counts="device": the count rows travel by the library's own stores into every rank's mailbox
+        # (moe_push_counts / moe_notify_peers) instead of an all-gather of the process group; no generations travel
+        # with them, so the addresses are static
+        assert counts in ("collective", "device") and (counts == "collective" or mode == "static")
+        self.counts, self.plan_epoch = counts, 0
         self.group, self.mode, self.device = group, mode, device
         self.sync, self.host_fence, self.epoch = sync, host_fence, 0
         self.rank = dist.get_rank(group)
@@ -110,7 +115,8 @@ class EpRank:
         quantised dispatch behind that; attaches it and returns the [capacity_rows, H] view of the rows."""
         assert not (quant and quant_group)
         flags = binding.MOE_WINDOW_STATE | (binding.MOE_WINDOW_QUANT if quant else 0) | \
-            (binding.MOE_WINDOW_QUANT_GROUP if quant_group else 0)
+            (binding.MOE_WINDOW_QUANT_GROUP if quant_group else 0) | \
+            (binding.MOE_WINDOW_COUNTS if self.counts == "device" else 0)
         nbytes = self.comm.moe_window_bytes(capacity_rows, flags)
         backing = torch.zeros(nbytes // 2, dtype=torch.bfloat16, device=self.device)
         self.attach_window(backing, capacity_rows, flags)
@@ -182,6 +188,18 @@ class EpRank:
 
     # -- the phases ------------------------------------------------------------------------------------
     def plan(self, schedule: int, topk_idx_local: torch.Tensor) -> torch.Tensor:
+        if self.counts == "device":
+            # Layout, then the row goes into every rank's mailbox and the offsets are built from this rank's own
+            # mailbox once all rows are there: no collective, nothing read back on the host
+            self._ensure_addresses()
+            self.plan_epoch += 1
+            self.comm.moe_layout(schedule, topk_idx_local, self.rank, self.counts_row)
+            self.comm.moe_push_counts(self.plan_epoch)
+            if self.host_fence:                  # ranks share a GPU: every push is sent before any notify is enqueued
+                self._host_barrier()
+            self.comm.moe_notify_peers(self.plan_epoch)
+            self.announced = None
+            return None
         self.comm.moe_layout(schedule, topk_idx_local, self.rank, self.counts_row)
         gathered = all_gather_rows(self.message, self.group)             # metadata only, no payload
         counts_all = gathered[:, :self.E].contiguous()

@@ -81,13 +81,21 @@ def test_window_and_state_sizes_host_logic(lib):
     assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_QUANT | binding.MOE_WINDOW_QUANT_GROUP) == 0
     odd = binding.MoeShape(2048, 7168 + 64, 256, 16, 8)                                # H % 128 != 0: no group-wise parts
     assert lib.moe_window_bytes(ctypes.byref(odd), 1300, binding.MOE_WINDOW_QUANT_GROUP) == 0
-    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 8) == 0                       # unknown flag
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_COUNTS) == 0   # only behind the state region
+    box = 2 * (16 * 256 + 16) * 4                                                      # two buffers of [R][E] counts + [R] epochs
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_COUNTS) == \
+        up(rows) + 256 + up(box)
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_COUNTS |
+                                binding.MOE_WINDOW_QUANT) == up(rows) + 256 + up(box) + up(1300 * 7168) + up(1300 * 4)
+    assert lib.moe_window_bytes(ctypes.byref(shape), 1300, 16) == 0                      # unknown flag
     assert lib.moe_window_bytes(ctypes.byref(shape), -1, 1) == 0 and lib.moe_window_bytes(None, 8, 1) == 0
     assert ctypes.sizeof(binding.MoeWindowHandle) == 96
     # calls that need a context reject a missing one before touching anything
     assert lib.moe_peers_check(None, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_signal_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_wait_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_push_counts(None, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_notify_peers(None, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_dispatch_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_window_export(None, 16, 1, 0, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_dispatch_quant_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG

@@ -248,6 +248,90 @@ def test_group_quantised_dispatch_through_the_installed_table(case):
         c.close()
 
 
+@pytest.mark.parametrize("case", [CASES[0], CASES[1], CASES[3]], ids=lambda c: c[0])
+def test_counts_exchanged_through_the_mailboxes_of_one_process(case):
+    """The count exchange by the library's own stores (moe_push_counts, moe_notify_peers), every rank a context of
+    this process, so every push is enqueued before any notify: the offsets and receive counts equal the oracle's, two
+    steps with different routing use the two buffers in turn, dispatch and combine through the table reproduce the
+    global result, and a notify nobody pushed for runs out after its bound, reports MOE_ERR_TIMEOUT without
+    trapping and leaves no plan behind."""
+    name, T, H, E, R, K, sch, routing, per = case
+    dev = torch.device("cuda:0")
+    FLAGS = binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_COUNTS
+    comms, backings, bases, C_alloc = None, None, None, None
+    for step, seed in enumerate((7100, 7200, 7300)):
+        wl = Workload(name, T, H, E, R, K, sch, routing, "identity", seed + T, rank_tokens=per)
+        inp = synth.make_inputs(wl)
+        rts = inp.rank_tok_start
+        p = oracle.plan(inp.topk_idx.numpy(), E, R, rts)
+        idx, w, X = inp.topk_idx.to(dev), inp.topk_w.to(dev), inp.X.to(dev)
+        if comms is None:
+            comms = [binding.MoeComm(max(int(rts[r + 1] - rts[r]), 1), H, E, R, K, dev) for r in range(R)]
+            C_alloc = int(p.n_recv.max()) + 64                       # room for the other steps' routing
+            total = comms[0].moe_window_bytes(C_alloc, FLAGS) // 2
+            backings = [torch.zeros(total, dtype=torch.bfloat16, device=dev) for _ in range(R)]   # state and mailbox zeroed
+            bases = [b.data_ptr() for b in backings]
+            # a table without the mailbox refuses the exchange; so does a context that has not laid out its tokens
+            comms[0].moe_peers_set(bases, None, C_alloc, my_rank=0, flags=binding.MOE_WINDOW_STATE)
+            comms[0].moe_layout(sch, idx[rts[0]:rts[1]].contiguous(), 0, torch.zeros(E, dtype=torch.int32, device=dev))
+            assert comms[0].moe_push_counts(1, check=False) == binding.MOE_ERR_STALE_PEERS
+            assert comms[0].moe_notify_peers(1, check=False) == binding.MOE_ERR_STALE_PEERS
+            for r, c in enumerate(comms):
+                c.moe_peers_set(bases, None, C_alloc, my_rank=r, flags=FLAGS)
+            assert comms[1].moe_push_counts(1, check=False) == binding.MOE_ERR_NOT_PLANNED
+        C = C_alloc
+        assert int(p.n_recv.max()) <= C
+        want = harness.oracle_run(inp, C)
+        epoch = step + 1
+        row = torch.zeros(E, dtype=torch.int32, device=dev)
+        for r, c in enumerate(comms):                              # every rank lays out and pushes ...
+            c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, row)
+            c.moe_push_counts(epoch)
+        for r, c in enumerate(comms):                              # ... then every rank builds its offsets
+            c.moe_notify_peers(epoch)
+            assert c.moe_status() == 0
+            v = c.moe_plan_view()
+            assert np.array_equal(v["large_off"].cpu().numpy(), p.o), (step, r)
+            assert np.array_equal(v["n_recv"].cpu().numpy(), p.n_recv)
+            if sch == PREFILL:
+                assert np.array_equal(v["counts"].cpu().numpy(), p.M) and np.array_equal(v["n_exp"].cpu().numpy(), p.n_exp)
+                assert np.array_equal(v["c_rank"].cpu().numpy(), p.c_rank)
+        rows = [b[:C * H].view(C, H) for b in backings]
+        for t in rows:
+            t.view(torch.int16).fill_(int(np.int16(np.uint16(harness.CANARY))))
+        for r, c in enumerate(comms):
+            c.moe_dispatch_cached(X[rts[r]:rts[r + 1]].contiguous())
+            assert c.moe_status() == 0
+        assert np.array_equal(torch.cat(rows).cpu().view(torch.int16).numpy().view(np.uint16), want.windows)
+        Y = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
+        for r, c in enumerate(comms):
+            y_r = torch.empty((int(rts[r + 1] - rts[r]), H), dtype=torch.bfloat16, device=dev)
+            c.moe_combine_cached(None, w[rts[r]:rts[r + 1]].contiguous(), y_r)
+            assert c.moe_status() == 0
+            Y[rts[r]:rts[r + 1]] = y_r
+        assert harness.max_ulp_diff(Y.cpu().view(torch.int16).numpy().view(np.uint16), want.Y) <= 1
+    # epoch 4: only rank 0 pushes; rank 1's notify is bounded (50 ms here), reports, and leaves no plan
+    c = comms[1]
+    c.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 50)
+    row = torch.zeros(E, dtype=torch.int32, device=dev)
+    for r in (0, 1):
+        comms[r].moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, row)
+    comms[0].moe_push_counts(4)
+    c.moe_notify_peers(4)
+    assert c.moe_status() == binding.MOE_ERR_TIMEOUT
+    assert c.moe_dispatch_cached(X[rts[1]:rts[2]].contiguous(), check=False) == binding.MOE_ERR_NOT_PLANNED
+    c.moe_set_option(binding.MOE_OPT_TEST_STARVE_WAIT_MS, 0)
+    # the others push: the same epoch now completes
+    for r in range(1, R):
+        comms[r].moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, row)
+        comms[r].moe_push_counts(4)
+    c.moe_notify_peers(4)
+    assert c.moe_status() == 0
+    assert np.array_equal(c.moe_plan_view()["large_off"].cpu().numpy(), p.o)
+    for cc in comms:
+        cc.close()
+
+
 def test_signals_and_bounded_waits_between_ranks_of_one_process():
     """The device-side phase order with every rank a context of this process (all on the one GPU, so every signal
     is enqueued before any wait): signals reach every rank's state region, waits pass once all R signals of the
@@ -557,7 +641,8 @@ def test_benchmark_expert_parallel_leg_as_two_processes_on_one_gpu():
         for variant, want_handshakes in (("cached_addresses__host_phase_order", 0),
                                          ("handshake_addresses__host_phase_order", 3),
                                          ("cached_addresses__device_phase_order", 0),
-                                         ("static_addresses__device_phase_order", 0)):
+                                         ("static_addresses__device_phase_order", 0),
+                                         ("static_addresses__device_phase_order__counts_through_mailboxes", 0)):
             got = leg["decode"][variant]
             assert got["verified"]["window_equals_single_gpu_path"] and got["verified"]["Y_equals_X"]
             assert got["handshakes_in_timed_steps"] == want_handshakes
