@@ -509,6 +509,7 @@ def sweeps(dev, n: int = 20) -> dict:
             whole = binding.MoeComm(wl.T, H, E, R, K, dev)
             whole.moe_plan(P, idx)
             counts = whole.moe_plan_view()["counts"].clone()
+            whole_n_recv = whole.moe_plan_view()["n_recv"].clone()
             whole.close()
             mine = idx[:per].contiguous()
             c = binding.MoeComm(per, H, E, R, K, dev)
@@ -516,10 +517,31 @@ def sweeps(dev, n: int = 20) -> dict:
             noti = lambda: c.moe_notify(counts)
             lay(), noti()
             assert c.moe_status() == 0
-            res["layout_notify"][f"R{R}_{per}_tokens_per_rank"] = {
-                "layout_us": time_graphed(lay), "notify_us": time_graphed(noti),
-                "both_us": time_graphed(lambda: (lay(), noti())), "note": "back to back inside a CUDA graph"}
+            entry = {"layout_us": time_graphed(lay), "notify_us": time_graphed(noti),
+                     "both_us": time_graphed(lambda: (lay(), noti())), "note": "back to back inside a CUDA graph"}
+            # the same with the counts going through the mailboxes: every window of this one GPU behind the table,
+            # the other ranks' rows pushed once beforehand (so the notify finds them and never waits)
+            flags = binding.MOE_WINDOW_STATE | binding.MOE_WINDOW_COUNTS
+            nbytes = c.moe_window_bytes(8, flags)
+            backings = [torch.zeros(nbytes // 2, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+            bases = [b.data_ptr() for b in backings]
+            others = binding.MoeComm(per, H, E, R, K, dev)
+            for r in range(1, R):
+                others.moe_peers_set(bases, None, 8, my_rank=r, flags=flags)
+                others.moe_layout(wl.schedule, idx[r * per:(r + 1) * per].contiguous(), r, counts[r].clone())
+                others.moe_push_counts(1)
+            c.moe_peers_set(bases, None, 8, my_rank=0, flags=flags)
+            boxed = lambda: (lay(), c.moe_push_counts(1), c.moe_notify_peers(1))
+            boxed()
+            assert c.moe_status() == 0 and others.moe_status() == 0
+            assert torch.equal(c.moe_plan_view()["n_recv"], whole_n_recv)
+            entry["layout_push_notify_peers_us"] = time_graphed(boxed)
+            entry["push_us"] = time_graphed(lambda: c.moe_push_counts(1))
+            entry["notify_peers_us"] = time_graphed(lambda: c.moe_notify_peers(1))
+            res["layout_notify"][f"R{R}_{per}_tokens_per_rank"] = entry
+            others.close()
             c.close()
+            del backings
     return res
 
 

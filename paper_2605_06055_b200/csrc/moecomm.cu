@@ -1370,7 +1370,7 @@ moe_status_t moe_push_counts(moe_ctx_t* ctx, uint32_t epoch, void* stream) {
   if (!ctx->layout_done) return MOE_ERR_NOT_PLANNED;
   if (!ctx->peers_installed || !ctx->peers_have_counts) return MOE_ERR_STALE_PEERS;
   const moe_shape_t& sh = ctx->shape;
-  push_counts_kernel<<<sh.R, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+  push_counts_kernel<<<(sh.R + PUSH_RANKS_PER_CTA - 1) / PUSH_RANKS_PER_CTA, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
       ctx->box_table, ctx->M + (size_t)ctx->my_rank * sh.E, sh.E, sh.R, ctx->my_rank, epoch);
   return launch_ok(ctx);
 }
