@@ -608,8 +608,11 @@ void launch_gate_form(const float* logits, int32_t T, int32_t E, int32_t K, int3
   // Two tokens per warp (they share the rank / softmax / store instructions) once that still leaves every SM a
   // full CTA of pairs; small batches keep one token per warp and so more warps.  3.0 against 2.7 us at T=2048,
   // 4.7 against 5.1 us at T=8192, 12.3 against 14.3 us at T=32768 (256 logits, top-8).
+  // A pair needs at most 16 candidates per token, which from K = 12 on fails too often (both tokens are then
+  // taken one by one after the attempt): 32768 tokens of 256 logits, K=11 16.2 against 18.0 us, K=12 19.6 against
+  // 18.6, K=16 27.2 against 21.5.
   if constexpr (VPT >= 4) {
-    if (K <= 16 && (int64_t)T / 2 >= (int64_t)num_sms * 8) {
+    if (K <= 11 && (int64_t)T / 2 >= (int64_t)num_sms * 8) {
       launch_gate_kernel<VPT, true>(logits, T, E, K, idx, w, num_sms, dev, st);
       return;
     }
