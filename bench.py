@@ -531,11 +531,11 @@ def sweeps(dev, n: int = 20) -> dict:
                 others.moe_layout(wl.schedule, idx[r * per:(r + 1) * per].contiguous(), r, counts[r].clone())
                 others.moe_push_counts(1)
             c.moe_peers_set(bases, None, 8, my_rank=0, flags=flags)
-            boxed = lambda: (lay(), c.moe_push_counts(1), c.moe_notify_peers(1))
+            boxed = lambda: (c.moe_layout_push(wl.schedule, mine, 0, 1), c.moe_notify_peers(1))
             boxed()
             assert c.moe_status() == 0 and others.moe_status() == 0
             assert torch.equal(c.moe_plan_view()["n_recv"], whole_n_recv)
-            entry["layout_push_notify_peers_us"] = time_graphed(boxed)
+            entry["layout_push_then_notify_peers_us"] = time_graphed(boxed)
             entry["push_us"] = time_graphed(lambda: c.moe_push_counts(1))
             entry["notify_peers_us"] = time_graphed(lambda: c.moe_notify_peers(1))
             res["layout_notify"][f"R{R}_{per}_tokens_per_rank"] = entry

@@ -375,6 +375,12 @@ moe_status_t moe_peers_close(moe_ctx_t* ctx, void* stream);
  * MOE_ERR_STALE_PEERS without an installed table whose windows have the mailbox; MOE_ERR_NOT_PLANNED before
  * moe_layout.  (No counterpart call in the paper: its Notify kernel does both halves.) */
 moe_status_t moe_push_counts(moe_ctx_t* ctx, uint32_t epoch, void* stream);
+/* moe_layout followed by moe_push_counts in one call (my_rank must be the rank of the installed table): for batches
+ * the single-launch planner takes (at most 4096 branches on this rank) and up to 16 ranks the one CTA that lays the
+ * tokens out also sends the row, straight from its shared memory -- a launch less in front of every multi-rank step; larger batches
+ * enqueue the two calls one behind the other.  Same results and errors as the two calls. */
+moe_status_t moe_layout_push(moe_ctx_t* ctx, moe_schedule_t schedule, const int32_t* topk_idx /*DEVICE [T_local,K]*/,
+                             int32_t T_local, int32_t my_rank, uint32_t epoch, void* stream);
 moe_status_t moe_notify_peers(moe_ctx_t* ctx, uint32_t epoch, void* stream);
 size_t moe_state_bytes(int32_t R);
 size_t moe_window_bytes(const moe_shape_t* shape /*HOST*/, int64_t capacity_rows, int32_t flags);

@@ -30,7 +30,7 @@ EXPORTS = [
     "moe_window_export", "moe_peers_open", "moe_peers_set", "moe_peers_check", "moe_peers_close",
     "moe_dispatch_cached", "moe_combine_cached", "moe_state_bytes", "moe_window_bytes", "moe_signal_peers",
     "moe_wait_peers", "moe_dispatch_quant_cached", "moe_dispatch_quant_group", "moe_plan_dispatch_quant_group",
-    "moe_dispatch_quant_group_cached", "moe_push_counts", "moe_notify_peers",
+    "moe_dispatch_quant_group_cached", "moe_push_counts", "moe_notify_peers", "moe_layout_push",
 ]
 MOE_SYNC_SLOTS = 4
 MOE_WINDOW_STATE, MOE_WINDOW_QUANT, MOE_WINDOW_QUANT_GROUP, MOE_WINDOW_COUNTS = 1, 2, 4, 8
@@ -133,6 +133,8 @@ def load() -> ctypes.CDLL:
     L.moe_signal_peers.restype = L.moe_wait_peers.restype = ctypes.c_int
     L.moe_push_counts.argtypes = L.moe_notify_peers.argtypes = [vp, ctypes.c_uint32, vp]
     L.moe_push_counts.restype = L.moe_notify_peers.restype = ctypes.c_int
+    L.moe_layout_push.argtypes = [vp, i32, vp, i32, i32, ctypes.c_uint32, vp]
+    L.moe_layout_push.restype = ctypes.c_int
     L.moe_peers_check.argtypes = [vp, vp]
     L.moe_peers_close.argtypes = [vp, vp]
     L.moe_dispatch_cached.argtypes = [vp, vp, vp, vp]
@@ -487,6 +489,18 @@ class MoeComm:
             rc = self.lib.moe_wait_peers(self._h, int(slot), int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
         if rc != MOE_OK and check:
             raise MoeError(rc, "moe_wait_peers")
+        return rc
+
+    def moe_layout_push(self, schedule: int, topk_idx: torch.Tensor, my_rank: int, epoch: int, stream=None,
+                        check: bool = True) -> int:
+        T = topk_idx.shape[0]
+        with self._on_device():
+            rc = self.lib.moe_layout_push(self._h, schedule, _dev_ptr(topk_idx, torch.int32), T, my_rank,
+                                          int(epoch) & 0xFFFFFFFF, _stream_handle(stream))
+        if rc == MOE_OK:
+            self.T, self.schedule, self._keep = T, schedule, topk_idx
+        elif check:
+            raise MoeError(rc, "moe_layout_push")
         return rc
 
     def moe_push_counts(self, epoch: int, stream=None, check: bool = True) -> int:

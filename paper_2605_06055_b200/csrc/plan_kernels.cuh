@@ -416,6 +416,16 @@ plan_scan_kernel(int32_t* __restrict__ tile_hist /* in: histograms, out: exclusi
   if (threadIdx.x == 0) ctl->scan_ticket = 0;  // ready for the next plan on this stream
 }
 
+// Count exchange through the pooled memory (Section 5.2, Notify: the ranks exchange count metadata only).  Behind
+// the arrival flags of a rank's state region lies a mailbox of two buffers, each [R][E] counts and [R] epoch
+// words; an exchange with epoch e uses buffer e & 1.
+__host__ __device__ constexpr size_t counts_box_bytes(int E, int R) {
+  return 2 * ((size_t)R * E + R) * sizeof(int32_t);
+}
+__device__ __forceinline__ int32_t* box_counts(unsigned char* box, int E, int R, uint32_t epoch) {
+  return reinterpret_cast<int32_t*>(box) + (size_t)(epoch & 1u) * ((size_t)R * E + R);
+}
+
 // Compact planner for batches in which every source rank holds few branches (every decode step,
 // small prefill chunks): ONE launch, one CTA per source rank.  The CTA walks its rank's branches in
 // passes of WARPS*32, carrying the running per-expert count in shared memory, so the small offsets
@@ -434,7 +444,9 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
                  int32_t full_table, int32_t align, int32_t* __restrict__ s, int32_t* __restrict__ M,
                  int32_t* __restrict__ c_rank,
                  int32_t* __restrict__ o, int32_t* __restrict__ n_exp, int32_t* __restrict__ n_recv, Control* ctl,
-                 int32_t mode /* PLAN_TICKET, PLAN_CLUSTER or PLAN_LOCAL, see plan_scan_kernel */, int32_t first_rank) {
+                 int32_t mode /* PLAN_TICKET, PLAN_CLUSTER or PLAN_LOCAL, see plan_scan_kernel */, int32_t first_rank,
+                 unsigned char* const* __restrict__ box_of_rank /* PLAN_LOCAL: the ranks' count mailboxes, or nullptr */,
+                 uint32_t epoch) {
   extern __shared__ int32_t sm[];
   __shared__ int is_last;
   const bool as_cluster = mode == PLAN_CLUSTER;
@@ -503,7 +515,21 @@ plan_rank_kernel(const int32_t* __restrict__ topk_idx, const __grid_constant__ R
     cluster_notify(rank_base, sm + (P + 1) * E, E, R, r, full_table, align, c_rank, o, n_exp, n_recv);
     return;
   }
-  if (mode == PLAN_LOCAL) return;   // s and this rank's row of M: the offsets come from moe_notify
+  if (mode == PLAN_LOCAL) {   // s and this rank's row of M: the offsets come from moe_notify / moe_notify_peers
+    if (box_of_rank != nullptr) {
+      // moe_layout_push: the row goes straight from shared memory into every rank's mailbox (see push_counts_kernel)
+      for (int q = threadIdx.x; q < R * E; q += WARPS * 32) {
+        const int d = q / E, e = q - d * E;
+        box_counts(box_of_rank[d], E, R, epoch)[(size_t)r * E + e] = rank_base[e];
+      }
+      __syncthreads();
+      for (int d = threadIdx.x; d < R; d += WARPS * 32) {
+        uint32_t* word = reinterpret_cast<uint32_t*>(box_counts(box_of_rank[d], E, R, epoch) + (size_t)R * E) + r;
+        asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(word), "r"(epoch) : "memory");
+      }
+    }
+    return;
+  }
 
   __threadfence();
   __syncthreads();
@@ -535,16 +561,6 @@ notify_rank_kernel(const int32_t* counts_all, int32_t E, int32_t R, int32_t full
     for (int e = threadIdx.x; e < E; e += (int)blockDim.x) M[(size_t)d * E + e] = counts_all[(size_t)d * E + e];
   __syncthreads();
   window_offsets(sm, E, R, d, full_table, align, c_rank, o, n_exp, n_recv);
-}
-
-// Count exchange through the pooled memory (Section 5.2, Notify: the ranks exchange count metadata only).  Behind
-// the arrival flags of a rank's state region lies a mailbox of two buffers, each [R][E] counts and [R] epoch
-// words; an exchange with epoch e uses buffer e & 1.
-__host__ __device__ constexpr size_t counts_box_bytes(int E, int R) {
-  return 2 * ((size_t)R * E + R) * sizeof(int32_t);
-}
-__device__ __forceinline__ int32_t* box_counts(unsigned char* box, int E, int R, uint32_t epoch) {
-  return reinterpret_cast<int32_t*>(box) + (size_t)(epoch & 1u) * ((size_t)R * E + R);
 }
 
 // push: a CTA stores this rank's row of counts into entry [my_rank] of the mailboxes of 16 ranks (plain peer stores),

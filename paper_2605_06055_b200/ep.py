@@ -193,8 +193,7 @@ class EpRank:
             # mailbox once all rows are there: no collective, nothing read back on the host
             self._ensure_addresses()
             self.plan_epoch += 1
-            self.comm.moe_layout(schedule, topk_idx_local, self.rank, self.counts_row)
-            self.comm.moe_push_counts(self.plan_epoch)
+            self.comm.moe_layout_push(schedule, topk_idx_local, self.rank, self.plan_epoch)
             if self.host_fence:                  # ranks share a GPU: every push is sent before any notify is enqueued
                 self._host_barrier()
             self.comm.moe_notify_peers(self.plan_epoch)

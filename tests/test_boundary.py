@@ -96,6 +96,7 @@ def test_window_and_state_sizes_host_logic(lib):
     assert lib.moe_wait_peers(None, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_push_counts(None, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_notify_peers(None, 1, None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_layout_push(None, 0, None, 0, 0, 1, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_dispatch_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_window_export(None, 16, 1, 0, None) == binding.MOE_ERR_INVALID_ARG
     assert lib.moe_dispatch_quant_cached(None, None, None, None) == binding.MOE_ERR_INVALID_ARG

@@ -279,14 +279,19 @@ def test_counts_exchanged_through_the_mailboxes_of_one_process(case):
             for r, c in enumerate(comms):
                 c.moe_peers_set(bases, None, C_alloc, my_rank=r, flags=FLAGS)
             assert comms[1].moe_push_counts(1, check=False) == binding.MOE_ERR_NOT_PLANNED
+            assert comms[1].moe_layout_push(sch, idx[rts[1]:rts[2]].contiguous(), 0, 1, check=False) == \
+                binding.MOE_ERR_STALE_PEERS                          # not the rank of the installed table
         C = C_alloc
         assert int(p.n_recv.max()) <= C
         want = harness.oracle_run(inp, C)
         epoch = step + 1
         row = torch.zeros(E, dtype=torch.int32, device=dev)
         for r, c in enumerate(comms):                              # every rank lays out and pushes ...
-            c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, row)
-            c.moe_push_counts(epoch)
+            if step == 1:                                          # ... as one call (one kernel for small batches)
+                c.moe_layout_push(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, epoch)
+            else:
+                c.moe_layout(sch, idx[rts[r]:rts[r + 1]].contiguous(), r, row)
+                c.moe_push_counts(epoch)
         for r, c in enumerate(comms):                              # ... then every rank builds its offsets
             c.moe_notify_peers(epoch)
             assert c.moe_status() == 0
